@@ -1,0 +1,232 @@
+"""ctypes front end of the CPU oracle (test infrastructure, not product code).
+
+The oracle is ``nvfp4_oracle.cpp`` beside this file: a plain scalar C++
+restatement of the NVFP4 Root Newton-Schulz step.  Only tests, the smoke check
+and the benchmark's CPU-baseline leg may import this package; the CUDA library
+and its Python binding never do.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "nvfp4_oracle.cpp")
+_LIB = os.path.join(_HERE, "libnvfp4_oracle.so")
+_lib = None
+
+_u8p = C.POINTER(C.c_uint8)
+_f32p = C.POINTER(C.c_float)
+
+
+class OrcParams(C.Structure):
+    _fields_ = [("a", C.c_float), ("b", C.c_float), ("c", C.c_float),
+                ("clip_quantile", C.c_float), ("eps", C.c_float),
+                ("quantize", C.c_int32), ("exact_scales", C.c_int32)]
+
+
+class OrcTrace(C.Structure):
+    _fields_ = [("iter", C.c_int32),
+                ("tau", _f32p), ("nu", _f32p), ("X0", _f32p), ("amax_in", _f32p), ("X_in", _f32p),
+                ("qX_codes", _u8p), ("qX_scales", _u8p), ("qXt_codes", _u8p), ("qXt_scales", _u8p),
+                ("sg_X", _f32p), ("A", _f32p),
+                ("qA_codes", _u8p), ("qA_scales", _u8p), ("sg_A", _f32p),
+                ("S", _f32p), ("B", _f32p),
+                ("qB_codes", _u8p), ("qB_scales", _u8p), ("sg_B", _f32p),
+                ("X_out", _f32p)]
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with g++ (no CUDA involved); returns the library path."""
+    if (not force and os.path.exists(_LIB)
+            and os.path.getmtime(_LIB) >= os.path.getmtime(_SRC)):
+        return _LIB
+    cmd = ["g++", "-O2", "-std=c++17", "-ffp-contract=off", "-fopenmp", "-shared", "-fPIC",
+           _SRC, "-o", _LIB]
+    subprocess.run(cmd, check=True)
+    return _LIB
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        L = C.CDLL(build())
+        L.orc_e2m1_encode.argtypes = [C.c_float]; L.orc_e2m1_encode.restype = C.c_uint8
+        L.orc_e2m1_decode.argtypes = [C.c_uint8]; L.orc_e2m1_decode.restype = C.c_float
+        L.orc_ue4m3_encode.argtypes = [C.c_float]; L.orc_ue4m3_encode.restype = C.c_uint8
+        L.orc_ue4m3_decode.argtypes = [C.c_uint8]; L.orc_ue4m3_decode.restype = C.c_float
+        L.orc_amax.argtypes = [_f32p, C.c_int64]; L.orc_amax.restype = C.c_float
+        L.orc_tensor_scale_exact.argtypes = [C.c_float]; L.orc_tensor_scale_exact.restype = C.c_float
+        L.orc_tensor_scale_predicted.argtypes = [C.c_float]; L.orc_tensor_scale_predicted.restype = C.c_float
+        L.orc_quantile_rank.argtypes = [C.c_int64, C.c_float]; L.orc_quantile_rank.restype = C.c_int64
+        L.orc_quantize.argtypes = [_f32p, C.c_int64, C.c_int64, C.c_float, _u8p, _u8p]
+        L.orc_quantize.restype = None
+        L.orc_dequantize.argtypes = [_u8p, _u8p, C.c_float, C.c_int64, C.c_int64, _f32p]
+        L.orc_dequantize.restype = None
+        L.orc_gemm_nt_q.argtypes = [_u8p, _u8p, C.c_float, _u8p, _u8p, C.c_float,
+                                    C.c_int64, C.c_int64, C.c_int64, _f32p, C.c_int]
+        L.orc_gemm_nt_q.restype = None
+        L.orc_clip_threshold.argtypes = [_f32p, C.c_int64, C.c_float]
+        L.orc_clip_threshold.restype = C.c_float
+        L.orc_root_coeffs.argtypes = [C.c_int64, C.c_int64, C.c_int, _f32p]
+        L.orc_root_coeffs.restype = None
+        L.orc_root_ns.argtypes = [_f32p, C.c_int64, C.c_int64, C.c_int, C.POINTER(OrcParams),
+                                  _f32p, C.POINTER(OrcTrace)]
+        L.orc_root_ns.restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def _f32(a):
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    return a, a.ctypes.data_as(_f32p)
+
+
+def _u8(a):
+    a = np.ascontiguousarray(a, dtype=np.uint8)
+    return a, a.ctypes.data_as(_u8p)
+
+
+# --- codecs -----------------------------------------------------------------
+def e2m1_encode(y: float) -> int:
+    return int(lib().orc_e2m1_encode(float(np.float32(y))))
+
+
+def e2m1_decode(nib: int) -> float:
+    return float(lib().orc_e2m1_decode(int(nib)))
+
+
+def ue4m3_encode(t: float) -> int:
+    return int(lib().orc_ue4m3_encode(float(np.float32(t))))
+
+
+def ue4m3_decode(b: int) -> float:
+    return float(lib().orc_ue4m3_decode(int(b)))
+
+
+def tensor_scale_exact(amax: float) -> float:
+    return float(lib().orc_tensor_scale_exact(float(np.float32(amax))))
+
+
+def tensor_scale_predicted(bound: float) -> float:
+    return float(lib().orc_tensor_scale_predicted(float(np.float32(bound))))
+
+
+def quantile_rank(n: int, q: float) -> int:
+    return int(lib().orc_quantile_rank(int(n), float(np.float32(q))))
+
+
+# --- quantiser ----------------------------------------------------------------
+def quantize(x, s_g=None):
+    """Q_1x16 of a 2-D FP32 array.  s_g None: exact rule amax/2688.
+
+    Returns (codes[rows, cols/2] u8, scales[rows, cols/16] u8, s_g)."""
+    x, xp = _f32(x)
+    rows, cols = x.shape
+    assert cols % 16 == 0
+    if s_g is None:
+        s_g = tensor_scale_exact(float(lib().orc_amax(xp, x.size)))
+    codes = np.empty((rows, cols // 2), np.uint8)
+    scales = np.empty((rows, cols // 16), np.uint8)
+    lib().orc_quantize(xp, rows, cols, float(np.float32(s_g)),
+                       codes.ctypes.data_as(_u8p), scales.ctypes.data_as(_u8p))
+    return codes, scales, float(np.float32(s_g))
+
+
+def dequantize(codes, scales, s_g):
+    codes, cp = _u8(codes)
+    scales, sp = _u8(scales)
+    rows, cols = codes.shape[0], codes.shape[1] * 2
+    out = np.empty((rows, cols), np.float32)
+    lib().orc_dequantize(cp, sp, float(np.float32(s_g)), rows, cols, out.ctypes.data_as(_f32p))
+    return out
+
+
+def gemm_nt_q(a, b=None):
+    """FP32(deq(a) @ deq(b).T) with FP64 sums; a, b = (codes, scales, s_g).
+    b None: symmetric product a a^T (upper triangle computed, mirrored)."""
+    ac, acp = _u8(a[0]); as_, asp = _u8(a[1])
+    M, K = ac.shape[0], ac.shape[1] * 2
+    if b is None:
+        out = np.empty((M, M), np.float32)
+        lib().orc_gemm_nt_q(acp, asp, float(a[2]), acp, asp, float(a[2]), M, M, K,
+                            out.ctypes.data_as(_f32p), 1)
+        return out
+    bc, bcp = _u8(b[0]); bs, bsp = _u8(b[1])
+    N = bc.shape[0]
+    assert bc.shape[1] * 2 == K
+    out = np.empty((M, N), np.float32)
+    lib().orc_gemm_nt_q(acp, asp, float(a[2]), bcp, bsp, float(b[2]), M, N, K,
+                        out.ctypes.data_as(_f32p), 0)
+    return out
+
+
+# --- clip, coefficients, the whole step ---------------------------------------
+def clip_threshold(g, q=0.99) -> float:
+    g, gp = _f32(g)
+    return float(lib().orc_clip_threshold(gp, g.size, float(np.float32(q))))
+
+
+def root_coeffs(m, n, steps=5):
+    abc = (C.c_float * 3)()
+    lib().orc_root_coeffs(int(m), int(n), int(steps), abc)
+    return float(abc[0]), float(abc[1]), float(abc[2])
+
+
+def root_ns(G, steps=5, abc=None, clip_quantile=0.99, eps=1e-7, quantize=True,
+            exact_scales=False, trace_iter=None):
+    """The Root Newton-Schulz step on one m x n FP32 matrix.
+
+    Returns out (m x n FP32), or (out, trace dict) when trace_iter is given; the
+    trace holds the intermediates of that iteration in the work orientation
+    (s x l, s = min(m, n))."""
+    G, gp = _f32(G)
+    m, n = G.shape
+    s, l = min(m, n), max(m, n)
+    p = OrcParams()
+    if abc is None:
+        p.a = p.b = p.c = float("nan")
+    else:
+        p.a, p.b, p.c = [float(np.float32(v)) for v in abc]
+    p.clip_quantile = float(np.float32(clip_quantile))
+    p.eps = float(np.float32(eps))
+    p.quantize = 1 if quantize else 0
+    p.exact_scales = 1 if exact_scales else 0
+    out = np.empty((m, n), np.float32)
+    if trace_iter is None:
+        rc = lib().orc_root_ns(gp, m, n, int(steps), C.byref(p), out.ctypes.data_as(_f32p), None)
+        if rc:
+            raise ValueError(f"orc_root_ns failed with code {rc}")
+        return out
+    t = OrcTrace()
+    t.iter = int(trace_iter)
+    bufs = {}
+
+    def f(name, shape):
+        bufs[name] = np.zeros(shape, np.float32)
+        setattr(t, name, bufs[name].ctypes.data_as(_f32p))
+
+    def u(name, shape):
+        bufs[name] = np.zeros(shape, np.uint8)
+        setattr(t, name, bufs[name].ctypes.data_as(_u8p))
+
+    for name in ("tau", "nu", "amax_in", "sg_X", "sg_A", "sg_B"):
+        f(name, (1,))
+    for name in ("X0", "X_in", "X_out"):
+        f(name, (s, l))
+    for name in ("A", "S", "B"):
+        f(name, (s, s))
+    if quantize:
+        u("qX_codes", (s, l // 2)); u("qX_scales", (s, l // 16))
+        u("qXt_codes", (l, s // 2)); u("qXt_scales", (l, s // 16))
+        u("qA_codes", (s, s // 2)); u("qA_scales", (s, s // 16))
+        u("qB_codes", (s, s // 2)); u("qB_scales", (s, s // 16))
+    rc = lib().orc_root_ns(gp, m, n, int(steps), C.byref(p), out.ctypes.data_as(_f32p), C.byref(t))
+    if rc:
+        raise ValueError(f"orc_root_ns failed with code {rc}")
+    for name in ("tau", "nu", "amax_in", "sg_X", "sg_A", "sg_B"):
+        bufs[name] = float(bufs[name][0])
+    return out, bufs

@@ -1,0 +1,457 @@
+// CPU oracle for the NVFP4 Root Newton-Schulz step.
+//
+// THIS IS TEST INFRASTRUCTURE, NOT PRODUCT CODE.  It is a plain, slow, scalar
+// restatement of what the method computes, written from the paper so that the
+// CUDA library can be checked against it.  Nothing in the CUDA library includes,
+// links or calls this file, and this file includes nothing of the library.
+// Only the tests, the smoke check and the benchmark's CPU-baseline leg use it.
+//
+// What follows the paper, and where:
+//   * NVFP4 format (Section 2, "NVFP4 format"): E2M1 values (1 sign, 2 exponent,
+//     1 mantissa bit), one FP8-E4M3 scale s per block of 1x16 elements, one FP32
+//     global scale s_g, decoded value  x^ = x_E2M1 * s * s_g.
+//   * Rounding (Section 2, "Others"; Section 3.4 last paragraph): round to
+//     nearest.  Ties go to the even mantissa, conversions saturate.
+//   * Root Newton-Schulz iteration (Section 2, "Root optimizer", and the display
+//     equations of Section 3.4):  qX = Q_1x16(X), A = qX qX^T,
+//     qA = Q_1x16(A), qA^{16x1} = Q_16x1(A), B = b A + c qA qA^{16x1},
+//     qB = Q_1x16(B), qX^{16x1} = Q_16x1(X), X+ = a X + qB qX^{16x1}.
+//     Q_16x1(T) is Q_1x16 of the transpose: the 16 elements of a block always
+//     run along the contraction axis of the product that consumes them.
+//   * Outlier removal (Section 2 "soft-thresholding for ... outlier removal",
+//     Section 3.4 "p99 outlier clipping", appendix hyper-parameter "quantile
+//     ratio 0.99"): the soft-thresholded outlier part sign(g)*max(|g|-tau,0)
+//     is removed, which leaves clamp(g,-tau,tau); tau is the nearest-rank
+//     q-quantile of |G|.
+//
+// Readings taken where the paper is silent (each is repeated in the design
+// document of the repository):
+//   * input normalisation: X0 = G_c / (||G_c||_F + eps), norm summed in FP64;
+//   * per-tensor scale: exact amax/2688 for the initial operand (2688 = 6*448,
+//     the largest E2M1 value times the largest E4M3 value), and a power of two
+//     predicted from running maxima for tensors produced inside the loop;
+//   * coefficient provider: a one-parameter quintic family with p(1)=1, p'(1)=0
+//     chosen by aspect ratio.  The paper's own coefficient values are not
+//     printed: parity unpinned for orc_root_coeffs (the identities it satisfies
+//     are pinned, the values are a stand-in).
+//   * all FP32 steps are single IEEE operations with no fused multiply-add
+//     (build with -ffp-contract=off); GEMM sums are taken in FP64 in index
+//     order and rounded once to FP32.
+//
+// Build:  g++ -O2 -std=c++17 -ffp-contract=off -fopenmp -shared -fPIC
+
+#include <algorithm>
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+#include <vector>
+
+namespace {
+
+const float kE2M1Grid[8] = {0.0f, 0.5f, 1.0f, 1.5f, 2.0f, 3.0f, 4.0f, 6.0f};
+
+// Magnitude index on the E2M1 grid, round to nearest, ties to the even index
+// (even index == even mantissa bit), saturating at 6.
+int e2m1_index(float mag) {
+  if (!(mag == mag)) return 7;  // NaN: saturating conversion returns the largest value
+  if (mag >= 6.0f) return 7;
+  int idx = 0;
+  for (int i = 0; i < 7; ++i) {
+    // midpoint between grid[i] and grid[i+1]; all midpoints are exact in FP32
+    float mid = 0.5f * (kE2M1Grid[i] + kE2M1Grid[i + 1]);
+    if (mag > mid) {
+      idx = i + 1;
+    } else {
+      if (mag == mid) idx = (i % 2 == 0) ? i : i + 1;  // tie: the even index
+      break;
+    }
+  }
+  return idx;
+}
+
+// Unsigned E4M3 ("fn" variant: bias 7, 3 mantissa bits, no infinity, largest
+// finite value 448 = 0x7E).  Round to nearest even, saturate to 448.
+uint8_t ue4m3_encode(float t) {
+  if (!(t == t)) return 0x7E;
+  if (t <= 0.0f) return 0;
+  if (t >= 448.0f) return 0x7E;
+  const float min_normal = 0.015625f;  // 2^-6
+  if (t < min_normal) {
+    // subnormal step is 2^-9; nearbyint rounds half to even in the default mode
+    float q = std::nearbyint(t * 512.0f);  // exact scaling by a power of two
+    return (uint8_t)q;                     // q == 8 is exactly the code of 2^-6
+  }
+  int e;
+  float f = std::frexp(t, &e);  // t = f * 2^e, f in [0.5,1)
+  e -= 1;                       // t = (2f) * 2^e, 2f in [1,2)
+  float q = std::nearbyint(f * 16.0f);  // 2f*8 in [8,16]
+  if (q == 16.0f) { q = 8.0f; e += 1; }
+  int code = ((e + 7) << 3) | ((int)q - 8);
+  if (code > 0x7E) code = 0x7E;
+  return (uint8_t)code;
+}
+
+float ue4m3_decode(uint8_t b) {
+  int e = (b >> 3) & 0xF, m = b & 7;
+  if (e == 0) return std::ldexp((float)m, -9);
+  return std::ldexp((float)(8 + m), e - 7 - 3);
+}
+
+float e2m1_decode(uint8_t nib) {
+  float v = kE2M1Grid[nib & 7];
+  return (nib & 8) ? -v : v;
+}
+
+float amax_of(const float* x, int64_t n) {
+  float m = 0.0f;
+  for (int64_t i = 0; i < n; ++i) {
+    float a = std::fabs(x[i]);
+    if (a > m) m = a;
+  }
+  return m;
+}
+
+// Q_1x16 of a row-major rows x cols tensor with a given global scale.
+// codes: rows x cols/2 bytes, element 2j in the low nibble of byte j.
+// scales: rows x cols/16 bytes, plain row-major.
+void quantize_1x16(const float* x, int64_t rows, int64_t cols, float s_g,
+                   uint8_t* codes, uint8_t* scales) {
+  const int64_t nb = cols / 16;
+  const float six_sg = 6.0f * s_g;
+#pragma omp parallel for schedule(static)
+  for (int64_t r = 0; r < rows; ++r) {
+    for (int64_t kb = 0; kb < nb; ++kb) {
+      const float* blk = x + r * cols + kb * 16;
+      float amax_b = amax_of(blk, 16);
+      float t = amax_b / six_sg;
+      uint8_t sb = ue4m3_encode(t);
+      scales[r * nb + kb] = sb;
+      float s = ue4m3_decode(sb);
+      float d = s * s_g;
+      uint8_t nib[16];
+      if (d == 0.0f) {
+        for (int i = 0; i < 16; ++i) nib[i] = 0;
+      } else {
+        float rcp = 1.0f / d;
+        for (int i = 0; i < 16; ++i) {
+          float y = blk[i] * rcp;
+          int idx = e2m1_index(std::fabs(y));
+          nib[i] = (uint8_t)((std::signbit(y) ? 8 : 0) | idx);
+        }
+      }
+      uint8_t* out = codes + r * (cols / 2) + kb * 8;
+      for (int i = 0; i < 8; ++i) out[i] = (uint8_t)(nib[2 * i] | (nib[2 * i + 1] << 4));
+    }
+  }
+}
+
+void dequantize_1x16(const uint8_t* codes, const uint8_t* scales, float s_g,
+                     int64_t rows, int64_t cols, float* out) {
+  const int64_t nb = cols / 16;
+#pragma omp parallel for schedule(static)
+  for (int64_t r = 0; r < rows; ++r) {
+    for (int64_t kb = 0; kb < nb; ++kb) {
+      // grid value (<= 2 significant bits) * E4M3 (<= 4 bits) * FP32: the FP64
+      // product is exact, and it is representable in FP32 whenever s_g is a
+      // power of two; otherwise it is rounded once here, and the GEMMs below
+      // read the FP64 product again from its three factors.
+      double d = (double)ue4m3_decode(scales[r * nb + kb]) * (double)s_g;
+      for (int i = 0; i < 16; ++i) {
+        uint8_t byte = codes[r * (cols / 2) + kb * 8 + i / 2];
+        uint8_t nib = (i & 1) ? (byte >> 4) : (byte & 0xF);
+        out[r * cols + kb * 16 + i] = (float)((double)e2m1_decode(nib) * d);
+      }
+    }
+  }
+}
+
+// FP64 decoded operand for the GEMMs (exact products of the three factors).
+std::vector<double> decode_f64(const uint8_t* codes, const uint8_t* scales, float s_g,
+                               int64_t rows, int64_t cols) {
+  std::vector<double> out((size_t)rows * cols);
+  const int64_t nb = cols / 16;
+#pragma omp parallel for schedule(static)
+  for (int64_t r = 0; r < rows; ++r)
+    for (int64_t kb = 0; kb < nb; ++kb) {
+      double d = (double)ue4m3_decode(scales[r * nb + kb]) * (double)s_g;
+      for (int i = 0; i < 16; ++i) {
+        uint8_t byte = codes[r * (cols / 2) + kb * 8 + i / 2];
+        uint8_t nib = (i & 1) ? (byte >> 4) : (byte & 0xF);
+        out[(size_t)r * cols + kb * 16 + i] = (double)e2m1_decode(nib) * d;
+      }
+    }
+  return out;
+}
+
+// out[i][j] = FP32( sum_p a[i][p] * b[j][p] ), FP64 sum in index order.
+// symmetric != 0: a and b are the same operand, compute j >= i and mirror.
+void gemm_nt(const double* a, const double* b, int64_t M, int64_t N, int64_t K,
+             float* out, int symmetric) {
+#pragma omp parallel for schedule(dynamic, 4)
+  for (int64_t i = 0; i < M; ++i) {
+    const double* ai = a + i * K;
+    for (int64_t j = symmetric ? i : 0; j < N; ++j) {
+      const double* bj = b + j * K;
+      double acc = 0.0;
+      for (int64_t p = 0; p < K; ++p) acc += ai[p] * bj[p];
+      out[i * N + j] = (float)acc;
+    }
+  }
+  if (symmetric) {
+    for (int64_t i = 0; i < M; ++i)
+      for (int64_t j = 0; j < i; ++j) out[i * N + j] = out[j * N + i];
+  }
+}
+
+void transpose(const float* x, int64_t rows, int64_t cols, float* out) {
+  for (int64_t r = 0; r < rows; ++r)
+    for (int64_t c = 0; c < cols; ++c) out[c * rows + r] = x[r * cols + c];
+}
+
+float scale_exact(float amax) { return amax == 0.0f ? 1.0f : amax / 2688.0f; }
+
+// Smallest power of two >= bound/2688 (bound/2688 itself if it is one).
+float scale_predicted(float bound) {
+  if (!(bound > 0.0f)) return 1.0f;
+  float v = bound / 2688.0f;
+  int e;
+  float f = std::frexp(v, &e);  // v = f*2^e, f in [0.5,1)
+  float p = (f == 0.5f) ? std::ldexp(1.0f, e - 1) : std::ldexp(1.0f, e);
+  // keep the scale a normal FP32 number
+  const float tiny = std::ldexp(1.0f, -126);
+  return p < tiny ? tiny : p;
+}
+
+int64_t quantile_rank(int64_t n, float q) {
+  // the quantile is resolved to parts per million so that 0.99f means 99/100
+  int64_t ppm = (int64_t)std::llround((double)q * 1e6);
+  int64_t k = (ppm * n + 999999) / 1000000;
+  if (k < 1) k = 1;
+  if (k > n) k = n;
+  return k;
+}
+
+}  // namespace
+
+extern "C" {
+
+struct orc_params {
+  float a, b, c;        // NaN a: take orc_root_coeffs(m, n, steps)
+  float clip_quantile;  // <= 0 or >= 1: no clip
+  float eps;
+  int32_t quantize;     // 0: plain FP64-accumulated Newton-Schulz, no NVFP4
+  int32_t exact_scales; // 1: every tensor scale is amax/2688 (comparison only)
+};
+
+// Optional record of one iteration's intermediates (all row-major in the work
+// orientation s x l; scale arrays are plain row-major rows x K/16).  Null
+// pointers are skipped.
+struct orc_trace {
+  int32_t iter;           // which iteration to record
+  float* tau;             // [1]
+  float* nu;              // [1]
+  float* X0;              // s*l      normalised input
+  float* amax_in;         // [1]      amax of X at the start of iteration `iter`
+  float* X_in;            // s*l      X at the start of iteration `iter`
+  uint8_t* qX_codes;      // s*l/2    operand of G1
+  uint8_t* qX_scales;     // s*l/16
+  uint8_t* qXt_codes;     // l*s/2    operand of G3
+  uint8_t* qXt_scales;    // l*s/16
+  float* sg_X;            // [1]
+  float* A;               // s*s
+  uint8_t* qA_codes; uint8_t* qA_scales; float* sg_A;
+  float* S;               // s*s      qA qA^T
+  float* B;               // s*s
+  uint8_t* qB_codes; uint8_t* qB_scales; float* sg_B;
+  float* X_out;           // s*l      X after iteration `iter`
+};
+
+uint8_t orc_e2m1_encode(float y) {
+  return (uint8_t)((std::signbit(y) ? 8 : 0) | e2m1_index(std::fabs(y)));
+}
+float orc_e2m1_decode(uint8_t nib) { return e2m1_decode(nib); }
+uint8_t orc_ue4m3_encode(float t) { return ue4m3_encode(t); }
+float orc_ue4m3_decode(uint8_t b) { return ue4m3_decode(b); }
+float orc_amax(const float* x, int64_t n) { return amax_of(x, n); }
+float orc_tensor_scale_exact(float amax) { return scale_exact(amax); }
+float orc_tensor_scale_predicted(float bound) { return scale_predicted(bound); }
+int64_t orc_quantile_rank(int64_t n, float q) { return quantile_rank(n, q); }
+
+void orc_quantize(const float* x, int64_t rows, int64_t cols, float s_g,
+                  uint8_t* codes, uint8_t* scales) {
+  quantize_1x16(x, rows, cols, s_g, codes, scales);
+}
+
+void orc_dequantize(const uint8_t* codes, const uint8_t* scales, float s_g,
+                    int64_t rows, int64_t cols, float* out) {
+  dequantize_1x16(codes, scales, s_g, rows, cols, out);
+}
+
+// out = FP32(deq(a) deq(b)^T) with FP64 accumulation; operands are quantised
+// tensors (codes/scales/global scale), both rows x K.
+void orc_gemm_nt_q(const uint8_t* a_codes, const uint8_t* a_scales, float a_sg,
+                   const uint8_t* b_codes, const uint8_t* b_scales, float b_sg,
+                   int64_t M, int64_t N, int64_t K, float* out, int symmetric) {
+  std::vector<double> a = decode_f64(a_codes, a_scales, a_sg, M, K);
+  if (symmetric) { gemm_nt(a.data(), a.data(), M, N, K, out, 1); return; }
+  std::vector<double> b = decode_f64(b_codes, b_scales, b_sg, N, K);
+  gemm_nt(a.data(), b.data(), M, N, K, out, 0);
+}
+
+// nearest-rank q-quantile of |g|
+float orc_clip_threshold(const float* g, int64_t n, float q) {
+  std::vector<float> mag((size_t)n);
+  for (int64_t i = 0; i < n; ++i) mag[(size_t)i] = std::fabs(g[i]);
+  int64_t k = quantile_rank(n, q);
+  std::nth_element(mag.begin(), mag.begin() + (k - 1), mag.end());
+  return mag[(size_t)(k - 1)];
+}
+
+// Stand-in provider (the paper does not print Root's values).  Quintic
+// p(x) = a x + b x^3 + c x^5 with p(1) = 1 and p'(1) = 0, i.e. b = 2.5 - 2a,
+// c = a - 1.5; a grows as the matrix gets wider.  At aspect ratio 1 it is the
+// classical (15/8, -10/8, 3/8).
+void orc_root_coeffs(int64_t m, int64_t n, int steps, float abc[3]) {
+  (void)steps;
+  double s = (double)std::min(m, n), l = (double)std::max(m, n);
+  double gamma = s / l;
+  double delta = (std::sqrt(7.0 / 3.0) - 1.0) / 2.0;
+  double root_r = 1.0 + delta * (1.0 + std::sqrt(gamma));
+  double R = root_r * root_r;
+  double a = (1.5 * R - 1.0) / (R - 1.0);
+  abc[0] = (float)a;
+  abc[1] = (float)(2.5 - 2.0 * a);
+  abc[2] = (float)(a - 1.5);
+}
+
+// The whole step.  G is m x n row-major, out is m x n row-major.
+int orc_root_ns(const float* G, int64_t m, int64_t n, int steps, const orc_params* prm,
+                float* out, orc_trace* tr) {
+  if (m <= 0 || n <= 0 || steps < 0) return 1;
+  const bool tall = m > n;
+  const int64_t s = tall ? n : m, l = tall ? m : n;
+  if (prm->quantize && (s % 16 || l % 16)) return 2;
+  const size_t N = (size_t)s * l;
+
+  // orientation: work on the short side (XX^T is s x s)
+  std::vector<float> X(N);
+  if (tall) transpose(G, m, n, X.data()); else std::memcpy(X.data(), G, N * sizeof(float));
+
+  float abc[3] = {prm->a, prm->b, prm->c};
+  if (!(prm->a == prm->a)) orc_root_coeffs(m, n, steps, abc);
+  const float ca = abc[0], cb = abc[1], cc = abc[2];
+
+  // outlier removal: G_c = G - soft_threshold(G, tau) = clamp(G, -tau, tau)
+  float tau = INFINITY;
+  if (prm->clip_quantile > 0.0f && prm->clip_quantile < 1.0f) {
+    tau = orc_clip_threshold(X.data(), (int64_t)N, prm->clip_quantile);
+    for (size_t i = 0; i < N; ++i) {
+      float g = X[i];
+      X[i] = g > tau ? tau : (g < -tau ? -tau : g);
+    }
+  }
+  // Frobenius normalisation
+  double ss = 0.0;
+  for (size_t i = 0; i < N; ++i) ss += (double)X[i] * (double)X[i];
+  float nu = (float)std::sqrt(ss);
+  float inv = 1.0f / (nu + prm->eps);
+  for (size_t i = 0; i < N; ++i) X[i] = X[i] * inv;
+  if (tr) {
+    if (tr->tau) *tr->tau = tau;
+    if (tr->nu) *tr->nu = nu;
+    if (tr->X0) std::memcpy(tr->X0, X.data(), N * sizeof(float));
+  }
+
+  std::vector<float> Xt(N), A((size_t)s * s), S((size_t)s * s), B((size_t)s * s), P(N);
+  std::vector<uint8_t> qXc(N / 2 + 1), qXs(N / 16 + 1), qXtc(N / 2 + 1), qXts(N / 16 + 1);
+  std::vector<uint8_t> qAc((size_t)s * s / 2 + 1), qAs((size_t)s * s / 16 + 1);
+  std::vector<uint8_t> qBc((size_t)s * s / 2 + 1), qBs((size_t)s * s / 16 + 1);
+
+  float amax_X = amax_of(X.data(), (int64_t)N);
+  float sg_X = scale_exact(amax_X);  // initial operand: exact rule
+
+  for (int k = 0; k < steps; ++k) {
+    const bool rec = tr && tr->iter == k;
+    if (rec) {
+      if (tr->amax_in) *tr->amax_in = amax_X;
+      if (tr->X_in) std::memcpy(tr->X_in, X.data(), N * sizeof(float));
+    }
+    if (!prm->quantize) {
+      // textbook iteration, FP64 sums, FP32 storage
+      std::vector<double> Xd(X.begin(), X.end());
+      gemm_nt(Xd.data(), Xd.data(), s, s, l, A.data(), 1);
+      std::vector<double> Ad(A.begin(), A.end());
+      gemm_nt(Ad.data(), Ad.data(), s, s, s, S.data(), 1);
+      for (size_t i = 0; i < (size_t)s * s; ++i) B[i] = cb * A[i] + cc * S[i];
+      transpose(X.data(), s, l, Xt.data());
+      std::vector<double> Bd(B.begin(), B.end()), Xtd(Xt.begin(), Xt.end());
+      gemm_nt(Bd.data(), Xtd.data(), s, l, s, P.data(), 0);
+      for (size_t i = 0; i < N; ++i) X[i] = ca * X[i] + P[i];
+    } else {
+      // qX = Q_1x16(X), qX^{16x1} = Q_16x1(X) = Q_1x16(X^T), one global scale
+      transpose(X.data(), s, l, Xt.data());
+      quantize_1x16(X.data(), s, l, sg_X, qXc.data(), qXs.data());
+      quantize_1x16(Xt.data(), l, s, sg_X, qXtc.data(), qXts.data());
+      // A = qX qX^T
+      {
+        std::vector<double> d = decode_f64(qXc.data(), qXs.data(), sg_X, s, l);
+        gemm_nt(d.data(), d.data(), s, s, l, A.data(), 1);
+      }
+      float amax_A = amax_of(A.data(), (int64_t)s * s);
+      float bound_A = std::min(2.0f * (float)l * amax_X * amax_X, 4.0f);
+      float sg_A = prm->exact_scales ? scale_exact(amax_A) : scale_predicted(bound_A);
+      // qA = Q_1x16(A); A is symmetric so Q_16x1(A) is the transpose of qA
+      quantize_1x16(A.data(), s, s, sg_A, qAc.data(), qAs.data());
+      {
+        std::vector<double> d = decode_f64(qAc.data(), qAs.data(), sg_A, s, s);
+        gemm_nt(d.data(), d.data(), s, s, s, S.data(), 1);
+      }
+      // B = b A + c (qA qA^{16x1}), each product and the sum rounded to FP32
+      for (size_t i = 0; i < (size_t)s * s; ++i) {
+        float t1 = cb * A[i];
+        float t2 = cc * S[i];
+        B[i] = t1 + t2;
+      }
+      float amax_B = amax_of(B.data(), (int64_t)s * s);
+      float bound_B = (std::fabs(cb) + 4.0f * std::fabs(cc)) * amax_A;
+      float sg_B = prm->exact_scales ? scale_exact(amax_B) : scale_predicted(bound_B);
+      quantize_1x16(B.data(), s, s, sg_B, qBc.data(), qBs.data());
+      // X+ = a X + qB qX^{16x1}
+      {
+        std::vector<double> db = decode_f64(qBc.data(), qBs.data(), sg_B, s, s);
+        std::vector<double> dx = decode_f64(qXtc.data(), qXts.data(), sg_X, l, s);
+        gemm_nt(db.data(), dx.data(), s, l, s, P.data(), 0);
+      }
+      if (rec) {
+        if (tr->qX_codes) std::memcpy(tr->qX_codes, qXc.data(), N / 2);
+        if (tr->qX_scales) std::memcpy(tr->qX_scales, qXs.data(), N / 16);
+        if (tr->qXt_codes) std::memcpy(tr->qXt_codes, qXtc.data(), N / 2);
+        if (tr->qXt_scales) std::memcpy(tr->qXt_scales, qXts.data(), N / 16);
+        if (tr->sg_X) *tr->sg_X = sg_X;
+        if (tr->A) std::memcpy(tr->A, A.data(), (size_t)s * s * 4);
+        if (tr->qA_codes) std::memcpy(tr->qA_codes, qAc.data(), (size_t)s * s / 2);
+        if (tr->qA_scales) std::memcpy(tr->qA_scales, qAs.data(), (size_t)s * s / 16);
+        if (tr->sg_A) *tr->sg_A = sg_A;
+        if (tr->S) std::memcpy(tr->S, S.data(), (size_t)s * s * 4);
+        if (tr->B) std::memcpy(tr->B, B.data(), (size_t)s * s * 4);
+        if (tr->qB_codes) std::memcpy(tr->qB_codes, qBc.data(), (size_t)s * s / 2);
+        if (tr->qB_scales) std::memcpy(tr->qB_scales, qBs.data(), (size_t)s * s / 16);
+        if (tr->sg_B) *tr->sg_B = sg_B;
+      }
+      float amax_prev = amax_X;
+      for (size_t i = 0; i < N; ++i) {
+        float t1 = ca * X[i];
+        X[i] = t1 + P[i];
+      }
+      amax_X = amax_of(X.data(), (int64_t)N);
+      float bound_X = 4.0f * std::fabs(ca) * amax_prev;
+      sg_X = prm->exact_scales ? scale_exact(amax_X) : scale_predicted(bound_X);
+    }
+    if (rec && tr->X_out) std::memcpy(tr->X_out, X.data(), N * sizeof(float));
+  }
+
+  if (tall) transpose(X.data(), s, l, out); else std::memcpy(out, X.data(), N * sizeof(float));
+  return 0;
+}
+
+}  // extern "C"
