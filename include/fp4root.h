@@ -1,0 +1,170 @@
+/* fp4root.h -- C ABI of the NVFP4 Root Newton-Schulz library for B200 (sm_100a).
+ *
+ * One hot path of the paper "Full-Stack FP4": the NVFP4 Root step (Section 3.4),
+ * i.e. outlier clip, Frobenius normalisation and k Newton-Schulz iterations whose
+ * three matrix products per iteration run on NVFP4 operands (Section 2, "NVFP4
+ * format": E2M1 values, one E4M3 scale per 16 contiguous elements of the
+ * contraction axis, one FP32 scale per tensor) with FP32 accumulation.
+ *
+ * General rules
+ *   - Every pointer named "device" is a CUDA device pointer on the current device;
+ *     every other pointer is host memory that is read before the call returns.
+ *   - The caller owns all buffers.  The library keeps no state between calls except
+ *     the driver entry point it resolves on first use.  It allocates no device
+ *     memory.
+ *   - All work is enqueued on `stream`; no call synchronises the host except
+ *     fp4_last_device_status.
+ *   - Shapes: every matrix dimension must be a positive multiple of 128, else
+ *     FP4_ERR_SHAPE.  Device pointers must be 16-byte aligned (the workspace 1024),
+ *     else FP4_ERR_ALIGNMENT.
+ *   - Errors are return codes.  A kernel that gives up on a bounded wait records
+ *     FP4_ERR_DEVICE_TIMEOUT in the workspace header and ends normally; it never
+ *     traps.  Read it with fp4_last_device_status.
+ *   - Non-finite inputs give unspecified values but no fault (conversions saturate).
+ *   - There is no CPU fallback: on a device that is not compute capability 10.x
+ *     every compute entry point returns FP4_ERR_ARCH.
+ */
+#ifndef FP4ROOT_H_
+#define FP4ROOT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct CUstream_st* cudaStream_t;
+
+typedef enum {
+  FP4_OK = 0,
+  FP4_ERR_INVALID_ARG = 1,
+  FP4_ERR_SHAPE = 2,
+  FP4_ERR_ALIGNMENT = 3,
+  FP4_ERR_WORKSPACE = 4,
+  FP4_ERR_ARCH = 5,
+  FP4_ERR_CUDA = 6,
+  FP4_ERR_DEVICE_TIMEOUT = 7,
+  FP4_ERR_UNIMPLEMENTED = 8
+} fp4_status;
+
+/* flags of fp4_ns_params */
+#define FP4_FLAG_KEEP_OPERANDS 1u /* the last iteration also writes the NVFP4 copies of
+                                     its result (otherwise skipped as dead work); for
+                                     inspection through fp4_root_ns_workspace_layout */
+
+/* Parameters of the step.  Pass NULL for the defaults noted on each field. */
+typedef struct {
+  float a, b, c;       /* quintic coefficients of X+ = aX + (bA + cA^2)X (Section 2, "Root
+                          optimizer").  a = NaN (default): fp4_root_coeffs(m, n, steps).   */
+  float clip_quantile; /* outlier clip (Section 3.4, "p99 outlier clipping"): entries are
+                          clamped to the nearest-rank quantile of |G|, resolved to parts
+                          per million.  Default 0.99; <= 0 or >= 1 disables the clip.      */
+  float eps;           /* X0 = G_c / (||G_c||_F + eps).  Default 1e-7.                     */
+  uint32_t flags;      /* FP4_FLAG_*; default 0                                            */
+} fp4_ns_params;
+
+const char* fp4_status_string(fp4_status s);
+
+/* ---- NVFP4 block quantiser (Section 2, "NVFP4 format"; Q_1x16 of Section 3.4) ----------
+ *
+ * x: device, row-major rows x cols FP32 (leading dimension = cols).
+ * codes: device, out, rows x cols/2 bytes row-major; byte j of a row holds element 2j in
+ *   bits 3:0 and element 2j+1 in bits 7:4; a nibble is sign<<3 | index into
+ *   {0, 0.5, 1, 1.5, 2, 3, 4, 6}.
+ * scales: device, out, fp4_scale_bytes(rows, cols) bytes of unsigned E4M3 block scales in
+ *   the layout the tcgen05 block-scaled MMA reads: 512-byte atoms that hold 128 rows x 4
+ *   consecutive blocks; the scale of (row r, block kb) is at
+ *     ((r/128) * (cols/64) + kb/4) * 512 + (r%32)*16 + ((r%128)/32)*4 + kb%4.
+ * tensor_scale: device, out, one FP32: s_g = amax(x)/2688 (1 if x is all zero).  It is
+ *   also used as scratch while the call runs.
+ * Decoded value of an element = E2M1 value * E4M3 scale * s_g.  Rounding is to nearest,
+ * ties to even, saturating.  Block scale = E4M3(amax_block / (6 s_g)); elements are
+ * multiplied by the FP32 reciprocal of (scale * s_g) before conversion.
+ * flags: must be 0.
+ */
+size_t fp4_scale_bytes(int64_t rows, int64_t cols);
+fp4_status fp4_quantize(const float* x, int64_t rows, int64_t cols, uint8_t* codes,
+                        uint8_t* scales, float* tensor_scale, uint32_t flags,
+                        cudaStream_t stream);
+
+/* ---- shape-dependent coefficients (Section 3.4: "Root's shape-dependent coefficients") --
+ * Host function, pure.  The paper does not print the values; this provider returns a
+ * quintic with p(1) = 1, p'(1) = 0 whose slope at zero grows with max(m,n)/min(m,n)
+ * (15/8, -10/8, 3/8 for square matrices).  abc: host, out, 3 floats.
+ */
+fp4_status fp4_root_coeffs(int64_t m, int64_t n, int steps, float abc[3]);
+
+/* ---- the Root Newton-Schulz step on one matrix (Section 3.4, display equations) --------
+ *
+ * G: device, m x n FP32 row-major.  out: device, m x n FP32 row-major; may equal G exactly
+ *   (no partial overlap).  steps >= 0 iterations (0: clip and normalise only).
+ * ws: device workspace of at least fp4_root_ns_workspace_bytes(m, n, steps, flags) bytes,
+ *   1024-byte aligned; its contents need not be initialised and are overwritten.
+ * Computes, with s = min(m,n), l = max(m,n) and X = G or G^T so that X is s x l:
+ *   tau = quantile of |G|, G_c = clamp(G, -tau, tau), X0 = G_c/(||G_c||_F + eps), then
+ *   per iteration A = qX qX^T, B = bA + c qA qA^T, X+ = aX + qB qX^{16x1}, every q*
+ *   an NVFP4 quantisation with 16-element blocks along the contraction axis; the
+ *   result is X_steps (transposed back when m > n).
+ * Two calls that share a workspace must not overlap in time.
+ */
+size_t fp4_root_ns_workspace_bytes(int64_t m, int64_t n, int steps, uint32_t flags);
+fp4_status fp4_root_ns(const float* G, float* out, int64_t m, int64_t n, int steps,
+                       const fp4_ns_params* p, void* ws, size_t ws_bytes, cudaStream_t stream);
+
+/* ---- many matrices of different shapes in one call (the matrices of a layer stack) ------
+ * count matrices; G, out, m, n: host arrays of length count (G[i], out[i] device pointers).
+ * One parameter block applies to all (coefficients per matrix when p->a is NaN).
+ * ws: device, at least fp4_root_ns_batched_workspace_bytes(...) bytes, 1024-byte aligned.
+ */
+size_t fp4_root_ns_batched_workspace_bytes(int count, const int64_t* m, const int64_t* n,
+                                           int steps, uint32_t flags);
+fp4_status fp4_root_ns_batched(int count, const float* const* G, float* const* out,
+                               const int64_t* m, const int64_t* n, int steps,
+                               const fp4_ns_params* p, void* ws, size_t ws_bytes,
+                               cudaStream_t stream);
+
+/* Synchronises `stream`, then returns the status word that the kernels of the last call
+ * on workspace `ws` left in its header: FP4_OK or FP4_ERR_DEVICE_TIMEOUT. */
+fp4_status fp4_last_device_status(const void* ws, cudaStream_t stream);
+
+/* ---- inspection (tests) -----------------------------------------------------------------
+ * Byte offsets, inside the workspace of fp4_root_ns(m, n, ...), of the intermediates the
+ * last executed iteration leaves behind.  All are in the work orientation (s x l).
+ * Operands are NVFP4 tensors: codes as in fp4_quantize, scales in the atom layout, tensor
+ * scale in the FP32 array `scalars` at the given index.
+ */
+typedef struct {
+  size_t header;      /* uint32 status word first                                  */
+  size_t scalars;     /* float array, see the idx_* fields                          */
+  size_t X;           /* FP32 s x l: X (only when m > n; otherwise X lives in out)  */
+  size_t A;           /* FP32 s x s: A of the last iteration, upper-triangle tiles  */
+  size_t qX_codes, qX_scales;       /* Q_1x16(X): G1 operand, s x l                 */
+  size_t qXt_codes[2], qXt_scales[2]; /* Q_1x16(X^T): G3 operand, l x s, ping-pong  */
+  size_t qA_codes, qA_scales;       /* s x s                                        */
+  size_t qB_codes, qB_scales;       /* s x s                                        */
+  int32_t idx_tau, idx_nu, idx_inv; /* scalars[idx]                                 */
+  int32_t idx_amax_X0;              /* scalars[idx + k] = amax of X_k               */
+  int32_t idx_amax_A0;              /* scalars[idx + k] = amax of A_k               */
+  int32_t idx_sg_X0;                /* scalars[idx + k] = tensor scale of qX_k      */
+  int32_t idx_sg_A0, idx_sg_B0;     /* likewise for qA_k, qB_k                      */
+  size_t total;
+} fp4_ws_layout;
+fp4_status fp4_root_ns_workspace_layout(int64_t m, int64_t n, int steps, uint32_t flags,
+                                        fp4_ws_layout* layout);
+
+/* One block-scaled product on the tcgen05 path, for testing the GEMM alone:
+ * D = (deq(A) deq(B)^T) as FP32, A: M x K, B: N x K NVFP4 tensors (device; codes, scales in
+ * the atom layout, host tensor scales).  D: device, M x N FP32 row-major.  M, N, K
+ * multiples of 128. */
+fp4_status fp4_gemm_nt(const uint8_t* a_codes, const uint8_t* a_scales, float a_tensor_scale,
+                       const uint8_t* b_codes, const uint8_t* b_scales, float b_tensor_scale,
+                       int64_t M, int64_t N, int64_t K, float* D,
+                       uint32_t* device_status /* device, may be NULL: receives
+                       FP4_ERR_DEVICE_TIMEOUT if a bounded wait gives up */,
+                       cudaStream_t stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FP4ROOT_H_ */

@@ -1,2 +1,13 @@
-"""NVFP4 Root Newton-Schulz step for B200 (sm_100a)."""
+"""NVFP4 Root Newton-Schulz step for B200 (sm_100a).
+
+The product is the C-ABI library ``libfp4root.so`` built from ``csrc/``;
+``binding`` is its thin ctypes front end and ``workloads`` the seeded synthetic
+input generators.  There is no CPU fallback: every entry point raises if the
+CUDA library is missing.
+"""
 from . import workloads  # noqa: F401
+from .binding import (  # noqa: F401
+    Fp4Error, NsParams, fp4_gemm_nt, fp4_last_device_status, fp4_quantize, fp4_root_coeffs, fp4_root_ns,
+    fp4_root_ns_batched, fp4_root_ns_batched_workspace_bytes, fp4_root_ns_workspace_bytes,
+    fp4_root_ns_workspace_layout, fp4_scale_bytes, fp4_status_string, library_path, load_library,
+)

@@ -1,0 +1,179 @@
+"""ctypes binding of libfp4root.so: argument marshalling only.
+
+Functions carry the names of the C ABI (include/fp4root.h).  Tensors are torch CUDA
+tensors used purely as device memory; streams are torch streams.  Every step of the
+path runs in the library's kernels; if the library is missing the first call raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libfp4root.so")
+_lib = None
+
+FP4_FLAG_KEEP_OPERANDS = 1
+STATUS_NAMES = {0: "FP4_OK", 1: "FP4_ERR_INVALID_ARG", 2: "FP4_ERR_SHAPE", 3: "FP4_ERR_ALIGNMENT",
+                4: "FP4_ERR_WORKSPACE", 5: "FP4_ERR_ARCH", 6: "FP4_ERR_CUDA", 7: "FP4_ERR_DEVICE_TIMEOUT",
+                8: "FP4_ERR_UNIMPLEMENTED"}
+
+EXPORTS = ("fp4_status_string", "fp4_scale_bytes", "fp4_quantize", "fp4_root_coeffs",
+           "fp4_root_ns_workspace_bytes", "fp4_root_ns", "fp4_root_ns_batched_workspace_bytes",
+           "fp4_root_ns_batched", "fp4_last_device_status", "fp4_root_ns_workspace_layout", "fp4_gemm_nt")
+
+
+class Fp4Error(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = int(code)
+        super().__init__(f"{where}: {STATUS_NAMES.get(self.code, self.code)} ({fp4_status_string(self.code)})")
+
+
+class NsParams(C.Structure):
+    """fp4_ns_params"""
+    _fields_ = [("a", C.c_float), ("b", C.c_float), ("c", C.c_float), ("clip_quantile", C.c_float),
+                ("eps", C.c_float), ("flags", C.c_uint32)]
+
+    @classmethod
+    def make(cls, abc=None, clip_quantile=0.99, eps=1e-7, flags=0):
+        p = cls()
+        if abc is None:
+            p.a = p.b = p.c = float("nan")
+        else:
+            p.a, p.b, p.c = [float(v) for v in abc]
+        p.clip_quantile, p.eps, p.flags = float(clip_quantile), float(eps), int(flags)
+        return p
+
+
+class WsLayout(C.Structure):
+    """fp4_ws_layout"""
+    _fields_ = [("header", C.c_size_t), ("scalars", C.c_size_t), ("X", C.c_size_t), ("A", C.c_size_t),
+                ("qX_codes", C.c_size_t), ("qX_scales", C.c_size_t),
+                ("qXt_codes", C.c_size_t * 2), ("qXt_scales", C.c_size_t * 2),
+                ("qA_codes", C.c_size_t), ("qA_scales", C.c_size_t),
+                ("qB_codes", C.c_size_t), ("qB_scales", C.c_size_t),
+                ("idx_tau", C.c_int32), ("idx_nu", C.c_int32), ("idx_inv", C.c_int32),
+                ("idx_amax_X0", C.c_int32), ("idx_amax_A0", C.c_int32),
+                ("idx_sg_X0", C.c_int32), ("idx_sg_A0", C.c_int32), ("idx_sg_B0", C.c_int32),
+                ("total", C.c_size_t)]
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def load_library():
+    """Loads libfp4root.so (built in-tree by build.py).  Raises if it is missing:
+    there is no fallback implementation."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(_LIB_PATH):
+        raise RuntimeError(f"{_LIB_PATH} is missing: build it with `python -m paper_2607_04422_b200.build` "
+                           "(nvcc, sm_100a); this package has no CPU or PyTorch fallback")
+    L = C.CDLL(_LIB_PATH)
+    vp, i64, u32, sz = C.c_void_p, C.c_int64, C.c_uint32, C.c_size_t
+    L.fp4_status_string.argtypes = [C.c_int]; L.fp4_status_string.restype = C.c_char_p
+    L.fp4_scale_bytes.argtypes = [i64, i64]; L.fp4_scale_bytes.restype = sz
+    L.fp4_quantize.argtypes = [vp, i64, i64, vp, vp, vp, u32, vp]; L.fp4_quantize.restype = C.c_int
+    L.fp4_root_coeffs.argtypes = [i64, i64, C.c_int, C.POINTER(C.c_float)]; L.fp4_root_coeffs.restype = C.c_int
+    L.fp4_root_ns_workspace_bytes.argtypes = [i64, i64, C.c_int, u32]; L.fp4_root_ns_workspace_bytes.restype = sz
+    L.fp4_root_ns.argtypes = [vp, vp, i64, i64, C.c_int, C.POINTER(NsParams), vp, sz, vp]
+    L.fp4_root_ns.restype = C.c_int
+    L.fp4_root_ns_batched_workspace_bytes.argtypes = [C.c_int, C.POINTER(i64), C.POINTER(i64), C.c_int, u32]
+    L.fp4_root_ns_batched_workspace_bytes.restype = sz
+    L.fp4_root_ns_batched.argtypes = [C.c_int, C.POINTER(vp), C.POINTER(vp), C.POINTER(i64), C.POINTER(i64),
+                                      C.c_int, C.POINTER(NsParams), vp, sz, vp]
+    L.fp4_root_ns_batched.restype = C.c_int
+    L.fp4_last_device_status.argtypes = [vp, vp]; L.fp4_last_device_status.restype = C.c_int
+    L.fp4_root_ns_workspace_layout.argtypes = [i64, i64, C.c_int, u32, C.POINTER(WsLayout)]
+    L.fp4_root_ns_workspace_layout.restype = C.c_int
+    L.fp4_gemm_nt.argtypes = [vp, vp, C.c_float, vp, vp, C.c_float, i64, i64, i64, vp, vp, vp]
+    L.fp4_gemm_nt.restype = C.c_int
+    _lib = L
+    return L
+
+
+def _stream(stream=None) -> int:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return int(s.cuda_stream)
+
+
+def _check(rc: int, where: str):
+    if rc != 0:
+        raise Fp4Error(rc, where)
+
+
+def fp4_status_string(code: int) -> str:
+    return load_library().fp4_status_string(int(code)).decode()
+
+
+def fp4_scale_bytes(rows: int, cols: int) -> int:
+    return int(load_library().fp4_scale_bytes(rows, cols))
+
+
+def fp4_root_coeffs(m: int, n: int, steps: int = 5):
+    abc = (C.c_float * 3)()
+    _check(load_library().fp4_root_coeffs(m, n, steps, abc), "fp4_root_coeffs")
+    return float(abc[0]), float(abc[1]), float(abc[2])
+
+
+def fp4_quantize(x: torch.Tensor, codes: torch.Tensor, scales: torch.Tensor, tensor_scale: torch.Tensor,
+                 flags: int = 0, stream=None) -> None:
+    rows, cols = x.shape
+    _check(load_library().fp4_quantize(x.data_ptr(), rows, cols, codes.data_ptr(), scales.data_ptr(),
+                                       tensor_scale.data_ptr(), flags, _stream(stream)), "fp4_quantize")
+
+
+def fp4_root_ns_workspace_bytes(m: int, n: int, steps: int = 5, flags: int = 0) -> int:
+    return int(load_library().fp4_root_ns_workspace_bytes(m, n, steps, flags))
+
+
+def fp4_root_ns_workspace_layout(m: int, n: int, steps: int = 5, flags: int = 0) -> WsLayout:
+    lay = WsLayout()
+    _check(load_library().fp4_root_ns_workspace_layout(m, n, steps, flags, C.byref(lay)),
+           "fp4_root_ns_workspace_layout")
+    return lay
+
+
+def fp4_root_ns(G: torch.Tensor, out: torch.Tensor, steps: int, params: NsParams | None, ws: torch.Tensor,
+                stream=None) -> None:
+    m, n = G.shape
+    p = C.byref(params) if params is not None else None
+    _check(load_library().fp4_root_ns(G.data_ptr(), out.data_ptr(), m, n, steps, p, ws.data_ptr(),
+                                      ws.numel() * ws.element_size(), _stream(stream)), "fp4_root_ns")
+
+
+def fp4_root_ns_batched_workspace_bytes(shapes, steps: int = 5, flags: int = 0) -> int:
+    cnt = len(shapes)
+    m = (C.c_int64 * cnt)(*[s[0] for s in shapes])
+    n = (C.c_int64 * cnt)(*[s[1] for s in shapes])
+    return int(load_library().fp4_root_ns_batched_workspace_bytes(cnt, m, n, steps, flags))
+
+
+def fp4_root_ns_batched(Gs, outs, steps: int, params: NsParams | None, ws: torch.Tensor, stream=None) -> None:
+    cnt = len(Gs)
+    g = (C.c_void_p * cnt)(*[t.data_ptr() for t in Gs])
+    o = (C.c_void_p * cnt)(*[t.data_ptr() for t in outs])
+    m = (C.c_int64 * cnt)(*[t.shape[0] for t in Gs])
+    n = (C.c_int64 * cnt)(*[t.shape[1] for t in Gs])
+    p = C.byref(params) if params is not None else None
+    _check(load_library().fp4_root_ns_batched(cnt, g, o, m, n, steps, p, ws.data_ptr(),
+                                              ws.numel() * ws.element_size(), _stream(stream)),
+           "fp4_root_ns_batched")
+
+
+def fp4_last_device_status(ws: torch.Tensor, stream=None) -> int:
+    return int(load_library().fp4_last_device_status(ws.data_ptr(), _stream(stream)))
+
+
+def fp4_gemm_nt(a_codes, a_scales, a_sg: float, b_codes, b_scales, b_sg: float, D: torch.Tensor,
+                status: torch.Tensor | None = None, stream=None) -> None:
+    M, K = a_codes.shape[0], a_codes.shape[1] * 2
+    N = b_codes.shape[0]
+    _check(load_library().fp4_gemm_nt(a_codes.data_ptr(), a_scales.data_ptr(), float(a_sg), b_codes.data_ptr(),
+                                      b_scales.data_ptr(), float(b_sg), M, N, K, D.data_ptr(),
+                                      status.data_ptr() if status is not None else None, _stream(stream)),
+           "fp4_gemm_nt")

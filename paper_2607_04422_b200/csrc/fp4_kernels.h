@@ -1,0 +1,83 @@
+// Internal interfaces between the translation units of the library.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <string.h>
+
+#include "fp4_common.cuh"
+
+namespace fp4 {
+
+constexpr int kMaxSteps = 64;
+
+// First 128 bytes of a workspace.
+struct NsHeader {
+  uint32_t status;       // fp4_status left by the kernels (0 or FP4_ERR_DEVICE_TIMEOUT)
+  uint32_t reserved[3];
+  uint32_t sel_prefix;   // radix select: magnitude bits fixed so far
+  uint32_t sel_rank;     // radix select: rank still to find inside the prefix
+  uint32_t maxabs_bits;  // max |clamped g| as a bit pattern
+  uint32_t pad[25];
+};
+
+// Indices into the FP32 `scalars` array of a workspace.
+struct NsScalarIdx {
+  int tau, nu, inv;
+  int amax_X0, amax_A0;        // + k
+  int sg_X0, sg_A0, sg_B0;     // + k
+};
+
+struct NsPlan {
+  fp4_ws_layout lay;
+  NsScalarIdx ix;
+  int64_t m, n, s, l;
+  int tall;
+  int clip;
+  int64_t clip_rank;
+  float eps;
+  int sms;
+  int stat_blocks;
+  size_t off_hist, off_partial;
+  size_t zero_bytes;  // header + scalars + histogram, cleared at the start of a call
+};
+
+// Epilogue variants of the GEMM kernel.
+enum GemmMode : int {
+  kPlain = 0,  // D = acc * sgA*sgB                                  (fp4_gemm_nt)
+  kG1 = 1,     // A = qX qX^T; store A, emit qA (both triangles), track amax(A)
+  kG2 = 2,     // S = qA qA^T; B = bA + cS; emit qB (both triangles)
+  kG3 = 3      // P = qB qXt^T; X+ = aX + P; store X+, emit qX+, qXt+, track amax(X+)
+};
+
+struct GemmArgs {
+  const uint8_t* sfa;  // scale atoms of the row operand
+  const uint8_t* sfb;  // scale atoms of the column operand
+  int K;               // contraction length in elements (multiple of 128)
+  int tiles_m, tiles_n;
+  int symmetric;       // only tiles with tile_n >= tile_m; mirrored quantised output
+  float* scalars;      // workspace scalars (device)
+  NsScalarIdx ix;
+  int iter;            // Newton-Schulz iteration index k
+  float ca, cb, cc;    // coefficients
+  float l_cols;        // (float) l, for the bound on amax(A)
+  float sg_a, sg_b;    // kPlain: tensor scales from the host
+  uint8_t* rq_codes; uint8_t* rq_sf; int rq_K;  // quantised output, blocks along this tile's columns
+  uint8_t* cq_codes; uint8_t* cq_sf; int cq_K;  // quantised output, blocks along this tile's rows
+  int write_q;         // emit the quantised outputs
+  uint32_t* status;
+};
+
+cudaError_t launch_quantize(const float* x, int64_t rows, int64_t cols, uint8_t* codes, uint8_t* scales,
+                            float* tensor_scale, int sms, cudaStream_t st);
+cudaError_t launch_prologue(const float* G, int64_t m, int64_t n, const NsPlan& pl, uint8_t* ws, float* X,
+                            int write_q, bool clear_status, cudaStream_t st);
+cudaError_t launch_transpose_out(const float* X, int64_t s, int64_t l, float* out, cudaStream_t st);
+cudaError_t prologue_set_attributes();
+
+cudaError_t gemm_set_attributes();
+cudaError_t launch_gemm(GemmMode mode, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmAux,
+                        const CUtensorMap& tmOut, const GemmArgs& args, int sms, cudaStream_t st);
+
+}  // namespace fp4

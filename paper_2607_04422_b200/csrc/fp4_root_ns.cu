@@ -1,0 +1,379 @@
+// Host side of the library: argument checks, workspace layout, TMA descriptors, and the
+// sequence of launches of the Root Newton-Schulz step (Section 3.4).  Everything here
+// only enqueues work on the caller's stream.
+#include <cmath>
+#include <mutex>
+
+#include "fp4_kernels.h"
+
+namespace fp4 {
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct DeviceInfo {
+  bool ready = false;
+  fp4_status status = FP4_OK;
+  int sms = 0;
+  EncodeTiledFn encode = nullptr;
+};
+DeviceInfo g_dev[64];
+std::mutex g_mu;
+
+// Per-device set-up on first use: architecture check, driver entry point, kernel attributes.
+const DeviceInfo* device_info() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  std::lock_guard<std::mutex> lock(g_mu);
+  DeviceInfo& d = g_dev[dev];
+  if (d.ready) return &d;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) { d.status = FP4_ERR_CUDA; d.ready = true; return &d; }
+  if (prop.major != 10) { d.status = FP4_ERR_ARCH; d.ready = true; return &d; }
+  d.sms = prop.multiProcessorCount;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess || fn == nullptr) {
+    d.status = FP4_ERR_CUDA; d.ready = true; return &d;
+  }
+  d.encode = reinterpret_cast<EncodeTiledFn>(fn);
+  if (gemm_set_attributes() != cudaSuccess || prologue_set_attributes() != cudaSuccess) d.status = FP4_ERR_CUDA;
+  d.ready = true;
+  return &d;
+}
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+inline bool shape_ok(int64_t v) { return v >= 128 && v % 128 == 0 && v <= (1 << 20); }
+
+// 2-D map over a row-major byte matrix (NVFP4 codes): box = 64 bytes x 128 rows, 64-byte swizzle.
+bool make_codes_map(const DeviceInfo* d, CUtensorMap* tm, const void* base, int64_t rows, int64_t row_bytes) {
+  cuuint64_t dims[2] = {(cuuint64_t)row_bytes, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)row_bytes};
+  cuuint32_t box[2] = {64, 128};
+  cuuint32_t estr[2] = {1, 1};
+  return d->encode(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+// 2-D map over a row-major FP32 matrix: box = 16 columns x 128 rows, 64-byte swizzle.
+bool make_f32_map(const DeviceInfo* d, CUtensorMap* tm, const void* base, int64_t rows, int64_t cols) {
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)cols * 4};
+  cuuint32_t box[2] = {16, 128};
+  cuuint32_t estr[2] = {1, 1};
+  return d->encode(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+void default_params(fp4_ns_params* p) {
+  p->a = p->b = p->c = NAN;
+  p->clip_quantile = 0.99f;
+  p->eps = 1e-7f;
+  p->flags = 0;
+}
+
+int64_t quantile_rank(int64_t n, float q) {
+  // resolved to parts per million so that 0.99f means 99/100
+  int64_t ppm = (int64_t)llround((double)q * 1e6);
+  int64_t k = (ppm * n + 999999) / 1000000;
+  if (k < 1) k = 1;
+  if (k > n) k = n;
+  return k;
+}
+
+void coeffs(int64_t m, int64_t n, float abc[3]) {
+  // quintic with p(1) = 1, p'(1) = 0: b = 2.5 - 2a, c = a - 1.5; a from the aspect ratio
+  double s = (double)(m < n ? m : n), l = (double)(m < n ? n : m);
+  double delta = (std::sqrt(7.0 / 3.0) - 1.0) / 2.0;
+  double rr = 1.0 + delta * (1.0 + std::sqrt(s / l));
+  double R = rr * rr;
+  double a = (1.5 * R - 1.0) / (R - 1.0);
+  abc[0] = (float)a;
+  abc[1] = (float)(2.5 - 2.0 * a);
+  abc[2] = (float)(a - 1.5);
+}
+
+// Workspace layout of one matrix.
+fp4_status make_plan(int64_t m, int64_t n, int steps, const fp4_ns_params* p, int sms, NsPlan* pl) {
+  if (!shape_ok(m) || !shape_ok(n)) return FP4_ERR_SHAPE;
+  if (steps < 0 || steps > kMaxSteps) return FP4_ERR_INVALID_ARG;
+  memset(pl, 0, sizeof(*pl));
+  pl->m = m; pl->n = n;
+  pl->tall = m > n;
+  pl->s = m < n ? m : n;
+  pl->l = m < n ? n : m;
+  const int64_t s = pl->s, l = pl->l;
+  pl->clip = p->clip_quantile > 0.0f && p->clip_quantile < 1.0f;
+  pl->clip_rank = pl->clip ? quantile_rank(m * n, p->clip_quantile) : 0;
+  pl->eps = p->eps;
+  pl->sms = sms;
+  int64_t blocks = (m * n / 4 + 1023) / 1024;
+  pl->stat_blocks = (int)(blocks < 1024 ? blocks : 1024);
+
+  NsScalarIdx& ix = pl->ix;
+  ix.tau = 0; ix.nu = 1; ix.inv = 2;
+  const int span = kMaxSteps + 2;
+  ix.amax_X0 = 8; ix.amax_A0 = 8 + span; ix.sg_X0 = 8 + 2 * span; ix.sg_A0 = 8 + 3 * span; ix.sg_B0 = 8 + 4 * span;
+  const size_t scalar_bytes = align_up((size_t)(8 + 5 * span) * 4, 1024);
+
+  fp4_ws_layout& L = pl->lay;
+  size_t off = 0;
+  L.header = off; off += 1024;
+  L.scalars = off; off += scalar_bytes;
+  pl->off_hist = off; off += 2048 * 4;
+  pl->zero_bytes = off;
+  pl->off_partial = off; off += 1024 * 8;
+  off = align_up(off, 1024);
+  L.X = off; if (pl->tall) off += align_up((size_t)s * l * 4, 1024);
+  L.A = off; off += align_up((size_t)s * s * 4, 1024);
+  L.qX_codes = off; off += align_up((size_t)s * l / 2, 1024);
+  L.qX_scales = off; off += align_up((size_t)s * l / 16, 1024);
+  for (int i = 0; i < 2; ++i) {
+    L.qXt_codes[i] = off; off += align_up((size_t)s * l / 2, 1024);
+    L.qXt_scales[i] = off; off += align_up((size_t)s * l / 16, 1024);
+  }
+  L.qA_codes = off; off += align_up((size_t)s * s / 2, 1024);
+  L.qA_scales = off; off += align_up((size_t)s * s / 16, 1024);
+  L.qB_codes = off; off += align_up((size_t)s * s / 2, 1024);
+  L.qB_scales = off; off += align_up((size_t)s * s / 16, 1024);
+  L.idx_tau = ix.tau; L.idx_nu = ix.nu; L.idx_inv = ix.inv;
+  L.idx_amax_X0 = ix.amax_X0; L.idx_amax_A0 = ix.amax_A0;
+  L.idx_sg_X0 = ix.sg_X0; L.idx_sg_A0 = ix.sg_A0; L.idx_sg_B0 = ix.sg_B0;
+  L.total = off;
+  return FP4_OK;
+}
+
+// Enqueue the whole step for one matrix.
+fp4_status run_one(const DeviceInfo* d, const float* G, float* out, int64_t m, int64_t n, int steps,
+                   const fp4_ns_params* p, uint8_t* ws, bool clear_status, cudaStream_t st) {
+  NsPlan pl;
+  fp4_status rc = make_plan(m, n, steps, p, d->sms, &pl);
+  if (rc != FP4_OK) return rc;
+  const fp4_ws_layout& L = pl.lay;
+  const int64_t s = pl.s, l = pl.l;
+  float abc[3] = {p->a, p->b, p->c};
+  if (std::isnan(p->a)) coeffs(m, n, abc);
+  const bool keep = (p->flags & FP4_FLAG_KEEP_OPERANDS) != 0;
+
+  // X lives in `out` unless the input is tall (then it is transposed back at the end)
+  float* X = pl.tall ? reinterpret_cast<float*>(ws + L.X) : out;
+  float* scalars = reinterpret_cast<float*>(ws + L.scalars);
+  uint32_t* status = reinterpret_cast<uint32_t*>(ws + L.header);
+
+  if (launch_prologue(G, m, n, pl, ws, X, steps > 0 || keep, clear_status, st) != cudaSuccess) return FP4_ERR_CUDA;
+
+  if (steps > 0) {
+    CUtensorMap tm_qX, tm_qXt[2], tm_qA, tm_qB, tm_A, tm_X;
+    bool ok = make_codes_map(d, &tm_qX, ws + L.qX_codes, s, l / 2) &&
+              make_codes_map(d, &tm_qXt[0], ws + L.qXt_codes[0], l, s / 2) &&
+              make_codes_map(d, &tm_qXt[1], ws + L.qXt_codes[1], l, s / 2) &&
+              make_codes_map(d, &tm_qA, ws + L.qA_codes, s, s / 2) &&
+              make_codes_map(d, &tm_qB, ws + L.qB_codes, s, s / 2) &&
+              make_f32_map(d, &tm_A, ws + L.A, s, s) && make_f32_map(d, &tm_X, X, s, l);
+    if (!ok) return FP4_ERR_CUDA;
+
+    GemmArgs base;
+    memset(&base, 0, sizeof(base));
+    base.scalars = scalars;
+    base.ix = pl.ix;
+    base.ca = abc[0]; base.cb = abc[1]; base.cc = abc[2];
+    base.l_cols = (float)l;
+    base.status = status;
+
+    for (int k = 0; k < steps; ++k) {
+      const int cur = k & 1, nxt = cur ^ 1;
+      const bool last = (k == steps - 1);
+      // G1: A = qX qX^T (upper-triangle tiles), qA in both triangles
+      GemmArgs a1 = base;
+      a1.iter = k; a1.K = (int)l; a1.tiles_m = a1.tiles_n = (int)(s / 128); a1.symmetric = 1;
+      a1.sfa = a1.sfb = ws + L.qX_scales;
+      a1.rq_codes = a1.cq_codes = ws + L.qA_codes; a1.rq_sf = a1.cq_sf = ws + L.qA_scales;
+      a1.rq_K = a1.cq_K = (int)s; a1.write_q = 1;
+      if (launch_gemm(kG1, tm_qX, tm_qX, tm_A, tm_A, a1, d->sms, st) != cudaSuccess) return FP4_ERR_CUDA;
+      // G2: B = bA + c qA qA^T, qB in both triangles
+      GemmArgs a2 = base;
+      a2.iter = k; a2.K = (int)s; a2.tiles_m = a2.tiles_n = (int)(s / 128); a2.symmetric = 1;
+      a2.sfa = a2.sfb = ws + L.qA_scales;
+      a2.rq_codes = a2.cq_codes = ws + L.qB_codes; a2.rq_sf = a2.cq_sf = ws + L.qB_scales;
+      a2.rq_K = a2.cq_K = (int)s; a2.write_q = 1;
+      if (launch_gemm(kG2, tm_qA, tm_qA, tm_A, tm_A, a2, d->sms, st) != cudaSuccess) return FP4_ERR_CUDA;
+      // G3: X+ = aX + qB qXt^T, in place on X; new operand copies unless this is the last iteration
+      GemmArgs a3 = base;
+      a3.iter = k; a3.K = (int)s; a3.tiles_m = (int)(s / 128); a3.tiles_n = (int)(l / 128); a3.symmetric = 0;
+      a3.sfa = ws + L.qB_scales; a3.sfb = ws + L.qXt_scales[cur];
+      a3.rq_codes = ws + L.qX_codes; a3.rq_sf = ws + L.qX_scales; a3.rq_K = (int)l;
+      a3.cq_codes = ws + L.qXt_codes[nxt]; a3.cq_sf = ws + L.qXt_scales[nxt]; a3.cq_K = (int)s;
+      a3.write_q = (!last || keep) ? 1 : 0;
+      if (launch_gemm(kG3, tm_qB, tm_qXt[cur], tm_X, tm_X, a3, d->sms, st) != cudaSuccess) return FP4_ERR_CUDA;
+    }
+  }
+  if (pl.tall) {
+    if (launch_transpose_out(X, s, l, out, st) != cudaSuccess) return FP4_ERR_CUDA;
+  }
+  return FP4_OK;
+}
+
+fp4_status check_common(const DeviceInfo** d) {
+  *d = device_info();
+  if (*d == nullptr) return FP4_ERR_CUDA;
+  return (*d)->status;
+}
+
+}  // namespace
+}  // namespace fp4
+
+using namespace fp4;
+
+extern "C" {
+
+const char* fp4_status_string(fp4_status s) {
+  switch (s) {
+    case FP4_OK: return "ok";
+    case FP4_ERR_INVALID_ARG: return "invalid argument";
+    case FP4_ERR_SHAPE: return "unsupported shape (dimensions must be positive multiples of 128)";
+    case FP4_ERR_ALIGNMENT: return "misaligned pointer";
+    case FP4_ERR_WORKSPACE: return "workspace too small";
+    case FP4_ERR_ARCH: return "device is not compute capability 10.x (sm_100a kernels only, no fallback)";
+    case FP4_ERR_CUDA: return "CUDA runtime or driver call failed";
+    case FP4_ERR_DEVICE_TIMEOUT: return "a kernel gave up on a bounded wait";
+    case FP4_ERR_UNIMPLEMENTED: return "not implemented";
+  }
+  return "unknown status";
+}
+
+size_t fp4_scale_bytes(int64_t rows, int64_t cols) {
+  if (rows <= 0 || cols <= 0) return 0;
+  return (size_t)((rows + 127) / 128) * (size_t)((cols + 63) / 64) * 512;
+}
+
+fp4_status fp4_quantize(const float* x, int64_t rows, int64_t cols, uint8_t* codes, uint8_t* scales,
+                        float* tensor_scale, uint32_t flags, cudaStream_t stream) {
+  if (!x || !codes || !scales || !tensor_scale || flags != 0) return FP4_ERR_INVALID_ARG;
+  if (!shape_ok(rows) || !shape_ok(cols)) return FP4_ERR_SHAPE;
+  if (!aligned(x, 16) || !aligned(codes, 16) || !aligned(scales, 16) || !aligned(tensor_scale, 4))
+    return FP4_ERR_ALIGNMENT;
+  const DeviceInfo* d;
+  fp4_status rc = check_common(&d);
+  if (rc != FP4_OK) return rc;
+  return launch_quantize(x, rows, cols, codes, scales, tensor_scale, d->sms, stream) == cudaSuccess ? FP4_OK
+                                                                                                      : FP4_ERR_CUDA;
+}
+
+fp4_status fp4_root_coeffs(int64_t m, int64_t n, int steps, float abc[3]) {
+  if (m <= 0 || n <= 0 || steps < 0 || !abc) return FP4_ERR_INVALID_ARG;
+  coeffs(m, n, abc);
+  return FP4_OK;
+}
+
+fp4_status fp4_root_ns_workspace_layout(int64_t m, int64_t n, int steps, uint32_t flags, fp4_ws_layout* layout) {
+  if (!layout) return FP4_ERR_INVALID_ARG;
+  fp4_ns_params p;
+  default_params(&p);
+  p.flags = flags;
+  NsPlan pl;
+  fp4_status rc = make_plan(m, n, steps, &p, 1, &pl);
+  if (rc != FP4_OK) return rc;
+  *layout = pl.lay;
+  return FP4_OK;
+}
+
+size_t fp4_root_ns_workspace_bytes(int64_t m, int64_t n, int steps, uint32_t flags) {
+  fp4_ws_layout L;
+  if (fp4_root_ns_workspace_layout(m, n, steps, flags, &L) != FP4_OK) return 0;
+  return L.total;
+}
+
+fp4_status fp4_root_ns(const float* G, float* out, int64_t m, int64_t n, int steps, const fp4_ns_params* p,
+                       void* ws, size_t ws_bytes, cudaStream_t stream) {
+  fp4_ns_params dp;
+  if (!p) { default_params(&dp); p = &dp; }
+  if (!G || !out || !ws) return FP4_ERR_INVALID_ARG;
+  if (!shape_ok(m) || !shape_ok(n)) return FP4_ERR_SHAPE;
+  if (steps < 0 || steps > kMaxSteps) return FP4_ERR_INVALID_ARG;
+  if (!aligned(G, 16) || !aligned(out, 16) || !aligned(ws, 1024)) return FP4_ERR_ALIGNMENT;
+  const size_t need = fp4_root_ns_workspace_bytes(m, n, steps, p->flags);
+  if (need == 0 || ws_bytes < need) return FP4_ERR_WORKSPACE;
+  const DeviceInfo* d;
+  fp4_status rc = check_common(&d);
+  if (rc != FP4_OK) return rc;
+  return run_one(d, G, out, m, n, steps, p, static_cast<uint8_t*>(ws), true, stream);
+}
+
+size_t fp4_root_ns_batched_workspace_bytes(int count, const int64_t* m, const int64_t* n, int steps,
+                                           uint32_t flags) {
+  if (count <= 0 || !m || !n) return 0;
+  size_t need = 0;
+  for (int i = 0; i < count; ++i) {
+    size_t b = fp4_root_ns_workspace_bytes(m[i], n[i], steps, flags);
+    if (b == 0) return 0;
+    if (b > need) need = b;
+  }
+  return need;
+}
+
+fp4_status fp4_root_ns_batched(int count, const float* const* G, float* const* out, const int64_t* m,
+                               const int64_t* n, int steps, const fp4_ns_params* p, void* ws, size_t ws_bytes,
+                               cudaStream_t stream) {
+  fp4_ns_params dp;
+  if (!p) { default_params(&dp); p = &dp; }
+  if (count < 0 || (count > 0 && (!G || !out || !m || !n)) || !ws) return FP4_ERR_INVALID_ARG;
+  if (steps < 0 || steps > kMaxSteps) return FP4_ERR_INVALID_ARG;
+  if (!aligned(ws, 1024)) return FP4_ERR_ALIGNMENT;
+  for (int i = 0; i < count; ++i) {
+    if (!G[i] || !out[i]) return FP4_ERR_INVALID_ARG;
+    if (!shape_ok(m[i]) || !shape_ok(n[i])) return FP4_ERR_SHAPE;
+    if (!aligned(G[i], 16) || !aligned(out[i], 16)) return FP4_ERR_ALIGNMENT;
+  }
+  if (count == 0) return FP4_OK;
+  const size_t need = fp4_root_ns_batched_workspace_bytes(count, m, n, steps, p->flags);
+  if (need == 0 || ws_bytes < need) return FP4_ERR_WORKSPACE;
+  const DeviceInfo* d;
+  fp4_status rc = check_common(&d);
+  if (rc != FP4_OK) return rc;
+  // Matrix after matrix on the one stream: the working set of a matrix (operands, A, X)
+  // stays in L2 across its stages, and the shared workspace is reused.
+  for (int i = 0; i < count; ++i) {
+    rc = run_one(d, G[i], out[i], m[i], n[i], steps, p, static_cast<uint8_t*>(ws), i == 0, stream);
+    if (rc != FP4_OK) return rc;
+  }
+  return FP4_OK;
+}
+
+fp4_status fp4_last_device_status(const void* ws, cudaStream_t stream) {
+  if (!ws) return FP4_ERR_INVALID_ARG;
+  uint32_t word = 0;
+  if (cudaMemcpyAsync(&word, ws, 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return FP4_ERR_CUDA;
+  if (cudaStreamSynchronize(stream) != cudaSuccess) return FP4_ERR_CUDA;
+  return word == 0 ? FP4_OK : (fp4_status)word;
+}
+
+fp4_status fp4_gemm_nt(const uint8_t* a_codes, const uint8_t* a_scales, float a_tensor_scale,
+                       const uint8_t* b_codes, const uint8_t* b_scales, float b_tensor_scale, int64_t M, int64_t N,
+                       int64_t K, float* D, uint32_t* device_status, cudaStream_t stream) {
+  if (!a_codes || !a_scales || !b_codes || !b_scales || !D) return FP4_ERR_INVALID_ARG;
+  if (!shape_ok(M) || !shape_ok(N) || !shape_ok(K)) return FP4_ERR_SHAPE;
+  if (!aligned(a_codes, 16) || !aligned(a_scales, 16) || !aligned(b_codes, 16) || !aligned(b_scales, 16) ||
+      !aligned(D, 16))
+    return FP4_ERR_ALIGNMENT;
+  const DeviceInfo* d;
+  fp4_status rc = check_common(&d);
+  if (rc != FP4_OK) return rc;
+  CUtensorMap tmA, tmB, tmD;
+  if (!make_codes_map(d, &tmA, a_codes, M, K / 2) || !make_codes_map(d, &tmB, b_codes, N, K / 2) ||
+      !make_f32_map(d, &tmD, D, M, N))
+    return FP4_ERR_CUDA;
+  GemmArgs a;
+  memset(&a, 0, sizeof(a));
+  a.sfa = a_scales; a.sfb = b_scales;
+  a.K = (int)K; a.tiles_m = (int)(M / 128); a.tiles_n = (int)(N / 128);
+  a.sg_a = a_tensor_scale; a.sg_b = b_tensor_scale;
+  a.status = device_status;
+  return launch_gemm(kPlain, tmA, tmB, tmD, tmD, a, d->sms, stream) == cudaSuccess ? FP4_OK : FP4_ERR_CUDA;
+}
+
+}  // extern "C"

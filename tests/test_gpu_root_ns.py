@@ -1,0 +1,200 @@
+"""fp4_root_ns / fp4_root_ns_batched against the oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2607_04422_b200 as fp4
+from paper_2607_04422_b200 import workloads
+from paper_2607_04422_b200.binding import FP4_FLAG_KEEP_OPERANDS, fp4_root_ns_workspace_layout
+from helpers import nibbles, sf_from_atoms
+
+pytestmark = pytest.mark.gpu
+
+# Tolerances.  BASELINE: relative Frobenius error of the NS output <= 2e-3 per iteration
+# count, orthogonality error within 1e-2 of the oracle's.  Stage outputs that have
+# bit-identical inputs on both sides differ only by FP32-vs-FP64 accumulation.
+TOL_OUT = 2e-3
+TOL_STAGE = 1e-5
+TOL_ORTH = 1e-2
+
+
+def rel(a, b):
+    a = a.astype(np.float64); b = b.astype(np.float64)
+    return np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-300)
+
+
+def orth_err(x):
+    x = x.astype(np.float64)
+    if x.shape[0] > x.shape[1]:
+        x = x.T
+    return np.linalg.norm(x @ x.T - np.eye(x.shape[0])) / np.sqrt(x.shape[0])
+
+
+def run_gpu(G_np, steps, abc=None, clip_quantile=0.99, flags=0, in_place=False):
+    m, n = G_np.shape
+    G = torch.from_numpy(G_np).cuda()
+    out = G if in_place else torch.full((m, n), float("nan"), device="cuda")
+    ws = torch.empty(fp4.fp4_root_ns_workspace_bytes(m, n, steps, flags), dtype=torch.uint8, device="cuda")
+    p = fp4.NsParams.make(abc=abc, clip_quantile=clip_quantile, flags=flags)
+    fp4.fp4_root_ns(G, out, steps, p, ws)
+    assert fp4.fp4_last_device_status(ws) == 0
+    return out.cpu().numpy(), ws
+
+
+def ws_view(ws, m, n, steps, flags):
+    """Decodes the intermediates the last iteration left in the workspace."""
+    lay = fp4_root_ns_workspace_layout(m, n, steps, flags)
+    s, l = min(m, n), max(m, n)
+    raw = ws.cpu().numpy()
+    sc = raw[lay.scalars:lay.scalars + 4096].view(np.float32)
+
+    def f32(off, r, c):
+        return raw[off:off + r * c * 4].view(np.float32).reshape(r, c)
+
+    def q(coff, soff, r, c):
+        codes = raw[coff:coff + r * c // 2].reshape(r, c // 2)
+        sf = sf_from_atoms(raw[soff:soff + r * c // 16], r, c // 16)
+        return codes, sf
+
+    return lay, sc, f32, q, s, l
+
+
+def code_mismatch(got, want):
+    """fraction of differing 4-bit codes and the largest index distance among them"""
+    g, w = nibbles(got), nibbles(want)
+    bad = g != w
+    if not bad.any():
+        return 0.0, 0
+    dist = np.abs((g[bad] & 7).astype(int) - (w[bad] & 7).astype(int))
+    return bad.mean(), int(dist.max())
+
+
+# --------------------------------------------------------------------------------------
+@pytest.mark.parametrize("gen,shape", [(workloads.lowrank_outliers, (256, 512)),
+                                       (workloads.gradient_like, (384, 128)),
+                                       (workloads.gaussian, (1024, 1024))])
+def test_clip_and_normalise_only(gen, shape):
+    G = gen(*shape, seed=2)
+    got, ws = run_gpu(G, steps=0)
+    want, tr = oracle.root_ns(G, steps=0, trace_iter=0)
+    lay, sc, *_ = ws_view(ws, *shape, 0, 0)
+    assert sc[lay.idx_tau] == np.float32(tr["tau"])       # tau is an element of the input
+    assert abs(sc[lay.idx_nu] - tr["nu"]) <= 1.2e-7 * tr["nu"]
+    if sc[lay.idx_nu] == np.float32(tr["nu"]):
+        assert np.array_equal(got, want)
+    assert rel(got, want) < 2e-7
+
+
+def test_no_clip_path():
+    G = workloads.gaussian(256, 384, seed=4)
+    got, _ = run_gpu(G, steps=0, clip_quantile=0.0)
+    want = oracle.root_ns(G, steps=0, clip_quantile=0.0)
+    assert rel(got, want) < 2e-7
+
+
+@pytest.mark.parametrize("shape", [(256, 512), (384, 384), (512, 256), (128, 1152)])
+def test_one_iteration_every_stage(shape):
+    """Iteration 0 has bit-identical inputs on both sides: every stage is checked."""
+    m, n = shape
+    G = workloads.gradient_like(m, n, seed=7)
+    flags = FP4_FLAG_KEEP_OPERANDS
+    got, ws = run_gpu(G, steps=1, flags=flags)
+    want, tr = oracle.root_ns(G, steps=1, trace_iter=0)
+    lay, sc, f32, q, s, l = ws_view(ws, m, n, 1, flags)
+    assert sc[lay.idx_nu] == np.float32(tr["nu"]), "norm differs in the last bit: pick another seed"
+    assert sc[lay.idx_sg_X0] == np.float32(tr["sg_X"])
+    assert sc[lay.idx_amax_X0] == np.float32(tr["amax_in"])
+    # A: upper-triangle 128-tiles are stored
+    A = f32(lay.A, s, s)
+    mask = np.kron(np.triu(np.ones((s // 128, s // 128))), np.ones((128, 128))).astype(bool)
+    assert np.abs(A[mask] - tr["A"][mask]).max() <= TOL_STAGE * np.abs(tr["A"]).max()
+    assert sc[lay.idx_sg_A0] == np.float32(tr["sg_A"])
+    assert abs(sc[lay.idx_amax_A0] - np.abs(tr["A"]).max()) <= 1e-6 * np.abs(tr["A"]).max()
+    # qA, qB: full matrices (both triangles), a few codes may sit on rounding boundaries
+    for name, co, so in (("qA", lay.qA_codes, lay.qA_scales), ("qB", lay.qB_codes, lay.qB_scales)):
+        codes, sf = q(co, so, s, s)
+        frac, dist = code_mismatch(codes, tr[name + "_codes"])
+        assert frac < 2e-3 and dist <= 1, (name, frac, dist)
+        assert (sf != tr[name + "_scales"]).mean() < 2e-3, name
+        # the quantised tensor is symmetric as a decoded matrix
+        dq = oracle.dequantize(codes, sf, 1.0)
+    assert sc[lay.idx_sg_B0] == np.float32(tr["sg_B"])
+    # X1 and its two operand copies
+    assert rel(got if m <= n else got.T, tr["X_out"]) < 2e-4
+    X1 = got if m <= n else np.ascontiguousarray(got.T)
+    sgX1 = sc[lay.idx_sg_X0 + 1]
+    oc, os_, _ = oracle.quantize(X1, s_g=float(sgX1))      # the GPU's own X1, quantised by the oracle
+    codes, sf = q(lay.qX_codes, lay.qX_scales, s, l)
+    assert np.array_equal(codes, oc) and np.array_equal(sf, os_)
+    oc, os_, _ = oracle.quantize(np.ascontiguousarray(X1.T), s_g=float(sgX1))
+    codes, sf = q(lay.qXt_codes[1], lay.qXt_scales[1], l, s)
+    assert np.array_equal(codes, oc) and np.array_equal(sf, os_)
+    assert abs(sc[lay.idx_amax_X0 + 1] - np.abs(X1).max()) == 0
+
+
+@pytest.mark.parametrize("shape,gen", [((256, 512), workloads.gaussian),
+                                       ((640, 384), workloads.row_lognormal),
+                                       ((512, 512), workloads.lowrank_outliers)])
+def test_iteration_counts_1_to_5(shape, gen):
+    G = gen(*shape, seed=0)
+    for steps in (1, 2, 3, 4, 5):
+        got, _ = run_gpu(G, steps=steps)
+        want = oracle.root_ns(G, steps=steps)
+        r = rel(got, want)
+        assert r <= TOL_OUT, (steps, r)
+        assert abs(orth_err(got) - orth_err(want)) <= TOL_ORTH
+
+
+def test_in_place_and_determinism():
+    G = workloads.gradient_like(384, 640, seed=5)
+    a, _ = run_gpu(G, steps=3)
+    b, _ = run_gpu(G, steps=3)
+    c, _ = run_gpu(G.copy(), steps=3, in_place=True)
+    assert np.array_equal(a, b) and np.array_equal(a, c)
+
+
+def test_tall_equals_transposed_wide():
+    G = workloads.gaussian(256, 640, seed=6)
+    wide, _ = run_gpu(G, steps=2)
+    tall, _ = run_gpu(np.ascontiguousarray(G.T), steps=2)
+    assert np.array_equal(tall, wide.T)
+
+
+def test_user_coefficients():
+    G = workloads.gaussian(256, 256, seed=8)
+    abc = (1.6, -0.9, 0.3)
+    got, _ = run_gpu(G, steps=2, abc=abc)
+    want = oracle.root_ns(G, steps=2, abc=abc)
+    assert rel(got, want) <= TOL_OUT
+
+
+def test_batched_matches_single_calls():
+    mats = workloads.stack_3b(blocks=1, scale_down=8)     # 7 matrices: 384^2, 384x1024, 1024x384
+    Gs = [torch.from_numpy(g).cuda() for g in mats]
+    outs = [torch.empty_like(g) for g in Gs]
+    shapes = [tuple(g.shape) for g in Gs]
+    ws = torch.empty(fp4.fp4_root_ns_batched_workspace_bytes(shapes, 5), dtype=torch.uint8, device="cuda")
+    fp4.fp4_root_ns_batched(Gs, outs, 5, None, ws)
+    assert fp4.fp4_last_device_status(ws) == 0
+    for g, o in zip(mats, outs):
+        single, _ = run_gpu(g, steps=5)
+        assert np.array_equal(o.cpu().numpy(), single)
+        assert rel(single, oracle.root_ns(g, steps=5)) <= TOL_OUT
+
+
+def test_argument_errors():
+    G = torch.zeros((128, 256), device="cuda")
+    ws = torch.empty(fp4.fp4_root_ns_workspace_bytes(128, 256, 5), dtype=torch.uint8, device="cuda")
+    with pytest.raises(fp4.Fp4Error) as e:
+        fp4.fp4_root_ns(torch.zeros((100, 256), device="cuda"), G, 5, None, ws)
+    assert e.value.code == 2
+    with pytest.raises(fp4.Fp4Error) as e:
+        fp4.fp4_root_ns(G, G, 5, None, ws[:4096])
+    assert e.value.code == 4
+    with pytest.raises(fp4.Fp4Error) as e:
+        fp4.fp4_root_ns(G, G, -1, None, ws)
+    assert e.value.code == 1
+    with pytest.raises(fp4.Fp4Error) as e:
+        fp4.fp4_root_ns(G, G, 5, None, ws[1:])
+    assert e.value.code == 3
