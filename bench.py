@@ -1,0 +1,310 @@
+#!/usr/bin/env python
+"""Benchmark of the NVFP4 Root Newton-Schulz step.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+A step is one pass of the whole hot path (clip, normalise, quantise, 5 Newton-Schulz
+iterations) over the decoder-stack batch: 4 blocks x {Wq, Wk, Wv, Wo 3072x3072,
+Wgate, Wup 3072x8192, Wdown 8192x3072} = 28 seeded synthetic matrices, through one
+fp4_root_ns_batched call.  Prints one JSON line (rank 0).
+
+With N > 1 (launched by torch.distributed.run) every rank runs the same batch on its own
+GPU: the matrices are independent, there is no data-path collective (weak scaling).
+
+--impl reference times the CPU oracle on the host cores on a bounded sample of the same
+workload (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+STEPS_NS = 5
+METRIC = "ns_orthogonalisations_per_s"
+UNIT = "matrices/s"
+FP4_NOMINAL_TFLOPS = 9000.0  # dense NVFP4, nominal
+FP4_OVER_BF16 = 4.0          # nominal ratio of the dense FP4 and BF16 tensor peaks
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+def batch_flops(shapes, steps=STEPS_NS):
+    """(algorithmic, dense-equivalent) FLOPs of the Newton-Schulz loops of a batch."""
+    alg = dense = 0.0
+    for m, n in shapes:
+        s, l = min(m, n), max(m, n)
+        alg += steps * (3.0 * s * s * l + 1.0 * s ** 3)
+        dense += steps * (4.0 * s * s * l + 2.0 * s ** 3)
+    return alg, dense
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in out.strip().splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------
+def run_reference(args):
+    """The oracle as it stands, on the host cores, on a bounded sample of the batch."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    from paper_2607_04422_b200 import workloads
+    shapes = [(m, n) for _, m, n, _ in workloads.stack_3b_shapes(4)]
+    alg_batch, _ = batch_flops(shapes)
+    name, m, n, seed = workloads.stack_3b_shapes(4)[0]
+    G = workloads.gradient_like(m, n, seed=seed)
+    sample_steps = 1
+    alg_sample, _ = batch_flops([(m, n)], steps=sample_steps)
+    cores = os.cpu_count() or 1
+    for _ in range(args.warmup):
+        oracle.root_ns(G, steps=sample_steps)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.root_ns(G, steps=sample_steps)
+    dt = (time.perf_counter() - t0) / max(args.steps, 1)
+    # scale the sample to the batch by its share of the algorithmic FLOPs
+    batch_s = dt * alg_batch / alg_sample
+    value = len(shapes) / batch_s
+    sample = (f"{name} {m}x{n}, {sample_steps} of {STEPS_NS} iterations per step, scaled to the 28-matrix batch "
+              f"by algorithmic FLOPs (x{alg_batch / alg_sample:.1f})")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": batch_s * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "nvfp4 operands, fp64 accumulate (CPU oracle)",
+            "data": "synthetic",
+            "config": {"workload": "cfg4: 3B-style decoder stack, 4 blocks x 7 projections = 28 matrices, "
+                                   "5 NVFP4 Newton-Schulz iterations", "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "tflops_algorithmic": alg_sample / dt / 1e12}
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------
+def cpu_baseline_leg(mats_np, shapes):
+    """Oracle on the host cores: one 3072 x 3072 matrix, all 5 iterations (about 10-30 s)."""
+    import oracle
+    alg_batch, _ = batch_flops(shapes)
+    G = mats_np[0]
+    alg_sample, _ = batch_flops([G.shape])
+    t0 = time.perf_counter()
+    oracle.root_ns(G, steps=STEPS_NS)
+    dt = time.perf_counter() - t0
+    batch_s = dt * alg_batch / alg_sample
+    return {"value": len(shapes) / batch_s, "unit": UNIT, "cores": os.cpu_count() or 1, "kind": "oracle",
+            "sample": f"block0.Wq {G.shape[0]}x{G.shape[1]}, 5 iterations, {dt:.1f} s; scaled to the 28-matrix "
+                      f"batch by algorithmic FLOPs (x{alg_batch / alg_sample:.1f})",
+            "gflops_algorithmic": alg_sample / dt / 1e9}
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2607_04422_b200 as fp4
+    from paper_2607_04422_b200 import workloads
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    fp4.load_library()
+
+    specs = workloads.stack_3b_shapes(4)
+    shapes = [(m, n) for _, m, n, _ in specs]
+    mats_np = [workloads.gradient_like(m, n, seed=seed + 7919 * rank) for _, m, n, seed in specs]
+    in_bytes = sum(g.nbytes for g in mats_np)
+    host_in = [torch.from_numpy(g).pin_memory() for g in mats_np]
+    host_out = [torch.empty_like(h).pin_memory() for h in host_in]
+    Gs = [h.cuda(non_blocking=True) for h in host_in]
+    outs = [torch.empty_like(g) for g in Gs]
+    ws = torch.empty(fp4.fp4_root_ns_batched_workspace_bytes(shapes, STEPS_NS), dtype=torch.uint8, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def step():
+        fp4.fp4_root_ns_batched(Gs, outs, STEPS_NS, None, ws, stream)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing ------------------------------------------------------------
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    launches0 = fp4.fp4_kernel_launches()
+    sampler = ClockSampler(local) if rank == 0 else None
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    barrier()
+    ms = e0.elapsed_time(e1)
+    launches = fp4.fp4_kernel_launches() - launches0
+    clocks = sampler.stop() if sampler else None
+    status = fp4.fp4_last_device_status(ws)
+    if status != 0:
+        raise SystemExit(f"device status {status}: {fp4.fp4_status_string(status)}")
+    t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms = float(t.item())
+    ms_per_step = ms / args.steps
+    value = world * len(shapes) * args.steps / (ms / 1e3)
+
+    # ---- per-kernel times: one more pass with event brackets around every launch group ------
+    fp4.fp4_profile_enable(True)
+    prof_steps = min(args.steps, 3)
+    for _ in range(prof_steps):
+        step()
+    torch.cuda.synchronize()
+    prof = fp4.fp4_profile_collect()
+    fp4.fp4_profile_enable(False)
+
+    # ---- end to end: host buffers in, host buffers out, copies inside the timed region --------
+    def e2e_step():
+        for h, g in zip(host_in, Gs):
+            g.copy_(h, non_blocking=True)
+        step()
+        for o, h in zip(outs, host_out):
+            h.copy_(o, non_blocking=True)
+
+    e2e_step()
+    barrier()
+    n_e2e = max(2, min(args.steps, 5))
+    e0.record(stream)
+    for _ in range(n_e2e):
+        e2e_step()
+    e1.record(stream)
+    barrier()
+    t = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    e2e_value = world * len(shapes) * n_e2e / (float(t.item()) / 1e3)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel -----------------------------------------------------
+    pk = peaks()
+    alg, dense = batch_flops(shapes)
+    total_prof = sum(v[0] for v in prof.values())
+    shares = {k: (v[0] / total_prof if total_prof else 0.0) for k, v in prof.items()}
+    dom = max(("G1", "G2", "G3"), key=lambda k: prof[k][0])
+    per_launch_ms = prof[dom][0] / max(prof[dom][1], 1)
+    # algorithmic FLOPs of one launch of each GEMM, averaged over the batch's launches
+    flops = {"G1": 0.0, "G2": 0.0, "G3": 0.0}
+    for m, n in shapes:
+        s, l = min(m, n), max(m, n)
+        flops["G1"] += 1.0 * s * s * l      # symmetric: half of 2 s^2 l
+        flops["G2"] += 1.0 * s ** 3
+        flops["G3"] += 2.0 * s * s * l
+    avg_flops = flops[dom] / len(shapes)
+    achieved = avg_flops / (per_launch_ms / 1e3) / 1e12
+    fp4_peak = pk["bf16_tflops_sustained"] * FP4_OVER_BF16
+    roofline = {"kernel": f"k_gemm<{dom}>", "bound": "tensor", "achieved": achieved, "peak": fp4_peak,
+                "unit": "TFLOP/s", "frac": achieved / fp4_peak, "traffic": None,
+                "peak_source": f"{pk['source']} sustained bf16 x {FP4_OVER_BF16:.0f} (nominal FP4/BF16 ratio)",
+                "avg_launch_ms": per_launch_ms, "launches_profiled": prof[dom][1],
+                "time_share": shares}
+
+    cpu = cpu_baseline_leg(mats_np, shapes)
+    step_s = ms_per_step / 1e3
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "nvfp4 operands, fp32 accumulate", "data": "synthetic",
+            "config": {"workload": "cfg4: 3B-style decoder stack, 4 blocks x 7 projections = 28 matrices "
+                                   "(16x 3072x3072, 8x 3072x8192, 4x 8192x3072), 5 NVFP4 Newton-Schulz iterations, "
+                                   "one fp4_root_ns_batched call per step",
+                       "l2": f"inputs {in_bytes / 1e9:.2f} GB per step, larger than L2; no flush needed",
+                       "parallelism": f"replicas x{world}, no collective"},
+            "tflops_algorithmic": alg / step_s / 1e12, "tflops_dense_equivalent": dense / step_s / 1e12,
+            "pct_of_nominal_fp4_peak": 100.0 * alg / step_s / 1e12 / FP4_NOMINAL_TFLOPS,
+            "pct_of_measured_fp4_peak": 100.0 * alg / step_s / 1e12 / fp4_peak,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": in_bytes, "d2h_bytes_per_step": in_bytes},
+            "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "cpu_baseline": cpu}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -164,6 +164,20 @@ fp4_status fp4_gemm_nt(const uint8_t* a_codes, const uint8_t* a_scales, float a_
                        FP4_ERR_DEVICE_TIMEOUT if a bounded wait gives up */,
                        cudaStream_t stream);
 
+/* ---- measurement support (the paper has no counterpart) -----------------------------------
+ * While profiling is enabled, every group of launches of the step is bracketed by a pair of
+ * CUDA events on the caller's stream; fp4_profile_collect waits for them, adds the elapsed
+ * times per class into ms[class] and the number of bracketed groups into groups[class]
+ * (both host arrays of FP4_PROF_CLASSES entries), then forgets them.  Off by default; the
+ * events add stream operations, so time whole calls with profiling off.
+ * fp4_kernel_launches returns how many kernels this library has launched in this process.
+ */
+enum { FP4_PROF_CLIP = 0, FP4_PROF_STATS = 1, FP4_PROF_PREP = 2, FP4_PROF_G1 = 3, FP4_PROF_G2 = 4,
+       FP4_PROF_G3 = 5, FP4_PROF_TRANSPOSE = 6, FP4_PROF_QUANTIZE = 7, FP4_PROF_CLASSES = 8 };
+void fp4_profile_enable(int on);
+fp4_status fp4_profile_collect(float* ms, int* groups);
+uint64_t fp4_kernel_launches(void);
+
 #ifdef __cplusplus
 }
 #endif

@@ -22,7 +22,9 @@ STATUS_NAMES = {0: "FP4_OK", 1: "FP4_ERR_INVALID_ARG", 2: "FP4_ERR_SHAPE", 3: "F
 
 EXPORTS = ("fp4_status_string", "fp4_scale_bytes", "fp4_quantize", "fp4_root_coeffs",
            "fp4_root_ns_workspace_bytes", "fp4_root_ns", "fp4_root_ns_batched_workspace_bytes",
-           "fp4_root_ns_batched", "fp4_last_device_status", "fp4_root_ns_workspace_layout", "fp4_gemm_nt")
+           "fp4_root_ns_batched", "fp4_last_device_status", "fp4_root_ns_workspace_layout", "fp4_gemm_nt",
+           "fp4_profile_enable", "fp4_profile_collect", "fp4_kernel_launches")
+PROF_CLASSES = ("clip", "stats", "prep", "G1", "G2", "G3", "transpose", "quantize")
 
 
 class Fp4Error(RuntimeError):
@@ -92,6 +94,10 @@ def load_library():
     L.fp4_root_ns_workspace_layout.restype = C.c_int
     L.fp4_gemm_nt.argtypes = [vp, vp, C.c_float, vp, vp, C.c_float, i64, i64, i64, vp, vp, vp]
     L.fp4_gemm_nt.restype = C.c_int
+    L.fp4_profile_enable.argtypes = [C.c_int]; L.fp4_profile_enable.restype = None
+    L.fp4_profile_collect.argtypes = [C.POINTER(C.c_float), C.POINTER(C.c_int)]
+    L.fp4_profile_collect.restype = C.c_int
+    L.fp4_kernel_launches.argtypes = []; L.fp4_kernel_launches.restype = C.c_uint64
     _lib = L
     return L
 
@@ -177,3 +183,20 @@ def fp4_gemm_nt(a_codes, a_scales, a_sg: float, b_codes, b_scales, b_sg: float, 
                                       b_scales.data_ptr(), float(b_sg), M, N, K, D.data_ptr(),
                                       status.data_ptr() if status is not None else None, _stream(stream)),
            "fp4_gemm_nt")
+
+
+def fp4_profile_enable(on: bool) -> None:
+    load_library().fp4_profile_enable(1 if on else 0)
+
+
+def fp4_profile_collect():
+    """{class name: (milliseconds, bracketed launch groups)} since the last collect."""
+    n = len(PROF_CLASSES)
+    ms = (C.c_float * n)()
+    groups = (C.c_int * n)()
+    _check(load_library().fp4_profile_collect(ms, groups), "fp4_profile_collect")
+    return {PROF_CLASSES[i]: (float(ms[i]), int(groups[i])) for i in range(n)}
+
+
+def fp4_kernel_launches() -> int:
+    return int(load_library().fp4_kernel_launches())

@@ -376,6 +376,7 @@ cudaError_t launch_mode(const CUtensorMap& tmA, const CUtensorMap& tmB, const CU
   const int num_tiles = args.symmetric ? args.tiles_n * (args.tiles_n + 1) / 2 : args.tiles_m * args.tiles_n;
   int grid = 2 * sms;
   if (grid > num_tiles) grid = num_tiles;
+  count_launches(1);
   k_gemm<MODE><<<grid, NTHREADS, SMEM_BYTES, st>>>(tmA, tmB, tmAux, tmOut, args);
   return cudaGetLastError();
 }

@@ -69,6 +69,15 @@ struct GemmArgs {
   uint32_t* status;
 };
 
+// Measurement support: counts kernel launches and, when profiling is on, brackets a group of
+// launches with events.
+void count_launches(int n);
+struct ProfScope {
+  int cls; cudaStream_t st; cudaEvent_t e0; bool on;
+  ProfScope(int cls, cudaStream_t st);
+  ~ProfScope();
+};
+
 cudaError_t launch_quantize(const float* x, int64_t rows, int64_t cols, uint8_t* codes, uint8_t* scales,
                             float* tensor_scale, int sms, cudaStream_t st);
 cudaError_t launch_prologue(const float* G, int64_t m, int64_t n, const NsPlan& pl, uint8_t* ws, float* X,

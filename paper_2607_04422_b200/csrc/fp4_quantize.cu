@@ -317,6 +317,7 @@ cudaError_t launch_quantize(const float* x, int64_t rows, int64_t cols, uint8_t*
   k_quantize_rows<<<grid_for(n4, 256 * 2, sms), 256, 0, st>>>(reinterpret_cast<const float4*>(x), rows, cols, codes,
                                                             scales, reinterpret_cast<const uint32_t*>(tensor_scale));
   k_finish_tensor_scale<<<1, 1, 0, st>>>(tensor_scale);
+  count_launches(3);
   return cudaGetLastError();
 }
 
@@ -333,6 +334,8 @@ cudaError_t launch_prologue(const float* G, int64_t m, int64_t n, const NsPlan& 
   cudaError_t e = cudaMemsetAsync(ws + pl.lay.header + skip, 0, pl.zero_bytes - skip, st);
   if (e != cudaSuccess) return e;
   if (pl.clip) {
+    ProfScope ps(FP4_PROF_CLIP, st);
+    count_launches(7);
     k_select_init<<<1, 1, 0, st>>>(hdr, (uint32_t)pl.clip_rank);
     const int gh = grid_for(n4, 512 * 4, pl.sms);
     k_radix_hist<20, 11><<<gh, 512, 0, st>>>(g4, n4, hdr, hist);
@@ -342,10 +345,16 @@ cudaError_t launch_prologue(const float* G, int64_t m, int64_t n, const NsPlan& 
     k_radix_hist<0, 9><<<gh, 512, 0, st>>>(g4, n4, hdr, hist);
     k_radix_pick<0, 9><<<1, 256, 0, st>>>(hdr, hist, scalars, pl.ix.tau);
   }
-  k_clamp_stats<<<pl.stat_blocks, 256, 0, st>>>(g4, n4, scalars, pl.ix.tau, pl.clip, partial, &hdr->maxabs_bits);
-  k_norm_finish<<<1, 256, 0, st>>>(partial, pl.stat_blocks, hdr, scalars, pl.ix, pl.eps);
+  {
+    ProfScope ps(FP4_PROF_STATS, st);
+    count_launches(2);
+    k_clamp_stats<<<pl.stat_blocks, 256, 0, st>>>(g4, n4, scalars, pl.ix.tau, pl.clip, partial, &hdr->maxabs_bits);
+    k_norm_finish<<<1, 256, 0, st>>>(partial, pl.stat_blocks, hdr, scalars, pl.ix, pl.eps);
+  }
   const int tall = m > n;
   dim3 grid((unsigned)(pl.l / 128), (unsigned)(pl.s / 128));
+  ProfScope ps(FP4_PROF_PREP, st);
+  count_launches(1);
   k_prep_operands<<<grid, 256, 128 * 129 * 4, st>>>(G, n, tall, scalars, pl.ix, pl.clip, X, pl.s, pl.l,
                                                     ws + pl.lay.qX_codes, ws + pl.lay.qX_scales,
                                                     ws + pl.lay.qXt_codes[0], ws + pl.lay.qXt_scales[0], write_q);
@@ -354,6 +363,7 @@ cudaError_t launch_prologue(const float* G, int64_t m, int64_t n, const NsPlan& 
 
 cudaError_t launch_transpose_out(const float* X, int64_t s, int64_t l, float* out, cudaStream_t st) {
   dim3 grid((unsigned)(l / 32), (unsigned)(s / 32));
+  count_launches(1);
   k_transpose_out<<<grid, 256, 0, st>>>(X, s, l, out);
   return cudaGetLastError();
 }

@@ -1,12 +1,40 @@
 // Host side of the library: argument checks, workspace layout, TMA descriptors, and the
 // sequence of launches of the Root Newton-Schulz step (Section 3.4).  Everything here
 // only enqueues work on the caller's stream.
+#include <atomic>
 #include <cmath>
 #include <mutex>
+#include <vector>
 
 #include "fp4_kernels.h"
 
 namespace fp4 {
+
+namespace {
+std::atomic<uint64_t> g_launches{0};
+std::atomic<int> g_prof_on{0};
+struct ProfRec { int cls; cudaEvent_t e0, e1; };
+std::vector<ProfRec> g_prof;
+std::mutex g_prof_mu;
+}  // namespace
+
+void count_launches(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+ProfScope::ProfScope(int cls_, cudaStream_t st_) : cls(cls_), st(st_), e0(nullptr), on(g_prof_on.load() != 0) {
+  if (on) {
+    if (cudaEventCreate(&e0) != cudaSuccess) { on = false; return; }
+    cudaEventRecord(e0, st);
+  }
+}
+ProfScope::~ProfScope() {
+  if (!on) return;
+  cudaEvent_t e1;
+  if (cudaEventCreate(&e1) != cudaSuccess) { cudaEventDestroy(e0); return; }
+  cudaEventRecord(e1, st);
+  std::lock_guard<std::mutex> lock(g_prof_mu);
+  g_prof.push_back({cls, e0, e1});
+}
+
 namespace {
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -194,14 +222,20 @@ fp4_status run_one(const DeviceInfo* d, const float* G, float* out, int64_t m, i
       a1.sfa = a1.sfb = ws + L.qX_scales;
       a1.rq_codes = a1.cq_codes = ws + L.qA_codes; a1.rq_sf = a1.cq_sf = ws + L.qA_scales;
       a1.rq_K = a1.cq_K = (int)s; a1.write_q = 1;
-      if (launch_gemm(kG1, tm_qX, tm_qX, tm_A, tm_A, a1, d->sms, st) != cudaSuccess) return FP4_ERR_CUDA;
+      {
+        ProfScope ps(FP4_PROF_G1, st);
+        if (launch_gemm(kG1, tm_qX, tm_qX, tm_A, tm_A, a1, d->sms, st) != cudaSuccess) return FP4_ERR_CUDA;
+      }
       // G2: B = bA + c qA qA^T, qB in both triangles
       GemmArgs a2 = base;
       a2.iter = k; a2.K = (int)s; a2.tiles_m = a2.tiles_n = (int)(s / 128); a2.symmetric = 1;
       a2.sfa = a2.sfb = ws + L.qA_scales;
       a2.rq_codes = a2.cq_codes = ws + L.qB_codes; a2.rq_sf = a2.cq_sf = ws + L.qB_scales;
       a2.rq_K = a2.cq_K = (int)s; a2.write_q = 1;
-      if (launch_gemm(kG2, tm_qA, tm_qA, tm_A, tm_A, a2, d->sms, st) != cudaSuccess) return FP4_ERR_CUDA;
+      {
+        ProfScope ps(FP4_PROF_G2, st);
+        if (launch_gemm(kG2, tm_qA, tm_qA, tm_A, tm_A, a2, d->sms, st) != cudaSuccess) return FP4_ERR_CUDA;
+      }
       // G3: X+ = aX + qB qXt^T, in place on X; new operand copies unless this is the last iteration
       GemmArgs a3 = base;
       a3.iter = k; a3.K = (int)s; a3.tiles_m = (int)(s / 128); a3.tiles_n = (int)(l / 128); a3.symmetric = 0;
@@ -209,10 +243,14 @@ fp4_status run_one(const DeviceInfo* d, const float* G, float* out, int64_t m, i
       a3.rq_codes = ws + L.qX_codes; a3.rq_sf = ws + L.qX_scales; a3.rq_K = (int)l;
       a3.cq_codes = ws + L.qXt_codes[nxt]; a3.cq_sf = ws + L.qXt_scales[nxt]; a3.cq_K = (int)s;
       a3.write_q = (!last || keep) ? 1 : 0;
-      if (launch_gemm(kG3, tm_qB, tm_qXt[cur], tm_X, tm_X, a3, d->sms, st) != cudaSuccess) return FP4_ERR_CUDA;
+      {
+        ProfScope ps(FP4_PROF_G3, st);
+        if (launch_gemm(kG3, tm_qB, tm_qXt[cur], tm_X, tm_X, a3, d->sms, st) != cudaSuccess) return FP4_ERR_CUDA;
+      }
     }
   }
   if (pl.tall) {
+    ProfScope ps(FP4_PROF_TRANSPOSE, st);
     if (launch_transpose_out(X, s, l, out, st) != cudaSuccess) return FP4_ERR_CUDA;
   }
   return FP4_OK;
@@ -260,6 +298,7 @@ fp4_status fp4_quantize(const float* x, int64_t rows, int64_t cols, uint8_t* cod
   const DeviceInfo* d;
   fp4_status rc = check_common(&d);
   if (rc != FP4_OK) return rc;
+  ProfScope ps(FP4_PROF_QUANTIZE, stream);
   return launch_quantize(x, rows, cols, codes, scales, tensor_scale, d->sms, stream) == cudaSuccess ? FP4_OK
                                                                                                       : FP4_ERR_CUDA;
 }
@@ -375,5 +414,26 @@ fp4_status fp4_gemm_nt(const uint8_t* a_codes, const uint8_t* a_scales, float a_
   a.status = device_status;
   return launch_gemm(kPlain, tmA, tmB, tmD, tmD, a, d->sms, stream) == cudaSuccess ? FP4_OK : FP4_ERR_CUDA;
 }
+
+void fp4_profile_enable(int on) { g_prof_on.store(on ? 1 : 0); }
+
+fp4_status fp4_profile_collect(float* ms, int* groups) {
+  if (!ms || !groups) return FP4_ERR_INVALID_ARG;
+  for (int i = 0; i < FP4_PROF_CLASSES; ++i) { ms[i] = 0.0f; groups[i] = 0; }
+  std::lock_guard<std::mutex> lock(g_prof_mu);
+  fp4_status rc = FP4_OK;
+  for (const ProfRec& r : g_prof) {
+    float t = 0.0f;
+    if (cudaEventSynchronize(r.e1) != cudaSuccess || cudaEventElapsedTime(&t, r.e0, r.e1) != cudaSuccess)
+      rc = FP4_ERR_CUDA;
+    if (r.cls >= 0 && r.cls < FP4_PROF_CLASSES) { ms[r.cls] += t; groups[r.cls] += 1; }
+    cudaEventDestroy(r.e0);
+    cudaEventDestroy(r.e1);
+  }
+  g_prof.clear();
+  return rc;
+}
+
+uint64_t fp4_kernel_launches(void) { return g_launches.load(); }
 
 }  // extern "C"
