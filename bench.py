@@ -56,6 +56,26 @@ def batch_flops(shapes, steps=STEPS_NS):
     return alg, dense
 
 
+def rank_seed(seed: int, rank: int) -> int:
+    """Every rank draws its own batch."""
+    return int(seed) + 7919 * int(rank)
+
+
+def max_over_ranks(ms: float, device, world: int) -> float:
+    """Step time of the job = the slowest rank's device time."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_value(world: int, matrices: int, steps: int, ms: float) -> float:
+    """Whole-job matrices per second: every rank processed matrices * steps."""
+    return world * matrices * steps / (ms / 1e3)
+
+
 class ClockSampler:
     """nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
@@ -172,7 +192,7 @@ def run_ours(args):
 
     specs = workloads.stack_3b_shapes(4)
     shapes = [(m, n) for _, m, n, _ in specs]
-    mats_np = [workloads.gradient_like(m, n, seed=seed + 7919 * rank) for _, m, n, seed in specs]
+    mats_np = [workloads.gradient_like(m, n, seed=rank_seed(seed, rank)) for _, m, n, seed in specs]
     in_bytes = sum(g.nbytes for g in mats_np)
     host_in = [torch.from_numpy(g).pin_memory() for g in mats_np]
     host_out = [torch.empty_like(h).pin_memory() for h in host_in]
@@ -208,12 +228,9 @@ def run_ours(args):
     status = fp4.fp4_last_device_status(ws)
     if status != 0:
         raise SystemExit(f"device status {status}: {fp4.fp4_status_string(status)}")
-    t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms = float(t.item())
+    ms = max_over_ranks(ms, torch.device("cuda"), world)
     ms_per_step = ms / args.steps
-    value = world * len(shapes) * args.steps / (ms / 1e3)
+    value = aggregate_value(world, len(shapes), args.steps, ms)
 
     # ---- per-kernel times: one more pass with event brackets around every launch group ------
     fp4.fp4_profile_enable(True)
@@ -240,10 +257,7 @@ def run_ours(args):
         e2e_step()
     e1.record(stream)
     barrier()
-    t = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    e2e_value = world * len(shapes) * n_e2e / (float(t.item()) / 1e3)
+    e2e_value = aggregate_value(world, len(shapes), n_e2e, max_over_ranks(e0.elapsed_time(e1), torch.device("cuda"), world))
 
     if rank != 0:
         if world > 1:

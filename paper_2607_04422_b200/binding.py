@@ -12,7 +12,7 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_LIB_PATH = os.path.join(_HERE, "libfp4root.so")
+_LIB_PATH = os.environ.get("FP4ROOT_LIB") or os.path.join(_HERE, "libfp4root.so")
 _lib = None
 
 FP4_FLAG_KEEP_OPERANDS = 1

@@ -23,7 +23,10 @@ namespace fp4 {
 namespace {
 
 constexpr int BM = 128, BN = 128, BK = 128;
-constexpr int STAGES = 4;
+#ifndef FP4_STAGES
+#define FP4_STAGES 4
+#endif
+constexpr int STAGES = FP4_STAGES;
 constexpr int OPER_BYTES = BM * BK / 2;      // 8192: one operand tile of a stage (64-byte rows)
 constexpr int SF_BYTES = 2 * 512;            // two scale atoms (128 rows x 8 blocks) per operand and stage
 constexpr uint32_t STAGE_TX = 2 * OPER_BYTES + 2 * SF_BYTES;
