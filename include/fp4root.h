@@ -15,7 +15,7 @@
  *   - All work is enqueued on `stream`; no call synchronises the host except
  *     fp4_last_device_status.
  *   - Shapes: every matrix dimension must be a positive multiple of 128, else
- *     FP4_ERR_SHAPE.  Device pointers must be 16-byte aligned (the workspace 1024),
+ *     FP4_ERR_SHAPE.  Device pointers must be 16-byte aligned (the workspace 256),
  *     else FP4_ERR_ALIGNMENT.
  *   - Errors are return codes.  A kernel that gives up on a bounded wait records
  *     FP4_ERR_DEVICE_TIMEOUT in the workspace header and ends normally; it never
@@ -100,7 +100,7 @@ fp4_status fp4_root_coeffs(int64_t m, int64_t n, int steps, float abc[3]);
  * G: device, m x n FP32 row-major.  out: device, m x n FP32 row-major; may equal G exactly
  *   (no partial overlap).  steps >= 0 iterations (0: clip and normalise only).
  * ws: device workspace of at least fp4_root_ns_workspace_bytes(m, n, steps, flags) bytes,
- *   1024-byte aligned; its contents need not be initialised and are overwritten.
+ *   256-byte aligned; its contents need not be initialised and are overwritten.
  * Computes, with s = min(m,n), l = max(m,n) and X = G or G^T so that X is s x l:
  *   tau = quantile of |G|, G_c = clamp(G, -tau, tau), X0 = G_c/(||G_c||_F + eps), then
  *   per iteration A = qX qX^T, B = bA + c qA qA^T, X+ = aX + qB qX^{16x1}, every q*
@@ -115,7 +115,7 @@ fp4_status fp4_root_ns(const float* G, float* out, int64_t m, int64_t n, int ste
 /* ---- many matrices of different shapes in one call (the matrices of a layer stack) ------
  * count matrices; G, out, m, n: host arrays of length count (G[i], out[i] device pointers).
  * One parameter block applies to all (coefficients per matrix when p->a is NaN).
- * ws: device, at least fp4_root_ns_batched_workspace_bytes(...) bytes, 1024-byte aligned.
+ * ws: device, at least fp4_root_ns_batched_workspace_bytes(...) bytes, 256-byte aligned.
  */
 size_t fp4_root_ns_batched_workspace_bytes(int count, const int64_t* m, const int64_t* n,
                                            int steps, uint32_t flags);

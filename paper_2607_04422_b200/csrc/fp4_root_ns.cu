@@ -334,7 +334,7 @@ fp4_status fp4_root_ns(const float* G, float* out, int64_t m, int64_t n, int ste
   if (!G || !out || !ws) return FP4_ERR_INVALID_ARG;
   if (!shape_ok(m) || !shape_ok(n)) return FP4_ERR_SHAPE;
   if (steps < 0 || steps > kMaxSteps) return FP4_ERR_INVALID_ARG;
-  if (!aligned(G, 16) || !aligned(out, 16) || !aligned(ws, 1024)) return FP4_ERR_ALIGNMENT;
+  if (!aligned(G, 16) || !aligned(out, 16) || !aligned(ws, 256)) return FP4_ERR_ALIGNMENT;
   const size_t need = fp4_root_ns_workspace_bytes(m, n, steps, p->flags);
   if (need == 0 || ws_bytes < need) return FP4_ERR_WORKSPACE;
   const DeviceInfo* d;
@@ -362,7 +362,7 @@ fp4_status fp4_root_ns_batched(int count, const float* const* G, float* const* o
   if (!p) { default_params(&dp); p = &dp; }
   if (count < 0 || (count > 0 && (!G || !out || !m || !n)) || !ws) return FP4_ERR_INVALID_ARG;
   if (steps < 0 || steps > kMaxSteps) return FP4_ERR_INVALID_ARG;
-  if (!aligned(ws, 1024)) return FP4_ERR_ALIGNMENT;
+  if (!aligned(ws, 256)) return FP4_ERR_ALIGNMENT;
   for (int i = 0; i < count; ++i) {
     if (!G[i] || !out[i]) return FP4_ERR_INVALID_ARG;
     if (!shape_ok(m[i]) || !shape_ok(n[i])) return FP4_ERR_SHAPE;

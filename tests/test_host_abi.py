@@ -67,6 +67,7 @@ def test_argument_validation_happens_before_any_device_work():
     assert lib.fp4_root_ns(p, p, 100, 128, 5, None, p, 1 << 30, None) == 2        # shape
     assert lib.fp4_root_ns(p, p, 128, 128, 65, None, p, 1 << 30, None) == 1       # steps
     assert lib.fp4_root_ns(p + 4, p, 128, 128, 5, None, p, 1 << 30, None) == 3    # alignment
+    assert lib.fp4_root_ns(p, p, 128, 128, 5, None, p + 128, 1 << 30, None) == 3  # workspace alignment
     assert lib.fp4_root_ns(p, p, 128, 128, 5, None, p, 16, None) == 4             # workspace
     assert lib.fp4_quantize(p, 128, 120, p, p, p, 0, None) == 2
     assert lib.fp4_gemm_nt(p, p, 1.0, p, p, 1.0, 128, 128, 64, p, None, None) == 2
