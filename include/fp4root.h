@@ -45,7 +45,8 @@ typedef enum {
   FP4_ERR_ARCH = 5,
   FP4_ERR_CUDA = 6,
   FP4_ERR_DEVICE_TIMEOUT = 7,
-  FP4_ERR_UNIMPLEMENTED = 8
+  FP4_ERR_UNIMPLEMENTED = 8,
+  FP4_ERR_STATIC_LIMIT = 9
 } fp4_status;
 
 /* flags of fp4_ns_params */
@@ -123,6 +124,37 @@ fp4_status fp4_root_ns_batched(int count, const float* const* G, float* const* o
                                const int64_t* m, const int64_t* n, int steps,
                                const fp4_ns_params* p, void* ws, size_t ws_bytes,
                                cudaStream_t stream);
+
+/* ---- the same step for callers that cannot allocate device memory --------------------------
+ * (The paper has no counterpart; this is a packaging variant of fp4_root_ns.)
+ *
+ * Some callers have nowhere to get a workspace from: code that runs inside another
+ * framework's callback or a real-time loop where cudaMalloc is forbidden because it may
+ * synchronise the device, plug-ins that are handed input and output buffers and nothing
+ * else, and programs whose memory pool is already fully committed.  For them this entry
+ * point keeps the workspace inside the library: a fixed array of
+ * FP4_STATIC_SCRATCH_BYTES (16 MiB) in the device's global memory, part of the loaded
+ * module, held by every GPU that uses the library until the process exits.
+ *
+ * Arguments as for fp4_root_ns, without ws.  Works for every (m, n, steps, flags) with
+ * fp4_root_ns_workspace_bytes(m, n, steps, flags) <= FP4_STATIC_SCRATCH_BYTES -- for example
+ * 1024 x 1024 and 1024 x 2048; a tall 2048 x 1024 needs more -- and returns
+ * FP4_ERR_STATIC_LIMIT for anything larger, before any work is enqueued.
+ * device_status: device, optional (may be NULL): one uint32 that receives, in stream order,
+ *   the status word of this call (FP4_OK or FP4_ERR_DEVICE_TIMEOUT).
+ *
+ * It calls no cudaMalloc, cudaFree or other allocating routine.  The first call on each
+ * device looks up the array's device address (a one-time, per-device set-up done with that
+ * device current); make that first call outside any stream capture.  All calls on a device
+ * share the one array, which keeps whatever the previous call left in it; the call itself
+ * clears the parts that must start from zero.  Two calls whose kernels could overlap on the
+ * GPU (different streams without an ordering between them) race on the array: order them.
+ * Results are identical to fp4_root_ns on the same input.
+ */
+#define FP4_STATIC_SCRATCH_BYTES ((size_t)16 << 20)
+fp4_status fp4_root_ns_static(const float* G, float* out, int64_t m, int64_t n, int steps,
+                              const fp4_ns_params* p, uint32_t* device_status,
+                              cudaStream_t stream);
 
 /* Synchronises `stream`, then returns the status word that the kernels of the last call
  * on workspace `ws` left in its header: FP4_OK or FP4_ERR_DEVICE_TIMEOUT. */

@@ -18,12 +18,13 @@ _lib = None
 FP4_FLAG_KEEP_OPERANDS = 1
 STATUS_NAMES = {0: "FP4_OK", 1: "FP4_ERR_INVALID_ARG", 2: "FP4_ERR_SHAPE", 3: "FP4_ERR_ALIGNMENT",
                 4: "FP4_ERR_WORKSPACE", 5: "FP4_ERR_ARCH", 6: "FP4_ERR_CUDA", 7: "FP4_ERR_DEVICE_TIMEOUT",
-                8: "FP4_ERR_UNIMPLEMENTED"}
+                8: "FP4_ERR_UNIMPLEMENTED", 9: "FP4_ERR_STATIC_LIMIT"}
+FP4_STATIC_SCRATCH_BYTES = 16 << 20
 
 EXPORTS = ("fp4_status_string", "fp4_scale_bytes", "fp4_quantize", "fp4_root_coeffs",
            "fp4_root_ns_workspace_bytes", "fp4_root_ns", "fp4_root_ns_batched_workspace_bytes",
            "fp4_root_ns_batched", "fp4_last_device_status", "fp4_root_ns_workspace_layout", "fp4_gemm_nt",
-           "fp4_profile_enable", "fp4_profile_collect", "fp4_kernel_launches")
+           "fp4_profile_enable", "fp4_profile_collect", "fp4_kernel_launches", "fp4_root_ns_static")
 PROF_CLASSES = ("clip", "stats", "prep", "G1", "G2", "G3", "transpose", "quantize")
 
 
@@ -94,6 +95,8 @@ def load_library():
     L.fp4_root_ns_workspace_layout.restype = C.c_int
     L.fp4_gemm_nt.argtypes = [vp, vp, C.c_float, vp, vp, C.c_float, i64, i64, i64, vp, vp, vp]
     L.fp4_gemm_nt.restype = C.c_int
+    L.fp4_root_ns_static.argtypes = [vp, vp, i64, i64, C.c_int, C.POINTER(NsParams), vp, vp]
+    L.fp4_root_ns_static.restype = C.c_int
     L.fp4_profile_enable.argtypes = [C.c_int]; L.fp4_profile_enable.restype = None
     L.fp4_profile_collect.argtypes = [C.POINTER(C.c_float), C.POINTER(C.c_int)]
     L.fp4_profile_collect.restype = C.c_int
@@ -150,6 +153,18 @@ def fp4_root_ns(G: torch.Tensor, out: torch.Tensor, steps: int, params: NsParams
     p = C.byref(params) if params is not None else None
     _check(load_library().fp4_root_ns(G.data_ptr(), out.data_ptr(), m, n, steps, p, ws.data_ptr(),
                                       ws.numel() * ws.element_size(), _stream(stream)), "fp4_root_ns")
+
+
+def fp4_root_ns_static(G: torch.Tensor, out: torch.Tensor, steps: int, params: NsParams | None = None,
+                       device_status: torch.Tensor | None = None, stream=None) -> None:
+    """fp4_root_ns for callers that cannot allocate a workspace: the library's own 16 MiB
+    static device array is the scratch.  Shapes that need more raise FP4_ERR_STATIC_LIMIT.
+    Calls that could overlap on the GPU must be ordered by the caller."""
+    m, n = G.shape
+    p = C.byref(params) if params is not None else None
+    _check(load_library().fp4_root_ns_static(G.data_ptr(), out.data_ptr(), m, n, steps, p,
+                                             device_status.data_ptr() if device_status is not None else None,
+                                             _stream(stream)), "fp4_root_ns_static")
 
 
 def fp4_root_ns_batched_workspace_bytes(shapes, steps: int = 5, flags: int = 0) -> int:

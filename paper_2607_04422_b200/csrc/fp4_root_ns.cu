@@ -280,6 +280,7 @@ const char* fp4_status_string(fp4_status s) {
     case FP4_ERR_CUDA: return "CUDA runtime or driver call failed";
     case FP4_ERR_DEVICE_TIMEOUT: return "a kernel gave up on a bounded wait";
     case FP4_ERR_UNIMPLEMENTED: return "not implemented";
+    case FP4_ERR_STATIC_LIMIT: return "problem needs more scratch than the library's built-in static array holds";
   }
   return "unknown status";
 }
@@ -413,6 +414,62 @@ fp4_status fp4_gemm_nt(const uint8_t* a_codes, const uint8_t* a_scales, float a_
   a.sg_a = a_tensor_scale; a.sg_b = b_tensor_scale;
   a.status = device_status;
   return launch_gemm(kPlain, tmA, tmB, tmD, tmD, a, d->sms, stream) == cudaSuccess ? FP4_OK : FP4_ERR_CUDA;
+}
+
+}  // extern "C"
+
+// ---- fp4_root_ns_static: the step with the workspace in a static device array ------------
+// For callers that cannot allocate device memory (no cudaMalloc allowed where they run, or
+// no pool to take a workspace from).  The array is part of the module image: every device
+// that loads the library holds these 16 MiB until the process ends.  In host code the
+// array's name stands for the symbol, it is not a device address; the address is looked up
+// once per device with cudaGetSymbolAddress and handed to the kernels like any workspace.
+namespace {
+static __device__ __align__(256) unsigned char g_static_scratch[FP4_STATIC_SCRATCH_BYTES];
+void* g_static_ptr[64] = {nullptr};
+std::mutex g_static_mu;
+
+// Device address of the static array on the current device; looked up on the first call.
+fp4_status static_scratch_address(void** ptr) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return FP4_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_static_mu);
+  if (g_static_ptr[dev] == nullptr) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) return FP4_ERR_CUDA;
+    g_static_ptr[dev] = p;
+  }
+  *ptr = g_static_ptr[dev];
+  return FP4_OK;
+}
+}  // namespace
+
+extern "C" {
+
+fp4_status fp4_root_ns_static(const float* G, float* out, int64_t m, int64_t n, int steps, const fp4_ns_params* p,
+                              uint32_t* device_status, cudaStream_t stream) {
+  fp4_ns_params dp;
+  if (!p) { default_params(&dp); p = &dp; }
+  if (!G || !out) return FP4_ERR_INVALID_ARG;
+  if (!shape_ok(m) || !shape_ok(n)) return FP4_ERR_SHAPE;
+  if (steps < 0 || steps > kMaxSteps) return FP4_ERR_INVALID_ARG;
+  if (!aligned(G, 16) || !aligned(out, 16) || (device_status && !aligned(device_status, 4))) return FP4_ERR_ALIGNMENT;
+  const size_t need = fp4_root_ns_workspace_bytes(m, n, steps, p->flags);
+  if (need == 0) return FP4_ERR_SHAPE;
+  if (need > FP4_STATIC_SCRATCH_BYTES) return FP4_ERR_STATIC_LIMIT;
+  const DeviceInfo* d;
+  fp4_status rc = check_common(&d);
+  if (rc != FP4_OK) return rc;
+  void* scratch = nullptr;
+  rc = static_scratch_address(&scratch);
+  if (rc != FP4_OK) return rc;
+  // run_one clears the header, the scalars and the histogram of the shared array itself
+  rc = run_one(d, G, out, m, n, steps, p, static_cast<uint8_t*>(scratch), true, stream);
+  if (rc != FP4_OK) return rc;
+  if (device_status &&
+      cudaMemcpyAsync(device_status, scratch, 4, cudaMemcpyDeviceToDevice, stream) != cudaSuccess)
+    return FP4_ERR_CUDA;
+  return FP4_OK;
 }
 
 void fp4_profile_enable(int on) { g_prof_on.store(on ? 1 : 0); }
