@@ -14,8 +14,12 @@
 //
 // One CTA owns 128 x 128 output tiles.  Warp roles: 0 = TMA producer of operand stages,
 // 1 = MMA issuer (one thread) and TMEM owner, 2 = TMA producer of the FP32 tile the
-// epilogue combines with, 3..6 = epilogue (TMEM lane quadrant = warp % 4).  Two CTAs
-// share an SM, so one CTA's epilogue overlaps the other's main loop.
+// epilogue combines with, 3 = TMA-store issuer, 4..7 = drain (TMEM lane quadrant =
+// warp % 4), 8..11 = finish.  The epilogue is a pipeline over a ring of 8 KB chunk buffers
+// (16 FP32 columns x 128 rows) connected by mbarriers only: TMA load of the FP32 tile
+// chunk -> drain (combine, quantise along the row, write the result chunk in place) ->
+// TMA store and, concurrently, finish (quantise down the columns) -> slot free.  Two CTAs
+// share an SM, so one CTA's epilogue also overlaps the other's main loop.
 #include "fp4_kernels.h"
 
 namespace fp4 {
@@ -24,9 +28,13 @@ namespace {
 
 constexpr int BM = 128, BN = 128, BK = 128;
 #ifndef FP4_STAGES
-#define FP4_STAGES 4
+#define FP4_STAGES 3
 #endif
-constexpr int STAGES = FP4_STAGES;
+#ifndef FP4_RING
+#define FP4_RING 7
+#endif
+constexpr int STAGES = FP4_STAGES;          // operand stages of the main loop
+constexpr int RING = FP4_RING;              // FP32 chunk buffers of the epilogue
 constexpr int OPER_BYTES = BM * BK / 2;      // 8192: one operand tile of a stage (64-byte rows)
 constexpr int SF_BYTES = 2 * 512;            // two scale atoms (128 rows x 8 blocks) per operand and stage
 constexpr uint32_t STAGE_TX = 2 * OPER_BYTES + 2 * SF_BYTES;
@@ -38,13 +46,14 @@ constexpr int OFF_A = 0;
 constexpr int OFF_B = OFF_A + STAGES * OPER_BYTES;
 constexpr int OFF_SFA = OFF_B + STAGES * OPER_BYTES;
 constexpr int OFF_SFB = OFF_SFA + STAGES * SF_BYTES;
-constexpr int OFF_AUX = OFF_SFB + STAGES * SF_BYTES;
-constexpr int OFF_OUT = OFF_AUX + 2 * CHUNK_BYTES;
-constexpr int OFF_BAR = OFF_OUT + 2 * CHUNK_BYTES;
-constexpr int SMEM_BYTES = OFF_BAR + 256 + 1024;  // + slack to align the base to 1024
+constexpr int OFF_RING = OFF_SFB + STAGES * SF_BYTES;
+constexpr int OFF_BAR = OFF_RING + RING * CHUNK_BYTES;
+constexpr int SMEM_BYTES = OFF_BAR + 512 + 1024;  // + slack to align the base to 1024
+static_assert(2 * (SMEM_BYTES + 1024) <= 233472, "two CTAs must fit in one SM's shared memory");
 
-constexpr int NTHREADS = 224;
-constexpr int EPI_THREADS = 128;
+// warps: 0 operand producer, 1 MMA issuer, 2 producer of the FP32 tile, 3 TMA-store issuer,
+// 4..7 drain (TMEM -> registers -> ring), 8..11 finish (transposed quantisation from the ring)
+constexpr int NTHREADS = 384;
 constexpr uint32_t TMEM_COLS = 256;
 constexpr uint32_t TMEM_SF_COL = 128;  // scale factors: 16 columns per stage after the accumulator
 
@@ -53,15 +62,17 @@ constexpr uint32_t IDESC = (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) 
                            ((uint32_t)(BM >> 4) << 24);
 
 struct Barriers {
-  uint64_t full[STAGES];
-  uint64_t empty[STAGES];
-  uint64_t acc_full;
-  uint64_t acc_empty;
-  uint64_t aux_full[2];
-  uint64_t aux_empty[2];
+  uint64_t full[STAGES];     // operand stage landed (TMA bytes)
+  uint64_t empty[STAGES];    // operand stage consumed (MMA commit)
+  uint64_t acc_full;         // accumulator complete (MMA commit)
+  uint64_t acc_empty;        // accumulator drained (4 drain warps)
+  uint64_t aux_full[RING];   // FP32 tile chunk landed in a ring slot (TMA bytes)
+  uint64_t v_ready[RING];    // result chunk written to the slot (4 drain warps)
+  uint64_t slot_free[RING];  // slot read by everyone: 4 finish warps + the store warp
   uint32_t tmem_base;
   uint32_t abort_flag;
 };
+static_assert(sizeof(Barriers) <= 512, "barrier block");
 
 __device__ __forceinline__ uint64_t globaltimer_ns() {
   uint64_t t;
@@ -88,18 +99,6 @@ __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatil
   return wait_slow(bar, parity, abort_flag);
 }
 
-// barrier over the epilogue threads that also ANDs a predicate
-__device__ __forceinline__ bool epi_barrier_and(bool pred) {
-  uint32_t r;
-  asm volatile(
-      "{\n\t.reg .pred p, q;\n\tsetp.ne.b32 p, %1, 0;\n\t"
-      "barrier.cta.red.and.pred q, 1, 128, p;\n\tselp.u32 %0, 1, 0, q;\n\t}"
-      : "=r"(r)
-      : "r"((uint32_t)pred)
-      : "memory");
-  return r != 0;
-}
-
 __device__ __forceinline__ void decode_tile(int t, int tiles_n, int symmetric, int& ti, int& tj) {
   if (!symmetric) {
     ti = t / tiles_n;
@@ -109,6 +108,40 @@ __device__ __forceinline__ void decode_tile(int t, int tiles_n, int symmetric, i
     while (rem >= tiles_n - row) { rem -= tiles_n - row; ++row; }
     ti = row;
     tj = row + rem;
+  }
+}
+
+// Per-call scalars of an epilogue: the factor that turns the accumulator into the
+// product (tensor scales of the two operands) and the tensor scale of the quantised
+// output, predicted from the running maxima (power of two).
+template <int MODE>
+__device__ __forceinline__ void epilogue_scalars(const GemmArgs& args, float& scale, float& sg_out, bool publish) {
+  float* sc = args.scalars;
+  sg_out = 1.0f;
+  if (MODE == kPlain) {
+    scale = __fmul_rn(args.sg_a, args.sg_b);
+  } else if (MODE == kG1) {
+    const float sgx = sc[args.ix.sg_X0 + args.iter];
+    const float ax = sc[args.ix.amax_X0 + args.iter];
+    scale = __fmul_rn(sgx, sgx);
+    float bound = __fmul_rn(__fmul_rn(__fmul_rn(2.0f, args.l_cols), ax), ax);
+    sg_out = scale_predicted(fminf(bound, 4.0f));
+    if (publish) sc[args.ix.sg_A0 + args.iter] = sg_out;
+  } else if (MODE == kG2) {
+    const float sga = sc[args.ix.sg_A0 + args.iter];
+    const float aa = sc[args.ix.amax_A0 + args.iter];
+    scale = __fmul_rn(sga, sga);
+    float bound = __fmul_rn(__fadd_rn(fabsf(args.cb), __fmul_rn(4.0f, fabsf(args.cc))), aa);
+    sg_out = scale_predicted(bound);
+    if (publish) sc[args.ix.sg_B0 + args.iter] = sg_out;
+  } else {
+    const float sgb = sc[args.ix.sg_B0 + args.iter];
+    const float sgx = sc[args.ix.sg_X0 + args.iter];
+    const float ax = sc[args.ix.amax_X0 + args.iter];
+    scale = __fmul_rn(sgb, sgx);
+    float bound = __fmul_rn(__fmul_rn(4.0f, fabsf(args.ca)), ax);
+    sg_out = scale_predicted(bound);
+    if (publish) sc[args.ix.sg_X0 + args.iter + 1] = sg_out;
   }
 }
 
@@ -123,15 +156,24 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int num_tiles = args.symmetric ? args.tiles_n * (args.tiles_n + 1) / 2 : args.tiles_m * args.tiles_n;
+#ifdef FP4_DEBUG_ONE_KBLOCK
+  const int num_kb = 1;  // timing experiments only: epilogue cost without the main loop
+#else
   const int num_kb = args.K / BK;
+#endif
   constexpr bool HAS_AUX = (MODE == kG2 || MODE == kG3);
   constexpr bool STORE_F32 = (MODE == kPlain || MODE == kG1 || MODE == kG3);
+  const bool do_q = (MODE != kPlain) && args.write_q;
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < STAGES; ++i) { mbar_init(&bars->full[i], 1); mbar_init(&bars->empty[i], 1); }
     mbar_init(&bars->acc_full, 1);
-    mbar_init(&bars->acc_empty, EPI_THREADS);
-    for (int i = 0; i < 2; ++i) { mbar_init(&bars->aux_full[i], 1); mbar_init(&bars->aux_empty[i], EPI_THREADS); }
+    mbar_init(&bars->acc_empty, 4);
+    for (int i = 0; i < RING; ++i) {
+      mbar_init(&bars->aux_full[i], 1);
+      mbar_init(&bars->v_ready[i], 4);
+      mbar_init(&bars->slot_free[i], 5);
+    }
     bars->abort_flag = 0;
     mbar_fence_init();
     tma_prefetch_desc(&tmA);
@@ -202,56 +244,64 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
     }
   } else if (warp == 2) {
     // ------------------------------------------------------------ producer of the FP32 tile
+    // Loads the chunk the epilogue combines with (A for G2, X for G3) into the ring slot
+    // that will afterwards hold the result chunk, as soon as the slot is free: the loads
+    // of a tile run ahead of its main loop.
     if (HAS_AUX && elect_one()) {
       uint32_t it = 0; bool ok = true;
       for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
         int ti, tj;
         decode_tile(t, args.tiles_n, args.symmetric, ti, tj);
         for (int c = 0; c < NCHUNK; ++c, ++it) {
-          const int b = it & 1;
-          if (!wait_bar(&bars->aux_empty[b], ((it >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
+          const int b = it % RING;
+          const uint32_t use = it / RING;
+          if (!wait_bar(&bars->slot_free[b], (use & 1) ^ 1, abort_flag)) { ok = false; break; }
           mbar_expect_tx(&bars->aux_full[b], CHUNK_BYTES);
-          tma_load_2d(smem + OFF_AUX + b * CHUNK_BYTES, &tmAux, tj * BN + c * CHUNK, ti * BM, &bars->aux_full[b]);
+          tma_load_2d(smem + OFF_RING + b * CHUNK_BYTES, &tmAux, tj * BN + c * CHUNK, ti * BM, &bars->aux_full[b]);
         }
       }
     }
-  } else {
-    // ------------------------------------------------------------ epilogue
-    const int quad = warp & 3;
-    const int row = quad * 32 + lane;           // row of the tile this thread owns (TMEM lane)
-    const int et = (warp - 3) * 32 + lane;      // index among the epilogue threads
-    const bool leader = (et == 0);
-
-    // per-call scalars (written by earlier kernels of the stream)
-    float scale, sg_out = 1.0f;
-    float* sc = args.scalars;
-    if (MODE == kPlain) {
-      scale = __fmul_rn(args.sg_a, args.sg_b);
-    } else if (MODE == kG1) {
-      const float sgx = sc[args.ix.sg_X0 + args.iter];
-      const float ax = sc[args.ix.amax_X0 + args.iter];
-      scale = __fmul_rn(sgx, sgx);
-      float bound = __fmul_rn(__fmul_rn(__fmul_rn(2.0f, args.l_cols), ax), ax);
-      sg_out = scale_predicted(fminf(bound, 4.0f));
-      if (blockIdx.x == 0 && leader) sc[args.ix.sg_A0 + args.iter] = sg_out;
-    } else if (MODE == kG2) {
-      const float sga = sc[args.ix.sg_A0 + args.iter];
-      const float aa = sc[args.ix.amax_A0 + args.iter];
-      scale = __fmul_rn(sga, sga);
-      float bound = __fmul_rn(__fadd_rn(fabsf(args.cb), __fmul_rn(4.0f, fabsf(args.cc))), aa);
-      sg_out = scale_predicted(bound);
-      if (blockIdx.x == 0 && leader) sc[args.ix.sg_B0 + args.iter] = sg_out;
-    } else {
-      const float sgb = sc[args.ix.sg_B0 + args.iter];
-      const float sgx = sc[args.ix.sg_X0 + args.iter];
-      const float ax = sc[args.ix.amax_X0 + args.iter];
-      scale = __fmul_rn(sgb, sgx);
-      float bound = __fmul_rn(__fmul_rn(4.0f, fabsf(args.ca)), ax);
-      sg_out = scale_predicted(bound);
-      if (blockIdx.x == 0 && leader) sc[args.ix.sg_X0 + args.iter + 1] = sg_out;
+  } else if (warp == 3) {
+    // ------------------------------------------------------------ TMA-store issuer
+    // Stores each finished chunk and hands the slot back once the store has read it.
+    if (elect_one()) {
+      uint32_t it = 0; bool ok = true;
+      int prev_slot = -1;
+      for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+        int ti, tj;
+        decode_tile(t, args.tiles_n, args.symmetric, ti, tj);
+        for (int c = 0; c < NCHUNK; ++c, ++it) {
+          const int b = it % RING;
+          const uint32_t use = it / RING;
+          if (!wait_bar(&bars->v_ready[b], use & 1, abort_flag)) { ok = false; break; }
+          if (STORE_F32) {
+            tma_store_2d(&tmOut, tj * BN + c * CHUNK, ti * BM, smem + OFF_RING + b * CHUNK_BYTES);
+            bulk_commit();
+            bulk_wait_read<1>();  // every store but the newest has read its slot
+            if (prev_slot >= 0) mbar_arrive(&bars->slot_free[prev_slot]);
+            prev_slot = b;
+          } else {
+            mbar_arrive(&bars->slot_free[b]);
+          }
+        }
+      }
+      if (STORE_F32) {
+        bulk_wait_read<0>();
+        if (prev_slot >= 0) mbar_arrive(&bars->slot_free[prev_slot]);
+        bulk_wait_all<0>();
+      }
     }
+  } else if (warp < 8) {
+    // ------------------------------------------------------------ drain warps
+    // TMEM -> registers (thread = row), combine with the FP32 tile, quantise the blocks
+    // that run along the row, write the result chunk into the ring slot.
+    const int quad = warp & 3;
+    const int row = quad * 32 + lane;
+    float scale, sg_out;
+    epilogue_scalars<MODE>(args, scale, sg_out, blockIdx.x == 0 && threadIdx.x == 128);
     const float six_sg = __fmul_rn(6.0f, sg_out);
-    const bool do_q = (MODE != kPlain) && args.write_q;
+    const int sw = (row >> 1) & 3;
+    const uint32_t tm_lane = tmem_base + ((uint32_t)(quad * 32) << 16);
 
     uint32_t acc_ph = 0, it = 0;
     float amax = 0.0f;
@@ -261,95 +311,71 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
       decode_tile(t, args.tiles_n, args.symmetric, ti, tj);
       const bool mirror = do_q && (MODE == kG3 || (args.symmetric && ti != tj));
       // give-up decisions are made warp-uniform: the TMEM loads below are warp-collective
-      bool tile_ok = __all_sync(0xffffffffu, wait_bar(&bars->acc_full, acc_ph, abort_flag));
+      ok = __all_sync(0xffffffffu, wait_bar(&bars->acc_full, acc_ph, abort_flag));
       acc_ph ^= 1;
+      if (!ok) break;
       tc_fence_after();
-      const int64_t grow = (int64_t)ti * BM + row;  // global row of this thread
+      const int64_t grow = (int64_t)ti * BM + row;
       uint32_t sfw = 0;
+      uint32_t acc[16];
+      tc_ld16_issue(tm_lane, acc);
       for (int c = 0; c < NCHUNK; ++c, ++it) {
-        const int b = it & 1;
+        const int b = it % RING;
+        const uint32_t use = it / RING;
+        uint8_t* slot_row = smem + OFF_RING + b * CHUNK_BYTES + row * 64;
         float v[16];
-        if (tile_ok) {
-          float acc[16];
-          tc_ld16(tmem_base + ((uint32_t)(quad * 32) << 16) + c * CHUNK, acc);
-          if (c == NCHUNK - 1) {  // accumulator drained: the next tile's MMAs may start
-            tc_fence_before();
-            mbar_arrive(&bars->acc_empty);
-          }
-          if (HAS_AUX) {
-            tile_ok = __all_sync(0xffffffffu, wait_bar(&bars->aux_full[b], (it >> 1) & 1, abort_flag));
-            if (tile_ok) {
-              const uint8_t* arow = smem + OFF_AUX + b * CHUNK_BYTES + row * 64;
-              const int sw = (row >> 1) & 3;
+        // the slot: holds the FP32 tile chunk (G2, G3) or must be free (G1, plain)
+        if (HAS_AUX) ok = __all_sync(0xffffffffu, wait_bar(&bars->aux_full[b], use & 1, abort_flag));
+        else ok = __all_sync(0xffffffffu, wait_bar(&bars->slot_free[b], (use & 1) ^ 1, abort_flag));
+        if (!ok) break;
+        tc_wait_ld16(acc);
+        if (HAS_AUX) {
 #pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                float4 x = *reinterpret_cast<const float4*>(arow + ((j ^ sw) << 4));
-                float e[4] = {x.x, x.y, x.z, x.w};
+          for (int j = 0; j < 4; ++j) {
+            float4 x = *reinterpret_cast<const float4*>(slot_row + ((j ^ sw) << 4));
+            float e[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                  const float p = __fmul_rn(acc[4 * j + q], scale);
-                  if (MODE == kG2) v[4 * j + q] = __fadd_rn(__fmul_rn(args.cb, e[q]), __fmul_rn(args.cc, p));
-                  else v[4 * j + q] = __fadd_rn(__fmul_rn(args.ca, e[q]), p);
-                }
-              }
-              mbar_arrive(&bars->aux_empty[b]);
-            }
-          } else {
-#pragma unroll
-            for (int i = 0; i < 16; ++i) v[i] = __fmul_rn(acc[i], scale);
-          }
-        }
-        if (tile_ok) {
-          if (MODE == kG1 || MODE == kG3) {
-#pragma unroll
-            for (int i = 0; i < 16; ++i) amax = fmaxf(amax, fabsf(v[i]));
-          }
-          if (do_q) {
-            // blocks of 16 along this tile's columns: in-thread
-            uint32_t lo, hi;
-            uint32_t sb = quantize_block16(v, six_sg, sg_out, lo, hi);
-            const int64_t gcol = (int64_t)tj * BN + c * CHUNK;
-            *reinterpret_cast<uint2*>(args.rq_codes + grow * (args.rq_K / 2) + gcol / 2) = make_uint2(lo, hi);
-            sfw |= sb << (8 * (c & 3));
-            if ((c & 3) == 3) {
-              *reinterpret_cast<uint32_t*>(args.rq_sf + sf_offset(grow, (gcol >> 4) & ~3ll, args.rq_K >> 4)) = sfw;
-              sfw = 0;
+            for (int q = 0; q < 4; ++q) {
+              const float p = __fmul_rn(__uint_as_float(acc[4 * j + q]), scale);
+              if (MODE == kG2) v[4 * j + q] = __fadd_rn(__fmul_rn(args.cb, e[q]), __fmul_rn(args.cc, p));
+              else v[4 * j + q] = __fadd_rn(__fmul_rn(args.ca, e[q]), p);
             }
           }
-          if (STORE_F32 || mirror) {
-            // stage the FP32 chunk in the 64-byte-swizzled layout TMA stores from
-            uint8_t* orow = smem + OFF_OUT + b * CHUNK_BYTES + row * 64;
-            const int sw = (row >> 1) & 3;
+        } else {
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-              *reinterpret_cast<float4*>(orow + ((j ^ sw) << 4)) = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-            fence_proxy_async_smem();
-          }
+          for (int i = 0; i < 16; ++i) v[i] = __fmul_rn(__uint_as_float(acc[i]), scale);
         }
-        // the previous chunk's store must have read its staging buffer before the next
-        // chunk overwrites it
-        if (STORE_F32 && leader) bulk_wait_read<0>();
-        if (!epi_barrier_and(tile_ok)) { ok = false; break; }
-        if (STORE_F32 && leader) {
-          tma_store_2d(&tmOut, tj * BN + c * CHUNK, ti * BM, smem + OFF_OUT + b * CHUNK_BYTES);
-          bulk_commit();
+        // the next chunk's accumulator columns are fetched while this chunk is finished
+        if (c + 1 < NCHUNK) {
+          tc_ld16_issue(tm_lane + (c + 1) * CHUNK, acc);
+        } else {
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&bars->acc_empty);  // the next tile's MMAs may start
         }
-        if (mirror) {
-          // blocks of 16 down this tile's rows: thread = (column cc, row group g)
-          const int cc = et & 15, g = et >> 4;
-          const uint8_t* obase = smem + OFF_OUT + b * CHUNK_BYTES;
-          float w[16];
+        if (STORE_F32 || mirror) {
 #pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const int r = g * 16 + i;
-            w[i] = *reinterpret_cast<const float*>(obase + r * 64 + ((((cc >> 2) ^ ((r >> 1) & 3))) << 4) + (cc & 3) * 4);
-          }
+          for (int j = 0; j < 4; ++j)
+            *reinterpret_cast<float4*>(slot_row + ((j ^ sw) << 4)) =
+                make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+          fence_proxy_async_smem();
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bars->v_ready[b]);
+        if (MODE == kG1 || MODE == kG3) {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) amax = fmaxf(amax, fabsf(v[i]));
+        }
+        if (do_q) {
           uint32_t lo, hi;
-          uint32_t sb = quantize_block16(w, six_sg, sg_out, lo, hi);
-          const int64_t trow = (int64_t)tj * BN + c * CHUNK + cc;  // row of the mirrored / transposed tensor
-          const int64_t tcol = (int64_t)ti * BM + g * 16;
-          *reinterpret_cast<uint2*>(args.cq_codes + trow * (args.cq_K / 2) + tcol / 2) = make_uint2(lo, hi);
-          args.cq_sf[sf_offset(trow, tcol >> 4, args.cq_K >> 4)] = (uint8_t)sb;
+          uint32_t sb = quantize_block16(v, six_sg, sg_out, lo, hi);
+          const int64_t gcol = (int64_t)tj * BN + c * CHUNK;
+          *reinterpret_cast<uint2*>(args.rq_codes + grow * (args.rq_K / 2) + gcol / 2) = make_uint2(lo, hi);
+          sfw |= sb << (8 * (c & 3));
+          if ((c & 3) == 3) {
+            *reinterpret_cast<uint32_t*>(args.rq_sf + sf_offset(grow, (gcol >> 4) & ~3ll, args.rq_K >> 4)) = sfw;
+            sfw = 0;
+          }
         }
       }
     }
@@ -358,10 +384,51 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
       for (int o = 16; o; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
       if (lane == 0) {
         const int slot = (MODE == kG1) ? args.ix.amax_A0 + args.iter : args.ix.amax_X0 + args.iter + 1;
-        atomicMax(reinterpret_cast<uint32_t*>(sc + slot), __float_as_uint(amax));
+        atomicMax(reinterpret_cast<uint32_t*>(args.scalars + slot), __float_as_uint(amax));
       }
     }
-    if (STORE_F32 && leader) bulk_wait_all<0>();
+  } else {
+    // ------------------------------------------------------------ finish warps
+    // Blocks of 16 that run down this tile's rows (the transposed operand copy in G3, the
+    // mirrored triangle in G1/G2): thread = (column cc of the chunk, row group g).
+    const int et = threadIdx.x - 256;
+    const int cc = et & 15, g = et >> 4;
+    float scale, sg_out;
+    epilogue_scalars<MODE>(args, scale, sg_out, false);
+    const float six_sg = __fmul_rn(6.0f, sg_out);
+    uint32_t it = 0;
+    bool ok = true;
+    for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+      int ti, tj;
+      decode_tile(t, args.tiles_n, args.symmetric, ti, tj);
+      const bool mirror = do_q && (MODE == kG3 || (args.symmetric && ti != tj));
+      for (int c = 0; c < NCHUNK; ++c, ++it) {
+        const int b = it % RING;
+        const uint32_t use = it / RING;
+        ok = __all_sync(0xffffffffu, wait_bar(&bars->v_ready[b], use & 1, abort_flag));
+        if (!ok) break;
+        if (mirror) {
+          const uint8_t* obase = smem + OFF_RING + b * CHUNK_BYTES;
+          float w[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const int r = g * 16 + i;
+            w[i] = *reinterpret_cast<const float*>(obase + r * 64 + ((((cc >> 2) ^ ((r >> 1) & 3))) << 4) + (cc & 3) * 4);
+          }
+          uint32_t lo, hi;
+          uint32_t sb = quantize_block16(w, six_sg, sg_out, lo, hi);
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&bars->slot_free[b]);  // the slot's values are in registers
+          const int64_t trow = (int64_t)tj * BN + c * CHUNK + cc;  // row of the mirrored / transposed tensor
+          const int64_t tcol = (int64_t)ti * BM + g * 16;
+          *reinterpret_cast<uint2*>(args.cq_codes + trow * (args.cq_K / 2) + tcol / 2) = make_uint2(lo, hi);
+          args.cq_sf[sf_offset(trow, tcol >> 4, args.cq_K >> 4)] = (uint8_t)sb;
+        } else {
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&bars->slot_free[b]);
+        }
+      }
+    }
   }
 
   tc_fence_before();
