@@ -63,6 +63,8 @@ typedef struct {
                           per million.  Default 0.99; <= 0 or >= 1 disables the clip.      */
   float eps;           /* X0 = G_c / (||G_c||_F + eps).  Default 1e-7.                     */
   uint32_t flags;      /* FP4_FLAG_*; default 0                                            */
+  uint32_t max_group;  /* fp4_root_ns_batched: at most this many equal-shape matrices run their
+                          stages in lockstep as single launches; 0 = library default (8)      */
 } fp4_ns_params;
 
 const char* fp4_status_string(fp4_status s);
@@ -116,7 +118,11 @@ fp4_status fp4_root_ns(const float* G, float* out, int64_t m, int64_t n, int ste
 /* ---- many matrices of different shapes in one call (the matrices of a layer stack) ------
  * count matrices; G, out, m, n: host arrays of length count (G[i], out[i] device pointers).
  * One parameter block applies to all (coefficients per matrix when p->a is NaN).
- * ws: device, at least fp4_root_ns_batched_workspace_bytes(...) bytes, 256-byte aligned.
+ * ws: device, at least fp4_root_ns_batched_workspace_bytes(...) bytes, 256-byte aligned: one
+ *   single-matrix workspace per matrix plus the tables of the grouped launches.
+ * Matrices of equal shape (after orientation) are grouped: each Newton-Schulz stage of a
+ * group is one launch whose tile list spans all its matrices.  Results are bit-identical to
+ * calling fp4_root_ns on each matrix.
  */
 size_t fp4_root_ns_batched_workspace_bytes(int count, const int64_t* m, const int64_t* n,
                                            int steps, uint32_t flags);

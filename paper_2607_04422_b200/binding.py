@@ -37,16 +37,17 @@ class Fp4Error(RuntimeError):
 class NsParams(C.Structure):
     """fp4_ns_params"""
     _fields_ = [("a", C.c_float), ("b", C.c_float), ("c", C.c_float), ("clip_quantile", C.c_float),
-                ("eps", C.c_float), ("flags", C.c_uint32)]
+                ("eps", C.c_float), ("flags", C.c_uint32), ("max_group", C.c_uint32)]
 
     @classmethod
-    def make(cls, abc=None, clip_quantile=0.99, eps=1e-7, flags=0):
+    def make(cls, abc=None, clip_quantile=0.99, eps=1e-7, flags=0, max_group=0):
         p = cls()
         if abc is None:
             p.a = p.b = p.c = float("nan")
         else:
             p.a, p.b, p.c = [float(v) for v in abc]
         p.clip_quantile, p.eps, p.flags = float(clip_quantile), float(eps), int(flags)
+        p.max_group = int(max_group)
         return p
 
 

@@ -99,8 +99,13 @@ __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatil
   return wait_slow(bar, parity, abort_flag);
 }
 
-__device__ __forceinline__ void decode_tile(int t, int tiles_n, int symmetric, int& ti, int& tj) {
-  if (!symmetric) {
+// tile index of a launch -> (problem, tile row, tile column)
+__device__ __forceinline__ void decode_tile(int t, const GemmLaunch& L, int tiles_per_problem, int& p, int& ti,
+                                            int& tj) {
+  p = t / tiles_per_problem;
+  t -= p * tiles_per_problem;
+  const int tiles_n = L.tiles_n;
+  if (!L.symmetric) {
     ti = t / tiles_n;
     tj = t - ti * tiles_n;
   } else {
@@ -115,11 +120,12 @@ __device__ __forceinline__ void decode_tile(int t, int tiles_n, int symmetric, i
 // product (tensor scales of the two operands) and the tensor scale of the quantised
 // output, predicted from the running maxima (power of two).
 template <int MODE>
-__device__ __forceinline__ void epilogue_scalars(const GemmArgs& args, float& scale, float& sg_out, bool publish) {
-  float* sc = args.scalars;
+__device__ __forceinline__ void epilogue_scalars(const GemmProblem& pr, const GemmLaunch& args, float& scale,
+                                                 float& sg_out, bool publish) {
+  float* sc = pr.scalars;
   sg_out = 1.0f;
   if (MODE == kPlain) {
-    scale = __fmul_rn(args.sg_a, args.sg_b);
+    scale = __fmul_rn(pr.sg_a, pr.sg_b);
   } else if (MODE == kG1) {
     const float sgx = sc[args.ix.sg_X0 + args.iter];
     const float ax = sc[args.ix.amax_X0 + args.iter];
@@ -131,7 +137,7 @@ __device__ __forceinline__ void epilogue_scalars(const GemmArgs& args, float& sc
     const float sga = sc[args.ix.sg_A0 + args.iter];
     const float aa = sc[args.ix.amax_A0 + args.iter];
     scale = __fmul_rn(sga, sga);
-    float bound = __fmul_rn(__fadd_rn(fabsf(args.cb), __fmul_rn(4.0f, fabsf(args.cc))), aa);
+    float bound = __fmul_rn(__fadd_rn(fabsf(pr.cb), __fmul_rn(4.0f, fabsf(pr.cc))), aa);
     sg_out = scale_predicted(bound);
     if (publish) sc[args.ix.sg_B0 + args.iter] = sg_out;
   } else {
@@ -139,7 +145,7 @@ __device__ __forceinline__ void epilogue_scalars(const GemmArgs& args, float& sc
     const float sgx = sc[args.ix.sg_X0 + args.iter];
     const float ax = sc[args.ix.amax_X0 + args.iter];
     scale = __fmul_rn(sgb, sgx);
-    float bound = __fmul_rn(__fmul_rn(4.0f, fabsf(args.ca)), ax);
+    float bound = __fmul_rn(__fmul_rn(4.0f, fabsf(pr.ca)), ax);
     sg_out = scale_predicted(bound);
     if (publish) sc[args.ix.sg_X0 + args.iter + 1] = sg_out;
   }
@@ -147,15 +153,16 @@ __device__ __forceinline__ void epilogue_scalars(const GemmArgs& args, float& sc
 
 template <int MODE>
 __global__ void __launch_bounds__(NTHREADS, 2)
-k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-       const __grid_constant__ CUtensorMap tmAux, const __grid_constant__ CUtensorMap tmOut, const GemmArgs args) {
+k_gemm(const __grid_constant__ GemmProblem single, const GemmProblem* __restrict__ table, const GemmLaunch args) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   Barriers* bars = reinterpret_cast<Barriers*>(smem + OFF_BAR);
   volatile uint32_t* abort_flag = &bars->abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int num_tiles = args.symmetric ? args.tiles_n * (args.tiles_n + 1) / 2 : args.tiles_m * args.tiles_n;
+  const GemmProblem* probs = table ? table : &single;
+  const int tiles_per_problem = args.symmetric ? args.tiles_n * (args.tiles_n + 1) / 2 : args.tiles_m * args.tiles_n;
+  const int num_tiles = tiles_per_problem * args.num_problems;
 #ifdef FP4_DEBUG_ONE_KBLOCK
   const int num_kb = 1;  // timing experiments only: epilogue cost without the main loop
 #else
@@ -176,10 +183,6 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
     }
     bars->abort_flag = 0;
     mbar_fence_init();
-    tma_prefetch_desc(&tmA);
-    tma_prefetch_desc(&tmB);
-    if (HAS_AUX) tma_prefetch_desc(&tmAux);
-    if (STORE_F32) tma_prefetch_desc(&tmOut);
   }
   if (warp == 1) {
     tmem_alloc(&bars->tmem_base, TMEM_COLS);
@@ -195,15 +198,16 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
     if (elect_one()) {
       int st = 0; uint32_t ph = 0; bool ok = true;
       for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
-        int ti, tj;
-        decode_tile(t, args.tiles_n, args.symmetric, ti, tj);
-        const uint8_t* sfa = args.sfa + (size_t)ti * (args.K / 64) * 512;
-        const uint8_t* sfb = args.sfb + (size_t)tj * (args.K / 64) * 512;
+        int p, ti, tj;
+        decode_tile(t, args, tiles_per_problem, p, ti, tj);
+        const GemmProblem* pr = probs + p;
+        const uint8_t* sfa = pr->sfa + (size_t)ti * (args.K / 64) * 512;
+        const uint8_t* sfb = pr->sfb + (size_t)tj * (args.K / 64) * 512;
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!wait_bar(&bars->empty[st], ph ^ 1, abort_flag)) { ok = false; break; }
           mbar_expect_tx(&bars->full[st], STAGE_TX);
-          tma_load_2d(smem + OFF_A + st * OPER_BYTES, &tmA, kb * (BK / 2), ti * BM, &bars->full[st]);
-          tma_load_2d(smem + OFF_B + st * OPER_BYTES, &tmB, kb * (BK / 2), tj * BN, &bars->full[st]);
+          tma_load_2d(smem + OFF_A + st * OPER_BYTES, &pr->tmA, kb * (BK / 2), ti * BM, &bars->full[st]);
+          tma_load_2d(smem + OFF_B + st * OPER_BYTES, &pr->tmB, kb * (BK / 2), tj * BN, &bars->full[st]);
           bulk_load_1d(smem + OFF_SFA + st * SF_BYTES, sfa + (size_t)kb * SF_BYTES, SF_BYTES, &bars->full[st]);
           bulk_load_1d(smem + OFF_SFB + st * SF_BYTES, sfb + (size_t)kb * SF_BYTES, SF_BYTES, &bars->full[st]);
           if (++st == STAGES) { st = 0; ph ^= 1; }
@@ -250,14 +254,15 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
     if (HAS_AUX && elect_one()) {
       uint32_t it = 0; bool ok = true;
       for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
-        int ti, tj;
-        decode_tile(t, args.tiles_n, args.symmetric, ti, tj);
+        int p, ti, tj;
+        decode_tile(t, args, tiles_per_problem, p, ti, tj);
+        const GemmProblem* pr = probs + p;
         for (int c = 0; c < NCHUNK; ++c, ++it) {
           const int b = it % RING;
           const uint32_t use = it / RING;
           if (!wait_bar(&bars->slot_free[b], (use & 1) ^ 1, abort_flag)) { ok = false; break; }
           mbar_expect_tx(&bars->aux_full[b], CHUNK_BYTES);
-          tma_load_2d(smem + OFF_RING + b * CHUNK_BYTES, &tmAux, tj * BN + c * CHUNK, ti * BM, &bars->aux_full[b]);
+          tma_load_2d(smem + OFF_RING + b * CHUNK_BYTES, &pr->tmAux, tj * BN + c * CHUNK, ti * BM, &bars->aux_full[b]);
         }
       }
     }
@@ -268,14 +273,15 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
       uint32_t it = 0; bool ok = true;
       int prev_slot = -1;
       for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
-        int ti, tj;
-        decode_tile(t, args.tiles_n, args.symmetric, ti, tj);
+        int p, ti, tj;
+        decode_tile(t, args, tiles_per_problem, p, ti, tj);
+        const GemmProblem* pr = probs + p;
         for (int c = 0; c < NCHUNK; ++c, ++it) {
           const int b = it % RING;
           const uint32_t use = it / RING;
           if (!wait_bar(&bars->v_ready[b], use & 1, abort_flag)) { ok = false; break; }
           if (STORE_F32) {
-            tma_store_2d(&tmOut, tj * BN + c * CHUNK, ti * BM, smem + OFF_RING + b * CHUNK_BYTES);
+            tma_store_2d(&pr->tmOut, tj * BN + c * CHUNK, ti * BM, smem + OFF_RING + b * CHUNK_BYTES);
             bulk_commit();
             bulk_wait_read<1>();  // every store but the newest has read its slot
             if (prev_slot >= 0) mbar_arrive(&bars->slot_free[prev_slot]);
@@ -297,9 +303,10 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
     // that run along the row, write the result chunk into the ring slot.
     const int quad = warp & 3;
     const int row = quad * 32 + lane;
-    float scale, sg_out;
-    epilogue_scalars<MODE>(args, scale, sg_out, blockIdx.x == 0 && threadIdx.x == 128);
-    const float six_sg = __fmul_rn(6.0f, sg_out);
+    float scale = 0.0f, sg_out = 1.0f, six_sg = 6.0f;
+    float ca = 0.0f, cb = 0.0f, cc = 0.0f;
+    const GemmProblem* pr = nullptr;
+    int cur_p = -1;
     const int sw = (row >> 1) & 3;
     const uint32_t tm_lane = tmem_base + ((uint32_t)(quad * 32) << 16);
 
@@ -307,8 +314,26 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
     float amax = 0.0f;
     bool ok = true;
     for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
-      int ti, tj;
-      decode_tile(t, args.tiles_n, args.symmetric, ti, tj);
+      int p, ti, tj;
+      decode_tile(t, args, tiles_per_problem, p, ti, tj);
+      if (p != cur_p) {
+        // a new matrix: hand in the running maximum of the previous one, fetch this one's scalars
+        if ((MODE == kG1 || MODE == kG3) && cur_p >= 0) {
+#pragma unroll
+          for (int o = 16; o; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+          if (lane == 0) {
+            const int slot = (MODE == kG1) ? args.ix.amax_A0 + args.iter : args.ix.amax_X0 + args.iter + 1;
+            atomicMax(reinterpret_cast<uint32_t*>(pr->scalars + slot), __float_as_uint(amax));
+          }
+          amax = 0.0f;
+        }
+        cur_p = p;
+        pr = probs + p;
+        // the CTA that owns a matrix's first tile publishes its output scale
+        epilogue_scalars<MODE>(*pr, args, scale, sg_out, t == p * tiles_per_problem && threadIdx.x == 128);
+        six_sg = __fmul_rn(6.0f, sg_out);
+        ca = pr->ca; cb = pr->cb; cc = pr->cc;
+      }
       const bool mirror = do_q && (MODE == kG3 || (args.symmetric && ti != tj));
       // give-up decisions are made warp-uniform: the TMEM loads below are warp-collective
       ok = __all_sync(0xffffffffu, wait_bar(&bars->acc_full, acc_ph, abort_flag));
@@ -336,9 +361,9 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
             float e[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
-              const float p = __fmul_rn(__uint_as_float(acc[4 * j + q]), scale);
-              if (MODE == kG2) v[4 * j + q] = __fadd_rn(__fmul_rn(args.cb, e[q]), __fmul_rn(args.cc, p));
-              else v[4 * j + q] = __fadd_rn(__fmul_rn(args.ca, e[q]), p);
+              const float prod = __fmul_rn(__uint_as_float(acc[4 * j + q]), scale);
+              if (MODE == kG2) v[4 * j + q] = __fadd_rn(__fmul_rn(cb, e[q]), __fmul_rn(cc, prod));
+              else v[4 * j + q] = __fadd_rn(__fmul_rn(ca, e[q]), prod);
             }
           }
         } else {
@@ -370,21 +395,21 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
           uint32_t lo, hi;
           uint32_t sb = quantize_block16(v, six_sg, sg_out, lo, hi);
           const int64_t gcol = (int64_t)tj * BN + c * CHUNK;
-          *reinterpret_cast<uint2*>(args.rq_codes + grow * (args.rq_K / 2) + gcol / 2) = make_uint2(lo, hi);
+          *reinterpret_cast<uint2*>(pr->rq_codes + grow * (args.rq_K / 2) + gcol / 2) = make_uint2(lo, hi);
           sfw |= sb << (8 * (c & 3));
           if ((c & 3) == 3) {
-            *reinterpret_cast<uint32_t*>(args.rq_sf + sf_offset(grow, (gcol >> 4) & ~3ll, args.rq_K >> 4)) = sfw;
+            *reinterpret_cast<uint32_t*>(pr->rq_sf + sf_offset(grow, (gcol >> 4) & ~3ll, args.rq_K >> 4)) = sfw;
             sfw = 0;
           }
         }
       }
     }
-    if (MODE == kG1 || MODE == kG3) {
+    if ((MODE == kG1 || MODE == kG3) && cur_p >= 0) {
 #pragma unroll
       for (int o = 16; o; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
       if (lane == 0) {
         const int slot = (MODE == kG1) ? args.ix.amax_A0 + args.iter : args.ix.amax_X0 + args.iter + 1;
-        atomicMax(reinterpret_cast<uint32_t*>(args.scalars + slot), __float_as_uint(amax));
+        atomicMax(reinterpret_cast<uint32_t*>(pr->scalars + slot), __float_as_uint(amax));
       }
     }
   } else {
@@ -393,14 +418,20 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
     // mirrored triangle in G1/G2): thread = (column cc of the chunk, row group g).
     const int et = threadIdx.x - 256;
     const int cc = et & 15, g = et >> 4;
-    float scale, sg_out;
-    epilogue_scalars<MODE>(args, scale, sg_out, false);
-    const float six_sg = __fmul_rn(6.0f, sg_out);
+    float scale, sg_out = 1.0f, six_sg = 6.0f;
+    const GemmProblem* pr = nullptr;
+    int cur_p = -1;
     uint32_t it = 0;
     bool ok = true;
     for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
-      int ti, tj;
-      decode_tile(t, args.tiles_n, args.symmetric, ti, tj);
+      int p, ti, tj;
+      decode_tile(t, args, tiles_per_problem, p, ti, tj);
+      if (p != cur_p) {
+        cur_p = p;
+        pr = probs + p;
+        epilogue_scalars<MODE>(*pr, args, scale, sg_out, false);
+        six_sg = __fmul_rn(6.0f, sg_out);
+      }
       const bool mirror = do_q && (MODE == kG3 || (args.symmetric && ti != tj));
       for (int c = 0; c < NCHUNK; ++c, ++it) {
         const int b = it % RING;
@@ -421,8 +452,8 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
           if (lane == 0) mbar_arrive(&bars->slot_free[b]);  // the slot's values are in registers
           const int64_t trow = (int64_t)tj * BN + c * CHUNK + cc;  // row of the mirrored / transposed tensor
           const int64_t tcol = (int64_t)ti * BM + g * 16;
-          *reinterpret_cast<uint2*>(args.cq_codes + trow * (args.cq_K / 2) + tcol / 2) = make_uint2(lo, hi);
-          args.cq_sf[sf_offset(trow, tcol >> 4, args.cq_K >> 4)] = (uint8_t)sb;
+          *reinterpret_cast<uint2*>(pr->cq_codes + trow * (args.cq_K / 2) + tcol / 2) = make_uint2(lo, hi);
+          pr->cq_sf[sf_offset(trow, tcol >> 4, args.cq_K >> 4)] = (uint8_t)sb;
         } else {
           __syncwarp();
           if (lane == 0) mbar_arrive(&bars->slot_free[b]);
@@ -441,13 +472,15 @@ k_gemm(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensor
 }
 
 template <int MODE>
-cudaError_t launch_mode(const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmAux,
-                        const CUtensorMap& tmOut, const GemmArgs& args, int sms, cudaStream_t st) {
-  const int num_tiles = args.symmetric ? args.tiles_n * (args.tiles_n + 1) / 2 : args.tiles_m * args.tiles_n;
+cudaError_t launch_mode(const GemmProblem* single, const GemmProblem* table, const GemmLaunch& L, int sms,
+                        cudaStream_t st) {
+  const int tpp = L.symmetric ? L.tiles_n * (L.tiles_n + 1) / 2 : L.tiles_m * L.tiles_n;
+  const int num_tiles = tpp * L.num_problems;
   int grid = 2 * sms;
   if (grid > num_tiles) grid = num_tiles;
   count_launches(1);
-  k_gemm<MODE><<<grid, NTHREADS, SMEM_BYTES, st>>>(tmA, tmB, tmAux, tmOut, args);
+  static const GemmProblem kNone = {};
+  k_gemm<MODE><<<grid, NTHREADS, SMEM_BYTES, st>>>(single ? *single : kNone, table, L);
   return cudaGetLastError();
 }
 
@@ -462,13 +495,14 @@ cudaError_t gemm_set_attributes() {
   return cudaSuccess;
 }
 
-cudaError_t launch_gemm(GemmMode mode, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmAux,
-                        const CUtensorMap& tmOut, const GemmArgs& args, int sms, cudaStream_t st) {
+cudaError_t launch_gemm(GemmMode mode, const GemmProblem* single, const GemmProblem* table, const GemmLaunch& launch,
+                        int sms, cudaStream_t st) {
+  if ((single == nullptr) == (table == nullptr)) return cudaErrorInvalidValue;
   switch (mode) {
-    case kPlain: return launch_mode<kPlain>(tmA, tmB, tmAux, tmOut, args, sms, st);
-    case kG1: return launch_mode<kG1>(tmA, tmB, tmAux, tmOut, args, sms, st);
-    case kG2: return launch_mode<kG2>(tmA, tmB, tmAux, tmOut, args, sms, st);
-    default: return launch_mode<kG3>(tmA, tmB, tmAux, tmOut, args, sms, st);
+    case kPlain: return launch_mode<kPlain>(single, table, launch, sms, st);
+    case kG1: return launch_mode<kG1>(single, table, launch, sms, st);
+    case kG2: return launch_mode<kG2>(single, table, launch, sms, st);
+    default: return launch_mode<kG3>(single, table, launch, sms, st);
   }
 }
 

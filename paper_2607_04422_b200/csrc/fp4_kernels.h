@@ -51,21 +51,32 @@ enum GemmMode : int {
   kG3 = 3      // P = qB qXt^T; X+ = aX + P; store X+, emit qX+, qXt+, track amax(X+)
 };
 
-struct GemmArgs {
-  const uint8_t* sfa;  // scale atoms of the row operand
-  const uint8_t* sfb;  // scale atoms of the column operand
+// One matrix product of a launch.  A launch runs the same stage for a group of matrices
+// of one shape; the problems of a group sit in an array in device memory (or, for a single
+// problem, in the kernel's parameter space).
+struct alignas(64) GemmProblem {
+  CUtensorMap tmA, tmB;      // NVFP4 codes of the row and the column operand
+  CUtensorMap tmAux, tmOut;  // FP32 tile combined in the epilogue / FP32 result
+  const uint8_t* sfa;        // scale atoms of the row operand
+  const uint8_t* sfb;        // scale atoms of the column operand
+  float* scalars;            // workspace scalars of this matrix (device)
+  uint8_t* rq_codes; uint8_t* rq_sf;  // quantised output, blocks along the tile's columns
+  uint8_t* cq_codes; uint8_t* cq_sf;  // quantised output, blocks along the tile's rows
+  float ca, cb, cc;          // coefficients
+  float sg_a, sg_b;          // kPlain: tensor scales from the host
+};
+
+// What all problems of a launch share.
+struct GemmLaunch {
+  int num_problems;
   int K;               // contraction length in elements (multiple of 128)
   int tiles_m, tiles_n;
   int symmetric;       // only tiles with tile_n >= tile_m; mirrored quantised output
-  float* scalars;      // workspace scalars (device)
-  NsScalarIdx ix;
   int iter;            // Newton-Schulz iteration index k
-  float ca, cb, cc;    // coefficients
-  float l_cols;        // (float) l, for the bound on amax(A)
-  float sg_a, sg_b;    // kPlain: tensor scales from the host
-  uint8_t* rq_codes; uint8_t* rq_sf; int rq_K;  // quantised output, blocks along this tile's columns
-  uint8_t* cq_codes; uint8_t* cq_sf; int cq_K;  // quantised output, blocks along this tile's rows
   int write_q;         // emit the quantised outputs
+  int rq_K, cq_K;      // row lengths (elements) of the two quantised outputs
+  float l_cols;        // (float) l, for the bound on amax(A)
+  NsScalarIdx ix;
   uint32_t* status;
 };
 
@@ -86,7 +97,9 @@ cudaError_t launch_transpose_out(const float* X, int64_t s, int64_t l, float* ou
 cudaError_t prologue_set_attributes();
 
 cudaError_t gemm_set_attributes();
-cudaError_t launch_gemm(GemmMode mode, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmAux,
-                        const CUtensorMap& tmOut, const GemmArgs& args, int sms, cudaStream_t st);
+// single: the one problem of the launch (host copy, passed by value) when table is null;
+// table: device array of launch.num_problems problems.
+cudaError_t launch_gemm(GemmMode mode, const GemmProblem* single, const GemmProblem* table, const GemmLaunch& launch,
+                        int sms, cudaStream_t st);
 
 }  // namespace fp4

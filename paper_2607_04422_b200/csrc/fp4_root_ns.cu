@@ -98,11 +98,14 @@ bool make_f32_map(const DeviceInfo* d, CUtensorMap* tm, const void* base, int64_
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+constexpr int kDefaultMaxGroup = 8;
+
 void default_params(fp4_ns_params* p) {
   p->a = p->b = p->c = NAN;
   p->clip_quantile = 0.99f;
   p->eps = 1e-7f;
   p->flags = 0;
+  p->max_group = 0;
 }
 
 int64_t quantile_rank(int64_t n, float q) {
@@ -176,84 +179,158 @@ fp4_status make_plan(int64_t m, int64_t n, int steps, const fp4_ns_params* p, in
   return FP4_OK;
 }
 
-// Enqueue the whole step for one matrix.
-fp4_status run_one(const DeviceInfo* d, const float* G, float* out, int64_t m, int64_t n, int steps,
-                   const fp4_ns_params* p, uint8_t* ws, bool clear_status, cudaStream_t st) {
+// Everything the launches need to know about one matrix of a call.
+struct MatrixCtx {
   NsPlan pl;
-  fp4_status rc = make_plan(m, n, steps, p, d->sms, &pl);
+  const float* G;
+  float* out;
+  float* X;        // FP32 X in the work orientation: `out` itself, or the workspace when tall
+  uint8_t* ws;     // this matrix's workspace
+  GemmProblem g1, g2, g3[2];  // g3[cur]: reads qXt[cur], writes qXt[cur ^ 1]
+};
+
+fp4_status prepare_matrix(const DeviceInfo* d, const float* G, float* out, int64_t m, int64_t n, int steps,
+                          const fp4_ns_params* p, uint8_t* ws, MatrixCtx* c) {
+  fp4_status rc = make_plan(m, n, steps, p, d->sms, &c->pl);
   if (rc != FP4_OK) return rc;
-  const fp4_ws_layout& L = pl.lay;
-  const int64_t s = pl.s, l = pl.l;
+  const fp4_ws_layout& L = c->pl.lay;
+  const int64_t s = c->pl.s, l = c->pl.l;
+  c->G = G; c->out = out; c->ws = ws;
+  c->X = c->pl.tall ? reinterpret_cast<float*>(ws + L.X) : out;
+  if (steps == 0) return FP4_OK;
   float abc[3] = {p->a, p->b, p->c};
   if (std::isnan(p->a)) coeffs(m, n, abc);
+  CUtensorMap tm_qX, tm_qXt[2], tm_qA, tm_qB, tm_A, tm_X;
+  bool ok = make_codes_map(d, &tm_qX, ws + L.qX_codes, s, l / 2) &&
+            make_codes_map(d, &tm_qXt[0], ws + L.qXt_codes[0], l, s / 2) &&
+            make_codes_map(d, &tm_qXt[1], ws + L.qXt_codes[1], l, s / 2) &&
+            make_codes_map(d, &tm_qA, ws + L.qA_codes, s, s / 2) &&
+            make_codes_map(d, &tm_qB, ws + L.qB_codes, s, s / 2) &&
+            make_f32_map(d, &tm_A, ws + L.A, s, s) && make_f32_map(d, &tm_X, c->X, s, l);
+  if (!ok) return FP4_ERR_CUDA;
+  GemmProblem base;
+  memset(&base, 0, sizeof(base));
+  base.scalars = reinterpret_cast<float*>(ws + L.scalars);
+  base.ca = abc[0]; base.cb = abc[1]; base.cc = abc[2];
+  // G1: A = qX qX^T (upper-triangle tiles), qA in both triangles
+  c->g1 = base;
+  c->g1.tmA = c->g1.tmB = tm_qX; c->g1.tmAux = c->g1.tmOut = tm_A;
+  c->g1.sfa = c->g1.sfb = ws + L.qX_scales;
+  c->g1.rq_codes = c->g1.cq_codes = ws + L.qA_codes; c->g1.rq_sf = c->g1.cq_sf = ws + L.qA_scales;
+  // G2: B = bA + c qA qA^T, qB in both triangles
+  c->g2 = base;
+  c->g2.tmA = c->g2.tmB = tm_qA; c->g2.tmAux = c->g2.tmOut = tm_A;
+  c->g2.sfa = c->g2.sfb = ws + L.qA_scales;
+  c->g2.rq_codes = c->g2.cq_codes = ws + L.qB_codes; c->g2.rq_sf = c->g2.cq_sf = ws + L.qB_scales;
+  // G3: X+ = aX + qB qXt^T in place on X; new operand copies
+  for (int cur = 0; cur < 2; ++cur) {
+    GemmProblem& g = c->g3[cur];
+    g = base;
+    g.tmA = tm_qB; g.tmB = tm_qXt[cur]; g.tmAux = g.tmOut = tm_X;
+    g.sfa = ws + L.qB_scales; g.sfb = ws + L.qXt_scales[cur];
+    g.rq_codes = ws + L.qX_codes; g.rq_sf = ws + L.qX_scales;
+    g.cq_codes = ws + L.qXt_codes[cur ^ 1]; g.cq_sf = ws + L.qXt_scales[cur ^ 1];
+  }
+  return FP4_OK;
+}
+
+constexpr int kPackMax = 6;
+struct ProblemPack { GemmProblem p[kPackMax]; };
+
+// Copies problem descriptions from kernel parameters into a device table (the tables of a
+// batched call are filled this way so that the call stays asynchronous).
+__global__ void k_write_problems(GemmProblem* dst, const __grid_constant__ ProblemPack pack, int n) {
+  const uint4* src = reinterpret_cast<const uint4*>(&pack);
+  uint4* out = reinterpret_cast<uint4*>(dst);
+  const int words = n * (int)(sizeof(GemmProblem) / 16);
+  for (int i = threadIdx.x; i < words; i += blockDim.x) out[i] = src[i];
+}
+
+// Enqueue the whole step for a group of matrices of one shape (s, l): the prologue per matrix,
+// then every Newton-Schulz stage as one launch over all matrices of the group.
+// table: device memory for 4 * count problems (unused when count == 1).
+fp4_status run_group(const DeviceInfo* d, MatrixCtx* mats, int count, int steps, const fp4_ns_params* p,
+                     uint32_t* status, GemmProblem* table, bool clear_first_status, cudaStream_t st) {
   const bool keep = (p->flags & FP4_FLAG_KEEP_OPERANDS) != 0;
-
-  // X lives in `out` unless the input is tall (then it is transposed back at the end)
-  float* X = pl.tall ? reinterpret_cast<float*>(ws + L.X) : out;
-  float* scalars = reinterpret_cast<float*>(ws + L.scalars);
-  uint32_t* status = reinterpret_cast<uint32_t*>(ws + L.header);
-
-  if (launch_prologue(G, m, n, pl, ws, X, steps > 0 || keep, clear_status, st) != cudaSuccess) return FP4_ERR_CUDA;
-
+  const NsPlan& pl0 = mats[0].pl;
+  const int64_t s = pl0.s, l = pl0.l;
+  for (int i = 0; i < count; ++i) {
+    MatrixCtx& c = mats[i];
+    if (launch_prologue(c.G, c.pl.m, c.pl.n, c.pl, c.ws, c.X, steps > 0 || keep, clear_first_status && i == 0, st) !=
+        cudaSuccess)
+      return FP4_ERR_CUDA;
+  }
   if (steps > 0) {
-    CUtensorMap tm_qX, tm_qXt[2], tm_qA, tm_qB, tm_A, tm_X;
-    bool ok = make_codes_map(d, &tm_qX, ws + L.qX_codes, s, l / 2) &&
-              make_codes_map(d, &tm_qXt[0], ws + L.qXt_codes[0], l, s / 2) &&
-              make_codes_map(d, &tm_qXt[1], ws + L.qXt_codes[1], l, s / 2) &&
-              make_codes_map(d, &tm_qA, ws + L.qA_codes, s, s / 2) &&
-              make_codes_map(d, &tm_qB, ws + L.qB_codes, s, s / 2) &&
-              make_f32_map(d, &tm_A, ws + L.A, s, s) && make_f32_map(d, &tm_X, X, s, l);
-    if (!ok) return FP4_ERR_CUDA;
-
-    GemmArgs base;
+    const GemmProblem* tabs[4] = {nullptr, nullptr, nullptr, nullptr};
+    if (count > 1) {
+      for (int kind = 0; kind < 4; ++kind) {
+        GemmProblem* dst = table + (size_t)kind * count;
+        tabs[kind] = dst;
+        for (int i0 = 0; i0 < count; i0 += kPackMax) {
+          ProblemPack pack;
+          const int nn = count - i0 < kPackMax ? count - i0 : kPackMax;
+          for (int j = 0; j < nn; ++j) {
+            const MatrixCtx& c = mats[i0 + j];
+            pack.p[j] = kind == 0 ? c.g1 : kind == 1 ? c.g2 : c.g3[kind - 2];
+          }
+          for (int j = nn; j < kPackMax; ++j) pack.p[j] = pack.p[0];
+          count_launches(1);
+          k_write_problems<<<1, 128, 0, st>>>(dst + i0, pack, nn);
+        }
+      }
+      if (cudaGetLastError() != cudaSuccess) return FP4_ERR_CUDA;
+    }
+    GemmLaunch base;
     memset(&base, 0, sizeof(base));
-    base.scalars = scalars;
-    base.ix = pl.ix;
-    base.ca = abc[0]; base.cb = abc[1]; base.cc = abc[2];
+    base.num_problems = count;
+    base.ix = pl0.ix;
     base.l_cols = (float)l;
     base.status = status;
-
     for (int k = 0; k < steps; ++k) {
-      const int cur = k & 1, nxt = cur ^ 1;
+      const int cur = k & 1;
       const bool last = (k == steps - 1);
-      // G1: A = qX qX^T (upper-triangle tiles), qA in both triangles
-      GemmArgs a1 = base;
-      a1.iter = k; a1.K = (int)l; a1.tiles_m = a1.tiles_n = (int)(s / 128); a1.symmetric = 1;
-      a1.sfa = a1.sfb = ws + L.qX_scales;
-      a1.rq_codes = a1.cq_codes = ws + L.qA_codes; a1.rq_sf = a1.cq_sf = ws + L.qA_scales;
-      a1.rq_K = a1.cq_K = (int)s; a1.write_q = 1;
+      GemmLaunch L1 = base;
+      L1.iter = k; L1.K = (int)l; L1.tiles_m = L1.tiles_n = (int)(s / 128); L1.symmetric = 1;
+      L1.rq_K = L1.cq_K = (int)s; L1.write_q = 1;
       {
         ProfScope ps(FP4_PROF_G1, st);
-        if (launch_gemm(kG1, tm_qX, tm_qX, tm_A, tm_A, a1, d->sms, st) != cudaSuccess) return FP4_ERR_CUDA;
+        if (launch_gemm(kG1, count == 1 ? &mats[0].g1 : nullptr, tabs[0], L1, d->sms, st) != cudaSuccess)
+          return FP4_ERR_CUDA;
       }
-      // G2: B = bA + c qA qA^T, qB in both triangles
-      GemmArgs a2 = base;
-      a2.iter = k; a2.K = (int)s; a2.tiles_m = a2.tiles_n = (int)(s / 128); a2.symmetric = 1;
-      a2.sfa = a2.sfb = ws + L.qA_scales;
-      a2.rq_codes = a2.cq_codes = ws + L.qB_codes; a2.rq_sf = a2.cq_sf = ws + L.qB_scales;
-      a2.rq_K = a2.cq_K = (int)s; a2.write_q = 1;
+      GemmLaunch L2 = L1;
+      L2.K = (int)s;
       {
         ProfScope ps(FP4_PROF_G2, st);
-        if (launch_gemm(kG2, tm_qA, tm_qA, tm_A, tm_A, a2, d->sms, st) != cudaSuccess) return FP4_ERR_CUDA;
+        if (launch_gemm(kG2, count == 1 ? &mats[0].g2 : nullptr, tabs[1], L2, d->sms, st) != cudaSuccess)
+          return FP4_ERR_CUDA;
       }
-      // G3: X+ = aX + qB qXt^T, in place on X; new operand copies unless this is the last iteration
-      GemmArgs a3 = base;
-      a3.iter = k; a3.K = (int)s; a3.tiles_m = (int)(s / 128); a3.tiles_n = (int)(l / 128); a3.symmetric = 0;
-      a3.sfa = ws + L.qB_scales; a3.sfb = ws + L.qXt_scales[cur];
-      a3.rq_codes = ws + L.qX_codes; a3.rq_sf = ws + L.qX_scales; a3.rq_K = (int)l;
-      a3.cq_codes = ws + L.qXt_codes[nxt]; a3.cq_sf = ws + L.qXt_scales[nxt]; a3.cq_K = (int)s;
-      a3.write_q = (!last || keep) ? 1 : 0;
+      GemmLaunch L3 = base;
+      L3.iter = k; L3.K = (int)s; L3.tiles_m = (int)(s / 128); L3.tiles_n = (int)(l / 128); L3.symmetric = 0;
+      L3.rq_K = (int)l; L3.cq_K = (int)s;
+      L3.write_q = (!last || keep) ? 1 : 0;
       {
         ProfScope ps(FP4_PROF_G3, st);
-        if (launch_gemm(kG3, tm_qB, tm_qXt[cur], tm_X, tm_X, a3, d->sms, st) != cudaSuccess) return FP4_ERR_CUDA;
+        if (launch_gemm(kG3, count == 1 ? &mats[0].g3[cur] : nullptr, tabs[2 + cur], L3, d->sms, st) != cudaSuccess)
+          return FP4_ERR_CUDA;
       }
     }
   }
-  if (pl.tall) {
-    ProfScope ps(FP4_PROF_TRANSPOSE, st);
-    if (launch_transpose_out(X, s, l, out, st) != cudaSuccess) return FP4_ERR_CUDA;
+  for (int i = 0; i < count; ++i) {
+    if (mats[i].pl.tall) {
+      ProfScope ps(FP4_PROF_TRANSPOSE, st);
+      if (launch_transpose_out(mats[i].X, s, l, mats[i].out, st) != cudaSuccess) return FP4_ERR_CUDA;
+    }
   }
   return FP4_OK;
+}
+
+// Enqueue the whole step for one matrix.
+fp4_status run_one(const DeviceInfo* d, const float* G, float* out, int64_t m, int64_t n, int steps,
+                   const fp4_ns_params* p, uint8_t* ws, bool clear_status, cudaStream_t st) {
+  MatrixCtx c;
+  fp4_status rc = prepare_matrix(d, G, out, m, n, steps, p, ws, &c);
+  if (rc != FP4_OK) return rc;
+  return run_group(d, &c, 1, steps, p, reinterpret_cast<uint32_t*>(ws + c.pl.lay.header), nullptr, clear_status, st);
 }
 
 fp4_status check_common(const DeviceInfo** d) {
@@ -344,6 +421,8 @@ fp4_status fp4_root_ns(const float* G, float* out, int64_t m, int64_t n, int ste
   return run_one(d, G, out, m, n, steps, p, static_cast<uint8_t*>(ws), true, stream);
 }
 
+// Batched workspace: one workspace per matrix (the stages of equal-shape matrices run in
+// lockstep, so none can be shared), then the problem tables.
 size_t fp4_root_ns_batched_workspace_bytes(int count, const int64_t* m, const int64_t* n, int steps,
                                            uint32_t flags) {
   if (count <= 0 || !m || !n) return 0;
@@ -351,8 +430,9 @@ size_t fp4_root_ns_batched_workspace_bytes(int count, const int64_t* m, const in
   for (int i = 0; i < count; ++i) {
     size_t b = fp4_root_ns_workspace_bytes(m[i], n[i], steps, flags);
     if (b == 0) return 0;
-    if (b > need) need = b;
+    need += align_up(b, 1024);
   }
+  need += align_up((size_t)4 * count * sizeof(GemmProblem), 1024);
   return need;
 }
 
@@ -375,11 +455,39 @@ fp4_status fp4_root_ns_batched(int count, const float* const* G, float* const* o
   const DeviceInfo* d;
   fp4_status rc = check_common(&d);
   if (rc != FP4_OK) return rc;
-  // Matrix after matrix on the one stream: the working set of a matrix (operands, A, X)
-  // stays in L2 across its stages, and the shared workspace is reused.
+
+  uint8_t* base = static_cast<uint8_t*>(ws);
+  std::vector<MatrixCtx> ctx((size_t)count);
+  size_t off = 0;
   for (int i = 0; i < count; ++i) {
-    rc = run_one(d, G[i], out[i], m[i], n[i], steps, p, static_cast<uint8_t*>(ws), i == 0, stream);
+    rc = prepare_matrix(d, G[i], out[i], m[i], n[i], steps, p, base + off, &ctx[(size_t)i]);
     if (rc != FP4_OK) return rc;
+    off += align_up(ctx[(size_t)i].pl.lay.total, 1024);
+  }
+  GemmProblem* table = reinterpret_cast<GemmProblem*>(base + off);
+  uint32_t* status = reinterpret_cast<uint32_t*>(base);  // header of the first matrix
+
+  // Matrices of one shape form a group whose stages run as single launches over all of
+  // them (many tiles per launch: no idle SMs in a last partial wave, the two CTAs of an SM
+  // fall out of step so that main loops and epilogues overlap).  A group is split when it
+  // exceeds max_group matrices, which bounds the working set competing for L2.
+  const int cap = p->max_group > 0 ? (int)p->max_group : kDefaultMaxGroup;
+  std::vector<char> done((size_t)count, 0);
+  std::vector<MatrixCtx> group;
+  bool first = true;
+  for (int i = 0; i < count; ++i) {
+    if (done[(size_t)i]) continue;
+    group.clear();
+    for (int j = i; j < count && (int)group.size() < cap; ++j) {
+      if (done[(size_t)j]) continue;
+      if (ctx[(size_t)j].pl.s == ctx[(size_t)i].pl.s && ctx[(size_t)j].pl.l == ctx[(size_t)i].pl.l) {
+        group.push_back(ctx[(size_t)j]);
+        done[(size_t)j] = 1;
+      }
+    }
+    rc = run_group(d, group.data(), (int)group.size(), steps, p, status, table, first, stream);
+    if (rc != FP4_OK) return rc;
+    first = false;
   }
   return FP4_OK;
 }
@@ -403,17 +511,20 @@ fp4_status fp4_gemm_nt(const uint8_t* a_codes, const uint8_t* a_scales, float a_
   const DeviceInfo* d;
   fp4_status rc = check_common(&d);
   if (rc != FP4_OK) return rc;
-  CUtensorMap tmA, tmB, tmD;
-  if (!make_codes_map(d, &tmA, a_codes, M, K / 2) || !make_codes_map(d, &tmB, b_codes, N, K / 2) ||
-      !make_f32_map(d, &tmD, D, M, N))
+  GemmProblem pr;
+  memset(&pr, 0, sizeof(pr));
+  if (!make_codes_map(d, &pr.tmA, a_codes, M, K / 2) || !make_codes_map(d, &pr.tmB, b_codes, N, K / 2) ||
+      !make_f32_map(d, &pr.tmOut, D, M, N))
     return FP4_ERR_CUDA;
-  GemmArgs a;
-  memset(&a, 0, sizeof(a));
-  a.sfa = a_scales; a.sfb = b_scales;
-  a.K = (int)K; a.tiles_m = (int)(M / 128); a.tiles_n = (int)(N / 128);
-  a.sg_a = a_tensor_scale; a.sg_b = b_tensor_scale;
-  a.status = device_status;
-  return launch_gemm(kPlain, tmA, tmB, tmD, tmD, a, d->sms, stream) == cudaSuccess ? FP4_OK : FP4_ERR_CUDA;
+  pr.tmAux = pr.tmOut;
+  pr.sfa = a_scales; pr.sfb = b_scales;
+  pr.sg_a = a_tensor_scale; pr.sg_b = b_tensor_scale;
+  GemmLaunch L;
+  memset(&L, 0, sizeof(L));
+  L.num_problems = 1;
+  L.K = (int)K; L.tiles_m = (int)(M / 128); L.tiles_n = (int)(N / 128);
+  L.status = device_status;
+  return launch_gemm(kPlain, &pr, nullptr, L, d->sms, stream) == cudaSuccess ? FP4_OK : FP4_ERR_CUDA;
 }
 
 }  // extern "C"
