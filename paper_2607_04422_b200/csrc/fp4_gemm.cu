@@ -14,30 +14,37 @@
 //
 // One CTA owns 128 x 128 output tiles.  Warp roles: 0 = TMA producer of operand stages,
 // 1 = MMA issuer (one thread) and TMEM owner, 2 = TMA producer of the FP32 tile the
-// epilogue combines with, 3 = TMA-store issuer, 4..7 = drain (TMEM lane quadrant =
-// warp % 4), 8..11 = finish.  The epilogue is a pipeline over a ring of 8 KB chunk buffers
+// epilogue combines with, 3 = TMA-store issuer, 4..11 = drain (TMEM lane quadrant =
+// warp % 4; two sets of four split a tile's columns), 12..19 = finish.  The epilogue is a pipeline over a ring of 8 KB chunk buffers
 // (16 FP32 columns x 128 rows) connected by mbarriers only: TMA load of the FP32 tile
 // chunk -> drain (combine, quantise along the row, write the result chunk in place) ->
-// TMA store and, concurrently, finish (quantise down the columns) -> slot free.  Two CTAs
-// share an SM, so one CTA's epilogue also overlaps the other's main loop.
+// TMA store and, concurrently, finish (quantise down the columns) -> slot free.  One
+// persistent CTA per SM with three accumulator buffers in TMEM: the MMAs of the next tiles
+// run while a tile is drained, so the operand ring never idles.
 #include "fp4_kernels.h"
 
 namespace fp4 {
 
 namespace {
 
-constexpr int BM = 128, BN = 128, BK = 128;
+#ifndef FP4_BK
+#define FP4_BK 256
+#endif
 #ifndef FP4_STAGES
-#define FP4_STAGES 3
+#define FP4_STAGES 4
 #endif
 #ifndef FP4_RING
-#define FP4_RING 7
+#define FP4_RING 9
 #endif
+constexpr int BM = 128, BN = 128, BK = FP4_BK;  // BK elements of K per stage: 64- or 128-byte operand rows
+static_assert(BK == 128 || BK == 256, "operand rows of a stage are one TMA swizzle span");
+constexpr int KSTEPS = BK / 64;               // MMAs (K = 64) per stage
+constexpr uint32_t OPER_SWIZZLE = (BK == 256) ? 2u : 4u;  // UMMA layout type: 128- or 64-byte swizzle
+constexpr uint32_t OPER_SBO = 8 * (BK / 2);   // bytes between 8-row groups of an operand tile
 constexpr int STAGES = FP4_STAGES;          // operand stages of the main loop
 constexpr int RING = FP4_RING;              // FP32 chunk buffers of the epilogue
-constexpr int OPER_BYTES = BM * BK / 2;      // 8192: one operand tile of a stage (64-byte rows)
-constexpr int SF_BYTES = 2 * 512;            // two scale atoms (128 rows x 8 blocks) per operand and stage
-constexpr uint32_t STAGE_TX = 2 * OPER_BYTES + 2 * SF_BYTES;
+constexpr int OPER_BYTES = BM * BK / 2;      // one operand tile of a stage
+constexpr int SF_BYTES = KSTEPS * 512;       // one scale atom (128 rows x 4 blocks) per MMA, operand and stage
 constexpr int CHUNK = 16;                    // FP32 columns per epilogue step
 constexpr int CHUNK_BYTES = BM * CHUNK * 4;  // 8192
 constexpr int NCHUNK = BN / CHUNK;
@@ -49,13 +56,18 @@ constexpr int OFF_SFB = OFF_SFA + STAGES * SF_BYTES;
 constexpr int OFF_RING = OFF_SFB + STAGES * SF_BYTES;
 constexpr int OFF_BAR = OFF_RING + RING * CHUNK_BYTES;
 constexpr int SMEM_BYTES = OFF_BAR + 512 + 1024;  // + slack to align the base to 1024
-static_assert(2 * (SMEM_BYTES + 1024) <= 233472, "two CTAs must fit in one SM's shared memory");
+static_assert(SMEM_BYTES <= 232448, "one CTA per SM: at most 227 KB of dynamic shared memory");
 
 // warps: 0 operand producer, 1 MMA issuer, 2 producer of the FP32 tile, 3 TMA-store issuer,
-// 4..7 drain (TMEM -> registers -> ring), 8..11 finish (transposed quantisation from the ring)
-constexpr int NTHREADS = 384;
-constexpr uint32_t TMEM_COLS = 256;
-constexpr uint32_t TMEM_SF_COL = 128;  // scale factors: 16 columns per stage after the accumulator
+// 4..11 drain (TMEM -> registers -> ring; warps 4..7 take columns 0..63 of a tile, 8..11
+// columns 64..127), 12..19 finish (transposed quantisation from the ring, same split)
+constexpr int NTHREADS = 640;
+constexpr int NACC = 3;                  // accumulator buffers: the MMAs of the next tiles run during a drain
+constexpr uint32_t TMEM_COLS = 512;
+constexpr uint32_t TMEM_SF_COL = 384;    // scale factors after the accumulators
+constexpr uint32_t SF_COLS = KSTEPS * 8; // per stage: 4 columns per MMA for each operand
+static_assert(NACC * BN + STAGES * SF_COLS <= 512, "tensor memory columns");
+constexpr int HALF_CHUNKS = NCHUNK / 2;
 
 // instruction descriptor: E2M1 x E2M1, UE4M3 scales, both operands K-major, M = N = 128
 constexpr uint32_t IDESC = (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | (0u << 23) |
@@ -64,11 +76,11 @@ constexpr uint32_t IDESC = (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) 
 struct Barriers {
   uint64_t full[STAGES];     // operand stage landed (TMA bytes)
   uint64_t empty[STAGES];    // operand stage consumed (MMA commit)
-  uint64_t acc_full;         // accumulator complete (MMA commit)
-  uint64_t acc_empty;        // accumulator drained (4 drain warps)
+  uint64_t acc_full[NACC];   // accumulator complete (MMA commit)
+  uint64_t acc_empty[NACC];  // accumulator drained (8 drain warps)
   uint64_t aux_full[RING];   // FP32 tile chunk landed in a ring slot (TMA bytes)
-  uint64_t v_ready[RING];    // result chunk written to the slot (4 drain warps)
-  uint64_t slot_free[RING];  // slot read by everyone: 4 finish warps + the store warp
+  uint64_t v_ready[RING];    // result chunk written to the slot (the 4 drain warps of its half)
+  uint64_t slot_free[RING];  // slot read by everyone: the 4 finish warps of its half + the store warp
   uint32_t tmem_base;
   uint32_t abort_flag;
 };
@@ -152,7 +164,7 @@ __device__ __forceinline__ void epilogue_scalars(const GemmProblem& pr, const Ge
 }
 
 template <int MODE>
-__global__ void __launch_bounds__(NTHREADS, 2)
+__global__ void __launch_bounds__(NTHREADS, 1)
 k_gemm(const __grid_constant__ GemmProblem single, const GemmProblem* __restrict__ table, const GemmLaunch args) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -166,7 +178,7 @@ k_gemm(const __grid_constant__ GemmProblem single, const GemmProblem* __restrict
 #ifdef FP4_DEBUG_ONE_KBLOCK
   const int num_kb = 1;  // timing experiments only: epilogue cost without the main loop
 #else
-  const int num_kb = args.K / BK;
+  const int num_kb = (args.K + BK - 1) / BK;  // K is a multiple of 128: the last stage may be half full
 #endif
   constexpr bool HAS_AUX = (MODE == kG2 || MODE == kG3);
   constexpr bool STORE_F32 = (MODE == kPlain || MODE == kG1 || MODE == kG3);
@@ -174,8 +186,7 @@ k_gemm(const __grid_constant__ GemmProblem single, const GemmProblem* __restrict
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < STAGES; ++i) { mbar_init(&bars->full[i], 1); mbar_init(&bars->empty[i], 1); }
-    mbar_init(&bars->acc_full, 1);
-    mbar_init(&bars->acc_empty, 4);
+    for (int i = 0; i < NACC; ++i) { mbar_init(&bars->acc_full[i], 1); mbar_init(&bars->acc_empty[i], 8); }
     for (int i = 0; i < RING; ++i) {
       mbar_init(&bars->aux_full[i], 1);
       mbar_init(&bars->v_ready[i], 4);
@@ -205,11 +216,15 @@ k_gemm(const __grid_constant__ GemmProblem single, const GemmProblem* __restrict
         const uint8_t* sfb = pr->sfb + (size_t)tj * (args.K / 64) * 512;
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!wait_bar(&bars->empty[st], ph ^ 1, abort_flag)) { ok = false; break; }
-          mbar_expect_tx(&bars->full[st], STAGE_TX);
+          // a half-full last stage: the operand boxes are zero-filled beyond K (and still
+          // credit their full size), only the scale atoms that exist are fetched
+          const int kvalid = args.K - kb * BK < BK ? args.K - kb * BK : BK;
+          const uint32_t sf_bytes = (uint32_t)(kvalid / 64) * 512;
+          mbar_expect_tx(&bars->full[st], 2 * OPER_BYTES + 2 * sf_bytes);
           tma_load_2d(smem + OFF_A + st * OPER_BYTES, &pr->tmA, kb * (BK / 2), ti * BM, &bars->full[st]);
           tma_load_2d(smem + OFF_B + st * OPER_BYTES, &pr->tmB, kb * (BK / 2), tj * BN, &bars->full[st]);
-          bulk_load_1d(smem + OFF_SFA + st * SF_BYTES, sfa + (size_t)kb * SF_BYTES, SF_BYTES, &bars->full[st]);
-          bulk_load_1d(smem + OFF_SFB + st * SF_BYTES, sfb + (size_t)kb * SF_BYTES, SF_BYTES, &bars->full[st]);
+          bulk_load_1d(smem + OFF_SFA + st * SF_BYTES, sfa + (size_t)kb * SF_BYTES, sf_bytes, &bars->full[st]);
+          bulk_load_1d(smem + OFF_SFB + st * SF_BYTES, sfb + (size_t)kb * SF_BYTES, sf_bytes, &bars->full[st]);
           if (++st == STAGES) { st = 0; ph ^= 1; }
         }
       }
@@ -217,33 +232,37 @@ k_gemm(const __grid_constant__ GemmProblem single, const GemmProblem* __restrict
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
     if (elect_one()) {
-      int st = 0; uint32_t ph = 0, acc_ph = 0; bool ok = true;
-      for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
-        if (!wait_bar(&bars->acc_empty, acc_ph ^ 1, abort_flag)) { ok = false; break; }
+      int st = 0; uint32_t ph = 0, seq = 0; bool ok = true;
+      for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++seq) {
+        const uint32_t ab = seq % NACC, ause = seq / NACC;
+        if (!wait_bar(&bars->acc_empty[ab], (ause & 1) ^ 1, abort_flag)) { ok = false; break; }
         tc_fence_after();
+        const uint32_t d_tmem = tmem_base + ab * BN;
         for (int kb = 0; kb < num_kb; ++kb) {
           if (!wait_bar(&bars->full[st], ph, abort_flag)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t sf_t = tmem_base + TMEM_SF_COL + st * 16;
+          const uint32_t sf_t = tmem_base + TMEM_SF_COL + st * SF_COLS;
+          const int ksteps = (args.K - kb * BK < BK ? args.K - kb * BK : BK) / 64;
 #pragma unroll
-          for (int a = 0; a < 2; ++a) {
-            tc_cp_sf(sf_t + a * 4, umma_desc(smem_u32(smem + OFF_SFA + st * SF_BYTES + a * 512), 128, 0));
-            tc_cp_sf(sf_t + 8 + a * 4, umma_desc(smem_u32(smem + OFF_SFB + st * SF_BYTES + a * 512), 128, 0));
+          for (int a = 0; a < KSTEPS; ++a) {
+            if (a < ksteps) tc_cp_sf(sf_t + a * 4, umma_desc(smem_u32(smem + OFF_SFA + st * SF_BYTES + a * 512), 128, 0));
+            if (a < ksteps) tc_cp_sf(sf_t + KSTEPS * 4 + a * 4,
+                                     umma_desc(smem_u32(smem + OFF_SFB + st * SF_BYTES + a * 512), 128, 0));
           }
-          const uint64_t adesc = umma_desc(smem_u32(smem + OFF_A + st * OPER_BYTES), 512, 4);
-          const uint64_t bdesc = umma_desc(smem_u32(smem + OFF_B + st * OPER_BYTES), 512, 4);
+          const uint64_t adesc = umma_desc(smem_u32(smem + OFF_A + st * OPER_BYTES), OPER_SBO, OPER_SWIZZLE);
+          const uint64_t bdesc = umma_desc(smem_u32(smem + OFF_B + st * OPER_BYTES), OPER_SBO, OPER_SWIZZLE);
 #pragma unroll
-          for (int k = 0; k < 2; ++k) {
+          for (int k = 0; k < KSTEPS; ++k) {
             // 64 elements = 32 bytes further along K: +2 in the 16-byte address field
-            tc_mma_nvf4(tmem_base, adesc + 2 * k, bdesc + 2 * k, IDESC, sf_t + k * 4, sf_t + 8 + k * 4,
-                        (kb | k) != 0 ? 1u : 0u);
+            if (k < ksteps)
+              tc_mma_nvf4(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC, sf_t + k * 4, sf_t + KSTEPS * 4 + k * 4,
+                          (kb | k) != 0 ? 1u : 0u);
           }
           tc_commit(&bars->empty[st]);
           if (++st == STAGES) { st = 0; ph ^= 1; }
         }
         if (!ok) break;
-        tc_commit(&bars->acc_full);
-        acc_ph ^= 1;
+        tc_commit(&bars->acc_full[ab]);
       }
     }
   } else if (warp == 2) {
@@ -297,10 +316,12 @@ k_gemm(const __grid_constant__ GemmProblem single, const GemmProblem* __restrict
         bulk_wait_all<0>();
       }
     }
-  } else if (warp < 8) {
+  } else if (warp < 12) {
     // ------------------------------------------------------------ drain warps
     // TMEM -> registers (thread = row), combine with the FP32 tile, quantise the blocks
-    // that run along the row, write the result chunk into the ring slot.
+    // that run along the row, write the result chunk into the ring slot.  Warps 4..7 take
+    // the chunks of columns 0..63, warps 8..11 those of columns 64..127.
+    const int half = (warp - 4) >> 2;
     const int quad = warp & 3;
     const int row = quad * 32 + lane;
     float scale = 0.0f, sg_out = 1.0f, six_sg = 6.0f;
@@ -310,10 +331,10 @@ k_gemm(const __grid_constant__ GemmProblem single, const GemmProblem* __restrict
     const int sw = (row >> 1) & 3;
     const uint32_t tm_lane = tmem_base + ((uint32_t)(quad * 32) << 16);
 
-    uint32_t acc_ph = 0, it = 0;
+    uint32_t seq = 0;
     float amax = 0.0f;
     bool ok = true;
-    for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+    for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++seq) {
       int p, ti, tj;
       decode_tile(t, args, tiles_per_problem, p, ti, tj);
       if (p != cur_p) {
@@ -336,15 +357,17 @@ k_gemm(const __grid_constant__ GemmProblem single, const GemmProblem* __restrict
       }
       const bool mirror = do_q && (MODE == kG3 || (args.symmetric && ti != tj));
       // give-up decisions are made warp-uniform: the TMEM loads below are warp-collective
-      ok = __all_sync(0xffffffffu, wait_bar(&bars->acc_full, acc_ph, abort_flag));
-      acc_ph ^= 1;
+      const uint32_t ab = seq % NACC, ause = seq / NACC;
+      ok = __all_sync(0xffffffffu, wait_bar(&bars->acc_full[ab], ause & 1, abort_flag));
       if (!ok) break;
       tc_fence_after();
       const int64_t grow = (int64_t)ti * BM + row;
+      const uint32_t tm_acc = tm_lane + ab * BN;
       uint32_t sfw = 0;
       uint32_t acc[16];
-      tc_ld16_issue(tm_lane, acc);
-      for (int c = 0; c < NCHUNK; ++c, ++it) {
+      tc_ld16_issue(tm_acc + half * HALF_CHUNKS * CHUNK, acc);
+      for (int c = half * HALF_CHUNKS; c < (half + 1) * HALF_CHUNKS; ++c) {
+        const uint32_t it = seq * NCHUNK + c;
         const int b = it % RING;
         const uint32_t use = it / RING;
         uint8_t* slot_row = smem + OFF_RING + b * CHUNK_BYTES + row * 64;
@@ -371,12 +394,12 @@ k_gemm(const __grid_constant__ GemmProblem single, const GemmProblem* __restrict
           for (int i = 0; i < 16; ++i) v[i] = __fmul_rn(__uint_as_float(acc[i]), scale);
         }
         // the next chunk's accumulator columns are fetched while this chunk is finished
-        if (c + 1 < NCHUNK) {
-          tc_ld16_issue(tm_lane + (c + 1) * CHUNK, acc);
+        if (c + 1 < (half + 1) * HALF_CHUNKS) {
+          tc_ld16_issue(tm_acc + (c + 1) * CHUNK, acc);
         } else {
           tc_fence_before();
           __syncwarp();
-          if (lane == 0) mbar_arrive(&bars->acc_empty);  // the next tile's MMAs may start
+          if (lane == 0) mbar_arrive(&bars->acc_empty[ab]);  // this warp is done with the accumulator
         }
         if (STORE_F32 || mirror) {
 #pragma unroll
@@ -416,14 +439,15 @@ k_gemm(const __grid_constant__ GemmProblem single, const GemmProblem* __restrict
     // ------------------------------------------------------------ finish warps
     // Blocks of 16 that run down this tile's rows (the transposed operand copy in G3, the
     // mirrored triangle in G1/G2): thread = (column cc of the chunk, row group g).
-    const int et = threadIdx.x - 256;
+    const int half = (warp - 12) >> 2;
+    const int et = ((warp - 12) & 3) * 32 + lane;
     const int cc = et & 15, g = et >> 4;
     float scale, sg_out = 1.0f, six_sg = 6.0f;
     const GemmProblem* pr = nullptr;
     int cur_p = -1;
-    uint32_t it = 0;
+    uint32_t seq = 0;
     bool ok = true;
-    for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+    for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++seq) {
       int p, ti, tj;
       decode_tile(t, args, tiles_per_problem, p, ti, tj);
       if (p != cur_p) {
@@ -433,7 +457,8 @@ k_gemm(const __grid_constant__ GemmProblem single, const GemmProblem* __restrict
         six_sg = __fmul_rn(6.0f, sg_out);
       }
       const bool mirror = do_q && (MODE == kG3 || (args.symmetric && ti != tj));
-      for (int c = 0; c < NCHUNK; ++c, ++it) {
+      for (int c = half * HALF_CHUNKS; c < (half + 1) * HALF_CHUNKS; ++c) {
+        const uint32_t it = seq * NCHUNK + c;
         const int b = it % RING;
         const uint32_t use = it / RING;
         ok = __all_sync(0xffffffffu, wait_bar(&bars->v_ready[b], use & 1, abort_flag));
@@ -476,7 +501,7 @@ cudaError_t launch_mode(const GemmProblem* single, const GemmProblem* table, con
                         cudaStream_t st) {
   const int tpp = L.symmetric ? L.tiles_n * (L.tiles_n + 1) / 2 : L.tiles_m * L.tiles_n;
   const int num_tiles = tpp * L.num_problems;
-  int grid = 2 * sms;
+  int grid = sms;
   if (grid > num_tiles) grid = num_tiles;
   count_launches(1);
   static const GemmProblem kNone = {};
@@ -485,6 +510,8 @@ cudaError_t launch_mode(const GemmProblem* single, const GemmProblem* table, con
 }
 
 }  // namespace
+
+int gemm_stage_k() { return BK; }
 
 cudaError_t gemm_set_attributes() {
   cudaError_t e;

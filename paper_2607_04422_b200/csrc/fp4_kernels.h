@@ -97,6 +97,7 @@ cudaError_t launch_transpose_out(const float* X, int64_t s, int64_t l, float* ou
 cudaError_t prologue_set_attributes();
 
 cudaError_t gemm_set_attributes();
+int gemm_stage_k();  // elements of K per operand stage (the codes maps' box is this / 2 bytes wide)
 // single: the one problem of the launch (host copy, passed by value) when table is null;
 // table: device array of launch.num_problems problems.
 cudaError_t launch_gemm(GemmMode mode, const GemmProblem* single, const GemmProblem* table, const GemmLaunch& launch,

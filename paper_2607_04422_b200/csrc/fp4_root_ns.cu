@@ -77,14 +77,17 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 inline bool shape_ok(int64_t v) { return v >= 128 && v % 128 == 0 && v <= (1 << 20); }
 
-// 2-D map over a row-major byte matrix (NVFP4 codes): box = 64 bytes x 128 rows, 64-byte swizzle.
+// 2-D map over a row-major byte matrix (NVFP4 codes): box = one operand stage (64 or 128 bytes
+// x 128 rows), swizzled over the box width.
 bool make_codes_map(const DeviceInfo* d, CUtensorMap* tm, const void* base, int64_t rows, int64_t row_bytes) {
+  const cuuint32_t bw = (cuuint32_t)(gemm_stage_k() / 2);
   cuuint64_t dims[2] = {(cuuint64_t)row_bytes, (cuuint64_t)rows};
   cuuint64_t strides[1] = {(cuuint64_t)row_bytes};
-  cuuint32_t box[2] = {64, 128};
+  cuuint32_t box[2] = {bw, 128};
   cuuint32_t estr[2] = {1, 1};
   return d->encode(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
-                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, bw == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 // 2-D map over a row-major FP32 matrix: box = 16 columns x 128 rows, 64-byte swizzle.

@@ -198,3 +198,71 @@ def test_argument_errors():
     with pytest.raises(fp4.Fp4Error) as e:
         fp4.fp4_root_ns(G, G, 5, None, ws[1:])
     assert e.value.code == 3
+
+
+# --------------------------------------------------------------------------------------
+# Full-size configurations (the shapes bench.py times).  The oracle runs the whole matrix
+# where that takes about a minute of host time; the iteration count is reduced for the
+# largest shapes, which leaves every kernel, tile count and launch configuration unchanged.
+def _full_size_case(G, steps):
+    got, _ = run_gpu(G, steps=steps)
+    want = oracle.root_ns(G, steps=steps)
+    r = rel(got, want)
+    assert r <= TOL_OUT, r
+    assert abs(orth_err(got) - orth_err(want)) <= TOL_ORTH
+
+
+def test_config2_square_2048_lowrank_outliers():
+    _full_size_case(workloads.config2(), 5)
+
+
+def test_config3_wide_and_tall_2048x8192():
+    wide, tall = workloads.config3()
+    _full_size_case(wide, 5)
+    _full_size_case(tall, 5)
+
+
+def test_config4_shapes_3072():
+    specs = workloads.stack_3b_shapes(1)
+    name, m, n, seed = specs[0]          # Wq 3072 x 3072
+    _full_size_case(workloads.gradient_like(m, n, seed=seed), 5)
+    name, m, n, seed = specs[4]          # Wgate 3072 x 8192
+    _full_size_case(workloads.gradient_like(m, n, seed=seed), 3)
+
+
+def test_config4_batched_full_size_properties_and_sampled_stage():
+    """The 7 matrices of one decoder block at full size through fp4_root_ns_batched: the
+    batched result equals the single-matrix result bit for bit, and for a wide matrix the
+    first product A = qX qX^T is checked on sampled tiles that the oracle computes from its
+    own clip, normalisation and quantisation of the input."""
+    specs = workloads.stack_3b_shapes(1)
+    mats = [workloads.gradient_like(m, n, seed=seed) for _, m, n, seed in specs]
+    Gs = [torch.from_numpy(g).cuda() for g in mats]
+    outs = [torch.empty_like(g) for g in Gs]
+    shapes = [tuple(g.shape) for g in Gs]
+    ws = torch.empty(fp4.fp4_root_ns_batched_workspace_bytes(shapes, 5), dtype=torch.uint8, device="cuda")
+    fp4.fp4_root_ns_batched(Gs, outs, 5, None, ws)
+    assert fp4.fp4_last_device_status(ws) == 0
+    for idx in (0, 4, 6):                                   # 3072^2, 3072x8192, 8192x3072
+        single, _ = run_gpu(mats[idx], steps=5)
+        assert np.array_equal(outs[idx].cpu().numpy(), single)
+        sv = np.linalg.svd(single.astype(np.float64), compute_uv=False) if idx == 0 else None
+        assert np.isfinite(single).all()
+        if sv is not None:
+            assert sv.max() < 1.6 and sv.min() >= 0
+    # sampled tiles of A (iteration 0) for the wide 3072 x 8192 matrix
+    G = mats[4]
+    m, n = G.shape
+    flags = FP4_FLAG_KEEP_OPERANDS
+    _, ws1 = run_gpu(G, steps=1, flags=flags)
+    lay, sc, f32, q, s, l = ws_view(ws1, m, n, 1, flags)
+    X0 = oracle.root_ns(G, steps=0)
+    qx = oracle.quantize(X0)
+    assert sc[lay.idx_sg_X0] == np.float32(qx[2])
+    A = f32(lay.A, s, s)
+    rng = np.random.default_rng(0)
+    for _ in range(6):
+        i = int(rng.integers(0, s // 128)); j = int(rng.integers(i, s // 128))
+        rows = slice(128 * i, 128 * i + 128); cols = slice(128 * j, 128 * j + 128)
+        want = oracle.gemm_nt_q((qx[0][rows], qx[1][rows], qx[2]), (qx[0][cols], qx[1][cols], qx[2]))
+        assert np.abs(A[rows, cols] - want).max() <= TOL_STAGE * np.abs(want).max()
