@@ -21,7 +21,7 @@
 // TMA store and, concurrently, finish (quantise down the columns) -> slot free.  One
 // persistent CTA per SM with three accumulator buffers in TMEM: the MMAs of the next tiles
 // run while a tile is drained, so the operand ring never idles.
-#include "fp4_kernels.h"
+#include "fp4_gemm_common.cuh"
 
 namespace fp4 {
 
@@ -34,7 +34,7 @@ namespace {
 #define FP4_STAGES 4
 #endif
 #ifndef FP4_RING
-#define FP4_RING 9
+#define FP4_RING 10
 #endif
 constexpr int BM = 128, BN = 128, BK = FP4_BK;  // BK elements of K per stage: 64- or 128-byte operand rows
 static_assert(BK == 128 || BK == 256, "operand rows of a stage are one TMA swizzle span");
@@ -68,6 +68,20 @@ constexpr uint32_t TMEM_SF_COL = 384;    // scale factors after the accumulators
 constexpr uint32_t SF_COLS = KSTEPS * 8; // per stage: 4 columns per MMA for each operand
 static_assert(NACC * BN + STAGES * SF_COLS <= 512, "tensor memory columns");
 constexpr int HALF_CHUNKS = NCHUNK / 2;
+static_assert(RING % 2 == 0, "the ring is split between the two column halves of a tile");
+constexpr int RING_HALF = RING / 2;
+
+// Ring slot and use count of chunk c of the seq-th tile of this CTA.  Each column half of a
+// tile has its own slots, used strictly in order by that half's drain and finish warps, so
+// every waiter sees every phase of the barriers it waits on.
+__device__ __forceinline__ void chunk_slot(uint32_t seq, int c, int& b, uint32_t& use) {
+  const int h = c / HALF_CHUNKS;
+  const uint32_t j = seq * HALF_CHUNKS + (uint32_t)(c - h * HALF_CHUNKS);
+  b = h * RING_HALF + (int)(j % RING_HALF);
+  use = j / RING_HALF;
+}
+// the single-thread roles walk the chunks of a tile alternating between the two halves
+__device__ __forceinline__ int interleaved_chunk(int i) { return (i & 1) * HALF_CHUNKS + (i >> 1); }
 
 // instruction descriptor: E2M1 x E2M1, UE4M3 scales, both operands K-major, M = N = 128
 constexpr uint32_t IDESC = (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | (0u << 23) |
@@ -85,83 +99,6 @@ struct Barriers {
   uint32_t abort_flag;
 };
 static_assert(sizeof(Barriers) <= 512, "barrier block");
-
-__device__ __forceinline__ uint64_t globaltimer_ns() {
-  uint64_t t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
-
-// Wait on an mbarrier phase for at most two seconds; false on give-up (own time-out or
-// another thread's abort flag).
-__device__ __noinline__ bool wait_slow(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag) {
-  const uint64_t t0 = globaltimer_ns();
-  for (;;) {
-    for (int i = 0; i < 256; ++i)
-      if (mbar_try_wait(bar, parity)) return true;
-    if (*abort_flag) return false;
-    if (globaltimer_ns() - t0 > 2000000000ull) {
-      *abort_flag = 1;
-      return false;
-    }
-  }
-}
-__device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag) {
-  if (mbar_try_wait(bar, parity)) return true;
-  return wait_slow(bar, parity, abort_flag);
-}
-
-// tile index of a launch -> (problem, tile row, tile column)
-__device__ __forceinline__ void decode_tile(int t, const GemmLaunch& L, int tiles_per_problem, int& p, int& ti,
-                                            int& tj) {
-  p = t / tiles_per_problem;
-  t -= p * tiles_per_problem;
-  const int tiles_n = L.tiles_n;
-  if (!L.symmetric) {
-    ti = t / tiles_n;
-    tj = t - ti * tiles_n;
-  } else {
-    int row = 0, rem = t;
-    while (rem >= tiles_n - row) { rem -= tiles_n - row; ++row; }
-    ti = row;
-    tj = row + rem;
-  }
-}
-
-// Per-call scalars of an epilogue: the factor that turns the accumulator into the
-// product (tensor scales of the two operands) and the tensor scale of the quantised
-// output, predicted from the running maxima (power of two).
-template <int MODE>
-__device__ __forceinline__ void epilogue_scalars(const GemmProblem& pr, const GemmLaunch& args, float& scale,
-                                                 float& sg_out, bool publish) {
-  float* sc = pr.scalars;
-  sg_out = 1.0f;
-  if (MODE == kPlain) {
-    scale = __fmul_rn(pr.sg_a, pr.sg_b);
-  } else if (MODE == kG1) {
-    const float sgx = sc[args.ix.sg_X0 + args.iter];
-    const float ax = sc[args.ix.amax_X0 + args.iter];
-    scale = __fmul_rn(sgx, sgx);
-    float bound = __fmul_rn(__fmul_rn(__fmul_rn(2.0f, args.l_cols), ax), ax);
-    sg_out = scale_predicted(fminf(bound, 4.0f));
-    if (publish) sc[args.ix.sg_A0 + args.iter] = sg_out;
-  } else if (MODE == kG2) {
-    const float sga = sc[args.ix.sg_A0 + args.iter];
-    const float aa = sc[args.ix.amax_A0 + args.iter];
-    scale = __fmul_rn(sga, sga);
-    float bound = __fmul_rn(__fadd_rn(fabsf(pr.cb), __fmul_rn(4.0f, fabsf(pr.cc))), aa);
-    sg_out = scale_predicted(bound);
-    if (publish) sc[args.ix.sg_B0 + args.iter] = sg_out;
-  } else {
-    const float sgb = sc[args.ix.sg_B0 + args.iter];
-    const float sgx = sc[args.ix.sg_X0 + args.iter];
-    const float ax = sc[args.ix.amax_X0 + args.iter];
-    scale = __fmul_rn(sgb, sgx);
-    float bound = __fmul_rn(__fmul_rn(4.0f, fabsf(pr.ca)), ax);
-    sg_out = scale_predicted(bound);
-    if (publish) sc[args.ix.sg_X0 + args.iter + 1] = sg_out;
-  }
-}
 
 template <int MODE>
 __global__ void __launch_bounds__(NTHREADS, 1)
@@ -271,14 +208,15 @@ k_gemm(const __grid_constant__ GemmProblem single, const GemmProblem* __restrict
     // that will afterwards hold the result chunk, as soon as the slot is free: the loads
     // of a tile run ahead of its main loop.
     if (HAS_AUX && elect_one()) {
-      uint32_t it = 0; bool ok = true;
-      for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+      uint32_t seq = 0; bool ok = true;
+      for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++seq) {
         int p, ti, tj;
         decode_tile(t, args, tiles_per_problem, p, ti, tj);
         const GemmProblem* pr = probs + p;
-        for (int c = 0; c < NCHUNK; ++c, ++it) {
-          const int b = it % RING;
-          const uint32_t use = it / RING;
+        for (int i = 0; i < NCHUNK; ++i) {
+          const int c = interleaved_chunk(i);
+          int b; uint32_t use;
+          chunk_slot(seq, c, b, use);
           if (!wait_bar(&bars->slot_free[b], (use & 1) ^ 1, abort_flag)) { ok = false; break; }
           mbar_expect_tx(&bars->aux_full[b], CHUNK_BYTES);
           tma_load_2d(smem + OFF_RING + b * CHUNK_BYTES, &pr->tmAux, tj * BN + c * CHUNK, ti * BM, &bars->aux_full[b]);
@@ -289,15 +227,16 @@ k_gemm(const __grid_constant__ GemmProblem single, const GemmProblem* __restrict
     // ------------------------------------------------------------ TMA-store issuer
     // Stores each finished chunk and hands the slot back once the store has read it.
     if (elect_one()) {
-      uint32_t it = 0; bool ok = true;
+      uint32_t seq = 0; bool ok = true;
       int prev_slot = -1;
-      for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+      for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++seq) {
         int p, ti, tj;
         decode_tile(t, args, tiles_per_problem, p, ti, tj);
         const GemmProblem* pr = probs + p;
-        for (int c = 0; c < NCHUNK; ++c, ++it) {
-          const int b = it % RING;
-          const uint32_t use = it / RING;
+        for (int i = 0; i < NCHUNK; ++i) {
+          const int c = interleaved_chunk(i);
+          int b; uint32_t use;
+          chunk_slot(seq, c, b, use);
           if (!wait_bar(&bars->v_ready[b], use & 1, abort_flag)) { ok = false; break; }
           if (STORE_F32) {
             tma_store_2d(&pr->tmOut, tj * BN + c * CHUNK, ti * BM, smem + OFF_RING + b * CHUNK_BYTES);
@@ -367,9 +306,8 @@ k_gemm(const __grid_constant__ GemmProblem single, const GemmProblem* __restrict
       uint32_t acc[16];
       tc_ld16_issue(tm_acc + half * HALF_CHUNKS * CHUNK, acc);
       for (int c = half * HALF_CHUNKS; c < (half + 1) * HALF_CHUNKS; ++c) {
-        const uint32_t it = seq * NCHUNK + c;
-        const int b = it % RING;
-        const uint32_t use = it / RING;
+        int b; uint32_t use;
+        chunk_slot(seq, c, b, use);
         uint8_t* slot_row = smem + OFF_RING + b * CHUNK_BYTES + row * 64;
         float v[16];
         // the slot: holds the FP32 tile chunk (G2, G3) or must be free (G1, plain)
@@ -458,9 +396,8 @@ k_gemm(const __grid_constant__ GemmProblem single, const GemmProblem* __restrict
       }
       const bool mirror = do_q && (MODE == kG3 || (args.symmetric && ti != tj));
       for (int c = half * HALF_CHUNKS; c < (half + 1) * HALF_CHUNKS; ++c) {
-        const uint32_t it = seq * NCHUNK + c;
-        const int b = it % RING;
-        const uint32_t use = it / RING;
+        int b; uint32_t use;
+        chunk_slot(seq, c, b, use);
         ok = __all_sync(0xffffffffu, wait_bar(&bars->v_ready[b], use & 1, abort_flag));
         if (!ok) break;
         if (mirror) {

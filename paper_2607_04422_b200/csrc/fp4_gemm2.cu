@@ -1,0 +1,519 @@
+// The same block-scaled NVFP4 GEMM and fused Newton-Schulz epilogues as fp4_gemm.cu
+// (Section 3.4, display equations), for shapes whose dimensions are multiples of 256:
+// a pair of CTAs on two SMs (a cluster of 2) computes one 256 x 256 output tile with
+// tcgen05.mma.cta_group::2.  Each CTA holds 128 rows of the row operand and 128 of the 256
+// rows of the column operand in its shared memory, so every byte fetched from L2 and every
+// byte the tensor core reads from shared memory feeds twice as many multiply-adds as in the
+// 128 x 128 single-CTA kernel, whose main loop is bound by exactly that traffic.
+//
+// Per CTA: accumulator 128 lanes x 256 FP32 columns in tensor memory, drained in sixteen
+// 16-column chunks through the same mbarrier-connected ring pipeline as the single-CTA
+// kernel.  Only the even CTA of a pair issues MMAs; both CTAs run every other role on
+// their own 128 rows.  TMA loads of both CTAs signal the even CTA's stage barrier; MMA
+// completion is multicast to the stage and accumulator barriers of both CTAs.
+#include "fp4_gemm_common.cuh"
+
+namespace fp4 {
+
+namespace {
+
+#ifndef FP4_STAGES2
+#define FP4_STAGES2 4
+#endif
+#ifndef FP4_RING2
+#define FP4_RING2 8
+#endif
+constexpr int PM = 256, PN = 256;              // output tile of a CTA pair
+constexpr int BM = 128;                        // rows per CTA
+constexpr int BK = 256;                        // elements of K per stage: 128-byte operand rows
+constexpr int KSTEPS = BK / 64;
+constexpr int STAGES = FP4_STAGES2;
+constexpr int RING = FP4_RING2;
+constexpr int OPER_BYTES = BM * BK / 2;        // 16 KB: 128 rows of one operand
+constexpr int SF_ATOMS = KSTEPS * 512;         // scale atoms of one 128-row block and stage
+constexpr int SF_BYTES = 3 * SF_ATOMS;         // row operand: own block; column operand: both blocks
+constexpr uint32_t STAGE_BYTES_CTA = 2 * OPER_BYTES + SF_BYTES;
+constexpr int CHUNK = 16;
+constexpr int CHUNK_BYTES = BM * CHUNK * 4;    // 8 KB
+constexpr int NCHUNK = PN / CHUNK;             // 16
+constexpr int HALF_CHUNKS = NCHUNK / 2;
+static_assert(RING % 2 == 0, "the ring is split between the two column halves of a tile");
+constexpr int RING_HALF = RING / 2;
+
+// Ring slot and use count of chunk c of the seq-th tile of this CTA.  Each column half of a
+// tile has its own slots, used strictly in order by that half's drain and finish warps, so
+// every waiter sees every phase of the barriers it waits on.
+__device__ __forceinline__ void chunk_slot(uint32_t seq, int c, int& b, uint32_t& use) {
+  const int h = c / HALF_CHUNKS;
+  const uint32_t j = seq * HALF_CHUNKS + (uint32_t)(c - h * HALF_CHUNKS);
+  b = h * RING_HALF + (int)(j % RING_HALF);
+  use = j / RING_HALF;
+}
+// the single-thread roles walk the chunks of a tile alternating between the two halves
+__device__ __forceinline__ int interleaved_chunk(int i) { return (i & 1) * HALF_CHUNKS + (i >> 1); }
+
+constexpr int OFF_A = 0;
+constexpr int OFF_B = OFF_A + STAGES * OPER_BYTES;
+constexpr int OFF_SF = OFF_B + STAGES * OPER_BYTES;
+constexpr int OFF_RING = OFF_SF + STAGES * SF_BYTES;
+constexpr int OFF_BAR = OFF_RING + RING * CHUNK_BYTES;
+constexpr int SMEM_BYTES = OFF_BAR + 512 + 1024;
+static_assert(SMEM_BYTES <= 232448, "at most 227 KB of dynamic shared memory");
+
+constexpr int NTHREADS = 640;  // warp roles as in the single-CTA kernel
+constexpr uint32_t TMEM_COLS = 512;
+constexpr uint32_t TMEM_SF_COL = 256;          // scale factors after the accumulator
+constexpr uint32_t SF_COLS = KSTEPS * 12;      // per stage: 4 columns (row operand) + 8 (column operand) per MMA
+constexpr int SF_SLOTS = 2;
+static_assert(PN + SF_SLOTS * SF_COLS <= 512, "tensor memory columns");
+
+// instruction descriptor: E2M1 x E2M1, UE4M3 scales, K-major operands, M = 256 (pair), N = 256
+constexpr uint32_t IDESC = (1u << 7) | (1u << 10) | ((uint32_t)(PN >> 3) << 17) | ((uint32_t)(PM >> 4) << 24);
+
+struct Barriers {
+  uint64_t full[STAGES];     // even CTA: both CTAs' operand bytes of a stage have landed
+  uint64_t empty[STAGES];    // stage consumed (MMA commit, multicast to both CTAs)
+  uint64_t acc_full;         // accumulator complete (MMA commit, multicast)
+  uint64_t acc_empty;        // even CTA: accumulator drained by the 16 drain warps of the pair
+  uint64_t aux_full[RING];
+  uint64_t v_ready[RING];
+  uint64_t slot_free[RING];
+  uint32_t tmem_base;
+  uint32_t abort_flag;
+};
+static_assert(sizeof(Barriers) <= 512, "barrier block");
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// shared::cluster address of `p` (a shared-memory object of this CTA) in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t map_to_cta(const void* p, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_u32(p)), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// TMA load whose completion bytes are credited to a barrier that may live in the peer CTA
+__device__ __forceinline__ void tma_load_2d_pair(void* smem_dst, const void* tmap, int x, int y, uint32_t bar_cluster) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+      "[%0], [%1, {%2, %3}], [%4];" ::"r"(smem_u32(smem_dst)),
+      "l"(tmap), "r"(x), "r"(y), "r"(bar_cluster)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_alloc2(uint32_t* smem_dst, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_dst)),
+               "r"(ncols)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish2() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc2(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_cp_sf2(uint32_t taddr, uint64_t sdesc) {
+  asm volatile("tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+}
+__device__ __forceinline__ void tc_mma_nvf4_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                                 uint32_t sfa_tmem, uint32_t sfb_tmem, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::mxf4nvf4.block_scale.block16 [%0], %1, %2, %3, [%5], [%6], p;\n\t}" ::"r"(
+          d_tmem),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(sfa_tmem), "r"(sfb_tmem)
+      : "memory");
+}
+// arrive on the barrier at this shared-memory offset in both CTAs of the pair when all MMAs
+// issued so far have completed
+__device__ __forceinline__ void tc_commit_pair(uint64_t* bar) {
+  const uint16_t mask = 3;
+  asm volatile(
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(
+          smem_u32(bar)),
+      "h"(mask)
+      : "memory");
+}
+
+template <int MODE>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
+k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __restrict__ table, const GemmLaunch args) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  Barriers* bars = reinterpret_cast<Barriers*>(smem + OFF_BAR);
+  volatile uint32_t* abort_flag = &bars->abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const bool leader = (rank == 0);
+  const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+  const GemmProblem* probs = table ? table : &single;
+  // args.tiles_m / tiles_n count 256 x 256 tiles here
+  const int tiles_per_problem = args.symmetric ? args.tiles_n * (args.tiles_n + 1) / 2 : args.tiles_m * args.tiles_n;
+  const int num_tiles = tiles_per_problem * args.num_problems;
+  const int num_kb = args.K / BK;
+  constexpr bool HAS_AUX = (MODE == kG2 || MODE == kG3);
+  constexpr bool STORE_F32 = (MODE == kPlain || MODE == kG1 || MODE == kG3);
+  const bool do_q = (MODE != kPlain) && args.write_q;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < STAGES; ++i) { mbar_init(&bars->full[i], 1); mbar_init(&bars->empty[i], 1); }
+    mbar_init(&bars->acc_full, 1);
+    mbar_init(&bars->acc_empty, 16);
+    for (int i = 0; i < RING; ++i) {
+      mbar_init(&bars->aux_full[i], 1);
+      mbar_init(&bars->v_ready[i], 4);
+      mbar_init(&bars->slot_free[i], 5);
+    }
+    bars->abort_flag = 0;
+    mbar_fence_init();
+  }
+  if (warp == 1) {
+    tmem_alloc2(&bars->tmem_base, TMEM_COLS);
+    tmem_relinquish2();
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();  // the peer's barriers are initialised before anything signals them
+  tc_fence_after();
+  const uint32_t tmem_base = bars->tmem_base;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ operand producer (both CTAs)
+    if (elect_one()) {
+      int st = 0; uint32_t ph = 0; bool ok = true;
+      for (int t = pair; t < num_tiles && ok; t += num_pairs) {
+        int p, ti, tj;
+        decode_tile(t, args, tiles_per_problem, p, ti, tj);
+        const GemmProblem* pr = probs + p;
+        const int arow = ti * PM + (int)rank * BM;   // this CTA's rows of the row operand
+        const int brow = tj * PN + (int)rank * BM;   // this CTA's half of the column operand
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!wait_bar(&bars->empty[st], ph ^ 1, abort_flag)) { ok = false; break; }
+          const uint32_t full_leader = map_to_cta(&bars->full[st], 0);
+          if (leader) mbar_expect_tx(&bars->full[st], 2 * STAGE_BYTES_CTA);
+          tma_load_2d_pair(smem + OFF_A + st * OPER_BYTES, &pr->tmA, kb * (BK / 2), arow, full_leader);
+          tma_load_2d_pair(smem + OFF_B + st * OPER_BYTES, &pr->tmB, kb * (BK / 2), brow, full_leader);
+          // scale atoms: 64-bit elements, one row of the map per 128-row block
+          uint8_t* sf = smem + OFF_SF + st * SF_BYTES;
+          tma_load_2d_pair(sf, &pr->tmSfa, kb * (SF_ATOMS / 8), arow / 128, full_leader);
+          tma_load_2d_pair(sf + SF_ATOMS, &pr->tmSfb, kb * (SF_ATOMS / 8), tj * 2, full_leader);
+          tma_load_2d_pair(sf + 2 * SF_ATOMS, &pr->tmSfb, kb * (SF_ATOMS / 8), tj * 2 + 1, full_leader);
+          if (++st == STAGES) { st = 0; ph ^= 1; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer (even CTA only)
+    if (leader && elect_one()) {
+      int st = 0; uint32_t ph = 0, seq = 0, kstage = 0; bool ok = true;
+      for (int t = pair; t < num_tiles && ok; t += num_pairs, ++seq) {
+        if (!wait_bar(&bars->acc_empty, (seq & 1) ^ 1, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        for (int kb = 0; kb < num_kb; ++kb, ++kstage) {
+          if (!wait_bar(&bars->full[st], ph, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sf_t = tmem_base + TMEM_SF_COL + (kstage % SF_SLOTS) * SF_COLS;
+          const uint8_t* sf = smem + OFF_SF + st * SF_BYTES;
+#pragma unroll
+          for (int a = 0; a < KSTEPS; ++a) {
+            tc_cp_sf2(sf_t + a * 4, umma_desc(smem_u32(sf + a * 512), 128, 0));
+            tc_cp_sf2(sf_t + KSTEPS * 4 + a * 8, umma_desc(smem_u32(sf + SF_ATOMS + a * 512), 128, 0));
+            tc_cp_sf2(sf_t + KSTEPS * 4 + a * 8 + 4, umma_desc(smem_u32(sf + 2 * SF_ATOMS + a * 512), 128, 0));
+          }
+          const uint64_t adesc = umma_desc(smem_u32(smem + OFF_A + st * OPER_BYTES), 1024, 2);
+          const uint64_t bdesc = umma_desc(smem_u32(smem + OFF_B + st * OPER_BYTES), 1024, 2);
+#pragma unroll
+          for (int k = 0; k < KSTEPS; ++k) {
+            tc_mma_nvf4_pair(tmem_base, adesc + 2 * k, bdesc + 2 * k, IDESC, sf_t + k * 4,
+                             sf_t + KSTEPS * 4 + k * 8, (kb | k) != 0 ? 1u : 0u);
+          }
+          tc_commit_pair(&bars->empty[st]);
+          if (++st == STAGES) { st = 0; ph ^= 1; }
+        }
+        if (!ok) break;
+        tc_commit_pair(&bars->acc_full);
+      }
+    }
+  } else if (warp == 2) {
+    // ------------------------------------------------------------ producer of the FP32 tile
+    if (HAS_AUX && elect_one()) {
+      uint32_t seq = 0; bool ok = true;
+      for (int t = pair; t < num_tiles && ok; t += num_pairs, ++seq) {
+        int p, ti, tj;
+        decode_tile(t, args, tiles_per_problem, p, ti, tj);
+        const GemmProblem* pr = probs + p;
+        const int bi = ti * 2 + (int)rank;
+        for (int i = 0; i < NCHUNK; ++i) {
+          const int c = interleaved_chunk(i);
+          int b; uint32_t use;
+          chunk_slot(seq, c, b, use);
+          if (!wait_bar(&bars->slot_free[b], (use & 1) ^ 1, abort_flag)) { ok = false; break; }
+          const int bj = tj * 2 + c / 8;
+          if (args.symmetric && bj < bi) {
+            // a 128 x 128 block below the diagonal: nothing to combine, the slot is passed on empty
+            mbar_arrive(&bars->aux_full[b]);
+          } else {
+            mbar_expect_tx(&bars->aux_full[b], CHUNK_BYTES);
+            tma_load_2d(smem + OFF_RING + b * CHUNK_BYTES, &pr->tmAux, tj * PN + c * CHUNK, bi * BM, &bars->aux_full[b]);
+          }
+        }
+      }
+    }
+  } else if (warp == 3) {
+    // ------------------------------------------------------------ TMA-store issuer
+    if (elect_one()) {
+      uint32_t seq = 0; bool ok = true;
+      int prev_slot = -1;
+      for (int t = pair; t < num_tiles && ok; t += num_pairs, ++seq) {
+        int p, ti, tj;
+        decode_tile(t, args, tiles_per_problem, p, ti, tj);
+        const GemmProblem* pr = probs + p;
+        const int bi = ti * 2 + (int)rank;
+        for (int i = 0; i < NCHUNK; ++i) {
+          const int c = interleaved_chunk(i);
+          int b; uint32_t use;
+          chunk_slot(seq, c, b, use);
+          if (!wait_bar(&bars->v_ready[b], use & 1, abort_flag)) { ok = false; break; }
+          const bool below = args.symmetric && (tj * 2 + c / 8) < bi;
+          if (STORE_F32 && !below) {
+            tma_store_2d(&pr->tmOut, tj * PN + c * CHUNK, bi * BM, smem + OFF_RING + b * CHUNK_BYTES);
+            bulk_commit();
+            bulk_wait_read<1>();
+            if (prev_slot >= 0) mbar_arrive(&bars->slot_free[prev_slot]);
+            prev_slot = b;
+          } else {
+            mbar_arrive(&bars->slot_free[b]);
+          }
+        }
+      }
+      if (STORE_F32) {
+        bulk_wait_read<0>();
+        if (prev_slot >= 0) mbar_arrive(&bars->slot_free[prev_slot]);
+        bulk_wait_all<0>();
+      }
+    }
+  } else if (warp < 12) {
+    // ------------------------------------------------------------ drain warps
+    const int half = (warp - 4) >> 2;
+    const int quad = warp & 3;
+    const int row = quad * 32 + lane;
+    float scale = 0.0f, sg_out = 1.0f, six_sg = 6.0f;
+    float ca = 0.0f, cb = 0.0f, cc = 0.0f;
+    const GemmProblem* pr = nullptr;
+    int cur_p = -1;
+    const int sw = (row >> 1) & 3;
+    const uint32_t tm_lane = tmem_base + ((uint32_t)(quad * 32) << 16);
+    const uint32_t acc_empty_leader = map_to_cta(&bars->acc_empty, 0);
+
+    uint32_t seq = 0;
+    float amax = 0.0f;
+    bool ok = true;
+    for (int t = pair; t < num_tiles && ok; t += num_pairs, ++seq) {
+      int p, ti, tj;
+      decode_tile(t, args, tiles_per_problem, p, ti, tj);
+      if (p != cur_p) {
+        if ((MODE == kG1 || MODE == kG3) && cur_p >= 0) {
+#pragma unroll
+          for (int o = 16; o; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+          if (lane == 0) {
+            const int slot = (MODE == kG1) ? args.ix.amax_A0 + args.iter : args.ix.amax_X0 + args.iter + 1;
+            atomicMax(reinterpret_cast<uint32_t*>(pr->scalars + slot), __float_as_uint(amax));
+          }
+          amax = 0.0f;
+        }
+        cur_p = p;
+        pr = probs + p;
+        epilogue_scalars<MODE>(*pr, args, scale, sg_out,
+                               leader && t == p * tiles_per_problem && threadIdx.x == 128);
+        six_sg = __fmul_rn(6.0f, sg_out);
+        ca = pr->ca; cb = pr->cb; cc = pr->cc;
+      }
+      const int bi = ti * 2 + (int)rank;              // 128-row block of this CTA
+      const int bj = tj * 2 + half;                   // 128-column block of this half
+      const bool below = args.symmetric && bj < bi;   // redundant block of a diagonal tile
+      const bool mirror = do_q && !below && (MODE == kG3 || (args.symmetric && bi != bj));
+      ok = __all_sync(0xffffffffu, wait_bar(&bars->acc_full, seq & 1, abort_flag));
+      if (!ok) break;
+      tc_fence_after();
+      const int64_t grow = (int64_t)bi * BM + row;
+      uint32_t sfw = 0;
+      uint32_t acc[16];
+      tc_ld16_issue(tm_lane + half * HALF_CHUNKS * CHUNK, acc);
+      for (int c = half * HALF_CHUNKS; c < (half + 1) * HALF_CHUNKS; ++c) {
+        int b; uint32_t use;
+        chunk_slot(seq, c, b, use);
+        uint8_t* slot_row = smem + OFF_RING + b * CHUNK_BYTES + row * 64;
+        float v[16];
+        if (HAS_AUX) ok = __all_sync(0xffffffffu, wait_bar(&bars->aux_full[b], use & 1, abort_flag));
+        else ok = __all_sync(0xffffffffu, wait_bar(&bars->slot_free[b], (use & 1) ^ 1, abort_flag));
+        if (!ok) break;
+        tc_wait_ld16(acc);
+        if (HAS_AUX && !below) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            float4 x = *reinterpret_cast<const float4*>(slot_row + ((j ^ sw) << 4));
+            float e[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              const float prod = __fmul_rn(__uint_as_float(acc[4 * j + q]), scale);
+              if (MODE == kG2) v[4 * j + q] = __fadd_rn(__fmul_rn(cb, e[q]), __fmul_rn(cc, prod));
+              else v[4 * j + q] = __fadd_rn(__fmul_rn(ca, e[q]), prod);
+            }
+          }
+        } else {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) v[i] = __fmul_rn(__uint_as_float(acc[i]), scale);
+        }
+        if (c + 1 < (half + 1) * HALF_CHUNKS) {
+          tc_ld16_issue(tm_lane + (c + 1) * CHUNK, acc);
+        } else {
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(acc_empty_leader);  // this warp is done with the accumulator
+        }
+        if (!below && (STORE_F32 || mirror)) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+            *reinterpret_cast<float4*>(slot_row + ((j ^ sw) << 4)) =
+                make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+          fence_proxy_async_smem();
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bars->v_ready[b]);
+        if (below) continue;
+        if (MODE == kG1 || MODE == kG3) {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) amax = fmaxf(amax, fabsf(v[i]));
+        }
+        if (do_q) {
+          uint32_t lo, hi;
+          uint32_t sb = quantize_block16(v, six_sg, sg_out, lo, hi);
+          const int64_t gcol = (int64_t)tj * PN + c * CHUNK;
+          *reinterpret_cast<uint2*>(pr->rq_codes + grow * (args.rq_K / 2) + gcol / 2) = make_uint2(lo, hi);
+          sfw |= sb << (8 * (c & 3));
+          if ((c & 3) == 3) {
+            *reinterpret_cast<uint32_t*>(pr->rq_sf + sf_offset(grow, (gcol >> 4) & ~3ll, args.rq_K >> 4)) = sfw;
+            sfw = 0;
+          }
+        }
+      }
+    }
+    if ((MODE == kG1 || MODE == kG3) && cur_p >= 0) {
+#pragma unroll
+      for (int o = 16; o; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+      if (lane == 0) {
+        const int slot = (MODE == kG1) ? args.ix.amax_A0 + args.iter : args.ix.amax_X0 + args.iter + 1;
+        atomicMax(reinterpret_cast<uint32_t*>(pr->scalars + slot), __float_as_uint(amax));
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ finish warps
+    const int half = (warp - 12) >> 2;
+    const int et = ((warp - 12) & 3) * 32 + lane;
+    const int cc = et & 15, g = et >> 4;
+    float scale, sg_out = 1.0f, six_sg = 6.0f;
+    const GemmProblem* pr = nullptr;
+    int cur_p = -1;
+    uint32_t seq = 0;
+    bool ok = true;
+    for (int t = pair; t < num_tiles && ok; t += num_pairs, ++seq) {
+      int p, ti, tj;
+      decode_tile(t, args, tiles_per_problem, p, ti, tj);
+      if (p != cur_p) {
+        cur_p = p;
+        pr = probs + p;
+        epilogue_scalars<MODE>(*pr, args, scale, sg_out, false);
+        six_sg = __fmul_rn(6.0f, sg_out);
+      }
+      const int bi = ti * 2 + (int)rank;
+      const int bj = tj * 2 + half;
+      const bool below = args.symmetric && bj < bi;
+      const bool mirror = do_q && !below && (MODE == kG3 || (args.symmetric && bi != bj));
+      for (int c = half * HALF_CHUNKS; c < (half + 1) * HALF_CHUNKS; ++c) {
+        int b; uint32_t use;
+        chunk_slot(seq, c, b, use);
+        ok = __all_sync(0xffffffffu, wait_bar(&bars->v_ready[b], use & 1, abort_flag));
+        if (!ok) break;
+        if (mirror) {
+          const uint8_t* obase = smem + OFF_RING + b * CHUNK_BYTES;
+          float w[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const int r = g * 16 + i;
+            w[i] = *reinterpret_cast<const float*>(obase + r * 64 + ((((cc >> 2) ^ ((r >> 1) & 3))) << 4) + (cc & 3) * 4);
+          }
+          uint32_t lo, hi;
+          uint32_t sb = quantize_block16(w, six_sg, sg_out, lo, hi);
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&bars->slot_free[b]);
+          const int64_t trow = (int64_t)tj * PN + c * CHUNK + cc;
+          const int64_t tcol = (int64_t)bi * BM + g * 16;
+          *reinterpret_cast<uint2*>(pr->cq_codes + trow * (args.cq_K / 2) + tcol / 2) = make_uint2(lo, hi);
+          pr->cq_sf[sf_offset(trow, tcol >> 4, args.cq_K >> 4)] = (uint8_t)sb;
+        } else {
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&bars->slot_free[b]);
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();  // neither CTA leaves while the other may still signal it or read its shared memory
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc2(tmem_base, TMEM_COLS);
+  }
+  if (threadIdx.x == 0 && bars->abort_flag) report_timeout(args.status);
+}
+
+template <int MODE>
+cudaError_t launch_pair_mode(const GemmProblem* single, const GemmProblem* table, const GemmLaunch& L, int sms,
+                             cudaStream_t st) {
+  const int tpp = L.symmetric ? L.tiles_n * (L.tiles_n + 1) / 2 : L.tiles_m * L.tiles_n;
+  const int num_tiles = tpp * L.num_problems;
+  int pairs = sms / 2;
+  if (pairs > num_tiles) pairs = num_tiles;
+  count_launches(1);
+  static const GemmProblem kNone = {};
+  k_gemm_pair<MODE><<<2 * pairs, NTHREADS, SMEM_BYTES, st>>>(single ? *single : kNone, table, L);
+  return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t gemm_pair_set_attributes() {
+  cudaError_t e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kPlain>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG2>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG3>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
+  return cudaSuccess;
+}
+
+// `launch` carries tile counts in 128-blocks; all of M, N, K must be multiples of 256.
+cudaError_t launch_gemm_pair(GemmMode mode, const GemmProblem* single, const GemmProblem* table,
+                             const GemmLaunch& launch, int sms, cudaStream_t st) {
+  if ((single == nullptr) == (table == nullptr)) return cudaErrorInvalidValue;
+  if ((launch.tiles_m & 1) || (launch.tiles_n & 1) || (launch.K % BK)) return cudaErrorInvalidValue;
+  GemmLaunch L = launch;
+  L.tiles_m = launch.tiles_m / 2;
+  L.tiles_n = launch.tiles_n / 2;
+  switch (mode) {
+    case kPlain: return launch_pair_mode<kPlain>(single, table, L, sms, st);
+    case kG1: return launch_pair_mode<kG1>(single, table, L, sms, st);
+    case kG2: return launch_pair_mode<kG2>(single, table, L, sms, st);
+    default: return launch_pair_mode<kG3>(single, table, L, sms, st);
+  }
+}
+
+}  // namespace fp4

@@ -1,0 +1,85 @@
+// Device helpers shared by the two GEMM kernels (one CTA per tile / a pair of CTAs per tile).
+#pragma once
+
+#include "fp4_kernels.h"
+
+namespace fp4 {
+
+__device__ __forceinline__ uint64_t globaltimer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+
+// Wait on an mbarrier phase for at most two seconds; false on give-up (own time-out or
+// another thread's abort flag).
+static __device__ __noinline__ bool wait_slow(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag) {
+  const uint64_t t0 = globaltimer_ns();
+  for (;;) {
+    for (int i = 0; i < 256; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (globaltimer_ns() - t0 > 2000000000ull) {
+      *abort_flag = 1;
+      return false;
+    }
+  }
+}
+__device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  return wait_slow(bar, parity, abort_flag);
+}
+
+// tile index of a launch -> (problem, tile row, tile column)
+__device__ __forceinline__ void decode_tile(int t, const GemmLaunch& L, int tiles_per_problem, int& p, int& ti,
+                                            int& tj) {
+  p = t / tiles_per_problem;
+  t -= p * tiles_per_problem;
+  const int tiles_n = L.tiles_n;
+  if (!L.symmetric) {
+    ti = t / tiles_n;
+    tj = t - ti * tiles_n;
+  } else {
+    int row = 0, rem = t;
+    while (rem >= tiles_n - row) { rem -= tiles_n - row; ++row; }
+    ti = row;
+    tj = row + rem;
+  }
+}
+
+// Per-call scalars of an epilogue: the factor that turns the accumulator into the
+// product (tensor scales of the two operands) and the tensor scale of the quantised
+// output, predicted from the running maxima (power of two).
+template <int MODE>
+__device__ __forceinline__ void epilogue_scalars(const GemmProblem& pr, const GemmLaunch& args, float& scale,
+                                                 float& sg_out, bool publish) {
+  float* sc = pr.scalars;
+  sg_out = 1.0f;
+  if (MODE == kPlain) {
+    scale = __fmul_rn(pr.sg_a, pr.sg_b);
+  } else if (MODE == kG1) {
+    const float sgx = sc[args.ix.sg_X0 + args.iter];
+    const float ax = sc[args.ix.amax_X0 + args.iter];
+    scale = __fmul_rn(sgx, sgx);
+    float bound = __fmul_rn(__fmul_rn(__fmul_rn(2.0f, args.l_cols), ax), ax);
+    sg_out = scale_predicted(fminf(bound, 4.0f));
+    if (publish) sc[args.ix.sg_A0 + args.iter] = sg_out;
+  } else if (MODE == kG2) {
+    const float sga = sc[args.ix.sg_A0 + args.iter];
+    const float aa = sc[args.ix.amax_A0 + args.iter];
+    scale = __fmul_rn(sga, sga);
+    float bound = __fmul_rn(__fadd_rn(fabsf(pr.cb), __fmul_rn(4.0f, fabsf(pr.cc))), aa);
+    sg_out = scale_predicted(bound);
+    if (publish) sc[args.ix.sg_B0 + args.iter] = sg_out;
+  } else {
+    const float sgb = sc[args.ix.sg_B0 + args.iter];
+    const float sgx = sc[args.ix.sg_X0 + args.iter];
+    const float ax = sc[args.ix.amax_X0 + args.iter];
+    scale = __fmul_rn(sgb, sgx);
+    float bound = __fmul_rn(__fmul_rn(4.0f, fabsf(pr.ca)), ax);
+    sg_out = scale_predicted(bound);
+    if (publish) sc[args.ix.sg_X0 + args.iter + 1] = sg_out;
+  }
+}
+
+}  // namespace fp4

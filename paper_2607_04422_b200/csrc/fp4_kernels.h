@@ -57,6 +57,7 @@ enum GemmMode : int {
 struct alignas(64) GemmProblem {
   CUtensorMap tmA, tmB;      // NVFP4 codes of the row and the column operand
   CUtensorMap tmAux, tmOut;  // FP32 tile combined in the epilogue / FP32 result
+  CUtensorMap tmSfa, tmSfb;  // scale atoms of the two operands as 2-D maps (CTA-pair kernel)
   const uint8_t* sfa;        // scale atoms of the row operand
   const uint8_t* sfb;        // scale atoms of the column operand
   float* scalars;            // workspace scalars of this matrix (device)
@@ -97,6 +98,9 @@ cudaError_t launch_transpose_out(const float* X, int64_t s, int64_t l, float* ou
 cudaError_t prologue_set_attributes();
 
 cudaError_t gemm_set_attributes();
+cudaError_t gemm_pair_set_attributes();
+cudaError_t launch_gemm_pair(GemmMode mode, const GemmProblem* single, const GemmProblem* table,
+                             const GemmLaunch& launch, int sms, cudaStream_t st);
 int gemm_stage_k();  // elements of K per operand stage (the codes maps' box is this / 2 bytes wide)
 // single: the one problem of the launch (host copy, passed by value) when table is null;
 // table: device array of launch.num_problems problems.

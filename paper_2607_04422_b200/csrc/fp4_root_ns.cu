@@ -68,7 +68,9 @@ const DeviceInfo* device_info() {
     d.status = FP4_ERR_CUDA; d.ready = true; return &d;
   }
   d.encode = reinterpret_cast<EncodeTiledFn>(fn);
-  if (gemm_set_attributes() != cudaSuccess || prologue_set_attributes() != cudaSuccess) d.status = FP4_ERR_CUDA;
+  if (gemm_set_attributes() != cudaSuccess || gemm_pair_set_attributes() != cudaSuccess ||
+      prologue_set_attributes() != cudaSuccess)
+    d.status = FP4_ERR_CUDA;
   d.ready = true;
   return &d;
 }
@@ -102,6 +104,29 @@ bool make_f32_map(const DeviceInfo* d, CUtensorMap* tm, const void* base, int64_
 }
 
 constexpr int kDefaultMaxGroup = 8;
+
+// 2-D map over the scale atoms of a rows x K operand: one map row per 128-row block, 64-bit
+// elements, box = the atoms of one operand stage (256 elements = 2 KB), no swizzle.
+bool make_sf_map(const DeviceInfo* d, CUtensorMap* tm, const void* base, int64_t rows, int64_t K) {
+  if (K < 256) { memset(tm, 0, sizeof(*tm)); return true; }   // never used by the CTA-pair kernel
+  cuuint64_t dims[2] = {(cuuint64_t)(K / 64) * 64, (cuuint64_t)(rows / 128)};
+  cuuint64_t strides[1] = {(cuuint64_t)(K / 64) * 512};
+  cuuint32_t box[2] = {256, 1};
+  cuuint32_t estr[2] = {1, 1};
+  return d->encode(tm, CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, const_cast<void*>(base), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// The CTA-pair kernel takes every product whose dimensions are all multiples of 256.
+cudaError_t launch_gemm_auto(GemmMode mode, const GemmProblem* single, const GemmProblem* table,
+                             const GemmLaunch& L, int sms, cudaStream_t st) {
+#ifndef FP4_DISABLE_PAIR
+  if (!(L.tiles_m & 1) && !(L.tiles_n & 1) && L.K % 256 == 0 && sms >= 2)
+    return launch_gemm_pair(mode, single, table, L, sms, st);
+#endif
+  return launch_gemm(mode, single, table, L, sms, st);
+}
 
 void default_params(fp4_ns_params* p) {
   p->a = p->b = p->c = NAN;
@@ -204,7 +229,11 @@ fp4_status prepare_matrix(const DeviceInfo* d, const float* G, float* out, int64
   float abc[3] = {p->a, p->b, p->c};
   if (std::isnan(p->a)) coeffs(m, n, abc);
   CUtensorMap tm_qX, tm_qXt[2], tm_qA, tm_qB, tm_A, tm_X;
-  bool ok = make_codes_map(d, &tm_qX, ws + L.qX_codes, s, l / 2) &&
+  CUtensorMap sf_qX, sf_qXt[2], sf_qA, sf_qB;
+  bool ok = make_sf_map(d, &sf_qX, ws + L.qX_scales, s, l) && make_sf_map(d, &sf_qXt[0], ws + L.qXt_scales[0], l, s) &&
+            make_sf_map(d, &sf_qXt[1], ws + L.qXt_scales[1], l, s) && make_sf_map(d, &sf_qA, ws + L.qA_scales, s, s) &&
+            make_sf_map(d, &sf_qB, ws + L.qB_scales, s, s) &&
+            make_codes_map(d, &tm_qX, ws + L.qX_codes, s, l / 2) &&
             make_codes_map(d, &tm_qXt[0], ws + L.qXt_codes[0], l, s / 2) &&
             make_codes_map(d, &tm_qXt[1], ws + L.qXt_codes[1], l, s / 2) &&
             make_codes_map(d, &tm_qA, ws + L.qA_codes, s, s / 2) &&
@@ -218,11 +247,13 @@ fp4_status prepare_matrix(const DeviceInfo* d, const float* G, float* out, int64
   // G1: A = qX qX^T (upper-triangle tiles), qA in both triangles
   c->g1 = base;
   c->g1.tmA = c->g1.tmB = tm_qX; c->g1.tmAux = c->g1.tmOut = tm_A;
+  c->g1.tmSfa = c->g1.tmSfb = sf_qX;
   c->g1.sfa = c->g1.sfb = ws + L.qX_scales;
   c->g1.rq_codes = c->g1.cq_codes = ws + L.qA_codes; c->g1.rq_sf = c->g1.cq_sf = ws + L.qA_scales;
   // G2: B = bA + c qA qA^T, qB in both triangles
   c->g2 = base;
   c->g2.tmA = c->g2.tmB = tm_qA; c->g2.tmAux = c->g2.tmOut = tm_A;
+  c->g2.tmSfa = c->g2.tmSfb = sf_qA;
   c->g2.sfa = c->g2.sfb = ws + L.qA_scales;
   c->g2.rq_codes = c->g2.cq_codes = ws + L.qB_codes; c->g2.rq_sf = c->g2.cq_sf = ws + L.qB_scales;
   // G3: X+ = aX + qB qXt^T in place on X; new operand copies
@@ -230,6 +261,7 @@ fp4_status prepare_matrix(const DeviceInfo* d, const float* G, float* out, int64
     GemmProblem& g = c->g3[cur];
     g = base;
     g.tmA = tm_qB; g.tmB = tm_qXt[cur]; g.tmAux = g.tmOut = tm_X;
+    g.tmSfa = sf_qB; g.tmSfb = sf_qXt[cur];
     g.sfa = ws + L.qB_scales; g.sfb = ws + L.qXt_scales[cur];
     g.rq_codes = ws + L.qX_codes; g.rq_sf = ws + L.qX_scales;
     g.cq_codes = ws + L.qXt_codes[cur ^ 1]; g.cq_sf = ws + L.qXt_scales[cur ^ 1];
@@ -237,7 +269,7 @@ fp4_status prepare_matrix(const DeviceInfo* d, const float* G, float* out, int64
   return FP4_OK;
 }
 
-constexpr int kPackMax = 6;
+constexpr int kPackMax = 4;
 struct ProblemPack { GemmProblem p[kPackMax]; };
 
 // Copies problem descriptions from kernel parameters into a device table (the tables of a
@@ -297,14 +329,14 @@ fp4_status run_group(const DeviceInfo* d, MatrixCtx* mats, int count, int steps,
       L1.rq_K = L1.cq_K = (int)s; L1.write_q = 1;
       {
         ProfScope ps(FP4_PROF_G1, st);
-        if (launch_gemm(kG1, count == 1 ? &mats[0].g1 : nullptr, tabs[0], L1, d->sms, st) != cudaSuccess)
+        if (launch_gemm_auto(kG1, count == 1 ? &mats[0].g1 : nullptr, tabs[0], L1, d->sms, st) != cudaSuccess)
           return FP4_ERR_CUDA;
       }
       GemmLaunch L2 = L1;
       L2.K = (int)s;
       {
         ProfScope ps(FP4_PROF_G2, st);
-        if (launch_gemm(kG2, count == 1 ? &mats[0].g2 : nullptr, tabs[1], L2, d->sms, st) != cudaSuccess)
+        if (launch_gemm_auto(kG2, count == 1 ? &mats[0].g2 : nullptr, tabs[1], L2, d->sms, st) != cudaSuccess)
           return FP4_ERR_CUDA;
       }
       GemmLaunch L3 = base;
@@ -313,7 +345,7 @@ fp4_status run_group(const DeviceInfo* d, MatrixCtx* mats, int count, int steps,
       L3.write_q = (!last || keep) ? 1 : 0;
       {
         ProfScope ps(FP4_PROF_G3, st);
-        if (launch_gemm(kG3, count == 1 ? &mats[0].g3[cur] : nullptr, tabs[2 + cur], L3, d->sms, st) != cudaSuccess)
+        if (launch_gemm_auto(kG3, count == 1 ? &mats[0].g3[cur] : nullptr, tabs[2 + cur], L3, d->sms, st) != cudaSuccess)
           return FP4_ERR_CUDA;
       }
     }
@@ -517,7 +549,8 @@ fp4_status fp4_gemm_nt(const uint8_t* a_codes, const uint8_t* a_scales, float a_
   GemmProblem pr;
   memset(&pr, 0, sizeof(pr));
   if (!make_codes_map(d, &pr.tmA, a_codes, M, K / 2) || !make_codes_map(d, &pr.tmB, b_codes, N, K / 2) ||
-      !make_f32_map(d, &pr.tmOut, D, M, N))
+      !make_f32_map(d, &pr.tmOut, D, M, N) || !make_sf_map(d, &pr.tmSfa, a_scales, M, K) ||
+      !make_sf_map(d, &pr.tmSfb, b_scales, N, K))
     return FP4_ERR_CUDA;
   pr.tmAux = pr.tmOut;
   pr.sfa = a_scales; pr.sfb = b_scales;
@@ -527,7 +560,7 @@ fp4_status fp4_gemm_nt(const uint8_t* a_codes, const uint8_t* a_scales, float a_
   L.num_problems = 1;
   L.K = (int)K; L.tiles_m = (int)(M / 128); L.tiles_n = (int)(N / 128);
   L.status = device_status;
-  return launch_gemm(kPlain, &pr, nullptr, L, d->sms, stream) == cudaSuccess ? FP4_OK : FP4_ERR_CUDA;
+  return launch_gemm_auto(kPlain, &pr, nullptr, L, d->sms, stream) == cudaSuccess ? FP4_OK : FP4_ERR_CUDA;
 }
 
 }  // extern "C"

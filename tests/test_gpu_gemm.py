@@ -27,7 +27,8 @@ def _gemm(qa, qb):
     return D.cpu().numpy()
 
 
-@pytest.mark.parametrize("M,N,K", [(128, 128, 128), (128, 128, 512), (256, 384, 640), (640, 256, 2048)])
+@pytest.mark.parametrize("M,N,K", [(128, 128, 128), (128, 128, 512), (256, 384, 640), (640, 256, 2048),
+                                   (256, 256, 256), (512, 768, 1024), (256, 512, 2048)])  # last three: CTA-pair kernel
 def test_gemm_nt_matches_oracle(M, N, K):
     qa = oracle.quantize(workloads.row_lognormal(M, K, seed=1))
     qb = oracle.quantize(workloads.gaussian(N, K, seed=2))
