@@ -81,6 +81,49 @@ __device__ __forceinline__ uint32_t quantize_block16(const float (&v)[16], float
   return sb;
 }
 
+// The same quantisation when the tensor scale is a power of two (every tensor produced
+// inside the Newton-Schulz loop), with the two IEEE divisions replaced by exact equivalents:
+//   amax / (6 sg)  = RN(amax / 6) * (1/sg): the division by the constant 6 is one multiply
+//     and two fused multiply-adds (quotient, exact remainder, correction), which gives the
+//     correctly rounded quotient; the scaling by a power of two is exact;
+//   1 / (s sg): s has 3 mantissa bits, so the correctly rounded reciprocal is one of eight
+//     constants with the exponent shifted.
+// inv_sg = 1/sg; rcp_base = (7 - log2 sg) << 23.  Also returns the block's amax.
+__constant__ uint32_t kRcpMantissa[8] = {0x3F800000u, 0x3F638E39u, 0x3F4CCCCDu, 0x3F3A2E8Cu,
+                                         0x3F2AAAABu, 0x3F1D89D9u, 0x3F124925u, 0x3F088889u};
+__device__ __forceinline__ uint32_t quantize_block16_pow2(const float (&v)[16], float sg, float inv_sg,
+                                                          uint32_t rcp_base, uint32_t& lo, uint32_t& hi,
+                                                          float& amax_out) {
+  float m8[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) m8[i] = fmaxf(fabsf(v[2 * i]), fabsf(v[2 * i + 1]));
+  const float amax = fmaxf(fmaxf(fmaxf(m8[0], m8[1]), fmaxf(m8[2], m8[3])),
+                           fmaxf(fmaxf(m8[4], m8[5]), fmaxf(m8[6], m8[7])));
+  amax_out = amax;
+  const float sixth = 0.16666667163372039794921875f;  // RN(1/6)
+  float q = __fmul_rn(amax, sixth);
+  const float r = __fmaf_rn(-q, 6.0f, amax);
+  q = __fmaf_rn(r, sixth, q);                          // RN(amax / 6)
+  const uint32_t sb = cvt_ue4m3(__fmul_rn(q, inv_sg));
+  lo = 0; hi = 0;
+  if (sb != 0) {
+    const uint32_t e = sb >> 3;
+    const float rcp = e != 0 ? __uint_as_float(kRcpMantissa[sb & 7] + rcp_base - (e << 23))
+                             : __frcp_rn(__fmul_rn(ue4m3_to_float(sb), sg));
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      lo |= cvt_e2m1x2(__fmul_rn(v[2 * i], rcp), __fmul_rn(v[2 * i + 1], rcp)) << (8 * i);
+      hi |= cvt_e2m1x2(__fmul_rn(v[8 + 2 * i], rcp), __fmul_rn(v[9 + 2 * i], rcp)) << (8 * i);
+    }
+  }
+  return sb;
+}
+// rcp_base of a power-of-two tensor scale
+__device__ __forceinline__ uint32_t rcp_base_of(float sg) {
+  const int esg = (int)(__float_as_uint(sg) >> 23) - 127;
+  return (uint32_t)(7 - esg) << 23;
+}
+
 // ----------------------------------------------------------------------------------
 // status word
 // ----------------------------------------------------------------------------------

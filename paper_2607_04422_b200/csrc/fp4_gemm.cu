@@ -263,7 +263,8 @@ k_gemm(const __grid_constant__ GemmProblem single, const GemmProblem* __restrict
     const int half = (warp - 4) >> 2;
     const int quad = warp & 3;
     const int row = quad * 32 + lane;
-    float scale = 0.0f, sg_out = 1.0f, six_sg = 6.0f;
+    float scale = 0.0f, sg_out = 1.0f, inv_sg = 1.0f;
+    uint32_t rcp_base = 0;
     float ca = 0.0f, cb = 0.0f, cc = 0.0f;
     const GemmProblem* pr = nullptr;
     int cur_p = -1;
@@ -291,7 +292,8 @@ k_gemm(const __grid_constant__ GemmProblem single, const GemmProblem* __restrict
         pr = probs + p;
         // the CTA that owns a matrix's first tile publishes its output scale
         epilogue_scalars<MODE>(*pr, args, scale, sg_out, t == p * tiles_per_problem && threadIdx.x == 128);
-        six_sg = __fmul_rn(6.0f, sg_out);
+        inv_sg = __frcp_rn(sg_out);  // exact: the predicted scales are powers of two
+        rcp_base = rcp_base_of(sg_out);
         ca = pr->ca; cb = pr->cb; cc = pr->cc;
       }
       const bool mirror = do_q && (MODE == kG3 || (args.symmetric && ti != tj));
@@ -348,13 +350,11 @@ k_gemm(const __grid_constant__ GemmProblem single, const GemmProblem* __restrict
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(&bars->v_ready[b]);
-        if (MODE == kG1 || MODE == kG3) {
-#pragma unroll
-          for (int i = 0; i < 16; ++i) amax = fmaxf(amax, fabsf(v[i]));
-        }
         if (do_q) {
           uint32_t lo, hi;
-          uint32_t sb = quantize_block16(v, six_sg, sg_out, lo, hi);
+          float bmax;
+          uint32_t sb = quantize_block16_pow2(v, sg_out, inv_sg, rcp_base, lo, hi, bmax);
+          if (MODE == kG1 || MODE == kG3) amax = fmaxf(amax, bmax);
           const int64_t gcol = (int64_t)tj * BN + c * CHUNK;
           *reinterpret_cast<uint2*>(pr->rq_codes + grow * (args.rq_K / 2) + gcol / 2) = make_uint2(lo, hi);
           sfw |= sb << (8 * (c & 3));
@@ -380,7 +380,8 @@ k_gemm(const __grid_constant__ GemmProblem single, const GemmProblem* __restrict
     const int half = (warp - 12) >> 2;
     const int et = ((warp - 12) & 3) * 32 + lane;
     const int cc = et & 15, g = et >> 4;
-    float scale, sg_out = 1.0f, six_sg = 6.0f;
+    float scale, sg_out = 1.0f, inv_sg = 1.0f;
+    uint32_t rcp_base = 0;
     const GemmProblem* pr = nullptr;
     int cur_p = -1;
     uint32_t seq = 0;
@@ -392,7 +393,8 @@ k_gemm(const __grid_constant__ GemmProblem single, const GemmProblem* __restrict
         cur_p = p;
         pr = probs + p;
         epilogue_scalars<MODE>(*pr, args, scale, sg_out, false);
-        six_sg = __fmul_rn(6.0f, sg_out);
+        inv_sg = __frcp_rn(sg_out);
+        rcp_base = rcp_base_of(sg_out);
       }
       const bool mirror = do_q && (MODE == kG3 || (args.symmetric && ti != tj));
       for (int c = half * HALF_CHUNKS; c < (half + 1) * HALF_CHUNKS; ++c) {
@@ -409,7 +411,8 @@ k_gemm(const __grid_constant__ GemmProblem single, const GemmProblem* __restrict
             w[i] = *reinterpret_cast<const float*>(obase + r * 64 + ((((cc >> 2) ^ ((r >> 1) & 3))) << 4) + (cc & 3) * 4);
           }
           uint32_t lo, hi;
-          uint32_t sb = quantize_block16(w, six_sg, sg_out, lo, hi);
+          float bmax;
+          uint32_t sb = quantize_block16_pow2(w, sg_out, inv_sg, rcp_base, lo, hi, bmax);
           __syncwarp();
           if (lane == 0) mbar_arrive(&bars->slot_free[b]);  // the slot's values are in registers
           const int64_t trow = (int64_t)tj * BN + c * CHUNK + cc;  // row of the mirrored / transposed tensor
