@@ -18,8 +18,12 @@ struct NsHeader {
   uint32_t reserved[3];
   uint32_t sel_prefix;   // radix select: magnitude bits fixed so far
   uint32_t sel_rank;     // radix select: rank still to find inside the prefix
-  uint32_t maxabs_bits;  // max |clamped g| as a bit pattern
-  uint32_t pad[25];
+  uint32_t maxabs_bits;  // max |g| below the clip bin (or of everything without a clip), bit pattern
+  uint32_t bin_count;    // elements in the bin picked by the first radix pass
+  uint32_t count_below;  // elements in the bins below it
+  uint32_t cand_count;   // candidates appended by the second pass (may exceed the list's capacity)
+  uint32_t overflow;     // 1: the candidate list overflowed, the fallback passes run
+  uint32_t pad[21];
 };
 
 // Indices into the FP32 `scalars` array of a workspace.
@@ -92,8 +96,15 @@ struct ProfScope {
 
 cudaError_t launch_quantize(const float* x, int64_t rows, int64_t cols, uint8_t* codes, uint8_t* scales,
                             float* tensor_scale, int sms, cudaStream_t st);
-cudaError_t launch_prologue(const float* G, int64_t m, int64_t n, const NsPlan& pl, uint8_t* ws, float* X,
-                            int write_q, bool clear_status, cudaStream_t st);
+struct PrologueItem {
+  const float* G;
+  float* X;
+  uint8_t* ws;
+  const NsPlan* pl;
+  bool clear_status;
+};
+// count matrices that share the shape (s, l) and the clip / eps parameters
+cudaError_t launch_prologue_group(const PrologueItem* items, int count, int write_q, cudaStream_t st);
 cudaError_t launch_transpose_out(const float* X, int64_t s, int64_t l, float* out, cudaStream_t st);
 cudaError_t prologue_set_attributes();
 

@@ -184,7 +184,7 @@ fp4_status make_plan(int64_t m, int64_t n, int steps, const fp4_ns_params* p, in
   size_t off = 0;
   L.header = off; off += 1024;
   L.scalars = off; off += scalar_bytes;
-  pl->off_hist = off; off += 2048 * 4;
+  pl->off_hist = off; off += 8192 * 4;
   pl->zero_bytes = off;
   pl->off_partial = off; off += 1024 * 8;
   off = align_up(off, 1024);
@@ -289,11 +289,13 @@ fp4_status run_group(const DeviceInfo* d, MatrixCtx* mats, int count, int steps,
   const bool keep = (p->flags & FP4_FLAG_KEEP_OPERANDS) != 0;
   const NsPlan& pl0 = mats[0].pl;
   const int64_t s = pl0.s, l = pl0.l;
-  for (int i = 0; i < count; ++i) {
-    MatrixCtx& c = mats[i];
-    if (launch_prologue(c.G, c.pl.m, c.pl.n, c.pl, c.ws, c.X, steps > 0 || keep, clear_first_status && i == 0, st) !=
-        cudaSuccess)
-      return FP4_ERR_CUDA;
+  {
+    std::vector<PrologueItem> items((size_t)count);
+    for (int i = 0; i < count; ++i) {
+      MatrixCtx& c = mats[i];
+      items[(size_t)i] = PrologueItem{c.G, c.X, c.ws, &c.pl, clear_first_status && i == 0};
+    }
+    if (launch_prologue_group(items.data(), count, steps > 0 || keep, st) != cudaSuccess) return FP4_ERR_CUDA;
   }
   if (steps > 0) {
     const GemmProblem* tabs[4] = {nullptr, nullptr, nullptr, nullptr};

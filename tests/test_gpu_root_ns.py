@@ -266,3 +266,30 @@ def test_config4_batched_full_size_properties_and_sampled_stage():
         rows = slice(128 * i, 128 * i + 128); cols = slice(128 * j, 128 * j + 128)
         want = oracle.gemm_nt_q((qx[0][rows], qx[1][rows], qx[2]), (qx[0][cols], qx[1][cols], qx[2]))
         assert np.abs(A[rows, cols] - want).max() <= TOL_STAGE * np.abs(want).max()
+
+
+# --------------------------------------------------------------------------------------
+# Degenerate inputs for the clip: so many equal magnitudes that the candidate list of the
+# two-pass select overflows and the fallback passes run.
+@pytest.mark.parametrize("kind", ["constant", "zero", "two_values", "ties_at_quantile"])
+def test_clip_degenerate_inputs(kind):
+    rng = np.random.default_rng(3)
+    m, n = 256, 384
+    if kind == "constant":
+        G = (3.0 * rng.choice([-1.0, 1.0], (m, n))).astype(np.float32)
+    elif kind == "zero":
+        G = np.zeros((m, n), np.float32)
+    elif kind == "two_values":
+        G = rng.choice([0.5, 2.0, -2.0], (m, n)).astype(np.float32)
+    else:
+        G = rng.standard_normal((m, n)).astype(np.float32)
+        G[np.abs(G) > 2.0] = np.float32(2.25) * np.sign(G[np.abs(G) > 2.0])   # ~4.5 % of entries tie
+    got, ws = run_gpu(G, steps=0)
+    want, tr = oracle.root_ns(G, steps=0, trace_iter=0)
+    lay, sc, *_ = ws_view(ws, m, n, 0, 0)
+    assert sc[lay.idx_tau] == np.float32(tr["tau"])
+    assert abs(sc[lay.idx_nu] - tr["nu"]) <= 1.2e-7 * max(tr["nu"], 1e-30)
+    assert rel(got, want) < 2e-7 or not want.any()
+    if kind != "zero":
+        got2, _ = run_gpu(G, steps=2)
+        assert rel(got2, oracle.root_ns(G, steps=2)) <= TOL_OUT
