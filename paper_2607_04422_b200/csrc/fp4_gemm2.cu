@@ -64,7 +64,7 @@ constexpr int NTHREADS = 640;  // warp roles as in the single-CTA kernel
 constexpr uint32_t TMEM_COLS = 512;
 constexpr uint32_t TMEM_SF_COL = 256;          // scale factors after the accumulator
 constexpr uint32_t SF_COLS = KSTEPS * 12;      // per stage: 4 columns (row operand) + 8 (column operand) per MMA
-constexpr int SF_SLOTS = 2;
+constexpr int SF_SLOTS = 1;
 static_assert(PN + SF_SLOTS * SF_COLS <= 512, "tensor memory columns");
 
 // instruction descriptor: E2M1 x E2M1, UE4M3 scales, K-major operands, M = 256 (pair), N = 256
