@@ -40,17 +40,28 @@ constexpr int HALF_CHUNKS = NCHUNK / 2;
 static_assert(RING % 2 == 0, "the ring is split between the two column halves of a tile");
 constexpr int RING_HALF = RING / 2;
 
-// Ring slot and use count of chunk c of the seq-th tile of this CTA.  Each column half of a
-// tile has its own slots, used strictly in order by that half's drain and finish warps, so
-// every waiter sees every phase of the barriers it waits on.
-__device__ __forceinline__ void chunk_slot(uint32_t seq, int c, int& b, uint32_t& use) {
-  const int h = c / HALF_CHUNKS;
-  const uint32_t j = seq * HALF_CHUNKS + (uint32_t)(c - h * HALF_CHUNKS);
+// Two consecutive tiles use two accumulator buffers that share OV_CHUNKS chunks of tensor
+// memory (512 columns cannot hold two 256-column accumulators plus the scale factors):
+// buffer 0 = columns [0, 256), buffer 1 = columns [208, 464), scale factors [464, 512).
+// The shared columns are buffer 0's last three chunks and buffer 1's first three; the half
+// that owns them drains them first and reports it, then the next tile's MMAs may start
+// while the rest of the tile is still being drained.
+constexpr int OV_CHUNKS = 3;
+constexpr uint32_t ACC1_COL = PN - OV_CHUNKS * CHUNK;  // 208
+
+// chunk handled at position i (0..7) by column half h in a tile that uses buffer `par`
+__device__ __forceinline__ int half_chunk(int par, int h, int i) {
+  if (par == 0 && h == 1) return i < OV_CHUNKS ? NCHUNK - OV_CHUNKS + i : HALF_CHUNKS + (i - OV_CHUNKS);
+  return h * HALF_CHUNKS + i;
+}
+// Ring slot and use count of position i of half h in the seq-th tile of this CTA.  Each
+// column half has its own slots, used strictly in order by that half's drain and finish
+// warps, so every waiter sees every phase of the barriers it waits on.
+__device__ __forceinline__ void chunk_slot(uint32_t seq, int h, int i, int& b, uint32_t& use) {
+  const uint32_t j = seq * HALF_CHUNKS + (uint32_t)i;
   b = h * RING_HALF + (int)(j % RING_HALF);
   use = j / RING_HALF;
 }
-// the single-thread roles walk the chunks of a tile alternating between the two halves
-__device__ __forceinline__ int interleaved_chunk(int i) { return (i & 1) * HALF_CHUNKS + (i >> 1); }
 
 constexpr int OFF_A = 0;
 constexpr int OFF_B = OFF_A + STAGES * OPER_BYTES;
@@ -62,10 +73,10 @@ static_assert(SMEM_BYTES <= 232448, "at most 227 KB of dynamic shared memory");
 
 constexpr int NTHREADS = 640;  // warp roles as in the single-CTA kernel
 constexpr uint32_t TMEM_COLS = 512;
-constexpr uint32_t TMEM_SF_COL = 256;          // scale factors after the accumulator
+constexpr uint32_t TMEM_SF_COL = ACC1_COL + PN;  // scale factors after the second accumulator buffer
 constexpr uint32_t SF_COLS = KSTEPS * 12;      // per stage: 4 columns (row operand) + 8 (column operand) per MMA
-constexpr int SF_SLOTS = 1;
-static_assert(PN + SF_SLOTS * SF_COLS <= 512, "tensor memory columns");
+constexpr int SF_SLOTS = 1;                    // copies and MMAs execute in issue order: one slot suffices
+static_assert(TMEM_SF_COL + SF_SLOTS * SF_COLS <= 512, "tensor memory columns");
 
 // instruction descriptor: E2M1 x E2M1, UE4M3 scales, K-major operands, M = 256 (pair), N = 256
 constexpr uint32_t IDESC = (1u << 7) | (1u << 10) | ((uint32_t)(PN >> 3) << 17) | ((uint32_t)(PM >> 4) << 24);
@@ -73,8 +84,9 @@ constexpr uint32_t IDESC = (1u << 7) | (1u << 10) | ((uint32_t)(PN >> 3) << 17) 
 struct Barriers {
   uint64_t full[STAGES];     // even CTA: both CTAs' operand bytes of a stage have landed
   uint64_t empty[STAGES];    // stage consumed (MMA commit, multicast to both CTAs)
-  uint64_t acc_full;         // accumulator complete (MMA commit, multicast)
-  uint64_t acc_empty;        // even CTA: accumulator drained by the 16 drain warps of the pair
+  uint64_t acc_full[2];      // accumulator buffer complete (MMA commit, multicast)
+  uint64_t acc_empty[2];     // even CTA: buffer drained by the 16 drain warps of the pair
+  uint64_t ov_free;          // even CTA: the columns shared with the other buffer are drained (8 warps)
   uint64_t aux_full[RING];
   uint64_t v_ready[RING];
   uint64_t slot_free[RING];
@@ -165,8 +177,8 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < STAGES; ++i) { mbar_init(&bars->full[i], 1); mbar_init(&bars->empty[i], 1); }
-    mbar_init(&bars->acc_full, 1);
-    mbar_init(&bars->acc_empty, 16);
+    for (int i = 0; i < 2; ++i) { mbar_init(&bars->acc_full[i], 1); mbar_init(&bars->acc_empty[i], 16); }
+    mbar_init(&bars->ov_free, 8);
     for (int i = 0; i < RING; ++i) {
       mbar_init(&bars->aux_full[i], 1);
       mbar_init(&bars->v_ready[i], 4);
@@ -215,8 +227,13 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
     if (leader && elect_one()) {
       int st = 0; uint32_t ph = 0, seq = 0, kstage = 0; bool ok = true;
       for (int t = pair; t < num_tiles && ok; t += num_pairs, ++seq) {
-        if (!wait_bar(&bars->acc_empty, (seq & 1) ^ 1, abort_flag)) { ok = false; break; }
+        const uint32_t par = seq & 1, buse = seq >> 1;
+        // this buffer's previous tile is drained, and so are the columns it shares with the
+        // buffer of the tile before this one
+        if (!wait_bar(&bars->acc_empty[par], (buse & 1) ^ 1, abort_flag)) { ok = false; break; }
+        if (seq > 0 && !wait_bar(&bars->ov_free, (seq - 1) & 1, abort_flag)) { ok = false; break; }
         tc_fence_after();
+        const uint32_t d_tmem = tmem_base + par * ACC1_COL;
         for (int kb = 0; kb < num_kb; ++kb, ++kstage) {
           if (!wait_bar(&bars->full[st], ph, abort_flag)) { ok = false; break; }
           tc_fence_after();
@@ -232,14 +249,14 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
           const uint64_t bdesc = umma_desc(smem_u32(smem + OFF_B + st * OPER_BYTES), 1024, 2);
 #pragma unroll
           for (int k = 0; k < KSTEPS; ++k) {
-            tc_mma_nvf4_pair(tmem_base, adesc + 2 * k, bdesc + 2 * k, IDESC, sf_t + k * 4,
+            tc_mma_nvf4_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC, sf_t + k * 4,
                              sf_t + KSTEPS * 4 + k * 8, (kb | k) != 0 ? 1u : 0u);
           }
           tc_commit_pair(&bars->empty[st]);
           if (++st == STAGES) { st = 0; ph ^= 1; }
         }
         if (!ok) break;
-        tc_commit_pair(&bars->acc_full);
+        tc_commit_pair(&bars->acc_full[par]);
       }
     }
   } else if (warp == 2) {
@@ -251,10 +268,10 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
         decode_tile(t, args, tiles_per_problem, p, ti, tj);
         const GemmProblem* pr = probs + p;
         const int bi = ti * 2 + (int)rank;
-        for (int i = 0; i < NCHUNK; ++i) {
-          const int c = interleaved_chunk(i);
+        for (int i2 = 0; i2 < NCHUNK; ++i2) {
+          const int h = i2 & 1, c = half_chunk((int)(seq & 1), h, i2 >> 1);
           int b; uint32_t use;
-          chunk_slot(seq, c, b, use);
+          chunk_slot(seq, h, i2 >> 1, b, use);
           if (!wait_bar(&bars->slot_free[b], (use & 1) ^ 1, abort_flag)) { ok = false; break; }
           const int bj = tj * 2 + c / 8;
           if (args.symmetric && bj < bi) {
@@ -277,10 +294,10 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
         decode_tile(t, args, tiles_per_problem, p, ti, tj);
         const GemmProblem* pr = probs + p;
         const int bi = ti * 2 + (int)rank;
-        for (int i = 0; i < NCHUNK; ++i) {
-          const int c = interleaved_chunk(i);
+        for (int i2 = 0; i2 < NCHUNK; ++i2) {
+          const int h = i2 & 1, c = half_chunk((int)(seq & 1), h, i2 >> 1);
           int b; uint32_t use;
-          chunk_slot(seq, c, b, use);
+          chunk_slot(seq, h, i2 >> 1, b, use);
           if (!wait_bar(&bars->v_ready[b], use & 1, abort_flag)) { ok = false; break; }
           const bool below = args.symmetric && (tj * 2 + c / 8) < bi;
           if (STORE_F32 && !below) {
@@ -312,7 +329,9 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
     int cur_p = -1;
     const int sw = (row >> 1) & 3;
     const uint32_t tm_lane = tmem_base + ((uint32_t)(quad * 32) << 16);
-    const uint32_t acc_empty_leader = map_to_cta(&bars->acc_empty, 0);
+    const uint32_t acc_empty_leader0 = map_to_cta(&bars->acc_empty[0], 0);
+    const uint32_t acc_empty_leader1 = map_to_cta(&bars->acc_empty[1], 0);
+    const uint32_t ov_free_leader = map_to_cta(&bars->ov_free, 0);
 
     uint32_t seq = 0;
     float amax = 0.0f;
@@ -342,16 +361,20 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
       const int bj = tj * 2 + half;                   // 128-column block of this half
       const bool below = args.symmetric && bj < bi;   // redundant block of a diagonal tile
       const bool mirror = do_q && !below && (MODE == kG3 || (args.symmetric && bi != bj));
-      ok = __all_sync(0xffffffffu, wait_bar(&bars->acc_full, seq & 1, abort_flag));
+      const int par = (int)(seq & 1);
+      ok = __all_sync(0xffffffffu, wait_bar(&bars->acc_full[par], (seq >> 1) & 1, abort_flag));
       if (!ok) break;
       tc_fence_after();
       const int64_t grow = (int64_t)bi * BM + row;
-      uint32_t sfw = 0;
+      const uint32_t tm_acc = tm_lane + par * ACC1_COL;
+      const bool owns_overlap = (half == (par == 0 ? 1 : 0));
+      uint32_t sfw0 = 0, sfw1 = 0;
       uint32_t acc[16];
-      tc_ld16_issue(tm_lane + half * HALF_CHUNKS * CHUNK, acc);
-      for (int c = half * HALF_CHUNKS; c < (half + 1) * HALF_CHUNKS; ++c) {
+      tc_ld16_issue(tm_acc + half_chunk(par, half, 0) * CHUNK, acc);
+      for (int i = 0; i < HALF_CHUNKS; ++i) {
+        const int c = half_chunk(par, half, i);
         int b; uint32_t use;
-        chunk_slot(seq, c, b, use);
+        chunk_slot(seq, half, i, b, use);
         uint8_t* slot_row = smem + OFF_RING + b * CHUNK_BYTES + row * 64;
         float v[16];
         if (HAS_AUX) ok = __all_sync(0xffffffffu, wait_bar(&bars->aux_full[b], use & 1, abort_flag));
@@ -374,12 +397,18 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
 #pragma unroll
           for (int i = 0; i < 16; ++i) v[i] = __fmul_rn(__uint_as_float(acc[i]), scale);
         }
-        if (c + 1 < (half + 1) * HALF_CHUNKS) {
-          tc_ld16_issue(tm_lane + (c + 1) * CHUNK, acc);
+        if (owns_overlap && i == OV_CHUNKS - 1) {
+          // the columns shared with the other buffer are in registers: the next tile may use them
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(ov_free_leader);
+        }
+        if (i + 1 < HALF_CHUNKS) {
+          tc_ld16_issue(tm_acc + half_chunk(par, half, i + 1) * CHUNK, acc);
         } else {
           tc_fence_before();
           __syncwarp();
-          if (lane == 0) mbar_arrive_cluster(acc_empty_leader);  // this warp is done with the accumulator
+          if (lane == 0) mbar_arrive_cluster(par ? acc_empty_leader1 : acc_empty_leader0);  // done with the buffer
         }
         if (!below && (STORE_F32 || mirror)) {
 #pragma unroll
@@ -398,12 +427,14 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
           if (MODE == kG1 || MODE == kG3) amax = fmaxf(amax, bmax);
           const int64_t gcol = (int64_t)tj * PN + c * CHUNK;
           *reinterpret_cast<uint2*>(pr->rq_codes + grow * (args.rq_K / 2) + gcol / 2) = make_uint2(lo, hi);
-          sfw |= sb << (8 * (c & 3));
-          if ((c & 3) == 3) {
-            *reinterpret_cast<uint32_t*>(pr->rq_sf + sf_offset(grow, (gcol >> 4) & ~3ll, args.rq_K >> 4)) = sfw;
-            sfw = 0;
-          }
+          if ((c >> 2) & 1) sfw1 |= sb << (8 * (c & 3)); else sfw0 |= sb << (8 * (c & 3));
         }
+      }
+      if (ok && do_q && !below) {
+        // the two scale words of this half's 128 columns of the row
+        const int64_t kb0 = ((int64_t)tj * PN + half * (PN / 2)) >> 4;
+        *reinterpret_cast<uint32_t*>(pr->rq_sf + sf_offset(grow, kb0, args.rq_K >> 4)) = sfw0;
+        *reinterpret_cast<uint32_t*>(pr->rq_sf + sf_offset(grow, kb0 + 4, args.rq_K >> 4)) = sfw1;
       }
     }
     if ((MODE == kG1 || MODE == kG3) && cur_p >= 0) {
@@ -439,9 +470,10 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
       const int bj = tj * 2 + half;
       const bool below = args.symmetric && bj < bi;
       const bool mirror = do_q && !below && (MODE == kG3 || (args.symmetric && bi != bj));
-      for (int c = half * HALF_CHUNKS; c < (half + 1) * HALF_CHUNKS; ++c) {
+      for (int i = 0; i < HALF_CHUNKS; ++i) {
+        const int c = half_chunk((int)(seq & 1), half, i);
         int b; uint32_t use;
-        chunk_slot(seq, c, b, use);
+        chunk_slot(seq, half, i, b, use);
         ok = __all_sync(0xffffffffu, wait_bar(&bars->v_ready[b], use & 1, abort_flag));
         if (!ok) break;
         if (mirror) {
