@@ -380,6 +380,7 @@ k_gemm(const __grid_constant__ GemmProblem single, const GemmProblem* __restrict
     const int half = (warp - 12) >> 2;
     const int et = ((warp - 12) & 3) * 32 + lane;
     const int cc = et & 15, g = et >> 4;
+    const int rot = (lane >> 4) & 1;
     float scale, sg_out = 1.0f, inv_sg = 1.0f;
     uint32_t rcp_base = 0;
     const GemmProblem* pr = nullptr;
@@ -407,12 +408,19 @@ k_gemm(const __grid_constant__ GemmProblem single, const GemmProblem* __restrict
           float w[16];
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
-            const int r = g * 16 + i;
+            // the upper half-warp starts one row later (and wraps), so that the two half-warps
+            // read rows of different parity, i.e. different banks
+            const int r = g * 16 + ((i + rot) & 15);
             w[i] = *reinterpret_cast<const float*>(obase + r * 64 + ((((cc >> 2) ^ ((r >> 1) & 3))) << 4) + (cc & 3) * 4);
           }
           uint32_t lo, hi;
           float bmax;
           uint32_t sb = quantize_block16_pow2(w, sg_out, inv_sg, rcp_base, lo, hi, bmax);
+          if (rot) {
+            // the codes were packed one row early: rotate the 16 nibbles back into row order
+            const uint32_t nlo = (lo << 4) | (hi >> 28), nhi = (hi << 4) | (lo >> 28);
+            lo = nlo; hi = nhi;
+          }
           __syncwarp();
           if (lane == 0) mbar_arrive(&bars->slot_free[b]);  // the slot's values are in registers
           const int64_t trow = (int64_t)tj * BN + c * CHUNK + cc;  // row of the mirrored / transposed tensor
