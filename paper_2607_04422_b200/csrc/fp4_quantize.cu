@@ -5,15 +5,24 @@
 namespace fp4 {
 
 // ----------------------------------------------------------------------------------
-// amax over a tensor: 128-bit loads, warp shuffle reduction, one atomicMax per block on
-// the bit pattern (non-negative floats order like unsigned integers).
+// amax over a tensor: 128-bit loads (four independent ones in flight per thread), warp
+// shuffle reduction, one atomicMax per block on the bit pattern (non-negative floats order
+// like unsigned integers).
 // ----------------------------------------------------------------------------------
+__device__ __forceinline__ float amax4(float4 v) {
+  return fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w)));
+}
+
 __global__ void __launch_bounds__(256) k_amax(const float4* __restrict__ x, int64_t n4, uint32_t* amax_bits) {
   float m = 0.0f;
-  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n4; i += (int64_t)gridDim.x * blockDim.x) {
-    float4 v = __ldg(x + i);
-    m = fmaxf(fmaxf(m, fmaxf(fabsf(v.x), fabsf(v.y))), fmaxf(fabsf(v.z), fabsf(v.w)));
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+  for (; i + 3 * stride < n4; i += 4 * stride) {
+    const float4 a = __ldg(x + i), b = __ldg(x + i + stride), c = __ldg(x + i + 2 * stride),
+                 d = __ldg(x + i + 3 * stride);
+    m = fmaxf(m, fmaxf(fmaxf(amax4(a), amax4(b)), fmaxf(amax4(c), amax4(d))));
   }
+  for (; i < n4; i += stride) m = fmaxf(m, amax4(__ldg(x + i)));
 #pragma unroll
   for (int o = 16; o; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
   __shared__ float wm[8];
@@ -27,48 +36,65 @@ __global__ void __launch_bounds__(256) k_amax(const float4* __restrict__ x, int6
 }
 
 // ----------------------------------------------------------------------------------
-// Row quantiser.  Four neighbouring lanes own one block of 16 elements (one float4
-// each): block amax by two xor-shuffles, the 8 code bytes and the 4 scale bytes of a
-// 64-element group are gathered by shuffles so that each store is 8 or 4 bytes wide.
+// Row quantiser.  A warp walks one row segment: each lane loads one float4 per step, so a
+// step covers 128 consecutive elements = 8 blocks of 16 with fully coalesced 512-byte
+// requests.  Four neighbouring lanes own one block: block amax by two xor-shuffles; the
+// 8 code bytes of a block and the 4 scale bytes of a 64-element group are gathered by
+// shuffles so that each store is 8 or 4 bytes wide.  Four steps are in flight per lane.
+// grid: x = segments of kSegment columns, y = groups of 8 rows (one per warp).
 // amax_bits holds the tensor amax on entry (bit pattern).
 // ----------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) k_quantize_rows(const float4* __restrict__ x, int64_t rows, int64_t cols,
+constexpr int kSegment = 4096;  // columns per block and row
+
+__device__ __forceinline__ void quantize_step(float4 v, float six_sg, float sg, int lane, uint8_t* code_dst,
+                                              uint8_t* sf_dst) {
+  float a = amax4(v);
+  a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 1));
+  a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 2));
+  const uint32_t sb = cvt_ue4m3(__fdiv_rn(a, six_sg));
+  const float d = __fmul_rn(ue4m3_to_float(sb), sg);
+  uint32_t w = 0;
+  if (d != 0.0f) {
+    const float rcp = __frcp_rn(d);
+    w = cvt_e2m1x2(__fmul_rn(v.x, rcp), __fmul_rn(v.y, rcp)) |
+        (cvt_e2m1x2(__fmul_rn(v.z, rcp), __fmul_rn(v.w, rcp)) << 8);
+  }
+  // codes: 4 lanes x 16 bits -> one 8-byte store by the first lane of the block
+  const uint32_t w2 = w | (__shfl_down_sync(0xffffffffu, w, 1) << 16);
+  const uint32_t w3 = __shfl_down_sync(0xffffffffu, w2, 2);
+  // scales: 4 blocks (16 lanes) -> one 4-byte store
+  const uint32_t s2 = sb | (__shfl_down_sync(0xffffffffu, sb, 4) << 8);
+  const uint32_t s4 = s2 | (__shfl_down_sync(0xffffffffu, s2, 8) << 16);
+  if ((lane & 3) == 0) *reinterpret_cast<uint2*>(code_dst + (lane >> 2) * 8) = make_uint2(w2, w3);
+  if ((lane & 15) == 0) *reinterpret_cast<uint32_t*>(sf_dst + (lane >> 4) * 512) = s4;
+}
+
+__global__ void __launch_bounds__(256) k_quantize_rows(const float* __restrict__ x, int64_t rows, int64_t cols,
                                                        uint8_t* __restrict__ codes, uint8_t* __restrict__ scales,
                                                        const uint32_t* __restrict__ amax_bits) {
   const float sg = scale_exact(__uint_as_float(*amax_bits));
   const float six_sg = __fmul_rn(6.0f, sg);
-  const int64_t n4 = rows * cols / 4;
-  const int64_t c4 = cols / 4;
-  const int lane = threadIdx.x & 31;
-  // n4 is a multiple of 32*... (cols multiple of 128): whole warps stay in range together
-  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n4; i += (int64_t)gridDim.x * blockDim.x) {
-    float4 v = __ldg(x + i);
-    float a = fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w)));
-    a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 1));
-    a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 2));
-    uint32_t sb = cvt_ue4m3(__fdiv_rn(a, six_sg));
-    float d = __fmul_rn(ue4m3_to_float(sb), sg);
-    uint32_t w = 0;
-    if (d != 0.0f) {
-      float rcp = __frcp_rn(d);
-      w = cvt_e2m1x2(__fmul_rn(v.x, rcp), __fmul_rn(v.y, rcp)) |
-          (cvt_e2m1x2(__fmul_rn(v.z, rcp), __fmul_rn(v.w, rcp)) << 8);
-    }
-    // codes: 4 lanes x 16 bits -> one 8-byte store by the first lane of the block
-    uint32_t w2 = w | (__shfl_down_sync(0xffffffffu, w, 1) << 16);
-    uint32_t w3 = __shfl_down_sync(0xffffffffu, w2, 2);
-    // scales: 4 blocks (16 lanes) -> one 4-byte store
-    uint32_t s2 = sb | (__shfl_down_sync(0xffffffffu, sb, 4) << 8);
-    uint32_t s4 = s2 | (__shfl_down_sync(0xffffffffu, s2, 8) << 16);
-    int64_t r = i / c4;
-    int64_t cb = (i - r * c4) >> 2;  // block index in the row
-    if ((lane & 3) == 0) {
-      *reinterpret_cast<uint2*>(codes + (i >> 2) * 8) = make_uint2(w2, w3);
-    }
-    if ((lane & 15) == 0) {
-      *reinterpret_cast<uint32_t*>(scales + sf_offset(r, cb, cols >> 4)) = s4;
-    }
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int64_t r = (int64_t)blockIdx.y * 8 + warp;
+  if (r >= rows) return;
+  const int64_t c_begin = (int64_t)blockIdx.x * kSegment;
+  const int64_t c_end = c_begin + kSegment < cols ? c_begin + kSegment : cols;
+  const float4* src = reinterpret_cast<const float4*>(x + r * cols);
+  uint8_t* crow = codes + r * (cols / 2);
+  // scale atoms of this row: atom (r / 128, c / 64) is 512 bytes; within it this row owns
+  // 4 consecutive bytes at (r % 32) * 16 + ((r % 128) / 32) * 4
+  uint8_t* srow = scales + (size_t)(r >> 7) * (size_t)(cols >> 6) * 512 + (r & 31) * 16 + ((r & 127) >> 5) * 4;
+  int64_t c = c_begin;
+  for (; c + 512 <= c_end; c += 512) {
+    float4 v[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) v[u] = __ldg(src + (c + u * 128) / 4 + lane);
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      quantize_step(v[u], six_sg, sg, lane, crow + (c + u * 128) / 2, srow + ((c + u * 128) >> 6) * 512);
   }
+  for (; c < c_end; c += 128)
+    quantize_step(__ldg(src + c / 4 + lane), six_sg, sg, lane, crow + c / 2, srow + (c >> 6) * 512);
 }
 
 __global__ void k_finish_tensor_scale(float* ts) {
@@ -100,10 +126,11 @@ cudaError_t launch_quantize(const float* x, int64_t rows, int64_t cols, uint8_t*
   const int64_t n4 = rows * cols / 4;
   cudaError_t e = cudaMemsetAsync(tensor_scale, 0, 4, st);
   if (e != cudaSuccess) return e;
-  k_amax<<<grid_for(n4, 256 * 4, sms), 256, 0, st>>>(reinterpret_cast<const float4*>(x), n4,
+  k_amax<<<grid_for(n4, 256 * 8, sms), 256, 0, st>>>(reinterpret_cast<const float4*>(x), n4,
                                                     reinterpret_cast<uint32_t*>(tensor_scale));
-  k_quantize_rows<<<grid_for(n4, 256 * 2, sms), 256, 0, st>>>(reinterpret_cast<const float4*>(x), rows, cols, codes,
-                                                            scales, reinterpret_cast<const uint32_t*>(tensor_scale));
+  const dim3 qgrid((unsigned)((cols + kSegment - 1) / kSegment), (unsigned)((rows + 7) / 8));
+  k_quantize_rows<<<qgrid, 256, 0, st>>>(x, rows, cols, codes, scales,
+                                         reinterpret_cast<const uint32_t*>(tensor_scale));
   k_finish_tensor_scale<<<1, 1, 0, st>>>(tensor_scale);
   count_launches(3);
   return cudaGetLastError();
