@@ -241,6 +241,19 @@ def run_ours(args):
     prof = fp4.fp4_profile_collect()
     fp4.fp4_profile_enable(False)
 
+    # ---- the standalone quantiser on one 8192 x 8192 tensor (HBM-bound: 8.5625 B per element)
+    qx = torch.randn((8192, 8192), device="cuda")
+    qc = torch.empty((8192, 4096), dtype=torch.uint8, device="cuda")
+    qs = torch.empty(fp4.fp4_scale_bytes(8192, 8192), dtype=torch.uint8, device="cuda")
+    qt = torch.empty(1, device="cuda")
+    q_ms = []
+    for _ in range(5):
+        e0.record(stream); fp4.fp4_quantize(qx, qc, qs, qt, 0, stream); e1.record(stream)
+        torch.cuda.synchronize()
+        q_ms.append(e0.elapsed_time(e1))
+    q_gbs = 8192 * 8192 * 8.5625 / (min(q_ms[1:]) / 1e3) / 1e9
+    del qx, qc, qs
+
     # ---- end to end: host buffers in, host buffers out, copies inside the timed region --------
     def e2e_step():
         for h, g in zip(host_in, Gs):
@@ -305,6 +318,8 @@ def run_ours(args):
             "pct_of_nominal_fp4_peak": 100.0 * alg / step_s / 1e12 / FP4_NOMINAL_TFLOPS,
             "pct_of_measured_fp4_peak": 100.0 * alg / step_s / 1e12 / fp4_peak,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": in_bytes, "d2h_bytes_per_step": in_bytes},
+            "quantizer": {"workload": "fp4_quantize 8192x8192 FP32", "gbs": q_gbs, "peak_gbs": pk["hbm_gbs"],
+                          "frac": q_gbs / pk["hbm_gbs"], "bytes_per_element": 8.5625},
             "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "cpu_baseline": cpu}
     print(json.dumps(line), flush=True)
     if world > 1:
