@@ -33,6 +33,10 @@ METRIC = "ns_orthogonalisations_per_s"
 UNIT = "matrices/s"
 FP4_NOMINAL_TFLOPS = 9000.0  # dense NVFP4, nominal
 FP4_OVER_BF16 = 4.0          # nominal ratio of the dense FP4 and BF16 tensor peaks
+# DRAM bytes per element of X that one G3 launch moves (dram__bytes_read + dram__bytes_write of
+# k_gemm_pair<G3> on one 3072 x 8192 matrix, profiles/k_gemm_pair_3072x8192.md: 170.3 MB for
+# 25.2 M elements); a grouped launch is scaled by the elements it covers
+G3_DRAM_BYTES_PER_ELEMENT = 170.3e6 / (3072 * 8192)
 
 
 def peaks():
@@ -297,7 +301,10 @@ def run_ours(args):
     achieved = dom_flops / (dom_ms / 1e3) / 1e12
     fp4_peak = pk["bf16_tflops_sustained"] * FP4_OVER_BF16
     roofline = {"kernel": f"k_gemm<{dom}>", "bound": "tensor", "achieved": achieved, "peak": fp4_peak,
-                "unit": "TFLOP/s", "frac": achieved / fp4_peak, "traffic": None,
+                "unit": "TFLOP/s", "frac": achieved / fp4_peak,
+                "traffic": (G3_DRAM_BYTES_PER_ELEMENT * sum(m * n for m, n in shapes) * STEPS_NS * prof_steps
+                            / max(prof[dom][1], 1)) if dom == "G3" else None,
+                "traffic_note": "DRAM bytes per launch, scaled from an ncu capture of one 3072x8192 matrix",
                 "peak_source": f"{pk['source']} sustained bf16 x {FP4_OVER_BF16:.0f} (nominal FP4/BF16 ratio)",
                 "avg_launch_ms": per_launch_ms, "launches_profiled": prof[dom][1],
                 "flops_per_launch": dom_flops / max(prof[dom][1], 1),
