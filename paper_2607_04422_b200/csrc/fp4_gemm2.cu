@@ -261,59 +261,106 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
     }
   } else if (warp == 2) {
     // ------------------------------------------------------------ producer of the FP32 tile
+    // One thread serves the rings of both column halves without blocking on either: it
+    // polls the next slot of each half in turn and loads a chunk as soon as its slot is free.
     if (HAS_AUX && elect_one()) {
-      uint32_t seq = 0; bool ok = true;
-      for (int t = pair; t < num_tiles && ok; t += num_pairs, ++seq) {
-        int p, ti, tj;
-        decode_tile(t, args, tiles_per_problem, p, ti, tj);
-        const GemmProblem* pr = probs + p;
-        const int bi = ti * 2 + (int)rank;
-        for (int i2 = 0; i2 < NCHUNK; ++i2) {
-          const int h = i2 & 1, c = half_chunk((int)(seq & 1), h, i2 >> 1);
+      const uint32_t my_tiles = pair < num_tiles ? (uint32_t)((num_tiles - pair + num_pairs - 1) / num_pairs) : 0u;
+      const uint32_t total = my_tiles * HALF_CHUNKS;
+      uint32_t n[2] = {0, 0}, seq_dec[2] = {0xFFFFFFFFu, 0xFFFFFFFFu};
+      int pp[2] = {0, 0}, tis[2] = {0, 0}, tjs[2] = {0, 0};
+      uint32_t idle = 0;
+      uint64_t t_idle = 0;
+      while ((n[0] < total || n[1] < total)) {
+        bool progressed = false;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          if (n[h] >= total) continue;
+          const uint32_t seq = n[h] / HALF_CHUNKS;
+          const int i = (int)(n[h] % HALF_CHUNKS);
           int b; uint32_t use;
-          chunk_slot(seq, h, i2 >> 1, b, use);
-          if (!wait_bar(&bars->slot_free[b], (use & 1) ^ 1, abort_flag)) { ok = false; break; }
-          const int bj = tj * 2 + c / 8;
+          chunk_slot(seq, h, i, b, use);
+          if (!mbar_try_wait(&bars->slot_free[b], (use & 1) ^ 1)) continue;
+          if (seq_dec[h] != seq) {
+            decode_tile(pair + (int)seq * num_pairs, args, tiles_per_problem, pp[h], tis[h], tjs[h]);
+            seq_dec[h] = seq;
+          }
+          const GemmProblem* pr = probs + pp[h];
+          const int bi = tis[h] * 2 + (int)rank;
+          const int c = half_chunk((int)(seq & 1), h, i);
+          const int bj = tjs[h] * 2 + c / 8;
           if (args.symmetric && bj < bi) {
             // a 128 x 128 block below the diagonal: nothing to combine, the slot is passed on empty
             mbar_arrive(&bars->aux_full[b]);
           } else {
             mbar_expect_tx(&bars->aux_full[b], CHUNK_BYTES);
-            tma_load_2d(smem + OFF_RING + b * CHUNK_BYTES, &pr->tmAux, tj * PN + c * CHUNK, bi * BM, &bars->aux_full[b]);
+            tma_load_2d(smem + OFF_RING + b * CHUNK_BYTES, &pr->tmAux, tjs[h] * PN + c * CHUNK, bi * BM, &bars->aux_full[b]);
           }
+          ++n[h];
+          progressed = true;
+        }
+        if (progressed) { idle = 0; continue; }
+        if ((++idle & 1023u) == 0) {
+          if (*abort_flag) break;
+          const uint64_t now = globaltimer_ns();
+          if (idle == 1024u) t_idle = now;
+          else if (now - t_idle > 2000000000ull) { *abort_flag = 1; break; }
         }
       }
     }
   } else if (warp == 3) {
     // ------------------------------------------------------------ TMA-store issuer
+    // One thread, both halves, polling like the producer above; up to three stores are in
+    // flight, a slot is handed back once two newer stores have been issued.
     if (elect_one()) {
-      uint32_t seq = 0; bool ok = true;
-      int prev_slot = -1;
-      for (int t = pair; t < num_tiles && ok; t += num_pairs, ++seq) {
-        int p, ti, tj;
-        decode_tile(t, args, tiles_per_problem, p, ti, tj);
-        const GemmProblem* pr = probs + p;
-        const int bi = ti * 2 + (int)rank;
-        for (int i2 = 0; i2 < NCHUNK; ++i2) {
-          const int h = i2 & 1, c = half_chunk((int)(seq & 1), h, i2 >> 1);
+      const uint32_t my_tiles = pair < num_tiles ? (uint32_t)((num_tiles - pair + num_pairs - 1) / num_pairs) : 0u;
+      const uint32_t total = my_tiles * HALF_CHUNKS;
+      uint32_t n[2] = {0, 0}, seq_dec[2] = {0xFFFFFFFFu, 0xFFFFFFFFu};
+      int pp[2] = {0, 0}, tis[2] = {0, 0}, tjs[2] = {0, 0};
+      int q0 = -1, q1 = -1;  // slots of the two newest stores, not yet handed back
+      uint32_t idle = 0;
+      uint64_t t_idle = 0;
+      while ((n[0] < total || n[1] < total)) {
+        bool progressed = false;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          if (n[h] >= total) continue;
+          const uint32_t seq = n[h] / HALF_CHUNKS;
+          const int i = (int)(n[h] % HALF_CHUNKS);
           int b; uint32_t use;
-          chunk_slot(seq, h, i2 >> 1, b, use);
-          if (!wait_bar(&bars->v_ready[b], use & 1, abort_flag)) { ok = false; break; }
-          const bool below = args.symmetric && (tj * 2 + c / 8) < bi;
+          chunk_slot(seq, h, i, b, use);
+          if (!mbar_try_wait(&bars->v_ready[b], use & 1)) continue;
+          if (seq_dec[h] != seq) {
+            decode_tile(pair + (int)seq * num_pairs, args, tiles_per_problem, pp[h], tis[h], tjs[h]);
+            seq_dec[h] = seq;
+          }
+          const GemmProblem* pr = probs + pp[h];
+          const int bi = tis[h] * 2 + (int)rank;
+          const int c = half_chunk((int)(seq & 1), h, i);
+          const bool below = args.symmetric && (tjs[h] * 2 + c / 8) < bi;
           if (STORE_F32 && !below) {
-            tma_store_2d(&pr->tmOut, tj * PN + c * CHUNK, bi * BM, smem + OFF_RING + b * CHUNK_BYTES);
+            tma_store_2d(&pr->tmOut, tjs[h] * PN + c * CHUNK, bi * BM, smem + OFF_RING + b * CHUNK_BYTES);
             bulk_commit();
-            bulk_wait_read<1>();
-            if (prev_slot >= 0) mbar_arrive(&bars->slot_free[prev_slot]);
-            prev_slot = b;
+            bulk_wait_read<2>();  // every store but the two newest has read its slot
+            if (q0 >= 0) mbar_arrive(&bars->slot_free[q0]);
+            q0 = q1; q1 = b;
           } else {
             mbar_arrive(&bars->slot_free[b]);
           }
+          ++n[h];
+          progressed = true;
+        }
+        if (progressed) { idle = 0; continue; }
+        if ((++idle & 1023u) == 0) {
+          if (*abort_flag) break;
+          const uint64_t now = globaltimer_ns();
+          if (idle == 1024u) t_idle = now;
+          else if (now - t_idle > 2000000000ull) { *abort_flag = 1; break; }
         }
       }
       if (STORE_F32) {
         bulk_wait_read<0>();
-        if (prev_slot >= 0) mbar_arrive(&bars->slot_free[prev_slot]);
+        if (q0 >= 0) mbar_arrive(&bars->slot_free[q0]);
+        if (q1 >= 0) mbar_arrive(&bars->slot_free[q1]);
         bulk_wait_all<0>();
       }
     }
