@@ -25,7 +25,8 @@ _f32p = C.POINTER(C.c_float)
 class OrcParams(C.Structure):
     _fields_ = [("a", C.c_float), ("b", C.c_float), ("c", C.c_float),
                 ("clip_quantile", C.c_float), ("eps", C.c_float),
-                ("quantize", C.c_int32), ("exact_scales", C.c_int32)]
+                ("quantize", C.c_int32), ("exact_scales", C.c_int32),
+                ("rht", C.c_int32), ("four_six", C.c_int32), ("seed", C.c_uint64)]
 
 
 class OrcTrace(C.Structure):
@@ -64,6 +65,10 @@ def lib():
         L.orc_quantile_rank.argtypes = [C.c_int64, C.c_float]; L.orc_quantile_rank.restype = C.c_int64
         L.orc_quantize.argtypes = [_f32p, C.c_int64, C.c_int64, C.c_float, _u8p, _u8p]
         L.orc_quantize.restype = None
+        L.orc_quantize_opts.argtypes = [_f32p, C.c_int64, C.c_int64, C.c_float, _u8p, _u8p, C.c_int, C.c_uint16, C.c_int]
+        L.orc_quantize_opts.restype = None
+        L.orc_hadamard16.argtypes = [_f32p, C.c_uint16, _f32p]; L.orc_hadamard16.restype = None
+        L.orc_rht_mask.argtypes = [C.c_uint64, C.c_uint64]; L.orc_rht_mask.restype = C.c_uint16
         L.orc_dequantize.argtypes = [_u8p, _u8p, C.c_float, C.c_int64, C.c_int64, _f32p]
         L.orc_dequantize.restype = None
         L.orc_gemm_nt_q.argtypes = [_u8p, _u8p, C.c_float, _u8p, _u8p, C.c_float,
@@ -120,20 +125,35 @@ def quantile_rank(n: int, q: float) -> int:
 
 
 # --- quantiser ----------------------------------------------------------------
-def quantize(x, s_g=None):
-    """Q_1x16 of a 2-D FP32 array.  s_g None: exact rule amax/2688.
+def quantize(x, s_g=None, rht=False, mask=0, four_six=False):
+    """Q_1x16 of a 2-D FP32 array.  s_g None: exact rule amax/2688 (4 amax/2688 with rht).
+    rht: every 16-block is first multiplied by the random Hadamard matrix of `mask`;
+    four_six: adaptive 4/6 block scaling.
 
     Returns (codes[rows, cols/2] u8, scales[rows, cols/16] u8, s_g)."""
     x, xp = _f32(x)
     rows, cols = x.shape
     assert cols % 16 == 0
     if s_g is None:
-        s_g = tensor_scale_exact(float(lib().orc_amax(xp, x.size)))
+        amax = float(lib().orc_amax(xp, x.size))
+        s_g = tensor_scale_exact(float(np.float32(4.0) * np.float32(amax)) if rht else amax)
     codes = np.empty((rows, cols // 2), np.uint8)
     scales = np.empty((rows, cols // 16), np.uint8)
-    lib().orc_quantize(xp, rows, cols, float(np.float32(s_g)),
-                       codes.ctypes.data_as(_u8p), scales.ctypes.data_as(_u8p))
+    lib().orc_quantize_opts(xp, rows, cols, float(np.float32(s_g)), codes.ctypes.data_as(_u8p),
+                            scales.ctypes.data_as(_u8p), int(bool(rht)), int(mask), int(bool(four_six)))
     return codes, scales, float(np.float32(s_g))
+
+
+def hadamard16(x, mask=0):
+    """x diag(r) H_16 / 4 for one block of 16 (bit i of mask set: r_i = -1)."""
+    x, xp = _f32(x)
+    y = np.empty(16, np.float32)
+    lib().orc_hadamard16(xp, int(mask), y.ctypes.data_as(_f32p))
+    return y
+
+
+def rht_mask(seed, idx):
+    return int(lib().orc_rht_mask(int(seed), int(idx)))
 
 
 def dequantize(codes, scales, s_g):
@@ -177,7 +197,7 @@ def root_coeffs(m, n, steps=5):
 
 
 def root_ns(G, steps=5, abc=None, clip_quantile=0.99, eps=1e-7, quantize=True,
-            exact_scales=False, trace_iter=None):
+            exact_scales=False, trace_iter=None, rht=False, four_six=False, seed=0):
     """The Root Newton-Schulz step on one m x n FP32 matrix.
 
     Returns out (m x n FP32), or (out, trace dict) when trace_iter is given; the
@@ -195,6 +215,9 @@ def root_ns(G, steps=5, abc=None, clip_quantile=0.99, eps=1e-7, quantize=True,
     p.eps = float(np.float32(eps))
     p.quantize = 1 if quantize else 0
     p.exact_scales = 1 if exact_scales else 0
+    p.rht = 1 if rht else 0
+    p.four_six = 1 if four_six else 0
+    p.seed = int(seed)
     out = np.empty((m, n), np.float32)
     if trace_iter is None:
         rc = lib().orc_root_ns(gp, m, n, int(steps), C.byref(p), out.ctypes.data_as(_f32p), None)

@@ -38,6 +38,20 @@
 //     (build with -ffp-contract=off); GEMM sums are taken in FP64 in index
 //     order and rounded once to FP32.
 //
+//   * paper-faithful quantiser mode (Section 3.4: every operand is written Q(. H_16^r) and
+//     "all quantizations use RTN and adaptive 4/6 scaling"; Section 3.1: H_16^r is a fresh
+//     16 x 16 random Hadamard transform): the paper gives no formulas, the readings are
+//       - H^r = diag(r) H_16 / 4 with r in {+1,-1}^16 drawn per (call, iteration, tensor) from
+//         a splitmix64 counter generator; each 16-block along the contraction axis is
+//         multiplied by it (signs, then a natural-order fast Walsh-Hadamard butterfly of
+//         FP32 additions, then * 0.25), the same for both operands of a product, so it
+//         cancels; tensor-scale bounds are multiplied by 4 (|y| <= 4 amax);
+//       - adaptive 4/6: a block is also quantised with its maximum mapped to 4 instead of 6
+//         (scale E4M3(amax / (4 s_g))); the candidate with the smaller sum of squared FP32
+//         errors is kept, ties keep 6.
+//     Parity unpinned against the cited sources (Four Over Six, TE's RHT); the invariances
+//     (the transform cancels, the error never grows) are pinned.
+//
 // Build:  g++ -O2 -std=c++17 -ffp-contract=off -fopenmp -shared -fPIC
 
 #include <algorithm>
@@ -111,38 +125,81 @@ float amax_of(const float* x, int64_t n) {
   return m;
 }
 
+// y = x diag(r) H_16 / 4 for one block: signs (bit i of mask set: -x_i), natural-order fast
+// Walsh-Hadamard butterfly in FP32, then the exact factor 1/4.
+void hadamard16(const float* x, uint16_t mask, float* y) {
+  for (int i = 0; i < 16; ++i) y[i] = ((mask >> i) & 1) ? -x[i] : x[i];
+  for (int h = 1; h < 16; h *= 2)
+    for (int j0 = 0; j0 < 16; j0 += 2 * h)
+      for (int j = j0; j < j0 + h; ++j) {
+        float a = y[j], b = y[j + h];
+        y[j] = a + b;
+        y[j + h] = a - b;
+      }
+  for (int i = 0; i < 16; ++i) y[i] = y[i] * 0.25f;
+}
+
+// Codes of one block for the block scale byte sb; returns the sum of squared FP32 errors.
+float encode_block(const float* v, uint8_t sb, float s_g, uint8_t* nib) {
+  float d = ue4m3_decode(sb) * s_g;
+  float err = 0.0f;
+  if (d == 0.0f) {
+    for (int i = 0; i < 16; ++i) { nib[i] = 0; float q = v[i] * v[i]; err = err + q; }
+    return err;
+  }
+  float rcp = 1.0f / d;
+  for (int i = 0; i < 16; ++i) {
+    float y = v[i] * rcp;
+    int idx = e2m1_index(std::fabs(y));
+    nib[i] = (uint8_t)((std::signbit(y) ? 8 : 0) | idx);
+    float dq = e2m1_decode(nib[i]) * d;
+    float diff = v[i] - dq;
+    float q = diff * diff;
+    err = err + q;
+  }
+  return err;
+}
+
 // Q_1x16 of a row-major rows x cols tensor with a given global scale.
 // codes: rows x cols/2 bytes, element 2j in the low nibble of byte j.
 // scales: rows x cols/16 bytes, plain row-major.
+// rht: each block is first multiplied by the random Hadamard matrix of `mask`;
+// four_six: adaptive 4/6 block scaling.
 void quantize_1x16(const float* x, int64_t rows, int64_t cols, float s_g,
-                   uint8_t* codes, uint8_t* scales) {
+                   uint8_t* codes, uint8_t* scales, int rht = 0, uint16_t mask = 0, int four_six = 0) {
   const int64_t nb = cols / 16;
   const float six_sg = 6.0f * s_g;
+  const float four_sg = 4.0f * s_g;
 #pragma omp parallel for schedule(static)
   for (int64_t r = 0; r < rows; ++r) {
     for (int64_t kb = 0; kb < nb; ++kb) {
-      const float* blk = x + r * cols + kb * 16;
+      const float* src = x + r * cols + kb * 16;
+      float blk[16];
+      if (rht) hadamard16(src, mask, blk); else for (int i = 0; i < 16; ++i) blk[i] = src[i];
       float amax_b = amax_of(blk, 16);
-      float t = amax_b / six_sg;
-      uint8_t sb = ue4m3_encode(t);
-      scales[r * nb + kb] = sb;
-      float s = ue4m3_decode(sb);
-      float d = s * s_g;
+      uint8_t sb = ue4m3_encode(amax_b / six_sg);
       uint8_t nib[16];
-      if (d == 0.0f) {
-        for (int i = 0; i < 16; ++i) nib[i] = 0;
-      } else {
-        float rcp = 1.0f / d;
-        for (int i = 0; i < 16; ++i) {
-          float y = blk[i] * rcp;
-          int idx = e2m1_index(std::fabs(y));
-          nib[i] = (uint8_t)((std::signbit(y) ? 8 : 0) | idx);
-        }
+      float err6 = encode_block(blk, sb, s_g, nib);
+      if (four_six) {
+        uint8_t sb4 = ue4m3_encode(amax_b / four_sg);
+        uint8_t nib4[16];
+        float err4 = encode_block(blk, sb4, s_g, nib4);
+        if (err4 < err6) { sb = sb4; for (int i = 0; i < 16; ++i) nib[i] = nib4[i]; }
       }
+      scales[r * nb + kb] = sb;
       uint8_t* out = codes + r * (cols / 2) + kb * 8;
       for (int i = 0; i < 8; ++i) out[i] = (uint8_t)(nib[2 * i] | (nib[2 * i + 1] << 4));
     }
   }
+}
+
+// splitmix64 counter generator: the 16 signs of the idx-th random Hadamard matrix of a call
+uint16_t rht_mask(uint64_t seed, uint64_t idx) {
+  uint64_t z = seed + 0x9E3779B97F4A7C15ull * (idx + 1);
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  z = z ^ (z >> 31);
+  return (uint16_t)(z & 0xFFFF);
 }
 
 void dequantize_1x16(const uint8_t* codes, const uint8_t* scales, float s_g,
@@ -241,6 +298,9 @@ struct orc_params {
   float eps;
   int32_t quantize;     // 0: plain FP64-accumulated Newton-Schulz, no NVFP4
   int32_t exact_scales; // 1: every tensor scale is amax/2688 (comparison only)
+  int32_t rht;          // 1: random Hadamard transform of every 16-block before quantisation
+  int32_t four_six;     // 1: adaptive 4/6 block scaling
+  uint64_t seed;        // signs of the Hadamard matrices
 };
 
 // Optional record of one iteration's intermediates (all row-major in the work
@@ -281,6 +341,12 @@ void orc_quantize(const float* x, int64_t rows, int64_t cols, float s_g,
                   uint8_t* codes, uint8_t* scales) {
   quantize_1x16(x, rows, cols, s_g, codes, scales);
 }
+void orc_quantize_opts(const float* x, int64_t rows, int64_t cols, float s_g, uint8_t* codes, uint8_t* scales,
+                       int rht, uint16_t mask, int four_six) {
+  quantize_1x16(x, rows, cols, s_g, codes, scales, rht, mask, four_six);
+}
+void orc_hadamard16(const float* x, uint16_t mask, float* y) { hadamard16(x, mask, y); }
+uint16_t orc_rht_mask(uint64_t seed, uint64_t idx) { return rht_mask(seed, idx); }
 
 void orc_dequantize(const uint8_t* codes, const uint8_t* scales, float s_g,
                     int64_t rows, int64_t cols, float* out) {
@@ -368,7 +434,9 @@ int orc_root_ns(const float* G, int64_t m, int64_t n, int steps, const orc_param
   std::vector<uint8_t> qBc((size_t)s * s / 2 + 1), qBs((size_t)s * s / 16 + 1);
 
   float amax_X = amax_of(X.data(), (int64_t)N);
-  float sg_X = scale_exact(amax_X);  // initial operand: exact rule
+  const int rht = prm->rht, f46 = prm->four_six;
+  const float widen = rht ? 4.0f : 1.0f;  // |x H^r| <= 4 amax(x)
+  float sg_X = scale_exact(widen * amax_X);  // initial operand: exact rule
 
   for (int k = 0; k < steps; ++k) {
     const bool rec = tr && tr->iter == k;
@@ -390,8 +458,12 @@ int orc_root_ns(const float* G, int64_t m, int64_t n, int steps, const orc_param
     } else {
       // qX = Q_1x16(X), qX^{16x1} = Q_16x1(X) = Q_1x16(X^T), one global scale
       transpose(X.data(), s, l, Xt.data());
-      quantize_1x16(X.data(), s, l, sg_X, qXc.data(), qXs.data());
-      quantize_1x16(Xt.data(), l, s, sg_X, qXtc.data(), qXts.data());
+      // one Hadamard matrix for X_k (both operand copies and B_k, which meets qX^{16x1}),
+      // another for A_k
+      const uint16_t mask_X = rht ? rht_mask(prm->seed, 2 * (uint64_t)k) : 0;
+      const uint16_t mask_A = rht ? rht_mask(prm->seed, 2 * (uint64_t)k + 1) : 0;
+      quantize_1x16(X.data(), s, l, sg_X, qXc.data(), qXs.data(), rht, mask_X, f46);
+      quantize_1x16(Xt.data(), l, s, sg_X, qXtc.data(), qXts.data(), rht, mask_X, f46);
       // A = qX qX^T
       {
         std::vector<double> d = decode_f64(qXc.data(), qXs.data(), sg_X, s, l);
@@ -399,9 +471,9 @@ int orc_root_ns(const float* G, int64_t m, int64_t n, int steps, const orc_param
       }
       float amax_A = amax_of(A.data(), (int64_t)s * s);
       float bound_A = std::min(2.0f * (float)l * amax_X * amax_X, 4.0f);
-      float sg_A = prm->exact_scales ? scale_exact(amax_A) : scale_predicted(bound_A);
+      float sg_A = prm->exact_scales ? scale_exact(widen * amax_A) : scale_predicted(widen * bound_A);
       // qA = Q_1x16(A); A is symmetric so Q_16x1(A) is the transpose of qA
-      quantize_1x16(A.data(), s, s, sg_A, qAc.data(), qAs.data());
+      quantize_1x16(A.data(), s, s, sg_A, qAc.data(), qAs.data(), rht, mask_A, f46);
       {
         std::vector<double> d = decode_f64(qAc.data(), qAs.data(), sg_A, s, s);
         gemm_nt(d.data(), d.data(), s, s, s, S.data(), 1);
@@ -414,8 +486,8 @@ int orc_root_ns(const float* G, int64_t m, int64_t n, int steps, const orc_param
       }
       float amax_B = amax_of(B.data(), (int64_t)s * s);
       float bound_B = (std::fabs(cb) + 4.0f * std::fabs(cc)) * amax_A;
-      float sg_B = prm->exact_scales ? scale_exact(amax_B) : scale_predicted(bound_B);
-      quantize_1x16(B.data(), s, s, sg_B, qBc.data(), qBs.data());
+      float sg_B = prm->exact_scales ? scale_exact(widen * amax_B) : scale_predicted(widen * bound_B);
+      quantize_1x16(B.data(), s, s, sg_B, qBc.data(), qBs.data(), rht, mask_X, f46);
       // X+ = a X + qB qX^{16x1}
       {
         std::vector<double> db = decode_f64(qBc.data(), qBs.data(), sg_B, s, s);
@@ -445,7 +517,7 @@ int orc_root_ns(const float* G, int64_t m, int64_t n, int steps, const orc_param
       }
       amax_X = amax_of(X.data(), (int64_t)N);
       float bound_X = 4.0f * std::fabs(ca) * amax_prev;
-      sg_X = prm->exact_scales ? scale_exact(amax_X) : scale_predicted(bound_X);
+      sg_X = prm->exact_scales ? scale_exact(widen * amax_X) : scale_predicted(widen * bound_X);
     }
     if (rec && tr->X_out) std::memcpy(tr->X_out, X.data(), N * sizeof(float));
   }

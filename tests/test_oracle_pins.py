@@ -314,3 +314,88 @@ def test_gemm_nt_q_against_numpy():
     sym = oracle.gemm_nt_q(a)
     np.testing.assert_array_equal(sym, sym.T)
     np.testing.assert_allclose(sym, _decode64(*a) @ _decode64(*a).T, rtol=1e-7, atol=1e-7)
+
+
+# ---- paper-faithful quantiser mode: random Hadamard transform and adaptive 4/6 -----------
+def _splitmix_mask(seed, idx):
+    m = (1 << 64) - 1
+    z = (seed + 0x9E3779B97F4A7C15 * (idx + 1)) & m
+    z = ((z ^ (z >> 30)) * 0xBF58476D1CE4E5B9) & m
+    z = ((z ^ (z >> 27)) * 0x94D049BB133111EB) & m
+    z ^= z >> 31
+    return z & 0xFFFF
+
+
+def test_rht_mask_is_splitmix64():
+    for seed, idx in ((0, 0), (1, 5), (2 ** 63 + 12345, 9), (42, 2 ** 40)):
+        assert oracle.rht_mask(seed, idx) == _splitmix_mask(seed, idx)
+
+
+def test_hadamard16_matches_scipy_and_is_orthonormal():
+    import scipy.linalg
+    H = scipy.linalg.hadamard(16).astype(np.float64) / 4.0      # natural (Sylvester) order
+    eye = np.eye(16, dtype=np.float32)
+    M = np.stack([oracle.hadamard16(eye[i]) for i in range(16)])  # row i = e_i H
+    np.testing.assert_array_equal(M, H.astype(np.float32))
+    np.testing.assert_allclose(M.astype(np.float64) @ M.astype(np.float64).T, np.eye(16), atol=1e-12)
+    mask = 0b1010_0000_1111_0001
+    r = np.array([-1.0 if (mask >> i) & 1 else 1.0 for i in range(16)])
+    x = np.random.default_rng(0).standard_normal(16).astype(np.float32)
+    np.testing.assert_allclose(oracle.hadamard16(x, mask), (x * r) @ H, rtol=1e-6, atol=1e-6)
+
+
+def test_rht_cancels_in_the_product():
+    # (X H)(Y H)^T = X Y^T when the same transform is applied to every 16-block along K
+    rng = np.random.default_rng(1)
+    X = rng.standard_normal((8, 64)).astype(np.float32)
+    Y = rng.standard_normal((6, 64)).astype(np.float32)
+    mask = oracle.rht_mask(7, 3)
+    tx = np.stack([np.concatenate([oracle.hadamard16(row[k:k + 16], mask) for k in range(0, 64, 16)]) for row in X])
+    ty = np.stack([np.concatenate([oracle.hadamard16(row[k:k + 16], mask) for k in range(0, 64, 16)]) for row in Y])
+    np.testing.assert_allclose(tx.astype(np.float64) @ ty.astype(np.float64).T,
+                               X.astype(np.float64) @ Y.astype(np.float64).T, rtol=0, atol=2e-5)
+
+
+def test_rht_quantiser_quantises_the_transformed_blocks():
+    x = workloads.gaussian(16, 128, seed=8)
+    mask = oracle.rht_mask(3, 0)
+    c, s, sg = oracle.quantize(x, rht=True, mask=mask)
+    tx = np.stack([np.concatenate([oracle.hadamard16(row[k:k + 16], mask) for k in range(0, 128, 16)]) for row in x])
+    c2, s2, _ = oracle.quantize(tx, s_g=sg)
+    np.testing.assert_array_equal(c, c2)
+    np.testing.assert_array_equal(s, s2)
+    assert sg == oracle.tensor_scale_exact(float(np.float32(4) * np.abs(x).max()))
+    assert s.max() < 0x7E
+
+
+def test_four_six_golden_blocks():
+    for name, vals, sbyte, cbytes in _lines("four_six_examples.txt"):
+        x = np.array([float(v) for v in vals.split()], np.float32).reshape(1, 16)
+        codes, scales, _ = oracle.quantize(x, s_g=1.0, four_six=True)
+        assert scales[0, 0] == int(sbyte, 16), name
+        assert [int(b) for b in codes[0]] == [int(b, 16) for b in cbytes.split()], name
+
+
+def test_four_six_never_increases_the_block_error():
+    x = workloads.row_lognormal(64, 256, seed=12)
+    base = oracle.quantize(x)
+    fs = oracle.quantize(x, four_six=True)
+    eb = ((_decode64(*base) - x) ** 2).reshape(64, 16, 16).sum(-1)
+    ef = ((_decode64(*fs) - x) ** 2).reshape(64, 16, 16).sum(-1)
+    assert np.all(ef <= eb * (1 + 1e-5) + 1e-30)
+    changed = fs[1] != base[1]
+    assert 0.05 < changed.mean() < 0.95          # both mappings are in use
+    assert ef.sum() < 0.97 * eb.sum()             # and the total error drops
+
+
+@pytest.mark.parametrize("gen,shape", [(workloads.gaussian, (256, 512)), (workloads.lowrank_outliers, (256, 256))])
+def test_paper_faithful_ns_is_at_least_as_close_to_exact_ns(gen, shape):
+    g = gen(*shape, seed=0)
+    e = oracle.root_ns(g, steps=5, quantize=False).astype(np.float64)
+    base = oracle.root_ns(g, steps=5).astype(np.float64)
+    pf = oracle.root_ns(g, steps=5, rht=True, four_six=True, seed=11).astype(np.float64)
+    err = lambda q: np.linalg.norm(q - e) / np.linalg.norm(e)
+    assert err(pf) < err(base) * 1.05
+    # a different seed changes the signs, not the quality
+    pf2 = oracle.root_ns(g, steps=5, rht=True, four_six=True, seed=12).astype(np.float64)
+    assert not np.array_equal(pf, pf2) and abs(err(pf2) - err(pf)) < 0.03
