@@ -53,6 +53,23 @@ typedef enum {
 #define FP4_FLAG_KEEP_OPERANDS 1u /* the last iteration also writes the NVFP4 copies of
                                      its result (otherwise skipped as dead work); for
                                      inspection through fp4_root_ns_workspace_layout */
+/* Paper-faithful quantiser options (Section 3.4: operands are rotated by a random Hadamard
+ * transform along the contraction axis, and every quantisation uses adaptive 4/6 scaling).
+ * Off by default; each costs epilogue arithmetic.
+ *   FP4_FLAG_RHT: every 16-block b along the contraction axis becomes b diag(r) H_16 / 4
+ *     before it is quantised, r = 16 random signs and H_16 the Sylvester Hadamard matrix.
+ *     Both operands of a product share r, so the transform cancels in exact arithmetic.
+ *     Tensor scales are derived from 4 amax (|b H| <= 4 amax(b)).
+ *   FP4_FLAG_FOUR_SIX: a block is encoded twice, with its maximum mapped to 6 (block scale
+ *     E4M3(amax/(6 s_g))) and to 4 (E4M3(amax/(4 s_g))); the encoding with the smaller sum
+ *     of squared errors (FP32, summed in element order) is kept, a tie keeps 6.
+ * fp4_root_ns draws the signs of product j of a call (j = 2k: X_k, B_k; j = 2k+1: A_k) from
+ * splitmix64: z = seed + 0x9E3779B97F4A7C15 (j+1), the generator's output mix of z, low 16
+ * bits; bit i set means element i is negated.  fp4_quantize takes the 16 sign bits in the
+ * upper half of its flags word: FP4_FLAG_RHT | FP4_QUANT_SIGNS(mask). */
+#define FP4_FLAG_RHT 2u
+#define FP4_FLAG_FOUR_SIX 4u
+#define FP4_QUANT_SIGNS(mask) ((uint32_t)(mask) << 16)
 
 /* Parameters of the step.  Pass NULL for the defaults noted on each field. */
 typedef struct {
@@ -65,6 +82,7 @@ typedef struct {
   uint32_t flags;      /* FP4_FLAG_*; default 0                                            */
   uint32_t max_group;  /* fp4_root_ns_batched: at most this many equal-shape matrices run their
                           stages in lockstep as single launches; 0 = library default (8)      */
+  uint64_t seed;       /* FP4_FLAG_RHT: seed of the sign draws; default 0                    */
 } fp4_ns_params;
 
 const char* fp4_status_string(fp4_status s);
@@ -84,7 +102,8 @@ const char* fp4_status_string(fp4_status s);
  * Decoded value of an element = E2M1 value * E4M3 scale * s_g.  Rounding is to nearest,
  * ties to even, saturating.  Block scale = E4M3(amax_block / (6 s_g)); elements are
  * multiplied by the FP32 reciprocal of (scale * s_g) before conversion.
- * flags: must be 0.
+ * flags: 0, or FP4_FLAG_RHT | FP4_QUANT_SIGNS(mask) and / or FP4_FLAG_FOUR_SIX (see above);
+ *   with FP4_FLAG_RHT, s_g = 4 amax(x)/2688.
  */
 size_t fp4_scale_bytes(int64_t rows, int64_t cols);
 fp4_status fp4_quantize(const float* x, int64_t rows, int64_t cols, uint8_t* codes,

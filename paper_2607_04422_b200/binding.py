@@ -16,6 +16,8 @@ _LIB_PATH = os.environ.get("FP4ROOT_LIB") or os.path.join(_HERE, "libfp4root.so"
 _lib = None
 
 FP4_FLAG_KEEP_OPERANDS = 1
+FP4_FLAG_RHT = 2
+FP4_FLAG_FOUR_SIX = 4
 STATUS_NAMES = {0: "FP4_OK", 1: "FP4_ERR_INVALID_ARG", 2: "FP4_ERR_SHAPE", 3: "FP4_ERR_ALIGNMENT",
                 4: "FP4_ERR_WORKSPACE", 5: "FP4_ERR_ARCH", 6: "FP4_ERR_CUDA", 7: "FP4_ERR_DEVICE_TIMEOUT",
                 8: "FP4_ERR_UNIMPLEMENTED", 9: "FP4_ERR_STATIC_LIMIT"}
@@ -37,10 +39,10 @@ class Fp4Error(RuntimeError):
 class NsParams(C.Structure):
     """fp4_ns_params"""
     _fields_ = [("a", C.c_float), ("b", C.c_float), ("c", C.c_float), ("clip_quantile", C.c_float),
-                ("eps", C.c_float), ("flags", C.c_uint32), ("max_group", C.c_uint32)]
+                ("eps", C.c_float), ("flags", C.c_uint32), ("max_group", C.c_uint32), ("seed", C.c_uint64)]
 
     @classmethod
-    def make(cls, abc=None, clip_quantile=0.99, eps=1e-7, flags=0, max_group=0):
+    def make(cls, abc=None, clip_quantile=0.99, eps=1e-7, flags=0, max_group=0, seed=0):
         p = cls()
         if abc is None:
             p.a = p.b = p.c = float("nan")
@@ -48,6 +50,7 @@ class NsParams(C.Structure):
             p.a, p.b, p.c = [float(v) for v in abc]
         p.clip_quantile, p.eps, p.flags = float(clip_quantile), float(eps), int(flags)
         p.max_group = int(max_group)
+        p.seed = int(seed)
         return p
 
 

@@ -125,6 +125,101 @@ __device__ __forceinline__ uint32_t rcp_base_of(float sg) {
 }
 
 // ----------------------------------------------------------------------------------
+// Paper-faithful quantiser options (Section 3.4): a random Hadamard transform of every
+// 16-block along the contraction axis, and adaptive 4/6 block scaling.
+// ----------------------------------------------------------------------------------
+struct QuantOpts {
+  uint32_t rht;       // 1: multiply each block by diag(signs) H_16 / 4 before quantising
+  uint32_t mask;      // bit i set: element i of a block is negated
+  uint32_t four_six;  // 1: try the max->4 mapping too, keep the smaller squared error
+  float widen;        // factor on the amax bounds of predicted tensor scales: 4 with rht, else 1
+};
+
+// One byte of two E2M1 codes -> two FP32 values (x = low nibble), exact.
+__device__ __forceinline__ float2 e2m1x2_to_float2(uint32_t byte) {
+  uint32_t h2;
+  asm("{\n\t.reg .b8 t;\n\tcvt.u8.u32 t, %1;\n\tcvt.rn.f16x2.e2m1x2 %0, t;\n\t}" : "=r"(h2) : "r"(byte));
+  float2 f;
+  asm("{\n\t.reg .f16 a, b;\n\tmov.b32 {a, b}, %2;\n\tcvt.f32.f16 %0, a;\n\tcvt.f32.f16 %1, b;\n\t}"
+      : "=f"(f.x), "=f"(f.y)
+      : "r"(h2));
+  return f;
+}
+
+// v <- v diag(signs) H_16 / 4 in FP32: signs, the natural-order butterfly (strides 1, 2, 4, 8;
+// sum to the lower index, difference to the upper), then the factor 1/4.
+__device__ __forceinline__ void hadamard16(float (&v)[16], uint32_t mask) {
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = (mask >> i) & 1 ? -v[i] : v[i];
+#pragma unroll
+  for (int h = 1; h < 16; h *= 2) {
+#pragma unroll
+    for (int j = 0; j < 16; ++j) {
+      if ((j & h) == 0) {
+        const float a = v[j], b = v[j + h];
+        v[j] = __fadd_rn(a, b);
+        v[j + h] = __fsub_rn(a, b);
+      }
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __fmul_rn(v[i], 0.25f);
+}
+
+// Codes of one block for the scale byte sb; returns the sum of the squared FP32 errors,
+// accumulated in element order (the 4/6 choice compares two such sums, so the order of the
+// roundings is part of the definition).
+__device__ __forceinline__ float encode_block16(const float (&v)[16], uint32_t sb, float sg, uint32_t& lo,
+                                                uint32_t& hi) {
+  const float d = __fmul_rn(ue4m3_to_float(sb), sg);
+  lo = 0; hi = 0;
+  float err = 0.0f;
+  if (d == 0.0f) {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) err = __fadd_rn(err, __fmul_rn(v[i], v[i]));
+    return err;
+  }
+  const float rcp = __frcp_rn(d);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const uint32_t byte = cvt_e2m1x2(__fmul_rn(v[2 * i], rcp), __fmul_rn(v[2 * i + 1], rcp));
+    const float2 q = e2m1x2_to_float2(byte);
+    const float d0 = __fsub_rn(v[2 * i], __fmul_rn(q.x, d));
+    err = __fadd_rn(err, __fmul_rn(d0, d0));
+    const float d1 = __fsub_rn(v[2 * i + 1], __fmul_rn(q.y, d));
+    err = __fadd_rn(err, __fmul_rn(d1, d1));
+    if (i < 4) lo |= byte << (8 * i); else hi |= byte << (8 * (i - 4));
+  }
+  return err;
+}
+
+// Quantise one block with the options above; any tensor scale.  v is transformed in place.
+// Returns the scale byte; amax_in is the block's amax before the transform (what the
+// predicted tensor scales of the next stage are derived from).
+__device__ __forceinline__ uint32_t quantize_block16_opts(float (&v)[16], const QuantOpts& q, float sg, uint32_t& lo,
+                                                          uint32_t& hi, float& amax_in) {
+  float a = 0.0f;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) a = fmaxf(a, fabsf(v[i]));
+  amax_in = a;
+  if (q.rht) {
+    hadamard16(v, q.mask);
+    a = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) a = fmaxf(a, fabsf(v[i]));
+  }
+  uint32_t sb = cvt_ue4m3(__fdiv_rn(a, __fmul_rn(6.0f, sg)));
+  const float err6 = encode_block16(v, sb, sg, lo, hi);
+  if (q.four_six) {
+    const uint32_t sb4 = cvt_ue4m3(__fdiv_rn(a, __fmul_rn(4.0f, sg)));
+    uint32_t lo4, hi4;
+    const float err4 = encode_block16(v, sb4, sg, lo4, hi4);
+    if (err4 < err6) { sb = sb4; lo = lo4; hi = hi4; }
+  }
+  return sb;
+}
+
+// ----------------------------------------------------------------------------------
 // status word
 // ----------------------------------------------------------------------------------
 __device__ __forceinline__ void report_timeout(uint32_t* status) {

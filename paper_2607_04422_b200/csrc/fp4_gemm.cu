@@ -100,7 +100,7 @@ struct Barriers {
 };
 static_assert(sizeof(Barriers) <= 512, "barrier block");
 
-template <int MODE>
+template <int MODE, bool PF>
 __global__ void __launch_bounds__(NTHREADS, 1)
 k_gemm(const __grid_constant__ GemmProblem single, const GemmProblem* __restrict__ table, const GemmLaunch args) {
   extern __shared__ uint8_t smem_raw[];
@@ -353,7 +353,9 @@ k_gemm(const __grid_constant__ GemmProblem single, const GemmProblem* __restrict
         if (do_q) {
           uint32_t lo, hi;
           float bmax;
-          uint32_t sb = quantize_block16_pow2(v, sg_out, inv_sg, rcp_base, lo, hi, bmax);
+          uint32_t sb;
+          if (PF) sb = quantize_block16_opts(v, args.q, sg_out, lo, hi, bmax);
+          else sb = quantize_block16_pow2(v, sg_out, inv_sg, rcp_base, lo, hi, bmax);
           if (MODE == kG1 || MODE == kG3) amax = fmaxf(amax, bmax);
           const int64_t gcol = (int64_t)tj * BN + c * CHUNK;
           *reinterpret_cast<uint2*>(pr->rq_codes + grow * (args.rq_K / 2) + gcol / 2) = make_uint2(lo, hi);
@@ -415,11 +417,20 @@ k_gemm(const __grid_constant__ GemmProblem single, const GemmProblem* __restrict
           }
           uint32_t lo, hi;
           float bmax;
-          uint32_t sb = quantize_block16_pow2(w, sg_out, inv_sg, rcp_base, lo, hi, bmax);
-          if (rot) {
-            // the codes were packed one row early: rotate the 16 nibbles back into row order
-            const uint32_t nlo = (lo << 4) | (hi >> 28), nhi = (hi << 4) | (lo >> 28);
-            lo = nlo; hi = nhi;
+          uint32_t sb;
+          if (PF) {
+            // the transform and the error sums need the block in row order
+            float x[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) x[i] = rot ? w[(i + 15) & 15] : w[i];
+            sb = quantize_block16_opts(x, args.q, sg_out, lo, hi, bmax);
+          } else {
+            sb = quantize_block16_pow2(w, sg_out, inv_sg, rcp_base, lo, hi, bmax);
+            if (rot) {
+              // the codes were packed one row early: rotate the 16 nibbles back into row order
+              const uint32_t nlo = (lo << 4) | (hi >> 28), nhi = (hi << 4) | (lo >> 28);
+              lo = nlo; hi = nhi;
+            }
           }
           __syncwarp();
           if (lane == 0) mbar_arrive(&bars->slot_free[b]);  // the slot's values are in registers
@@ -444,7 +455,7 @@ k_gemm(const __grid_constant__ GemmProblem single, const GemmProblem* __restrict
   if (threadIdx.x == 0 && bars->abort_flag) report_timeout(args.status);
 }
 
-template <int MODE>
+template <int MODE, bool PF>
 cudaError_t launch_mode(const GemmProblem* single, const GemmProblem* table, const GemmLaunch& L, int sms,
                         cudaStream_t st) {
   const int tpp = L.symmetric ? L.tiles_n * (L.tiles_n + 1) / 2 : L.tiles_m * L.tiles_n;
@@ -453,7 +464,7 @@ cudaError_t launch_mode(const GemmProblem* single, const GemmProblem* table, con
   if (grid > num_tiles) grid = num_tiles;
   count_launches(1);
   static const GemmProblem kNone = {};
-  k_gemm<MODE><<<grid, NTHREADS, SMEM_BYTES, st>>>(single ? *single : kNone, table, L);
+  k_gemm<MODE, PF><<<grid, NTHREADS, SMEM_BYTES, st>>>(single ? *single : kNone, table, L);
   return cudaGetLastError();
 }
 
@@ -463,21 +474,25 @@ int gemm_stage_k() { return BK; }
 
 cudaError_t gemm_set_attributes() {
   cudaError_t e;
-  if ((e = cudaFuncSetAttribute(k_gemm<kPlain>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
-  if ((e = cudaFuncSetAttribute(k_gemm<kG1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
-  if ((e = cudaFuncSetAttribute(k_gemm<kG2>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
-  if ((e = cudaFuncSetAttribute(k_gemm<kG3>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm<kPlain, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm<kG1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm<kG1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm<kG2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm<kG2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm<kG3, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm<kG3, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
   return cudaSuccess;
 }
 
 cudaError_t launch_gemm(GemmMode mode, const GemmProblem* single, const GemmProblem* table, const GemmLaunch& launch,
                         int sms, cudaStream_t st) {
   if ((single == nullptr) == (table == nullptr)) return cudaErrorInvalidValue;
+  const bool pf = launch.q.rht || launch.q.four_six;
   switch (mode) {
-    case kPlain: return launch_mode<kPlain>(single, table, launch, sms, st);
-    case kG1: return launch_mode<kG1>(single, table, launch, sms, st);
-    case kG2: return launch_mode<kG2>(single, table, launch, sms, st);
-    default: return launch_mode<kG3>(single, table, launch, sms, st);
+    case kPlain: return launch_mode<kPlain, false>(single, table, launch, sms, st);
+    case kG1: return pf ? launch_mode<kG1, true>(single, table, launch, sms, st) : launch_mode<kG1, false>(single, table, launch, sms, st);
+    case kG2: return pf ? launch_mode<kG2, true>(single, table, launch, sms, st) : launch_mode<kG2, false>(single, table, launch, sms, st);
+    default: return pf ? launch_mode<kG3, true>(single, table, launch, sms, st) : launch_mode<kG3, false>(single, table, launch, sms, st);
   }
 }
 

@@ -154,7 +154,7 @@ __device__ __forceinline__ void tc_commit_pair(uint64_t* bar) {
       : "memory");
 }
 
-template <int MODE>
+template <int MODE, bool PF>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
 k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __restrict__ table, const GemmLaunch args) {
   extern __shared__ uint8_t smem_raw[];
@@ -470,7 +470,9 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
         if (do_q) {
           uint32_t lo, hi;
           float bmax;
-          uint32_t sb = quantize_block16_pow2(v, sg_out, inv_sg, rcp_base, lo, hi, bmax);
+          uint32_t sb;
+          if (PF) sb = quantize_block16_opts(v, args.q, sg_out, lo, hi, bmax);
+          else sb = quantize_block16_pow2(v, sg_out, inv_sg, rcp_base, lo, hi, bmax);
           if (MODE == kG1 || MODE == kG3) amax = fmaxf(amax, bmax);
           const int64_t gcol = (int64_t)tj * PN + c * CHUNK;
           *reinterpret_cast<uint2*>(pr->rq_codes + grow * (args.rq_K / 2) + gcol / 2) = make_uint2(lo, hi);
@@ -536,11 +538,20 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
           }
           uint32_t lo, hi;
           float bmax;
-          uint32_t sb = quantize_block16_pow2(w, sg_out, inv_sg, rcp_base, lo, hi, bmax);
-          if (rot) {
-            // the codes were packed one row early: rotate the 16 nibbles back into row order
-            const uint32_t nlo = (lo << 4) | (hi >> 28), nhi = (hi << 4) | (lo >> 28);
-            lo = nlo; hi = nhi;
+          uint32_t sb;
+          if (PF) {
+            // the transform and the error sums need the block in row order
+            float x[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) x[i] = rot ? w[(i + 15) & 15] : w[i];
+            sb = quantize_block16_opts(x, args.q, sg_out, lo, hi, bmax);
+          } else {
+            sb = quantize_block16_pow2(w, sg_out, inv_sg, rcp_base, lo, hi, bmax);
+            if (rot) {
+              // the codes were packed one row early: rotate the 16 nibbles back into row order
+              const uint32_t nlo = (lo << 4) | (hi >> 28), nhi = (hi << 4) | (lo >> 28);
+              lo = nlo; hi = nhi;
+            }
           }
           __syncwarp();
           if (lane == 0) mbar_arrive(&bars->slot_free[b]);
@@ -566,7 +577,7 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
   if (threadIdx.x == 0 && bars->abort_flag) report_timeout(args.status);
 }
 
-template <int MODE>
+template <int MODE, bool PF>
 cudaError_t launch_pair_mode(const GemmProblem* single, const GemmProblem* table, const GemmLaunch& L, int sms,
                              cudaStream_t st) {
   const int tpp = L.symmetric ? L.tiles_n * (L.tiles_n + 1) / 2 : L.tiles_m * L.tiles_n;
@@ -575,7 +586,7 @@ cudaError_t launch_pair_mode(const GemmProblem* single, const GemmProblem* table
   if (pairs > num_tiles) pairs = num_tiles;
   count_launches(1);
   static const GemmProblem kNone = {};
-  k_gemm_pair<MODE><<<2 * pairs, NTHREADS, SMEM_BYTES, st>>>(single ? *single : kNone, table, L);
+  k_gemm_pair<MODE, PF><<<2 * pairs, NTHREADS, SMEM_BYTES, st>>>(single ? *single : kNone, table, L);
   return cudaGetLastError();
 }
 
@@ -583,10 +594,13 @@ cudaError_t launch_pair_mode(const GemmProblem* single, const GemmProblem* table
 
 cudaError_t gemm_pair_set_attributes() {
   cudaError_t e;
-  if ((e = cudaFuncSetAttribute(k_gemm_pair<kPlain>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
-  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG1>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
-  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG2>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
-  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG3>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kPlain, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG3, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG3, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
   return cudaSuccess;
 }
 
@@ -598,11 +612,12 @@ cudaError_t launch_gemm_pair(GemmMode mode, const GemmProblem* single, const Gem
   GemmLaunch L = launch;
   L.tiles_m = launch.tiles_m / 2;
   L.tiles_n = launch.tiles_n / 2;
+  const bool pf = launch.q.rht || launch.q.four_six;
   switch (mode) {
-    case kPlain: return launch_pair_mode<kPlain>(single, table, L, sms, st);
-    case kG1: return launch_pair_mode<kG1>(single, table, L, sms, st);
-    case kG2: return launch_pair_mode<kG2>(single, table, L, sms, st);
-    default: return launch_pair_mode<kG3>(single, table, L, sms, st);
+    case kPlain: return launch_pair_mode<kPlain, false>(single, table, L, sms, st);
+    case kG1: return pf ? launch_pair_mode<kG1, true>(single, table, L, sms, st) : launch_pair_mode<kG1, false>(single, table, L, sms, st);
+    case kG2: return pf ? launch_pair_mode<kG2, true>(single, table, L, sms, st) : launch_pair_mode<kG2, false>(single, table, L, sms, st);
+    default: return pf ? launch_pair_mode<kG3, true>(single, table, L, sms, st) : launch_pair_mode<kG3, false>(single, table, L, sms, st);
   }
 }
 

@@ -49,7 +49,8 @@ __device__ __forceinline__ void decode_tile(int t, const GemmLaunch& L, int tile
 
 // Per-call scalars of an epilogue: the factor that turns the accumulator into the
 // product (tensor scales of the two operands) and the tensor scale of the quantised
-// output, predicted from the running maxima (power of two).
+// output, predicted from the running maxima (power of two); the bound is widened by
+// args.q.widen when the output is rotated before quantisation (|x H| <= 4 amax(x)).
 template <int MODE>
 __device__ __forceinline__ void epilogue_scalars(const GemmProblem& pr, const GemmLaunch& args, float& scale,
                                                  float& sg_out, bool publish) {
@@ -62,14 +63,14 @@ __device__ __forceinline__ void epilogue_scalars(const GemmProblem& pr, const Ge
     const float ax = sc[args.ix.amax_X0 + args.iter];
     scale = __fmul_rn(sgx, sgx);
     float bound = __fmul_rn(__fmul_rn(__fmul_rn(2.0f, args.l_cols), ax), ax);
-    sg_out = scale_predicted(fminf(bound, 4.0f));
+    sg_out = scale_predicted(__fmul_rn(args.q.widen, fminf(bound, 4.0f)));
     if (publish) sc[args.ix.sg_A0 + args.iter] = sg_out;
   } else if (MODE == kG2) {
     const float sga = sc[args.ix.sg_A0 + args.iter];
     const float aa = sc[args.ix.amax_A0 + args.iter];
     scale = __fmul_rn(sga, sga);
     float bound = __fmul_rn(__fadd_rn(fabsf(pr.cb), __fmul_rn(4.0f, fabsf(pr.cc))), aa);
-    sg_out = scale_predicted(bound);
+    sg_out = scale_predicted(__fmul_rn(args.q.widen, bound));
     if (publish) sc[args.ix.sg_B0 + args.iter] = sg_out;
   } else {
     const float sgb = sc[args.ix.sg_B0 + args.iter];
@@ -77,7 +78,7 @@ __device__ __forceinline__ void epilogue_scalars(const GemmProblem& pr, const Ge
     const float ax = sc[args.ix.amax_X0 + args.iter];
     scale = __fmul_rn(sgb, sgx);
     float bound = __fmul_rn(__fmul_rn(4.0f, fabsf(pr.ca)), ax);
-    sg_out = scale_predicted(bound);
+    sg_out = scale_predicted(__fmul_rn(args.q.widen, bound));
     if (publish) sc[args.ix.sg_X0 + args.iter + 1] = sg_out;
   }
 }

@@ -81,6 +81,7 @@ struct GemmLaunch {
   int write_q;         // emit the quantised outputs
   int rq_K, cq_K;      // row lengths (elements) of the two quantised outputs
   float l_cols;        // (float) l, for the bound on amax(A)
+  QuantOpts q;         // how this stage's output is quantised (q.widen = 1 in the base mode)
   NsScalarIdx ix;
   uint32_t* status;
 };
@@ -95,7 +96,7 @@ struct ProfScope {
 };
 
 cudaError_t launch_quantize(const float* x, int64_t rows, int64_t cols, uint8_t* codes, uint8_t* scales,
-                            float* tensor_scale, int sms, cudaStream_t st);
+                            float* tensor_scale, const QuantOpts& q, int sms, cudaStream_t st);
 struct PrologueItem {
   const float* G;
   float* X;
@@ -104,7 +105,8 @@ struct PrologueItem {
   bool clear_status;
 };
 // count matrices that share the shape (s, l) and the clip / eps parameters
-cudaError_t launch_prologue_group(const PrologueItem* items, int count, int write_q, cudaStream_t st);
+cudaError_t launch_prologue_group(const PrologueItem* items, int count, int write_q, const QuantOpts& q,
+                                  cudaStream_t st);
 cudaError_t launch_transpose_out(const float* X, int64_t s, int64_t l, float* out, cudaStream_t st);
 cudaError_t prologue_set_attributes();
 

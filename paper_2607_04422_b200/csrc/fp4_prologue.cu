@@ -51,6 +51,7 @@ struct PrepGroup {
   int stat_blocks;
   int write_q;
   int zero_words;      // 32-bit words of header + scalars + histogram to clear
+  QuantOpts q;         // quantiser options of X0's operand copies
   NsScalarIdx ix;
 };
 
@@ -227,14 +228,14 @@ __device__ __forceinline__ double sum_partials(const double* partial, int nparts
 }
 
 __device__ __forceinline__ void write_norm_scalars(float* scalars, const NsScalarIdx& ix, double sumsq, float maxabs,
-                                                   float eps) {
+                                                   float eps, float widen) {
   const float nu = (float)sqrt(sumsq);
   const float inv = __fdiv_rn(1.0f, __fadd_rn(nu, eps));
   const float amax0 = __fmul_rn(maxabs, inv);
   scalars[ix.nu] = nu;
   scalars[ix.inv] = inv;
   scalars[ix.amax_X0] = amax0;
-  scalars[ix.sg_X0] = scale_exact(amax0);
+  scalars[ix.sg_X0] = scale_exact(__fmul_rn(widen, amax0));
 }
 
 // ---- finish: select tau among the candidates and derive the normalisation scalars
@@ -248,7 +249,8 @@ __global__ void __launch_bounds__(1024) kp_finalize(const __grid_constant__ Prep
   NsHeader* hdr = m.hdr;
   if (!g.clip) {
     const double total = sum_partials(m.partial, g.stat_blocks, shd);
-    if (threadIdx.x == 0) write_norm_scalars(m.scalars, g.ix, total, __uint_as_float(hdr->maxabs_bits), g.eps);
+    if (threadIdx.x == 0) write_norm_scalars(m.scalars, g.ix, total, __uint_as_float(hdr->maxabs_bits), g.eps,
+                                               g.q.widen);
     return;
   }
   const uint32_t count = hdr->cand_count;
@@ -349,7 +351,7 @@ __global__ void __launch_bounds__(1024) kp_finalize(const __grid_constant__ Prep
     const double n_clipped = n_total - (double)hdr->count_below - (double)hdr->bin_count + (double)s_above;
     const double total = below + cand_sq + n_clipped * (double)tau * (double)tau;
     m.scalars[g.ix.tau] = tau;
-    write_norm_scalars(m.scalars, g.ix, total, tau, g.eps);
+    write_norm_scalars(m.scalars, g.ix, total, tau, g.eps, g.q.widen);
     hdr->overflow = 0;
   }
 }
@@ -417,12 +419,13 @@ __global__ void __launch_bounds__(1024) kp_fb_finish(const __grid_constant__ Pre
   if (threadIdx.x == 0) {
     const float tau = __uint_as_float(m.hdr->sel_prefix);
     m.scalars[g.ix.tau] = tau;
-    write_norm_scalars(m.scalars, g.ix, total, tau, g.eps);
+    write_norm_scalars(m.scalars, g.ix, total, tau, g.eps, g.q.widen);
   }
 }
 
 // ---- X0 = clamp(G) * inv in the work orientation (s x l; transposed when G is tall), its FP32
 // copy, and both NVFP4 operand copies.  One 128 x 128 tile of X per block, gridDim.z = matrix.
+template <bool PF>
 __global__ void __launch_bounds__(512) kp_prep_operands(const __grid_constant__ PrepGroup g) {
   extern __shared__ float xs[];  // [128][129]
   constexpr int P = 129;
@@ -471,7 +474,10 @@ __global__ void __launch_bounds__(512) kp_prep_operands(const __grid_constant__ 
 #pragma unroll
       for (int i = 0; i < 16; ++i) v[i] = xs[rr * P + kb * 16 + i];
       uint32_t lo, hi;
-      uint32_t sb = quantize_block16(v, six_sg, sg, lo, hi);
+      uint32_t sb;
+      float unused;
+      if (PF) sb = quantize_block16_opts(v, g.q, sg, lo, hi, unused);
+      else sb = quantize_block16(v, six_sg, sg, lo, hi);
       *reinterpret_cast<uint2*>(m.qx_codes + (r0 + rr) * (l / 2) + (c0 + kb * 16) / 2) = make_uint2(lo, hi);
       sfw |= sb << (8 * q);
     }
@@ -487,7 +493,10 @@ __global__ void __launch_bounds__(512) kp_prep_operands(const __grid_constant__ 
 #pragma unroll
       for (int i = 0; i < 16; ++i) v[i] = xs[(gq * 16 + i) * P + cc];
       uint32_t lo, hi;
-      uint32_t sb = quantize_block16(v, six_sg, sg, lo, hi);
+      uint32_t sb;
+      float unused;
+      if (PF) sb = quantize_block16_opts(v, g.q, sg, lo, hi, unused);
+      else sb = quantize_block16(v, six_sg, sg, lo, hi);
       *reinterpret_cast<uint2*>(m.qt_codes + (c0 + cc) * (s / 2) + (r0 + gq * 16) / 2) = make_uint2(lo, hi);
       sfw |= sb << (8 * q);
     }
@@ -498,11 +507,14 @@ __global__ void __launch_bounds__(512) kp_prep_operands(const __grid_constant__ 
 }  // namespace
 
 cudaError_t prologue_set_attributes() {
-  return cudaFuncSetAttribute(kp_prep_operands, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 129 * 4);
+  cudaError_t e = cudaFuncSetAttribute(kp_prep_operands<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 129 * 4);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(kp_prep_operands<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 129 * 4);
 }
 
 // Enqueue the prologue for `count` matrices of one shape (s, l) and one parameter set.
-cudaError_t launch_prologue_group(const PrologueItem* items, int count, int write_q, cudaStream_t st) {
+cudaError_t launch_prologue_group(const PrologueItem* items, int count, int write_q, const QuantOpts& q,
+                                  cudaStream_t st) {
   for (int i0 = 0; i0 < count; i0 += kMaxPack) {
     const int nn = count - i0 < kMaxPack ? count - i0 : kMaxPack;
     const NsPlan& pl = *items[i0].pl;
@@ -520,6 +532,7 @@ cudaError_t launch_prologue_group(const PrologueItem* items, int count, int writ
     g.write_q = write_q;
     g.zero_words = (int)(pl.zero_bytes / 4);
     g.ix = pl.ix;
+    g.q = q;
     for (int j = 0; j < nn; ++j) {
       const PrologueItem& it = items[i0 + j];
       const fp4_ws_layout& L = it.pl->lay;
@@ -568,7 +581,8 @@ cudaError_t launch_prologue_group(const PrologueItem* items, int count, int writ
     {
       ProfScope ps(FP4_PROF_PREP, st);
       const dim3 gp((unsigned)(pl.l / 128), (unsigned)(pl.s / 128), (unsigned)nn);
-      kp_prep_operands<<<gp, 512, 128 * 129 * 4, st>>>(g);
+      if (q.rht || q.four_six) kp_prep_operands<true><<<gp, 512, 128 * 129 * 4, st>>>(g);
+      else kp_prep_operands<false><<<gp, 512, 128 * 129 * 4, st>>>(g);
       count_launches(1);
     }
     cudaError_t e = cudaGetLastError();

@@ -97,8 +97,34 @@ __global__ void __launch_bounds__(256) k_quantize_rows(const float* __restrict__
     quantize_step(__ldg(src + c / 4 + lane), six_sg, sg, lane, crow + c / 2, srow + (c >> 6) * 512);
 }
 
-__global__ void k_finish_tensor_scale(float* ts) {
-  *ts = scale_exact(*ts);  // amax (bit pattern of a float) -> s_g
+__global__ void k_finish_tensor_scale(float* ts, float widen) {
+  *ts = scale_exact(__fmul_rn(widen, *ts));  // amax (bit pattern of a float) -> s_g
+}
+
+// Row quantiser with the paper-faithful options (Section 3.4): one thread per block of 16
+// (the transform and the two candidate encodings are local to a block), a warp covers 512
+// consecutive elements of a row.  grid: rows x ceil(cols / 4096) thread blocks, row-major.
+__global__ void __launch_bounds__(256) k_quantize_rows_opts(const float* __restrict__ x, int64_t rows, int64_t cols,
+                                                            uint8_t* __restrict__ codes, uint8_t* __restrict__ scales,
+                                                            const uint32_t* __restrict__ amax_bits,
+                                                            const QuantOpts q) {
+  const float sg = scale_exact(__fmul_rn(q.widen, __uint_as_float(*amax_bits)));
+  const int64_t groups = ((cols >> 4) + 255) / 256;  // thread blocks per row
+  const int64_t r = blockIdx.x / groups;
+  const int64_t kb = (blockIdx.x % groups) * 256 + threadIdx.x;
+  if (r >= rows || kb >= (cols >> 4)) return;
+  const float4* src = reinterpret_cast<const float4*>(x + r * cols + kb * 16);
+  float v[16];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const float4 t = __ldg(src + j);
+    v[4 * j] = t.x; v[4 * j + 1] = t.y; v[4 * j + 2] = t.z; v[4 * j + 3] = t.w;
+  }
+  uint32_t lo, hi;
+  float unused;
+  const uint32_t sb = quantize_block16_opts(v, q, sg, lo, hi, unused);
+  *reinterpret_cast<uint2*>(codes + r * (cols / 2) + kb * 8) = make_uint2(lo, hi);
+  scales[sf_offset(r, kb, cols >> 4)] = (uint8_t)sb;
 }
 
 // out (m x n, m > n) = X^T where X is n x m: 32 x 32 tiles through shared memory
@@ -122,16 +148,22 @@ static int grid_for(int64_t n4, int threads, int sms) {
 }
 
 cudaError_t launch_quantize(const float* x, int64_t rows, int64_t cols, uint8_t* codes, uint8_t* scales,
-                            float* tensor_scale, int sms, cudaStream_t st) {
+                            float* tensor_scale, const QuantOpts& q, int sms, cudaStream_t st) {
   const int64_t n4 = rows * cols / 4;
   cudaError_t e = cudaMemsetAsync(tensor_scale, 0, 4, st);
   if (e != cudaSuccess) return e;
   k_amax<<<grid_for(n4, 256 * 8, sms), 256, 0, st>>>(reinterpret_cast<const float4*>(x), n4,
                                                     reinterpret_cast<uint32_t*>(tensor_scale));
-  const dim3 qgrid((unsigned)((cols + kSegment - 1) / kSegment), (unsigned)((rows + 7) / 8));
-  k_quantize_rows<<<qgrid, 256, 0, st>>>(x, rows, cols, codes, scales,
-                                         reinterpret_cast<const uint32_t*>(tensor_scale));
-  k_finish_tensor_scale<<<1, 1, 0, st>>>(tensor_scale);
+  if (q.rht || q.four_six) {
+    const unsigned qgrid = (unsigned)(((cols / 16 + 255) / 256) * rows);
+    k_quantize_rows_opts<<<qgrid, 256, 0, st>>>(x, rows, cols, codes, scales,
+                                                reinterpret_cast<const uint32_t*>(tensor_scale), q);
+  } else {
+    const dim3 qgrid((unsigned)((cols + kSegment - 1) / kSegment), (unsigned)((rows + 7) / 8));
+    k_quantize_rows<<<qgrid, 256, 0, st>>>(x, rows, cols, codes, scales,
+                                           reinterpret_cast<const uint32_t*>(tensor_scale));
+  }
+  k_finish_tensor_scale<<<1, 1, 0, st>>>(tensor_scale, q.widen);
   count_launches(3);
   return cudaGetLastError();
 }

@@ -134,6 +134,26 @@ void default_params(fp4_ns_params* p) {
   p->eps = 1e-7f;
   p->flags = 0;
   p->max_group = 0;
+  p->seed = 0;
+}
+
+// The 16 signs of the j-th random Hadamard matrix of a call: splitmix64 on seed + j.
+uint32_t rht_signs(uint64_t seed, uint64_t j) {
+  uint64_t z = seed + 0x9E3779B97F4A7C15ull * (j + 1);
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  z ^= z >> 31;
+  return (uint32_t)(z & 0xFFFFu);
+}
+
+// Quantiser options of the j-th product of a call.
+QuantOpts quant_opts(const fp4_ns_params* p, uint64_t j) {
+  QuantOpts q;
+  q.rht = (p->flags & FP4_FLAG_RHT) ? 1u : 0u;
+  q.four_six = (p->flags & FP4_FLAG_FOUR_SIX) ? 1u : 0u;
+  q.mask = q.rht ? rht_signs(p->seed, j) : 0u;
+  q.widen = q.rht ? 4.0f : 1.0f;
+  return q;
 }
 
 int64_t quantile_rank(int64_t n, float q) {
@@ -295,7 +315,8 @@ fp4_status run_group(const DeviceInfo* d, MatrixCtx* mats, int count, int steps,
       MatrixCtx& c = mats[i];
       items[(size_t)i] = PrologueItem{c.G, c.X, c.ws, &c.pl, clear_first_status && i == 0};
     }
-    if (launch_prologue_group(items.data(), count, steps > 0 || keep, st) != cudaSuccess) return FP4_ERR_CUDA;
+    if (launch_prologue_group(items.data(), count, steps > 0 || keep, quant_opts(p, 0), st) != cudaSuccess)
+      return FP4_ERR_CUDA;
   }
   if (steps > 0) {
     const GemmProblem* tabs[4] = {nullptr, nullptr, nullptr, nullptr};
@@ -329,6 +350,7 @@ fp4_status run_group(const DeviceInfo* d, MatrixCtx* mats, int count, int steps,
       GemmLaunch L1 = base;
       L1.iter = k; L1.K = (int)l; L1.tiles_m = L1.tiles_n = (int)(s / 128); L1.symmetric = 1;
       L1.rq_K = L1.cq_K = (int)s; L1.write_q = 1;
+      L1.q = quant_opts(p, 2 * (uint64_t)k + 1);  // qA_k
       {
         ProfScope ps(FP4_PROF_G1, st);
         if (launch_gemm_auto(kG1, count == 1 ? &mats[0].g1 : nullptr, tabs[0], L1, d->sms, st) != cudaSuccess)
@@ -336,6 +358,7 @@ fp4_status run_group(const DeviceInfo* d, MatrixCtx* mats, int count, int steps,
       }
       GemmLaunch L2 = L1;
       L2.K = (int)s;
+      L2.q = quant_opts(p, 2 * (uint64_t)k);      // qB_k meets qX_k^{16x1}
       {
         ProfScope ps(FP4_PROF_G2, st);
         if (launch_gemm_auto(kG2, count == 1 ? &mats[0].g2 : nullptr, tabs[1], L2, d->sms, st) != cudaSuccess)
@@ -345,6 +368,7 @@ fp4_status run_group(const DeviceInfo* d, MatrixCtx* mats, int count, int steps,
       L3.iter = k; L3.K = (int)s; L3.tiles_m = (int)(s / 128); L3.tiles_n = (int)(l / 128); L3.symmetric = 0;
       L3.rq_K = (int)l; L3.cq_K = (int)s;
       L3.write_q = (!last || keep) ? 1 : 0;
+      L3.q = quant_opts(p, 2 * (uint64_t)k + 2);  // both copies of X_{k+1}
       {
         ProfScope ps(FP4_PROF_G3, st);
         if (launch_gemm_auto(kG3, count == 1 ? &mats[0].g3[cur] : nullptr, tabs[2 + cur], L3, d->sms, st) != cudaSuccess)
@@ -406,7 +430,14 @@ size_t fp4_scale_bytes(int64_t rows, int64_t cols) {
 
 fp4_status fp4_quantize(const float* x, int64_t rows, int64_t cols, uint8_t* codes, uint8_t* scales,
                         float* tensor_scale, uint32_t flags, cudaStream_t stream) {
-  if (!x || !codes || !scales || !tensor_scale || flags != 0) return FP4_ERR_INVALID_ARG;
+  if (!x || !codes || !scales || !tensor_scale) return FP4_ERR_INVALID_ARG;
+  if (flags & 0xFFFFu & ~(FP4_FLAG_RHT | FP4_FLAG_FOUR_SIX)) return FP4_ERR_INVALID_ARG;
+  if (!(flags & FP4_FLAG_RHT) && (flags >> 16)) return FP4_ERR_INVALID_ARG;
+  QuantOpts q;
+  q.rht = (flags & FP4_FLAG_RHT) ? 1u : 0u;
+  q.four_six = (flags & FP4_FLAG_FOUR_SIX) ? 1u : 0u;
+  q.mask = flags >> 16;
+  q.widen = q.rht ? 4.0f : 1.0f;
   if (!shape_ok(rows) || !shape_ok(cols)) return FP4_ERR_SHAPE;
   if (!aligned(x, 16) || !aligned(codes, 16) || !aligned(scales, 16) || !aligned(tensor_scale, 4))
     return FP4_ERR_ALIGNMENT;
@@ -414,7 +445,7 @@ fp4_status fp4_quantize(const float* x, int64_t rows, int64_t cols, uint8_t* cod
   fp4_status rc = check_common(&d);
   if (rc != FP4_OK) return rc;
   ProfScope ps(FP4_PROF_QUANTIZE, stream);
-  return launch_quantize(x, rows, cols, codes, scales, tensor_scale, d->sms, stream) == cudaSuccess ? FP4_OK
+  return launch_quantize(x, rows, cols, codes, scales, tensor_scale, q, d->sms, stream) == cudaSuccess ? FP4_OK
                                                                                                       : FP4_ERR_CUDA;
 }
 

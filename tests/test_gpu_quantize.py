@@ -6,18 +6,19 @@ import torch
 import oracle
 import paper_2607_04422_b200 as fp4
 from paper_2607_04422_b200 import workloads
+from paper_2607_04422_b200.binding import FP4_FLAG_FOUR_SIX, FP4_FLAG_RHT
 from helpers import mismatch_report, sf_from_atoms
 
 pytestmark = pytest.mark.gpu
 
 
-def _run(x_np):
+def _run(x_np, flags=0):
     rows, cols = x_np.shape
     x = torch.from_numpy(x_np).cuda()
     codes = torch.empty((rows, cols // 2), dtype=torch.uint8, device="cuda")
     scales = torch.zeros(fp4.fp4_scale_bytes(rows, cols), dtype=torch.uint8, device="cuda")
     ts = torch.zeros(1, dtype=torch.float32, device="cuda")
-    fp4.fp4_quantize(x, codes, scales, ts)
+    fp4.fp4_quantize(x, codes, scales, ts, flags=flags)
     torch.cuda.synchronize()
     return codes.cpu().numpy(), sf_from_atoms(scales.cpu().numpy(), rows, cols // 16), float(ts.item())
 
@@ -77,6 +78,45 @@ def test_large_tensor_sampled_rows():
     assert np.array_equal(c[rows], oc) and np.array_equal(s[rows], os_)
 
 
+@pytest.mark.parametrize("rht,four_six", [(True, False), (False, True), (True, True)])
+@pytest.mark.parametrize("gen,shape", [
+    (workloads.gaussian, (256, 512)),
+    (workloads.row_lognormal, (384, 1024)),
+    (workloads.gradient_like, (128, 4224)),     # a row is longer than one thread block covers
+])
+def test_paper_faithful_options_bit_exact(gen, shape, rht, four_six):
+    """Random Hadamard transform and adaptive 4/6 (Section 3.4): the transform's butterfly
+    order and the order of the error sums are part of the definition, so codes, block
+    scales and the tensor scale agree bit for bit."""
+    x = gen(*shape, seed=5)
+    mask = oracle.rht_mask(17, 3) if rht else 0
+    flags = (FP4_FLAG_RHT | (mask << 16) if rht else 0) | (FP4_FLAG_FOUR_SIX if four_six else 0)
+    c, s, sg = _run(x, flags)
+    oc, os_, osg = oracle.quantize(x, rht=rht, mask=mask, four_six=four_six)
+    assert np.float32(sg) == np.float32(osg)
+    assert np.array_equal(s, os_), mismatch_report(s, os_)
+    assert np.array_equal(c, oc), mismatch_report(c, oc)
+    if four_six:
+        base = oracle.quantize(x, rht=rht, mask=mask)
+        assert (s != base[1]).mean() > 0.05      # the 4-mapping is really taken
+
+
+def test_paper_faithful_options_edge_blocks():
+    """Blocks whose two candidate encodings tie or underflow."""
+    x = np.zeros((128, 128), np.float32)
+    x[0, :16] = [6, 3, 1.5, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0]        # tie: keeps the 6-mapping
+    x[1, :16] = [4, 3, 2, 1, 0.5, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, -4]       # the 4-mapping is exact
+    x[2, :16] = 1e-9                                                       # block scale underflows to 0
+    x[3, 16:32] = np.float32(2688.0)                                       # sets the tensor scale to 1
+    x[4, :16] = 5.0 / 1024                                                  # 6-scale 0, 4-scale the smallest subnormal
+    c, s, sg = _run(x, FP4_FLAG_FOUR_SIX)
+    oc, os_, osg = oracle.quantize(x, four_six=True)
+    assert sg == osg == 1.0
+    assert np.array_equal(s, os_), mismatch_report(s, os_)
+    assert np.array_equal(c, oc), mismatch_report(c, oc)
+    assert s[0, 0] == 0x38 and s[1, 0] == 0x38 and s[2, 0] == 0 and s[4, 0] == 1
+
+
 def test_argument_errors():
     x = torch.zeros((128, 128), device="cuda")
     codes = torch.empty((128, 64), dtype=torch.uint8, device="cuda")
@@ -87,4 +127,7 @@ def test_argument_errors():
     assert e.value.code == 2
     with pytest.raises(fp4.Fp4Error) as e:
         fp4.fp4_quantize(x, codes, scales, ts, flags=7)
+    assert e.value.code == 1
+    with pytest.raises(fp4.Fp4Error) as e:       # sign bits without the transform flag
+        fp4.fp4_quantize(x, codes, scales, ts, flags=FP4_FLAG_FOUR_SIX | (0x1234 << 16))
     assert e.value.code == 1

