@@ -42,12 +42,17 @@ constexpr int RING_HALF = RING / 2;
 
 // Two consecutive tiles use two accumulator buffers that share OV_CHUNKS chunks of tensor
 // memory (512 columns cannot hold two 256-column accumulators plus the scale factors):
-// buffer 0 = columns [0, 256), buffer 1 = columns [208, 464), scale factors [464, 512).
-// The shared columns are buffer 0's last three chunks and buffer 1's first three; the half
-// that owns them drains them first and reports it, then the next tile's MMAs may start
-// while the rest of the tile is still being drained.
-constexpr int OV_CHUNKS = 3;
-constexpr uint32_t ACC1_COL = PN - OV_CHUNKS * CHUNK;  // 208
+// buffer 0 = columns [0, 256), buffer 1 = columns [240, 496), scale factors [496, 508).
+// The shared columns are buffer 0's last chunk and buffer 1's first; the half that owns them
+// drains them first and reports it, then the next tile's MMAs may start while the rest of
+// the tile is still being drained.  The time from "accumulator complete" to that report is
+// on the critical path of every tile (drain of the shared chunk, then the next main loop),
+// which is why the scale factors get only the 12 columns one MMA needs.
+#ifndef FP4_OV_CHUNKS
+#define FP4_OV_CHUNKS 1
+#endif
+constexpr int OV_CHUNKS = FP4_OV_CHUNKS;
+constexpr uint32_t ACC1_COL = PN - OV_CHUNKS * CHUNK;  // 240
 
 // chunk handled at position i (0..7) by column half h in a tile that uses buffer `par`
 __device__ __forceinline__ int half_chunk(int par, int h, int i) {
@@ -74,9 +79,10 @@ static_assert(SMEM_BYTES <= 232448, "at most 227 KB of dynamic shared memory");
 constexpr int NTHREADS = 640;  // warp roles as in the single-CTA kernel
 constexpr uint32_t TMEM_COLS = 512;
 constexpr uint32_t TMEM_SF_COL = ACC1_COL + PN;  // scale factors after the second accumulator buffer
-constexpr uint32_t SF_COLS = KSTEPS * 12;      // per stage: 4 columns (row operand) + 8 (column operand) per MMA
-constexpr int SF_SLOTS = 1;                    // copies and MMAs execute in issue order: one slot suffices
-static_assert(TMEM_SF_COL + SF_SLOTS * SF_COLS <= 512, "tensor memory columns");
+// Scale factors of ONE MMA (K = 64): 4 columns (row operand) + 8 (column operand, N = 256).  Copies and
+// MMAs execute in issue order, so the copies for the next MMA may target the same columns.
+constexpr uint32_t SF_COLS = 12;
+static_assert(TMEM_SF_COL + SF_COLS <= 512, "tensor memory columns");
 
 // instruction descriptor: E2M1 x E2M1, UE4M3 scales, K-major operands, M = 256 (pair), N = 256
 constexpr uint32_t IDESC = (1u << 7) | (1u << 10) | ((uint32_t)(PN >> 3) << 17) | ((uint32_t)(PM >> 4) << 24);
@@ -109,8 +115,12 @@ __device__ __forceinline__ uint32_t map_to_cta(const void* p, uint32_t rank) {
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_u32(p)), "r"(rank));
   return r;
 }
+// Arrive on a barrier of (possibly) the peer CTA.  Relaxed: the barriers signalled this way guard
+// tensor memory that the arriving warp has finished reading (tcgen05.wait::ld has returned), not data
+// in memory; a release at cluster scope would first wait for all of the thread's earlier global
+// stores to be performed, thousands of cycles on the critical path of every tile.
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+  asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
 }
 // TMA load whose completion bytes are credited to a barrier that may live in the peer CTA
 __device__ __forceinline__ void tma_load_2d_pair(void* smem_dst, const void* tmap, int x, int y, uint32_t bar_cluster) {
@@ -225,7 +235,7 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer (even CTA only)
     if (leader && elect_one()) {
-      int st = 0; uint32_t ph = 0, seq = 0, kstage = 0; bool ok = true;
+      int st = 0; uint32_t ph = 0, seq = 0; bool ok = true;
       for (int t = pair; t < num_tiles && ok; t += num_pairs, ++seq) {
         const uint32_t par = seq & 1, buse = seq >> 1;
         // this buffer's previous tile is drained, and so are the columns it shares with the
@@ -234,23 +244,19 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
         if (seq > 0 && !wait_bar(&bars->ov_free, (seq - 1) & 1, abort_flag)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + par * ACC1_COL;
-        for (int kb = 0; kb < num_kb; ++kb, ++kstage) {
+        for (int kb = 0; kb < num_kb; ++kb) {
           if (!wait_bar(&bars->full[st], ph, abort_flag)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t sf_t = tmem_base + TMEM_SF_COL + (kstage % SF_SLOTS) * SF_COLS;
+          const uint32_t sf_t = tmem_base + TMEM_SF_COL;
           const uint8_t* sf = smem + OFF_SF + st * SF_BYTES;
-#pragma unroll
-          for (int a = 0; a < KSTEPS; ++a) {
-            tc_cp_sf2(sf_t + a * 4, umma_desc(smem_u32(sf + a * 512), 128, 0));
-            tc_cp_sf2(sf_t + KSTEPS * 4 + a * 8, umma_desc(smem_u32(sf + SF_ATOMS + a * 512), 128, 0));
-            tc_cp_sf2(sf_t + KSTEPS * 4 + a * 8 + 4, umma_desc(smem_u32(sf + 2 * SF_ATOMS + a * 512), 128, 0));
-          }
           const uint64_t adesc = umma_desc(smem_u32(smem + OFF_A + st * OPER_BYTES), 1024, 2);
           const uint64_t bdesc = umma_desc(smem_u32(smem + OFF_B + st * OPER_BYTES), 1024, 2);
 #pragma unroll
           for (int k = 0; k < KSTEPS; ++k) {
-            tc_mma_nvf4_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC, sf_t + k * 4,
-                             sf_t + KSTEPS * 4 + k * 8, (kb | k) != 0 ? 1u : 0u);
+            tc_cp_sf2(sf_t, umma_desc(smem_u32(sf + k * 512), 128, 0));
+            tc_cp_sf2(sf_t + 4, umma_desc(smem_u32(sf + SF_ATOMS + k * 512), 128, 0));
+            tc_cp_sf2(sf_t + 8, umma_desc(smem_u32(sf + 2 * SF_ATOMS + k * 512), 128, 0));
+            tc_mma_nvf4_pair(d_tmem, adesc + 2 * k, bdesc + 2 * k, IDESC, sf_t, sf_t + 4, (kb | k) != 0 ? 1u : 0u);
           }
           tc_commit_pair(&bars->empty[st]);
           if (++st == STAGES) { st = 0; ph ^= 1; }
@@ -268,6 +274,8 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
       const uint32_t total = my_tiles * HALF_CHUNKS;
       uint32_t n[2] = {0, 0}, seq_dec[2] = {0xFFFFFFFFu, 0xFFFFFFFFu};
       int pp[2] = {0, 0}, tis[2] = {0, 0}, tjs[2] = {0, 0};
+      uint32_t pf_seq[2] = {0xFFFFFFFFu, 0xFFFFFFFFu};
+      int pf_p[2] = {0, 0}, pf_ti[2] = {0, 0}, pf_tj[2] = {0, 0};
       uint32_t idle = 0;
       uint64_t t_idle = 0;
       while ((n[0] < total || n[1] < total)) {
@@ -295,6 +303,26 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
             mbar_expect_tx(&bars->aux_full[b], CHUNK_BYTES);
             tma_load_2d(smem + OFF_RING + b * CHUNK_BYTES, &pr->tmAux, tjs[h] * PN + c * CHUNK, bi * BM, &bars->aux_full[b]);
           }
+#ifndef FP4_NO_AUX_PREFETCH
+          // Ahead of its use, pull this CTA's part of the next tile's FP32 operand into L2 in
+          // whole 1 KB row segments (the chunk loads above touch only 64 bytes of a row at a
+          // time, which DRAM serves poorly): each of the 16 chunk loads of a tile prefetches 8 rows.
+          {
+            const int tn = pair + (int)(seq + 1) * num_pairs;
+            if (tn < num_tiles) {
+              if (pf_seq[h] != seq + 1) {
+                decode_tile(tn, args, tiles_per_problem, pf_p[h], pf_ti[h], pf_tj[h]);
+                pf_seq[h] = seq + 1;
+              }
+              const GemmProblem* pn = probs + pf_p[h];
+              const int part = h * HALF_CHUNKS + i;  // 0..15
+              const float* src = pn->aux + ((int64_t)(pf_ti[h] * 2 + (int)rank) * BM + part * 8) * pn->aux_ld +
+                                 (int64_t)pf_tj[h] * PN;
+#pragma unroll
+              for (int r = 0; r < 8; ++r) l2_prefetch(src + r * pn->aux_ld, PN * 4);
+            }
+          }
+#endif
           ++n[h];
           progressed = true;
         }
