@@ -81,6 +81,36 @@ __device__ __forceinline__ uint32_t quantize_block16(const float (&v)[16], float
   return sb;
 }
 
+// Packed FP32 pairs: sm_100 multiplies two FP32 lanes per instruction, each lane rounded to
+// nearest like the scalar operation.  Only used where the product feeds a conversion: a packed
+// multiply followed by a packed add was seen to be contracted into a fused multiply-add, which
+// changes the rounding the method defines.
+__device__ __forceinline__ uint64_t pack2(float a, float b) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t r, float& a, float& b) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(r));
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+// Four FP32 -> two bytes of E2M1 codes (a in bits 3:0, b in 7:4, c in 11:8, d in 15:12).
+__device__ __forceinline__ uint32_t cvt_e2m1x4(float a, float b, float c, float d) {
+  uint32_t r;
+  asm("{\n\t.reg .b8 t0, t1;\n\t.reg .b16 h;\n\t"
+      "cvt.rn.satfinite.e2m1x2.f32 t0, %2, %1;\n\t"
+      "cvt.rn.satfinite.e2m1x2.f32 t1, %4, %3;\n\t"
+      "mov.b16 h, {t0, t1};\n\t"
+      "cvt.u32.u16 %0, h;\n\t}"
+      : "=r"(r)
+      : "f"(a), "f"(b), "f"(c), "f"(d));
+  return r;
+}
+
 // The same quantisation when the tensor scale is a power of two (every tensor produced
 // inside the Newton-Schulz loop), with the two IEEE divisions replaced by exact equivalents:
 //   amax / (6 sg)  = RN(amax / 6) * (1/sg): the division by the constant 6 is one multiply
@@ -105,17 +135,27 @@ __device__ __forceinline__ uint32_t quantize_block16_pow2(const float (&v)[16], 
   const float r = __fmaf_rn(-q, 6.0f, amax);
   q = __fmaf_rn(r, sixth, q);                          // RN(amax / 6)
   const uint32_t sb = cvt_ue4m3(__fmul_rn(q, inv_sg));
-  lo = 0; hi = 0;
-  if (sb != 0) {
-    const uint32_t e = sb >> 3;
-    const float rcp = e != 0 ? __uint_as_float(kRcpMantissa[sb & 7] + rcp_base - (e << 23))
-                             : __frcp_rn(__fmul_rn(ue4m3_to_float(sb), sg));
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      lo |= cvt_e2m1x2(__fmul_rn(v[2 * i], rcp), __fmul_rn(v[2 * i + 1], rcp)) << (8 * i);
-      hi |= cvt_e2m1x2(__fmul_rn(v[8 + 2 * i], rcp), __fmul_rn(v[9 + 2 * i], rcp)) << (8 * i);
-    }
+  const uint32_t e = sb >> 3;
+  // scale bytes below 8 (E4M3 subnormals, zero included) are rare: keep their division out of
+  // the common path of the warp
+  float rcp = __uint_as_float(kRcpMantissa[sb & 7] + rcp_base - (e << 23));
+  if (__any_sync(0xffffffffu, e == 0)) {
+    if (e == 0) rcp = sb ? __frcp_rn(__fmul_rn(ue4m3_to_float(sb), sg)) : 0.0f;
   }
+  // y = v * rcp, two lanes per instruction; an all-zero block (rcp = 0) gets codes 0 with the
+  // sign bits of its elements cleared below
+  const uint64_t rcp2 = pack2(rcp, rcp);
+  uint32_t w[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float a, b, c, d;
+    unpack2(mul2(pack2(v[4 * i], v[4 * i + 1]), rcp2), a, b);
+    unpack2(mul2(pack2(v[4 * i + 2], v[4 * i + 3]), rcp2), c, d);
+    w[i] = cvt_e2m1x4(a, b, c, d);
+  }
+  lo = w[0] | (w[1] << 16);
+  hi = w[2] | (w[3] << 16);
+  if (sb == 0) { lo = 0; hi = 0; }
   return sb;
 }
 // rcp_base of a power-of-two tensor scale
@@ -298,10 +338,6 @@ __device__ __forceinline__ void bulk_load_1d(void* smem_dst, const void* gsrc, u
           smem_u32(smem_dst)),
       "l"(gsrc), "r"(bytes), "r"(smem_u32(bar))
       : "memory");
-}
-// hint: bring `bytes` (a multiple of 16, 16-byte aligned) of global memory into L2
-__device__ __forceinline__ void l2_prefetch(const void* gsrc, uint32_t bytes) {
-  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(gsrc), "r"(bytes) : "memory");
 }
 __device__ __forceinline__ void tma_store_2d(const void* tmap, int x, int y, const void* smem_src) {
   asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];" ::"l"(

@@ -7,10 +7,15 @@
 // 128 x 128 single-CTA kernel, whose main loop is bound by exactly that traffic.
 //
 // Per CTA: accumulator 128 lanes x 256 FP32 columns in tensor memory, drained in sixteen
-// 16-column chunks through the same mbarrier-connected ring pipeline as the single-CTA
-// kernel.  Only the even CTA of a pair issues MMAs; both CTAs run every other role on
-// their own 128 rows.  TMA loads of both CTAs signal the even CTA's stage barrier; MMA
-// completion is multicast to the stage and accumulator barriers of both CTAs.
+// 16-column chunks by sixteen epilogue warps: four teams of four warps, a team owns four
+// chunks of a tile, a warp of a team the 32 accumulator lanes of its quadrant.  For one chunk
+// a warp combines its 32 x 16 block with the FP32 tile, quantises it along the rows, stages
+// it in shared memory for the TMA store and, reading its own block back column-wise,
+// quantises it down the columns (the transposed / mirrored operand copy): both
+// quantisations of a block stay inside one warp, no hand-over between warps.  Only the even
+// CTA of a pair issues MMAs; both CTAs run every other role on their own 128 rows.  TMA
+// loads of both CTAs signal the even CTA's stage barrier; MMA completion is multicast to the
+// stage and accumulator barriers of both CTAs.
 #include "fp4_gemm_common.cuh"
 
 namespace fp4 {
@@ -36,9 +41,10 @@ constexpr uint32_t STAGE_BYTES_CTA = 2 * OPER_BYTES + SF_BYTES;
 constexpr int CHUNK = 16;
 constexpr int CHUNK_BYTES = BM * CHUNK * 4;    // 8 KB
 constexpr int NCHUNK = PN / CHUNK;             // 16
-constexpr int HALF_CHUNKS = NCHUNK / 2;
-static_assert(RING % 2 == 0, "the ring is split between the two column halves of a tile");
-constexpr int RING_HALF = RING / 2;
+constexpr int TEAMS = 4;                       // epilogue teams (of four warps) per CTA
+constexpr int TEAM_CHUNKS = NCHUNK / TEAMS;    // 4: one 64-column group, one 32-bit word of row scales
+static_assert(RING % TEAMS == 0, "the ring is split between the teams");
+constexpr int RING_TEAM = RING / TEAMS;
 
 // Two consecutive tiles use two accumulator buffers that share OV_CHUNKS chunks of tensor
 // memory (512 columns cannot hold two 256-column accumulators plus the scale factors):
@@ -54,18 +60,22 @@ constexpr int RING_HALF = RING / 2;
 constexpr int OV_CHUNKS = FP4_OV_CHUNKS;
 constexpr uint32_t ACC1_COL = PN - OV_CHUNKS * CHUNK;  // 240
 
-// chunk handled at position i (0..7) by column half h in a tile that uses buffer `par`
-__device__ __forceinline__ int half_chunk(int par, int h, int i) {
-  if (par == 0 && h == 1) return i < OV_CHUNKS ? NCHUNK - OV_CHUNKS + i : HALF_CHUNKS + (i - OV_CHUNKS);
-  return h * HALF_CHUNKS + i;
+static_assert(OV_CHUNKS <= TEAM_CHUNKS, "the shared chunks belong to one team");
+static_assert(TEAM_CHUNKS == 4, "a team writes one 32-bit word of row scales per row and tile");
+// chunk handled at position i by team t in a tile that uses buffer `par`: buffer 0 shares its
+// last chunks, which the last team therefore takes first; buffer 1 shares its first chunks
+__device__ __forceinline__ int team_chunk(int par, int t, int i) {
+  if (par == 0 && t == TEAMS - 1)
+    return i < OV_CHUNKS ? NCHUNK - OV_CHUNKS + i : t * TEAM_CHUNKS + (i - OV_CHUNKS);
+  return t * TEAM_CHUNKS + i;
 }
-// Ring slot and use count of position i of half h in the seq-th tile of this CTA.  Each
-// column half has its own slots, used strictly in order by that half's drain and finish
-// warps, so every waiter sees every phase of the barriers it waits on.
-__device__ __forceinline__ void chunk_slot(uint32_t seq, int h, int i, int& b, uint32_t& use) {
-  const uint32_t j = seq * HALF_CHUNKS + (uint32_t)i;
-  b = h * RING_HALF + (int)(j % RING_HALF);
-  use = j / RING_HALF;
+// Ring slot and use count of position i of team t in the seq-th tile of this CTA.  Each team
+// has its own slots, used strictly in order, so every waiter sees every phase of the
+// barriers it waits on.
+__device__ __forceinline__ void chunk_slot(uint32_t seq, int t, int i, int& b, uint32_t& use) {
+  const uint32_t j = seq * TEAM_CHUNKS + (uint32_t)i;
+  b = t * RING_TEAM + (int)(j % RING_TEAM);
+  use = j / RING_TEAM;
 }
 
 constexpr int OFF_A = 0;
@@ -76,7 +86,7 @@ constexpr int OFF_BAR = OFF_RING + RING * CHUNK_BYTES;
 constexpr int SMEM_BYTES = OFF_BAR + 512 + 1024;
 static_assert(SMEM_BYTES <= 232448, "at most 227 KB of dynamic shared memory");
 
-constexpr int NTHREADS = 640;  // warp roles as in the single-CTA kernel
+constexpr int NTHREADS = 128 + TEAMS * 128;  // four single-thread roles, then the epilogue teams
 constexpr uint32_t TMEM_COLS = 512;
 constexpr uint32_t TMEM_SF_COL = ACC1_COL + PN;  // scale factors after the second accumulator buffer
 // Scale factors of ONE MMA (K = 64): 4 columns (row operand) + 8 (column operand, N = 256).  Copies and
@@ -91,7 +101,7 @@ struct Barriers {
   uint64_t full[STAGES];     // even CTA: both CTAs' operand bytes of a stage have landed
   uint64_t empty[STAGES];    // stage consumed (MMA commit, multicast to both CTAs)
   uint64_t acc_full[2];      // accumulator buffer complete (MMA commit, multicast)
-  uint64_t acc_empty[2];     // even CTA: buffer drained by the 16 drain warps of the pair
+  uint64_t acc_empty[2];     // even CTA: buffer drained by all epilogue warps of the pair
   uint64_t ov_free;          // even CTA: the columns shared with the other buffer are drained (8 warps)
   uint64_t aux_full[RING];
   uint64_t v_ready[RING];
@@ -187,7 +197,7 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < STAGES; ++i) { mbar_init(&bars->full[i], 1); mbar_init(&bars->empty[i], 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&bars->acc_full[i], 1); mbar_init(&bars->acc_empty[i], 16); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&bars->acc_full[i], 1); mbar_init(&bars->acc_empty[i], 2 * 4 * TEAMS); }
     mbar_init(&bars->ov_free, 8);
     for (int i = 0; i < RING; ++i) {
       mbar_init(&bars->aux_full[i], 1);
@@ -267,24 +277,24 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
     }
   } else if (warp == 2) {
     // ------------------------------------------------------------ producer of the FP32 tile
-    // One thread serves the rings of both column halves without blocking on either: it
-    // polls the next slot of each half in turn and loads a chunk as soon as its slot is free.
+    // One thread serves the rings of all teams without blocking on any: it polls the next
+    // slot of each team in turn and loads a chunk as soon as its slot is free.
     if (HAS_AUX && elect_one()) {
       const uint32_t my_tiles = pair < num_tiles ? (uint32_t)((num_tiles - pair + num_pairs - 1) / num_pairs) : 0u;
-      const uint32_t total = my_tiles * HALF_CHUNKS;
-      uint32_t n[2] = {0, 0}, seq_dec[2] = {0xFFFFFFFFu, 0xFFFFFFFFu};
-      int pp[2] = {0, 0}, tis[2] = {0, 0}, tjs[2] = {0, 0};
-      uint32_t pf_seq[2] = {0xFFFFFFFFu, 0xFFFFFFFFu};
-      int pf_p[2] = {0, 0}, pf_ti[2] = {0, 0}, pf_tj[2] = {0, 0};
-      uint32_t idle = 0;
+      const uint32_t total = my_tiles * TEAM_CHUNKS;
+      uint32_t n[TEAMS], seq_dec[TEAMS];
+      int pp[TEAMS], tis[TEAMS], tjs[TEAMS];
+#pragma unroll
+      for (int h = 0; h < TEAMS; ++h) { n[h] = 0; seq_dec[h] = 0xFFFFFFFFu; pp[h] = tis[h] = tjs[h] = 0; }
+      uint32_t idle = 0, done = 0;
       uint64_t t_idle = 0;
-      while ((n[0] < total || n[1] < total)) {
+      while (done < TEAMS * total) {
         bool progressed = false;
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
+        for (int h = 0; h < TEAMS; ++h) {
           if (n[h] >= total) continue;
-          const uint32_t seq = n[h] / HALF_CHUNKS;
-          const int i = (int)(n[h] % HALF_CHUNKS);
+          const uint32_t seq = n[h] / TEAM_CHUNKS;
+          const int i = (int)(n[h] % TEAM_CHUNKS);
           int b; uint32_t use;
           chunk_slot(seq, h, i, b, use);
           if (!mbar_try_wait(&bars->slot_free[b], (use & 1) ^ 1)) continue;
@@ -294,7 +304,7 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
           }
           const GemmProblem* pr = probs + pp[h];
           const int bi = tis[h] * 2 + (int)rank;
-          const int c = half_chunk((int)(seq & 1), h, i);
+          const int c = team_chunk((int)(seq & 1), h, i);
           const int bj = tjs[h] * 2 + c / 8;
           if (args.symmetric && bj < bi) {
             // a 128 x 128 block below the diagonal: nothing to combine, the slot is passed on empty
@@ -303,30 +313,14 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
             mbar_expect_tx(&bars->aux_full[b], CHUNK_BYTES);
             tma_load_2d(smem + OFF_RING + b * CHUNK_BYTES, &pr->tmAux, tjs[h] * PN + c * CHUNK, bi * BM, &bars->aux_full[b]);
           }
-#ifndef FP4_NO_AUX_PREFETCH
-          // Ahead of its use, pull this CTA's part of the next tile's FP32 operand into L2 in
-          // whole 1 KB row segments (the chunk loads above touch only 64 bytes of a row at a
-          // time, which DRAM serves poorly): each of the 16 chunk loads of a tile prefetches 8 rows.
-          {
-            const int tn = pair + (int)(seq + 1) * num_pairs;
-            if (tn < num_tiles) {
-              if (pf_seq[h] != seq + 1) {
-                decode_tile(tn, args, tiles_per_problem, pf_p[h], pf_ti[h], pf_tj[h]);
-                pf_seq[h] = seq + 1;
-              }
-              const GemmProblem* pn = probs + pf_p[h];
-              const int part = h * HALF_CHUNKS + i;  // 0..15
-              const float* src = pn->aux + ((int64_t)(pf_ti[h] * 2 + (int)rank) * BM + part * 8) * pn->aux_ld +
-                                 (int64_t)pf_tj[h] * PN;
-#pragma unroll
-              for (int r = 0; r < 8; ++r) l2_prefetch(src + r * pn->aux_ld, PN * 4);
-            }
-          }
-#endif
           ++n[h];
+          ++done;
           progressed = true;
         }
         if (progressed) { idle = 0; continue; }
+#ifdef FP4_POLL_SLEEP
+        __nanosleep(FP4_POLL_SLEEP);
+#endif
         if ((++idle & 1023u) == 0) {
           if (*abort_flag) break;
           const uint64_t now = globaltimer_ns();
@@ -337,23 +331,26 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
     }
   } else if (warp == 3) {
     // ------------------------------------------------------------ TMA-store issuer
-    // One thread, both halves, polling like the producer above; up to three stores are in
-    // flight, a slot is handed back once two newer stores have been issued.
+    // One thread, all teams, polling like the producer above; up to three stores are in
+    // flight, a slot is handed back once two newer stores have been issued or, when no chunk
+    // is waiting to be sent, as soon as its store has read it.
     if (elect_one()) {
       const uint32_t my_tiles = pair < num_tiles ? (uint32_t)((num_tiles - pair + num_pairs - 1) / num_pairs) : 0u;
-      const uint32_t total = my_tiles * HALF_CHUNKS;
-      uint32_t n[2] = {0, 0}, seq_dec[2] = {0xFFFFFFFFu, 0xFFFFFFFFu};
-      int pp[2] = {0, 0}, tis[2] = {0, 0}, tjs[2] = {0, 0};
+      const uint32_t total = my_tiles * TEAM_CHUNKS;
+      uint32_t n[TEAMS], seq_dec[TEAMS];
+      int pp[TEAMS], tis[TEAMS], tjs[TEAMS];
+#pragma unroll
+      for (int h = 0; h < TEAMS; ++h) { n[h] = 0; seq_dec[h] = 0xFFFFFFFFu; pp[h] = tis[h] = tjs[h] = 0; }
       int q0 = -1, q1 = -1;  // slots of the two newest stores, not yet handed back
-      uint32_t idle = 0;
+      uint32_t idle = 0, done = 0;
       uint64_t t_idle = 0;
-      while ((n[0] < total || n[1] < total)) {
+      while (done < TEAMS * total) {
         bool progressed = false;
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
+        for (int h = 0; h < TEAMS; ++h) {
           if (n[h] >= total) continue;
-          const uint32_t seq = n[h] / HALF_CHUNKS;
-          const int i = (int)(n[h] % HALF_CHUNKS);
+          const uint32_t seq = n[h] / TEAM_CHUNKS;
+          const int i = (int)(n[h] % TEAM_CHUNKS);
           int b; uint32_t use;
           chunk_slot(seq, h, i, b, use);
           if (!mbar_try_wait(&bars->v_ready[b], use & 1)) continue;
@@ -363,7 +360,7 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
           }
           const GemmProblem* pr = probs + pp[h];
           const int bi = tis[h] * 2 + (int)rank;
-          const int c = half_chunk((int)(seq & 1), h, i);
+          const int c = team_chunk((int)(seq & 1), h, i);
           const bool below = args.symmetric && (tjs[h] * 2 + c / 8) < bi;
           if (STORE_F32 && !below) {
             tma_store_2d(&pr->tmOut, tjs[h] * PN + c * CHUNK, bi * BM, smem + OFF_RING + b * CHUNK_BYTES);
@@ -375,9 +372,22 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
             mbar_arrive(&bars->slot_free[b]);
           }
           ++n[h];
+          ++done;
           progressed = true;
         }
         if (progressed) { idle = 0; continue; }
+#ifdef FP4_POLL_SLEEP
+        __nanosleep(FP4_POLL_SLEEP);
+#endif
+        if (STORE_F32 && q1 >= 0) {
+          // nothing to send right now: do not sit on the slots of the newest stores (their team may
+          // need them back before anyone issues another store)
+          bulk_wait_read<0>();
+          if (q0 >= 0) mbar_arrive(&bars->slot_free[q0]);
+          mbar_arrive(&bars->slot_free[q1]);
+          q0 = q1 = -1;
+          continue;
+        }
         if ((++idle & 1023u) == 0) {
           if (*abort_flag) break;
           const uint64_t now = globaltimer_ns();
@@ -392,17 +402,25 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
         bulk_wait_all<0>();
       }
     }
-  } else if (warp < 12) {
-    // ------------------------------------------------------------ drain warps
-    const int half = (warp - 4) >> 2;
+  } else {
+    // ------------------------------------------------------------ epilogue warps
+    const int team = (warp - 4) >> 2;
     const int quad = warp & 3;
     const int row = quad * 32 + lane;
+    // column pass: lane = (column cq of the chunk, 16-row group g of this warp's 32 rows)
+    const int cq = lane & 15, g = lane >> 4;
     float scale = 0.0f, sg_out = 1.0f, inv_sg = 1.0f;
     uint32_t rcp_base = 0;
     float ca = 0.0f, cb = 0.0f, cc = 0.0f;
     const GemmProblem* pr = nullptr;
     int cur_p = -1;
     const int sw = (row >> 1) & 3;
+    // column pass: byte offset of (first row of this lane's 16-row group, column cq) in a slot, and the
+    // swizzled offsets of the column's 16-byte group for the four values of bits 1-2 of the row
+    const int col_off = (quad * 32 + g * 16) * 64 + (cq & 3) * 4;
+    int col_sw[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) col_sw[k] = ((cq >> 2) ^ k) << 4;
     const uint32_t tm_lane = tmem_base + ((uint32_t)(quad * 32) << 16);
     const uint32_t acc_empty_leader0 = map_to_cta(&bars->acc_empty[0], 0);
     const uint32_t acc_empty_leader1 = map_to_cta(&bars->acc_empty[1], 0);
@@ -432,25 +450,37 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
         rcp_base = rcp_base_of(sg_out);
         ca = pr->ca; cb = pr->cb; cc = pr->cc;
       }
-      const int bi = ti * 2 + (int)rank;              // 128-row block of this CTA
-      const int bj = tj * 2 + half;                   // 128-column block of this half
-      const bool below = args.symmetric && bj < bi;   // redundant block of a diagonal tile
+      const int bi = ti * 2 + (int)rank;                               // 128-row block of this CTA
+      const int bj = tj * 2 + (team * TEAM_CHUNKS * CHUNK) / 128;      // 128-column block of this team's chunks
+      const bool below = args.symmetric && bj < bi;                    // redundant block of a diagonal tile
       const bool mirror = do_q && !below && (MODE == kG3 || (args.symmetric && bi != bj));
+      const bool stage = !below && (STORE_F32 || mirror);
       const int par = (int)(seq & 1);
       ok = __all_sync(0xffffffffu, wait_bar(&bars->acc_full[par], (seq >> 1) & 1, abort_flag));
       if (!ok) break;
       tc_fence_after();
       const int64_t grow = (int64_t)bi * BM + row;
+      // store addresses of this tile: row-quantised codes of this thread's row; column-quantised
+      // codes and scale of (tensor row = tile column cq, 16-block = this lane's row group)
+      uint8_t* rq_row = nullptr; uint8_t* cq_col = nullptr; uint8_t* cq_sfp = nullptr;
+      if (do_q) {
+        rq_row = pr->rq_codes + grow * (args.rq_K / 2) + ((int64_t)tj * PN) / 2;
+        const int64_t tcol = (int64_t)bi * BM + quad * 32 + g * 16;
+        const int64_t kb = tcol >> 4, kblocks = args.cq_K >> 4;
+        cq_col = pr->cq_codes + ((int64_t)tj * PN + cq) * (args.cq_K / 2) + tcol / 2;
+        cq_sfp = pr->cq_sf + ((int64_t)tj * 2 * (kblocks >> 2) + (kb >> 2)) * 512 + (kb & 3) + cq * 16;
+      }
       const uint32_t tm_acc = tm_lane + par * ACC1_COL;
-      const bool owns_overlap = (half == (par == 0 ? 1 : 0));
-      uint32_t sfw0 = 0, sfw1 = 0;
+      const bool owns_overlap = (team == (par == 0 ? TEAMS - 1 : 0));
+      uint32_t sfw = 0;
       uint32_t acc[16];
-      tc_ld16_issue(tm_acc + half_chunk(par, half, 0) * CHUNK, acc);
-      for (int i = 0; i < HALF_CHUNKS; ++i) {
-        const int c = half_chunk(par, half, i);
+      tc_ld16_issue(tm_acc + team_chunk(par, team, 0) * CHUNK, acc);
+      for (int i = 0; i < TEAM_CHUNKS; ++i) {
+        const int c = team_chunk(par, team, i);
         int b; uint32_t use;
-        chunk_slot(seq, half, i, b, use);
-        uint8_t* slot_row = smem + OFF_RING + b * CHUNK_BYTES + row * 64;
+        chunk_slot(seq, team, i, b, use);
+        uint8_t* slot = smem + OFF_RING + b * CHUNK_BYTES;
+        uint8_t* slot_row = slot + row * 64;
         float v[16];
         if (HAS_AUX) ok = __all_sync(0xffffffffu, wait_bar(&bars->aux_full[b], use & 1, abort_flag));
         else ok = __all_sync(0xffffffffu, wait_bar(&bars->slot_free[b], (use & 1) ^ 1, abort_flag));
@@ -459,10 +489,11 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
         if (HAS_AUX && !below) {
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
-            float4 x = *reinterpret_cast<const float4*>(slot_row + ((j ^ sw) << 4));
-            float e[4] = {x.x, x.y, x.z, x.w};
+            const float4 x = *reinterpret_cast<const float4*>(slot_row + ((j ^ sw) << 4));
+            const float e[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
+              // every product and the sum rounded on its own (scalar intrinsics: never contracted)
               const float prod = __fmul_rn(__uint_as_float(acc[4 * j + q]), scale);
               if (MODE == kG2) v[4 * j + q] = __fadd_rn(__fmul_rn(cb, e[q]), __fmul_rn(cc, prod));
               else v[4 * j + q] = __fadd_rn(__fmul_rn(ca, e[q]), prod);
@@ -470,7 +501,7 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
           }
         } else {
 #pragma unroll
-          for (int i = 0; i < 16; ++i) v[i] = __fmul_rn(__uint_as_float(acc[i]), scale);
+          for (int k = 0; k < 16; ++k) v[k] = __fmul_rn(__uint_as_float(acc[k]), scale);
         }
         if (owns_overlap && i == OV_CHUNKS - 1) {
           // the columns shared with the other buffer are in registers: the next tile may use them
@@ -478,14 +509,14 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
           __syncwarp();
           if (lane == 0) mbar_arrive_cluster(ov_free_leader);
         }
-        if (i + 1 < HALF_CHUNKS) {
-          tc_ld16_issue(tm_acc + half_chunk(par, half, i + 1) * CHUNK, acc);
+        if (i + 1 < TEAM_CHUNKS) {
+          tc_ld16_issue(tm_acc + team_chunk(par, team, i + 1) * CHUNK, acc);
         } else {
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive_cluster(par ? acc_empty_leader1 : acc_empty_leader0);  // done with the buffer
         }
-        if (!below && (STORE_F32 || mirror)) {
+        if (stage) {
 #pragma unroll
           for (int j = 0; j < 4; ++j)
             *reinterpret_cast<float4*>(slot_row + ((j ^ sw) << 4)) =
@@ -493,25 +524,47 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
           fence_proxy_async_smem();
         }
         __syncwarp();
-        if (lane == 0) mbar_arrive(&bars->v_ready[b]);
-        if (below) continue;
-        if (do_q) {
+        if (lane == 0) mbar_arrive(&bars->v_ready[b]);  // the store issuer may send the chunk
+        // Blocks of 16 down the rows of this warp's own 32 x 16 block (the transposed operand
+        // copy in G3, the mirrored triangle in G1/G2), read back from the staging slot: row
+        // k of the block is at k * 64 bytes, its 16-byte column group XOR-swizzled with bits
+        // 1-2 of k.  (The two half-warps read rows 16 apart, a two-way bank conflict on these
+        // sixteen 4-byte loads; avoiding it costs more instructions than it saves.)
+        float w[16];
+        if (mirror) {
+          const uint8_t* colp = slot + col_off;
+#pragma unroll
+          for (int k = 0; k < 16; ++k)
+            w[k] = *reinterpret_cast<const float*>(colp + k * 64 + (col_sw[(k >> 1) & 3]));
+        }
+        if (!below && do_q) {
           uint32_t lo, hi;
           float bmax;
           uint32_t sb;
           if (PF) sb = quantize_block16_opts(v, args.q, sg_out, lo, hi, bmax);
           else sb = quantize_block16_pow2(v, sg_out, inv_sg, rcp_base, lo, hi, bmax);
           if (MODE == kG1 || MODE == kG3) amax = fmaxf(amax, bmax);
-          const int64_t gcol = (int64_t)tj * PN + c * CHUNK;
-          *reinterpret_cast<uint2*>(pr->rq_codes + grow * (args.rq_K / 2) + gcol / 2) = make_uint2(lo, hi);
-          if ((c >> 2) & 1) sfw1 |= sb << (8 * (c & 3)); else sfw0 |= sb << (8 * (c & 3));
+          *reinterpret_cast<uint2*>(rq_row + c * (CHUNK / 2)) = make_uint2(lo, hi);
+          sfw |= sb << (8 * (c & 3));
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bars->slot_free[b]);  // this warp's part of the slot is in registers
+        if (mirror) {
+          uint32_t lo, hi;
+          float bmax;
+          uint32_t sb;
+          if (PF) sb = quantize_block16_opts(w, args.q, sg_out, lo, hi, bmax);
+          else sb = quantize_block16_pow2(w, sg_out, inv_sg, rcp_base, lo, hi, bmax);
+          // tensor row = tj * 256 + c * 16 + cq: its codes are c * 16 rows further on; in the scale
+          // atoms, c / 8 selects the 128-row atom, c % 2 the upper 16 of 32 rows, (c % 8) / 2 the 32-row group
+          *reinterpret_cast<uint2*>(cq_col + (int64_t)c * CHUNK * (args.cq_K / 2)) = make_uint2(lo, hi);
+          cq_sfp[(int64_t)(c >> 3) * (args.cq_K >> 6) * 512 + (c & 1) * 256 + ((c & 7) >> 1) * 4] = (uint8_t)sb;
         }
       }
       if (ok && do_q && !below) {
-        // the two scale words of this half's 128 columns of the row
-        const int64_t kb0 = ((int64_t)tj * PN + half * (PN / 2)) >> 4;
-        *reinterpret_cast<uint32_t*>(pr->rq_sf + sf_offset(grow, kb0, args.rq_K >> 4)) = sfw0;
-        *reinterpret_cast<uint32_t*>(pr->rq_sf + sf_offset(grow, kb0 + 4, args.rq_K >> 4)) = sfw1;
+        // the scale word of this team's 64 columns of the row
+        const int64_t kb0 = ((int64_t)tj * PN + team * TEAM_CHUNKS * CHUNK) >> 4;
+        *reinterpret_cast<uint32_t*>(pr->rq_sf + sf_offset(grow, kb0, args.rq_K >> 4)) = sfw;
       }
     }
     if ((MODE == kG1 || MODE == kG3) && cur_p >= 0) {
@@ -520,77 +573,6 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
       if (lane == 0) {
         const int slot = (MODE == kG1) ? args.ix.amax_A0 + args.iter : args.ix.amax_X0 + args.iter + 1;
         atomicMax(reinterpret_cast<uint32_t*>(pr->scalars + slot), __float_as_uint(amax));
-      }
-    }
-  } else {
-    // ------------------------------------------------------------ finish warps
-    const int half = (warp - 12) >> 2;
-    const int et = ((warp - 12) & 3) * 32 + lane;
-    const int cc = et & 15, g = et >> 4;
-    const int rot = (lane >> 4) & 1;
-    float scale, sg_out = 1.0f, inv_sg = 1.0f;
-    uint32_t rcp_base = 0;
-    const GemmProblem* pr = nullptr;
-    int cur_p = -1;
-    uint32_t seq = 0;
-    bool ok = true;
-    for (int t = pair; t < num_tiles && ok; t += num_pairs, ++seq) {
-      int p, ti, tj;
-      decode_tile(t, args, tiles_per_problem, p, ti, tj);
-      if (p != cur_p) {
-        cur_p = p;
-        pr = probs + p;
-        epilogue_scalars<MODE>(*pr, args, scale, sg_out, false);
-        inv_sg = __frcp_rn(sg_out);
-        rcp_base = rcp_base_of(sg_out);
-      }
-      const int bi = ti * 2 + (int)rank;
-      const int bj = tj * 2 + half;
-      const bool below = args.symmetric && bj < bi;
-      const bool mirror = do_q && !below && (MODE == kG3 || (args.symmetric && bi != bj));
-      for (int i = 0; i < HALF_CHUNKS; ++i) {
-        const int c = half_chunk((int)(seq & 1), half, i);
-        int b; uint32_t use;
-        chunk_slot(seq, half, i, b, use);
-        ok = __all_sync(0xffffffffu, wait_bar(&bars->v_ready[b], use & 1, abort_flag));
-        if (!ok) break;
-        if (mirror) {
-          const uint8_t* obase = smem + OFF_RING + b * CHUNK_BYTES;
-          float w[16];
-#pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            // the upper half-warp starts one row later (and wraps), so that the two half-warps
-            // read rows of different parity, i.e. different banks
-            const int r = g * 16 + ((i + rot) & 15);
-            w[i] = *reinterpret_cast<const float*>(obase + r * 64 + ((((cc >> 2) ^ ((r >> 1) & 3))) << 4) + (cc & 3) * 4);
-          }
-          uint32_t lo, hi;
-          float bmax;
-          uint32_t sb;
-          if (PF) {
-            // the transform and the error sums need the block in row order
-            float x[16];
-#pragma unroll
-            for (int i = 0; i < 16; ++i) x[i] = rot ? w[(i + 15) & 15] : w[i];
-            sb = quantize_block16_opts(x, args.q, sg_out, lo, hi, bmax);
-          } else {
-            sb = quantize_block16_pow2(w, sg_out, inv_sg, rcp_base, lo, hi, bmax);
-            if (rot) {
-              // the codes were packed one row early: rotate the 16 nibbles back into row order
-              const uint32_t nlo = (lo << 4) | (hi >> 28), nhi = (hi << 4) | (lo >> 28);
-              lo = nlo; hi = nhi;
-            }
-          }
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&bars->slot_free[b]);
-          const int64_t trow = (int64_t)tj * PN + c * CHUNK + cc;
-          const int64_t tcol = (int64_t)bi * BM + g * 16;
-          *reinterpret_cast<uint2*>(pr->cq_codes + trow * (args.cq_K / 2) + tcol / 2) = make_uint2(lo, hi);
-          pr->cq_sf[sf_offset(trow, tcol >> 4, args.cq_K >> 4)] = (uint8_t)sb;
-        } else {
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&bars->slot_free[b]);
-        }
       }
     }
   }

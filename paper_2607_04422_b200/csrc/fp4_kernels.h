@@ -65,8 +65,6 @@ struct alignas(64) GemmProblem {
   const uint8_t* sfa;        // scale atoms of the row operand
   const uint8_t* sfb;        // scale atoms of the column operand
   float* scalars;            // workspace scalars of this matrix (device)
-  const float* aux;          // the FP32 matrix behind tmAux (row-major, leading dimension aux_ld), for L2 prefetch
-  int64_t aux_ld;
   uint8_t* rq_codes; uint8_t* rq_sf;  // quantised output, blocks along the tile's columns
   uint8_t* cq_codes; uint8_t* cq_sf;  // quantised output, blocks along the tile's rows
   float ca, cb, cc;          // coefficients

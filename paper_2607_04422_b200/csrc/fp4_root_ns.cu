@@ -267,14 +267,12 @@ fp4_status prepare_matrix(const DeviceInfo* d, const float* G, float* out, int64
   // G1: A = qX qX^T (upper-triangle tiles), qA in both triangles
   c->g1 = base;
   c->g1.tmA = c->g1.tmB = tm_qX; c->g1.tmAux = c->g1.tmOut = tm_A;
-  c->g1.aux = nullptr;
   c->g1.tmSfa = c->g1.tmSfb = sf_qX;
   c->g1.sfa = c->g1.sfb = ws + L.qX_scales;
   c->g1.rq_codes = c->g1.cq_codes = ws + L.qA_codes; c->g1.rq_sf = c->g1.cq_sf = ws + L.qA_scales;
   // G2: B = bA + c qA qA^T, qB in both triangles
   c->g2 = base;
   c->g2.tmA = c->g2.tmB = tm_qA; c->g2.tmAux = c->g2.tmOut = tm_A;
-  c->g2.aux = reinterpret_cast<const float*>(ws + L.A); c->g2.aux_ld = s;
   c->g2.tmSfa = c->g2.tmSfb = sf_qA;
   c->g2.sfa = c->g2.sfb = ws + L.qA_scales;
   c->g2.rq_codes = c->g2.cq_codes = ws + L.qB_codes; c->g2.rq_sf = c->g2.cq_sf = ws + L.qB_scales;
@@ -283,7 +281,6 @@ fp4_status prepare_matrix(const DeviceInfo* d, const float* G, float* out, int64
     GemmProblem& g = c->g3[cur];
     g = base;
     g.tmA = tm_qB; g.tmB = tm_qXt[cur]; g.tmAux = g.tmOut = tm_X;
-    g.aux = c->X; g.aux_ld = l;
     g.tmSfa = sf_qB; g.tmSfb = sf_qXt[cur];
     g.sfa = ws + L.qB_scales; g.sfb = ws + L.qXt_scales[cur];
     g.rq_codes = ws + L.qX_codes; g.rq_sf = ws + L.qX_scales;
