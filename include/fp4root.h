@@ -81,7 +81,7 @@ typedef struct {
   float eps;           /* X0 = G_c / (||G_c||_F + eps).  Default 1e-7.                     */
   uint32_t flags;      /* FP4_FLAG_*; default 0                                            */
   uint32_t max_group;  /* fp4_root_ns_batched: at most this many equal-shape matrices run their
-                          stages in lockstep as single launches; 0 = library default (8)      */
+                          stages in lockstep as single launches; 0 = library default (16)     */
   uint64_t seed;       /* FP4_FLAG_RHT: seed of the sign draws; default 0                    */
 } fp4_ns_params;
 

@@ -412,6 +412,8 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
     float scale = 0.0f, sg_out = 1.0f, inv_sg = 1.0f;
     uint32_t rcp_base = 0;
     float ca = 0.0f, cb = 0.0f, cc = 0.0f;
+    float tau = 0.0f, inv = 0.0f;  // first G3 stage on the raw input: X0 = clamp(G, tau) * inv
+    bool raw = false;
     const GemmProblem* pr = nullptr;
     int cur_p = -1;
     const int sw = (row >> 1) & 3;
@@ -449,6 +451,11 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
         inv_sg = __frcp_rn(sg_out);  // exact: the predicted scales are powers of two
         rcp_base = rcp_base_of(sg_out);
         ca = pr->ca; cb = pr->cb; cc = pr->cc;
+        raw = (MODE == kG3) && pr->aux_raw != 0;
+        if (raw) {
+          tau = args.clip ? pr->scalars[args.ix.tau] : __int_as_float(0x7f800000);
+          inv = pr->scalars[args.ix.inv];
+        }
       }
       const int bi = ti * 2 + (int)rank;                               // 128-row block of this CTA
       const int bj = tj * 2 + (team * TEAM_CHUNKS * CHUNK) / 128;      // 128-column block of this team's chunks
@@ -490,7 +497,11 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
             const float4 x = *reinterpret_cast<const float4*>(slot_row + ((j ^ sw) << 4));
-            const float e[4] = {x.x, x.y, x.z, x.w};
+            float e[4] = {x.x, x.y, x.z, x.w};
+            if (MODE == kG3 && raw) {
+#pragma unroll
+              for (int q = 0; q < 4; ++q) e[q] = __fmul_rn(fminf(fmaxf(e[q], -tau), tau), inv);
+            }
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
               // every product and the sum rounded on its own (scalar intrinsics: never contracted)

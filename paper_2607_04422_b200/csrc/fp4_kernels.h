@@ -69,6 +69,7 @@ struct alignas(64) GemmProblem {
   uint8_t* cq_codes; uint8_t* cq_sf;  // quantised output, blocks along the tile's rows
   float ca, cb, cc;          // coefficients
   float sg_a, sg_b;          // kPlain: tensor scales from the host
+  int aux_raw;               // kG3: tmAux maps the raw input G; X0 = clamp(G, tau) * inv is formed on the fly
 };
 
 // What all problems of a launch share.
@@ -82,6 +83,7 @@ struct GemmLaunch {
   int rq_K, cq_K;      // row lengths (elements) of the two quantised outputs
   float l_cols;        // (float) l, for the bound on amax(A)
   QuantOpts q;         // how this stage's output is quantised (q.widen = 1 in the base mode)
+  int clip;            // kG3 on a problem with aux_raw: whether tau applies
   NsScalarIdx ix;
   uint32_t* status;
 };
@@ -103,6 +105,7 @@ struct PrologueItem {
   uint8_t* ws;
   const NsPlan* pl;
   bool clear_status;
+  bool store_x;   // write X0 in FP32 (not needed when the first G3 stage reads G itself)
 };
 // count matrices that share the shape (s, l) and the clip / eps parameters
 cudaError_t launch_prologue_group(const PrologueItem* items, int count, int write_q, const QuantOpts& q,

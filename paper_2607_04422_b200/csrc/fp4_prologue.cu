@@ -37,6 +37,7 @@ struct PrepMatrix {
   uint8_t* qt_codes; uint8_t* qt_sf;
   int tall;
   int clear_status;
+  int store_x;
 };
 
 struct PrepGroup {
@@ -424,7 +425,7 @@ __global__ void __launch_bounds__(1024) kp_fb_finish(const __grid_constant__ Pre
 }
 
 // ---- X0 = clamp(G) * inv in the work orientation (s x l; transposed when G is tall), its FP32
-// copy, and both NVFP4 operand copies.  One 128 x 128 tile of X per block, gridDim.z = matrix.
+// copy (unless the first G3 stage will form X0 from G itself), and both NVFP4 operand copies.  One 128 x 128 tile of X per block, gridDim.z = matrix.
 template <bool PF>
 __global__ void __launch_bounds__(512) kp_prep_operands(const __grid_constant__ PrepGroup g) {
   extern __shared__ float xs[];  // [128][129]
@@ -455,11 +456,13 @@ __global__ void __launch_bounds__(512) kp_prep_operands(const __grid_constant__ 
     }
   }
   __syncthreads();
+  if (m.store_x) {
 #pragma unroll 4
-  for (int rr = warp; rr < 128; rr += 16) {
-    float4 v = make_float4(xs[rr * P + lane * 4], xs[rr * P + lane * 4 + 1], xs[rr * P + lane * 4 + 2],
-                           xs[rr * P + lane * 4 + 3]);
-    *reinterpret_cast<float4*>(m.X + (r0 + rr) * l + c0 + lane * 4) = v;
+    for (int rr = warp; rr < 128; rr += 16) {
+      float4 v = make_float4(xs[rr * P + lane * 4], xs[rr * P + lane * 4 + 1], xs[rr * P + lane * 4 + 2],
+                             xs[rr * P + lane * 4 + 3]);
+      *reinterpret_cast<float4*>(m.X + (r0 + rr) * l + c0 + lane * 4) = v;
+    }
   }
   if (!g.write_q) return;
   const int part = (warp & 7) >> 2;  // which four of the eight 16-blocks this thread takes
@@ -547,6 +550,7 @@ cudaError_t launch_prologue_group(const PrologueItem* items, int count, int writ
       m.qt_codes = it.ws + L.qXt_codes[0]; m.qt_sf = it.ws + L.qXt_scales[0];
       m.tall = it.pl->tall;
       m.clear_status = it.clear_status ? 1 : 0;
+      m.store_x = it.store_x ? 1 : 0;
     }
     const int sms = pl.sms;
     int64_t hb = (g.n4 + 512 * 4 - 1) / (512 * 4);

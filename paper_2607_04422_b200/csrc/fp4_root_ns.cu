@@ -103,7 +103,7 @@ bool make_f32_map(const DeviceInfo* d, CUtensorMap* tm, const void* base, int64_
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-constexpr int kDefaultMaxGroup = 8;
+constexpr int kDefaultMaxGroup = 16;
 
 // 2-D map over the scale atoms of a rows x K operand: one map row per 128-row block, 64-bit
 // elements, box = the atoms of one operand stage (256 elements = 2 KB), no swizzle.
@@ -235,6 +235,8 @@ struct MatrixCtx {
   float* X;        // FP32 X in the work orientation: `out` itself, or the workspace when tall
   uint8_t* ws;     // this matrix's workspace
   GemmProblem g1, g2, g3[2];  // g3[cur]: reads qXt[cur], writes qXt[cur ^ 1]
+  GemmProblem g3_first;       // iteration 0: as g3[0], but a wide input's FP32 tile is G itself (no X0 copy)
+  bool store_x0;              // the prologue writes X0 in FP32
 };
 
 fp4_status prepare_matrix(const DeviceInfo* d, const float* G, float* out, int64_t m, int64_t n, int steps,
@@ -245,6 +247,7 @@ fp4_status prepare_matrix(const DeviceInfo* d, const float* G, float* out, int64
   const int64_t s = c->pl.s, l = c->pl.l;
   c->G = G; c->out = out; c->ws = ws;
   c->X = c->pl.tall ? reinterpret_cast<float*>(ws + L.X) : out;
+  c->store_x0 = c->pl.tall || steps == 0;
   if (steps == 0) return FP4_OK;
   float abc[3] = {p->a, p->b, p->c};
   if (std::isnan(p->a)) coeffs(m, n, abc);
@@ -286,6 +289,13 @@ fp4_status prepare_matrix(const DeviceInfo* d, const float* G, float* out, int64
     g.rq_codes = ws + L.qX_codes; g.rq_sf = ws + L.qX_scales;
     g.cq_codes = ws + L.qXt_codes[cur ^ 1]; g.cq_sf = ws + L.qXt_scales[cur ^ 1];
   }
+  c->g3_first = c->g3[0];
+  if (!c->store_x0) {
+    CUtensorMap tm_G;
+    if (!make_f32_map(d, &tm_G, G, s, l)) return FP4_ERR_CUDA;
+    c->g3_first.tmAux = tm_G;
+    c->g3_first.aux_raw = 1;
+  }
   return FP4_OK;
 }
 
@@ -303,7 +313,7 @@ __global__ void k_write_problems(GemmProblem* dst, const __grid_constant__ Probl
 
 // Enqueue the whole step for a group of matrices of one shape (s, l): the prologue per matrix,
 // then every Newton-Schulz stage as one launch over all matrices of the group.
-// table: device memory for 4 * count problems (unused when count == 1).
+// table: device memory for 5 * count problems (unused when count == 1).
 fp4_status run_group(const DeviceInfo* d, MatrixCtx* mats, int count, int steps, const fp4_ns_params* p,
                      uint32_t* status, GemmProblem* table, bool clear_first_status, cudaStream_t st) {
   const bool keep = (p->flags & FP4_FLAG_KEEP_OPERANDS) != 0;
@@ -313,15 +323,15 @@ fp4_status run_group(const DeviceInfo* d, MatrixCtx* mats, int count, int steps,
     std::vector<PrologueItem> items((size_t)count);
     for (int i = 0; i < count; ++i) {
       MatrixCtx& c = mats[i];
-      items[(size_t)i] = PrologueItem{c.G, c.X, c.ws, &c.pl, clear_first_status && i == 0};
+      items[(size_t)i] = PrologueItem{c.G, c.X, c.ws, &c.pl, clear_first_status && i == 0, c.store_x0};
     }
     if (launch_prologue_group(items.data(), count, steps > 0 || keep, quant_opts(p, 0), st) != cudaSuccess)
       return FP4_ERR_CUDA;
   }
   if (steps > 0) {
-    const GemmProblem* tabs[4] = {nullptr, nullptr, nullptr, nullptr};
+    const GemmProblem* tabs[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
     if (count > 1) {
-      for (int kind = 0; kind < 4; ++kind) {
+      for (int kind = 0; kind < 5; ++kind) {
         GemmProblem* dst = table + (size_t)kind * count;
         tabs[kind] = dst;
         for (int i0 = 0; i0 < count; i0 += kPackMax) {
@@ -329,7 +339,7 @@ fp4_status run_group(const DeviceInfo* d, MatrixCtx* mats, int count, int steps,
           const int nn = count - i0 < kPackMax ? count - i0 : kPackMax;
           for (int j = 0; j < nn; ++j) {
             const MatrixCtx& c = mats[i0 + j];
-            pack.p[j] = kind == 0 ? c.g1 : kind == 1 ? c.g2 : c.g3[kind - 2];
+            pack.p[j] = kind == 0 ? c.g1 : kind == 1 ? c.g2 : kind == 4 ? c.g3_first : c.g3[kind - 2];
           }
           for (int j = nn; j < kPackMax; ++j) pack.p[j] = pack.p[0];
           count_launches(1);
@@ -344,6 +354,7 @@ fp4_status run_group(const DeviceInfo* d, MatrixCtx* mats, int count, int steps,
     base.ix = pl0.ix;
     base.l_cols = (float)l;
     base.status = status;
+    base.clip = pl0.clip;
     for (int k = 0; k < steps; ++k) {
       const int cur = k & 1;
       const bool last = (k == steps - 1);
@@ -371,7 +382,8 @@ fp4_status run_group(const DeviceInfo* d, MatrixCtx* mats, int count, int steps,
       L3.q = quant_opts(p, 2 * (uint64_t)k + 2);  // both copies of X_{k+1}
       {
         ProfScope ps(FP4_PROF_G3, st);
-        if (launch_gemm_auto(kG3, count == 1 ? &mats[0].g3[cur] : nullptr, tabs[2 + cur], L3, d->sms, st) != cudaSuccess)
+        const GemmProblem* one = k == 0 ? &mats[0].g3_first : &mats[0].g3[cur];
+        if (launch_gemm_auto(kG3, count == 1 ? one : nullptr, k == 0 ? tabs[4] : tabs[2 + cur], L3, d->sms, st) != cudaSuccess)
           return FP4_ERR_CUDA;
       }
     }
@@ -500,7 +512,7 @@ size_t fp4_root_ns_batched_workspace_bytes(int count, const int64_t* m, const in
     if (b == 0) return 0;
     need += align_up(b, 1024);
   }
-  need += align_up((size_t)4 * count * sizeof(GemmProblem), 1024);
+  need += align_up((size_t)5 * count * sizeof(GemmProblem), 1024);
   return need;
 }
 
