@@ -426,13 +426,18 @@ __global__ void __launch_bounds__(1024) kp_fb_finish(const __grid_constant__ Pre
 
 // ---- X0 = clamp(G) * inv in the work orientation (s x l; transposed when G is tall), its FP32
 // copy (unless the first G3 stage will form X0 from G itself), and both NVFP4 operand copies.  One 128 x 128 tile of X per block, gridDim.z = matrix.
+// Row pitch of the shared tile in floats: 132 (16-byte aligned rows: 128-bit shared accesses
+// along a row, conflict-free per quarter-warp) when the tile is filled row by row; 129 (odd)
+// for a tall input, whose tile is filled transposed with 4-byte stores.
+constexpr int kPitchWide = 132, kPitchTall = 129;
+
 template <bool PF>
-__global__ void __launch_bounds__(512) kp_prep_operands(const __grid_constant__ PrepGroup g) {
-  extern __shared__ float xs[];  // [128][129]
-  constexpr int P = 129;
+__global__ void __launch_bounds__(512, 3) kp_prep_operands(const __grid_constant__ PrepGroup g) {
+  extern __shared__ float xs[];  // [128][pitch]
   const PrepMatrix& m = g.mat[blockIdx.z];
   const int64_t s = g.s, l = g.l;
   const int tall = m.tall;
+  const int P = tall ? kPitchTall : kPitchWide;
   const int64_t ldg = tall ? s : l;  // row length of G: a tall G is l x s
   const float tau = g.clip ? m.scalars[g.ix.tau] : __int_as_float(0x7f800000);
   const float inv = m.scalars[g.ix.inv];
@@ -441,68 +446,83 @@ __global__ void __launch_bounds__(512) kp_prep_operands(const __grid_constant__ 
   const int64_t r0 = (int64_t)blockIdx.y * 128, c0 = (int64_t)blockIdx.x * 128;  // tile origin in X
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 
-#pragma unroll 4
-  for (int rr = warp; rr < 128; rr += 16) {
-    // G row: tall -> row (c0+rr), columns r0..; else row (r0+rr), columns c0..
-    const float* src = tall ? m.G + (c0 + rr) * ldg + r0 : m.G + (r0 + rr) * ldg + c0;
-    float4 v = __ldg(reinterpret_cast<const float4*>(src) + lane);
-    float e[4] = {v.x, v.y, v.z, v.w};
+  // The tile holds raw G values; clamp and scale are applied where a pass reads them.  A wide
+  // input's rows go straight to shared memory with asynchronous 16-byte copies (64 KB in flight
+  // per block without holding registers); a tall input's tile is filled transposed from registers.
+  auto x0 = [&](float gval) { return __fmul_rn(fminf(fmaxf(gval, -tau), tau), inv); };
+  if (!tall) {
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      float c = fminf(fmaxf(e[j], -tau), tau);
-      float xv = __fmul_rn(c, inv);
-      int cc = lane * 4 + j;
-      if (tall) xs[cc * P + rr] = xv; else xs[rr * P + cc] = xv;
+    for (int rr = warp; rr < 128; rr += 16) {
+      const float* src = m.G + (r0 + rr) * ldg + c0 + lane * 4;
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(xs + rr * P + lane * 4)), "l"(src) : "memory");
+    }
+    asm volatile("cp.async.wait_all;" ::: "memory");
+  } else {
+#pragma unroll 4
+    for (int rr = warp; rr < 128; rr += 16) {
+      const float4 v = __ldg(reinterpret_cast<const float4*>(m.G + (c0 + rr) * ldg + r0) + lane);
+      xs[(lane * 4 + 0) * P + rr] = v.x; xs[(lane * 4 + 1) * P + rr] = v.y;
+      xs[(lane * 4 + 2) * P + rr] = v.z; xs[(lane * 4 + 3) * P + rr] = v.w;
     }
   }
   __syncthreads();
   if (m.store_x) {
 #pragma unroll 4
     for (int rr = warp; rr < 128; rr += 16) {
-      float4 v = make_float4(xs[rr * P + lane * 4], xs[rr * P + lane * 4 + 1], xs[rr * P + lane * 4 + 2],
-                             xs[rr * P + lane * 4 + 3]);
-      *reinterpret_cast<float4*>(m.X + (r0 + rr) * l + c0 + lane * 4) = v;
+      const float* row = xs + rr * P + lane * 4;
+      *reinterpret_cast<float4*>(m.X + (r0 + rr) * l + c0 + lane * 4) =
+          make_float4(x0(row[0]), x0(row[1]), x0(row[2]), x0(row[3]));
     }
   }
   if (!g.write_q) return;
   const int part = (warp & 7) >> 2;  // which four of the eight 16-blocks this thread takes
+  uint32_t code[8];                  // the codes of those four blocks: 32 consecutive bytes of the operand row
+  uint32_t sfw = 0;
   if (warp < 8) {
     // blocks along the columns of X (contraction axis of G1): thread = row
     const int rr = (warp & 3) * 32 + lane;
-    uint32_t sfw = 0;
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
       const int kb = part * 4 + q;
       float v[16];
+      if (tall) {
 #pragma unroll
-      for (int i = 0; i < 16; ++i) v[i] = xs[rr * P + kb * 16 + i];
-      uint32_t lo, hi;
+        for (int i = 0; i < 16; ++i) v[i] = x0(xs[rr * P + kb * 16 + i]);
+      } else {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float4 t = *reinterpret_cast<const float4*>(xs + rr * P + kb * 16 + i * 4);
+          v[4 * i] = x0(t.x); v[4 * i + 1] = x0(t.y); v[4 * i + 2] = x0(t.z); v[4 * i + 3] = x0(t.w);
+        }
+      }
       uint32_t sb;
       float unused;
-      if (PF) sb = quantize_block16_opts(v, g.q, sg, lo, hi, unused);
-      else sb = quantize_block16(v, six_sg, sg, lo, hi);
-      *reinterpret_cast<uint2*>(m.qx_codes + (r0 + rr) * (l / 2) + (c0 + kb * 16) / 2) = make_uint2(lo, hi);
+      if (PF) sb = quantize_block16_opts(v, g.q, sg, code[2 * q], code[2 * q + 1], unused);
+      else sb = quantize_block16(v, six_sg, sg, code[2 * q], code[2 * q + 1]);
       sfw |= sb << (8 * q);
     }
+    uint4* dst = reinterpret_cast<uint4*>(m.qx_codes + (r0 + rr) * (l / 2) + (c0 + part * 64) / 2);
+    dst[0] = make_uint4(code[0], code[1], code[2], code[3]);
+    dst[1] = make_uint4(code[4], code[5], code[6], code[7]);
     *reinterpret_cast<uint32_t*>(m.qx_sf + sf_offset(r0 + rr, c0 / 16 + part * 4, l / 16)) = sfw;
   } else {
     // blocks along the rows of X (contraction axis of G3): thread = column of X = row of X^T
     const int cc = (warp & 3) * 32 + lane;
-    uint32_t sfw = 0;
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
       const int gq = part * 4 + q;
       float v[16];
 #pragma unroll
-      for (int i = 0; i < 16; ++i) v[i] = xs[(gq * 16 + i) * P + cc];
-      uint32_t lo, hi;
+      for (int i = 0; i < 16; ++i) v[i] = x0(xs[(gq * 16 + i) * P + cc]);
       uint32_t sb;
       float unused;
-      if (PF) sb = quantize_block16_opts(v, g.q, sg, lo, hi, unused);
-      else sb = quantize_block16(v, six_sg, sg, lo, hi);
-      *reinterpret_cast<uint2*>(m.qt_codes + (c0 + cc) * (s / 2) + (r0 + gq * 16) / 2) = make_uint2(lo, hi);
+      if (PF) sb = quantize_block16_opts(v, g.q, sg, code[2 * q], code[2 * q + 1], unused);
+      else sb = quantize_block16(v, six_sg, sg, code[2 * q], code[2 * q + 1]);
       sfw |= sb << (8 * q);
     }
+    uint4* dst = reinterpret_cast<uint4*>(m.qt_codes + (c0 + cc) * (s / 2) + (r0 + part * 64) / 2);
+    dst[0] = make_uint4(code[0], code[1], code[2], code[3]);
+    dst[1] = make_uint4(code[4], code[5], code[6], code[7]);
     *reinterpret_cast<uint32_t*>(m.qt_sf + sf_offset(c0 + cc, r0 / 16 + part * 4, s / 16)) = sfw;
   }
 }
@@ -510,9 +530,9 @@ __global__ void __launch_bounds__(512) kp_prep_operands(const __grid_constant__ 
 }  // namespace
 
 cudaError_t prologue_set_attributes() {
-  cudaError_t e = cudaFuncSetAttribute(kp_prep_operands<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 129 * 4);
+  cudaError_t e = cudaFuncSetAttribute(kp_prep_operands<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * kPitchWide * 4);
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(kp_prep_operands<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 129 * 4);
+  return cudaFuncSetAttribute(kp_prep_operands<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * kPitchWide * 4);
 }
 
 // Enqueue the prologue for `count` matrices of one shape (s, l) and one parameter set.
@@ -585,8 +605,8 @@ cudaError_t launch_prologue_group(const PrologueItem* items, int count, int writ
     {
       ProfScope ps(FP4_PROF_PREP, st);
       const dim3 gp((unsigned)(pl.l / 128), (unsigned)(pl.s / 128), (unsigned)nn);
-      if (q.rht || q.four_six) kp_prep_operands<true><<<gp, 512, 128 * 129 * 4, st>>>(g);
-      else kp_prep_operands<false><<<gp, 512, 128 * 129 * 4, st>>>(g);
+      if (q.rht || q.four_six) kp_prep_operands<true><<<gp, 512, 128 * kPitchWide * 4, st>>>(g);
+      else kp_prep_operands<false><<<gp, 512, 128 * kPitchWide * 4, st>>>(g);
       count_launches(1);
     }
     cudaError_t e = cudaGetLastError();
