@@ -23,7 +23,7 @@ namespace fp4 {
 
 namespace {
 
-constexpr int kMaxPack = 8;
+constexpr int kMaxPack = 16;
 
 struct PrepMatrix {
   const float* G;

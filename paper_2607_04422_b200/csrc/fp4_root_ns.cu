@@ -299,7 +299,7 @@ fp4_status prepare_matrix(const DeviceInfo* d, const float* G, float* out, int64
   return FP4_OK;
 }
 
-constexpr int kPackMax = 4;
+constexpr int kPackMax = 16;
 struct ProblemPack { GemmProblem p[kPackMax]; };
 
 // Copies problem descriptions from kernel parameters into a device table (the tables of a
