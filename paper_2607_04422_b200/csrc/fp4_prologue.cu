@@ -259,8 +259,15 @@ __global__ void __launch_bounds__(1024) kp_finalize(const __grid_constant__ Prep
     if (threadIdx.x == 0) hdr->overflow = 1;  // the fallback kernels take over
     return;
   }
-  // two radix rounds over the low 18 bits of the candidates: 9 bits each
+  // two radix rounds over the low 18 bits of the candidates: 9 bits each.  The second round
+  // also gathers what the norm needs: squares of the candidates below the sub-bin picked by
+  // the first round (certainly not clipped) as exact integers -- all candidates share the
+  // exponent field, so x = mant * 2^(e-150) with a 24-bit integer mant -- and the number above it.
   if (threadIdx.x == 0) { s_prefix = hdr->sel_prefix; s_rank = hdr->sel_rank; s_lo = 0; s_hi = 0; s_above = 0; }
+  unsigned long long lo = 0, hi = 0;
+  uint32_t above = 0;
+  const uint32_t efield = hdr->sel_prefix >> 23;
+  const uint32_t implicit = efield ? 0x800000u : 0u;
   for (int round = 0; round < 2; ++round) {
     const int shift = round == 0 ? 9 : 0;
     const uint32_t high_mask = ~((1u << (shift + 9)) - 1u) & 0x7FFFFFFFu;
@@ -275,8 +282,21 @@ __global__ void __launch_bounds__(1024) kp_finalize(const __grid_constant__ Prep
         k[u] = i < count ? m.cand[i] : 0xFFFFFFFFu;
       }
 #pragma unroll
-      for (int u = 0; u < 8; ++u)
-        if ((k[u] & high_mask) == (prefix & high_mask) && k[u] != 0xFFFFFFFFu) atomicAdd(&hist[(k[u] >> shift) & 511u], 1u);
+      for (int u = 0; u < 8; ++u) {
+        if (k[u] == 0xFFFFFFFFu) continue;
+        if ((k[u] & high_mask) == (prefix & high_mask)) {
+          atomicAdd(&hist[(k[u] >> shift) & 511u], 1u);
+        } else if (round == 1) {
+          if (k[u] < prefix) {
+            const unsigned long long mant = (k[u] & 0x7FFFFFu) | implicit;
+            const unsigned long long sq = mant * mant;
+            lo += sq & 0xFFFFFFull;
+            hi += sq >> 24;
+          } else {
+            above += 1;
+          }
+        }
+      }
     }
     __syncthreads();
     // the bin that holds the rank: inclusive scan of the 512 counters by the first warps
@@ -313,28 +333,19 @@ __global__ void __launch_bounds__(1024) kp_finalize(const __grid_constant__ Prep
     __syncthreads();
   }
   const uint32_t tau_bits = s_prefix;
-  // squares of the candidates that are not clipped, as exact integers: all candidates share
-  // the exponent field, so x = mant * 2^(e-150) with a 24-bit integer mant
-  unsigned long long lo = 0, hi = 0;
-  uint32_t above = 0;
-  const uint32_t efield = tau_bits >> 23;
-  for (uint32_t i0 = threadIdx.x; i0 < count; i0 += 8 * blockDim.x) {
-    uint32_t k[8];
-#pragma unroll
-    for (int u = 0; u < 8; ++u) {
-      const uint32_t i = i0 + u * blockDim.x;
-      k[u] = i < count ? m.cand[i] : 0u;
-    }
-#pragma unroll
-    for (int u = 0; u < 8; ++u) {
-      if (i0 + u * blockDim.x >= count) continue;
-      if (k[u] <= tau_bits) {
-        const unsigned long long mant = (k[u] & 0x7FFFFFu) | (efield ? 0x800000u : 0u);
+  // candidates inside the last sub-bin: a counter of the second round stands for one exact
+  // magnitude (all 31 bits known), so its members' squares are count * mant^2
+  if (threadIdx.x < 512) {
+    const uint32_t cnt = hist[threadIdx.x];
+    const uint32_t kk = (tau_bits & ~511u) | threadIdx.x;
+    if (cnt) {
+      if (kk <= tau_bits) {
+        const unsigned long long mant = (kk & 0x7FFFFFu) | implicit;
         const unsigned long long sq = mant * mant;
-        lo += sq & 0xFFFFFFull;
-        hi += sq >> 24;
+        lo += (unsigned long long)cnt * (sq & 0xFFFFFFull);
+        hi += (unsigned long long)cnt * (sq >> 24);
       } else {
-        above += 1;
+        above += cnt;
       }
     }
   }
