@@ -349,9 +349,18 @@ __global__ void __launch_bounds__(1024) kp_finalize(const __grid_constant__ Prep
       }
     }
   }
-  atomicAdd(&s_lo, lo);
-  atomicAdd(&s_hi, hi);
-  atomicAdd(&s_above, above);
+  // one shared atomic per warp (64-bit shared atomics from all 1024 threads serialise badly)
+#pragma unroll
+  for (int o = 16; o; o >>= 1) {
+    lo += __shfl_xor_sync(0xffffffffu, lo, o);
+    hi += __shfl_xor_sync(0xffffffffu, hi, o);
+    above += __shfl_xor_sync(0xffffffffu, above, o);
+  }
+  if ((threadIdx.x & 31) == 0) {
+    atomicAdd(&s_lo, lo);
+    atomicAdd(&s_hi, hi);
+    atomicAdd(&s_above, above);
+  }
   __syncthreads();
   const double below = sum_partials(m.partial, g.stat_blocks, shd);
   if (threadIdx.x == 0) {
