@@ -34,9 +34,10 @@ UNIT = "matrices/s"
 FP4_NOMINAL_TFLOPS = 9000.0  # dense NVFP4, nominal
 FP4_OVER_BF16 = 4.0          # nominal ratio of the dense FP4 and BF16 tensor peaks
 # DRAM bytes per element of X that one G3 launch moves (dram__bytes_read + dram__bytes_write of
-# k_gemm_pair<G3> on one 3072 x 8192 matrix, profiles/k_gemm_pair_3072x8192.md: 170.3 MB for
-# 25.2 M elements); a grouped launch is scaled by the elements it covers
-G3_DRAM_BYTES_PER_ELEMENT = 170.3e6 / (3072 * 8192)
+# k_gemm_pair<G3> on one 3072 x 8192 matrix with all quantised outputs written,
+# profiles/k_gemm_pair_3072x8192.md: 217.3 MB for 25.2 M elements); a grouped launch is scaled by
+# the elements it covers
+G3_DRAM_BYTES_PER_ELEMENT = 217.3e6 / (3072 * 8192)
 
 
 def peaks():
