@@ -99,5 +99,18 @@ def stack_3b(blocks: int = 4, scale_down: int = 1):
     return mats
 
 
+def gqa_stack_shapes(d: int, d_ff: int, kv: int = 1024, blocks: int = 4, fused: bool = False):
+    """(name, m, n) of the projections of `blocks` decoder blocks with hidden size d, gated FFN
+    width d_ff and grouped-query attention whose key / value projections are kv wide (the
+    paper's timing shapes: Section 4.3, d = 4096 / 6144, d_ff = 11008 / 13824, 8 KV heads of
+    128).  Weights are stored (out, in).  fused: one qkv and one gate_up matrix per block."""
+    if fused:
+        roles = (("Wqkv", d + 2 * kv, d), ("Wo", d, d), ("Wgate_up", 2 * d_ff, d), ("Wdown", d, d_ff))
+    else:
+        roles = (("Wq", d, d), ("Wk", kv, d), ("Wv", kv, d), ("Wo", d, d), ("Wgate", d_ff, d), ("Wup", d_ff, d),
+                 ("Wdown", d, d_ff))
+    return [(f"block{b}.{name}", m, n) for b in range(blocks) for name, m, n in roles]
+
+
 def sweep_square(size: int) -> np.ndarray:
     return gaussian(size, size, seed=1)
