@@ -170,6 +170,49 @@ def test_batched_matches_single_calls():
         assert rel(single, oracle.root_ns(g, steps=5)) <= TOL_OUT
 
 
+def test_batched_mixed_orientations_in_one_group_paper_options():
+    """Wide and tall matrices of one work shape share a lockstep group (the wide ones take
+    their first FP32 tile from the raw input, the tall ones from the transposed copy); with
+    the random Hadamard transform and adaptive 4/6 on, and in place for one of them."""
+    specs = [(512, 256, 1), (256, 512, 2), (512, 256, 3), (256, 512, 4), (256, 256, 5)]
+    mats = [workloads.gradient_like(m, n, seed=sd) for m, n, sd in specs]
+    Gs = [torch.from_numpy(g).cuda() for g in mats]
+    outs = [torch.empty_like(g) for g in Gs]
+    outs[1] = Gs[1]                                        # in place
+    shapes = [tuple(g.shape) for g in Gs]
+    flags = FP4_FLAG_RHT | FP4_FLAG_FOUR_SIX
+    ws = torch.empty(fp4.fp4_root_ns_batched_workspace_bytes(shapes, 3, flags), dtype=torch.uint8, device="cuda")
+    p = fp4.NsParams.make(flags=flags, seed=77)
+    fp4.fp4_root_ns_batched(Gs, outs, 3, p, ws)
+    assert fp4.fp4_last_device_status(ws) == 0
+    for g, o in zip(mats, outs):
+        single, _ = run_gpu(g, steps=3, flags=flags, seed=77)
+        assert np.array_equal(o.cpu().numpy(), single)
+        assert rel(single, oracle.root_ns(g, steps=3, rht=True, four_six=True, seed=77)) <= TOL_OUT
+
+
+def test_cuda_graph_replay_matches_direct_call():
+    """The call only enqueues kernels on its stream: it can be captured in a CUDA graph
+    (after one direct call has done the library's per-device set-up) and replayed."""
+    G_np = workloads.config1()
+    m, n = G_np.shape
+    G = torch.from_numpy(G_np).cuda()
+    direct = torch.empty_like(G)
+    ws = torch.empty(fp4.fp4_root_ns_workspace_bytes(m, n, 5), dtype=torch.uint8, device="cuda")
+    fp4.fp4_root_ns(G, direct, 5, None, ws)
+    torch.cuda.synchronize()
+    out = torch.zeros_like(G)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        fp4.fp4_root_ns(G, out, 5, None, ws, torch.cuda.current_stream())
+    for _ in range(2):
+        out.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert fp4.fp4_last_device_status(ws) == 0
+        assert torch.equal(out, direct)
+
+
 def test_argument_errors():
     G = torch.zeros((128, 256), device="cuda")
     ws = torch.empty(fp4.fp4_root_ns_workspace_bytes(128, 256, 5), dtype=torch.uint8, device="cuda")
