@@ -14,9 +14,11 @@
  *     memory.
  *   - All work is enqueued on `stream`; no call synchronises the host except
  *     fp4_last_device_status.
- *   - Shapes: every matrix dimension must be a positive multiple of 128, else
- *     FP4_ERR_SHAPE.  Device pointers must be 16-byte aligned (the workspace 256),
- *     else FP4_ERR_ALIGNMENT.
+ *   - Shapes: for fp4_root_ns, fp4_root_ns_batched and fp4_root_ns_static every matrix
+ *     dimension must be a positive multiple of 16 (the block length; the work matrices
+ *     are zero-padded to multiples of 128 inside the workspace, which changes no result);
+ *     for fp4_quantize and fp4_gemm_nt a positive multiple of 128.  Else FP4_ERR_SHAPE.
+ *     Device pointers must be 16-byte aligned (the workspace 256), else FP4_ERR_ALIGNMENT.
  *   - Errors are return codes.  A kernel that gives up on a bounded wait records
  *     FP4_ERR_DEVICE_TIMEOUT in the workspace header and ends normally; it never
  *     traps.  Read it with fp4_last_device_status.
@@ -123,6 +125,7 @@ fp4_status fp4_root_coeffs(int64_t m, int64_t n, int steps, float abc[3]);
  *   (no partial overlap).  steps >= 0 iterations (0: clip and normalise only).
  * ws: device workspace of at least fp4_root_ns_workspace_bytes(m, n, steps, flags) bytes,
  *   256-byte aligned; its contents need not be initialised and are overwritten.
+ * m, n: positive multiples of 16.
  * Computes, with s = min(m,n), l = max(m,n) and X = G or G^T so that X is s x l:
  *   tau = quantile of |G|, G_c = clamp(G, -tau, tau), X0 = G_c/(||G_c||_F + eps), then
  *   per iteration A = qX qX^T, B = bA + c qA qA^T, X+ = aX + qB qX^{16x1}, every q*

@@ -238,7 +238,8 @@ k_gemm(const __grid_constant__ GemmProblem single, const GemmProblem* __restrict
           int b; uint32_t use;
           chunk_slot(seq, c, b, use);
           if (!wait_bar(&bars->v_ready[b], use & 1, abort_flag)) { ok = false; break; }
-          if (STORE_F32) {
+          // a chunk that starts outside the stored matrix (zero padding of the work shape) is dropped
+          if (STORE_F32 && tj * BN + c * CHUNK < pr->out_cols && ti * BM < pr->out_rows) {
             tma_store_2d(&pr->tmOut, tj * BN + c * CHUNK, ti * BM, smem + OFF_RING + b * CHUNK_BYTES);
             bulk_commit();
             bulk_wait_read<1>();  // every store but the newest has read its slot

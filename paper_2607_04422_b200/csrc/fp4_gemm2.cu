@@ -362,7 +362,9 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
           const int bi = tis[h] * 2 + (int)rank;
           const int c = team_chunk((int)(seq & 1), h, i);
           const bool below = args.symmetric && (tjs[h] * 2 + c / 8) < bi;
-          if (STORE_F32 && !below) {
+          // a chunk that starts outside the stored matrix (zero padding of the work shape) is dropped
+          const bool inside = tjs[h] * PN + c * CHUNK < pr->out_cols && bi * BM < pr->out_rows;
+          if (STORE_F32 && !below && inside) {
             tma_store_2d(&pr->tmOut, tjs[h] * PN + c * CHUNK, bi * BM, smem + OFF_RING + b * CHUNK_BYTES);
             bulk_commit();
             bulk_wait_read<2>();  // every store but the two newest has read its slot

@@ -36,7 +36,9 @@ struct NsScalarIdx {
 struct NsPlan {
   fp4_ws_layout lay;
   NsScalarIdx ix;
-  int64_t m, n, s, l;
+  int64_t m, n;      // the caller's matrix
+  int64_t s0, l0;    // its short and long side
+  int64_t s, l;      // work shape: s0, l0 rounded up to multiples of 128 (zero padding)
   int tall;
   int clip;
   int64_t clip_rank;
@@ -70,6 +72,7 @@ struct alignas(64) GemmProblem {
   float ca, cb, cc;          // coefficients
   float sg_a, sg_b;          // kPlain: tensor scales from the host
   int aux_raw;               // kG3: tmAux maps the raw input G; X0 = clamp(G, tau) * inv is formed on the fly
+  int out_rows, out_cols;    // extent of the matrix behind tmOut (chunks that start outside it are not stored)
 };
 
 // What all problems of a launch share.
@@ -106,11 +109,14 @@ struct PrologueItem {
   const NsPlan* pl;
   bool clear_status;
   bool store_x;   // write X0 in FP32 (not needed when the first G3 stage reads G itself)
+  int64_t x_rows, x_cols;  // extent and row pitch of X: the work shape in the workspace, the caller's shape in `out`
 };
 // count matrices that share the shape (s, l) and the clip / eps parameters
 cudaError_t launch_prologue_group(const PrologueItem* items, int count, int write_q, const QuantOpts& q,
                                   cudaStream_t st);
-cudaError_t launch_transpose_out(const float* X, int64_t s, int64_t l, float* out, cudaStream_t st);
+// out (l0 x s0, row-major) = the leading s0 x l0 part of X^T, X being s x l with row pitch l
+cudaError_t launch_transpose_out(const float* X, int64_t s, int64_t l, float* out, int64_t s0, int64_t l0,
+                                 cudaStream_t st);
 cudaError_t prologue_set_attributes();
 
 cudaError_t gemm_set_attributes();

@@ -38,13 +38,15 @@ struct PrepMatrix {
   int tall;
   int clear_status;
   int store_x;
+  int64_t x_rows, x_cols;  // extent and row pitch of X
 };
 
 struct PrepGroup {
   PrepMatrix mat[kMaxPack];
   int count;
-  int64_t n4;          // elements / 4
-  int64_t s, l;
+  int64_t n4;          // elements of the caller's matrix / 4
+  int64_t s, l;        // work shape (multiples of 128)
+  int64_t s0, l0;      // the caller's short and long side; the rest of the work shape is zero padding
   int clip;
   uint32_t clip_rank;
   uint32_t cand_cap;
@@ -458,7 +460,7 @@ __global__ void __launch_bounds__(512, 3) kp_prep_operands(const __grid_constant
   const int64_t s = g.s, l = g.l;
   const int tall = m.tall;
   const int P = tall ? kPitchTall : kPitchWide;
-  const int64_t ldg = tall ? s : l;  // row length of G: a tall G is l x s
+  const int64_t ldg = tall ? g.s0 : g.l0;  // row length of G: a tall G is l0 x s0
   const float tau = g.clip ? m.scalars[g.ix.tau] : __int_as_float(0x7f800000);
   const float inv = m.scalars[g.ix.inv];
   const float sg = m.scalars[g.ix.sg_X0];
@@ -470,17 +472,24 @@ __global__ void __launch_bounds__(512, 3) kp_prep_operands(const __grid_constant
   // input's rows go straight to shared memory with asynchronous 16-byte copies (64 KB in flight
   // per block without holding registers); a tall input's tile is filled transposed from registers.
   auto x0 = [&](float gval) { return __fmul_rn(fminf(fmaxf(gval, -tau), tau), inv); };
+  // Rows and columns beyond the caller's matrix are zero padding (source size 0 of the copy
+  // fills with zeros); the dimensions are multiples of 16, so a 16-byte piece is all in or all out.
   if (!tall) {
 #pragma unroll
     for (int rr = warp; rr < 128; rr += 16) {
-      const float* src = m.G + (r0 + rr) * ldg + c0 + lane * 4;
-      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(xs + rr * P + lane * 4)), "l"(src) : "memory");
+      const bool in = (r0 + rr) < g.s0 && (c0 + lane * 4) < g.l0;
+      const float* src = in ? m.G + (r0 + rr) * ldg + c0 + lane * 4 : m.G;
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_u32(xs + rr * P + lane * 4)), "l"(src),
+                   "r"(in ? 16 : 0)
+                   : "memory");
     }
     asm volatile("cp.async.wait_all;" ::: "memory");
   } else {
 #pragma unroll 4
     for (int rr = warp; rr < 128; rr += 16) {
-      const float4 v = __ldg(reinterpret_cast<const float4*>(m.G + (c0 + rr) * ldg + r0) + lane);
+      const bool in = (c0 + rr) < g.l0 && (r0 + lane * 4) < g.s0;
+      float4 v = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+      if (in) v = __ldg(reinterpret_cast<const float4*>(m.G + (c0 + rr) * ldg + r0) + lane);
       xs[(lane * 4 + 0) * P + rr] = v.x; xs[(lane * 4 + 1) * P + rr] = v.y;
       xs[(lane * 4 + 2) * P + rr] = v.z; xs[(lane * 4 + 3) * P + rr] = v.w;
     }
@@ -490,8 +499,9 @@ __global__ void __launch_bounds__(512, 3) kp_prep_operands(const __grid_constant
 #pragma unroll 4
     for (int rr = warp; rr < 128; rr += 16) {
       const float* row = xs + rr * P + lane * 4;
-      *reinterpret_cast<float4*>(m.X + (r0 + rr) * l + c0 + lane * 4) =
-          make_float4(x0(row[0]), x0(row[1]), x0(row[2]), x0(row[3]));
+      if ((r0 + rr) < m.x_rows && (c0 + lane * 4) < m.x_cols)
+        *reinterpret_cast<float4*>(m.X + (r0 + rr) * m.x_cols + c0 + lane * 4) =
+            make_float4(x0(row[0]), x0(row[1]), x0(row[2]), x0(row[3]));
     }
   }
   if (!g.write_q) return;
@@ -564,11 +574,12 @@ cudaError_t launch_prologue_group(const PrologueItem* items, int count, int writ
     PrepGroup g;
     memset(&g, 0, sizeof(g));
     g.count = nn;
-    g.n4 = pl.s * pl.l / 4;
+    g.n4 = pl.s0 * pl.l0 / 4;
     g.s = pl.s; g.l = pl.l;
+    g.s0 = pl.s0; g.l0 = pl.l0;
     g.clip = pl.clip;
     g.clip_rank = (uint32_t)pl.clip_rank;
-    const int64_t cap = pl.s * pl.l / 8 < pl.s * pl.s ? pl.s * pl.l / 8 : pl.s * pl.s;
+    const int64_t cap = pl.s0 * pl.l0 / 8 < pl.s * pl.s ? pl.s0 * pl.l0 / 8 : pl.s * pl.s;
     g.cand_cap = (uint32_t)cap;
     g.eps = pl.eps;
     g.stat_blocks = pl.stat_blocks;
@@ -591,6 +602,7 @@ cudaError_t launch_prologue_group(const PrologueItem* items, int count, int writ
       m.tall = it.pl->tall;
       m.clear_status = it.clear_status ? 1 : 0;
       m.store_x = it.store_x ? 1 : 0;
+      m.x_rows = it.x_rows; m.x_cols = it.x_cols;
     }
     const int sms = pl.sms;
     int64_t hb = (g.n4 + 512 * 4 - 1) / (512 * 4);

@@ -127,15 +127,17 @@ __global__ void __launch_bounds__(256) k_quantize_rows_opts(const float* __restr
   scales[sf_offset(r, kb, cols >> 4)] = (uint8_t)sb;
 }
 
-// out (m x n, m > n) = X^T where X is n x m: 32 x 32 tiles through shared memory
-__global__ void __launch_bounds__(256) k_transpose_out(const float* __restrict__ X, int64_t s, int64_t l,
-                                                       float* __restrict__ out) {
+// out (l0 x s0) = the leading s0 x l0 part of X^T, X being s x l (row pitch l): 32 x 32 tiles through
+// shared memory
+__global__ void __launch_bounds__(256) k_transpose_out(const float* __restrict__ X, int64_t l, float* __restrict__ out,
+                                                       int64_t s0, int64_t l0) {
   __shared__ float t[32][33];
-  const int64_t r0 = (int64_t)blockIdx.y * 32, c0 = (int64_t)blockIdx.x * 32;  // in X (s x l)
+  const int64_t r0 = (int64_t)blockIdx.y * 32, c0 = (int64_t)blockIdx.x * 32;  // in X
   const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
-  for (int j = ty; j < 32; j += 8) t[j][tx] = X[(r0 + j) * l + c0 + tx];
+  for (int j = ty; j < 32; j += 8) t[j][tx] = X[(r0 + j) * l + c0 + tx];   // inside the padded work matrix
   __syncthreads();
-  for (int j = ty; j < 32; j += 8) out[(c0 + j) * s + r0 + tx] = t[tx][j];
+  for (int j = ty; j < 32; j += 8)
+    if (c0 + j < l0 && r0 + tx < s0) out[(c0 + j) * s0 + r0 + tx] = t[tx][j];
 }
 
 // ----------------------------------------------------------------------------------
@@ -168,10 +170,12 @@ cudaError_t launch_quantize(const float* x, int64_t rows, int64_t cols, uint8_t*
   return cudaGetLastError();
 }
 
-cudaError_t launch_transpose_out(const float* X, int64_t s, int64_t l, float* out, cudaStream_t st) {
-  dim3 grid((unsigned)(l / 32), (unsigned)(s / 32));
+cudaError_t launch_transpose_out(const float* X, int64_t s, int64_t l, float* out, int64_t s0, int64_t l0,
+                                 cudaStream_t st) {
+  dim3 grid((unsigned)((l0 + 31) / 32), (unsigned)((s0 + 31) / 32));
+  (void)s;
   count_launches(1);
-  k_transpose_out<<<grid, 256, 0, st>>>(X, s, l, out);
+  k_transpose_out<<<grid, 256, 0, st>>>(X, l, out, s0, l0);
   return cudaGetLastError();
 }
 

@@ -78,6 +78,9 @@ const DeviceInfo* device_info() {
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 inline bool shape_ok(int64_t v) { return v >= 128 && v % 128 == 0 && v <= (1 << 20); }
+// The Newton-Schulz entry points pad internally: any positive multiple of the block length.
+inline bool ns_shape_ok(int64_t v) { return v >= 16 && v % 16 == 0 && v <= (1 << 20); }
+inline int64_t pad128(int64_t v) { return (v + 127) / 128 * 128; }
 
 // 2-D map over a row-major byte matrix (NVFP4 codes): box = one operand stage (64 or 128 bytes
 // x 128 rows), swizzled over the box width.
@@ -179,13 +182,17 @@ void coeffs(int64_t m, int64_t n, float abc[3]) {
 
 // Workspace layout of one matrix.
 fp4_status make_plan(int64_t m, int64_t n, int steps, const fp4_ns_params* p, int sms, NsPlan* pl) {
-  if (!shape_ok(m) || !shape_ok(n)) return FP4_ERR_SHAPE;
+  if (!ns_shape_ok(m) || !ns_shape_ok(n)) return FP4_ERR_SHAPE;
   if (steps < 0 || steps > kMaxSteps) return FP4_ERR_INVALID_ARG;
   memset(pl, 0, sizeof(*pl));
   pl->m = m; pl->n = n;
   pl->tall = m > n;
-  pl->s = m < n ? m : n;
-  pl->l = m < n ? n : m;
+  pl->s0 = m < n ? m : n;
+  pl->l0 = m < n ? n : m;
+  // Zero rows and columns stay zero through the iteration and add nothing to any product or
+  // maximum; since the dimensions are multiples of 16 no block mixes data and padding.
+  pl->s = pad128(pl->s0);
+  pl->l = pad128(pl->l0);
   const int64_t s = pl->s, l = pl->l;
   pl->clip = p->clip_quantile > 0.0f && p->clip_quantile < 1.0f;
   pl->clip_rank = pl->clip ? quantile_rank(m * n, p->clip_quantile) : 0;
@@ -237,6 +244,7 @@ struct MatrixCtx {
   GemmProblem g1, g2, g3[2];  // g3[cur]: reads qXt[cur], writes qXt[cur ^ 1]
   GemmProblem g3_first;       // iteration 0: as g3[0], but a wide input's FP32 tile is G itself (no X0 copy)
   bool store_x0;              // the prologue writes X0 in FP32
+  int64_t x_rows, x_cols;     // extent (and row pitch) of X
 };
 
 fp4_status prepare_matrix(const DeviceInfo* d, const float* G, float* out, int64_t m, int64_t n, int steps,
@@ -247,6 +255,10 @@ fp4_status prepare_matrix(const DeviceInfo* d, const float* G, float* out, int64
   const int64_t s = c->pl.s, l = c->pl.l;
   c->G = G; c->out = out; c->ws = ws;
   c->X = c->pl.tall ? reinterpret_cast<float*>(ws + L.X) : out;
+  // extent of X: the padded work shape in the workspace, the caller's shape in `out` (TMA fills what
+  // lies outside with zeros on loads and drops it on stores)
+  const int64_t xr = c->pl.tall ? s : c->pl.s0, xc = c->pl.tall ? l : c->pl.l0;
+  c->x_rows = xr; c->x_cols = xc;
   c->store_x0 = c->pl.tall || steps == 0;
   if (steps == 0) return FP4_OK;
   float abc[3] = {p->a, p->b, p->c};
@@ -261,12 +273,13 @@ fp4_status prepare_matrix(const DeviceInfo* d, const float* G, float* out, int64
             make_codes_map(d, &tm_qXt[1], ws + L.qXt_codes[1], l, s / 2) &&
             make_codes_map(d, &tm_qA, ws + L.qA_codes, s, s / 2) &&
             make_codes_map(d, &tm_qB, ws + L.qB_codes, s, s / 2) &&
-            make_f32_map(d, &tm_A, ws + L.A, s, s) && make_f32_map(d, &tm_X, c->X, s, l);
+            make_f32_map(d, &tm_A, ws + L.A, s, s) && make_f32_map(d, &tm_X, c->X, xr, xc);
   if (!ok) return FP4_ERR_CUDA;
   GemmProblem base;
   memset(&base, 0, sizeof(base));
   base.scalars = reinterpret_cast<float*>(ws + L.scalars);
   base.ca = abc[0]; base.cb = abc[1]; base.cc = abc[2];
+  base.out_rows = (int)s; base.out_cols = (int)s;
   // G1: A = qX qX^T (upper-triangle tiles), qA in both triangles
   c->g1 = base;
   c->g1.tmA = c->g1.tmB = tm_qX; c->g1.tmAux = c->g1.tmOut = tm_A;
@@ -284,6 +297,7 @@ fp4_status prepare_matrix(const DeviceInfo* d, const float* G, float* out, int64
     GemmProblem& g = c->g3[cur];
     g = base;
     g.tmA = tm_qB; g.tmB = tm_qXt[cur]; g.tmAux = g.tmOut = tm_X;
+    g.out_rows = (int)xr; g.out_cols = (int)xc;
     g.tmSfa = sf_qB; g.tmSfb = sf_qXt[cur];
     g.sfa = ws + L.qB_scales; g.sfb = ws + L.qXt_scales[cur];
     g.rq_codes = ws + L.qX_codes; g.rq_sf = ws + L.qX_scales;
@@ -292,7 +306,7 @@ fp4_status prepare_matrix(const DeviceInfo* d, const float* G, float* out, int64
   c->g3_first = c->g3[0];
   if (!c->store_x0) {
     CUtensorMap tm_G;
-    if (!make_f32_map(d, &tm_G, G, s, l)) return FP4_ERR_CUDA;
+    if (!make_f32_map(d, &tm_G, G, c->pl.s0, c->pl.l0)) return FP4_ERR_CUDA;
     c->g3_first.tmAux = tm_G;
     c->g3_first.aux_raw = 1;
   }
@@ -323,7 +337,7 @@ fp4_status run_group(const DeviceInfo* d, MatrixCtx* mats, int count, int steps,
     std::vector<PrologueItem> items((size_t)count);
     for (int i = 0; i < count; ++i) {
       MatrixCtx& c = mats[i];
-      items[(size_t)i] = PrologueItem{c.G, c.X, c.ws, &c.pl, clear_first_status && i == 0, c.store_x0};
+      items[(size_t)i] = PrologueItem{c.G, c.X, c.ws, &c.pl, clear_first_status && i == 0, c.store_x0, c.x_rows, c.x_cols};
     }
     if (launch_prologue_group(items.data(), count, steps > 0 || keep, quant_opts(p, 0), st) != cudaSuccess)
       return FP4_ERR_CUDA;
@@ -391,7 +405,7 @@ fp4_status run_group(const DeviceInfo* d, MatrixCtx* mats, int count, int steps,
   for (int i = 0; i < count; ++i) {
     if (mats[i].pl.tall) {
       ProfScope ps(FP4_PROF_TRANSPOSE, st);
-      if (launch_transpose_out(mats[i].X, s, l, mats[i].out, st) != cudaSuccess) return FP4_ERR_CUDA;
+      if (launch_transpose_out(mats[i].X, s, l, mats[i].out, pl0.s0, pl0.l0, st) != cudaSuccess) return FP4_ERR_CUDA;
     }
   }
   return FP4_OK;
@@ -423,7 +437,7 @@ const char* fp4_status_string(fp4_status s) {
   switch (s) {
     case FP4_OK: return "ok";
     case FP4_ERR_INVALID_ARG: return "invalid argument";
-    case FP4_ERR_SHAPE: return "unsupported shape (dimensions must be positive multiples of 128)";
+    case FP4_ERR_SHAPE: return "unsupported shape (Newton-Schulz entry points: positive multiples of 16; fp4_quantize, fp4_gemm_nt: of 128)";
     case FP4_ERR_ALIGNMENT: return "misaligned pointer";
     case FP4_ERR_WORKSPACE: return "workspace too small";
     case FP4_ERR_ARCH: return "device is not compute capability 10.x (sm_100a kernels only, no fallback)";
@@ -490,7 +504,7 @@ fp4_status fp4_root_ns(const float* G, float* out, int64_t m, int64_t n, int ste
   fp4_ns_params dp;
   if (!p) { default_params(&dp); p = &dp; }
   if (!G || !out || !ws) return FP4_ERR_INVALID_ARG;
-  if (!shape_ok(m) || !shape_ok(n)) return FP4_ERR_SHAPE;
+  if (!ns_shape_ok(m) || !ns_shape_ok(n)) return FP4_ERR_SHAPE;
   if (steps < 0 || steps > kMaxSteps) return FP4_ERR_INVALID_ARG;
   if (!aligned(G, 16) || !aligned(out, 16) || !aligned(ws, 256)) return FP4_ERR_ALIGNMENT;
   const size_t need = fp4_root_ns_workspace_bytes(m, n, steps, p->flags);
@@ -526,7 +540,7 @@ fp4_status fp4_root_ns_batched(int count, const float* const* G, float* const* o
   if (!aligned(ws, 256)) return FP4_ERR_ALIGNMENT;
   for (int i = 0; i < count; ++i) {
     if (!G[i] || !out[i]) return FP4_ERR_INVALID_ARG;
-    if (!shape_ok(m[i]) || !shape_ok(n[i])) return FP4_ERR_SHAPE;
+    if (!ns_shape_ok(m[i]) || !ns_shape_ok(n[i])) return FP4_ERR_SHAPE;
     if (!aligned(G[i], 16) || !aligned(out[i], 16)) return FP4_ERR_ALIGNMENT;
   }
   if (count == 0) return FP4_OK;
@@ -560,7 +574,7 @@ fp4_status fp4_root_ns_batched(int count, const float* const* G, float* const* o
     group.clear();
     for (int j = i; j < count && (int)group.size() < cap; ++j) {
       if (done[(size_t)j]) continue;
-      if (ctx[(size_t)j].pl.s == ctx[(size_t)i].pl.s && ctx[(size_t)j].pl.l == ctx[(size_t)i].pl.l) {
+      if (ctx[(size_t)j].pl.s0 == ctx[(size_t)i].pl.s0 && ctx[(size_t)j].pl.l0 == ctx[(size_t)i].pl.l0) {
         group.push_back(ctx[(size_t)j]);
         done[(size_t)j] = 1;
       }
@@ -600,6 +614,7 @@ fp4_status fp4_gemm_nt(const uint8_t* a_codes, const uint8_t* a_scales, float a_
   pr.tmAux = pr.tmOut;
   pr.sfa = a_scales; pr.sfb = b_scales;
   pr.sg_a = a_tensor_scale; pr.sg_b = b_tensor_scale;
+  pr.out_rows = (int)M; pr.out_cols = (int)N;
   GemmLaunch L;
   memset(&L, 0, sizeof(L));
   L.num_problems = 1;
@@ -643,7 +658,7 @@ fp4_status fp4_root_ns_static(const float* G, float* out, int64_t m, int64_t n, 
   fp4_ns_params dp;
   if (!p) { default_params(&dp); p = &dp; }
   if (!G || !out) return FP4_ERR_INVALID_ARG;
-  if (!shape_ok(m) || !shape_ok(n)) return FP4_ERR_SHAPE;
+  if (!ns_shape_ok(m) || !ns_shape_ok(n)) return FP4_ERR_SHAPE;
   if (steps < 0 || steps > kMaxSteps) return FP4_ERR_INVALID_ARG;
   if (!aligned(G, 16) || !aligned(out, 16) || (device_status && !aligned(device_status, 4))) return FP4_ERR_ALIGNMENT;
   const size_t need = fp4_root_ns_workspace_bytes(m, n, steps, p->flags);

@@ -191,6 +191,41 @@ def test_batched_mixed_orientations_in_one_group_paper_options():
         assert rel(single, oracle.root_ns(g, steps=3, rht=True, four_six=True, seed=77)) <= TOL_OUT
 
 
+@pytest.mark.parametrize("shape", [(144, 272), (272, 144), (208, 208), (16, 64), (400, 1040), (1040, 400)])
+def test_shapes_that_are_not_multiples_of_128(shape):
+    """Dimensions that are multiples of the block length 16 are zero-padded to the tile size
+    inside the library; the oracle works on the matrix as it is.  Padding must be invisible:
+    the clip rank counts the caller's elements only, zero rows and columns stay zero."""
+    m, n = shape
+    G = workloads.gradient_like(m, n, seed=21)
+    for steps in (0, 1, 3):
+        got, ws = run_gpu(G, steps=steps)
+        want = oracle.root_ns(G, steps=steps)
+        assert got.shape == (m, n) and np.isfinite(got).all()
+        assert rel(got, want) <= (1e-6 if steps == 0 else TOL_OUT), (steps, rel(got, want))
+    # in place, and the two orientations agree bit for bit
+    inplace, _ = run_gpu(G, steps=3, in_place=True)
+    assert np.array_equal(inplace, got)
+    if m != n:
+        t, _ = run_gpu(np.ascontiguousarray(G.T), steps=3)
+        assert np.array_equal(t.T, got)
+
+
+def test_batched_with_padded_shapes():
+    specs = [(144, 272, 1), (272, 144, 2), (144, 272, 3), (256, 512, 4), (208, 208, 5)]
+    mats = [workloads.gradient_like(m, n, seed=sd) for m, n, sd in specs]
+    Gs = [torch.from_numpy(g).cuda() for g in mats]
+    outs = [torch.full_like(g, float("nan")) for g in Gs]
+    shapes = [tuple(g.shape) for g in Gs]
+    ws = torch.empty(fp4.fp4_root_ns_batched_workspace_bytes(shapes, 4), dtype=torch.uint8, device="cuda")
+    fp4.fp4_root_ns_batched(Gs, outs, 4, None, ws)
+    assert fp4.fp4_last_device_status(ws) == 0
+    for g, o in zip(mats, outs):
+        single, _ = run_gpu(g, steps=4)
+        assert np.array_equal(o.cpu().numpy(), single)
+        assert rel(single, oracle.root_ns(g, steps=4)) <= TOL_OUT
+
+
 def test_cuda_graph_replay_matches_direct_call():
     """The call only enqueues kernels on its stream: it can be captured in a CUDA graph
     (after one direct call has done the library's per-device set-up) and replayed."""
