@@ -36,65 +36,34 @@ __global__ void __launch_bounds__(256) k_amax(const float4* __restrict__ x, int6
 }
 
 // ----------------------------------------------------------------------------------
-// Row quantiser.  A warp walks one row segment: each lane loads one float4 per step, so a
-// step covers 128 consecutive elements = 8 blocks of 16 with fully coalesced 512-byte
-// requests.  Four neighbouring lanes own one block: block amax by two xor-shuffles; the
-// 8 code bytes of a block and the 4 scale bytes of a 64-element group are gathered by
-// shuffles so that each store is 8 or 4 bytes wide.  Four steps are in flight per lane.
-// grid: x = segments of kSegment columns, y = groups of 8 rows (one per warp).
+// Row quantiser: one thread per block of 16 (four 128-bit loads = 64 contiguous bytes, a warp
+// covers 512 consecutive elements of a row), so the two IEEE divisions of a block are done
+// once; 8-byte code store and 1-byte scale store per thread.  Thread blocks walk the tensor
+// from its end: the amax pass has just read it front to back, so the end is what L2 still
+// holds.  grid: rows x ceil(cols / 4096) thread blocks.
 // amax_bits holds the tensor amax on entry (bit pattern).
 // ----------------------------------------------------------------------------------
-constexpr int kSegment = 4096;  // columns per block and row
-
-__device__ __forceinline__ void quantize_step(float4 v, float six_sg, float sg, int lane, uint8_t* code_dst,
-                                              uint8_t* sf_dst) {
-  float a = amax4(v);
-  a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 1));
-  a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 2));
-  const uint32_t sb = cvt_ue4m3(__fdiv_rn(a, six_sg));
-  const float d = __fmul_rn(ue4m3_to_float(sb), sg);
-  uint32_t w = 0;
-  if (d != 0.0f) {
-    const float rcp = __frcp_rn(d);
-    w = cvt_e2m1x2(__fmul_rn(v.x, rcp), __fmul_rn(v.y, rcp)) |
-        (cvt_e2m1x2(__fmul_rn(v.z, rcp), __fmul_rn(v.w, rcp)) << 8);
-  }
-  // codes: 4 lanes x 16 bits -> one 8-byte store by the first lane of the block
-  const uint32_t w2 = w | (__shfl_down_sync(0xffffffffu, w, 1) << 16);
-  const uint32_t w3 = __shfl_down_sync(0xffffffffu, w2, 2);
-  // scales: 4 blocks (16 lanes) -> one 4-byte store
-  const uint32_t s2 = sb | (__shfl_down_sync(0xffffffffu, sb, 4) << 8);
-  const uint32_t s4 = s2 | (__shfl_down_sync(0xffffffffu, s2, 8) << 16);
-  if ((lane & 3) == 0) *reinterpret_cast<uint2*>(code_dst + (lane >> 2) * 8) = make_uint2(w2, w3);
-  if ((lane & 15) == 0) *reinterpret_cast<uint32_t*>(sf_dst + (lane >> 4) * 512) = s4;
-}
-
 __global__ void __launch_bounds__(256) k_quantize_rows(const float* __restrict__ x, int64_t rows, int64_t cols,
                                                        uint8_t* __restrict__ codes, uint8_t* __restrict__ scales,
                                                        const uint32_t* __restrict__ amax_bits) {
   const float sg = scale_exact(__uint_as_float(*amax_bits));
   const float six_sg = __fmul_rn(6.0f, sg);
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int64_t r = (int64_t)blockIdx.y * 8 + warp;
-  if (r >= rows) return;
-  const int64_t c_begin = (int64_t)blockIdx.x * kSegment;
-  const int64_t c_end = c_begin + kSegment < cols ? c_begin + kSegment : cols;
-  const float4* src = reinterpret_cast<const float4*>(x + r * cols);
-  uint8_t* crow = codes + r * (cols / 2);
-  // scale atoms of this row: atom (r / 128, c / 64) is 512 bytes; within it this row owns
-  // 4 consecutive bytes at (r % 32) * 16 + ((r % 128) / 32) * 4
-  uint8_t* srow = scales + (size_t)(r >> 7) * (size_t)(cols >> 6) * 512 + (r & 31) * 16 + ((r & 127) >> 5) * 4;
-  int64_t c = c_begin;
-  for (; c + 512 <= c_end; c += 512) {
-    float4 v[4];
+  const int64_t groups = ((cols >> 4) + 255) / 256;  // thread blocks per row
+  const int64_t bid = (int64_t)gridDim.x - 1 - blockIdx.x;
+  const int64_t r = bid / groups;
+  const int64_t kb = (bid % groups) * 256 + threadIdx.x;
+  if (r >= rows || kb >= (cols >> 4)) return;
+  const float4* src = reinterpret_cast<const float4*>(x + r * cols + kb * 16);
+  float v[16];
 #pragma unroll
-    for (int u = 0; u < 4; ++u) v[u] = __ldg(src + (c + u * 128) / 4 + lane);
-#pragma unroll
-    for (int u = 0; u < 4; ++u)
-      quantize_step(v[u], six_sg, sg, lane, crow + (c + u * 128) / 2, srow + ((c + u * 128) >> 6) * 512);
+  for (int j = 0; j < 4; ++j) {
+    const float4 t = __ldg(src + j);
+    v[4 * j] = t.x; v[4 * j + 1] = t.y; v[4 * j + 2] = t.z; v[4 * j + 3] = t.w;
   }
-  for (; c < c_end; c += 128)
-    quantize_step(__ldg(src + c / 4 + lane), six_sg, sg, lane, crow + c / 2, srow + (c >> 6) * 512);
+  uint32_t lo, hi;
+  const uint32_t sb = quantize_block16(v, six_sg, sg, lo, hi);
+  *reinterpret_cast<uint2*>(codes + r * (cols / 2) + kb * 8) = make_uint2(lo, hi);
+  scales[sf_offset(r, kb, cols >> 4)] = (uint8_t)sb;
 }
 
 __global__ void k_finish_tensor_scale(float* ts, float widen) {
@@ -110,8 +79,9 @@ __global__ void __launch_bounds__(256) k_quantize_rows_opts(const float* __restr
                                                             const QuantOpts q) {
   const float sg = scale_exact(__fmul_rn(q.widen, __uint_as_float(*amax_bits)));
   const int64_t groups = ((cols >> 4) + 255) / 256;  // thread blocks per row
-  const int64_t r = blockIdx.x / groups;
-  const int64_t kb = (blockIdx.x % groups) * 256 + threadIdx.x;
+  const int64_t bid = (int64_t)gridDim.x - 1 - blockIdx.x;  // from the end, as k_quantize_rows
+  const int64_t r = bid / groups;
+  const int64_t kb = (bid % groups) * 256 + threadIdx.x;
   if (r >= rows || kb >= (cols >> 4)) return;
   const float4* src = reinterpret_cast<const float4*>(x + r * cols + kb * 16);
   float v[16];
@@ -156,15 +126,13 @@ cudaError_t launch_quantize(const float* x, int64_t rows, int64_t cols, uint8_t*
   if (e != cudaSuccess) return e;
   k_amax<<<grid_for(n4, 256 * 8, sms), 256, 0, st>>>(reinterpret_cast<const float4*>(x), n4,
                                                     reinterpret_cast<uint32_t*>(tensor_scale));
-  if (q.rht || q.four_six) {
-    const unsigned qgrid = (unsigned)(((cols / 16 + 255) / 256) * rows);
+  const unsigned qgrid = (unsigned)(((cols / 16 + 255) / 256) * rows);
+  if (q.rht || q.four_six)
     k_quantize_rows_opts<<<qgrid, 256, 0, st>>>(x, rows, cols, codes, scales,
                                                 reinterpret_cast<const uint32_t*>(tensor_scale), q);
-  } else {
-    const dim3 qgrid((unsigned)((cols + kSegment - 1) / kSegment), (unsigned)((rows + 7) / 8));
+  else
     k_quantize_rows<<<qgrid, 256, 0, st>>>(x, rows, cols, codes, scales,
                                            reinterpret_cast<const uint32_t*>(tensor_scale));
-  }
   k_finish_tensor_scale<<<1, 1, 0, st>>>(tensor_scale, q.widen);
   count_launches(3);
   return cudaGetLastError();
