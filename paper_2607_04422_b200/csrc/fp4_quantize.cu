@@ -97,17 +97,28 @@ __global__ void __launch_bounds__(256) k_quantize_rows_opts(const float* __restr
   scales[sf_offset(r, kb, cols >> 4)] = (uint8_t)sb;
 }
 
-// out (l0 x s0) = the leading s0 x l0 part of X^T, X being s x l (row pitch l): 32 x 32 tiles through
-// shared memory
+// out (l0 x s0) = the leading s0 x l0 part of X^T, X being s x l (row pitch l): 64 x 64 tiles through
+// shared memory, 128-bit loads along the rows of X and 128-bit stores along the rows of out
+// (s0 and l0 are multiples of 16, so a 16-byte piece is all inside or all outside).
 __global__ void __launch_bounds__(256) k_transpose_out(const float* __restrict__ X, int64_t l, float* __restrict__ out,
                                                        int64_t s0, int64_t l0) {
-  __shared__ float t[32][33];
-  const int64_t r0 = (int64_t)blockIdx.y * 32, c0 = (int64_t)blockIdx.x * 32;  // in X
-  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
-  for (int j = ty; j < 32; j += 8) t[j][tx] = X[(r0 + j) * l + c0 + tx];   // inside the padded work matrix
+  __shared__ float t[64][65];
+  const int64_t r0 = (int64_t)blockIdx.y * 64, c0 = (int64_t)blockIdx.x * 64;  // tile origin in X
+  const int q = threadIdx.x & 15, row = threadIdx.x >> 4;                      // 16 pieces per row, 16 rows per sweep
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int r = row + 16 * j;
+    const float4 v = __ldg(reinterpret_cast<const float4*>(X + (r0 + r) * l + c0) + q);  // inside the padded work matrix
+    t[r][4 * q] = v.x; t[r][4 * q + 1] = v.y; t[r][4 * q + 2] = v.z; t[r][4 * q + 3] = v.w;
+  }
   __syncthreads();
-  for (int j = ty; j < 32; j += 8)
-    if (c0 + j < l0 && r0 + tx < s0) out[(c0 + j) * s0 + r0 + tx] = t[tx][j];
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const int c = row + 16 * j;  // column of X = row of out
+    if (c0 + c < l0 && r0 + 4 * q < s0)
+      *reinterpret_cast<float4*>(out + (c0 + c) * s0 + r0 + 4 * q) =
+          make_float4(t[4 * q][c], t[4 * q + 1][c], t[4 * q + 2][c], t[4 * q + 3][c]);
+  }
 }
 
 // ----------------------------------------------------------------------------------
@@ -140,7 +151,7 @@ cudaError_t launch_quantize(const float* x, int64_t rows, int64_t cols, uint8_t*
 
 cudaError_t launch_transpose_out(const float* X, int64_t s, int64_t l, float* out, int64_t s0, int64_t l0,
                                  cudaStream_t st) {
-  dim3 grid((unsigned)((l0 + 31) / 32), (unsigned)((s0 + 31) / 32));
+  dim3 grid((unsigned)((l0 + 63) / 64), (unsigned)((s0 + 63) / 64));
   (void)s;
   count_launches(1);
   k_transpose_out<<<grid, 256, 0, st>>>(X, l, out, s0, l0);
