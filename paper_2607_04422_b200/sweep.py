@@ -102,6 +102,14 @@ def main():
                               "tflops_algorithmic": round(alg / ms / 1e9, 1),
                               "tflops_dense_equivalent": round(1.5 * alg / ms / 1e9, 1),
                               "pct_of_9pf": round(alg / ms / 1e9 / 90.0, 2)}), flush=True)
+        if size <= 2048:
+            # launch-latency-bound sizes: the same 5-iteration call replayed from a CUDA graph
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                fp4.fp4_root_ns(G, out, 5, None, ws, torch.cuda.current_stream())
+            ms = _time(graph.replay, a.reps, stream)
+            print(json.dumps({"case": "fp4_root_ns_graph", "size": size, "steps": 5, "ms": round(ms, 4),
+                              "tflops_algorithmic": round(5 * 4.0 * size ** 3 / ms / 1e9, 1)}), flush=True)
         status = fp4.fp4_last_device_status(ws)
         assert status == 0, status
         del G, out, ws, codes, scales
