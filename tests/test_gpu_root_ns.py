@@ -211,6 +211,32 @@ def test_shapes_that_are_not_multiples_of_128(shape):
         assert np.array_equal(t.T, got)
 
 
+@pytest.mark.parametrize("shape", [(128, 4096), (4096, 128), (16, 16), (16, 2048)])
+def test_extreme_aspect_ratios(shape):
+    m, n = shape
+    G = workloads.gaussian(m, n, seed=4)
+    got, _ = run_gpu(G, steps=2)
+    want = oracle.root_ns(G, steps=2)
+    assert rel(got, want) <= TOL_OUT, rel(got, want)
+
+
+def test_largest_sweep_size_properties():
+    """16384 x 16384 (the largest size of the scaling sweep, 1 GiB of FP32): no oracle run at this
+    size; the result must be finite, and one iteration of the quintic must have moved the
+    singular values towards 1 (the Frobenius norm of X0 is 1, so ||X1||_F > 1)."""
+    size = 16384
+    gen = torch.Generator(device="cuda"); gen.manual_seed(1)
+    G = torch.randn((size, size), device="cuda", generator=gen)
+    out = torch.empty_like(G)
+    ws = torch.empty(fp4.fp4_root_ns_workspace_bytes(size, size, 1), dtype=torch.uint8, device="cuda")
+    fp4.fp4_root_ns(G, out, 1, None, ws)
+    assert fp4.fp4_last_device_status(ws) == 0
+    assert bool(torch.isfinite(out).all())
+    nrm = float(out.double().norm())
+    a = fp4.fp4_root_coeffs(size, size, 1)[0]
+    assert 1.2 < nrm < a * 1.05, nrm          # every singular value grows by at most the slope a at zero
+
+
 def test_batched_with_padded_shapes():
     specs = [(144, 272, 1), (272, 144, 2), (144, 272, 3), (256, 512, 4), (208, 208, 5)]
     mats = [workloads.gradient_like(m, n, seed=sd) for m, n, sd in specs]
