@@ -46,6 +46,10 @@ def test_scale_bytes_and_workspace_sizes():
     assert fp4.fp4_scale_bytes(128, 128) == 1024
     assert fp4.fp4_scale_bytes(256, 512) == 2 * 8 * 512
     assert fp4.fp4_root_ns_workspace_bytes(100, 128) == 0
+    # multiples of 16 are padded to multiples of 128 inside the workspace
+    assert fp4.fp4_root_ns_workspace_bytes(144, 272, 5) == fp4.fp4_root_ns_workspace_bytes(256, 384, 5)
+    assert fp4.fp4_root_ns_workspace_bytes(16, 16, 5) == fp4.fp4_root_ns_workspace_bytes(128, 128, 5)
+    assert fp4.fp4_root_ns_workspace_bytes(136, 128, 5) == 0                      # not a multiple of 16
     small = fp4.fp4_root_ns_workspace_bytes(128, 256, 5)
     big = fp4.fp4_root_ns_workspace_bytes(3072, 8192, 5)
     assert 0 < small < big
