@@ -238,6 +238,18 @@ void fp4_profile_enable(int on);
 fp4_status fp4_profile_collect(float* ms, int* groups);
 uint64_t fp4_kernel_launches(void);
 
+/* ---- self-test of the bounded device-side waits (the paper has no counterpart) -------------
+ * Every wait of the GEMM kernels on a shared-memory barrier gives up after a time limit,
+ * raises the CTA's abort flag and ends normally, leaving FP4_ERR_DEVICE_TIMEOUT in the status
+ * word.  This entry point runs that same wait routine in a one-warp kernel on a barrier that
+ * nothing ever arrives on, with a limit of limit_us microseconds (1 .. 100000), after a
+ * second barrier whose arrival it does see.
+ * device_status: device, one uint32, out: FP4_ERR_DEVICE_TIMEOUT if the first wait was seen
+ *   to succeed and the second to time out (what must happen), FP4_ERR_INVALID_ARG otherwise.
+ * The kernel neither traps nor spins past the limit; the context stays usable.
+ */
+fp4_status fp4_selftest_bounded_wait(uint32_t* device_status, uint32_t limit_us, cudaStream_t stream);
+
 #ifdef __cplusplus
 }
 #endif

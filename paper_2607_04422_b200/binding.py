@@ -26,7 +26,8 @@ FP4_STATIC_SCRATCH_BYTES = 16 << 20
 EXPORTS = ("fp4_status_string", "fp4_scale_bytes", "fp4_quantize", "fp4_root_coeffs",
            "fp4_root_ns_workspace_bytes", "fp4_root_ns", "fp4_root_ns_batched_workspace_bytes",
            "fp4_root_ns_batched", "fp4_last_device_status", "fp4_root_ns_workspace_layout", "fp4_gemm_nt",
-           "fp4_profile_enable", "fp4_profile_collect", "fp4_kernel_launches", "fp4_root_ns_static")
+           "fp4_profile_enable", "fp4_profile_collect", "fp4_kernel_launches", "fp4_root_ns_static",
+           "fp4_selftest_bounded_wait")
 PROF_CLASSES = ("clip", "stats", "prep", "G1", "G2", "G3", "transpose", "quantize")
 
 
@@ -105,6 +106,7 @@ def load_library():
     L.fp4_profile_collect.argtypes = [C.POINTER(C.c_float), C.POINTER(C.c_int)]
     L.fp4_profile_collect.restype = C.c_int
     L.fp4_kernel_launches.argtypes = []; L.fp4_kernel_launches.restype = C.c_uint64
+    L.fp4_selftest_bounded_wait.argtypes = [vp, u32, vp]; L.fp4_selftest_bounded_wait.restype = C.c_int
     _lib = L
     return L
 
@@ -215,6 +217,11 @@ def fp4_profile_collect():
     groups = (C.c_int * n)()
     _check(load_library().fp4_profile_collect(ms, groups), "fp4_profile_collect")
     return {PROF_CLASSES[i]: (float(ms[i]), int(groups[i])) for i in range(n)}
+
+
+def fp4_selftest_bounded_wait(status: torch.Tensor, limit_us: int, stream=None) -> None:
+    _check(load_library().fp4_selftest_bounded_wait(status.data_ptr(), int(limit_us), _stream(stream)),
+           "fp4_selftest_bounded_wait")
 
 
 def fp4_kernel_launches() -> int:

@@ -11,19 +11,24 @@ __device__ __forceinline__ uint64_t globaltimer_ns() {
   return t;
 }
 
-// Wait on an mbarrier phase for at most two seconds; false on give-up (own time-out or
-// another thread's abort flag).
-static __device__ __noinline__ bool wait_slow(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag) {
+// Wait on an mbarrier phase for at most limit_ns; false on give-up (own time-out or another
+// thread's abort flag).
+static __device__ __noinline__ bool wait_limited(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                                 uint64_t limit_ns) {
   const uint64_t t0 = globaltimer_ns();
   for (;;) {
     for (int i = 0; i < 256; ++i)
       if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (globaltimer_ns() - t0 > 2000000000ull) {
+    if (globaltimer_ns() - t0 > limit_ns) {
       *abort_flag = 1;
       return false;
     }
   }
+}
+constexpr uint64_t kWaitLimitNs = 2000000000ull;  // two seconds
+static __device__ __forceinline__ bool wait_slow(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag) {
+  return wait_limited(bar, parity, abort_flag, kWaitLimitNs);
 }
 __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag) {
   if (mbar_try_wait(bar, parity)) return true;

@@ -6,7 +6,7 @@
 #include <mutex>
 #include <vector>
 
-#include "fp4_kernels.h"
+#include "fp4_gemm_common.cuh"
 
 namespace fp4 {
 
@@ -624,6 +624,37 @@ fp4_status fp4_gemm_nt(const uint8_t* a_codes, const uint8_t* a_scales, float a_
 }
 
 }  // extern "C"
+
+// ---- fp4_selftest_bounded_wait ----------------------------------------------------------------
+namespace fp4 {
+static __global__ void __launch_bounds__(32) k_selftest_wait(uint32_t* status, uint64_t limit_ns) {
+  __shared__ uint64_t bar_seen, bar_never;
+  __shared__ uint32_t abort_flag;
+  if (threadIdx.x == 0) {
+    fp4::mbar_init(&bar_seen, 1);
+    fp4::mbar_init(&bar_never, 1);
+    abort_flag = 0;
+    fp4::mbar_fence_init();
+  }
+  __syncwarp();
+  if (threadIdx.x == 1) fp4::mbar_arrive(&bar_seen);
+  if (threadIdx.x == 0) {
+    const bool first = fp4::wait_bar(&bar_seen, 0, &abort_flag);                 // lane 1 arrives: must succeed
+    const bool second = fp4::wait_limited(&bar_never, 0, &abort_flag, limit_ns);  // nobody arrives: must give up
+    *status = (first && !second && abort_flag == 1) ? (uint32_t)FP4_ERR_DEVICE_TIMEOUT : (uint32_t)FP4_ERR_INVALID_ARG;
+  }
+}
+}  // namespace fp4
+
+extern "C" fp4_status fp4_selftest_bounded_wait(uint32_t* device_status, uint32_t limit_us, cudaStream_t stream) {
+  if (!device_status || limit_us < 1 || limit_us > 100000) return FP4_ERR_INVALID_ARG;
+  const fp4::DeviceInfo* d;
+  fp4_status rc = fp4::check_common(&d);
+  if (rc != FP4_OK) return rc;
+  fp4::count_launches(1);
+  fp4::k_selftest_wait<<<1, 32, 0, stream>>>(device_status, (uint64_t)limit_us * 1000ull);
+  return cudaGetLastError() == cudaSuccess ? FP4_OK : FP4_ERR_CUDA;
+}
 
 // ---- fp4_root_ns_static: the step with the workspace in a static device array ------------
 // For callers that cannot allocate device memory (no cudaMalloc allowed where they run, or

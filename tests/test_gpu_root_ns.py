@@ -274,6 +274,41 @@ def test_cuda_graph_replay_matches_direct_call():
         assert torch.equal(out, direct)
 
 
+def test_bounded_wait_gives_up_and_reports():
+    """The wait routine of the GEMM kernels, run on a barrier that nothing arrives on with a
+    0.2 ms limit: it must give up, report FP4_ERR_DEVICE_TIMEOUT through the status word and
+    leave the context usable (no trap, no endless spin)."""
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    fp4.fp4_selftest_bounded_wait(status, 200)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 7
+    with pytest.raises(fp4.Fp4Error) as e:
+        fp4.fp4_selftest_bounded_wait(status, 0)
+    assert e.value.code == 1
+    G = workloads.config1()
+    got, _ = run_gpu(G, steps=2)                      # the context still works
+    assert rel(got, oracle.root_ns(G, steps=2)) <= TOL_OUT
+
+
+@pytest.mark.parametrize("shape", [(256, 512), (512, 256), (144, 272), (272, 144)])
+def test_nothing_is_written_outside_the_buffers(shape):
+    """Guard regions around the workspace and the result keep their pattern (also with the
+    zero padding of shapes that are not multiples of 128)."""
+    m, n = shape
+    G = torch.from_numpy(workloads.gradient_like(m, n, seed=9)).cuda()
+    guard = 1 << 16
+    need = fp4.fp4_root_ns_workspace_bytes(m, n, 3)
+    big = torch.full((need + 2 * guard,), 0xA5, dtype=torch.uint8, device="cuda")
+    ws = big[guard:guard + need]
+    outbig = torch.full((m * n + 2 * 4096,), 12345.0, device="cuda")
+    out = outbig[4096:4096 + m * n].view(m, n)
+    fp4.fp4_root_ns(G, out, 3, None, ws)
+    assert fp4.fp4_last_device_status(ws) == 0
+    assert bool((big[:guard] == 0xA5).all()) and bool((big[guard + need:] == 0xA5).all())
+    assert bool((outbig[:4096] == 12345.0).all()) and bool((outbig[4096 + m * n:] == 12345.0).all())
+    assert rel(out.cpu().numpy(), oracle.root_ns(G.cpu().numpy(), steps=3)) <= TOL_OUT
+
+
 def test_argument_errors():
     G = torch.zeros((128, 256), device="cuda")
     ws = torch.empty(fp4.fp4_root_ns_workspace_bytes(128, 256, 5), dtype=torch.uint8, device="cuda")
