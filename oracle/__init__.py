@@ -26,7 +26,8 @@ class OrcParams(C.Structure):
     _fields_ = [("a", C.c_float), ("b", C.c_float), ("c", C.c_float),
                 ("clip_quantile", C.c_float), ("eps", C.c_float),
                 ("quantize", C.c_int32), ("exact_scales", C.c_int32),
-                ("rht", C.c_int32), ("four_six", C.c_int32), ("seed", C.c_uint64)]
+                ("rht", C.c_int32), ("four_six", C.c_int32), ("seed", C.c_uint64),
+                ("store_bf16", C.c_int32)]
 
 
 class OrcTrace(C.Structure):
@@ -69,6 +70,7 @@ def lib():
         L.orc_quantize_opts.restype = None
         L.orc_hadamard16.argtypes = [_f32p, C.c_uint16, _f32p]; L.orc_hadamard16.restype = None
         L.orc_rht_mask.argtypes = [C.c_uint64, C.c_uint64]; L.orc_rht_mask.restype = C.c_uint16
+        L.orc_bf16_round.argtypes = [C.c_float]; L.orc_bf16_round.restype = C.c_float
         L.orc_dequantize.argtypes = [_u8p, _u8p, C.c_float, C.c_int64, C.c_int64, _f32p]
         L.orc_dequantize.restype = None
         L.orc_gemm_nt_q.argtypes = [_u8p, _u8p, C.c_float, _u8p, _u8p, C.c_float,
@@ -156,6 +158,12 @@ def rht_mask(seed, idx):
     return int(lib().orc_rht_mask(int(seed), int(idx)))
 
 
+def bf16_round(x):
+    """FP32 -> nearest BF16 (ties to even), as FP32; scalar or array."""
+    f = np.vectorize(lambda v: lib().orc_bf16_round(float(v)), otypes=[np.float32])
+    return f(np.asarray(x, np.float32))
+
+
 def dequantize(codes, scales, s_g):
     codes, cp = _u8(codes)
     scales, sp = _u8(scales)
@@ -197,7 +205,7 @@ def root_coeffs(m, n, steps=5):
 
 
 def root_ns(G, steps=5, abc=None, clip_quantile=0.99, eps=1e-7, quantize=True,
-            exact_scales=False, trace_iter=None, rht=False, four_six=False, seed=0):
+            exact_scales=False, trace_iter=None, rht=False, four_six=False, seed=0, store_bf16=False):
     """The Root Newton-Schulz step on one m x n FP32 matrix.
 
     Returns out (m x n FP32), or (out, trace dict) when trace_iter is given; the
@@ -218,6 +226,7 @@ def root_ns(G, steps=5, abc=None, clip_quantile=0.99, eps=1e-7, quantize=True,
     p.rht = 1 if rht else 0
     p.four_six = 1 if four_six else 0
     p.seed = int(seed)
+    p.store_bf16 = 1 if store_bf16 else 0
     out = np.empty((m, n), np.float32)
     if trace_iter is None:
         rc = lib().orc_root_ns(gp, m, n, int(steps), C.byref(p), out.ctypes.data_as(_f32p), None)

@@ -125,6 +125,18 @@ float amax_of(const float* x, int64_t n) {
   return m;
 }
 
+// FP32 -> nearest BF16 (ties to even), returned as FP32
+float bf16_round(float x) {
+  uint32_t u;
+  std::memcpy(&u, &x, 4);
+  if ((u & 0x7F800000u) == 0x7F800000u) return x;  // inf / nan unchanged
+  u += 0x7FFFu + ((u >> 16) & 1u);
+  u &= 0xFFFF0000u;
+  float y;
+  std::memcpy(&y, &u, 4);
+  return y;
+}
+
 // y = x diag(r) H_16 / 4 for one block: signs (bit i of mask set: -x_i), natural-order fast
 // Walsh-Hadamard butterfly in FP32, then the exact factor 1/4.
 void hadamard16(const float* x, uint16_t mask, float* y) {
@@ -301,6 +313,8 @@ struct orc_params {
   int32_t rht;          // 1: random Hadamard transform of every 16-block before quantisation
   int32_t four_six;     // 1: adaptive 4/6 block scaling
   uint64_t seed;        // signs of the Hadamard matrices
+  int32_t store_bf16;   // 1: X_k (k >= 1) and A_k are kept in BF16 between the stages (round to nearest even);
+                        //    quantisation and maxima still see the FP32 values, the result is FP32
 };
 
 // Optional record of one iteration's intermediates (all row-major in the work
@@ -346,6 +360,7 @@ void orc_quantize_opts(const float* x, int64_t rows, int64_t cols, float s_g, ui
   quantize_1x16(x, rows, cols, s_g, codes, scales, rht, mask, four_six);
 }
 void orc_hadamard16(const float* x, uint16_t mask, float* y) { hadamard16(x, mask, y); }
+float orc_bf16_round(float x) { return bf16_round(x); }
 uint16_t orc_rht_mask(uint64_t seed, uint64_t idx) { return rht_mask(seed, idx); }
 
 void orc_dequantize(const uint8_t* codes, const uint8_t* scales, float s_g,
@@ -434,6 +449,10 @@ int orc_root_ns(const float* G, int64_t m, int64_t n, int steps, const orc_param
   std::vector<uint8_t> qBc((size_t)s * s / 2 + 1), qBs((size_t)s * s / 16 + 1);
 
   float amax_X = amax_of(X.data(), (int64_t)N);
+  const int bf16 = prm->store_bf16;
+  // Xq: the FP32 values the operand copies are quantised from; X: what is kept between the
+  // iterations and enters a X (the same unless BF16 storage is on)
+  std::vector<float> Xq(X);
   const int rht = prm->rht, f46 = prm->four_six;
   const float widen = rht ? 4.0f : 1.0f;  // |x H^r| <= 4 amax(x)
   float sg_X = scale_exact(widen * amax_X);  // initial operand: exact rule
@@ -457,12 +476,12 @@ int orc_root_ns(const float* G, int64_t m, int64_t n, int steps, const orc_param
       for (size_t i = 0; i < N; ++i) X[i] = ca * X[i] + P[i];
     } else {
       // qX = Q_1x16(X), qX^{16x1} = Q_16x1(X) = Q_1x16(X^T), one global scale
-      transpose(X.data(), s, l, Xt.data());
+      transpose(Xq.data(), s, l, Xt.data());
       // one Hadamard matrix for X_k (both operand copies and B_k, which meets qX^{16x1}),
       // another for A_k
       const uint16_t mask_X = rht ? rht_mask(prm->seed, 2 * (uint64_t)k) : 0;
       const uint16_t mask_A = rht ? rht_mask(prm->seed, 2 * (uint64_t)k + 1) : 0;
-      quantize_1x16(X.data(), s, l, sg_X, qXc.data(), qXs.data(), rht, mask_X, f46);
+      quantize_1x16(Xq.data(), s, l, sg_X, qXc.data(), qXs.data(), rht, mask_X, f46);
       quantize_1x16(Xt.data(), l, s, sg_X, qXtc.data(), qXts.data(), rht, mask_X, f46);
       // A = qX qX^T
       {
@@ -478,9 +497,10 @@ int orc_root_ns(const float* G, int64_t m, int64_t n, int steps, const orc_param
         std::vector<double> d = decode_f64(qAc.data(), qAs.data(), sg_A, s, s);
         gemm_nt(d.data(), d.data(), s, s, s, S.data(), 1);
       }
-      // B = b A + c (qA qA^{16x1}), each product and the sum rounded to FP32
+      // B = b A + c (qA qA^{16x1}), each product and the sum rounded to FP32; A as it is stored
       for (size_t i = 0; i < (size_t)s * s; ++i) {
-        float t1 = cb * A[i];
+        const float a_st = bf16 ? bf16_round(A[i]) : A[i];
+        float t1 = cb * a_st;
         float t2 = cc * S[i];
         B[i] = t1 + t2;
       }
@@ -511,18 +531,21 @@ int orc_root_ns(const float* G, int64_t m, int64_t n, int steps, const orc_param
         if (tr->sg_B) *tr->sg_B = sg_B;
       }
       float amax_prev = amax_X;
+      const bool last_it = (k == steps - 1);
       for (size_t i = 0; i < N; ++i) {
         float t1 = ca * X[i];
-        X[i] = t1 + P[i];
+        Xq[i] = t1 + P[i];
+        X[i] = (bf16 && !last_it) ? bf16_round(Xq[i]) : Xq[i];
       }
-      amax_X = amax_of(X.data(), (int64_t)N);
+      amax_X = amax_of(Xq.data(), (int64_t)N);
       float bound_X = 4.0f * std::fabs(ca) * amax_prev;
       sg_X = prm->exact_scales ? scale_exact(widen * amax_X) : scale_predicted(widen * bound_X);
     }
-    if (rec && tr->X_out) std::memcpy(tr->X_out, X.data(), N * sizeof(float));
+    if (rec && tr->X_out) std::memcpy(tr->X_out, prm->quantize ? Xq.data() : X.data(), N * sizeof(float));
   }
 
-  if (tall) transpose(X.data(), s, l, out); else std::memcpy(out, X.data(), N * sizeof(float));
+  const std::vector<float>& R = prm->quantize ? Xq : X;  // the last iteration's FP32 result
+  if (tall) transpose(R.data(), s, l, out); else std::memcpy(out, R.data(), N * sizeof(float));
   return 0;
 }
 

@@ -399,3 +399,35 @@ def test_paper_faithful_ns_is_at_least_as_close_to_exact_ns(gen, shape):
     # a different seed changes the signs, not the quality
     pf2 = oracle.root_ns(g, steps=5, rht=True, four_six=True, seed=12).astype(np.float64)
     assert not np.array_equal(pf, pf2) and abs(err(pf2) - err(pf)) < 0.03
+
+
+# ---- BF16 storage of X_k and A_k between the stages ------------------------------------------
+def test_bf16_round_matches_ml_dtypes():
+    import ml_dtypes
+    rng = np.random.default_rng(5)
+    x = np.concatenate([rng.standard_normal(4000).astype(np.float32) * 10.0 ** rng.integers(-20, 20, 4000),
+                        np.array([0.0, -0.0, 1.0, 1.00390625, 1.01171875, 3.3895314e38, 1e-40, -1e-40], np.float32)])
+    # 1.00390625 = 1 + 2^-8 is a tie (rounds to even: 1.0), 1.01171875 = 1 + 3 * 2^-8 a tie that rounds up
+    want = x.astype(ml_dtypes.bfloat16).astype(np.float32)
+    got = oracle.bf16_round(x)
+    np.testing.assert_array_equal(got.view(np.uint32), want.view(np.uint32))
+    assert oracle.bf16_round(np.float32(1.00390625)) == 1.0 and oracle.bf16_round(np.float32(1.01171875)) == np.float32(1.015625)
+
+
+def test_bf16_storage_is_a_small_perturbation_and_leaves_the_first_iteration_alone():
+    g = workloads.gradient_like(256, 384, seed=2)
+    base1, tr0 = oracle.root_ns(g, steps=1, trace_iter=0)
+    bf1, tr1 = oracle.root_ns(g, steps=1, trace_iter=0, store_bf16=True)
+    # one iteration: A is stored in BF16 (changes B), the result itself is FP32
+    np.testing.assert_array_equal(tr0["A"], tr1["A"])                       # the trace holds the FP32 A
+    np.testing.assert_array_equal(tr0["qA_codes"], tr1["qA_codes"])         # quantised from the FP32 values
+    assert not np.array_equal(tr0["B"], tr1["B"])
+    abc = oracle.root_coeffs(256, 384)
+    a_st = oracle.bf16_round(tr1["A"])
+    want_B = (np.float32(abc[1]) * a_st).astype(np.float32) + (np.float32(abc[2]) * tr1["S"]).astype(np.float32)
+    np.testing.assert_array_equal(tr1["B"], want_B.astype(np.float32))
+    e = oracle.root_ns(g, steps=5, quantize=False).astype(np.float64)
+    err = lambda q: np.linalg.norm(q.astype(np.float64) - e) / np.linalg.norm(e)
+    b5, f5 = oracle.root_ns(g, steps=5), oracle.root_ns(g, steps=5, store_bf16=True)
+    assert abs(err(f5) - err(b5)) < 0.01 and not np.array_equal(b5, f5)
+    assert f5.dtype == np.float32 and np.any(oracle.bf16_round(f5) != f5)      # the result is not rounded to BF16
