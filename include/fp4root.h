@@ -71,6 +71,14 @@ typedef enum {
  * upper half of its flags word: FP4_FLAG_RHT | FP4_QUANT_SIGNS(mask). */
 #define FP4_FLAG_RHT 2u
 #define FP4_FLAG_FOUR_SIX 4u
+/* BF16 storage of the high-precision copies between the stages (the paper does not state their
+ * precision; FP32 is the default): A_k and X_k (k >= 1) are kept in BF16, round to nearest
+ * even, which halves the FP32 traffic of the fused epilogues.  The NVFP4 operand copies and the
+ * running maxima are still derived from the FP32 values in the epilogue, X_0 stays FP32 and
+ * the result is FP32.  When every dimension of the work shape is a multiple of 256 the copies
+ * really are 2-byte tensors; otherwise they stay FP32 tensors that hold BF16-rounded values
+ * (same results, no traffic saved). */
+#define FP4_FLAG_STORE_BF16 8u
 #define FP4_QUANT_SIGNS(mask) ((uint32_t)(mask) << 16)
 
 /* Parameters of the step.  Pass NULL for the defaults noted on each field. */
@@ -209,6 +217,8 @@ typedef struct {
   int32_t idx_sg_X0;                /* scalars[idx + k] = tensor scale of qX_k      */
   int32_t idx_sg_A0, idx_sg_B0;     /* likewise for qA_k, qB_k                      */
   size_t total;
+  size_t Xh;          /* FP4_FLAG_STORE_BF16 with 2-byte storage: BF16 s x l, X_k (k >= 1); the A
+                         region then holds A as BF16 s x s.  0 otherwise.                  */
 } fp4_ws_layout;
 fp4_status fp4_root_ns_workspace_layout(int64_t m, int64_t n, int steps, uint32_t flags,
                                         fp4_ws_layout* layout);

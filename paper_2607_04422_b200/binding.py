@@ -18,6 +18,7 @@ _lib = None
 FP4_FLAG_KEEP_OPERANDS = 1
 FP4_FLAG_RHT = 2
 FP4_FLAG_FOUR_SIX = 4
+FP4_FLAG_STORE_BF16 = 8
 STATUS_NAMES = {0: "FP4_OK", 1: "FP4_ERR_INVALID_ARG", 2: "FP4_ERR_SHAPE", 3: "FP4_ERR_ALIGNMENT",
                 4: "FP4_ERR_WORKSPACE", 5: "FP4_ERR_ARCH", 6: "FP4_ERR_CUDA", 7: "FP4_ERR_DEVICE_TIMEOUT",
                 8: "FP4_ERR_UNIMPLEMENTED", 9: "FP4_ERR_STATIC_LIMIT"}
@@ -65,7 +66,7 @@ class WsLayout(C.Structure):
                 ("idx_tau", C.c_int32), ("idx_nu", C.c_int32), ("idx_inv", C.c_int32),
                 ("idx_amax_X0", C.c_int32), ("idx_amax_A0", C.c_int32),
                 ("idx_sg_X0", C.c_int32), ("idx_sg_A0", C.c_int32), ("idx_sg_B0", C.c_int32),
-                ("total", C.c_size_t)]
+                ("total", C.c_size_t), ("Xh", C.c_size_t)]
 
 
 def library_path() -> str:

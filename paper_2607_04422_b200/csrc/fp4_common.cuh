@@ -260,6 +260,18 @@ __device__ __forceinline__ uint32_t quantize_block16_opts(float (&v)[16], const 
 }
 
 // ----------------------------------------------------------------------------------
+// BF16 storage of the high-precision copies (round to nearest even)
+// ----------------------------------------------------------------------------------
+// two FP32 -> one word of two BF16 (lo in bits 15:0)
+__device__ __forceinline__ uint32_t cvt_bf16x2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
+
+// ----------------------------------------------------------------------------------
 // status word
 // ----------------------------------------------------------------------------------
 __device__ __forceinline__ void report_timeout(uint32_t* status) {

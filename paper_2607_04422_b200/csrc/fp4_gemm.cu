@@ -239,7 +239,7 @@ k_gemm(const __grid_constant__ GemmProblem single, const GemmProblem* __restrict
           chunk_slot(seq, c, b, use);
           if (!wait_bar(&bars->v_ready[b], use & 1, abort_flag)) { ok = false; break; }
           // a chunk that starts outside the stored matrix (zero padding of the work shape) is dropped
-          if (STORE_F32 && tj * BN + c * CHUNK < pr->out_cols && ti * BM < pr->out_rows) {
+          if (STORE_F32 && args.out_h == 0 && tj * BN + c * CHUNK < pr->out_cols && ti * BM < pr->out_rows) {
             tma_store_2d(&pr->tmOut, tj * BN + c * CHUNK, ti * BM, smem + OFF_RING + b * CHUNK_BYTES);
             bulk_commit();
             bulk_wait_read<1>();  // every store but the newest has read its slot
@@ -353,7 +353,19 @@ k_gemm(const __grid_constant__ GemmProblem single, const GemmProblem* __restrict
           __syncwarp();
           if (lane == 0) mbar_arrive(&bars->acc_empty[ab]);  // this warp is done with the accumulator
         }
-        if (STORE_F32 || mirror) {
+        if (STORE_F32 && MODE != kPlain && args.out_h == 2) {
+          // BF16 storage kept in an FP32 tensor: this thread stores the rounded values of its row itself
+          const int64_t gcol0 = (int64_t)tj * BN + c * CHUNK;
+          if (grow < pr->out_rows && gcol0 < pr->out_cols) {
+            float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(pr->out_direct) + grow * pr->out_direct_ld + gcol0);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const uint32_t w0 = cvt_bf16x2(v[4 * j], v[4 * j + 1]), w1 = cvt_bf16x2(v[4 * j + 2], v[4 * j + 3]);
+              dst[j] = make_float4(bf16_lo(w0), bf16_hi(w0), bf16_lo(w1), bf16_hi(w1));
+            }
+          }
+        }
+        if ((STORE_F32 && args.out_h == 0) || mirror) {
 #pragma unroll
           for (int j = 0; j < 4; ++j)
             *reinterpret_cast<float4*>(slot_row + ((j ^ sw) << 4)) =

@@ -174,7 +174,8 @@ __device__ __forceinline__ void tc_commit_pair(uint64_t* bar) {
       : "memory");
 }
 
-template <int MODE, bool PF>
+// BH: instantiation with BF16 storage of the FP32 tiles (args.aux_h / args.out_h may be set)
+template <int MODE, bool PF, bool BH>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
 k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __restrict__ table, const GemmLaunch args) {
   extern __shared__ uint8_t smem_raw[];
@@ -310,8 +311,16 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
             // a 128 x 128 block below the diagonal: nothing to combine, the slot is passed on empty
             mbar_arrive(&bars->aux_full[b]);
           } else {
-            mbar_expect_tx(&bars->aux_full[b], CHUNK_BYTES);
-            tma_load_2d(smem + OFF_RING + b * CHUNK_BYTES, &pr->tmAux, tjs[h] * PN + c * CHUNK, bi * BM, &bars->aux_full[b]);
+            if (BH && args.aux_h) {
+              // the tile is kept in BF16: four boxes of 32 rows x 32 bytes, each at the start of the 2 KB
+              // of the slot that the warp of those rows later stages its FP32 block in (no warp's
+              // staging can then overwrite rows another warp has not read yet)
+              mbar_expect_tx(&bars->aux_full[b], CHUNK_BYTES / 2);
+              tma_load_2d(smem + OFF_RING + b * CHUNK_BYTES, &pr->tmH, tjs[h] * PN + c * CHUNK, bi * BM, &bars->aux_full[b]);
+            } else {
+              mbar_expect_tx(&bars->aux_full[b], CHUNK_BYTES);
+              tma_load_2d(smem + OFF_RING + b * CHUNK_BYTES, &pr->tmAux, tjs[h] * PN + c * CHUNK, bi * BM, &bars->aux_full[b]);
+            }
           }
           ++n[h];
           ++done;
@@ -365,7 +374,12 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
           // a chunk that starts outside the stored matrix (zero padding of the work shape) is dropped
           const bool inside = tjs[h] * PN + c * CHUNK < pr->out_cols && bi * BM < pr->out_rows;
           if (STORE_F32 && !below && inside) {
-            tma_store_2d(&pr->tmOut, tjs[h] * PN + c * CHUNK, bi * BM, smem + OFF_RING + b * CHUNK_BYTES);
+            if (BH && args.out_h == 1) {
+              // the result was staged in BF16, 32 rows x 32 bytes at the start of each warp's part of the slot
+              tma_store_2d(&pr->tmH, tjs[h] * PN + c * CHUNK, bi * BM, smem + OFF_RING + b * CHUNK_BYTES);
+            } else {
+              tma_store_2d(&pr->tmOut, tjs[h] * PN + c * CHUNK, bi * BM, smem + OFF_RING + b * CHUNK_BYTES);
+            }
             bulk_commit();
             bulk_wait_read<2>();  // every store but the two newest has read its slot
             if (q0 >= 0) mbar_arrive(&bars->slot_free[q0]);
@@ -463,7 +477,8 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
       const int bj = tj * 2 + (team * TEAM_CHUNKS * CHUNK) / 128;      // 128-column block of this team's chunks
       const bool below = args.symmetric && bj < bi;                    // redundant block of a diagonal tile
       const bool mirror = do_q && !below && (MODE == kG3 || (args.symmetric && bi != bj));
-      const bool stage = !below && (STORE_F32 || mirror);
+      const bool hout = BH && STORE_F32 && MODE != kPlain && args.out_h == 1 && !below;  // result stored as BF16
+      const bool stage = !below && ((STORE_F32 && !hout) || mirror);
       const int par = (int)(seq & 1);
       ok = __all_sync(0xffffffffu, wait_bar(&bars->acc_full[par], (seq >> 1) & 1, abort_flag));
       if (!ok) break;
@@ -495,7 +510,21 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
         else ok = __all_sync(0xffffffffu, wait_bar(&bars->slot_free[b], (use & 1) ^ 1, abort_flag));
         if (!ok) break;
         tc_wait_ld16(acc);
-        if (HAS_AUX && !below) {
+        if (BH && HAS_AUX && !below && args.aux_h) {
+          // the FP32 tile is kept in BF16: this lane's row is 32 bytes at the start of its warp's part of the slot
+          const uint8_t* hrow = slot + row * 32;
+          const uint4 h0 = *reinterpret_cast<const uint4*>(hrow);
+          const uint4 h1 = *reinterpret_cast<const uint4*>(hrow + 16);
+          const uint32_t hw[8] = {h0.x, h0.y, h0.z, h0.w, h1.x, h1.y, h1.z, h1.w};
+          bar_sync(1 + team, 128);  // the four warps have their rows before any of them stages FP32 values over them
+#pragma unroll
+          for (int q = 0; q < 16; ++q) {
+            const float e = (q & 1) ? bf16_hi(hw[q >> 1]) : bf16_lo(hw[q >> 1]);
+            const float prod = __fmul_rn(__uint_as_float(acc[q]), scale);
+            if (MODE == kG2) v[q] = __fadd_rn(__fmul_rn(cb, e), __fmul_rn(cc, prod));
+            else v[q] = __fadd_rn(__fmul_rn(ca, e), prod);
+          }
+        } else if (HAS_AUX && !below) {
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
             const float4 x = *reinterpret_cast<const float4*>(slot_row + ((j ^ sw) << 4));
@@ -515,6 +544,11 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
         } else {
 #pragma unroll
           for (int k = 0; k < 16; ++k) v[k] = __fmul_rn(__uint_as_float(acc[k]), scale);
+        }
+        uint32_t hout_w[8];  // the row rounded to BF16 (before a quantiser option may transform v in place)
+        if (hout) {
+#pragma unroll
+          for (int q = 0; q < 8; ++q) hout_w[q] = cvt_bf16x2(v[2 * q], v[2 * q + 1]);
         }
         if (owns_overlap && i == OV_CHUNKS - 1) {
           // the columns shared with the other buffer are in registers: the next tile may use them
@@ -537,7 +571,7 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
           fence_proxy_async_smem();
         }
         __syncwarp();
-        if (lane == 0) mbar_arrive(&bars->v_ready[b]);  // the store issuer may send the chunk
+        if (!hout && lane == 0) mbar_arrive(&bars->v_ready[b]);  // the store issuer may send the chunk
         // Blocks of 16 down the rows of this warp's own 32 x 16 block (the transposed operand
         // copy in G3, the mirrored triangle in G1/G2), read back from the staging slot: row
         // k of the block is at k * 64 bytes, its 16-byte column group XOR-swizzled with bits
@@ -550,6 +584,18 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
           for (int k = 0; k < 16; ++k)
             w[k] = *reinterpret_cast<const float*>(colp + k * 64 + (col_sw[(k >> 1) & 3]));
         }
+        if (hout) {
+          bar_sync(1 + team, 128);  // the four warps have read their FP32 blocks back
+          // BF16 storage: the FP32 block has been read back (or was never staged); the rounded result
+          // takes its place, 32 bytes per row at the start of this warp's part of the slot, and
+          // the store issuer sends the four warps' rows as four boxes
+          uint8_t* hrow = slot + row * 32;
+          *reinterpret_cast<uint4*>(hrow) = make_uint4(hout_w[0], hout_w[1], hout_w[2], hout_w[3]);
+          *reinterpret_cast<uint4*>(hrow + 16) = make_uint4(hout_w[4], hout_w[5], hout_w[6], hout_w[7]);
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) { mbar_arrive(&bars->v_ready[b]); mbar_arrive(&bars->slot_free[b]); }  // done with the slot
+        }
         if (!below && do_q) {
           uint32_t lo, hi;
           float bmax;
@@ -560,8 +606,10 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
           *reinterpret_cast<uint2*>(rq_row + c * (CHUNK / 2)) = make_uint2(lo, hi);
           sfw |= sb << (8 * (c & 3));
         }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&bars->slot_free[b]);  // this warp's part of the slot is in registers
+        if (!hout) {
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&bars->slot_free[b]);  // this warp's part of the slot is in registers
+        }
         if (mirror) {
           uint32_t lo, hi;
           float bmax;
@@ -600,7 +648,7 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
   if (threadIdx.x == 0 && bars->abort_flag) report_timeout(args.status);
 }
 
-template <int MODE, bool PF>
+template <int MODE, bool PF, bool BH>
 cudaError_t launch_pair_mode(const GemmProblem* single, const GemmProblem* table, const GemmLaunch& L, int sms,
                              cudaStream_t st) {
   const int tpp = L.symmetric ? L.tiles_n * (L.tiles_n + 1) / 2 : L.tiles_m * L.tiles_n;
@@ -609,7 +657,7 @@ cudaError_t launch_pair_mode(const GemmProblem* single, const GemmProblem* table
   if (pairs > num_tiles) pairs = num_tiles;
   count_launches(1);
   static const GemmProblem kNone = {};
-  k_gemm_pair<MODE, PF><<<2 * pairs, NTHREADS, SMEM_BYTES, st>>>(single ? *single : kNone, table, L);
+  k_gemm_pair<MODE, PF, BH><<<2 * pairs, NTHREADS, SMEM_BYTES, st>>>(single ? *single : kNone, table, L);
   return cudaGetLastError();
 }
 
@@ -617,13 +665,19 @@ cudaError_t launch_pair_mode(const GemmProblem* single, const GemmProblem* table
 
 cudaError_t gemm_pair_set_attributes() {
   cudaError_t e;
-  if ((e = cudaFuncSetAttribute(k_gemm_pair<kPlain, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
-  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
-  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
-  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
-  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
-  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG3, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
-  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG3, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kPlain, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG1, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG1, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG1, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG1, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG2, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG2, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG2, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG2, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG3, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG3, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG3, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG3, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
   return cudaSuccess;
 }
 
@@ -636,12 +690,19 @@ cudaError_t launch_gemm_pair(GemmMode mode, const GemmProblem* single, const Gem
   L.tiles_m = launch.tiles_m / 2;
   L.tiles_n = launch.tiles_n / 2;
   const bool pf = launch.q.rht || launch.q.four_six;
+  const bool bh = launch.aux_h != 0 || launch.out_h != 0;
+#define FP4_PAIR_CASE(M)                                                                                    \
+  return pf ? (bh ? launch_pair_mode<M, true, true>(single, table, L, sms, st)                               \
+                  : launch_pair_mode<M, true, false>(single, table, L, sms, st))                             \
+            : (bh ? launch_pair_mode<M, false, true>(single, table, L, sms, st)                              \
+                  : launch_pair_mode<M, false, false>(single, table, L, sms, st))
   switch (mode) {
-    case kPlain: return launch_pair_mode<kPlain, false>(single, table, L, sms, st);
-    case kG1: return pf ? launch_pair_mode<kG1, true>(single, table, L, sms, st) : launch_pair_mode<kG1, false>(single, table, L, sms, st);
-    case kG2: return pf ? launch_pair_mode<kG2, true>(single, table, L, sms, st) : launch_pair_mode<kG2, false>(single, table, L, sms, st);
-    default: return pf ? launch_pair_mode<kG3, true>(single, table, L, sms, st) : launch_pair_mode<kG3, false>(single, table, L, sms, st);
+    case kPlain: return launch_pair_mode<kPlain, false, false>(single, table, L, sms, st);
+    case kG1: FP4_PAIR_CASE(kG1);
+    case kG2: FP4_PAIR_CASE(kG2);
+    default: FP4_PAIR_CASE(kG3);
   }
+#undef FP4_PAIR_CASE
 }
 
 }  // namespace fp4

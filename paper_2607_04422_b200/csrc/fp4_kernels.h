@@ -41,6 +41,8 @@ struct NsPlan {
   int64_t s, l;      // work shape: s0, l0 rounded up to multiples of 128 (zero padding)
   int tall;
   int clip;
+  int bf16_mode;     // 0: FP32 storage of X_k / A_k; 1: BF16 tensors; 2: FP32 tensors holding BF16-rounded values
+  size_t off_Xh;     // bf16_mode 1: BF16 X in the workspace
   int64_t clip_rank;
   float eps;
   int sms;
@@ -64,6 +66,8 @@ struct alignas(64) GemmProblem {
   CUtensorMap tmA, tmB;      // NVFP4 codes of the row and the column operand
   CUtensorMap tmAux, tmOut;  // FP32 tile combined in the epilogue / FP32 result
   CUtensorMap tmSfa, tmSfb;  // scale atoms of the two operands as 2-D maps (CTA-pair kernel)
+  CUtensorMap tmH;           // BF16 storage: the 2-byte tensor this stage reads its tile from and / or stores its
+                             // result to (A for G1 / G2, X for G3); box 16 columns x 32 rows, no swizzle
   const uint8_t* sfa;        // scale atoms of the row operand
   const uint8_t* sfb;        // scale atoms of the column operand
   float* scalars;            // workspace scalars of this matrix (device)
@@ -73,6 +77,8 @@ struct alignas(64) GemmProblem {
   float sg_a, sg_b;          // kPlain: tensor scales from the host
   int aux_raw;               // kG3: tmAux maps the raw input G; X0 = clamp(G, tau) * inv is formed on the fly
   int out_rows, out_cols;    // extent of the matrix behind tmOut (chunks that start outside it are not stored)
+  void* out_direct;          // out_h == 2: the FP32 tensor the epilogue warps store the rounded result to
+  int64_t out_direct_ld;     //   (row-major, leading dimension in elements)
 };
 
 // What all problems of a launch share.
@@ -87,6 +93,9 @@ struct GemmLaunch {
   float l_cols;        // (float) l, for the bound on amax(A)
   QuantOpts q;         // how this stage's output is quantised (q.widen = 1 in the base mode)
   int clip;            // kG3 on a problem with aux_raw: whether tau applies
+  int aux_h;           // the combined tile is read from tmH (BF16)
+  int out_h;           // 0: FP32 result by TMA store; 1: rounded to BF16, staged and stored through tmH (CTA-pair
+                       // kernel); 2: rounded to BF16, stored as FP32 by the epilogue warps (single-CTA kernel)
   NsScalarIdx ix;
   uint32_t* status;
 };

@@ -106,6 +106,18 @@ bool make_f32_map(const DeviceInfo* d, CUtensorMap* tm, const void* base, int64_
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// 2-D map over a row-major BF16 matrix: box = 16 columns x 32 rows (32-byte rows), no swizzle: one box per
+// epilogue warp of a team, so that a warp's rows sit inside its own part of the chunk slot.
+bool make_bf16_map(const DeviceInfo* d, CUtensorMap* tm, const void* base, int64_t rows, int64_t cols) {
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  cuuint32_t box[2] = {16, 128};
+  cuuint32_t estr[2] = {1, 1};
+  return d->encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 constexpr int kDefaultMaxGroup = 16;
 
 // 2-D map over the scale atoms of a rows x K operand: one map row per 128-row block, 64-bit
@@ -123,9 +135,9 @@ bool make_sf_map(const DeviceInfo* d, CUtensorMap* tm, const void* base, int64_t
 
 // The CTA-pair kernel takes every product whose dimensions are all multiples of 256.
 cudaError_t launch_gemm_auto(GemmMode mode, const GemmProblem* single, const GemmProblem* table,
-                             const GemmLaunch& L, int sms, cudaStream_t st) {
+                             const GemmLaunch& L, int sms, cudaStream_t st, bool force_single = false) {
 #ifndef FP4_DISABLE_PAIR
-  if (!(L.tiles_m & 1) && !(L.tiles_n & 1) && L.K % 256 == 0 && sms >= 2)
+  if (!force_single && !(L.tiles_m & 1) && !(L.tiles_n & 1) && L.K % 256 == 0 && sms >= 2)
     return launch_gemm_pair(mode, single, table, L, sms, st);
 #endif
   return launch_gemm(mode, single, table, L, sms, st);
@@ -193,6 +205,12 @@ fp4_status make_plan(int64_t m, int64_t n, int steps, const fp4_ns_params* p, in
   // maximum; since the dimensions are multiples of 16 no block mixes data and padding.
   pl->s = pad128(pl->s0);
   pl->l = pad128(pl->l0);
+  // BF16 storage: 2-byte tensors when all three stages run in the CTA-pair kernel, else FP32
+  // tensors that hold rounded values (and all stages in the single-CTA kernel)
+  if (p->flags & FP4_FLAG_STORE_BF16) pl->bf16_mode = (pl->s % 256 == 0 && pl->l % 256 == 0) ? 1 : 2;
+#ifdef FP4_DISABLE_PAIR
+  if (pl->bf16_mode == 1) pl->bf16_mode = 2;
+#endif
   const int64_t s = pl->s, l = pl->l;
   pl->clip = p->clip_quantile > 0.0f && p->clip_quantile < 1.0f;
   pl->clip_rank = pl->clip ? quantile_rank(m * n, p->clip_quantile) : 0;
@@ -227,6 +245,8 @@ fp4_status make_plan(int64_t m, int64_t n, int steps, const fp4_ns_params* p, in
   L.qA_scales = off; off += align_up((size_t)s * s / 16, 1024);
   L.qB_codes = off; off += align_up((size_t)s * s / 2, 1024);
   L.qB_scales = off; off += align_up((size_t)s * s / 16, 1024);
+  L.Xh = 0;
+  if (pl->bf16_mode == 1) { pl->off_Xh = off; L.Xh = off; off += align_up((size_t)s * l * 2, 1024); }
   L.idx_tau = ix.tau; L.idx_nu = ix.nu; L.idx_inv = ix.inv;
   L.idx_amax_X0 = ix.amax_X0; L.idx_amax_A0 = ix.amax_A0;
   L.idx_sg_X0 = ix.sg_X0; L.idx_sg_A0 = ix.sg_A0; L.idx_sg_B0 = ix.sg_B0;
@@ -280,17 +300,24 @@ fp4_status prepare_matrix(const DeviceInfo* d, const float* G, float* out, int64
   base.scalars = reinterpret_cast<float*>(ws + L.scalars);
   base.ca = abc[0]; base.cb = abc[1]; base.cc = abc[2];
   base.out_rows = (int)s; base.out_cols = (int)s;
+  const int bmode = c->pl.bf16_mode;
+  CUtensorMap tm_Ah, tm_Xh;
+  uint8_t* Xh = bmode == 1 ? ws + c->pl.off_Xh : nullptr;
+  if (bmode == 1 && (!make_bf16_map(d, &tm_Ah, ws + L.A, s, s) || !make_bf16_map(d, &tm_Xh, Xh, s, l))) return FP4_ERR_CUDA;
   // G1: A = qX qX^T (upper-triangle tiles), qA in both triangles
   c->g1 = base;
   c->g1.tmA = c->g1.tmB = tm_qX; c->g1.tmAux = c->g1.tmOut = tm_A;
   c->g1.tmSfa = c->g1.tmSfb = sf_qX;
   c->g1.sfa = c->g1.sfb = ws + L.qX_scales;
   c->g1.rq_codes = c->g1.cq_codes = ws + L.qA_codes; c->g1.rq_sf = c->g1.cq_sf = ws + L.qA_scales;
+  if (bmode == 1) c->g1.tmH = tm_Ah;                                           // A as a BF16 tensor
+  if (bmode == 2) { c->g1.out_direct = ws + L.A; c->g1.out_direct_ld = s; }   // A as rounded FP32
   // G2: B = bA + c qA qA^T, qB in both triangles
   c->g2 = base;
   c->g2.tmA = c->g2.tmB = tm_qA; c->g2.tmAux = c->g2.tmOut = tm_A;
   c->g2.tmSfa = c->g2.tmSfb = sf_qA;
   c->g2.sfa = c->g2.sfb = ws + L.qA_scales;
+  if (bmode == 1) c->g2.tmH = tm_Ah;
   c->g2.rq_codes = c->g2.cq_codes = ws + L.qB_codes; c->g2.rq_sf = c->g2.cq_sf = ws + L.qB_scales;
   // G3: X+ = aX + qB qXt^T in place on X; new operand copies
   for (int cur = 0; cur < 2; ++cur) {
@@ -298,6 +325,8 @@ fp4_status prepare_matrix(const DeviceInfo* d, const float* G, float* out, int64
     g = base;
     g.tmA = tm_qB; g.tmB = tm_qXt[cur]; g.tmAux = g.tmOut = tm_X;
     g.out_rows = (int)xr; g.out_cols = (int)xc;
+    if (bmode == 1) g.tmH = tm_Xh;
+    if (bmode == 2) { g.out_direct = c->X; g.out_direct_ld = xc; }
     g.tmSfa = sf_qB; g.tmSfb = sf_qXt[cur];
     g.sfa = ws + L.qB_scales; g.sfb = ws + L.qXt_scales[cur];
     g.rq_codes = ws + L.qX_codes; g.rq_sf = ws + L.qX_scales;
@@ -369,6 +398,8 @@ fp4_status run_group(const DeviceInfo* d, MatrixCtx* mats, int count, int steps,
     base.l_cols = (float)l;
     base.status = status;
     base.clip = pl0.clip;
+    const int bmode = pl0.bf16_mode;
+    const bool fs = bmode == 2;  // rounded-FP32 storage is implemented by the single-CTA kernel only
     for (int k = 0; k < steps; ++k) {
       const int cur = k & 1;
       const bool last = (k == steps - 1);
@@ -376,17 +407,19 @@ fp4_status run_group(const DeviceInfo* d, MatrixCtx* mats, int count, int steps,
       L1.iter = k; L1.K = (int)l; L1.tiles_m = L1.tiles_n = (int)(s / 128); L1.symmetric = 1;
       L1.rq_K = L1.cq_K = (int)s; L1.write_q = 1;
       L1.q = quant_opts(p, 2 * (uint64_t)k + 1);  // qA_k
+      L1.out_h = bmode;
       {
         ProfScope ps(FP4_PROF_G1, st);
-        if (launch_gemm_auto(kG1, count == 1 ? &mats[0].g1 : nullptr, tabs[0], L1, d->sms, st) != cudaSuccess)
+        if (launch_gemm_auto(kG1, count == 1 ? &mats[0].g1 : nullptr, tabs[0], L1, d->sms, st, fs) != cudaSuccess)
           return FP4_ERR_CUDA;
       }
       GemmLaunch L2 = L1;
       L2.K = (int)s;
       L2.q = quant_opts(p, 2 * (uint64_t)k);      // qB_k meets qX_k^{16x1}
+      L2.out_h = 0; L2.aux_h = bmode == 1;
       {
         ProfScope ps(FP4_PROF_G2, st);
-        if (launch_gemm_auto(kG2, count == 1 ? &mats[0].g2 : nullptr, tabs[1], L2, d->sms, st) != cudaSuccess)
+        if (launch_gemm_auto(kG2, count == 1 ? &mats[0].g2 : nullptr, tabs[1], L2, d->sms, st, fs) != cudaSuccess)
           return FP4_ERR_CUDA;
       }
       GemmLaunch L3 = base;
@@ -394,10 +427,12 @@ fp4_status run_group(const DeviceInfo* d, MatrixCtx* mats, int count, int steps,
       L3.rq_K = (int)l; L3.cq_K = (int)s;
       L3.write_q = (!last || keep) ? 1 : 0;
       L3.q = quant_opts(p, 2 * (uint64_t)k + 2);  // both copies of X_{k+1}
+      L3.aux_h = (bmode == 1 && k > 0) ? 1 : 0;   // X_0 is FP32 (or the raw input)
+      L3.out_h = last ? 0 : bmode;                 // the result itself is FP32
       {
         ProfScope ps(FP4_PROF_G3, st);
         const GemmProblem* one = k == 0 ? &mats[0].g3_first : &mats[0].g3[cur];
-        if (launch_gemm_auto(kG3, count == 1 ? one : nullptr, k == 0 ? tabs[4] : tabs[2 + cur], L3, d->sms, st) != cudaSuccess)
+        if (launch_gemm_auto(kG3, count == 1 ? one : nullptr, k == 0 ? tabs[4] : tabs[2 + cur], L3, d->sms, st, fs) != cudaSuccess)
           return FP4_ERR_CUDA;
       }
     }

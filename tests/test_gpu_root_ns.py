@@ -6,7 +6,7 @@ import torch
 import oracle
 import paper_2607_04422_b200 as fp4
 from paper_2607_04422_b200 import workloads
-from paper_2607_04422_b200.binding import (FP4_FLAG_FOUR_SIX, FP4_FLAG_KEEP_OPERANDS, FP4_FLAG_RHT,
+from paper_2607_04422_b200.binding import (FP4_FLAG_FOUR_SIX, FP4_FLAG_KEEP_OPERANDS, FP4_FLAG_RHT, FP4_FLAG_STORE_BF16,
                                            fp4_root_ns_workspace_layout)
 from helpers import nibbles, sf_from_atoms
 
@@ -272,6 +272,59 @@ def test_cuda_graph_replay_matches_direct_call():
         torch.cuda.synchronize()
         assert fp4.fp4_last_device_status(ws) == 0
         assert torch.equal(out, direct)
+
+
+@pytest.mark.parametrize("shape", [(256, 512), (512, 256), (512, 512), (384, 384), (640, 384), (144, 272), (1024, 2048)])
+def test_bf16_storage_of_the_high_precision_copies(shape):
+    """FP4_FLAG_STORE_BF16: A_k and X_k (k >= 1) are kept in BF16 between the stages; shapes whose
+    work dimensions are multiples of 256 use 2-byte tensors (CTA-pair kernel), the others FP32
+    tensors with rounded values (single-CTA kernel).  Both against the oracle's emulation."""
+    m, n = shape
+    G = workloads.gradient_like(m, n, seed=13)
+    for steps in (1, 2, 5):
+        got, _ = run_gpu(G, steps=steps, flags=FP4_FLAG_STORE_BF16)
+        want = oracle.root_ns(G, steps=steps, store_bf16=True)
+        assert rel(got, want) <= TOL_OUT, (steps, rel(got, want))
+        assert abs(orth_err(got) - orth_err(want)) <= TOL_ORTH
+    plain, _ = run_gpu(G, steps=5)
+    assert not np.array_equal(plain, got)                       # the option does change the numbers
+    assert np.any(oracle.bf16_round(got) != got)                # the result itself is not rounded
+    # iteration 0: qB is quantised from B = b bf16(A) + c S
+    flags = FP4_FLAG_STORE_BF16 | FP4_FLAG_KEEP_OPERANDS
+    _, ws = run_gpu(G, steps=1, flags=flags)
+    _, tr = oracle.root_ns(G, steps=1, trace_iter=0, store_bf16=True)
+    lay, sc, f32, q, s, l = ws_view(ws, m, n, 1, flags)
+    if s % 128 == 0 and l % 128 == 0:
+        codes, sf = q(lay.qB_codes, lay.qB_scales, s, s)
+        sf_diff = sf != tr["qB_scales"]
+        assert sf_diff.mean() < 2e-3
+        g, w = nibbles(codes), nibbles(tr["qB_codes"])
+        assert ((g != w) & ~np.repeat(sf_diff, 16, axis=1)).mean() < 2e-3
+        raw = ws.cpu().numpy()
+        if lay.Xh:   # 2-byte storage: the A region holds BF16 A (upper-triangle 128-blocks)
+            A16 = raw[lay.A:lay.A + s * s * 2].view(np.uint16).reshape(s, s)
+            A = (A16.astype(np.uint32) << 16).view(np.float32)
+        else:
+            A = f32(lay.A, s, s)
+        mask = np.kron(np.triu(np.ones((s // 128, s // 128))), np.ones((128, 128))).astype(bool)
+        want_A = oracle.bf16_round(tr["A"])
+        # the stored A is the BF16 rounding of an FP32 value that differs from the oracle's in the last bits
+        assert np.abs(A[mask] - want_A[mask]).max() <= 2.0 ** -7 * np.abs(tr["A"]).max()
+        assert np.array_equal(oracle.bf16_round(A[mask]), A[mask])
+
+
+def test_bf16_storage_batched_matches_single_calls():
+    specs = [(256, 512, 1), (512, 256, 2), (384, 384, 3), (256, 512, 4)]
+    mats = [workloads.gradient_like(m, n, seed=sd) for m, n, sd in specs]
+    Gs = [torch.from_numpy(g).cuda() for g in mats]
+    outs = [torch.empty_like(g) for g in Gs]
+    shapes = [tuple(g.shape) for g in Gs]
+    ws = torch.empty(fp4.fp4_root_ns_batched_workspace_bytes(shapes, 4, FP4_FLAG_STORE_BF16), dtype=torch.uint8, device="cuda")
+    fp4.fp4_root_ns_batched(Gs, outs, 4, fp4.NsParams.make(flags=FP4_FLAG_STORE_BF16), ws)
+    assert fp4.fp4_last_device_status(ws) == 0
+    for g, o in zip(mats, outs):
+        single, _ = run_gpu(g, steps=4, flags=FP4_FLAG_STORE_BF16)
+        assert np.array_equal(o.cpu().numpy(), single)
 
 
 def test_bounded_wait_gives_up_and_reports():
