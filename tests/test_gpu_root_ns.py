@@ -12,7 +12,7 @@ from helpers import nibbles, sf_from_atoms
 
 pytestmark = pytest.mark.gpu
 
-# Tolerances.  BASELINE: relative Frobenius error of the NS output <= 2e-3 per iteration
+# Tolerances.  Required of the path: relative Frobenius error of the NS output <= 2e-3 per iteration
 # count, orthogonality error within 1e-2 of the oracle's.  Stage outputs that have
 # bit-identical inputs on both sides differ only by FP32-vs-FP64 accumulation.
 TOL_OUT = 2e-3
