@@ -20,6 +20,8 @@ _lib = None
 
 _u8p = C.POINTER(C.c_uint8)
 _f32p = C.POINTER(C.c_float)
+_u16p = C.POINTER(C.c_uint16)
+_u32p = C.POINTER(C.c_uint32)
 
 
 class OrcParams(C.Structure):
@@ -71,6 +73,14 @@ def lib():
         L.orc_hadamard16.argtypes = [_f32p, C.c_uint16, _f32p]; L.orc_hadamard16.restype = None
         L.orc_rht_mask.argtypes = [C.c_uint64, C.c_uint64]; L.orc_rht_mask.restype = C.c_uint16
         L.orc_bf16_round.argtypes = [C.c_float]; L.orc_bf16_round.restype = C.c_float
+        L.orc_momentum_encode.argtypes = [_f32p, C.c_int64, C.c_int64, C.c_int, C.c_uint64, _u8p, _u16p]
+        L.orc_momentum_encode.restype = None
+        L.orc_momentum_decode.argtypes = [_u8p, _u16p, C.c_int64, C.c_int64, _f32p]
+        L.orc_momentum_decode.restype = None
+        L.orc_momentum_update.argtypes = [_f32p, C.c_int64, C.c_int64, C.c_float, C.c_float, C.c_int, C.c_uint64,
+                                          _u8p, _u16p, _f32p, _u32p]
+        L.orc_momentum_update.restype = None
+        L.orc_splitmix64_at.argtypes = [C.c_uint64, C.c_uint64]; L.orc_splitmix64_at.restype = C.c_uint64
         L.orc_dequantize.argtypes = [_u8p, _u8p, C.c_float, C.c_int64, C.c_int64, _f32p]
         L.orc_dequantize.restype = None
         L.orc_gemm_nt_q.argtypes = [_u8p, _u8p, C.c_float, _u8p, _u8p, C.c_float,
@@ -162,6 +172,46 @@ def bf16_round(x):
     """FP32 -> nearest BF16 (ties to even), as FP32; scalar or array."""
     f = np.vectorize(lambda v: lib().orc_bf16_round(float(v)), otypes=[np.float32])
     return f(np.asarray(x, np.float32))
+
+
+def splitmix64_at(seed, idx):
+    """Output number idx (from 0) of the splitmix64 generator seeded with `seed`."""
+    return int(lib().orc_splitmix64_at(int(seed), int(idx)))
+
+
+def momentum_encode(M, sr=False, seed=0):
+    """First-moment state of an FP32 matrix: (codes u8 rows x cols/2, scales u16 rows x cols/16)."""
+    M, mp = _f32(M)
+    rows, cols = M.shape
+    codes = np.empty((rows, cols // 2), np.uint8)
+    scales = np.empty((rows, cols // 16), np.uint16)
+    lib().orc_momentum_encode(mp, rows, cols, int(bool(sr)), int(seed), codes.ctypes.data_as(_u8p),
+                              scales.ctypes.data_as(_u16p))
+    return codes, scales
+
+
+def momentum_decode(codes, scales):
+    codes, cp = _u8(codes)
+    scales = np.ascontiguousarray(scales, np.uint16)
+    rows, cols = codes.shape[0], codes.shape[1] * 2
+    out = np.empty((rows, cols), np.float32)
+    lib().orc_momentum_decode(cp, scales.ctypes.data_as(_u16p), rows, cols, out.ctypes.data_as(_f32p))
+    return out
+
+
+def momentum_update(G, codes, scales, mu, g_scale=1.0, sr=False, seed=0, want_hist=True):
+    """One step on a stored state; returns (M_t, new codes, new scales, histogram or None)."""
+    G, gp = _f32(G)
+    rows, cols = G.shape
+    codes = np.array(codes, np.uint8, copy=True)
+    scales = np.array(scales, np.uint16, copy=True)
+    M = np.empty((rows, cols), np.float32)
+    hist = np.zeros(8192, np.uint32) if want_hist else None
+    lib().orc_momentum_update(gp, rows, cols, float(np.float32(mu)), float(np.float32(g_scale)), int(bool(sr)),
+                              int(seed), codes.ctypes.data_as(_u8p), scales.ctypes.data_as(_u16p),
+                              M.ctypes.data_as(_f32p),
+                              hist.ctypes.data_as(_u32p) if want_hist else None)
+    return M, codes, scales, hist
 
 
 def dequantize(codes, scales, s_g):

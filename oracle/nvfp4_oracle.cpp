@@ -52,6 +52,23 @@
 //     Parity unpinned against the cited sources (Four Over Six, TE's RHT); the invariances
 //     (the transform cancels, the error never grows) are pinned.
 //
+//   * first-moment momentum state (Section 3.3: "Hadamard mixing ... before SR and adaptive
+//     4/6 quantization", 5 bits per element in the appendix's memory accounting; Section 3.4:
+//     Root's momentum uses the same storage recipe).  The paper gives no formulas; readings:
+//       - each 1x16 block along a row is multiplied by the fixed H_16 / 4 (no signs), its own
+//         inverse; the block scale is a BF16 number (4 + 16/16 = 5 bits per element) and there
+//         is no tensor scale; the two 4/6 candidates are BF16(amax/6) and BF16(amax/4), chosen
+//         by the round-to-nearest error exactly as above;
+//       - stochastic rounding (optional) re-encodes the block with the chosen scale: a value
+//         between two neighbouring grid points goes up with probability equal to its
+//         fractional position, decided by a 24-bit uniform number from a splitmix64 counter
+//         generator indexed by element pair;
+//       - the update is M_t = fl(fl(mu M_{t-1}) + fl(g_scale G_t)) in FP32 on the decoded
+//         state, and the state is re-encoded from M_t.
+//     Parity unpinned against the authors' code; the transform's involution, the grid
+//     round trip, unbiasedness of the stochastic rounding and the generator's published
+//     test vector are pinned.
+//
 // Build:  g++ -O2 -std=c++17 -ffp-contract=off -fopenmp -shared -fPIC
 
 #include <algorithm>
@@ -298,6 +315,93 @@ int64_t quantile_rank(int64_t n, float q) {
   if (k < 1) k = 1;
   if (k > n) k = n;
   return k;
+}
+
+// ---- first-moment momentum state (Section 3.3 first-moment recipe, Section 3.4) ----
+
+uint64_t splitmix64_at(uint64_t seed, uint64_t idx) {
+  uint64_t z = seed + 0x9E3779B97F4A7C15ull * (idx + 1);
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  return z ^ (z >> 31);
+}
+
+uint16_t bf16_bits(float x) {  // x is already a BF16 value
+  uint32_t u;
+  std::memcpy(&u, &x, 4);
+  return (uint16_t)(u >> 16);
+}
+float bf16_from_bits(uint16_t b) {
+  uint32_t u = (uint32_t)b << 16;
+  float y;
+  std::memcpy(&y, &u, 4);
+  return y;
+}
+
+// Round-to-nearest codes of one transformed block for the block scale d; returns the sum of
+// squared FP32 errors.
+float mom_encode_rtn(const float* h, float d, uint8_t* nib) {
+  float err = 0.0f;
+  if (d == 0.0f) {
+    for (int i = 0; i < 16; ++i) { nib[i] = 0; float q = h[i] * h[i]; err = err + q; }
+    return err;
+  }
+  float rcp = 1.0f / d;
+  for (int i = 0; i < 16; ++i) {
+    float y = h[i] * rcp;
+    nib[i] = (uint8_t)((std::signbit(y) ? 8 : 0) | e2m1_index(std::fabs(y)));
+    float diff = h[i] - e2m1_decode(nib[i]) * d;
+    float q = diff * diff;
+    err = err + q;
+  }
+  return err;
+}
+
+// Stochastic rounding of |y| onto the grid with the uniform number u in [0,1)
+int e2m1_index_sr(float mag, float u) {
+  if (!(mag == mag) || mag >= 6.0f) return 7;
+  int i = 0;
+  while (i < 6 && mag >= kE2M1Grid[i + 1]) ++i;  // grid[i] <= mag < grid[i+1]
+  float p = (mag - kE2M1Grid[i]) / (kE2M1Grid[i + 1] - kE2M1Grid[i]);
+  return (u < p) ? i + 1 : i;
+}
+
+// Encode one 1x16 block of a momentum matrix; `first` is the index of its first element
+// in the matrix (it numbers the random stream).
+void mom_encode_block(const float* v, int sr, uint64_t seed, uint64_t first,
+                      uint8_t* nib, uint16_t* scale_bits) {
+  float h[16];
+  hadamard16(v, 0, h);
+  float amax = amax_of(h, 16);
+  float d6 = bf16_round(amax / 6.0f);
+  float d4 = bf16_round(amax / 4.0f);
+  uint8_t n4[16];
+  float err6 = mom_encode_rtn(h, d6, nib);
+  float err4 = mom_encode_rtn(h, d4, n4);
+  float d = d6;
+  if (err4 < err6) { d = d4; for (int i = 0; i < 16; ++i) nib[i] = n4[i]; }
+  if (sr && d != 0.0f) {
+    float rcp = 1.0f / d;
+    for (int i = 0; i < 16; i += 2) {
+      uint64_t z = splitmix64_at(seed, (first + (uint64_t)i) >> 1);
+      float u0 = (float)(uint32_t)(z >> 40) * 5.9604644775390625e-08f;               // 2^-24
+      float u1 = (float)(uint32_t)((z >> 8) & 0xFFFFFFu) * 5.9604644775390625e-08f;
+      float y0 = h[i] * rcp, y1 = h[i + 1] * rcp;
+      nib[i] = (uint8_t)((std::signbit(y0) ? 8 : 0) | e2m1_index_sr(std::fabs(y0), u0));
+      nib[i + 1] = (uint8_t)((std::signbit(y1) ? 8 : 0) | e2m1_index_sr(std::fabs(y1), u1));
+    }
+  }
+  *scale_bits = bf16_bits(d);
+}
+
+void mom_decode_block(const uint8_t* packed, uint16_t scale_bits, float* v) {
+  float d = bf16_from_bits(scale_bits);
+  float h[16];
+  for (int i = 0; i < 8; ++i) {
+    h[2 * i] = e2m1_decode(packed[i] & 0xF) * d;
+    h[2 * i + 1] = e2m1_decode(packed[i] >> 4) * d;
+  }
+  hadamard16(h, 0, v);
 }
 
 }  // namespace
@@ -548,5 +652,61 @@ int orc_root_ns(const float* G, int64_t m, int64_t n, int steps, const orc_param
   if (tall) transpose(R.data(), s, l, out); else std::memcpy(out, R.data(), N * sizeof(float));
   return 0;
 }
+
+// First-moment momentum state: see the file header.  codes rows x cols/2 bytes (element 2j of
+// the transformed block in the low nibble), scales rows x cols/16 BF16 bit patterns.
+void orc_momentum_encode(const float* M, int64_t rows, int64_t cols, int sr, uint64_t seed,
+                         uint8_t* codes, uint16_t* scales) {
+  const int64_t nb = cols / 16;
+#pragma omp parallel for schedule(static)
+  for (int64_t r = 0; r < rows; ++r)
+    for (int64_t kb = 0; kb < nb; ++kb) {
+      uint8_t nib[16];
+      mom_encode_block(M + r * cols + kb * 16, sr, seed, (uint64_t)(r * cols + kb * 16), nib,
+                       &scales[r * nb + kb]);
+      uint8_t* out = codes + r * (cols / 2) + kb * 8;
+      for (int i = 0; i < 8; ++i) out[i] = (uint8_t)(nib[2 * i] | (nib[2 * i + 1] << 4));
+    }
+}
+
+void orc_momentum_decode(const uint8_t* codes, const uint16_t* scales, int64_t rows, int64_t cols,
+                         float* M) {
+  const int64_t nb = cols / 16;
+#pragma omp parallel for schedule(static)
+  for (int64_t r = 0; r < rows; ++r)
+    for (int64_t kb = 0; kb < nb; ++kb)
+      mom_decode_block(codes + r * (cols / 2) + kb * 8, scales[r * nb + kb], M + r * cols + kb * 16);
+}
+
+// One momentum step on the stored state, in place: M_t = mu M_{t-1} + g_scale G_t, written to
+// M_out (may be null), re-encoded into codes/scales; hist (may be null, 8192 counters, added
+// to) counts the top 13 magnitude bits of every M_t element.
+void orc_momentum_update(const float* G, int64_t rows, int64_t cols, float mu, float g_scale,
+                         int sr, uint64_t seed, uint8_t* codes, uint16_t* scales, float* M_out,
+                         uint32_t* hist) {
+  const int64_t nb = cols / 16;
+  for (int64_t r = 0; r < rows; ++r)
+    for (int64_t kb = 0; kb < nb; ++kb) {
+      float prev[16], m[16];
+      mom_decode_block(codes + r * (cols / 2) + kb * 8, scales[r * nb + kb], prev);
+      for (int i = 0; i < 16; ++i) {
+        float t1 = mu * prev[i];
+        float t2 = g_scale * G[r * cols + kb * 16 + i];
+        m[i] = t1 + t2;
+        if (M_out) M_out[r * cols + kb * 16 + i] = m[i];
+        if (hist) {
+          uint32_t u;
+          std::memcpy(&u, &m[i], 4);
+          hist[(u & 0x7FFFFFFFu) >> 18] += 1;
+        }
+      }
+      uint8_t nib[16];
+      mom_encode_block(m, sr, seed, (uint64_t)(r * cols + kb * 16), nib, &scales[r * nb + kb]);
+      uint8_t* out = codes + r * (cols / 2) + kb * 8;
+      for (int i = 0; i < 8; ++i) out[i] = (uint8_t)(nib[2 * i] | (nib[2 * i + 1] << 4));
+    }
+}
+
+uint64_t orc_splitmix64_at(uint64_t seed, uint64_t idx) { return splitmix64_at(seed, idx); }
 
 }  // extern "C"

@@ -1,0 +1,187 @@
+"""Pins of the oracle's first-moment momentum state (Section 3.3 first-moment recipe, used by
+Root's momentum per Section 3.4) against things that are not the oracle: the generator's
+published test vector, scipy's Hadamard matrix, hand-worked blocks, numpy FP64 arithmetic and
+statistics of the stochastic rounding."""
+import numpy as np
+import pytest
+from scipy.linalg import hadamard
+
+import oracle
+
+GRID = np.array([0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0])
+H4 = hadamard(16).astype(np.float64) / 4.0   # Sylvester order; (H/4)(H/4) = I
+
+
+def nibbles(codes):
+    c = np.asarray(codes, np.uint8)
+    out = np.empty(c.shape[:-1] + (c.shape[-1] * 2,), np.uint8)
+    out[..., 0::2] = c & 0xF
+    out[..., 1::2] = c >> 4
+    return out
+
+
+def nib_values(nib):
+    return np.where(nib & 8, -1.0, 1.0) * GRID[nib & 7]
+
+
+def bf16_value(bits):
+    return (np.asarray(bits, np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def numpy_decode(codes, scales):
+    """Independent FP64 decode: grid value * BF16 scale, then the inverse transform."""
+    v = nib_values(nibbles(codes))
+    rows, cols = v.shape
+    h = v.reshape(rows, cols // 16, 16) * bf16_value(scales)[..., None]
+    return (h @ H4).reshape(rows, cols)
+
+
+def test_splitmix64_published_vector():
+    # the first outputs of the reference splitmix64 generator for the seed 1234567
+    want = [6457827717110365317, 3203168211198807973, 9817491932198370423,
+            4593380528125082431, 16408922859458223821]
+    assert [oracle.splitmix64_at(1234567, i) for i in range(5)] == want
+
+
+def test_state_is_five_bits_per_element():
+    M = np.ones((32, 128), np.float32)
+    c, s = oracle.momentum_encode(M)
+    assert (c.nbytes + s.nbytes) * 8 == 5 * M.size
+
+
+def test_grid_block_round_trip_exact():
+    # transformed values on the grid with maximum 6 * 2^k: the scale is 2^k, every code is the
+    # value itself, and decode returns the input bit for bit
+    rng = np.random.default_rng(5)
+    rows, nb = 8, 6
+    idx = rng.integers(0, 8, (rows, nb, 16))
+    sgn = rng.integers(0, 2, (rows, nb, 16))
+    idx[..., 3] = 7                                   # the block maximum
+    k = rng.integers(-20, 10, (rows, nb))
+    h = np.where(sgn == 1, -1.0, 1.0) * GRID[idx] * (2.0 ** k)[..., None]
+    x = (h @ H4).reshape(rows, nb * 16)               # exact: small dyadic numbers
+    assert np.array_equal(x, x.astype(np.float32))
+    c, s = oracle.momentum_encode(x.astype(np.float32))
+    nib = nibbles(c).reshape(rows, nb, 16)
+    assert np.array_equal(nib & 7, idx)
+    nz = idx != 0
+    assert np.array_equal((nib >> 3)[nz], sgn[nz])
+    assert np.array_equal(bf16_value(s), 2.0 ** k)
+    assert np.array_equal(oracle.momentum_decode(c, s), x.astype(np.float32))
+
+
+def test_four_is_chosen_when_it_is_exact():
+    # transformed block (4, 3, 2, 1, 0 ...): with the maximum on 4 the scale is 1 and the block
+    # is exact; with the maximum on 6 the scale BF16(2/3) leaves an error
+    h = np.zeros(16)
+    h[:4] = [4, -3, 2, 1]
+    x = (h @ H4).astype(np.float32)[None, :]
+    c, s = oracle.momentum_encode(x)
+    assert int(s[0, 0]) == 0x3F80
+    assert np.array_equal(nib_values(nibbles(c))[0], h)
+    assert np.array_equal(oracle.momentum_decode(c, s), x)
+
+
+def test_six_is_kept_on_ties_and_zero_block():
+    x = np.zeros((1, 32), np.float32)
+    h = np.zeros(16)
+    h[:3] = [6, 3, -1.5]                              # exact with 6 (scale 1) and with 4 (scale 1.5)
+    x[0, 16:] = (h @ H4).astype(np.float32)
+    c, s = oracle.momentum_encode(x)
+    assert int(s[0, 0]) == 0 and not c[0, :8].any()
+    assert int(s[0, 1]) == 0x3F80                     # the tie keeps the maximum on 6
+    assert np.array_equal(nib_values(nibbles(c))[0, 16:], h)
+
+
+@pytest.mark.parametrize("seed", [0, 1])
+def test_decode_matches_fp64_matrix_form(seed):
+    rng = np.random.default_rng(seed)
+    M = (rng.standard_normal((48, 320)) * np.exp(rng.standard_normal((48, 320)))).astype(np.float32)
+    c, s = oracle.momentum_encode(M)
+    D = oracle.momentum_decode(c, s)
+    want = numpy_decode(c, s)
+    assert np.allclose(D, want, rtol=0, atol=1e-6 * np.abs(want).max())
+    # a 4-bit code with the better of two scales: relative error well under 12 %
+    rel = np.linalg.norm(D - M) / np.linalg.norm(M)
+    assert 0.02 < rel < 0.12
+    # every scale is the BF16 of amax/6 or amax/4 of the transformed block
+    h = M.astype(np.float64).reshape(48, 20, 16) @ H4
+    amax = np.abs(h).max(-1)
+    d = bf16_value(s)
+    ok6 = np.abs(d - amax / 6) <= amax / 6 * 2.0 ** -8
+    ok4 = np.abs(d - amax / 4) <= amax / 4 * 2.0 ** -8
+    assert np.all(ok6 | ok4)
+    assert ok4.sum() > 0 and ok6.sum() > 0
+
+
+def test_update_arithmetic_and_histogram():
+    rng = np.random.default_rng(3)
+    rows, cols = 40, 192
+    M0 = rng.standard_normal((rows, cols)).astype(np.float32)
+    G = (rng.standard_normal((rows, cols)) * 0.3).astype(np.float32)
+    c0, s0 = oracle.momentum_encode(M0)
+    M1, c1, s1, hist = oracle.momentum_update(G, c0, s0, mu=0.95, g_scale=0.5)
+    want = 0.95 * numpy_decode(c0, s0) + 0.5 * G.astype(np.float64)
+    assert np.allclose(M1, want, rtol=0, atol=3e-7 * np.abs(want).max())
+    # the new state is the encoding of M1
+    c1b, s1b = oracle.momentum_encode(M1)
+    assert np.array_equal(c1, c1b) and np.array_equal(s1, s1b)
+    # the histogram counts the top 13 magnitude bits of M1
+    bins = (M1.view(np.uint32) & 0x7FFFFFFF) >> 18
+    assert np.array_equal(hist, np.bincount(bins.ravel(), minlength=8192).astype(np.uint32))
+
+
+def test_update_special_cases():
+    rng = np.random.default_rng(4)
+    G = rng.standard_normal((16, 64)).astype(np.float32)
+    zc = np.zeros((16, 32), np.uint8)
+    zs = np.zeros((16, 4), np.uint16)
+    # an all-zero state is zero momentum: M_1 = G
+    M1, c1, s1, _ = oracle.momentum_update(G, zc, zs, mu=0.9)
+    assert np.array_equal(M1, G)
+    # mu = 0 forgets the state
+    c0, s0 = oracle.momentum_encode(rng.standard_normal((16, 64)).astype(np.float32))
+    M2, c2, s2, _ = oracle.momentum_update(G, c0, s0, mu=0.0)
+    assert np.array_equal(M2, G) and np.array_equal(c2, c1) and np.array_equal(s2, s1)
+    # zero gradient with mu = 1 reads the state back
+    M3, _, _, _ = oracle.momentum_update(np.zeros_like(G), c0, s0, mu=1.0)
+    assert np.array_equal(M3, oracle.momentum_decode(c0, s0))
+
+
+def test_stochastic_rounding_probability_and_neighbours():
+    # transformed block (6, 1.125, -2.25, 0 ...): scale 1; 1.125 lies a quarter of the way from 1
+    # to 1.5, and 2.25 a quarter of the way from 2 to 3
+    h = np.zeros(16)
+    h[0], h[1], h[2] = 6.0, 1.125, -2.25
+    x = (h @ H4).astype(np.float32)[None, :]
+    ups = 0
+    ups2 = 0
+    n = 4000
+    for seed in range(n):
+        c, s = oracle.momentum_encode(x, sr=True, seed=seed)
+        assert int(s[0, 0]) == 0x3F80
+        v = nib_values(nibbles(c))[0]
+        assert v[0] == 6.0 and not v[3:].any()
+        assert v[1] in (1.0, 1.5) and v[2] in (-2.0, -3.0)
+        ups += v[1] == 1.5
+        ups2 += v[2] == -3.0
+    assert abs(ups / n - 0.25) < 0.03      # 4 sigma = 0.027
+    assert abs(ups2 / n - 0.25) < 0.03
+
+
+def test_stochastic_rounding_is_unbiased():
+    rng = np.random.default_rng(8)
+    M = rng.standard_normal((32, 256)).astype(np.float32)
+    c, s = oracle.momentum_encode(M)
+    rtn = np.linalg.norm(oracle.momentum_decode(c, s) - M) / np.linalg.norm(M)
+    acc = np.zeros(M.shape)
+    n = 256
+    for seed in range(n):
+        c, s = oracle.momentum_encode(M, sr=True, seed=1000 + seed)
+        acc += oracle.momentum_decode(c, s)
+    mean_err = np.linalg.norm(acc / n - M) / np.linalg.norm(M)
+    assert mean_err < 0.2 * rtn            # a biased rounding would stay near the RTN error
+    # and different seeds give different codes
+    ca, _ = oracle.momentum_encode(M, sr=True, seed=1)
+    cb, _ = oracle.momentum_encode(M, sr=True, seed=2)
+    assert not np.array_equal(ca, cb)
