@@ -275,6 +275,25 @@ def run_ours(args):
     q_gbs = 8192 * 8192 * 8.5625 / (min(q_ms[1:]) / 1e3) / 1e9
     del qx, qc, qs
 
+    # ---- the momentum step on one 8192 x 8192 matrix (HBM-bound: G in, M out, 5-bit state in
+    # and out = 9.25 B per element), with the clip histogram and with stochastic rounding
+    mg = torch.randn((8192, 8192), device="cuda")
+    mm = torch.empty_like(mg)
+    mc = torch.zeros((8192, 4096), dtype=torch.uint8, device="cuda")
+    msc = torch.zeros((8192, 512), dtype=torch.int16, device="cuda")
+    mh = torch.zeros(8192, dtype=torch.int32, device="cuda")
+    mom = {}
+    for name, flags in (("rtn", 0), ("sr", fp4.FP4_MOM_FLAG_SR)):
+        t_ms = []
+        for it in range(5):
+            e0.record(stream)
+            fp4.fp4_momentum_update(mg, mc, msc, mm, mh, 0.95, 1.0, flags, it, stream)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            t_ms.append(e0.elapsed_time(e1))
+        mom[name] = 8192 * 8192 * 9.25 / (min(t_ms[1:]) / 1e3) / 1e9
+    del mg, mm, mc, msc
+
     # ---- reference row: the same iterations in BF16 on cuBLAS (torch.matmul), dense products.
     # Context for the NVFP4 path, not part of the product.  The clip and the normalisation are
     # done once outside the timed region (torch has no fast exact quantile for 25 M elements),
@@ -412,6 +431,9 @@ def run_ours(args):
                     "how": "pinned host buffers; per decoder block: upload, fp4_root_ns_batched, download on three streams"},
             "quantizer": {"workload": "fp4_quantize 8192x8192 FP32", "gbs": q_gbs, "peak_gbs": pk["hbm_gbs"],
                           "frac": q_gbs / pk["hbm_gbs"], "bytes_per_element": 8.5625},
+            "momentum": {"workload": "fp4_momentum_update 8192x8192 FP32 with M_t and clip histogram out",
+                         "gbs": mom["rtn"], "gbs_stochastic_rounding": mom["sr"], "peak_gbs": pk["hbm_gbs"],
+                         "frac": mom["rtn"] / pk["hbm_gbs"], "bytes_per_element": 9.25},
             "bf16_cublas_ns": {"value": len(shapes) / (bf16_ms / 1e3), "unit": UNIT, "ms_per_step": bf16_ms,
                                "tflops_dense": dense / (bf16_ms / 1e3) / 1e12,
                                "what": "the 5 Newton-Schulz iterations of the batch with torch.matmul in BF16 "

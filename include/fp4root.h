@@ -234,6 +234,57 @@ fp4_status fp4_gemm_nt(const uint8_t* a_codes, const uint8_t* a_scales, float a_
                        FP4_ERR_DEVICE_TIMEOUT if a bounded wait gives up */,
                        cudaStream_t stream);
 
+/* ---- first-moment momentum in a 5-bit NVFP4 state ---------------------------------------------
+ * Section 3.3 (first-moment recipe: Hadamard mixing, then stochastic rounding and adaptive 4/6
+ * quantisation; 5 bits per element in the appendix's memory accounting) and Section 3.4 (Root's
+ * momentum is stored with that recipe).  The step that precedes fp4_root_ns in the optimiser:
+ *     M_t = mu * M_{t-1} + g_scale * G_t,
+ * with M_{t-1} read from the state, M_t written in FP32 (the Newton-Schulz input) and the state
+ * replaced by the encoding of M_t, all in one pass over the matrix.
+ *
+ * State of a rows x cols matrix (row-major; rows > 0, cols a positive multiple of 16, else
+ * FP4_ERR_SHAPE), blocks of 1x16 along the rows:
+ *   codes   device, rows*cols/2 bytes: E2M1 codes of each block multiplied by H_16 / 4 (the
+ *           Sylvester Hadamard matrix, no signs; its own inverse), element 2j of the transformed
+ *           block in the low nibble of byte j
+ *   scales  device, rows*cols/16 uint16: the block scales as BF16 bit patterns; no tensor scale
+ * An all-zero state is zero momentum.  Encoding a block h: the two candidate scales are
+ * BF16(amax/6) and BF16(amax/4); each is tried with round-to-nearest-even codes of h/scale, the
+ * one with the smaller sum of squared FP32 errors (element order) is kept, a tie keeps 6.
+ * FP4_MOM_FLAG_SR then encodes the block again with the chosen scale by stochastic rounding:
+ * with lo <= |y| < hi the neighbouring grid values and f = floor(65536 (|y| - lo) / (hi - lo)),
+ * y becomes hi when f + r >= 65536 (probability f / 65536).  The 16 random bits r: elements
+ * 8q .. 8q+7 of the matrix (row-major index) share output q of splitmix64 (z = seed +
+ * 0x9E3779B97F4A7C15 (q+1), then the generator's output mix), its low 32 bits for the first
+ * four; of a 32-bit word, the low half is r of element 0, the same 16 bits in reverse order
+ * r of element 1, the high half r of element 2, reversed r of element 3.
+ * Arithmetic: m_prev = (code * scale) H_16 / 4 (natural-order butterfly, FP32), then
+ * M = fl(fl(mu m_prev) + fl(g_scale G)).
+ *
+ * G       device, in : rows x cols FP32, 16-byte aligned
+ * codes, scales  device, in/out: the state, updated in place; 16-byte aligned
+ * M_out   device, out: rows x cols FP32 or NULL; must not overlap G
+ * hist    device, in/out or NULL: 8192 uint32 counters; counter ((bits of |M|) >> 18) is
+ *         incremented for every element of M_t (the top 13 magnitude bits: the first pass of the
+ *         outlier clip's quantile selection); the caller zeroes it
+ * Errors: FP4_ERR_INVALID_ARG (null pointer, unknown flag), FP4_ERR_SHAPE, FP4_ERR_ALIGNMENT,
+ * FP4_ERR_ARCH, FP4_ERR_CUDA.
+ */
+#define FP4_MOM_FLAG_SR 1u
+typedef struct fp4_momentum_params {
+  float mu;        /* momentum coefficient                                   */
+  float g_scale;   /* factor on the gradient: 1 (heavy ball) or 1 - mu (EMA) */
+  uint32_t flags;  /* FP4_MOM_FLAG_*                                         */
+  uint32_t reserved;
+  uint64_t seed;   /* FP4_MOM_FLAG_SR: a different seed every step           */
+} fp4_momentum_params;
+fp4_status fp4_momentum_update(const float* G, int64_t rows, int64_t cols, uint8_t* codes, uint16_t* scales,
+                               float* M_out, uint32_t* hist, const fp4_momentum_params* params,
+                               cudaStream_t stream);
+/* M_out = the decoded state (device, rows x cols FP32, 16-byte aligned); the state is not changed. */
+fp4_status fp4_momentum_decode(const uint8_t* codes, const uint16_t* scales, int64_t rows, int64_t cols,
+                               float* M_out, cudaStream_t stream);
+
 /* ---- measurement support (the paper has no counterpart) -----------------------------------
  * While profiling is enabled, every group of launches of the step is bracketed by a pair of
  * CUDA events on the caller's stream; fp4_profile_collect waits for them, adds the elapsed
@@ -243,7 +294,8 @@ fp4_status fp4_gemm_nt(const uint8_t* a_codes, const uint8_t* a_scales, float a_
  * fp4_kernel_launches returns how many kernels this library has launched in this process.
  */
 enum { FP4_PROF_CLIP = 0, FP4_PROF_STATS = 1, FP4_PROF_PREP = 2, FP4_PROF_G1 = 3, FP4_PROF_G2 = 4,
-       FP4_PROF_G3 = 5, FP4_PROF_TRANSPOSE = 6, FP4_PROF_QUANTIZE = 7, FP4_PROF_CLASSES = 8 };
+       FP4_PROF_G3 = 5, FP4_PROF_TRANSPOSE = 6, FP4_PROF_QUANTIZE = 7, FP4_PROF_MOMENTUM = 8,
+       FP4_PROF_CLASSES = 9 };
 void fp4_profile_enable(int on);
 fp4_status fp4_profile_collect(float* ms, int* groups);
 uint64_t fp4_kernel_launches(void);

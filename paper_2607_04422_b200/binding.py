@@ -19,6 +19,7 @@ FP4_FLAG_KEEP_OPERANDS = 1
 FP4_FLAG_RHT = 2
 FP4_FLAG_FOUR_SIX = 4
 FP4_FLAG_STORE_BF16 = 8
+FP4_MOM_FLAG_SR = 1
 STATUS_NAMES = {0: "FP4_OK", 1: "FP4_ERR_INVALID_ARG", 2: "FP4_ERR_SHAPE", 3: "FP4_ERR_ALIGNMENT",
                 4: "FP4_ERR_WORKSPACE", 5: "FP4_ERR_ARCH", 6: "FP4_ERR_CUDA", 7: "FP4_ERR_DEVICE_TIMEOUT",
                 8: "FP4_ERR_UNIMPLEMENTED", 9: "FP4_ERR_STATIC_LIMIT"}
@@ -29,7 +30,7 @@ EXPORTS = ("fp4_status_string", "fp4_scale_bytes", "fp4_quantize", "fp4_root_coe
            "fp4_root_ns_batched", "fp4_last_device_status", "fp4_root_ns_workspace_layout", "fp4_gemm_nt",
            "fp4_profile_enable", "fp4_profile_collect", "fp4_kernel_launches", "fp4_root_ns_static",
            "fp4_selftest_bounded_wait")
-PROF_CLASSES = ("clip", "stats", "prep", "G1", "G2", "G3", "transpose", "quantize")
+PROF_CLASSES = ("clip", "stats", "prep", "G1", "G2", "G3", "transpose", "quantize", "momentum")
 
 
 class Fp4Error(RuntimeError):
@@ -54,6 +55,12 @@ class NsParams(C.Structure):
         p.max_group = int(max_group)
         p.seed = int(seed)
         return p
+
+
+class MomentumParams(C.Structure):
+    """fp4_momentum_params of include/fp4root.h."""
+    _fields_ = [("mu", C.c_float), ("g_scale", C.c_float), ("flags", C.c_uint32), ("reserved", C.c_uint32),
+                ("seed", C.c_uint64)]
 
 
 class WsLayout(C.Structure):
@@ -107,6 +114,9 @@ def load_library():
     L.fp4_profile_collect.argtypes = [C.POINTER(C.c_float), C.POINTER(C.c_int)]
     L.fp4_profile_collect.restype = C.c_int
     L.fp4_kernel_launches.argtypes = []; L.fp4_kernel_launches.restype = C.c_uint64
+    L.fp4_momentum_update.argtypes = [vp, i64, i64, vp, vp, vp, vp, C.POINTER(MomentumParams), vp]
+    L.fp4_momentum_update.restype = C.c_int
+    L.fp4_momentum_decode.argtypes = [vp, vp, i64, i64, vp, vp]; L.fp4_momentum_decode.restype = C.c_int
     L.fp4_selftest_bounded_wait.argtypes = [vp, u32, vp]; L.fp4_selftest_bounded_wait.restype = C.c_int
     _lib = L
     return L
@@ -141,6 +151,25 @@ def fp4_quantize(x: torch.Tensor, codes: torch.Tensor, scales: torch.Tensor, ten
     rows, cols = x.shape
     _check(load_library().fp4_quantize(x.data_ptr(), rows, cols, codes.data_ptr(), scales.data_ptr(),
                                        tensor_scale.data_ptr(), flags, _stream(stream)), "fp4_quantize")
+
+
+def fp4_momentum_update(G: torch.Tensor, codes: torch.Tensor, scales: torch.Tensor, M_out: torch.Tensor | None,
+                        hist: torch.Tensor | None, mu: float, g_scale: float = 1.0, flags: int = 0, seed: int = 0,
+                        stream=None) -> None:
+    """One momentum step on the 5-bit state (codes uint8 rows x cols/2, scales int16/uint16 rows x cols/16),
+    in place; M_out (FP32) and hist (8192 int32 counters, added to) are optional."""
+    rows, cols = G.shape
+    prm = MomentumParams(mu, g_scale, flags, 0, seed)
+    _check(load_library().fp4_momentum_update(G.data_ptr(), rows, cols, codes.data_ptr(), scales.data_ptr(),
+                                              M_out.data_ptr() if M_out is not None else None,
+                                              hist.data_ptr() if hist is not None else None, C.byref(prm),
+                                              _stream(stream)), "fp4_momentum_update")
+
+
+def fp4_momentum_decode(codes: torch.Tensor, scales: torch.Tensor, M_out: torch.Tensor, stream=None) -> None:
+    rows, cols = M_out.shape
+    _check(load_library().fp4_momentum_decode(codes.data_ptr(), scales.data_ptr(), rows, cols, M_out.data_ptr(),
+                                              _stream(stream)), "fp4_momentum_decode")
 
 
 def fp4_root_ns_workspace_bytes(m: int, n: int, steps: int = 5, flags: int = 0) -> int:

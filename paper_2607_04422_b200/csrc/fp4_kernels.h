@@ -103,6 +103,14 @@ struct GemmLaunch {
 // Measurement support: counts kernel launches and, when profiling is on, brackets a group of
 // launches with events.
 void count_launches(int n);
+
+// First-moment momentum state (fp4_momentum.cu): one step in place on codes/scales; M_out and
+// hist may be null.
+cudaError_t launch_momentum_update(const float* G, int64_t rows, int64_t cols, float mu, float g_scale, bool sr,
+                                   uint64_t seed, uint8_t* codes, uint16_t* scales, float* M_out, uint32_t* hist,
+                                   int sms, cudaStream_t st);
+cudaError_t launch_momentum_decode(const uint8_t* codes, const uint16_t* scales, int64_t rows, int64_t cols,
+                                   float* M_out, int sms, cudaStream_t st);
 struct ProfScope {
   int cls; cudaStream_t st; cudaEvent_t e0; bool on;
   ProfScope(int cls, cudaStream_t st);

@@ -510,6 +510,37 @@ fp4_status fp4_quantize(const float* x, int64_t rows, int64_t cols, uint8_t* cod
                                                                                                       : FP4_ERR_CUDA;
 }
 
+fp4_status fp4_momentum_update(const float* G, int64_t rows, int64_t cols, uint8_t* codes, uint16_t* scales,
+                               float* M_out, uint32_t* hist, const fp4_momentum_params* params,
+                               cudaStream_t stream) {
+  if (!G || !codes || !scales || !params) return FP4_ERR_INVALID_ARG;
+  if (params->flags & ~FP4_MOM_FLAG_SR) return FP4_ERR_INVALID_ARG;
+  if (rows <= 0 || cols <= 0 || (cols & 15)) return FP4_ERR_SHAPE;
+  if (!aligned(G, 16) || !aligned(codes, 16) || !aligned(scales, 16) || (M_out && !aligned(M_out, 16)) ||
+      (hist && !aligned(hist, 4)))
+    return FP4_ERR_ALIGNMENT;
+  const DeviceInfo* d;
+  fp4_status rc = check_common(&d);
+  if (rc != FP4_OK) return rc;
+  ProfScope ps(FP4_PROF_MOMENTUM, stream);
+  return launch_momentum_update(G, rows, cols, params->mu, params->g_scale, (params->flags & FP4_MOM_FLAG_SR) != 0,
+                                params->seed, codes, scales, M_out, hist, d->sms, stream) == cudaSuccess
+             ? FP4_OK
+             : FP4_ERR_CUDA;
+}
+
+fp4_status fp4_momentum_decode(const uint8_t* codes, const uint16_t* scales, int64_t rows, int64_t cols,
+                               float* M_out, cudaStream_t stream) {
+  if (!codes || !scales || !M_out) return FP4_ERR_INVALID_ARG;
+  if (rows <= 0 || cols <= 0 || (cols & 15)) return FP4_ERR_SHAPE;
+  if (!aligned(codes, 16) || !aligned(scales, 16) || !aligned(M_out, 16)) return FP4_ERR_ALIGNMENT;
+  const DeviceInfo* d;
+  fp4_status rc = check_common(&d);
+  if (rc != FP4_OK) return rc;
+  return launch_momentum_decode(codes, scales, rows, cols, M_out, d->sms, stream) == cudaSuccess ? FP4_OK
+                                                                                                 : FP4_ERR_CUDA;
+}
+
 fp4_status fp4_root_coeffs(int64_t m, int64_t n, int steps, float abc[3]) {
   if (m <= 0 || n <= 0 || steps < 0 || !abc) return FP4_ERR_INVALID_ARG;
   coeffs(m, n, abc);

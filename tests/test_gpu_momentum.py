@@ -1,0 +1,172 @@
+"""fp4_momentum_update / fp4_momentum_decode against the oracle: M_t, codes, scales and the
+histogram bit for bit, over several steps, with and without stochastic rounding."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2607_04422_b200 as fp4
+from paper_2607_04422_b200 import workloads
+from helpers import mismatch_report
+
+pytestmark = pytest.mark.gpu
+
+
+class GpuState:
+    def __init__(self, rows, cols):
+        self.codes = torch.zeros((rows, cols // 2), dtype=torch.uint8, device="cuda")
+        self.scales = torch.zeros((rows, cols // 16), dtype=torch.int16, device="cuda")
+
+    def load(self, codes, scales):
+        self.codes.copy_(torch.from_numpy(codes))
+        self.scales.copy_(torch.from_numpy(scales.view(np.int16)))
+
+    def numpy(self):
+        return self.codes.cpu().numpy(), self.scales.cpu().numpy().view(np.uint16)
+
+
+def _step(G_np, st, mu, g_scale=1.0, sr=False, seed=0, want_m=True, want_hist=True):
+    G = torch.from_numpy(G_np).cuda()
+    M = torch.empty_like(G) if want_m else None
+    hist = torch.zeros(8192, dtype=torch.int32, device="cuda") if want_hist else None
+    fp4.fp4_momentum_update(G, st.codes, st.scales, M, hist, mu, g_scale,
+                            flags=fp4.FP4_MOM_FLAG_SR if sr else 0, seed=seed)
+    torch.cuda.synchronize()
+    return (M.cpu().numpy() if want_m else None,
+            hist.cpu().numpy().view(np.uint32) if want_hist else None)
+
+
+def _gradient(rows, cols, seed, scale=1.0):
+    return (workloads.row_lognormal(rows, cols, seed=seed) * np.float32(scale)).astype(np.float32)
+
+
+@pytest.mark.parametrize("sr", [False, True])
+@pytest.mark.parametrize("shape", [(16, 16), (1, 4096), (48, 272), (300, 1040), (1024, 3072)])
+def test_three_steps_bit_exact(shape, sr):
+    rows, cols = shape
+    st = GpuState(rows, cols)
+    oc = np.zeros((rows, cols // 2), np.uint8)
+    os_ = np.zeros((rows, cols // 16), np.uint16)
+    for t in range(3):
+        G = _gradient(rows, cols, seed=10 * t + rows, scale=1.0 + t)
+        M, hist = _step(G, st, mu=0.95, g_scale=1.0, sr=sr, seed=77 + t)
+        oM, oc, os_, oh = oracle.momentum_update(G, oc, os_, 0.95, 1.0, sr=sr, seed=77 + t)
+        c, s = st.numpy()
+        assert np.array_equal(M.view(np.uint32), oM.view(np.uint32)), mismatch_report(M, oM)
+        assert np.array_equal(s, os_), mismatch_report(s, os_)
+        assert np.array_equal(c, oc), mismatch_report(c, oc)
+        assert np.array_equal(hist, oh)
+
+
+def test_ema_form_and_optional_outputs():
+    rows, cols = 64, 512
+    G = _gradient(rows, cols, seed=3)
+    st = GpuState(rows, cols)
+    c0, s0 = oracle.momentum_encode(_gradient(rows, cols, seed=4))
+    st.load(c0, s0)
+    M, hist = _step(G, st, mu=0.9, g_scale=0.1, want_m=False, want_hist=False)
+    assert M is None and hist is None
+    _, oc, os_, _ = oracle.momentum_update(G, c0, s0, 0.9, 0.1)
+    c, s = st.numpy()
+    assert np.array_equal(c, oc) and np.array_equal(s, os_)
+
+
+def test_ties_zero_blocks_and_extreme_magnitudes():
+    f = np.float32
+    H4 = oracle.hadamard16  # only to place chosen values in the transformed domain
+    rng = np.random.default_rng(1)
+    rows, cols = 32, 256
+    G = np.zeros((rows, cols), f)
+    mids = np.array([0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0, 6.0, 4.0, 3.0, 0.0, 0.5, 1.0, 1.5, 2.0], f)
+    for r in range(rows):
+        for b in range(cols // 16):
+            h = rng.choice(np.concatenate([mids, -mids]), 16).astype(f)
+            h[rng.integers(16)] = [6.0, 4.0, 6.0 * 1.00390625, 5.0][(r + b) % 4]
+            h = h * f(2.0) ** int(rng.integers(-30, 30))
+            G[r, b * 16:(b + 1) * 16] = H4(h)      # the transform is its own inverse
+    G[3, 32:48] = 0
+    G[4, 0:16] = f(1e-42)                          # denormals
+    G[5, 16:32] = f(1e37) * np.sign(rng.standard_normal(16)).astype(f)   # sums stay finite
+    G[6, 0:16] = 0
+    G[6, 5] = f(-1e-30)
+    for sr in (False, True):
+        st = GpuState(rows, cols)
+        M, hist = _step(G, st, mu=0.5, sr=sr, seed=9)
+        oM, oc, os_, oh = oracle.momentum_update(G, np.zeros((rows, cols // 2), np.uint8),
+                                                 np.zeros((rows, cols // 16), np.uint16), 0.5, sr=sr, seed=9)
+        c, s = st.numpy()
+        assert np.array_equal(M.view(np.uint32), oM.view(np.uint32))
+        assert np.array_equal(s, os_), mismatch_report(s, os_)
+        assert np.array_equal(c, oc), mismatch_report(c, oc)
+        assert np.array_equal(hist, oh)
+        # second step from that state: the decode of every such block
+        G2 = np.zeros_like(G)
+        M2, _ = _step(G2, st, mu=1.0, sr=sr, seed=10)
+        oM2, _, _, _ = oracle.momentum_update(G2, oc, os_, 1.0, sr=sr, seed=10)
+        assert np.array_equal(M2.view(np.uint32), oM2.view(np.uint32))
+
+
+def test_decode_entry_point():
+    rows, cols = 96, 784
+    c0, s0 = oracle.momentum_encode(_gradient(rows, cols, seed=12))
+    st = GpuState(rows, cols)
+    st.load(c0, s0)
+    M = torch.empty((rows, cols), dtype=torch.float32, device="cuda")
+    fp4.fp4_momentum_decode(st.codes, st.scales, M)
+    torch.cuda.synchronize()
+    assert np.array_equal(M.cpu().numpy().view(np.uint32), oracle.momentum_decode(c0, s0).view(np.uint32))
+    c, s = st.numpy()
+    assert np.array_equal(c, c0) and np.array_equal(s, s0)
+
+
+def test_full_size_sampled_rows_and_histogram():
+    # the benchmark's size: rows checked one by one against the oracle, the histogram against the
+    # kernel's own M_t
+    rows, cols = 8192, 8192
+    gen = torch.Generator(device="cuda").manual_seed(5)
+    G = torch.randn((rows, cols), generator=gen, device="cuda", dtype=torch.float32)
+    G *= torch.exp(0.5 * torch.randn((rows, 1), generator=gen, device="cuda"))
+    st = GpuState(rows, cols)
+    M = torch.empty_like(G)
+    hist = torch.zeros(8192, dtype=torch.int32, device="cuda")
+    for t in range(2):
+        prev_c, prev_s = st.codes.clone(), st.scales.clone()
+        hist.zero_()
+        fp4.fp4_momentum_update(G, st.codes, st.scales, M, hist, 0.95, 1.0, flags=fp4.FP4_MOM_FLAG_SR, seed=t)
+    torch.cuda.synchronize()
+    assert int(hist.sum().item()) == rows * cols
+    bins = (M.view(torch.int32) & 0x7FFFFFFF) >> 18
+    want = torch.bincount(bins.flatten().long(), minlength=8192)
+    assert torch.equal(want.to(torch.int32), hist)
+    # without stochastic rounding any row can be checked alone; with it the random stream is
+    # numbered by matrix position, so the leading rows are
+    head = 8
+    oM, oc, os_, _ = oracle.momentum_update(G[:head].cpu().numpy(), prev_c[:head].cpu().numpy(),
+                                            prev_s[:head].cpu().numpy().view(np.uint16), 0.95, 1.0, sr=True, seed=1)
+    assert np.array_equal(M[:head].cpu().numpy().view(np.uint32), oM.view(np.uint32))
+    assert np.array_equal(st.codes[:head].cpu().numpy(), oc)
+    assert np.array_equal(st.scales[:head].cpu().numpy().view(np.uint16), os_)
+    idx = torch.tensor(np.random.default_rng(0).choice(rows, 24, replace=False), device="cuda")
+    Gs = G[idx].cpu().numpy()
+    pc, ps = prev_c[idx].cpu().numpy(), prev_s[idx].cpu().numpy().view(np.uint16)
+    st2_c, st2_s = prev_c.clone(), prev_s.clone()
+    fp4.fp4_momentum_update(G, st2_c, st2_s, M, None, 0.95, 1.0)
+    torch.cuda.synchronize()
+    oM, oc, os_, _ = oracle.momentum_update(Gs, pc, ps, 0.95, 1.0)
+    assert np.array_equal(M[idx].cpu().numpy().view(np.uint32), oM.view(np.uint32))
+    assert np.array_equal(st2_c[idx].cpu().numpy(), oc)
+    assert np.array_equal(st2_s[idx].cpu().numpy().view(np.uint16), os_)
+
+
+def test_argument_errors():
+    G = torch.zeros((16, 24), dtype=torch.float32, device="cuda")
+    c = torch.zeros((16, 12), dtype=torch.uint8, device="cuda")
+    s = torch.zeros((16, 2), dtype=torch.int16, device="cuda")
+    with pytest.raises(fp4.Fp4Error):
+        fp4.fp4_momentum_update(G, c, s, None, None, 0.9)            # cols not a multiple of 16
+    G = torch.zeros((16, 32), dtype=torch.float32, device="cuda")
+    c = torch.zeros((16, 16), dtype=torch.uint8, device="cuda")
+    with pytest.raises(fp4.Fp4Error):
+        fp4.fp4_momentum_update(G, c, s, None, None, 0.9, flags=4)   # unknown flag
+    with pytest.raises(fp4.Fp4Error):
+        fp4.fp4_momentum_update(G.flatten()[1:].reshape(1, -1)[:, :16], c, s, None, None, 0.9)  # misaligned

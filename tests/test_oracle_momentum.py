@@ -185,3 +185,28 @@ def test_stochastic_rounding_is_unbiased():
     ca, _ = oracle.momentum_encode(M, sr=True, seed=1)
     cb, _ = oracle.momentum_encode(M, sr=True, seed=2)
     assert not np.array_equal(ca, cb)
+
+
+def test_stochastic_rounding_random_bits_from_published_output():
+    # The first output of splitmix64(1234567) serves elements 0..7 of the matrix: its low word
+    # elements 0..3, its high word elements 4..7; in each word the low half decides element 0,
+    # the same bits reversed element 1, the high half element 2, reversed element 3.  A value at
+    # 1 + (65536 - r) / 131072 is the first that goes up to 1.5; the one before stays at 1.
+    z = 6457827717110365317
+    rev = lambda v: int(f"{v:016b}"[::-1], 2)
+    r = []
+    for w in (z & 0xFFFFFFFF, z >> 32):
+        r += [w & 0xFFFF, rev(w & 0xFFFF), w >> 16, rev(w >> 16)]
+    for delta, want in ((0, 1.5), (-1, 1.0)):
+        h = np.zeros(16)
+        h[15] = 6.0                                   # block scale 1
+        h[8:15] = 1.0                                 # keeps the maximum on 6
+        for e in range(8):
+            h[e] = 1.0 + (65536 - r[e] + delta) / 131072.0
+        x = (h @ H4).astype(np.float32)[None, :]
+        assert np.array_equal((x.astype(np.float64) @ H4)[0], h)   # exact in FP32
+        c, s = oracle.momentum_encode(x, sr=True, seed=1234567)
+        assert int(s[0, 0]) == 0x3F80
+        v = nib_values(nibbles(c))[0]
+        assert np.array_equal(v[:8], np.full(8, want)), (delta, v[:8])
+        assert np.array_equal(v[8:], h[8:])
