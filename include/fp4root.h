@@ -261,9 +261,9 @@ fp4_status fp4_gemm_nt(const uint8_t* a_codes, const uint8_t* a_scales, float a_
  * Arithmetic: m_prev = (code * scale) H_16 / 4 (natural-order butterfly, FP32), then
  * M = fl(fl(mu m_prev) + fl(g_scale G)).
  *
- * G       device, in : rows x cols FP32, 16-byte aligned
+ * G       device, in : rows x cols FP32, 32-byte aligned (the kernel moves 256 bits per access)
  * codes, scales  device, in/out: the state, updated in place; 16-byte aligned
- * M_out   device, out: rows x cols FP32 or NULL; must not overlap G
+ * M_out   device, out: rows x cols FP32 or NULL, 32-byte aligned; must not overlap G
  * hist    device, in/out or NULL: 8192 uint32 counters; counter ((bits of |M|) >> 18) is
  *         incremented for every element of M_t (the top 13 magnitude bits: the first pass of the
  *         outlier clip's quantile selection); the caller zeroes it
@@ -281,7 +281,7 @@ typedef struct fp4_momentum_params {
 fp4_status fp4_momentum_update(const float* G, int64_t rows, int64_t cols, uint8_t* codes, uint16_t* scales,
                                float* M_out, uint32_t* hist, const fp4_momentum_params* params,
                                cudaStream_t stream);
-/* M_out = the decoded state (device, rows x cols FP32, 16-byte aligned); the state is not changed. */
+/* M_out = the decoded state (device, rows x cols FP32, 32-byte aligned); the state is not changed. */
 fp4_status fp4_momentum_decode(const uint8_t* codes, const uint16_t* scales, int64_t rows, int64_t cols,
                                float* M_out, cudaStream_t stream);
 

@@ -123,73 +123,62 @@ __device__ __forceinline__ void mom_encode(float (&h)[16], uint64_t seed, uint64
   c = make_uint2(lo, hi);
 }
 
-// A warp's 32 blocks of M_t (2 KB) go to global memory through shared memory, so that every store
-// instruction of the warp writes 512 contiguous bytes: a thread writes its own block as four
-// 16-byte pieces, piece j at slot 4 lane + (j ^ ((lane >> 1) & 3)) (no bank conflicts on either
-// side), the warp syncs, and lane i of store t takes piece 32 t + i of the 2 KB.
-__device__ __forceinline__ void store_rows_coalesced(float4* stage, const float (&m)[16], bool valid, int lane,
-                                                     float* M_out, int64_t base, int64_t nblocks) {
-  if (valid) {
-#pragma unroll
-    for (int j = 0; j < 4; ++j)
-      stage[lane * 4 + (j ^ ((lane >> 1) & 3))] = make_float4(m[4 * j], m[4 * j + 1], m[4 * j + 2], m[4 * j + 3]);
-  }
-  __syncwarp();
-  float4* dst = reinterpret_cast<float4*>(M_out + base * 16);
-#pragma unroll
-  for (int t = 0; t < 4; ++t) {
-    const int i = t * 32 + lane, blk = i >> 2;
-    if (base + blk < nblocks) dst[i] = stage[blk * 4 + ((i & 3) ^ ((blk >> 1) & 3))];
-  }
-  __syncwarp();
+// 256-bit global accesses (32-byte aligned): a thread moves its block of 16 floats as two full
+// 32-byte sectors, so no sector is touched by two instructions -- with 128-bit pieces at a
+// 64-byte lane stride every sector is looked up twice on loads and written as two partial
+// sectors on stores.
+__device__ __forceinline__ void ldg_f32x8(const float* p, float* v) {
+  asm volatile("ld.global.nc.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7])
+               : "l"(p));
+}
+__device__ __forceinline__ void stg_f32x8(float* p, const float* v) {
+  asm volatile("st.global.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "f"(v[0]), "f"(v[1]), "f"(v[2]),
+               "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7])
+               : "memory");
 }
 
-// grid: any number of thread blocks of 256 threads; warps stride over groups of 32 consecutive
-// 16-blocks of the matrix.
+// grid: any number of thread blocks; threads stride over the 16-blocks of the matrix.
 template <bool SR, bool HIST>
 __global__ void __launch_bounds__(256) k_momentum_update(const float* __restrict__ G, int64_t nblocks, float mu,
                                                          float g_scale, uint64_t seed, uint8_t* codes,
                                                          uint16_t* scales, float* __restrict__ M_out,
                                                          uint32_t* __restrict__ hist) {
   __shared__ uint32_t sh[HIST ? kMomBins : 1];
-  __shared__ float4 stage_all[8 * 128];
   if (HIST) {
     for (int i = threadIdx.x; i < kMomBins; i += blockDim.x) sh[i] = 0;
     __syncthreads();
   }
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  float4* stage = stage_all + warp * 128;
-  const int64_t stride = (int64_t)gridDim.x * 256;
-  for (int64_t base = ((int64_t)blockIdx.x * 8 + warp) * 32; base < nblocks; base += stride) {
-    const int64_t b = base + lane;
-    const bool valid = b < nblocks;
-    float m[16];
-    if (valid) {
-      const uint2 c_in = *reinterpret_cast<const uint2*>(codes + b * 8);
-      const uint32_t s_in = scales[b];
-      const float4* src = reinterpret_cast<const float4*>(G + b * 16);
-      float g[16];
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  const uint64_t mu2 = pack2(mu, mu), gs2 = pack2(g_scale, g_scale);
+  for (int64_t b = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; b < nblocks; b += stride) {
+    const uint2 c_in = *reinterpret_cast<const uint2*>(codes + b * 8);
+    const uint32_t s_in = scales[b];
+    float g[16], m[16];
+    ldg_f32x8(G + b * 16, g);
+    ldg_f32x8(G + b * 16 + 8, g + 8);
+    mom_decode(c_in, s_in, m);
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const float4 t = __ldg(src + j);
-        g[4 * j] = t.x; g[4 * j + 1] = t.y; g[4 * j + 2] = t.z; g[4 * j + 3] = t.w;
-      }
-      mom_decode(c_in, s_in, m);
-#pragma unroll
-      for (int i = 0; i < 16; ++i) m[i] = __fadd_rn(__fmul_rn(mu, m[i]), __fmul_rn(g_scale, g[i]));
+    for (int i = 0; i < 8; ++i) {
+      float a0, a1, b0, b1;
+      unpack2(mul2(pack2(m[2 * i], m[2 * i + 1]), mu2), a0, a1);
+      unpack2(mul2(pack2(g[2 * i], g[2 * i + 1]), gs2), b0, b1);
+      m[2 * i] = __fadd_rn(a0, b0);       // scalar: the sum must not fuse with a product
+      m[2 * i + 1] = __fadd_rn(a1, b1);
     }
-    if (M_out) store_rows_coalesced(stage, m, valid, lane, M_out, base, nblocks);
-    if (valid) {
-      if (HIST) {
-#pragma unroll
-        for (int i = 0; i < 16; ++i) atomicAdd(&sh[(__float_as_uint(m[i]) & 0x7FFFFFFFu) >> 18], 1u);
-      }
-      uint2 c_out;
-      uint32_t s_out;
-      mom_encode<SR>(m, seed, (uint64_t)b * 16, c_out, s_out);
-      *reinterpret_cast<uint2*>(codes + b * 8) = c_out;
-      scales[b] = (uint16_t)s_out;
+    if (M_out) {
+      stg_f32x8(M_out + b * 16, m);
+      stg_f32x8(M_out + b * 16 + 8, m + 8);
     }
+    if (HIST) {
+#pragma unroll
+      for (int i = 0; i < 16; ++i) atomicAdd(&sh[(__float_as_uint(m[i]) & 0x7FFFFFFFu) >> 18], 1u);
+    }
+    uint2 c_out;
+    uint32_t s_out;
+    mom_encode<SR>(m, seed, (uint64_t)b * 16, c_out, s_out);
+    *reinterpret_cast<uint2*>(codes + b * 8) = c_out;
+    scales[b] = (uint16_t)s_out;
   }
   if (HIST) {
     __syncthreads();
@@ -201,29 +190,35 @@ __global__ void __launch_bounds__(256) k_momentum_update(const float* __restrict
 __global__ void __launch_bounds__(256) k_momentum_decode(const uint8_t* __restrict__ codes,
                                                          const uint16_t* __restrict__ scales, int64_t nblocks,
                                                          float* __restrict__ M_out) {
-  __shared__ float4 stage_all[8 * 128];
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int64_t stride = (int64_t)gridDim.x * 256;
-  for (int64_t base = ((int64_t)blockIdx.x * 8 + warp) * 32; base < nblocks; base += stride) {
-    const int64_t b = base + lane;
-    const bool valid = b < nblocks;
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  for (int64_t b = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; b < nblocks; b += stride) {
     float m[16];
-    if (valid) mom_decode(__ldg(reinterpret_cast<const uint2*>(codes + b * 8)), __ldg(scales + b), m);
-    store_rows_coalesced(stage_all + warp * 128, m, valid, lane, M_out, base, nblocks);
+    mom_decode(__ldg(reinterpret_cast<const uint2*>(codes + b * 8)), __ldg(scales + b), m);
+    stg_f32x8(M_out + b * 16, m);
+    stg_f32x8(M_out + b * 16 + 8, m + 8);
   }
 }
 
+// Without the histogram every thread block takes one group of 256 blocks.  With it a thread
+// block owns 32 KB of counters that it clears and flushes once, so the grid is what fits on the
+// GPU at once, shrunk so that all thread blocks run the same number of iterations.
 template <bool SR, bool HIST>
 cudaError_t launch_update(const float* G, int64_t nblocks, float mu, float g_scale, uint64_t seed, uint8_t* codes,
                           uint16_t* scales, float* M_out, uint32_t* hist, int sms, cudaStream_t st) {
-  int per_sm = 0;
-  cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_momentum_update<SR, HIST>, 256, 0);
-  if (e != cudaSuccess) return e;
-  if (per_sm < 1) per_sm = 1;
-  const int64_t need = (nblocks + 255) / 256;
-  const int64_t cap = (int64_t)sms * per_sm;
-  const unsigned grid = (unsigned)(need < cap ? need : cap);
-  k_momentum_update<SR, HIST><<<grid, 256, 0, st>>>(G, nblocks, mu, g_scale, seed, codes, scales, M_out, hist);
+  const int64_t units = (nblocks + 255) / 256;
+  int64_t grid = units;
+  if (HIST) {
+    int per_sm = 0;
+    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_momentum_update<SR, HIST>, 256, 0);
+    if (e != cudaSuccess) return e;
+    if (per_sm < 1) per_sm = 1;
+    if (per_sm > 4) per_sm = 4;  // measured: more resident counters only add clearing and flushing
+    const int64_t slots = (int64_t)sms * per_sm;
+    const int64_t iters = (units + slots - 1) / slots;
+    grid = (units + iters - 1) / iters;
+  }
+  k_momentum_update<SR, HIST><<<(unsigned)grid, 256, 0, st>>>(G, nblocks, mu, g_scale, seed, codes, scales, M_out,
+                                                              hist);
   count_launches(1);
   return cudaGetLastError();
 }

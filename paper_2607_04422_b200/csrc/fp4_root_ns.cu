@@ -516,7 +516,7 @@ fp4_status fp4_momentum_update(const float* G, int64_t rows, int64_t cols, uint8
   if (!G || !codes || !scales || !params) return FP4_ERR_INVALID_ARG;
   if (params->flags & ~FP4_MOM_FLAG_SR) return FP4_ERR_INVALID_ARG;
   if (rows <= 0 || cols <= 0 || (cols & 15)) return FP4_ERR_SHAPE;
-  if (!aligned(G, 16) || !aligned(codes, 16) || !aligned(scales, 16) || (M_out && !aligned(M_out, 16)) ||
+  if (!aligned(G, 32) || !aligned(codes, 16) || !aligned(scales, 16) || (M_out && !aligned(M_out, 32)) ||
       (hist && !aligned(hist, 4)))
     return FP4_ERR_ALIGNMENT;
   const DeviceInfo* d;
@@ -533,7 +533,7 @@ fp4_status fp4_momentum_decode(const uint8_t* codes, const uint16_t* scales, int
                                float* M_out, cudaStream_t stream) {
   if (!codes || !scales || !M_out) return FP4_ERR_INVALID_ARG;
   if (rows <= 0 || cols <= 0 || (cols & 15)) return FP4_ERR_SHAPE;
-  if (!aligned(codes, 16) || !aligned(scales, 16) || !aligned(M_out, 16)) return FP4_ERR_ALIGNMENT;
+  if (!aligned(codes, 16) || !aligned(scales, 16) || !aligned(M_out, 32)) return FP4_ERR_ALIGNMENT;
   const DeviceInfo* d;
   fp4_status rc = check_common(&d);
   if (rc != FP4_OK) return rc;

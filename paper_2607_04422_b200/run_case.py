@@ -23,11 +23,28 @@ def main():
     ap.add_argument("--reps", type=int, default=3)
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--quantize-only", action="store_true", help="time fp4_quantize instead of the NS step")
+    ap.add_argument("--momentum", choices=["rtn", "sr"], help="time fp4_momentum_update instead of the NS step")
     a = ap.parse_args()
     G = torch.from_numpy(workloads.gradient_like(a.m, a.n, seed=a.seed)).cuda()
     stream = torch.cuda.current_stream()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     times = []
+    if a.momentum:
+        codes = torch.zeros((a.m, a.n // 2), dtype=torch.uint8, device="cuda")
+        scales = torch.zeros((a.m, a.n // 16), dtype=torch.int16, device="cuda")
+        M = torch.empty_like(G)
+        hist = torch.zeros(8192, dtype=torch.int32, device="cuda")
+        flags = fp4.FP4_MOM_FLAG_SR if a.momentum == "sr" else 0
+        for i in range(a.reps):
+            e0.record(stream)
+            fp4.fp4_momentum_update(G, codes, scales, M, hist, 0.95, 1.0, flags, i)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            times.append(e0.elapsed_time(e1))
+        nbytes = a.m * a.n * 9.25
+        print(json.dumps({"case": "fp4_momentum_update", "mode": a.momentum, "m": a.m, "n": a.n, "ms": times,
+                          "gbs_best": nbytes / min(times) / 1e6}))
+        return
     if a.quantize_only:
         codes = torch.empty((a.m, a.n // 2), dtype=torch.uint8, device="cuda")
         scales = torch.empty(fp4.fp4_scale_bytes(a.m, a.n), dtype=torch.uint8, device="cuda")

@@ -170,3 +170,5 @@ def test_argument_errors():
         fp4.fp4_momentum_update(G, c, s, None, None, 0.9, flags=4)   # unknown flag
     with pytest.raises(fp4.Fp4Error):
         fp4.fp4_momentum_update(G.flatten()[1:].reshape(1, -1)[:, :16], c, s, None, None, 0.9)  # misaligned
+    with pytest.raises(fp4.Fp4Error):
+        fp4.fp4_momentum_update(G.flatten()[4:].reshape(1, -1)[:, :16], c, s, None, None, 0.9)  # 16 but not 32 bytes
