@@ -93,6 +93,14 @@ typedef struct {
   uint32_t max_group;  /* fp4_root_ns_batched: at most this many equal-shape matrices run their
                           stages in lockstep as single launches; 0 = library default (16)     */
   uint64_t seed;       /* FP4_FLAG_RHT: seed of the sign draws; default 0                    */
+  uint32_t* const* top_hist; /* NULL (default), or a host array with one entry per matrix of the call
+                          (one entry for fp4_root_ns and fp4_root_ns_static): NULL, or a device
+                          array of 8192 counters that already holds, for that matrix, the number
+                          of elements whose |g| has each value of its top 13 magnitude bits
+                          (bits >> 18), as fp4_momentum_update writes for its M_t.  The clip then
+                          skips its first pass over the matrix.  The counters must describe
+                          exactly the matrix passed as G; they are consumed: zero when the step
+                          has run.  Ignored when the clip is disabled.                        */
 } fp4_ns_params;
 
 const char* fp4_status_string(fp4_status s);

@@ -42,10 +42,11 @@ class Fp4Error(RuntimeError):
 class NsParams(C.Structure):
     """fp4_ns_params"""
     _fields_ = [("a", C.c_float), ("b", C.c_float), ("c", C.c_float), ("clip_quantile", C.c_float),
-                ("eps", C.c_float), ("flags", C.c_uint32), ("max_group", C.c_uint32), ("seed", C.c_uint64)]
+                ("eps", C.c_float), ("flags", C.c_uint32), ("max_group", C.c_uint32), ("seed", C.c_uint64),
+                ("top_hist", C.POINTER(C.c_void_p))]
 
     @classmethod
-    def make(cls, abc=None, clip_quantile=0.99, eps=1e-7, flags=0, max_group=0, seed=0):
+    def make(cls, abc=None, clip_quantile=0.99, eps=1e-7, flags=0, max_group=0, seed=0, top_hist=None):
         p = cls()
         if abc is None:
             p.a = p.b = p.c = float("nan")
@@ -54,6 +55,11 @@ class NsParams(C.Structure):
         p.clip_quantile, p.eps, p.flags = float(clip_quantile), float(eps), int(flags)
         p.max_group = int(max_group)
         p.seed = int(seed)
+        if top_hist is not None:
+            # one entry per matrix of the call: a tensor of 8192 int32 counters, or None
+            arr = (C.c_void_p * len(top_hist))(*[h.data_ptr() if h is not None else None for h in top_hist])
+            p._top_hist_keepalive = arr
+            p.top_hist = C.cast(arr, C.POINTER(C.c_void_p))
         return p
 
 

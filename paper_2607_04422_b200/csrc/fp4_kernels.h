@@ -127,6 +127,7 @@ struct PrologueItem {
   bool clear_status;
   bool store_x;   // write X0 in FP32 (not needed when the first G3 stage reads G itself)
   int64_t x_rows, x_cols;  // extent and row pitch of X: the work shape in the workspace, the caller's shape in `out`
+  uint32_t* hist_top;      // the caller's histogram of the top 13 magnitude bits of G, or null
 };
 // count matrices that share the shape (s, l) and the clip / eps parameters
 cudaError_t launch_prologue_group(const PrologueItem* items, int count, int write_q, const QuantOpts& q,

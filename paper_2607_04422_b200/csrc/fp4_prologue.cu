@@ -31,6 +31,7 @@ struct PrepMatrix {
   NsHeader* hdr;
   float* scalars;
   uint32_t* hist;      // 8192 counters
+  uint32_t* hist_top;  // the caller's counters of the first radix pass (then pass 1 is skipped), or null
   double* partial;     // one FP64 partial per statistics block
   uint32_t* cand;      // candidate list (the A buffer of the workspace, unused until G1)
   uint8_t* qx_codes; uint8_t* qx_sf;
@@ -82,6 +83,7 @@ constexpr int kTopBins = 1 << kTopBits;      // 8192
 __global__ void __launch_bounds__(512) kp_hist_top(const __grid_constant__ PrepGroup g) {
   __shared__ uint32_t sh[kTopBins];
   const PrepMatrix& m = g.mat[blockIdx.y];
+  if (m.hist_top) return;  // the caller counted this matrix already
   for (int i = threadIdx.x; i < kTopBins; i += blockDim.x) sh[i] = 0;
   __syncthreads();
   const float4* src = reinterpret_cast<const float4*>(m.G);
@@ -149,7 +151,7 @@ __device__ __forceinline__ void pick_bin(NsHeader* hdr, uint32_t* hist, int shif
 
 __global__ void __launch_bounds__(256) kp_pick_top(const __grid_constant__ PrepGroup g) {
   const PrepMatrix& m = g.mat[blockIdx.y];
-  pick_bin<kTopBins>(m.hdr, m.hist, kTopShift, &m.hdr->bin_count, &m.hdr->count_below);
+  pick_bin<kTopBins>(m.hdr, m.hist_top ? m.hist_top : m.hist, kTopShift, &m.hdr->bin_count, &m.hdr->count_below);
 }
 
 // ---- pass 2: candidates of the picked bin, FP64 sum of squares below the bin, max |g|.
@@ -587,6 +589,7 @@ cudaError_t launch_prologue_group(const PrologueItem* items, int count, int writ
     g.zero_words = (int)(pl.zero_bytes / 4);
     g.ix = pl.ix;
     g.q = q;
+    bool all_counted = true;
     for (int j = 0; j < nn; ++j) {
       const PrologueItem& it = items[i0 + j];
       const fp4_ws_layout& L = it.pl->lay;
@@ -603,6 +606,8 @@ cudaError_t launch_prologue_group(const PrologueItem* items, int count, int writ
       m.clear_status = it.clear_status ? 1 : 0;
       m.store_x = it.store_x ? 1 : 0;
       m.x_rows = it.x_rows; m.x_cols = it.x_cols;
+      m.hist_top = it.hist_top;
+      if (!it.hist_top) all_counted = false;
     }
     const int sms = pl.sms;
     int64_t hb = (g.n4 + 512 * 4 - 1) / (512 * 4);
@@ -614,9 +619,9 @@ cudaError_t launch_prologue_group(const PrologueItem* items, int count, int writ
       count_launches(1);
       if (g.clip) {
         kp_arm<<<gy1, 1, 0, st>>>(g);
-        kp_hist_top<<<gh, 512, 0, st>>>(g);
+        if (!all_counted) kp_hist_top<<<gh, 512, 0, st>>>(g);
         kp_pick_top<<<gy1, 256, 0, st>>>(g);
-        count_launches(3);
+        count_launches(all_counted ? 2 : 3);
       }
     }
     {

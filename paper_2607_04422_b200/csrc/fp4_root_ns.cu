@@ -150,6 +150,7 @@ void default_params(fp4_ns_params* p) {
   p->flags = 0;
   p->max_group = 0;
   p->seed = 0;
+  p->top_hist = nullptr;
 }
 
 // The 16 signs of the j-th random Hadamard matrix of a call: splitmix64 on seed + j.
@@ -265,6 +266,7 @@ struct MatrixCtx {
   GemmProblem g3_first;       // iteration 0: as g3[0], but a wide input's FP32 tile is G itself (no X0 copy)
   bool store_x0;              // the prologue writes X0 in FP32
   int64_t x_rows, x_cols;     // extent (and row pitch) of X
+  uint32_t* hist_top;         // the caller's first-pass histogram of G, or null
 };
 
 fp4_status prepare_matrix(const DeviceInfo* d, const float* G, float* out, int64_t m, int64_t n, int steps,
@@ -274,6 +276,7 @@ fp4_status prepare_matrix(const DeviceInfo* d, const float* G, float* out, int64
   const fp4_ws_layout& L = c->pl.lay;
   const int64_t s = c->pl.s, l = c->pl.l;
   c->G = G; c->out = out; c->ws = ws;
+  c->hist_top = nullptr;
   c->X = c->pl.tall ? reinterpret_cast<float*>(ws + L.X) : out;
   // extent of X: the padded work shape in the workspace, the caller's shape in `out` (TMA fills what
   // lies outside with zeros on loads and drops it on stores)
@@ -366,7 +369,8 @@ fp4_status run_group(const DeviceInfo* d, MatrixCtx* mats, int count, int steps,
     std::vector<PrologueItem> items((size_t)count);
     for (int i = 0; i < count; ++i) {
       MatrixCtx& c = mats[i];
-      items[(size_t)i] = PrologueItem{c.G, c.X, c.ws, &c.pl, clear_first_status && i == 0, c.store_x0, c.x_rows, c.x_cols};
+      items[(size_t)i] = PrologueItem{c.G, c.X, c.ws, &c.pl, clear_first_status && i == 0, c.store_x0, c.x_rows, c.x_cols,
+                                      c.hist_top};
     }
     if (launch_prologue_group(items.data(), count, steps > 0 || keep, quant_opts(p, 0), st) != cudaSuccess)
       return FP4_ERR_CUDA;
@@ -452,6 +456,7 @@ fp4_status run_one(const DeviceInfo* d, const float* G, float* out, int64_t m, i
   MatrixCtx c;
   fp4_status rc = prepare_matrix(d, G, out, m, n, steps, p, ws, &c);
   if (rc != FP4_OK) return rc;
+  if (p->top_hist) c.hist_top = p->top_hist[0];
   return run_group(d, &c, 1, steps, p, reinterpret_cast<uint32_t*>(ws + c.pl.lay.header), nullptr, clear_status, st);
 }
 
@@ -622,6 +627,7 @@ fp4_status fp4_root_ns_batched(int count, const float* const* G, float* const* o
   for (int i = 0; i < count; ++i) {
     rc = prepare_matrix(d, G[i], out[i], m[i], n[i], steps, p, base + off, &ctx[(size_t)i]);
     if (rc != FP4_OK) return rc;
+    if (p->top_hist) ctx[(size_t)i].hist_top = p->top_hist[i];
     off += align_up(ctx[(size_t)i].pl.lay.total, 1024);
   }
   GemmProblem* table = reinterpret_cast<GemmProblem*>(base + off);

@@ -172,3 +172,62 @@ def test_argument_errors():
         fp4.fp4_momentum_update(G.flatten()[1:].reshape(1, -1)[:, :16], c, s, None, None, 0.9)  # misaligned
     with pytest.raises(fp4.Fp4Error):
         fp4.fp4_momentum_update(G.flatten()[4:].reshape(1, -1)[:, :16], c, s, None, None, 0.9)  # 16 but not 32 bytes
+
+
+def _ns(G, steps=2, top_hist=None):
+    m, n = G.shape
+    out = torch.full((m, n), float("nan"), device="cuda")
+    ws = torch.empty(fp4.fp4_root_ns_workspace_bytes(m, n, steps, 0), dtype=torch.uint8, device="cuda")
+    p = fp4.NsParams.make(top_hist=top_hist)
+    fp4.fp4_root_ns(G, out, steps, p, ws)
+    assert fp4.fp4_last_device_status(ws) == 0
+    return out
+
+
+@pytest.mark.parametrize("shape", [(256, 512), (1024, 384), (400, 1136)])
+def test_momentum_histogram_feeds_the_clip(shape):
+    # M_t and its histogram from the momentum step; the Newton-Schulz step that takes the
+    # histogram must give exactly what it gives when it counts M_t itself, and the oracle chain
+    # (momentum step, then Root step) must agree with the GPU chain
+    rows, cols = shape
+    G = _gradient(rows, cols, seed=21)
+    st = GpuState(rows, cols)
+    c0, s0 = oracle.momentum_encode(_gradient(rows, cols, seed=22))
+    st.load(c0, s0)
+    Gd = torch.from_numpy(G).cuda()
+    M = torch.empty_like(Gd)
+    hist = torch.zeros(8192, dtype=torch.int32, device="cuda")
+    fp4.fp4_momentum_update(Gd, st.codes, st.scales, M, hist, 0.95, 1.0)
+    ref = _ns(M)
+    got = _ns(M, top_hist=[hist])
+    torch.cuda.synchronize()
+    assert torch.equal(ref, got)
+    assert int(hist.abs().sum().item()) == 0          # consumed
+    oM, _, _, _ = oracle.momentum_update(G, c0, s0, 0.95, 1.0)
+    assert np.array_equal(M.cpu().numpy().view(np.uint32), oM.view(np.uint32))
+    want = oracle.root_ns(oM, 2)
+    err = np.linalg.norm(got.cpu().numpy() - want) / np.linalg.norm(want)
+    assert err < 2e-3, err
+
+
+def test_momentum_histograms_in_a_batched_call():
+    shapes = [(256, 512), (256, 512), (512, 256), (384, 384), (256, 512)]
+    Ms, hists, outs_ref = [], [], []
+    for i, (r, c) in enumerate(shapes):
+        Gd = torch.from_numpy(_gradient(r, c, seed=30 + i)).cuda()
+        st = GpuState(r, c)
+        M = torch.empty_like(Gd)
+        h = torch.zeros(8192, dtype=torch.int32, device="cuda")
+        fp4.fp4_momentum_update(Gd, st.codes, st.scales, M, h, 0.9, 1.0)
+        Ms.append(M)
+        hists.append(h if i != 1 else None)           # one matrix of a group counts for itself
+        outs_ref.append(_ns(M, steps=3))
+    outs = [torch.empty_like(M) for M in Ms]
+    ws = torch.empty(fp4.fp4_root_ns_batched_workspace_bytes(shapes, 3, 0), dtype=torch.uint8, device="cuda")
+    fp4.fp4_root_ns_batched(Ms, outs, 3, fp4.NsParams.make(top_hist=hists), ws)
+    assert fp4.fp4_last_device_status(ws) == 0
+    for a, b in zip(outs, outs_ref):
+        assert torch.equal(a, b)
+    for h in hists:
+        if h is not None:
+            assert int(h.abs().sum().item()) == 0
