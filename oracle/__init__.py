@@ -54,6 +54,11 @@ def build(force: bool = False) -> str:
     return _LIB
 
 
+class AdamWParams(C.Structure):
+    _fields_ = [("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
+                ("weight_decay", C.c_float), ("step", C.c_int32), ("sr", C.c_int32), ("seed", C.c_uint64)]
+
+
 def lib():
     global _lib
     if _lib is None:
@@ -80,6 +85,11 @@ def lib():
         L.orc_momentum_update.argtypes = [_f32p, C.c_int64, C.c_int64, C.c_float, C.c_float, C.c_int, C.c_uint64,
                                           _u8p, _u16p, _f32p, _u32p]
         L.orc_momentum_update.restype = None
+        L.orc_v_encode.argtypes = [_f32p, C.c_int64, _u8p, _u16p, _u16p]; L.orc_v_encode.restype = None
+        L.orc_v_decode.argtypes = [_u8p, _u16p, _u16p, C.c_int64, _f32p]; L.orc_v_decode.restype = None
+        L.orc_adamw_update.argtypes = [_u16p, _u16p, C.c_int64, _u8p, _u16p, _u8p, _u16p, _u16p,
+                                       C.POINTER(AdamWParams), _f32p, _f32p]
+        L.orc_adamw_update.restype = None
         L.orc_splitmix64_at.argtypes = [C.c_uint64, C.c_uint64]; L.orc_splitmix64_at.restype = C.c_uint64
         L.orc_dequantize.argtypes = [_u8p, _u8p, C.c_float, C.c_int64, C.c_int64, _f32p]
         L.orc_dequantize.restype = None
@@ -212,6 +222,55 @@ def momentum_update(G, codes, scales, mu, g_scale=1.0, sr=False, seed=0, want_hi
                               M.ctypes.data_as(_f32p),
                               hist.ctypes.data_as(_u32p) if want_hist else None)
     return M, codes, scales, hist
+
+
+def bf16_bits(x):
+    """FP32 array -> BF16 bit patterns (uint16), round to nearest even."""
+    r = bf16_round(np.asarray(x, np.float32))
+    return (np.ascontiguousarray(r).view(np.uint32) >> 16).astype(np.uint16)
+
+
+def bf16_to_f32(bits):
+    return (np.asarray(bits, np.uint16).astype(np.uint32) << 16).view(np.float32)
+
+
+def v_encode(v):
+    """Second-moment state of a flat FP32 array (length a multiple of 256):
+    (codes u8 n/2, scales u16 n/16, means u16 n/256)."""
+    v, vp = _f32(np.asarray(v, np.float32).ravel())
+    n = v.size
+    codes = np.empty(n // 2, np.uint8); scales = np.empty(n // 16, np.uint16); means = np.empty(n // 256, np.uint16)
+    lib().orc_v_encode(vp, n, codes.ctypes.data_as(_u8p), scales.ctypes.data_as(_u16p), means.ctypes.data_as(_u16p))
+    return codes, scales, means
+
+
+def v_decode(codes, scales, means):
+    codes = np.ascontiguousarray(codes, np.uint8); scales = np.ascontiguousarray(scales, np.uint16)
+    means = np.ascontiguousarray(means, np.uint16)
+    n = codes.size * 2
+    out = np.empty(n, np.float32)
+    lib().orc_v_decode(codes.ctypes.data_as(_u8p), scales.ctypes.data_as(_u16p), means.ctypes.data_as(_u16p), n,
+                       out.ctypes.data_as(_f32p))
+    return out
+
+
+def adamw_update(W_bits, G_bits, state, lr, beta1=0.9, beta2=0.95, eps=1e-8, weight_decay=0.1, step=1, sr=False,
+                 seed=0):
+    """One packed AdamW step.  state = (m_codes, m_scales, v_codes, v_scales, v_means) or None for
+    zeros.  Returns (W_bits, new state, m FP32, v FP32); inputs are not modified."""
+    W = np.array(W_bits, np.uint16, copy=True).ravel()
+    G = np.ascontiguousarray(G_bits, np.uint16).ravel()
+    n = W.size
+    if state is None:
+        state = (np.zeros(n // 2, np.uint8), np.zeros(n // 16, np.uint16), np.zeros(n // 2, np.uint8),
+                 np.zeros(n // 16, np.uint16), np.zeros(n // 256, np.uint16))
+    mc, ms, vc, vs, vm = [np.array(a, copy=True) for a in state]
+    m = np.empty(n, np.float32); v = np.empty(n, np.float32)
+    prm = AdamWParams(lr, beta1, beta2, eps, weight_decay, step, int(bool(sr)), seed)
+    lib().orc_adamw_update(W.ctypes.data_as(_u16p), G.ctypes.data_as(_u16p), n, mc.ctypes.data_as(_u8p),
+                           ms.ctypes.data_as(_u16p), vc.ctypes.data_as(_u8p), vs.ctypes.data_as(_u16p),
+                           vm.ctypes.data_as(_u16p), C.byref(prm), m.ctypes.data_as(_f32p), v.ctypes.data_as(_f32p))
+    return W, (mc, ms, vc, vs, vm), m, v
 
 
 def dequantize(codes, scales, s_g):

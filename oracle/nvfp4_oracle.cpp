@@ -72,6 +72,28 @@
 //     round trip, unbiasedness of the stochastic rounding and the generator's published
 //     test vector are pinned.
 //
+//   * second-moment state and the packed AdamW update (Section 3.3: square root, BF16 tile mean,
+//     16-element Hadamard transform, NVFP4 storage with per-16 BF16 scales and per-256 BF16
+//     means = 5.0625 bits per element; reconstruction inverts the transform and the mean
+//     separation and squares; BF16 weights and gradients, no FP32 master weight; Section 2 gives
+//     the two moment recursions).  Readings, the paper giving no formulas:
+//       - a tensor is a flat array whose length is a multiple of 256; a tile is 256 consecutive
+//         elements, a block 16; s = sqrt(v) in FP32; the tile mean is BF16(sum / 256), the sum
+//         taken per block in element order and over the 16 block sums by a pairwise tree;
+//         residual s - mean, times the fixed H_16 / 4; block scale and codes exactly as for the
+//         first moment (two candidates BF16(amax/6), BF16(amax/4), the smaller squared error
+//         wins), round to nearest; decode: (code * scale) H_16 / 4 + mean, squared;
+//       - update with step count t (bias corrections from pow in FP64, rounded to FP32):
+//           m = fl(fl(b1 m') + fl((1-b1) g)),  v = fl(fl(b2 v') + fl((1-b2) fl(g g))),
+//           s = sqrt(v),  den = fl(fl(s * rsb2) + eps),  w1 = fl(w * fl(1 - fl(lr wd))),
+//           w2 = fl(w1 - fl(fl(lr / bc1) * fl(m / den))),  W = BF16(w2) to nearest even,
+//         m', v' the decoded states, bc1 = 1 - b1^t, rsb2 = 1 / sqrt(1 - b2^t); the states are
+//         re-encoded from m and v (the first moment optionally with stochastic rounding).
+//     Parity unpinned against the authors' code; pinned: the bit count, an exact round trip,
+//     the mean and the decode against numpy FP64, the first step against its closed form and
+//     against torch.optim.AdamW, and the paper's claim that the pipeline reconstructs a
+//     heavy-tailed second moment better than direct NVFP4.
+//
 // Build:  g++ -O2 -std=c++17 -ffp-contract=off -fopenmp -shared -fPIC
 
 #include <algorithm>
@@ -429,6 +451,61 @@ void mom_decode_block(const uint8_t* packed, uint16_t scale_bits, float* v) {
   hadamard16(h, 0, v);
 }
 
+// ---- second-moment state and packed AdamW (Section 3.3) ----
+
+// Two-candidate round-to-nearest encoding of one transformed block (shared by both moments).
+void state_encode_rtn(const float* h, uint8_t* nib, float* d_out) {
+  float amax = amax_of(h, 16);
+  float d6 = bf16_round(amax / 6.0f);
+  float d4 = bf16_round(amax / 4.0f);
+  uint8_t n4[16];
+  float err6 = mom_encode_rtn(h, d6, nib);
+  float err4 = mom_encode_rtn(h, d4, n4);
+  *d_out = d6;
+  if (err4 < err6) { *d_out = d4; for (int i = 0; i < 16; ++i) nib[i] = n4[i]; }
+}
+
+// BF16 mean of sqrt-domain values of one tile of 256: block sums in element order, then a
+// pairwise tree over the 16 block sums.
+float tile_mean_bf16(const float* s) {
+  float part[16];
+  for (int b = 0; b < 16; ++b) {
+    float acc = 0.0f;
+    for (int i = 0; i < 16; ++i) acc = acc + s[b * 16 + i];
+    part[b] = acc;
+  }
+  for (int stride = 1; stride < 16; stride *= 2)
+    for (int b = 0; b < 16; b += 2 * stride) part[b] = part[b] + part[b + stride];
+  return bf16_round(part[0] * 0.00390625f);
+}
+
+// Encode one tile of 256 second-moment values given in the square-root domain.
+void v_encode_tile(const float* s, uint8_t* codes /*128*/, uint16_t* scales /*16*/, uint16_t* mean_bits) {
+  float mean = tile_mean_bf16(s);
+  *mean_bits = bf16_bits(mean);
+  for (int b = 0; b < 16; ++b) {
+    float r[16], h[16], d;
+    uint8_t nib[16];
+    for (int i = 0; i < 16; ++i) r[i] = s[b * 16 + i] - mean;
+    hadamard16(r, 0, h);
+    state_encode_rtn(h, nib, &d);
+    scales[b] = bf16_bits(d);
+    for (int i = 0; i < 8; ++i) codes[b * 8 + i] = (uint8_t)(nib[2 * i] | (nib[2 * i + 1] << 4));
+  }
+}
+
+void v_decode_tile(const uint8_t* codes, const uint16_t* scales, uint16_t mean_bits, float* v) {
+  float mean = bf16_from_bits(mean_bits);
+  for (int b = 0; b < 16; ++b) {
+    float r[16];
+    mom_decode_block(codes + b * 8, scales[b], r);
+    for (int i = 0; i < 16; ++i) {
+      float u = r[i] + mean;
+      v[b * 16 + i] = u * u;
+    }
+  }
+}
+
 }  // namespace
 
 extern "C" {
@@ -733,5 +810,79 @@ void orc_momentum_update(const float* G, int64_t rows, int64_t cols, float mu, f
 }
 
 uint64_t orc_splitmix64_at(uint64_t seed, uint64_t idx) { return splitmix64_at(seed, idx); }
+
+void orc_v_encode(const float* v, int64_t n, uint8_t* codes, uint16_t* scales, uint16_t* means) {
+#pragma omp parallel for schedule(static)
+  for (int64_t t = 0; t < n / 256; ++t) {
+    float s[256];
+    for (int i = 0; i < 256; ++i) s[i] = std::sqrt(v[t * 256 + i]);
+    v_encode_tile(s, codes + t * 128, scales + t * 16, means + t);
+  }
+}
+
+void orc_v_decode(const uint8_t* codes, const uint16_t* scales, const uint16_t* means, int64_t n, float* v) {
+#pragma omp parallel for schedule(static)
+  for (int64_t t = 0; t < n / 256; ++t) v_decode_tile(codes + t * 128, scales + t * 16, means[t], v + t * 256);
+}
+
+struct orc_adamw_params {
+  float lr, beta1, beta2, eps, weight_decay;
+  int32_t step;   // t >= 1
+  int32_t sr;     // stochastic rounding of the first moment
+  uint64_t seed;
+};
+
+// One packed AdamW step in place: W (BF16 bits), the first-moment state (m_codes, m_scales) and
+// the second-moment state (v_codes, v_scales, v_means); G (BF16 bits) is read.  n: a multiple of
+// 256.  m_out / v_out (may be null): the FP32 moments of this step, before re-encoding.
+void orc_adamw_update(uint16_t* W, const uint16_t* G, int64_t n, uint8_t* m_codes, uint16_t* m_scales,
+                      uint8_t* v_codes, uint16_t* v_scales, uint16_t* v_means, const orc_adamw_params* p,
+                      float* m_out, float* v_out) {
+  const float b1 = p->beta1, b2 = p->beta2;
+  const float omb1 = 1.0f - b1, omb2 = 1.0f - b2;
+  const float bc1 = (float)(1.0 - std::pow((double)b1, (double)p->step));
+  const float rsb2 = (float)(1.0 / std::sqrt(1.0 - std::pow((double)b2, (double)p->step)));
+  const float step_size = p->lr / bc1;
+  const float lrwd = p->lr * p->weight_decay;
+  const float decay = 1.0f - lrwd;
+#pragma omp parallel for schedule(static)
+  for (int64_t t = 0; t < n / 256; ++t) {
+    float vprev[256], s[256], m[256];
+    v_decode_tile(v_codes + t * 128, v_scales + t * 16, v_means[t], vprev);
+    for (int b = 0; b < 16; ++b) {
+      float mprev[16];
+      const int64_t e0 = t * 256 + b * 16;
+      mom_decode_block(m_codes + e0 / 2, m_scales[e0 / 16], mprev);
+      for (int i = 0; i < 16; ++i) {
+        const int64_t e = e0 + i;
+        float g = bf16_from_bits(G[e]);
+        float w = bf16_from_bits(W[e]);
+        float t1 = b1 * mprev[i];
+        float t2 = omb1 * g;
+        float mi = t1 + t2;
+        float gg = g * g;
+        float t3 = b2 * vprev[b * 16 + i];
+        float t4 = omb2 * gg;
+        float vi = t3 + t4;
+        float si = std::sqrt(vi);
+        float den = si * rsb2;
+        den = den + p->eps;
+        float w1 = w * decay;
+        float upd = mi / den;
+        float su = step_size * upd;
+        float w2 = w1 - su;
+        W[e] = bf16_bits(bf16_round(w2));
+        m[b * 16 + i] = mi;
+        s[b * 16 + i] = si;
+        if (m_out) m_out[e] = mi;
+        if (v_out) v_out[e] = vi;
+      }
+      uint8_t nib[16];
+      mom_encode_block(m + b * 16, p->sr, p->seed, (uint64_t)e0, nib, &m_scales[e0 / 16]);
+      for (int i = 0; i < 8; ++i) m_codes[e0 / 2 + i] = (uint8_t)(nib[2 * i] | (nib[2 * i + 1] << 4));
+    }
+    v_encode_tile(s, v_codes + t * 128, v_scales + t * 16, v_means + t);
+  }
+}
 
 }  // extern "C"
