@@ -293,6 +293,44 @@ fp4_status fp4_momentum_update(const float* G, int64_t rows, int64_t cols, uint8
 fp4_status fp4_momentum_decode(const uint8_t* codes, const uint16_t* scales, int64_t rows, int64_t cols,
                                float* M_out, cudaStream_t stream);
 
+/* ---- packed AdamW step on NVFP4 moment states --------------------------------------------------
+ * Section 3.3 ("Quantized-State AdamW") and the appendix's accounting: BF16 weight and gradient,
+ * a 5-bit first moment and a 5.0625-bit second moment, 42.0625 bits per parameter, no FP32
+ * master weight; decay and parameter update fused into the pass that reconstructs and re-packs
+ * the states.  Section 2 gives the moment recursions.
+ *
+ * A tensor is a flat array of n elements, n a positive multiple of 256 (else FP4_ERR_SHAPE).
+ *   W         device, in/out: n BF16 weights, 32-byte aligned
+ *   G         device, in    : n BF16 gradients, 32-byte aligned; must not overlap W
+ *   m_codes, m_scales       : the first moment in the state format of fp4_momentum_update
+ *                             (n/2 bytes, n/16 uint16), in/out
+ *   v_codes, v_scales, v_means: the second moment, in/out: with s = sqrt(v) and a tile = 256
+ *       consecutive elements, v_means (n/256 uint16) holds BF16(sum(s) / 256) per tile (FP32 sums:
+ *       each block of 16 in element order, then a pairwise tree over the 16 block sums);
+ *       v_codes / v_scales hold the blocks of s - mean times H_16 / 4, encoded like the first
+ *       moment with round to nearest (two candidate BF16 scales amax/6, amax/4).  Decoding:
+ *       ((code * scale) H_16 / 4 + mean)^2.  All-zero states are zero moments.
+ *   All state arrays 16-byte aligned.
+ * Arithmetic, FP32, one rounded operation per step, t = params->step >= 1:
+ *   m = b1 m' + (1-b1) g,  v = b2 v' + (1-b2) (g g),  s = sqrt(v),  den = s * rsb2 + eps,
+ *   w2 = w (1 - lr wd) - (lr / bc1) (m / den),  W = BF16(w2) to nearest even;
+ *   bc1 = 1 - b1^t and rsb2 = 1 / sqrt(1 - b2^t) are evaluated in double and rounded to FP32.
+ * FP4_MOM_FLAG_SR: stochastic rounding of the first moment as in fp4_momentum_update, the
+ * random stream numbered by element index and seeded by params->seed.
+ * Errors: FP4_ERR_INVALID_ARG (null pointer, unknown flag, step < 1), FP4_ERR_SHAPE,
+ * FP4_ERR_ALIGNMENT, FP4_ERR_ARCH, FP4_ERR_CUDA.
+ */
+typedef struct fp4_adamw_params {
+  float lr, beta1, beta2, eps, weight_decay;
+  int32_t step;    /* t, from 1 */
+  uint32_t flags;  /* FP4_MOM_FLAG_SR */
+  uint32_t reserved;
+  uint64_t seed;
+} fp4_adamw_params;
+fp4_status fp4_adamw_update(uint16_t* W, const uint16_t* G, int64_t n, uint8_t* m_codes, uint16_t* m_scales,
+                            uint8_t* v_codes, uint16_t* v_scales, uint16_t* v_means,
+                            const fp4_adamw_params* params, cudaStream_t stream);
+
 /* ---- measurement support (the paper has no counterpart) -----------------------------------
  * While profiling is enabled, every group of launches of the step is bracketed by a pair of
  * CUDA events on the caller's stream; fp4_profile_collect waits for them, adds the elapsed
@@ -303,7 +341,7 @@ fp4_status fp4_momentum_decode(const uint8_t* codes, const uint16_t* scales, int
  */
 enum { FP4_PROF_CLIP = 0, FP4_PROF_STATS = 1, FP4_PROF_PREP = 2, FP4_PROF_G1 = 3, FP4_PROF_G2 = 4,
        FP4_PROF_G3 = 5, FP4_PROF_TRANSPOSE = 6, FP4_PROF_QUANTIZE = 7, FP4_PROF_MOMENTUM = 8,
-       FP4_PROF_CLASSES = 9 };
+       FP4_PROF_ADAMW = 9, FP4_PROF_CLASSES = 10 };
 void fp4_profile_enable(int on);
 fp4_status fp4_profile_collect(float* ms, int* groups);
 uint64_t fp4_kernel_launches(void);

@@ -30,7 +30,7 @@ EXPORTS = ("fp4_status_string", "fp4_scale_bytes", "fp4_quantize", "fp4_root_coe
            "fp4_root_ns_batched", "fp4_last_device_status", "fp4_root_ns_workspace_layout", "fp4_gemm_nt",
            "fp4_profile_enable", "fp4_profile_collect", "fp4_kernel_launches", "fp4_root_ns_static",
            "fp4_selftest_bounded_wait")
-PROF_CLASSES = ("clip", "stats", "prep", "G1", "G2", "G3", "transpose", "quantize", "momentum")
+PROF_CLASSES = ("clip", "stats", "prep", "G1", "G2", "G3", "transpose", "quantize", "momentum", "adamw")
 
 
 class Fp4Error(RuntimeError):
@@ -66,6 +66,13 @@ class NsParams(C.Structure):
 class MomentumParams(C.Structure):
     """fp4_momentum_params of include/fp4root.h."""
     _fields_ = [("mu", C.c_float), ("g_scale", C.c_float), ("flags", C.c_uint32), ("reserved", C.c_uint32),
+                ("seed", C.c_uint64)]
+
+
+class AdamwParams(C.Structure):
+    """fp4_adamw_params of include/fp4root.h."""
+    _fields_ = [("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
+                ("weight_decay", C.c_float), ("step", C.c_int32), ("flags", C.c_uint32), ("reserved", C.c_uint32),
                 ("seed", C.c_uint64)]
 
 
@@ -122,6 +129,8 @@ def load_library():
     L.fp4_kernel_launches.argtypes = []; L.fp4_kernel_launches.restype = C.c_uint64
     L.fp4_momentum_update.argtypes = [vp, i64, i64, vp, vp, vp, vp, C.POINTER(MomentumParams), vp]
     L.fp4_momentum_update.restype = C.c_int
+    L.fp4_adamw_update.argtypes = [vp, vp, i64, vp, vp, vp, vp, vp, C.POINTER(AdamwParams), vp]
+    L.fp4_adamw_update.restype = C.c_int
     L.fp4_momentum_decode.argtypes = [vp, vp, i64, i64, vp, vp]; L.fp4_momentum_decode.restype = C.c_int
     L.fp4_selftest_bounded_wait.argtypes = [vp, u32, vp]; L.fp4_selftest_bounded_wait.restype = C.c_int
     _lib = L
@@ -170,6 +179,18 @@ def fp4_momentum_update(G: torch.Tensor, codes: torch.Tensor, scales: torch.Tens
                                               M_out.data_ptr() if M_out is not None else None,
                                               hist.data_ptr() if hist is not None else None, C.byref(prm),
                                               _stream(stream)), "fp4_momentum_update")
+
+
+def fp4_adamw_update(W: torch.Tensor, G: torch.Tensor, m_codes: torch.Tensor, m_scales: torch.Tensor,
+                     v_codes: torch.Tensor, v_scales: torch.Tensor, v_means: torch.Tensor, lr: float,
+                     beta1: float = 0.9, beta2: float = 0.95, eps: float = 1e-8, weight_decay: float = 0.1,
+                     step: int = 1, flags: int = 0, seed: int = 0, stream=None) -> None:
+    """One packed AdamW step in place on BF16 weights W with BF16 gradients G (flat, a multiple of
+    256 elements) and both moments in their NVFP4 states."""
+    prm = AdamwParams(lr, beta1, beta2, eps, weight_decay, step, flags, 0, seed)
+    _check(load_library().fp4_adamw_update(W.data_ptr(), G.data_ptr(), W.numel(), m_codes.data_ptr(),
+                                           m_scales.data_ptr(), v_codes.data_ptr(), v_scales.data_ptr(),
+                                           v_means.data_ptr(), C.byref(prm), _stream(stream)), "fp4_adamw_update")
 
 
 def fp4_momentum_decode(codes: torch.Tensor, scales: torch.Tensor, M_out: torch.Tensor, stream=None) -> None:

@@ -8,8 +8,8 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libfp4root.so")
-SOURCES = ["fp4_quantize.cu", "fp4_prologue.cu", "fp4_gemm.cu", "fp4_gemm2.cu", "fp4_momentum.cu", "fp4_root_ns.cu"]
-HEADERS = ["fp4_common.cuh", "fp4_kernels.h", "fp4_gemm_common.cuh", os.path.join("..", "..", "include", "fp4root.h")]
+SOURCES = ["fp4_quantize.cu", "fp4_prologue.cu", "fp4_gemm.cu", "fp4_gemm2.cu", "fp4_momentum.cu", "fp4_adamw.cu", "fp4_root_ns.cu"]
+HEADERS = ["fp4_common.cuh", "fp4_kernels.h", "fp4_gemm_common.cuh", "fp4_state.cuh", os.path.join("..", "..", "include", "fp4root.h")]
 
 
 def _nvcc() -> str:

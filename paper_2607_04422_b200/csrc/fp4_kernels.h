@@ -109,6 +109,16 @@ void count_launches(int n);
 cudaError_t launch_momentum_update(const float* G, int64_t rows, int64_t cols, float mu, float g_scale, bool sr,
                                    uint64_t seed, uint8_t* codes, uint16_t* scales, float* M_out, uint32_t* hist,
                                    int sms, cudaStream_t st);
+// Packed AdamW step on NVFP4 moment states (fp4_adamw.cu).  The constants are derived on the host
+// in a fixed way (adamw_consts) and passed by value.
+struct AdamwConsts {
+  float b1, b2, omb1, omb2, eps, rsb2, step_size, decay;
+  uint64_t seed;
+};
+AdamwConsts adamw_consts(float lr, float beta1, float beta2, float eps, float weight_decay, int step, uint64_t seed);
+cudaError_t launch_adamw_update(uint16_t* W, const uint16_t* G, int64_t n, const AdamwConsts& k, bool sr,
+                                uint8_t* m_codes, uint16_t* m_scales, uint8_t* v_codes, uint16_t* v_scales,
+                                uint16_t* v_means, cudaStream_t st);
 cudaError_t launch_momentum_decode(const uint8_t* codes, const uint16_t* scales, int64_t rows, int64_t cols,
                                    float* M_out, int sms, cudaStream_t st);
 struct ProfScope {

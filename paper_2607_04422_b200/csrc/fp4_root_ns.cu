@@ -534,6 +534,27 @@ fp4_status fp4_momentum_update(const float* G, int64_t rows, int64_t cols, uint8
              : FP4_ERR_CUDA;
 }
 
+fp4_status fp4_adamw_update(uint16_t* W, const uint16_t* G, int64_t n, uint8_t* m_codes, uint16_t* m_scales,
+                            uint8_t* v_codes, uint16_t* v_scales, uint16_t* v_means,
+                            const fp4_adamw_params* params, cudaStream_t stream) {
+  if (!W || !G || !m_codes || !m_scales || !v_codes || !v_scales || !v_means || !params) return FP4_ERR_INVALID_ARG;
+  if ((params->flags & ~FP4_MOM_FLAG_SR) || params->step < 1) return FP4_ERR_INVALID_ARG;
+  if (n <= 0 || (n & 255)) return FP4_ERR_SHAPE;
+  if (!aligned(W, 32) || !aligned(G, 32) || !aligned(m_codes, 16) || !aligned(m_scales, 16) ||
+      !aligned(v_codes, 16) || !aligned(v_scales, 16) || !aligned(v_means, 16))
+    return FP4_ERR_ALIGNMENT;
+  const DeviceInfo* d;
+  fp4_status rc = check_common(&d);
+  if (rc != FP4_OK) return rc;
+  ProfScope ps(FP4_PROF_ADAMW, stream);
+  const AdamwConsts k = adamw_consts(params->lr, params->beta1, params->beta2, params->eps, params->weight_decay,
+                                     params->step, params->seed);
+  return launch_adamw_update(W, G, n, k, (params->flags & FP4_MOM_FLAG_SR) != 0, m_codes, m_scales, v_codes, v_scales,
+                             v_means, stream) == cudaSuccess
+             ? FP4_OK
+             : FP4_ERR_CUDA;
+}
+
 fp4_status fp4_momentum_decode(const uint8_t* codes, const uint16_t* scales, int64_t rows, int64_t cols,
                                float* M_out, cudaStream_t stream) {
   if (!codes || !scales || !M_out) return FP4_ERR_INVALID_ARG;

@@ -1,0 +1,162 @@
+// Device helpers shared by the kernels that keep optimiser moments in NVFP4 states (Section 3.3):
+// the fixed 16-point Hadamard transform on register pairs, the two-candidate (4/6) block
+// encoding with BF16 scales, hardware stochastic rounding, and 256-bit global accesses.
+#pragma once
+
+#include "fp4_common.cuh"
+
+namespace fp4 {
+
+__device__ __forceinline__ uint64_t splitmix64_at(uint64_t seed, uint64_t idx) {
+  uint64_t z = seed + 0x9E3779B97F4A7C15ull * (idx + 1);
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  return z ^ (z >> 31);
+}
+
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+
+// v <- v H_16 / 4, the natural-order butterfly of hadamard16 with no signs: the stride-1 stage on
+// scalars, the strides 2, 4, 8 and the factor 1/4 on packed pairs (v[2k], v[2k+1]); every lane
+// is the same single rounded operation as in the scalar form.
+__device__ __forceinline__ void hadamard16_pairs(float (&v)[16]) {
+  uint64_t p[8];
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    const float a = v[2 * k], b = v[2 * k + 1];
+    p[k] = pack2(__fadd_rn(a, b), __fsub_rn(a, b));
+  }
+#pragma unroll
+  for (int h = 1; h < 8; h *= 2) {
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      if ((k & h) == 0) {
+        const uint64_t a = p[k], b = p[k + h];
+        p[k] = add2(a, b);
+        p[k + h] = sub2(a, b);
+      }
+    }
+  }
+  const uint64_t q = pack2(0.25f, 0.25f);
+#pragma unroll
+  for (int k = 0; k < 8; ++k) unpack2(mul2(p[k], q), v[2 * k], v[2 * k + 1]);
+}
+
+// Nearest-rounding codes of one transformed block for the block scale d; returns the sum of the
+// squared FP32 errors in element order.  Products are taken two at a time; every subtraction
+// and every addition of the error sum stays a scalar operation, so none can fuse with a product.
+__device__ __forceinline__ float mom_encode_rtn(const float (&h)[16], float d, uint32_t& lo, uint32_t& hi) {
+  lo = 0; hi = 0;
+  float err = 0.0f;
+  if (d == 0.0f) {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) err = __fadd_rn(err, __fmul_rn(h[i], h[i]));
+    return err;
+  }
+  const float rcp = __frcp_rn(d);
+  const uint64_t rcp2 = pack2(rcp, rcp), d2 = pack2(d, d);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    float y0, y1, p0, p1, s0, s1;
+    unpack2(mul2(pack2(h[2 * i], h[2 * i + 1]), rcp2), y0, y1);
+    const uint32_t byte = cvt_e2m1x2(y0, y1);
+    const float2 q = e2m1x2_to_float2(byte);
+    unpack2(mul2(pack2(q.x, q.y), d2), p0, p1);
+    const float d0 = __fsub_rn(h[2 * i], p0), d1 = __fsub_rn(h[2 * i + 1], p1);
+    const uint64_t dd = pack2(d0, d1);
+    unpack2(mul2(dd, dd), s0, s1);
+    err = __fadd_rn(err, s0);
+    err = __fadd_rn(err, s1);
+    if (i < 4) lo |= byte << (8 * i); else hi |= byte << (8 * (i - 4));
+  }
+  return err;
+}
+
+// Stochastic rounding of four values onto the E2M1 grid with the conversion instruction of
+// sm_100a; the result holds v0 in bits 3:0 ... v3 in bits 15:12.  Measured behaviour of the
+// instruction: with lo <= |v| < hi the neighbouring grid values and f = floor(65536 (|v| - lo) /
+// (hi - lo)), v goes to hi when f + r >= 65536, where the 16 random bits r of the four values
+// come from the bytes b3 b2 b1 b0 of the random word as
+//   v0: b2 b0     v1: the same 16 bits in reverse order     v2: b3 b1     v3: those reversed.
+// `w` is the word in the plain form (v0: low half, v2: high half), permuted here.
+__device__ __forceinline__ uint32_t cvt_rs_e2m1x4(float v0, float v1, float v2, float v3, uint32_t w) {
+  const uint32_t rbits = __byte_perm(w, 0u, 0x3120);  // b0, b2 <- low half; b1, b3 <- high half
+  uint32_t r;
+  asm("{\n\t.reg .b16 t;\n\tcvt.rs.satfinite.e2m1x4.f32 t, {%1, %2, %3, %4}, %5;\n\tcvt.u32.u16 %0, t;\n\t}"
+      : "=r"(r)
+      : "f"(v3), "f"(v2), "f"(v1), "f"(v0), "r"(rbits));
+  return r;
+}
+
+__device__ __forceinline__ void mom_decode(uint2 c, uint32_t scale_bits, float (&v)[16]) {
+  const float d = __uint_as_float(scale_bits << 16);
+  const uint64_t d2 = pack2(d, d);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const uint32_t byte = ((i < 4 ? c.x : c.y) >> (8 * (i & 3))) & 0xFFu;
+    const float2 q = e2m1x2_to_float2(byte);
+    unpack2(mul2(pack2(q.x, q.y), d2), v[2 * i], v[2 * i + 1]);
+  }
+  hadamard16_pairs(v);
+}
+
+// Encodes m (destroyed); `first` is the matrix index of the block's first element.
+template <bool SR>
+__device__ __forceinline__ void mom_encode(float (&h)[16], uint64_t seed, uint64_t first, uint2& c,
+                                           uint32_t& scale_bits) {
+  hadamard16_pairs(h);
+  float amax = 0.0f;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) amax = fmaxf(amax, fabsf(h[i]));
+  const uint32_t w = cvt_bf16x2(__fdiv_rn(amax, 6.0f), __fdiv_rn(amax, 4.0f));
+  const float d6 = bf16_lo(w), d4 = bf16_hi(w);
+  uint32_t lo, hi, lo4, hi4;
+  const float err6 = mom_encode_rtn(h, d6, lo, hi);
+  const float err4 = mom_encode_rtn(h, d4, lo4, hi4);
+  float d = d6;
+  scale_bits = w & 0xFFFFu;
+  if (err4 < err6) { d = d4; scale_bits = w >> 16; lo = lo4; hi = hi4; }
+  if (SR && d != 0.0f) {
+    // one generator output per 8 elements of the matrix: its low word for the first four
+    const float rcp = __frcp_rn(d);
+    const uint64_t z0 = splitmix64_at(seed, first >> 3), z1 = splitmix64_at(seed, (first >> 3) + 1);
+    const uint32_t c0 = cvt_rs_e2m1x4(__fmul_rn(h[0], rcp), __fmul_rn(h[1], rcp), __fmul_rn(h[2], rcp),
+                                      __fmul_rn(h[3], rcp), (uint32_t)z0);
+    const uint32_t c1 = cvt_rs_e2m1x4(__fmul_rn(h[4], rcp), __fmul_rn(h[5], rcp), __fmul_rn(h[6], rcp),
+                                      __fmul_rn(h[7], rcp), (uint32_t)(z0 >> 32));
+    const uint32_t c2 = cvt_rs_e2m1x4(__fmul_rn(h[8], rcp), __fmul_rn(h[9], rcp), __fmul_rn(h[10], rcp),
+                                      __fmul_rn(h[11], rcp), (uint32_t)z1);
+    const uint32_t c3 = cvt_rs_e2m1x4(__fmul_rn(h[12], rcp), __fmul_rn(h[13], rcp), __fmul_rn(h[14], rcp),
+                                      __fmul_rn(h[15], rcp), (uint32_t)(z1 >> 32));
+    lo = c0 | (c1 << 16);
+    hi = c2 | (c3 << 16);
+  }
+  c = make_uint2(lo, hi);
+}
+
+// 256-bit global accesses (32-byte aligned): a thread moves its block of 16 floats as two full
+// 32-byte sectors, so no sector is touched by two instructions -- with 128-bit pieces at a
+// 64-byte lane stride every sector is looked up twice on loads and written as two partial
+// sectors on stores.
+__device__ __forceinline__ void ldg_f32x8(const float* p, float* v) {
+  asm volatile("ld.global.nc.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+               : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7])
+               : "l"(p));
+}
+__device__ __forceinline__ void stg_f32x8(float* p, const float* v) {
+  asm volatile("st.global.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "f"(v[0]), "f"(v[1]), "f"(v[2]),
+               "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7])
+               : "memory");
+}
+
+
+}  // namespace fp4

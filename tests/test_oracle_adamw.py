@@ -101,7 +101,7 @@ def test_pipeline_beats_direct_nvfp4_on_a_heavy_tailed_second_moment():
     sq_pipe = np.linalg.norm(np.sqrt(oracle.v_decode(c, s, m)) - np.sqrt(v)) / np.linalg.norm(np.sqrt(v))
     sq_direct = np.linalg.norm(np.sqrt(oracle.dequantize(qc, qs, sg)).ravel() - np.sqrt(v)) / np.linalg.norm(np.sqrt(v))
     assert sq_pipe < 0.75 * sq_direct, (sq_pipe, sq_direct)
-    assert err_pipe < 1.6 * err_direct, (err_pipe, err_direct)
+    assert err_pipe < 0.7 * err_direct, (err_pipe, err_direct)   # the paper: 0.0116 -> 0.0053 on its states
 
 
 def test_first_step_closed_form():
