@@ -24,7 +24,28 @@ def main():
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--quantize-only", action="store_true", help="time fp4_quantize instead of the NS step")
     ap.add_argument("--momentum", choices=["rtn", "sr"], help="time fp4_momentum_update instead of the NS step")
+    ap.add_argument("--adamw", choices=["rtn", "sr"], help="time fp4_adamw_update on m*n BF16 parameters instead")
     a = ap.parse_args()
+    if a.adamw:
+        n = a.m * a.n
+        gen = torch.Generator(device="cuda").manual_seed(a.seed)
+        W = (torch.randn(n, generator=gen, device="cuda") * 0.05).to(torch.bfloat16)
+        Gb = (torch.randn(n, generator=gen, device="cuda") * 1e-2).to(torch.bfloat16)
+        mc, vc = (torch.zeros(n // 2, dtype=torch.uint8, device="cuda") for _ in range(2))
+        ms, vs = (torch.zeros(n // 16, dtype=torch.int16, device="cuda") for _ in range(2))
+        vm = torch.zeros(n // 256, dtype=torch.int16, device="cuda")
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        times = []
+        for t in range(1, a.reps + 1):
+            e0.record()
+            fp4.fp4_adamw_update(W, Gb, mc, ms, vc, vs, vm, lr=1e-3, step=t,
+                                 flags=fp4.FP4_MOM_FLAG_SR if a.adamw == "sr" else 0, seed=t)
+            e1.record()
+            torch.cuda.synchronize()
+            times.append(e0.elapsed_time(e1))
+        print(json.dumps({"case": "fp4_adamw_update", "mode": a.adamw, "params": n, "ms": times,
+                          "gbs_best": n * 8.515625 / min(times) / 1e6}))
+        return
     G = torch.from_numpy(workloads.gradient_like(a.m, a.n, seed=a.seed)).cuda()
     stream = torch.cuda.current_stream()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
