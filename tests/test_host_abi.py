@@ -76,6 +76,32 @@ def test_argument_validation_happens_before_any_device_work():
     assert lib.fp4_root_ns(p, p, 128, 128, 5, None, p, 16, None) == 4             # workspace
     assert lib.fp4_quantize(p, 128, 120, p, p, p, 0, None) == 2
     assert lib.fp4_gemm_nt(p, p, 1.0, p, p, 1.0, 128, 128, 64, p, None, None) == 2
+    # the optimiser-state entry points
+    mp = binding.MomentumParams(0.9, 1.0, 0, 0, 0)
+    assert lib.fp4_momentum_update(None, 16, 16, p, p, None, None, ctypes.byref(mp), None) == 1   # null input
+    assert lib.fp4_momentum_update(p, 16, 24, p, p, None, None, ctypes.byref(mp), None) == 2      # shape
+    assert lib.fp4_momentum_update(p + 16, 16, 16, p, p, None, None, ctypes.byref(mp), None) == 3  # 32-byte rule
+    bad = binding.MomentumParams(0.9, 1.0, 8, 0, 0)
+    assert lib.fp4_momentum_update(p, 16, 16, p, p, None, None, ctypes.byref(bad), None) == 1     # unknown flag
+    assert lib.fp4_momentum_decode(p, p, 16, 16, None, None) == 1
+    ap = binding.AdamwParams(1e-3, 0.9, 0.95, 1e-8, 0.1, 1, 0, 0, 0)
+    assert lib.fp4_adamw_update(p, p, 384, p, p, p, p, p, ctypes.byref(ap), None) == 2            # not a multiple of 256
+    assert lib.fp4_adamw_update(p + 16, p, 256, p, p, p, p, p, ctypes.byref(ap), None) == 3
+    ap0 = binding.AdamwParams(1e-3, 0.9, 0.95, 1e-8, 0.1, 0, 0, 0, 0)
+    assert lib.fp4_adamw_update(p, p, 256, p, p, p, p, p, ctypes.byref(ap0), None) == 1           # step < 1
+
+
+def test_no_gpu_on_the_optimiser_state_entry_points():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("this check is for machines without a GPU")
+    lib = fp4.load_library()
+    buf = (ctypes.c_uint8 * (1 << 16))()
+    p = (ctypes.addressof(buf) + 1023) // 1024 * 1024
+    mp = binding.MomentumParams(0.9, 1.0, 0, 0, 0)
+    assert lib.fp4_momentum_update(p, 16, 16, p, p, None, None, ctypes.byref(mp), None) in (5, 6)
+    ap = binding.AdamwParams(1e-3, 0.9, 0.95, 1e-8, 0.1, 1, 0, 0, 0)
+    assert lib.fp4_adamw_update(p, p, 256, p, p, p, p, p, ctypes.byref(ap), None) in (5, 6)
 
 
 def test_no_gpu_means_an_error_not_a_fallback():
