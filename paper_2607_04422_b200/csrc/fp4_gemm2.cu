@@ -189,7 +189,9 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
   const int pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
   const GemmProblem* probs = table ? table : &single;
   // args.tiles_m / tiles_n count 256 x 256 tiles here
-  const int tiles_per_problem = args.symmetric ? args.tiles_n * (args.tiles_n + 1) / 2 : args.tiles_m * args.tiles_n;
+  // only the two symmetric products are ever launched with triangle tiles: a compile-time fact for the others
+  const bool sym = (MODE == kG1 || MODE == kG2) && args.symmetric != 0;
+  const int tiles_per_problem = sym ? args.tiles_n * (args.tiles_n + 1) / 2 : args.tiles_m * args.tiles_n;
   const int num_tiles = tiles_per_problem * args.num_problems;
   const int num_kb = args.K / BK;
   constexpr bool HAS_AUX = (MODE == kG2 || MODE == kG3);
@@ -224,7 +226,7 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
       int st = 0; uint32_t ph = 0; bool ok = true;
       for (int t = pair; t < num_tiles && ok; t += num_pairs) {
         int p, ti, tj;
-        decode_tile(t, args, tiles_per_problem, p, ti, tj);
+        decode_tile(t, args, tiles_per_problem, p, ti, tj, sym);
         const GemmProblem* pr = probs + p;
         const int arow = ti * PM + (int)rank * BM;   // this CTA's rows of the row operand
         const int brow = tj * PN + (int)rank * BM;   // this CTA's half of the column operand
@@ -300,14 +302,14 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
           chunk_slot(seq, h, i, b, use);
           if (!mbar_try_wait(&bars->slot_free[b], (use & 1) ^ 1)) continue;
           if (seq_dec[h] != seq) {
-            decode_tile(pair + (int)seq * num_pairs, args, tiles_per_problem, pp[h], tis[h], tjs[h]);
+            decode_tile(pair + (int)seq * num_pairs, args, tiles_per_problem, pp[h], tis[h], tjs[h], sym);
             seq_dec[h] = seq;
           }
           const GemmProblem* pr = probs + pp[h];
           const int bi = tis[h] * 2 + (int)rank;
           const int c = team_chunk((int)(seq & 1), h, i);
           const int bj = tjs[h] * 2 + c / 8;
-          if (args.symmetric && bj < bi) {
+          if (sym && bj < bi) {
             // a 128 x 128 block below the diagonal: nothing to combine, the slot is passed on empty
             mbar_arrive(&bars->aux_full[b]);
           } else {
@@ -364,13 +366,13 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
           chunk_slot(seq, h, i, b, use);
           if (!mbar_try_wait(&bars->v_ready[b], use & 1)) continue;
           if (seq_dec[h] != seq) {
-            decode_tile(pair + (int)seq * num_pairs, args, tiles_per_problem, pp[h], tis[h], tjs[h]);
+            decode_tile(pair + (int)seq * num_pairs, args, tiles_per_problem, pp[h], tis[h], tjs[h], sym);
             seq_dec[h] = seq;
           }
           const GemmProblem* pr = probs + pp[h];
           const int bi = tis[h] * 2 + (int)rank;
           const int c = team_chunk((int)(seq & 1), h, i);
-          const bool below = args.symmetric && (tjs[h] * 2 + c / 8) < bi;
+          const bool below = sym && (tjs[h] * 2 + c / 8) < bi;
           // a chunk that starts outside the stored matrix (zero padding of the work shape) is dropped
           const bool inside = tjs[h] * PN + c * CHUNK < pr->out_cols && bi * BM < pr->out_rows;
           if (STORE_F32 && !below && inside) {
@@ -449,7 +451,7 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
     bool ok = true;
     for (int t = pair; t < num_tiles && ok; t += num_pairs, ++seq) {
       int p, ti, tj;
-      decode_tile(t, args, tiles_per_problem, p, ti, tj);
+      decode_tile(t, args, tiles_per_problem, p, ti, tj, sym);
       if (p != cur_p) {
         if ((MODE == kG1 || MODE == kG3) && cur_p >= 0) {
 #pragma unroll
@@ -475,8 +477,8 @@ k_gemm_pair(const __grid_constant__ GemmProblem single, const GemmProblem* __res
       }
       const int bi = ti * 2 + (int)rank;                               // 128-row block of this CTA
       const int bj = tj * 2 + (team * TEAM_CHUNKS * CHUNK) / 128;      // 128-column block of this team's chunks
-      const bool below = args.symmetric && bj < bi;                    // redundant block of a diagonal tile
-      const bool mirror = do_q && !below && (MODE == kG3 || (args.symmetric && bi != bj));
+      const bool below = sym && bj < bi;                    // redundant block of a diagonal tile
+      const bool mirror = do_q && !below && (MODE == kG3 || (sym && bi != bj));
       const bool hout = BH && STORE_F32 && MODE != kPlain && args.out_h == 1 && !below;  // result stored as BF16
       const bool stage = !below && ((STORE_F32 && !hout) || mirror);
       const int par = (int)(seq & 1);

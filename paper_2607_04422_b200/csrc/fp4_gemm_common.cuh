@@ -37,11 +37,11 @@ __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatil
 
 // tile index of a launch -> (problem, tile row, tile column)
 __device__ __forceinline__ void decode_tile(int t, const GemmLaunch& L, int tiles_per_problem, int& p, int& ti,
-                                            int& tj) {
+                                            int& tj, bool sym) {
   p = t / tiles_per_problem;
   t -= p * tiles_per_problem;
   const int tiles_n = L.tiles_n;
-  if (!L.symmetric) {
+  if (!sym) {
     ti = t / tiles_n;
     tj = t - ti * tiles_n;
   } else {
@@ -50,6 +50,10 @@ __device__ __forceinline__ void decode_tile(int t, const GemmLaunch& L, int tile
     ti = row;
     tj = row + rem;
   }
+}
+__device__ __forceinline__ void decode_tile(int t, const GemmLaunch& L, int tiles_per_problem, int& p, int& ti,
+                                            int& tj) {
+  decode_tile(t, L, tiles_per_problem, p, ti, tj, L.symmetric != 0);
 }
 
 // Per-call scalars of an epilogue: the factor that turns the accumulator into the
