@@ -98,6 +98,12 @@ __device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
   asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
   return d;
 }
+// d = a * b + c per lane, one rounding (what the scalar fused multiply-add gives)
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
 // Four FP32 -> two bytes of E2M1 codes (a in bits 3:0, b in 7:4, c in 11:8, d in 15:12).
 __device__ __forceinline__ uint32_t cvt_e2m1x4(float a, float b, float c, float d) {
   uint32_t r;

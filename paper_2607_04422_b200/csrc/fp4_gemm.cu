@@ -102,14 +102,14 @@ static_assert(sizeof(Barriers) <= 512, "barrier block");
 
 template <int MODE, bool PF>
 __global__ void __launch_bounds__(NTHREADS, 1)
-k_gemm(const __grid_constant__ GemmProblem single, const GemmProblem* __restrict__ table, const GemmLaunch args) {
+k_gemm(const __grid_constant__ ProblemPack pack, const __grid_constant__ GemmLaunch args) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   Barriers* bars = reinterpret_cast<Barriers*>(smem + OFF_BAR);
   volatile uint32_t* abort_flag = &bars->abort_flag;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const GemmProblem* probs = table ? table : &single;
+  const GemmProblem* probs = pack.p;
   const int tiles_per_problem = args.symmetric ? args.tiles_n * (args.tiles_n + 1) / 2 : args.tiles_m * args.tiles_n;
   const int num_tiles = tiles_per_problem * args.num_problems;
 #ifdef FP4_DEBUG_ONE_KBLOCK
@@ -480,15 +480,13 @@ k_gemm(const __grid_constant__ GemmProblem single, const GemmProblem* __restrict
 }
 
 template <int MODE, bool PF>
-cudaError_t launch_mode(const GemmProblem* single, const GemmProblem* table, const GemmLaunch& L, int sms,
-                        cudaStream_t st) {
+cudaError_t launch_mode(const ProblemPack& pack, const GemmLaunch& L, int sms, cudaStream_t st) {
   const int tpp = L.symmetric ? L.tiles_n * (L.tiles_n + 1) / 2 : L.tiles_m * L.tiles_n;
   const int num_tiles = tpp * L.num_problems;
   int grid = sms;
   if (grid > num_tiles) grid = num_tiles;
   count_launches(1);
-  static const GemmProblem kNone = {};
-  k_gemm<MODE, PF><<<grid, NTHREADS, SMEM_BYTES, st>>>(single ? *single : kNone, table, L);
+  k_gemm<MODE, PF><<<grid, NTHREADS, SMEM_BYTES, st>>>(pack, L);
   return cudaGetLastError();
 }
 
@@ -508,15 +506,14 @@ cudaError_t gemm_set_attributes() {
   return cudaSuccess;
 }
 
-cudaError_t launch_gemm(GemmMode mode, const GemmProblem* single, const GemmProblem* table, const GemmLaunch& launch,
-                        int sms, cudaStream_t st) {
-  if ((single == nullptr) == (table == nullptr)) return cudaErrorInvalidValue;
+cudaError_t launch_gemm(GemmMode mode, const ProblemPack& pack, const GemmLaunch& launch, int sms, cudaStream_t st) {
+  if (launch.num_problems < 1 || launch.num_problems > kPackMax) return cudaErrorInvalidValue;
   const bool pf = launch.q.rht || launch.q.four_six;
   switch (mode) {
-    case kPlain: return launch_mode<kPlain, false>(single, table, launch, sms, st);
-    case kG1: return pf ? launch_mode<kG1, true>(single, table, launch, sms, st) : launch_mode<kG1, false>(single, table, launch, sms, st);
-    case kG2: return pf ? launch_mode<kG2, true>(single, table, launch, sms, st) : launch_mode<kG2, false>(single, table, launch, sms, st);
-    default: return pf ? launch_mode<kG3, true>(single, table, launch, sms, st) : launch_mode<kG3, false>(single, table, launch, sms, st);
+    case kPlain: return launch_mode<kPlain, false>(pack, launch, sms, st);
+    case kG1: return pf ? launch_mode<kG1, true>(pack, launch, sms, st) : launch_mode<kG1, false>(pack, launch, sms, st);
+    case kG2: return pf ? launch_mode<kG2, true>(pack, launch, sms, st) : launch_mode<kG2, false>(pack, launch, sms, st);
+    default: return pf ? launch_mode<kG3, true>(pack, launch, sms, st) : launch_mode<kG3, false>(pack, launch, sms, st);
   }
 }
 

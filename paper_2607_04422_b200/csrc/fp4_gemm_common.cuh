@@ -35,6 +35,47 @@ __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatil
   return wait_slow(bar, parity, abort_flag);
 }
 
+// The same wait for callers that do not branch on the outcome: when a wait gives up (its own
+// time-out, or another thread of the CTA gave up before) the abort flag is set and every later
+// wait of the CTA falls through at once, so the kernel runs to its end on whatever data it has
+// and the host reads FP4_ERR_DEVICE_TIMEOUT from the status word.  The polls carry a suspend-time
+// hint: the thread sleeps in hardware until the phase completes instead of spinning.
+__device__ __forceinline__ bool mbar_try_wait_hint(uint32_t bar_addr, uint32_t parity, uint32_t hint_ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar_addr), "r"(parity), "r"(hint_ns)
+      : "memory");
+  return ok != 0;
+}
+static __device__ __noinline__ void wait_slow_abort(uint32_t bar_addr, uint32_t parity, volatile uint32_t* abort_flag) {
+  const uint64_t t0 = globaltimer_ns();
+  for (;;) {
+    if (*abort_flag) return;
+    for (int i = 0; i < 64; ++i)
+      if (mbar_try_wait_hint(bar_addr, parity, 4000u)) return;
+    if (globaltimer_ns() - t0 > kWaitLimitNs) {
+      *abort_flag = 1;
+      return;
+    }
+  }
+}
+__device__ __forceinline__ void wait_or_abort(uint32_t bar_addr, uint32_t parity, volatile uint32_t* abort_flag) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar_addr), "r"(parity)
+      : "memory");
+  if (!ok) wait_slow_abort(bar_addr, parity, abort_flag);
+}
+__device__ __forceinline__ void wait_or_abort(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag) {
+  wait_or_abort(smem_u32(bar), parity, abort_flag);
+}
+
 // tile index of a launch -> (problem, tile row, tile column)
 __device__ __forceinline__ void decode_tile(int t, const GemmLaunch& L, int tiles_per_problem, int& p, int& ti,
                                             int& tj, bool sym) {

@@ -64,10 +64,13 @@ enum GemmMode : int {
 // problem, in the kernel's parameter space).
 struct alignas(64) GemmProblem {
   CUtensorMap tmA, tmB;      // NVFP4 codes of the row and the column operand
-  CUtensorMap tmAux, tmOut;  // FP32 tile combined in the epilogue / FP32 result
+  CUtensorMap tmAux, tmOut;  // FP32 tile combined in the epilogue / FP32 result (box: 16 columns x 128 rows in
+                             // the single-CTA kernel, 16 x 32 - one epilogue warp's block - in the CTA-pair kernel)
   CUtensorMap tmSfa, tmSfb;  // scale atoms of the two operands as 2-D maps (CTA-pair kernel)
   CUtensorMap tmH;           // BF16 storage: the 2-byte tensor this stage reads its tile from and / or stores its
                              // result to (A for G1 / G2, X for G3); box 16 columns x 32 rows, no swizzle
+  CUtensorMap tmRq, tmCq;    // CTA-pair kernel: byte maps over rq_codes (box 32 bytes x 32 rows) and cq_codes
+                             // (box 16 bytes x 64 rows), through which a warp stores the codes of its part of a tile
   const uint8_t* sfa;        // scale atoms of the row operand
   const uint8_t* sfb;        // scale atoms of the column operand
   float* scalars;            // workspace scalars of this matrix (device)
@@ -80,6 +83,12 @@ struct alignas(64) GemmProblem {
   void* out_direct;          // out_h == 2: the FP32 tensor the epilogue warps store the rounded result to
   int64_t out_direct_ld;     //   (row-major, leading dimension in elements)
 };
+
+// The problems of one launch travel as a kernel parameter (descriptors in parameter space need no
+// proxy fence before TMA uses them, and nothing has to be written to device memory first).
+constexpr int kPackMax = 16;
+struct ProblemPack { GemmProblem p[kPackMax]; };
+static_assert(sizeof(ProblemPack) + 256 <= 32764, "kernel parameter space");
 
 // What all problems of a launch share.
 struct GemmLaunch {
@@ -96,6 +105,7 @@ struct GemmLaunch {
   int aux_h;           // the combined tile is read from tmH (BF16)
   int out_h;           // 0: FP32 result by TMA store; 1: rounded to BF16, staged and stored through tmH (CTA-pair
                        // kernel); 2: rounded to BF16, stored as FP32 by the epilogue warps (single-CTA kernel)
+  int dry_operands;    // kPlain, CTA-pair kernel: measurement of the tensor-pipe ceiling - no operand is fetched
   NsScalarIdx ix;
   uint32_t* status;
 };
@@ -149,12 +159,10 @@ cudaError_t prologue_set_attributes();
 
 cudaError_t gemm_set_attributes();
 cudaError_t gemm_pair_set_attributes();
-cudaError_t launch_gemm_pair(GemmMode mode, const GemmProblem* single, const GemmProblem* table,
-                             const GemmLaunch& launch, int sms, cudaStream_t st);
+// pack: the launch.num_problems (<= kPackMax) problems of the launch
+cudaError_t launch_gemm_pair(GemmMode mode, const ProblemPack& pack, const GemmLaunch& launch, int sms,
+                             cudaStream_t st);
 int gemm_stage_k();  // elements of K per operand stage (the codes maps' box is this / 2 bytes wide)
-// single: the one problem of the launch (host copy, passed by value) when table is null;
-// table: device array of launch.num_problems problems.
-cudaError_t launch_gemm(GemmMode mode, const GemmProblem* single, const GemmProblem* table, const GemmLaunch& launch,
-                        int sms, cudaStream_t st);
+cudaError_t launch_gemm(GemmMode mode, const ProblemPack& pack, const GemmLaunch& launch, int sms, cudaStream_t st);
 
 }  // namespace fp4

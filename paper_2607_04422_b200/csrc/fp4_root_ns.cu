@@ -95,30 +95,44 @@ bool make_codes_map(const DeviceInfo* d, CUtensorMap* tm, const void* base, int6
                    CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
-// 2-D map over a row-major FP32 matrix: box = 16 columns x 128 rows, 64-byte swizzle.
-bool make_f32_map(const DeviceInfo* d, CUtensorMap* tm, const void* base, int64_t rows, int64_t cols) {
+// 2-D map over a row-major FP32 matrix: box = 16 columns x box_rows rows (128: a chunk of the single-CTA
+// kernel; 32: one epilogue warp's block in the CTA-pair kernel), 64-byte swizzle.
+bool make_f32_map(const DeviceInfo* d, CUtensorMap* tm, const void* base, int64_t rows, int64_t cols, int box_rows) {
   cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
   cuuint64_t strides[1] = {(cuuint64_t)cols * 4};
-  cuuint32_t box[2] = {16, 128};
+  cuuint32_t box[2] = {16, (cuuint32_t)box_rows};
   cuuint32_t estr[2] = {1, 1};
   return d->encode(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box, estr,
                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// 2-D map over a row-major BF16 matrix: box = 16 columns x 32 rows (32-byte rows), no swizzle: one box per
-// epilogue warp of a team, so that a warp's rows sit inside its own part of the chunk slot.
+// 2-D map over a row-major BF16 matrix: box = 16 columns x 32 rows (32-byte rows), no swizzle: the block of
+// one epilogue warp of the CTA-pair kernel.
 bool make_bf16_map(const DeviceInfo* d, CUtensorMap* tm, const void* base, int64_t rows, int64_t cols) {
   cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
   cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
-  cuuint32_t box[2] = {16, 128};
+  cuuint32_t box[2] = {16, 32};
   cuuint32_t estr[2] = {1, 1};
   return d->encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-constexpr int kDefaultMaxGroup = 16;
+// 2-D map over a row-major byte matrix (NVFP4 codes) for the stores of the CTA-pair kernel's epilogue
+// warps: box = box_bytes x box_rows, no swizzle.
+bool make_code_store_map(const DeviceInfo* d, CUtensorMap* tm, const void* base, int64_t rows, int64_t row_bytes,
+                         int box_bytes, int box_rows) {
+  cuuint64_t dims[2] = {(cuuint64_t)row_bytes, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)row_bytes};
+  cuuint32_t box[2] = {(cuuint32_t)box_bytes, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return d->encode(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+constexpr int kDefaultMaxGroup = kPackMax;
 
 // 2-D map over the scale atoms of a rows x K operand: one map row per 128-row block, 64-bit
 // elements, box = the atoms of one operand stage (256 elements = 2 KB), no swizzle.
@@ -133,14 +147,20 @@ bool make_sf_map(const DeviceInfo* d, CUtensorMap* tm, const void* base, int64_t
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// The CTA-pair kernel takes every product whose dimensions are all multiples of 256.
-cudaError_t launch_gemm_auto(GemmMode mode, const GemmProblem* single, const GemmProblem* table,
-                             const GemmLaunch& L, int sms, cudaStream_t st, bool force_single = false) {
+// The CTA-pair kernel takes every product whose dimensions are all multiples of 256 (tile counts in 128-blocks).
+// The descriptors of a problem are built for the kernel that runs it (pair_kernel decides both).
+bool pair_kernel(int64_t tiles_m, int64_t tiles_n, int64_t K, int sms, bool force_single = false) {
 #ifndef FP4_DISABLE_PAIR
-  if (!force_single && !(L.tiles_m & 1) && !(L.tiles_n & 1) && L.K % 256 == 0 && sms >= 2)
-    return launch_gemm_pair(mode, single, table, L, sms, st);
+  return !force_single && !(tiles_m & 1) && !(tiles_n & 1) && K % 256 == 0 && sms >= 2;
+#else
+  (void)tiles_m; (void)tiles_n; (void)K; (void)sms; (void)force_single;
+  return false;
 #endif
-  return launch_gemm(mode, single, table, L, sms, st);
+}
+cudaError_t launch_gemm_auto(GemmMode mode, const ProblemPack& pack, const GemmLaunch& L, int sms, cudaStream_t st,
+                             bool force_single = false) {
+  if (pair_kernel(L.tiles_m, L.tiles_n, L.K, sms, force_single)) return launch_gemm_pair(mode, pack, L, sms, st);
+  return launch_gemm(mode, pack, L, sms, st);
 }
 
 void default_params(fp4_ns_params* p) {
@@ -286,7 +306,11 @@ fp4_status prepare_matrix(const DeviceInfo* d, const float* G, float* out, int64
   if (steps == 0) return FP4_OK;
   float abc[3] = {p->a, p->b, p->c};
   if (std::isnan(p->a)) coeffs(m, n, abc);
-  CUtensorMap tm_qX, tm_qXt[2], tm_qA, tm_qB, tm_A, tm_X;
+  // which kernel runs each stage (rounded-FP32 storage is implemented by the single-CTA kernel only)
+  const bool fs = c->pl.bf16_mode == 2;
+  const bool pair1 = pair_kernel(s / 128, s / 128, l, d->sms, fs), pair2 = pair_kernel(s / 128, s / 128, s, d->sms, fs),
+             pair3 = pair_kernel(s / 128, l / 128, s, d->sms, fs);
+  CUtensorMap tm_qX, tm_qXt[2], tm_qA, tm_qB, tm_A1, tm_A2, tm_X;
   CUtensorMap sf_qX, sf_qXt[2], sf_qA, sf_qB;
   bool ok = make_sf_map(d, &sf_qX, ws + L.qX_scales, s, l) && make_sf_map(d, &sf_qXt[0], ws + L.qXt_scales[0], l, s) &&
             make_sf_map(d, &sf_qXt[1], ws + L.qXt_scales[1], l, s) && make_sf_map(d, &sf_qA, ws + L.qA_scales, s, s) &&
@@ -296,7 +320,19 @@ fp4_status prepare_matrix(const DeviceInfo* d, const float* G, float* out, int64
             make_codes_map(d, &tm_qXt[1], ws + L.qXt_codes[1], l, s / 2) &&
             make_codes_map(d, &tm_qA, ws + L.qA_codes, s, s / 2) &&
             make_codes_map(d, &tm_qB, ws + L.qB_codes, s, s / 2) &&
-            make_f32_map(d, &tm_A, ws + L.A, s, s) && make_f32_map(d, &tm_X, c->X, xr, xc);
+            make_f32_map(d, &tm_A1, ws + L.A, s, s, pair1 ? 32 : 128) &&
+            make_f32_map(d, &tm_A2, ws + L.A, s, s, pair2 ? 32 : 128) &&
+            make_f32_map(d, &tm_X, c->X, xr, xc, pair3 ? 32 : 128);
+  if (!ok) return FP4_ERR_CUDA;
+  // stores of the quantised outputs by the CTA-pair kernel's epilogue warps
+  CUtensorMap st_qA_r, st_qA_c, st_qB_r, st_qB_c, st_qX_r, st_qXt_c[2];
+  ok = make_code_store_map(d, &st_qA_r, ws + L.qA_codes, s, s / 2, 32, 32) &&
+       make_code_store_map(d, &st_qA_c, ws + L.qA_codes, s, s / 2, 16, 64) &&
+       make_code_store_map(d, &st_qB_r, ws + L.qB_codes, s, s / 2, 32, 32) &&
+       make_code_store_map(d, &st_qB_c, ws + L.qB_codes, s, s / 2, 16, 64) &&
+       make_code_store_map(d, &st_qX_r, ws + L.qX_codes, s, l / 2, 32, 32) &&
+       make_code_store_map(d, &st_qXt_c[0], ws + L.qXt_codes[0], l, s / 2, 16, 64) &&
+       make_code_store_map(d, &st_qXt_c[1], ws + L.qXt_codes[1], l, s / 2, 16, 64);
   if (!ok) return FP4_ERR_CUDA;
   GemmProblem base;
   memset(&base, 0, sizeof(base));
@@ -309,7 +345,8 @@ fp4_status prepare_matrix(const DeviceInfo* d, const float* G, float* out, int64
   if (bmode == 1 && (!make_bf16_map(d, &tm_Ah, ws + L.A, s, s) || !make_bf16_map(d, &tm_Xh, Xh, s, l))) return FP4_ERR_CUDA;
   // G1: A = qX qX^T (upper-triangle tiles), qA in both triangles
   c->g1 = base;
-  c->g1.tmA = c->g1.tmB = tm_qX; c->g1.tmAux = c->g1.tmOut = tm_A;
+  c->g1.tmA = c->g1.tmB = tm_qX; c->g1.tmAux = c->g1.tmOut = tm_A1;
+  c->g1.tmRq = st_qA_r; c->g1.tmCq = st_qA_c;
   c->g1.tmSfa = c->g1.tmSfb = sf_qX;
   c->g1.sfa = c->g1.sfb = ws + L.qX_scales;
   c->g1.rq_codes = c->g1.cq_codes = ws + L.qA_codes; c->g1.rq_sf = c->g1.cq_sf = ws + L.qA_scales;
@@ -317,7 +354,8 @@ fp4_status prepare_matrix(const DeviceInfo* d, const float* G, float* out, int64
   if (bmode == 2) { c->g1.out_direct = ws + L.A; c->g1.out_direct_ld = s; }   // A as rounded FP32
   // G2: B = bA + c qA qA^T, qB in both triangles
   c->g2 = base;
-  c->g2.tmA = c->g2.tmB = tm_qA; c->g2.tmAux = c->g2.tmOut = tm_A;
+  c->g2.tmA = c->g2.tmB = tm_qA; c->g2.tmAux = c->g2.tmOut = tm_A2;
+  c->g2.tmRq = st_qB_r; c->g2.tmCq = st_qB_c;
   c->g2.tmSfa = c->g2.tmSfb = sf_qA;
   c->g2.sfa = c->g2.sfb = ws + L.qA_scales;
   if (bmode == 1) c->g2.tmH = tm_Ah;
@@ -334,34 +372,24 @@ fp4_status prepare_matrix(const DeviceInfo* d, const float* G, float* out, int64
     g.sfa = ws + L.qB_scales; g.sfb = ws + L.qXt_scales[cur];
     g.rq_codes = ws + L.qX_codes; g.rq_sf = ws + L.qX_scales;
     g.cq_codes = ws + L.qXt_codes[cur ^ 1]; g.cq_sf = ws + L.qXt_scales[cur ^ 1];
+    g.tmRq = st_qX_r; g.tmCq = st_qXt_c[cur ^ 1];
   }
   c->g3_first = c->g3[0];
   if (!c->store_x0) {
     CUtensorMap tm_G;
-    if (!make_f32_map(d, &tm_G, G, c->pl.s0, c->pl.l0)) return FP4_ERR_CUDA;
+    if (!make_f32_map(d, &tm_G, G, c->pl.s0, c->pl.l0, pair3 ? 32 : 128)) return FP4_ERR_CUDA;
     c->g3_first.tmAux = tm_G;
     c->g3_first.aux_raw = 1;
   }
   return FP4_OK;
 }
 
-constexpr int kPackMax = 16;
-struct ProblemPack { GemmProblem p[kPackMax]; };
-
-// Copies problem descriptions from kernel parameters into a device table (the tables of a
-// batched call are filled this way so that the call stays asynchronous).
-__global__ void k_write_problems(GemmProblem* dst, const __grid_constant__ ProblemPack pack, int n) {
-  const uint4* src = reinterpret_cast<const uint4*>(&pack);
-  uint4* out = reinterpret_cast<uint4*>(dst);
-  const int words = n * (int)(sizeof(GemmProblem) / 16);
-  for (int i = threadIdx.x; i < words; i += blockDim.x) out[i] = src[i];
-}
-
 // Enqueue the whole step for a group of matrices of one shape (s, l): the prologue per matrix,
 // then every Newton-Schulz stage as one launch over all matrices of the group.
-// table: device memory for 5 * count problems (unused when count == 1).
+// count <= kPackMax: the problems of a launch travel as its parameter.
 fp4_status run_group(const DeviceInfo* d, MatrixCtx* mats, int count, int steps, const fp4_ns_params* p,
-                     uint32_t* status, GemmProblem* table, bool clear_first_status, cudaStream_t st) {
+                     uint32_t* status, bool clear_first_status, cudaStream_t st) {
+  if (count < 1 || count > kPackMax) return FP4_ERR_INVALID_ARG;
   const bool keep = (p->flags & FP4_FLAG_KEEP_OPERANDS) != 0;
   const NsPlan& pl0 = mats[0].pl;
   const int64_t s = pl0.s, l = pl0.l;
@@ -376,24 +404,13 @@ fp4_status run_group(const DeviceInfo* d, MatrixCtx* mats, int count, int steps,
       return FP4_ERR_CUDA;
   }
   if (steps > 0) {
-    const GemmProblem* tabs[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
-    if (count > 1) {
-      for (int kind = 0; kind < 5; ++kind) {
-        GemmProblem* dst = table + (size_t)kind * count;
-        tabs[kind] = dst;
-        for (int i0 = 0; i0 < count; i0 += kPackMax) {
-          ProblemPack pack;
-          const int nn = count - i0 < kPackMax ? count - i0 : kPackMax;
-          for (int j = 0; j < nn; ++j) {
-            const MatrixCtx& c = mats[i0 + j];
-            pack.p[j] = kind == 0 ? c.g1 : kind == 1 ? c.g2 : kind == 4 ? c.g3_first : c.g3[kind - 2];
-          }
-          for (int j = nn; j < kPackMax; ++j) pack.p[j] = pack.p[0];
-          count_launches(1);
-          k_write_problems<<<1, 128, 0, st>>>(dst + i0, pack, nn);
-        }
+    // the problems of the five kinds of launches: G1, G2, G3 reading qXt[0] / qXt[1], the first G3
+    std::vector<ProblemPack> packs(5);
+    for (int kind = 0; kind < 5; ++kind) {
+      for (int j = 0; j < kPackMax; ++j) {
+        const MatrixCtx& c = mats[j < count ? j : 0];
+        packs[(size_t)kind].p[j] = kind == 0 ? c.g1 : kind == 1 ? c.g2 : kind == 4 ? c.g3_first : c.g3[kind - 2];
       }
-      if (cudaGetLastError() != cudaSuccess) return FP4_ERR_CUDA;
     }
     GemmLaunch base;
     memset(&base, 0, sizeof(base));
@@ -414,7 +431,7 @@ fp4_status run_group(const DeviceInfo* d, MatrixCtx* mats, int count, int steps,
       L1.out_h = bmode;
       {
         ProfScope ps(FP4_PROF_G1, st);
-        if (launch_gemm_auto(kG1, count == 1 ? &mats[0].g1 : nullptr, tabs[0], L1, d->sms, st, fs) != cudaSuccess)
+        if (launch_gemm_auto(kG1, packs[0], L1, d->sms, st, fs) != cudaSuccess)
           return FP4_ERR_CUDA;
       }
       GemmLaunch L2 = L1;
@@ -423,7 +440,7 @@ fp4_status run_group(const DeviceInfo* d, MatrixCtx* mats, int count, int steps,
       L2.out_h = 0; L2.aux_h = bmode == 1;
       {
         ProfScope ps(FP4_PROF_G2, st);
-        if (launch_gemm_auto(kG2, count == 1 ? &mats[0].g2 : nullptr, tabs[1], L2, d->sms, st, fs) != cudaSuccess)
+        if (launch_gemm_auto(kG2, packs[1], L2, d->sms, st, fs) != cudaSuccess)
           return FP4_ERR_CUDA;
       }
       GemmLaunch L3 = base;
@@ -435,8 +452,7 @@ fp4_status run_group(const DeviceInfo* d, MatrixCtx* mats, int count, int steps,
       L3.out_h = last ? 0 : bmode;                 // the result itself is FP32
       {
         ProfScope ps(FP4_PROF_G3, st);
-        const GemmProblem* one = k == 0 ? &mats[0].g3_first : &mats[0].g3[cur];
-        if (launch_gemm_auto(kG3, count == 1 ? one : nullptr, k == 0 ? tabs[4] : tabs[2 + cur], L3, d->sms, st, fs) != cudaSuccess)
+        if (launch_gemm_auto(kG3, packs[k == 0 ? 4 : 2 + cur], L3, d->sms, st, fs) != cudaSuccess)
           return FP4_ERR_CUDA;
       }
     }
@@ -457,7 +473,7 @@ fp4_status run_one(const DeviceInfo* d, const float* G, float* out, int64_t m, i
   fp4_status rc = prepare_matrix(d, G, out, m, n, steps, p, ws, &c);
   if (rc != FP4_OK) return rc;
   if (p->top_hist) c.hist_top = p->top_hist[0];
-  return run_group(d, &c, 1, steps, p, reinterpret_cast<uint32_t*>(ws + c.pl.lay.header), nullptr, clear_status, st);
+  return run_group(d, &c, 1, steps, p, reinterpret_cast<uint32_t*>(ws + c.pl.lay.header), clear_status, st);
 }
 
 fp4_status check_common(const DeviceInfo** d) {
@@ -608,7 +624,7 @@ fp4_status fp4_root_ns(const float* G, float* out, int64_t m, int64_t n, int ste
 }
 
 // Batched workspace: one workspace per matrix (the stages of equal-shape matrices run in
-// lockstep, so none can be shared), then the problem tables.
+// lockstep, so none can be shared).
 size_t fp4_root_ns_batched_workspace_bytes(int count, const int64_t* m, const int64_t* n, int steps,
                                            uint32_t flags) {
   if (count <= 0 || !m || !n) return 0;
@@ -618,7 +634,6 @@ size_t fp4_root_ns_batched_workspace_bytes(int count, const int64_t* m, const in
     if (b == 0) return 0;
     need += align_up(b, 1024);
   }
-  need += align_up((size_t)5 * count * sizeof(GemmProblem), 1024);
   return need;
 }
 
@@ -651,14 +666,13 @@ fp4_status fp4_root_ns_batched(int count, const float* const* G, float* const* o
     if (p->top_hist) ctx[(size_t)i].hist_top = p->top_hist[i];
     off += align_up(ctx[(size_t)i].pl.lay.total, 1024);
   }
-  GemmProblem* table = reinterpret_cast<GemmProblem*>(base + off);
   uint32_t* status = reinterpret_cast<uint32_t*>(base);  // header of the first matrix
 
   // Matrices of one shape form a group whose stages run as single launches over all of
   // them (many tiles per launch: no idle SMs in a last partial wave, the two CTAs of an SM
   // fall out of step so that main loops and epilogues overlap).  A group is split when it
   // exceeds max_group matrices, which bounds the working set competing for L2.
-  const int cap = p->max_group > 0 ? (int)p->max_group : kDefaultMaxGroup;
+  const int cap = p->max_group > 0 && (int)p->max_group < kPackMax ? (int)p->max_group : kDefaultMaxGroup;
   std::vector<char> done((size_t)count, 0);
   std::vector<MatrixCtx> group;
   bool first = true;
@@ -672,7 +686,7 @@ fp4_status fp4_root_ns_batched(int count, const float* const* G, float* const* o
         done[(size_t)j] = 1;
       }
     }
-    rc = run_group(d, group.data(), (int)group.size(), steps, p, status, table, first, stream);
+    rc = run_group(d, group.data(), (int)group.size(), steps, p, status, first, stream);
     if (rc != FP4_OK) return rc;
     first = false;
   }
@@ -698,10 +712,11 @@ fp4_status fp4_gemm_nt(const uint8_t* a_codes, const uint8_t* a_scales, float a_
   const DeviceInfo* d;
   fp4_status rc = check_common(&d);
   if (rc != FP4_OK) return rc;
-  GemmProblem pr;
-  memset(&pr, 0, sizeof(pr));
+  ProblemPack pack;
+  memset(&pack, 0, sizeof(pack));
+  GemmProblem& pr = pack.p[0];
   if (!make_codes_map(d, &pr.tmA, a_codes, M, K / 2) || !make_codes_map(d, &pr.tmB, b_codes, N, K / 2) ||
-      !make_f32_map(d, &pr.tmOut, D, M, N) || !make_sf_map(d, &pr.tmSfa, a_scales, M, K) ||
+      !make_f32_map(d, &pr.tmOut, D, M, N, pair_kernel(M / 128, N / 128, K, d->sms) ? 32 : 128) || !make_sf_map(d, &pr.tmSfa, a_scales, M, K) ||
       !make_sf_map(d, &pr.tmSfb, b_scales, N, K))
     return FP4_ERR_CUDA;
   pr.tmAux = pr.tmOut;
@@ -713,7 +728,7 @@ fp4_status fp4_gemm_nt(const uint8_t* a_codes, const uint8_t* a_scales, float a_
   L.num_problems = 1;
   L.K = (int)K; L.tiles_m = (int)(M / 128); L.tiles_n = (int)(N / 128);
   L.status = device_status;
-  return launch_gemm_auto(kPlain, &pr, nullptr, L, d->sms, stream) == cudaSuccess ? FP4_OK : FP4_ERR_CUDA;
+  return launch_gemm_auto(kPlain, pack, L, d->sms, stream) == cudaSuccess ? FP4_OK : FP4_ERR_CUDA;
 }
 
 }  // extern "C"
