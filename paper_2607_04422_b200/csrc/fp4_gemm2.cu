@@ -45,8 +45,14 @@ constexpr int EPI_WARPS = 4 * TEAMS;           // one warp per (column group, la
 constexpr int XBUF = 2;                        // FP32 chunk buffers per warp
 constexpr int XBUF_BYTES = 32 * CHUNK * 4;     // 2 KB: 32 rows x 64 bytes (64-byte swizzle)
 constexpr int RQ_BYTES = 32 * 32;              // row-quantised codes of 32 rows x 64 columns
-constexpr int CQ_BYTES = 64 * 16;              // column-quantised codes of 64 columns x 32 rows
-constexpr int WARP_AREA = XBUF * XBUF_BYTES + RQ_BYTES + CQ_BYTES;
+constexpr int WARP_AREA = XBUF * XBUF_BYTES + RQ_BYTES;
+// What a warp alone would write as partial 32-byte sectors is collected for one 128-column half of the
+// CTA's tile (two column groups = eight warps) and leaves as whole sectors: the column-quantised codes
+// [128 tile columns][64 bytes = the CTA's 128 rows], their scale bytes (two atoms) and the row scales
+// (two atoms).  Writes of part of a sector make the L2 fetch the rest from memory first.
+constexpr int HALF_CQ_BYTES = 128 * 64;
+constexpr int HALF_SF_BYTES = 2 * 512;
+constexpr int HALF_AREA = HALF_CQ_BYTES + 2 * HALF_SF_BYTES;
 static_assert(TEAM_CHUNKS == 4 && XBUF == 2, "the chunk loop is written for four chunks on two buffers");
 
 // Two consecutive tiles use two accumulator buffers that share one chunk of tensor memory
@@ -62,12 +68,15 @@ constexpr int OFF_A = 0;
 constexpr int OFF_B = OFF_A + STAGES * OPER_BYTES;
 constexpr int OFF_SF = OFF_B + STAGES * OPER_BYTES;
 constexpr int OFF_EPI = OFF_SF + STAGES * SF_BYTES;
-constexpr int OFF_BAR = OFF_EPI + EPI_WARPS * WARP_AREA;
+constexpr int OFF_HALF = OFF_EPI + EPI_WARPS * WARP_AREA;
+constexpr int OFF_BAR = OFF_HALF + 2 * HALF_AREA;
 constexpr int SMEM_BYTES = OFF_BAR + 512 + 1024;
 static_assert(OFF_EPI % 1024 == 0 && WARP_AREA % 1024 == 0, "chunk buffers keep the swizzle phase");
+static_assert(OFF_HALF % 1024 == 0 && HALF_AREA % 1024 == 0, "code staging keeps the swizzle phase");
 static_assert(SMEM_BYTES <= 232448, "at most 227 KB of dynamic shared memory");
 
-constexpr int NTHREADS = 64 + EPI_WARPS * 32;  // operand producer, MMA issuer, then the epilogue warps
+constexpr int ROLE_WARPS = 3;                  // operand producer, MMA issuer, issuer of the half-tile stores
+constexpr int NTHREADS = (ROLE_WARPS + EPI_WARPS) * 32;
 constexpr uint32_t TMEM_COLS = 512;
 constexpr uint32_t TMEM_SF_COL = ACC1_COL + PN;  // scale factors after the second accumulator buffer
 // Scale factors of ONE MMA (K = 64): 4 columns (row operand) + 8 (column operand, N = 256).  Copies and
@@ -85,6 +94,8 @@ struct Barriers {
   uint64_t acc_empty[2];     // even CTA: buffer drained by all epilogue warps of the pair
   uint64_t ov_free;          // even CTA: the columns shared with the other buffer are drained (8 warps)
   uint64_t xfull[EPI_WARPS * XBUF];  // a warp's chunk buffer holds the FP32 block it asked for
+  uint64_t half_done[2];     // the eight warps of a half have staged their quantised output of the tile
+  uint64_t half_free[2];     // the stores of the half's staging area have read it
   uint32_t tmem_base;
   uint32_t abort_flag;
 };
@@ -173,6 +184,17 @@ __device__ __forceinline__ void sts128(uint32_t a, float x, float y, float z, fl
 __device__ __forceinline__ void sts128u(uint32_t a, uint32_t x, uint32_t y, uint32_t z, uint32_t w) {
   asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(x), "r"(y), "r"(z), "r"(w));
 }
+__device__ __forceinline__ void sts32(uint32_t a, uint32_t x) {
+  asm volatile("st.shared.b32 [%0], %1;" ::"r"(a), "r"(x));
+}
+__device__ __forceinline__ void sts8(uint32_t a, uint32_t x) {
+  asm volatile("st.shared.b8 [%0], %1;" ::"r"(a), "r"(x));
+}
+// contiguous bytes shared -> global (16-byte aligned, a multiple of 16 bytes), part of the thread's bulk group
+__device__ __forceinline__ void bulk_store_s(void* gdst, uint32_t smem_src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(smem_src), "r"(bytes)
+               : "memory");
+}
 __device__ __forceinline__ void sts64u(uint32_t a, uint32_t x, uint32_t y) {
   asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(a), "r"(x), "r"(y));
 }
@@ -246,6 +268,7 @@ k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ Ge
     for (int i = 0; i < 2; ++i) { mbar_init(&bars->acc_full[i], 1); mbar_init(&bars->acc_empty[i], 2 * EPI_WARPS); }
     mbar_init(&bars->ov_free, 8);
     for (int i = 0; i < EPI_WARPS * XBUF; ++i) mbar_init(&bars->xfull[i], 1);
+    for (int i = 0; i < 2; ++i) { mbar_init(&bars->half_done[i], EPI_WARPS / 2); mbar_init(&bars->half_free[i], 1); }
     bars->abort_flag = 0;
     mbar_fence_init();
   }
@@ -329,16 +352,53 @@ k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ Ge
       }
       TR_FLUSH
     }
+  } else if (warp == 2) {
+    // ------------------------------------------------------------ issuer of the half-tile stores
+    // When the eight warps of a half have staged their part of a tile, one thread sends the staging area
+    // off: column-quantised codes by TMA (64-byte rows), the two kinds of scale bytes as whole atoms.
+    if (do_q && elect_one()) {
+      uint32_t seq = 0;
+      for (int t = pair; t < num_tiles; t += num_pairs, ++seq) {
+        int p, ti, tj;
+        decode_tile(t, args, tiles_per_problem, p, ti, tj, sym);
+        const GemmProblem* pr = probs + p;
+        const int bi = ti * 2 + (int)rank;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const int hcol = (seq & 1) ? h : 1 - h;          // which 128 columns of the tile this half holds
+          const int bj = tj * 2 + hcol;
+          const bool below = sym && bj < bi;
+          const bool mirror = !below && (MODE == kG3 || (sym && bi != bj));
+          wait_or_abort(&bars->half_done[h], seq & 1, abort_flag);
+          if (!below) {
+            const uint32_t st = smem_u32(smem + OFF_HALF + h * HALF_AREA);
+            bulk_store_s(pr->rq_sf + ((int64_t)bi * (args.rq_K >> 6) + bj * 2) * 512, st + HALF_CQ_BYTES + HALF_SF_BYTES,
+                         HALF_SF_BYTES);
+            if (mirror) {
+              tma_store_2d_s(&pr->tmCq, bi * (BM / 2), bj * 128, st);
+              bulk_store_s(pr->cq_sf + ((int64_t)bj * (args.cq_K >> 6) + bi * 2) * 512, st + HALF_CQ_BYTES, HALF_SF_BYTES);
+            }
+          }
+        }
+        bulk_commit();
+        bulk_wait_read<0>();
+        mbar_arrive(&bars->half_free[0]);
+        mbar_arrive(&bars->half_free[1]);
+      }
+      bulk_wait_all<0>();
+    }
   } else {
     // ------------------------------------------------------------ epilogue warps
-    const int ew = warp - 2;
+    const int ew = warp - ROLE_WARPS;
     const int team = ew >> 2;      // which 64 columns of a tile (mirrored on buffer 0, see below)
     const int quad = warp & 3;     // tensor-memory lane quadrant this warp may read
     // column pass: lane = (column cq of the chunk, 16-row group g of this warp's 32 rows)
     const int cq = lane & 15, g = lane >> 4;
     const uint32_t area = smem_u32(smem + OFF_EPI + ew * WARP_AREA);
     const uint32_t rq_st = area + XBUF * XBUF_BYTES;   // [32 rows][32 bytes]
-    const uint32_t cq_st = rq_st + RQ_BYTES;           // [64 columns][16 bytes]
+    const int half = team >> 1;                         // the staging area this warp shares with seven others
+    const uint32_t half_st = smem_u32(smem + OFF_HALF + half * HALF_AREA);
+    const uint32_t half_done = smem_u32(&bars->half_done[half]), half_free = smem_u32(&bars->half_free[half]);
     const uint32_t xfull0 = smem_u32(&bars->xfull[ew * XBUF]);
     // row pass: this lane's row of a chunk buffer is 64 bytes whose 16-byte groups are XOR-swizzled with
     // bits 1-2 of the row; group j of the row sits at row_addr ^ (j << 4)
@@ -428,7 +488,7 @@ k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ Ge
         cur_p = p;
         pr = probs + p;
         epilogue_scalars<MODE>(*pr, args, scale, sg_out,
-                               leader && t == p * tiles_per_problem && threadIdx.x == 64);
+                               leader && t == p * tiles_per_problem && threadIdx.x == ROLE_WARPS * 32);
         inv_sg = __frcp_rn(sg_out);  // exact: the predicted scales are powers of two
         rcp_base = rcp_base_of(sg_out);
         ca = pr->ca; cb = pr->cb; cc = pr->cc;
@@ -467,6 +527,13 @@ k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ Ge
           if (team == 0) mbar_arrive_cluster(ov_free_leader);
           mbar_arrive_cluster(acc_empty_leader);
         }
+        if (do_q) {
+          // Nothing is staged, but the half's count still has to fill once per tile - and only after the
+          // store issuer has seen the previous tile's phase (two of these tiles can follow each other, and
+          // a barrier that completes twice unobserved looks unchanged to a parity wait).
+          wait_or_abort(half_free, (seq & 1) ^ 1, abort_flag);
+          if (lane == 0) mbar_arrive_s(half_done);
+        }
         if (HAS_AUX) {
 #pragma unroll
           for (int i = 0; i < TEAM_CHUNKS; ++i) {
@@ -481,13 +548,16 @@ k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ Ge
 
       // store addresses of this tile: the scale word of this lane's row; scale byte of (tensor row =
       // tile column cq, 16-block = this lane's row group) in the column-quantised output
-      uint8_t* rq_sfp = nullptr; uint8_t* cq_sfp = nullptr;
-      if (do_q) {
-        rq_sfp = pr->rq_sf + sf_offset((int64_t)y32 + lane, x64 >> 4, args.rq_K >> 4);
-        const int64_t kb = (y32 >> 4) + g, kblocks = args.cq_K >> 4;
-        cq_sfp = pr->cq_sf + ((int64_t)(x64 >> 7) * (kblocks >> 2) + (kb >> 2)) * 512 + (kb & 3) + cq * 16 +
-                 ((x64 >> 6) & 1) * 8;
-      }
+      // where this lane's outputs go in the half's staging area (cgl: which of its two column groups)
+      //   codes of (tile column = cgl * 64 + e * 16 + cq, rows quad * 32 + g * 16 ...): 64-byte rows, the
+      //     16-byte groups XOR-swizzled with bits 1-2 of the row index (which are those of cq);
+      //   their scale byte: atom quad / 2 (128 tile columns x 4 blocks of 16 rows), row e % 2 * 16 + cq,
+      //     group cgl * 2 + e / 2, byte quad % 2 * 2 + g;
+      //   the scale word of this lane's row: atom cgl, row lane, group quad.
+      const int cgl = cg & 1;
+      const uint32_t cq_st = half_st + (cgl * 64 + cq) * 64 + ((quad ^ ((cq >> 1) & 3)) << 4) + g * 8;
+      const uint32_t csf_st = half_st + HALF_CQ_BYTES + (quad >> 1) * 512 + cq * 16 + cgl * 8 + (quad & 1) * 2 + g;
+      const uint32_t rsf_st = half_st + HALF_CQ_BYTES + HALF_SF_BYTES + cgl * 512 + lane * 16 + quad * 4;
       const uint32_t tm_acc = tm_lane + par * ACC1_COL + cg * (TEAM_CHUNKS * CHUNK);
       uint32_t sfw = 0;
       uint32_t acc[16];
@@ -639,7 +709,11 @@ k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ Ge
           else if (has_next) fetch(probs + nxt.p, nxt.x64, nxt.y32, (i - 2) ^ (flip ^ 3), nxt.below, b);
         }
         if (do_q) {
-          if (i == 0) __syncwarp();
+          if (i == 0) {
+            __syncwarp();
+            // the stores of the previous tile have read the half's staging area
+            wait_or_abort(half_free, (seq & 1) ^ 1, abort_flag);
+          }
           sts64u(rq_st + lane * 32 + e * 8, rlo, rhi);
         }
         // ---- quantise down the columns
@@ -649,20 +723,20 @@ k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ Ge
           uint32_t sb;
           if (PF) sb = quantize_block16_opts(w, args.q, sg_out, lo, hi, bmax);
           else sb = quantize_block16_pow2(w, sg_out, inv_sg, rcp_base, lo, hi, bmax);
-          sts64u(cq_st + (e * CHUNK + cq) * 16 + g * 8, lo, hi);
+          sts64u(cq_st + e * (CHUNK * 64), lo, hi);
           // tensor row = x64 + e * 16 + cq: e % 2 selects the upper 16 of 32 rows of its scale atom,
           // e / 2 the 32-row group
-          cq_sfp[(e & 1) * 256 + (e >> 1) * 4] = (uint8_t)sb;
+          sts8(csf_st + (e & 1) * 256 + (e >> 1) * 4, sb);
         }
       }
       if (do_q) {
         // the scale word of this warp's 64 columns of the row; the codes of the warp's part of the tile
-        *reinterpret_cast<uint32_t*>(rq_sfp) = sfw;
+        sts32(rsf_st, sfw);
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) {
+          mbar_arrive_s(half_done);
           tma_store_2d_s(&pr->tmRq, x64 >> 1, y32, rq_st);
-          if (mirror) tma_store_2d_s(&pr->tmCq, y32 >> 1, x64, cq_st);
           bulk_commit();
         }
       }

@@ -69,8 +69,9 @@ struct alignas(64) GemmProblem {
   CUtensorMap tmSfa, tmSfb;  // scale atoms of the two operands as 2-D maps (CTA-pair kernel)
   CUtensorMap tmH;           // BF16 storage: the 2-byte tensor this stage reads its tile from and / or stores its
                              // result to (A for G1 / G2, X for G3); box 16 columns x 32 rows, no swizzle
-  CUtensorMap tmRq, tmCq;    // CTA-pair kernel: byte maps over rq_codes (box 32 bytes x 32 rows) and cq_codes
-                             // (box 16 bytes x 64 rows), through which a warp stores the codes of its part of a tile
+  CUtensorMap tmRq, tmCq;    // CTA-pair kernel: byte maps over rq_codes (box 32 bytes x 32 rows: one warp's part of a
+                             // tile) and cq_codes (box 64 bytes x 128 rows, 64-byte swizzle: a CTA's 128 rows of
+                             // 128 tile columns) for the stores of the quantised outputs
   const uint8_t* sfa;        // scale atoms of the row operand
   const uint8_t* sfb;        // scale atoms of the column operand
   float* scalars;            // workspace scalars of this matrix (device)

@@ -122,14 +122,14 @@ bool make_bf16_map(const DeviceInfo* d, CUtensorMap* tm, const void* base, int64
 // 2-D map over a row-major byte matrix (NVFP4 codes) for the stores of the CTA-pair kernel's epilogue
 // warps: box = box_bytes x box_rows, no swizzle.
 bool make_code_store_map(const DeviceInfo* d, CUtensorMap* tm, const void* base, int64_t rows, int64_t row_bytes,
-                         int box_bytes, int box_rows) {
+                         int box_bytes, int box_rows, bool swizzle64 = false) {
   cuuint64_t dims[2] = {(cuuint64_t)row_bytes, (cuuint64_t)rows};
   cuuint64_t strides[1] = {(cuuint64_t)row_bytes};
   cuuint32_t box[2] = {(cuuint32_t)box_bytes, (cuuint32_t)box_rows};
   cuuint32_t estr[2] = {1, 1};
   return d->encode(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
-                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 constexpr int kDefaultMaxGroup = kPackMax;
@@ -327,12 +327,12 @@ fp4_status prepare_matrix(const DeviceInfo* d, const float* G, float* out, int64
   // stores of the quantised outputs by the CTA-pair kernel's epilogue warps
   CUtensorMap st_qA_r, st_qA_c, st_qB_r, st_qB_c, st_qX_r, st_qXt_c[2];
   ok = make_code_store_map(d, &st_qA_r, ws + L.qA_codes, s, s / 2, 32, 32) &&
-       make_code_store_map(d, &st_qA_c, ws + L.qA_codes, s, s / 2, 16, 64) &&
+       make_code_store_map(d, &st_qA_c, ws + L.qA_codes, s, s / 2, 64, 128, true) &&
        make_code_store_map(d, &st_qB_r, ws + L.qB_codes, s, s / 2, 32, 32) &&
-       make_code_store_map(d, &st_qB_c, ws + L.qB_codes, s, s / 2, 16, 64) &&
+       make_code_store_map(d, &st_qB_c, ws + L.qB_codes, s, s / 2, 64, 128, true) &&
        make_code_store_map(d, &st_qX_r, ws + L.qX_codes, s, l / 2, 32, 32) &&
-       make_code_store_map(d, &st_qXt_c[0], ws + L.qXt_codes[0], l, s / 2, 16, 64) &&
-       make_code_store_map(d, &st_qXt_c[1], ws + L.qXt_codes[1], l, s / 2, 16, 64);
+       make_code_store_map(d, &st_qXt_c[0], ws + L.qXt_codes[0], l, s / 2, 64, 128, true) &&
+       make_code_store_map(d, &st_qXt_c[1], ws + L.qXt_codes[1], l, s / 2, 64, 128, true);
   if (!ok) return FP4_ERR_CUDA;
   GemmProblem base;
   memset(&base, 0, sizeof(base));
