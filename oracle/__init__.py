@@ -103,6 +103,9 @@ def lib():
         L.orc_root_ns.argtypes = [_f32p, C.c_int64, C.c_int64, C.c_int, C.POINTER(OrcParams),
                                   _f32p, C.POINTER(OrcTrace)]
         L.orc_root_ns.restype = C.c_int
+        L.orc_ns_iteration.argtypes = [_f32p, C.c_int64, C.c_int64, C.c_int, C.c_int, C.c_float, C.c_float,
+                                       C.POINTER(OrcParams), _f32p, _f32p, _f32p, C.POINTER(OrcTrace)]
+        L.orc_ns_iteration.restype = C.c_int
         _lib = L
     return _lib
 
@@ -342,8 +345,16 @@ def root_ns(G, steps=5, abc=None, clip_quantile=0.99, eps=1e-7, quantize=True,
         if rc:
             raise ValueError(f"orc_root_ns failed with code {rc}")
         return out
-    t = OrcTrace()
+    t, bufs = _make_trace(s, l, quantize)
     t.iter = int(trace_iter)
+    rc = lib().orc_root_ns(gp, m, n, int(steps), C.byref(p), out.ctypes.data_as(_f32p), C.byref(t))
+    if rc:
+        raise ValueError(f"orc_root_ns failed with code {rc}")
+    return out, _finish_trace(bufs)
+
+
+def _make_trace(s, l, quantize=True):
+    t = OrcTrace()
     bufs = {}
 
     def f(name, shape):
@@ -365,9 +376,41 @@ def root_ns(G, steps=5, abc=None, clip_quantile=0.99, eps=1e-7, quantize=True,
         u("qXt_codes", (l, s // 2)); u("qXt_scales", (l, s // 16))
         u("qA_codes", (s, s // 2)); u("qA_scales", (s, s // 16))
         u("qB_codes", (s, s // 2)); u("qB_scales", (s, s // 16))
-    rc = lib().orc_root_ns(gp, m, n, int(steps), C.byref(p), out.ctypes.data_as(_f32p), C.byref(t))
-    if rc:
-        raise ValueError(f"orc_root_ns failed with code {rc}")
+    return t, bufs
+
+
+def _finish_trace(bufs):
     for name in ("tau", "nu", "amax_in", "sg_X", "sg_A", "sg_B"):
         bufs[name] = float(bufs[name][0])
-    return out, bufs
+    return bufs
+
+
+def ns_iteration(X, k, amax_X, sg_X, abc=None, last=False, rht=False, four_six=False, seed=0):
+    """One quantised Newton-Schulz iteration (index k) from a given state: X is s x l FP32 in the
+    work orientation (s <= l), amax_X = max|X|, sg_X the tensor scale of its operand copies.
+    Returns (X_next, amax_next, sg_next, trace dict)."""
+    X, xp = _f32(X)
+    s, l = X.shape
+    p = OrcParams()
+    if abc is None:
+        p.a = p.b = p.c = float("nan")
+    else:
+        p.a, p.b, p.c = [float(np.float32(v)) for v in abc]
+    p.clip_quantile = 0.0
+    p.eps = 0.0
+    p.quantize = 1
+    p.exact_scales = 0
+    p.rht = 1 if rht else 0
+    p.four_six = 1 if four_six else 0
+    p.seed = int(seed)
+    p.store_bf16 = 0
+    t, bufs = _make_trace(s, l)
+    t.iter = int(k)
+    out = np.empty((s, l), np.float32)
+    am = np.zeros(1, np.float32); sg = np.zeros(1, np.float32)
+    rc = lib().orc_ns_iteration(xp, s, l, int(k), 1 if last else 0, float(np.float32(amax_X)), float(np.float32(sg_X)),
+                                C.byref(p), out.ctypes.data_as(_f32p), am.ctypes.data_as(_f32p),
+                                sg.ctypes.data_as(_f32p), C.byref(t))
+    if rc:
+        raise ValueError(f"orc_ns_iteration failed with code {rc}")
+    return out, float(am[0]), float(sg[0]), _finish_trace(bufs)

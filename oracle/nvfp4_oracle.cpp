@@ -611,6 +611,88 @@ void orc_root_coeffs(int64_t m, int64_t n, int steps, float abc[3]) {
   abc[2] = (float)(a - 1.5);
 }
 
+// One quantised iteration (Section 3.4, display equations) from the state at its start:
+// X (what is kept between the iterations and enters a X), Xq (the FP32 values the operand copies
+// are quantised from; the same as X unless BF16 storage is on), amax(Xq) and the tensor scale
+// of the operand copies.  Leaves the state at the start of the next iteration in the same
+// variables.  k picks the Hadamard sign vectors; rec: fill the trace.
+static void ns_iteration_quantised(int k, bool last_it, int64_t s, int64_t l, const orc_params* prm, float ca,
+                                   float cb, float cc, std::vector<float>& X, std::vector<float>& Xq,
+                                   float& amax_X, float& sg_X, orc_trace* tr, bool rec) {
+  const size_t N = (size_t)s * l;
+  std::vector<float> Xt(N), A((size_t)s * s), S((size_t)s * s), B((size_t)s * s), P(N);
+  std::vector<uint8_t> qXc(N / 2 + 1), qXs(N / 16 + 1), qXtc(N / 2 + 1), qXts(N / 16 + 1);
+  std::vector<uint8_t> qAc((size_t)s * s / 2 + 1), qAs((size_t)s * s / 16 + 1);
+  std::vector<uint8_t> qBc((size_t)s * s / 2 + 1), qBs((size_t)s * s / 16 + 1);
+  const int bf16 = prm->store_bf16;
+  const int rht = prm->rht, f46 = prm->four_six;
+  const float widen = rht ? 4.0f : 1.0f;  // |x H^r| <= 4 amax(x)
+    // qX = Q_1x16(X), qX^{16x1} = Q_16x1(X) = Q_1x16(X^T), one global scale
+    transpose(Xq.data(), s, l, Xt.data());
+    // one Hadamard matrix for X_k (both operand copies and B_k, which meets qX^{16x1}),
+    // another for A_k
+    const uint16_t mask_X = rht ? rht_mask(prm->seed, 2 * (uint64_t)k) : 0;
+    const uint16_t mask_A = rht ? rht_mask(prm->seed, 2 * (uint64_t)k + 1) : 0;
+    quantize_1x16(Xq.data(), s, l, sg_X, qXc.data(), qXs.data(), rht, mask_X, f46);
+    quantize_1x16(Xt.data(), l, s, sg_X, qXtc.data(), qXts.data(), rht, mask_X, f46);
+    // A = qX qX^T
+    {
+      std::vector<double> d = decode_f64(qXc.data(), qXs.data(), sg_X, s, l);
+      gemm_nt(d.data(), d.data(), s, s, l, A.data(), 1);
+    }
+    float amax_A = amax_of(A.data(), (int64_t)s * s);
+    float bound_A = std::min(2.0f * (float)l * amax_X * amax_X, 4.0f);
+    float sg_A = prm->exact_scales ? scale_exact(widen * amax_A) : scale_predicted(widen * bound_A);
+    // qA = Q_1x16(A); A is symmetric so Q_16x1(A) is the transpose of qA
+    quantize_1x16(A.data(), s, s, sg_A, qAc.data(), qAs.data(), rht, mask_A, f46);
+    {
+      std::vector<double> d = decode_f64(qAc.data(), qAs.data(), sg_A, s, s);
+      gemm_nt(d.data(), d.data(), s, s, s, S.data(), 1);
+    }
+    // B = b A + c (qA qA^{16x1}), each product and the sum rounded to FP32; A as it is stored
+    for (size_t i = 0; i < (size_t)s * s; ++i) {
+      const float a_st = bf16 ? bf16_round(A[i]) : A[i];
+      float t1 = cb * a_st;
+      float t2 = cc * S[i];
+      B[i] = t1 + t2;
+    }
+    float amax_B = amax_of(B.data(), (int64_t)s * s);
+    float bound_B = (std::fabs(cb) + 4.0f * std::fabs(cc)) * amax_A;
+    float sg_B = prm->exact_scales ? scale_exact(widen * amax_B) : scale_predicted(widen * bound_B);
+    quantize_1x16(B.data(), s, s, sg_B, qBc.data(), qBs.data(), rht, mask_X, f46);
+    // X+ = a X + qB qX^{16x1}
+    {
+      std::vector<double> db = decode_f64(qBc.data(), qBs.data(), sg_B, s, s);
+      std::vector<double> dx = decode_f64(qXtc.data(), qXts.data(), sg_X, l, s);
+      gemm_nt(db.data(), dx.data(), s, l, s, P.data(), 0);
+    }
+    if (rec) {
+      if (tr->qX_codes) std::memcpy(tr->qX_codes, qXc.data(), N / 2);
+      if (tr->qX_scales) std::memcpy(tr->qX_scales, qXs.data(), N / 16);
+      if (tr->qXt_codes) std::memcpy(tr->qXt_codes, qXtc.data(), N / 2);
+      if (tr->qXt_scales) std::memcpy(tr->qXt_scales, qXts.data(), N / 16);
+      if (tr->sg_X) *tr->sg_X = sg_X;
+      if (tr->A) std::memcpy(tr->A, A.data(), (size_t)s * s * 4);
+      if (tr->qA_codes) std::memcpy(tr->qA_codes, qAc.data(), (size_t)s * s / 2);
+      if (tr->qA_scales) std::memcpy(tr->qA_scales, qAs.data(), (size_t)s * s / 16);
+      if (tr->sg_A) *tr->sg_A = sg_A;
+      if (tr->S) std::memcpy(tr->S, S.data(), (size_t)s * s * 4);
+      if (tr->B) std::memcpy(tr->B, B.data(), (size_t)s * s * 4);
+      if (tr->qB_codes) std::memcpy(tr->qB_codes, qBc.data(), (size_t)s * s / 2);
+      if (tr->qB_scales) std::memcpy(tr->qB_scales, qBs.data(), (size_t)s * s / 16);
+      if (tr->sg_B) *tr->sg_B = sg_B;
+    }
+    float amax_prev = amax_X;
+    for (size_t i = 0; i < N; ++i) {
+      float t1 = ca * X[i];
+      Xq[i] = t1 + P[i];
+      X[i] = (bf16 && !last_it) ? bf16_round(Xq[i]) : Xq[i];
+    }
+    amax_X = amax_of(Xq.data(), (int64_t)N);
+    float bound_X = 4.0f * std::fabs(ca) * amax_prev;
+    sg_X = prm->exact_scales ? scale_exact(widen * amax_X) : scale_predicted(widen * bound_X);
+}
+
 // The whole step.  G is m x n row-major, out is m x n row-major.
 int orc_root_ns(const float* G, int64_t m, int64_t n, int steps, const orc_params* prm,
                 float* out, orc_trace* tr) {
@@ -681,77 +763,38 @@ int orc_root_ns(const float* G, int64_t m, int64_t n, int steps, const orc_param
       gemm_nt(Bd.data(), Xtd.data(), s, l, s, P.data(), 0);
       for (size_t i = 0; i < N; ++i) X[i] = ca * X[i] + P[i];
     } else {
-      // qX = Q_1x16(X), qX^{16x1} = Q_16x1(X) = Q_1x16(X^T), one global scale
-      transpose(Xq.data(), s, l, Xt.data());
-      // one Hadamard matrix for X_k (both operand copies and B_k, which meets qX^{16x1}),
-      // another for A_k
-      const uint16_t mask_X = rht ? rht_mask(prm->seed, 2 * (uint64_t)k) : 0;
-      const uint16_t mask_A = rht ? rht_mask(prm->seed, 2 * (uint64_t)k + 1) : 0;
-      quantize_1x16(Xq.data(), s, l, sg_X, qXc.data(), qXs.data(), rht, mask_X, f46);
-      quantize_1x16(Xt.data(), l, s, sg_X, qXtc.data(), qXts.data(), rht, mask_X, f46);
-      // A = qX qX^T
-      {
-        std::vector<double> d = decode_f64(qXc.data(), qXs.data(), sg_X, s, l);
-        gemm_nt(d.data(), d.data(), s, s, l, A.data(), 1);
-      }
-      float amax_A = amax_of(A.data(), (int64_t)s * s);
-      float bound_A = std::min(2.0f * (float)l * amax_X * amax_X, 4.0f);
-      float sg_A = prm->exact_scales ? scale_exact(widen * amax_A) : scale_predicted(widen * bound_A);
-      // qA = Q_1x16(A); A is symmetric so Q_16x1(A) is the transpose of qA
-      quantize_1x16(A.data(), s, s, sg_A, qAc.data(), qAs.data(), rht, mask_A, f46);
-      {
-        std::vector<double> d = decode_f64(qAc.data(), qAs.data(), sg_A, s, s);
-        gemm_nt(d.data(), d.data(), s, s, s, S.data(), 1);
-      }
-      // B = b A + c (qA qA^{16x1}), each product and the sum rounded to FP32; A as it is stored
-      for (size_t i = 0; i < (size_t)s * s; ++i) {
-        const float a_st = bf16 ? bf16_round(A[i]) : A[i];
-        float t1 = cb * a_st;
-        float t2 = cc * S[i];
-        B[i] = t1 + t2;
-      }
-      float amax_B = amax_of(B.data(), (int64_t)s * s);
-      float bound_B = (std::fabs(cb) + 4.0f * std::fabs(cc)) * amax_A;
-      float sg_B = prm->exact_scales ? scale_exact(widen * amax_B) : scale_predicted(widen * bound_B);
-      quantize_1x16(B.data(), s, s, sg_B, qBc.data(), qBs.data(), rht, mask_X, f46);
-      // X+ = a X + qB qX^{16x1}
-      {
-        std::vector<double> db = decode_f64(qBc.data(), qBs.data(), sg_B, s, s);
-        std::vector<double> dx = decode_f64(qXtc.data(), qXts.data(), sg_X, l, s);
-        gemm_nt(db.data(), dx.data(), s, l, s, P.data(), 0);
-      }
-      if (rec) {
-        if (tr->qX_codes) std::memcpy(tr->qX_codes, qXc.data(), N / 2);
-        if (tr->qX_scales) std::memcpy(tr->qX_scales, qXs.data(), N / 16);
-        if (tr->qXt_codes) std::memcpy(tr->qXt_codes, qXtc.data(), N / 2);
-        if (tr->qXt_scales) std::memcpy(tr->qXt_scales, qXts.data(), N / 16);
-        if (tr->sg_X) *tr->sg_X = sg_X;
-        if (tr->A) std::memcpy(tr->A, A.data(), (size_t)s * s * 4);
-        if (tr->qA_codes) std::memcpy(tr->qA_codes, qAc.data(), (size_t)s * s / 2);
-        if (tr->qA_scales) std::memcpy(tr->qA_scales, qAs.data(), (size_t)s * s / 16);
-        if (tr->sg_A) *tr->sg_A = sg_A;
-        if (tr->S) std::memcpy(tr->S, S.data(), (size_t)s * s * 4);
-        if (tr->B) std::memcpy(tr->B, B.data(), (size_t)s * s * 4);
-        if (tr->qB_codes) std::memcpy(tr->qB_codes, qBc.data(), (size_t)s * s / 2);
-        if (tr->qB_scales) std::memcpy(tr->qB_scales, qBs.data(), (size_t)s * s / 16);
-        if (tr->sg_B) *tr->sg_B = sg_B;
-      }
-      float amax_prev = amax_X;
-      const bool last_it = (k == steps - 1);
-      for (size_t i = 0; i < N; ++i) {
-        float t1 = ca * X[i];
-        Xq[i] = t1 + P[i];
-        X[i] = (bf16 && !last_it) ? bf16_round(Xq[i]) : Xq[i];
-      }
-      amax_X = amax_of(Xq.data(), (int64_t)N);
-      float bound_X = 4.0f * std::fabs(ca) * amax_prev;
-      sg_X = prm->exact_scales ? scale_exact(widen * amax_X) : scale_predicted(widen * bound_X);
+      ns_iteration_quantised(k, k == steps - 1, s, l, prm, ca, cb, cc, X, Xq, amax_X, sg_X, tr, rec);
     }
     if (rec && tr->X_out) std::memcpy(tr->X_out, prm->quantize ? Xq.data() : X.data(), N * sizeof(float));
   }
 
   const std::vector<float>& R = prm->quantize ? Xq : X;  // the last iteration's FP32 result
   if (tall) transpose(R.data(), s, l, out); else std::memcpy(out, R.data(), N * sizeof(float));
+  return 0;
+}
+
+// One quantised iteration from a state handed in by the caller (teacher-forced checks of a later
+// iteration: the state is another implementation's).  X is s x l in the work orientation
+// (s <= l), amax_X = max |X|, sg_X the tensor scale its operand copies are quantised with; k is
+// the iteration's index (it picks the Hadamard signs), a NaN coefficient a selects the
+// provider's values for the shape.  X_out receives the FP32 result, amax_out / sg_out the
+// state scalars of the next iteration; the trace (may be null) is filled as in orc_root_ns.
+int orc_ns_iteration(const float* X_in, int64_t s, int64_t l, int k, int last_it, float amax_X, float sg_X,
+                     const orc_params* prm, float* X_out, float* amax_out, float* sg_out, orc_trace* tr) {
+  if (s <= 0 || l < s || (s % 16) || (l % 16) || !prm->quantize || prm->store_bf16) return 1;
+  float abc[3] = {prm->a, prm->b, prm->c};
+  if (!(prm->a == prm->a)) orc_root_coeffs(s, l, 0, abc);
+  const size_t N = (size_t)s * l;
+  std::vector<float> X(X_in, X_in + N), Xq(X);
+  if (tr) {
+    if (tr->amax_in) *tr->amax_in = amax_X;
+    if (tr->X_in) std::memcpy(tr->X_in, X.data(), N * sizeof(float));
+  }
+  ns_iteration_quantised(k, last_it != 0, s, l, prm, abc[0], abc[1], abc[2], X, Xq, amax_X, sg_X, tr, tr != nullptr);
+  std::memcpy(X_out, Xq.data(), N * sizeof(float));
+  if (tr && tr->X_out) std::memcpy(tr->X_out, Xq.data(), N * sizeof(float));
+  if (amax_out) *amax_out = amax_X;
+  if (sg_out) *sg_out = sg_X;
   return 0;
 }
 

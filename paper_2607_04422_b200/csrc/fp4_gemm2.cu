@@ -700,6 +700,10 @@ k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ Ge
         // ---- the buffer is free once every lane has read its column and the store has read the
         // block; the block two chunks ahead is fetched into it.  (Waiting for the store's read here
         // also covers the code stores of the previous tile before the first chunk writes codes.)
+        // The column reads above belong to the generic proxy, the fetch below writes the buffer through the
+        // async proxy: without a fence between them nothing orders the two (the reads were seen to be
+        // scheduled after the fetch, and now and then the new block arrived first).
+        if (HAS_AUX) fence_proxy_async_smem();
         __syncwarp();
         TR_BEGIN
         if (lane == 0 && (STORE_F32 || i == 0)) bulk_wait_read<0>();
