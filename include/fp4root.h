@@ -89,9 +89,9 @@ typedef struct {
                           clamped to the nearest-rank quantile of |G|, resolved to parts
                           per million.  Default 0.99; <= 0 or >= 1 disables the clip.      */
   float eps;           /* X0 = G_c / (||G_c||_F + eps).  Default 1e-7.                     */
-  uint32_t flags;      /* FP4_FLAG_*; default 0                                            */
+  uint32_t flags;      /* FP4_FLAG_*; default 0; unknown bits: FP4_ERR_INVALID_ARG             */
   uint32_t max_group;  /* fp4_root_ns_batched: at most this many equal-shape matrices run their
-                          stages in lockstep as single launches; 0 = library default (16)     */
+                          stages in lockstep as single launches; 0 or more than 16 = 16        */
   uint64_t seed;       /* FP4_FLAG_RHT: seed of the sign draws; default 0                    */
   uint32_t* const* top_hist; /* NULL (default), or a host array with one entry per matrix of the call
                           (one entry for fp4_root_ns and fp4_root_ns_static): NULL, or a device
@@ -187,9 +187,13 @@ fp4_status fp4_root_ns_batched(int count, const float* const* G, float* const* o
  * device_status: device, optional (may be NULL): one uint32 that receives, in stream order,
  *   the status word of this call (FP4_OK or FP4_ERR_DEVICE_TIMEOUT).
  *
- * It calls no cudaMalloc, cudaFree or other allocating routine.  The first call on each
- * device looks up the array's device address (a one-time, per-device set-up done with that
- * device current); make that first call outside any stream capture.  All calls on a device
+ * It calls no cudaMalloc, cudaFree or other allocating routine (as long as fp4_profile_enable is
+ * off: the profiling brackets create events).  The first call on each device loads the module
+ * and resolves the array's device address, with that device current; make that first call
+ * outside any stream capture.  The address is looked up again on every call (a cheap table read),
+ * so a context that was destroyed and rebuilt between calls is handled; kernel attributes set
+ * during the library's per-device set-up are not re-applied after a cudaDeviceReset, which the
+ * library does not support while it is loaded.  All calls on a device
  * share the one array, which keeps whatever the previous call left in it; the call itself
  * clears the parts that must start from zero.  Two calls whose kernels could overlap on the
  * GPU (different streams without an ordering between them) race on the array: order them.

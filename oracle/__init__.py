@@ -103,6 +103,7 @@ def lib():
         L.orc_root_ns.argtypes = [_f32p, C.c_int64, C.c_int64, C.c_int, C.POINTER(OrcParams),
                                   _f32p, C.POINTER(OrcTrace)]
         L.orc_root_ns.restype = C.c_int
+        L.orc_sr_e2m1x4.argtypes = [_f32p, C.c_uint32]; L.orc_sr_e2m1x4.restype = C.c_uint16
         L.orc_ns_iteration.argtypes = [_f32p, C.c_int64, C.c_int64, C.c_int, C.c_int, C.c_float, C.c_float,
                                        C.POINTER(OrcParams), _f32p, _f32p, _f32p, C.POINTER(OrcTrace)]
         L.orc_ns_iteration.restype = C.c_int
@@ -190,6 +191,12 @@ def bf16_round(x):
 def splitmix64_at(seed, idx):
     """Output number idx (from 0) of the splitmix64 generator seeded with `seed`."""
     return int(lib().orc_splitmix64_at(int(seed), int(idx)))
+
+
+def sr_e2m1x4(y4, word: int) -> int:
+    """Four values rounded stochastically with one 32-bit random word; four nibbles, element 0 lowest."""
+    y, yp = _f32(np.asarray(y4, np.float32).reshape(4))
+    return int(lib().orc_sr_e2m1x4(yp, int(word) & 0xFFFFFFFF))
 
 
 def momentum_encode(M, sr=False, seed=0):

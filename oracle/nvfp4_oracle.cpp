@@ -773,6 +773,20 @@ int orc_root_ns(const float* G, int64_t m, int64_t n, int steps, const orc_param
   return 0;
 }
 
+// Stochastic rounding of four values with one 32-bit random word (the rule of the momentum state,
+// Section 3.3): element e takes the bits sr_bits_of_word assigns to it; result = four nibbles,
+// element 0 in bits 3:0.
+uint16_t orc_sr_e2m1x4(const float* y, uint32_t word) {
+  uint32_t r[4];
+  sr_bits_of_word(word, r);
+  uint16_t out = 0;
+  for (int e = 0; e < 4; ++e) {
+    const uint32_t nib = (std::signbit(y[e]) ? 8u : 0u) | (uint32_t)e2m1_index_sr(std::fabs(y[e]), r[e]);
+    out = (uint16_t)(out | (nib << (4 * e)));
+  }
+  return out;
+}
+
 // One quantised iteration from a state handed in by the caller (teacher-forced checks of a later
 // iteration: the state is another implementation's).  X is s x l in the work orientation
 // (s <= l), amax_X = max |X|, sg_X the tensor scale its operand copies are quantised with; k is

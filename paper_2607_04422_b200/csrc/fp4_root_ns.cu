@@ -81,6 +81,8 @@ inline bool shape_ok(int64_t v) { return v >= 128 && v % 128 == 0 && v <= (1 << 
 // The Newton-Schulz entry points pad internally: any positive multiple of the block length.
 inline bool ns_shape_ok(int64_t v) { return v >= 16 && v % 16 == 0 && v <= (1 << 20); }
 inline int64_t pad128(int64_t v) { return (v + 127) / 128 * 128; }
+// flag bits the Newton-Schulz entry points know
+constexpr uint32_t kNsFlags = FP4_FLAG_KEEP_OPERANDS | FP4_FLAG_RHT | FP4_FLAG_FOUR_SIX | FP4_FLAG_STORE_BF16;
 
 // 2-D map over a row-major byte matrix (NVFP4 codes): box = one operand stage (64 or 128 bytes
 // x 128 rows), swizzled over the box width.
@@ -590,7 +592,7 @@ fp4_status fp4_root_coeffs(int64_t m, int64_t n, int steps, float abc[3]) {
 }
 
 fp4_status fp4_root_ns_workspace_layout(int64_t m, int64_t n, int steps, uint32_t flags, fp4_ws_layout* layout) {
-  if (!layout) return FP4_ERR_INVALID_ARG;
+  if (!layout || (flags & ~kNsFlags)) return FP4_ERR_INVALID_ARG;
   fp4_ns_params p;
   default_params(&p);
   p.flags = flags;
@@ -611,7 +613,7 @@ fp4_status fp4_root_ns(const float* G, float* out, int64_t m, int64_t n, int ste
                        void* ws, size_t ws_bytes, cudaStream_t stream) {
   fp4_ns_params dp;
   if (!p) { default_params(&dp); p = &dp; }
-  if (!G || !out || !ws) return FP4_ERR_INVALID_ARG;
+  if (!G || !out || !ws || (p->flags & ~kNsFlags)) return FP4_ERR_INVALID_ARG;
   if (!ns_shape_ok(m) || !ns_shape_ok(n)) return FP4_ERR_SHAPE;
   if (steps < 0 || steps > kMaxSteps) return FP4_ERR_INVALID_ARG;
   if (!aligned(G, 16) || !aligned(out, 16) || !aligned(ws, 256)) return FP4_ERR_ALIGNMENT;
@@ -642,7 +644,7 @@ fp4_status fp4_root_ns_batched(int count, const float* const* G, float* const* o
                                cudaStream_t stream) {
   fp4_ns_params dp;
   if (!p) { default_params(&dp); p = &dp; }
-  if (count < 0 || (count > 0 && (!G || !out || !m || !n)) || !ws) return FP4_ERR_INVALID_ARG;
+  if (count < 0 || (count > 0 && (!G || !out || !m || !n)) || !ws || (p->flags & ~kNsFlags)) return FP4_ERR_INVALID_ARG;
   if (steps < 0 || steps > kMaxSteps) return FP4_ERR_INVALID_ARG;
   if (!aligned(ws, 256)) return FP4_ERR_ALIGNMENT;
   for (int i = 0; i < count; ++i) {
@@ -769,23 +771,18 @@ extern "C" fp4_status fp4_selftest_bounded_wait(uint32_t* device_status, uint32_
 // no pool to take a workspace from).  The array is part of the module image: every device
 // that loads the library holds these 16 MiB until the process ends.  In host code the
 // array's name stands for the symbol, it is not a device address; the address is looked up
-// once per device with cudaGetSymbolAddress and handed to the kernels like any workspace.
+// with cudaGetSymbolAddress, with the caller's device current, and handed to the kernels like
+// any workspace.
 namespace {
 static __device__ __align__(256) unsigned char g_static_scratch[FP4_STATIC_SCRATCH_BYTES];
-void* g_static_ptr[64] = {nullptr};
-std::mutex g_static_mu;
 
-// Device address of the static array on the current device; looked up on the first call.
+// Device address of the static array on the current device.  Looked up on every call: the lookup is a
+// table read once the module is loaded, allocates nothing, and stays right if the context was torn
+// down and rebuilt in between (a cached address would not).
 fp4_status static_scratch_address(void** ptr) {
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return FP4_ERR_CUDA;
-  std::lock_guard<std::mutex> lock(g_static_mu);
-  if (g_static_ptr[dev] == nullptr) {
-    void* p = nullptr;
-    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) return FP4_ERR_CUDA;
-    g_static_ptr[dev] = p;
-  }
-  *ptr = g_static_ptr[dev];
+  void* p = nullptr;
+  if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) return FP4_ERR_CUDA;
+  *ptr = p;
   return FP4_OK;
 }
 }  // namespace
@@ -796,7 +793,7 @@ fp4_status fp4_root_ns_static(const float* G, float* out, int64_t m, int64_t n, 
                               uint32_t* device_status, cudaStream_t stream) {
   fp4_ns_params dp;
   if (!p) { default_params(&dp); p = &dp; }
-  if (!G || !out) return FP4_ERR_INVALID_ARG;
+  if (!G || !out || (p->flags & ~kNsFlags)) return FP4_ERR_INVALID_ARG;
   if (!ns_shape_ok(m) || !ns_shape_ok(n)) return FP4_ERR_SHAPE;
   if (steps < 0 || steps > kMaxSteps) return FP4_ERR_INVALID_ARG;
   if (!aligned(G, 16) || !aligned(out, 16) || (device_status && !aligned(device_status, 4))) return FP4_ERR_ALIGNMENT;

@@ -133,12 +133,30 @@ def test_iteration_counts_1_to_5(shape, gen, qmode):
         assert abs(orth_err(got) - orth_err(want)) <= TOL_ORTH
 
 
-def test_in_place_and_determinism():
-    G = workloads.gradient_like(384, 640, seed=5)
-    a, _ = run_gpu(G, steps=3)
-    b, _ = run_gpu(G, steps=3)
-    c, _ = run_gpu(G.copy(), steps=3, in_place=True)
+@pytest.mark.parametrize("shape", [(384, 640), (512, 1024), (1024, 512), (768, 768)])
+@pytest.mark.parametrize("flags", [0, FP4_FLAG_STORE_BF16])
+def test_in_place_and_determinism(shape, flags):
+    """out == G, in the single-CTA kernel (384 x 640) and in the CTA-pair kernel (the others), whose
+    first G3 stage reads the raw input through one tensor map while it stores X1 to the same
+    addresses through another."""
+    G = workloads.gradient_like(*shape, seed=5)
+    a, _ = run_gpu(G, steps=3, flags=flags)
+    b, _ = run_gpu(G, steps=3, flags=flags)
+    c, _ = run_gpu(G.copy(), steps=3, flags=flags, in_place=True)
     assert np.array_equal(a, b) and np.array_equal(a, c)
+
+
+def test_batched_in_place_pair_kernel_shapes():
+    specs = [(512, 1024, 1), (1024, 512, 2), (512, 1024, 3), (512, 512, 4)]
+    mats = [workloads.gradient_like(m, n, seed=sd) for m, n, sd in specs]
+    Gs = [torch.from_numpy(g).cuda() for g in mats]
+    shapes = [tuple(g.shape) for g in Gs]
+    ws = torch.empty(fp4.fp4_root_ns_batched_workspace_bytes(shapes, 3), dtype=torch.uint8, device="cuda")
+    fp4.fp4_root_ns_batched(Gs, Gs, 3, None, ws)            # every matrix in place
+    assert fp4.fp4_last_device_status(ws) == 0
+    for g, o in zip(mats, Gs):
+        single, _ = run_gpu(g, steps=3)
+        assert np.array_equal(o.cpu().numpy(), single)
 
 
 def test_tall_equals_transposed_wide():
@@ -343,7 +361,7 @@ def test_bounded_wait_gives_up_and_reports():
     assert rel(got, oracle.root_ns(G, steps=2)) <= TOL_OUT
 
 
-@pytest.mark.parametrize("shape", [(256, 512), (512, 256), (144, 272), (272, 144)])
+@pytest.mark.parametrize("shape", [(256, 512), (512, 256), (144, 272), (272, 144), (768, 1024), (400, 512)])
 def test_nothing_is_written_outside_the_buffers(shape):
     """Guard regions around the workspace and the result keep their pattern (also with the
     zero padding of shapes that are not multiples of 128)."""
@@ -377,6 +395,13 @@ def test_argument_errors():
     with pytest.raises(fp4.Fp4Error) as e:
         fp4.fp4_root_ns(G, G, 5, None, ws[1:])
     assert e.value.code == 3
+    for bad_flags in (16, FP4_FLAG_RHT | (0x1234 << 16)):      # unknown bits, fp4_quantize's sign bits
+        with pytest.raises(fp4.Fp4Error) as e:
+            fp4.fp4_root_ns(G, G, 5, fp4.NsParams.make(flags=bad_flags), ws)
+        assert e.value.code == 1
+        with pytest.raises(fp4.Fp4Error) as e:
+            fp4.fp4_root_ns_batched([G], [G], 5, fp4.NsParams.make(flags=bad_flags), ws)
+        assert e.value.code == 1
 
 
 # --------------------------------------------------------------------------------------

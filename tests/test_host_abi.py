@@ -55,7 +55,11 @@ def test_scale_bytes_and_workspace_sizes():
     assert 0 < small < big
     assert fp4.fp4_root_ns_workspace_bytes(8192, 3072, 5) == big + 3072 * 8192 * 4  # tall: X lives in the workspace
     both = fp4.fp4_root_ns_batched_workspace_bytes([(128, 256), (3072, 8192)], 5)
-    assert both >= small + big and both < small + big + (1 << 16)  # one workspace per matrix + tables
+    assert both >= small + big and both < small + big + (1 << 16)  # one workspace per matrix
+    # flag bits the library does not know are an error, not ignored: the size query answers 0
+    assert fp4.fp4_root_ns_workspace_bytes(128, 256, 5, 16) == 0
+    assert fp4.fp4_root_ns_workspace_bytes(128, 256, 5, 0xABCD0000) == 0
+    assert fp4.fp4_root_ns_batched_workspace_bytes([(128, 256)], 5, 1 << 20) == 0
     lay = fp4.fp4_root_ns_workspace_layout(512, 256, 5)
     offs = [lay.header, lay.scalars, lay.X, lay.A, lay.qX_codes, lay.qX_scales, lay.qXt_codes[0],
             lay.qXt_scales[0], lay.qXt_codes[1], lay.qXt_scales[1], lay.qA_codes, lay.qA_scales,

@@ -431,3 +431,25 @@ def test_bf16_storage_is_a_small_perturbation_and_leaves_the_first_iteration_alo
     b5, f5 = oracle.root_ns(g, steps=5), oracle.root_ns(g, steps=5, store_bf16=True)
     assert abs(err(f5) - err(b5)) < 0.01 and not np.array_equal(b5, f5)
     assert f5.dtype == np.float32 and np.any(oracle.bf16_round(f5) != f5)      # the result is not rounded to BF16
+
+
+@pytest.mark.parametrize("opts", [dict(), dict(rht=True, four_six=True, seed=9)])
+def test_single_iteration_entry_equals_the_whole_step(opts):
+    """orc_ns_iteration (one iteration from a state handed in, used to teacher-force later iterations)
+    runs the same code as the loop of orc_root_ns: started from the whole step's X after iteration 0
+    and the scalars the step derives there, it must return the whole step's iteration 1 bit for bit."""
+    G = workloads.gradient_like(128, 384, seed=3)
+    _, tr0 = oracle.root_ns(G, steps=2, trace_iter=0, **opts)
+    out2, tr1 = oracle.root_ns(G, steps=2, trace_iter=1, **opts)
+    X1 = tr0["X_out"]
+    a = oracle.root_coeffs(128, 384)[0]
+    widen = np.float32(4.0 if opts.get("rht") else 1.0)
+    bound = np.float32(4.0) * np.float32(abs(a)) * np.float32(tr0["amax_in"])
+    sg1 = oracle.tensor_scale_predicted(widen * bound)
+    assert sg1 == tr1["sg_X"] and np.float32(np.abs(X1).max()) == np.float32(tr1["amax_in"])
+    X2, amax2, sg2, tr = oracle.ns_iteration(X1, 1, tr1["amax_in"], sg1, last=True, **opts)
+    assert np.array_equal(X2, out2)
+    for key in ("A", "S", "B", "qA_codes", "qA_scales", "qB_codes", "qB_scales", "qX_codes", "qXt_scales"):
+        assert np.array_equal(tr[key], tr1[key]), key
+    assert tr["sg_A"] == tr1["sg_A"] and tr["sg_B"] == tr1["sg_B"]
+    assert amax2 == np.float32(np.abs(out2).max())

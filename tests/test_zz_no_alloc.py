@@ -12,6 +12,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 import paper_2607_04422_b200 as fp4
 from paper_2607_04422_b200 import workloads
 from paper_2607_04422_b200.binding import FP4_STATIC_SCRATCH_BYTES
@@ -46,6 +47,10 @@ def test_static_scratch_matches_workspace_call_twice_in_a_row():
             got = out.cpu().numpy()
             rel = np.linalg.norm(got.astype(np.float64) - w) / np.linalg.norm(w.astype(np.float64))
             assert rel <= 2e-3 and np.array_equal(got, w), (round_, g.shape, rel)
+    # and against the CPU oracle, like every other parity test of the step
+    g, k = cases[1]
+    ref = oracle.root_ns(g, steps=k).astype(np.float64)
+    assert np.linalg.norm(got.astype(np.float64) - ref) / np.linalg.norm(ref) <= 2e-3
 
 
 def test_static_scratch_refuses_what_does_not_fit():
