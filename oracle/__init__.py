@@ -103,6 +103,8 @@ def lib():
         L.orc_root_ns.argtypes = [_f32p, C.c_int64, C.c_int64, C.c_int, C.POINTER(OrcParams),
                                   _f32p, C.POINTER(OrcTrace)]
         L.orc_root_ns.restype = C.c_int
+        L.orc_root_param_update.argtypes = [_u16p, _f32p, C.c_int64, C.c_float, C.c_float, C.c_float]
+        L.orc_root_param_update.restype = None
         L.orc_sr_e2m1x4.argtypes = [_f32p, C.c_uint32]; L.orc_sr_e2m1x4.restype = C.c_uint16
         L.orc_ns_iteration.argtypes = [_f32p, C.c_int64, C.c_int64, C.c_int, C.c_int, C.c_float, C.c_float,
                                        C.POINTER(OrcParams), _f32p, _f32p, _f32p, C.POINTER(OrcTrace)]
@@ -191,6 +193,16 @@ def bf16_round(x):
 def splitmix64_at(seed, idx):
     """Output number idx (from 0) of the splitmix64 generator seeded with `seed`."""
     return int(lib().orc_splitmix64_at(int(seed), int(idx)))
+
+
+def root_param_update(W_bits, O, lr, weight_decay=0.0, scale=1.0):
+    """Root's parameter update on BF16 weights (bit patterns, uint16): returns the new bit patterns."""
+    W = np.ascontiguousarray(W_bits, dtype=np.uint16).copy()
+    O_, op = _f32(O)
+    assert W.shape == O_.shape
+    lib().orc_root_param_update(W.ctypes.data_as(_u16p), op, W.size, float(np.float32(lr)),
+                                float(np.float32(weight_decay)), float(np.float32(scale)))
+    return W
 
 
 def sr_e2m1x4(y4, word: int) -> int:

@@ -773,6 +773,26 @@ int orc_root_ns(const float* G, int64_t m, int64_t n, int steps, const orc_param
   return 0;
 }
 
+// Root's parameter update (Section 3.4: the orthogonalised update is applied to the projection;
+// Section 3.3: weights are kept in BF16 without an FP32 master copy).  The paper gives no formula
+// beyond "other hyperparameters follow Root"; the reading taken is decoupled weight decay and a
+// step along the orthogonalised matrix O = X_k scaled by lr * scale, where the shape factor `scale`
+// (Muon-style optimisers use one such as sqrt(max(1, m/n))) is the caller's:
+//   w2 = fl( fl(w * fl(1 - fl(lr * wd))) - fl(fl(lr * scale) * o) ),   W = BF16(w2), nearest even.
+// W: n BF16 bit patterns, in place; O: n FP32 values in the same (row-major, m x n) order.
+void orc_root_param_update(uint16_t* W, const float* O, int64_t n, float lr, float weight_decay, float scale) {
+  const float t = lr * weight_decay;
+  const float decay = 1.0f - t;
+  const float step = lr * scale;
+  for (int64_t i = 0; i < n; ++i) {
+    const float w = bf16_from_bits(W[i]);
+    const float a = w * decay;
+    const float b = step * O[i];
+    const float w2 = a - b;
+    W[i] = bf16_bits(bf16_round(w2));
+  }
+}
+
 // Stochastic rounding of four values with one 32-bit random word (the rule of the momentum state,
 // Section 3.3): element e takes the bits sr_bits_of_word assigns to it; result = four nibbles,
 // element 0 in bits 3:0.

@@ -453,3 +453,45 @@ def test_single_iteration_entry_equals_the_whole_step(opts):
         assert np.array_equal(tr[key], tr1[key]), key
     assert tr["sg_A"] == tr1["sg_A"] and tr["sg_B"] == tr1["sg_B"]
     assert amax2 == np.float32(np.abs(out2).max())
+
+
+# ---- Root's parameter update on BF16 weights (Section 3.4 / 3.3; the formula is a reading) -----
+def _bf16(x):
+    return oracle.bf16_bits(oracle.bf16_round(np.asarray(x, np.float32)))
+
+
+def test_param_update_hand_worked_values():
+    # w = 1, no decay, step 2^-9: 1 - 2^-9 lies halfway between the BF16 neighbours 1 - 2^-8 and 1: ties to even -> 1
+    W = oracle.root_param_update(_bf16([1.0]), np.float32([1.0]), lr=2.0 ** -9, weight_decay=0.0, scale=1.0)
+    assert oracle.bf16_to_f32(W)[0] == 1.0
+    # a step of 3 * 2^-9 from 1: 1 - 3 * 2^-9 is halfway between 1 - 2^-7 and 1 - 2^-8: ties to even -> 1 - 2^-7
+    W = oracle.root_param_update(_bf16([1.0]), np.float32([3.0]), lr=2.0 ** -9, weight_decay=0.0, scale=1.0)
+    assert oracle.bf16_to_f32(W)[0] == 1.0 - 2.0 ** -7
+    # decay alone: 2 * (1 - 0.5 * 0.5) = 1.5 exactly
+    W = oracle.root_param_update(_bf16([2.0]), np.float32([0.0]), lr=0.5, weight_decay=0.5, scale=1.0)
+    assert oracle.bf16_to_f32(W)[0] == 1.5
+    # the shape factor multiplies the step: 0.25 * 4 * 0.5 = 0.5 off 3 -> 2.5
+    W = oracle.root_param_update(_bf16([3.0]), np.float32([0.5]), lr=0.25, weight_decay=0.0, scale=4.0)
+    assert oracle.bf16_to_f32(W)[0] == 2.5
+    # sign of the step: a negative update entry raises the weight
+    W = oracle.root_param_update(_bf16([0.0]), np.float32([-1.0]), lr=0.125, weight_decay=0.3, scale=1.0)
+    assert oracle.bf16_to_f32(W)[0] == 0.125
+    # nothing to do: lr = 0 leaves every representable weight as it is
+    w0 = _bf16(np.random.default_rng(0).standard_normal(64).astype(np.float32))
+    assert np.array_equal(oracle.root_param_update(w0, np.ones(64, np.float32), lr=0.0, weight_decay=0.1), w0)
+
+
+def test_param_update_against_fp64():
+    rng = np.random.default_rng(5)
+    w = oracle.bf16_to_f32(_bf16(rng.standard_normal(4096).astype(np.float32) * 0.05))
+    o = (rng.standard_normal(4096) * 0.02).astype(np.float32)
+    lr, wd, sc = 0.02, 0.1, 1.6
+    got = oracle.bf16_to_f32(oracle.root_param_update(_bf16(w), o, lr, wd, sc)).astype(np.float64)
+    exact = w.astype(np.float64) * (1.0 - lr * wd) - lr * sc * o.astype(np.float64)
+    # BF16 keeps 8 significant bits: half an ulp is at most 2^-8 of the value; the FP32 roundings add ~2^-22
+    assert np.all(np.abs(got - exact) <= np.abs(exact) * (2.0 ** -8 + 2.0 ** -20) + 1e-40)
+    assert np.abs(got - exact).mean() < np.abs(exact).mean() * 2.0 ** -9          # and half of that on average
+    # and it is the nearest BF16 of the FP32 value the formula gives
+    t = np.float32(1.0) - np.float32(lr) * np.float32(wd)
+    w2 = w * t - (np.float32(lr) * np.float32(sc)) * o
+    assert np.array_equal(oracle.root_param_update(_bf16(w), o, lr, wd, sc), oracle.bf16_bits(oracle.bf16_round(w2)))
