@@ -79,6 +79,10 @@ typedef enum {
  * really are 2-byte tensors; otherwise they stay FP32 tensors that hold BF16-rounded values
  * (same results, no traffic saved). */
 #define FP4_FLAG_STORE_BF16 8u
+/* With fp4_ns_params.weights: the FP32 result is not written (the parameter update is all the caller
+ * wants).  `out` is still required - it is the working copy of X during the iterations of a wide matrix -
+ * and its contents are unspecified afterwards. */
+#define FP4_FLAG_NO_OUT 16u
 #define FP4_QUANT_SIGNS(mask) ((uint32_t)(mask) << 16)
 
 /* Parameters of the step.  Pass NULL for the defaults noted on each field. */
@@ -101,6 +105,19 @@ typedef struct {
                           skips its first pass over the matrix.  The counters must describe
                           exactly the matrix passed as G; they are consumed: zero when the step
                           has run.  Ignored when the clip is disabled.                        */
+  uint16_t* const* weights;  /* NULL (default), or a host array with one entry per matrix of the call:
+                          NULL, or the device address of that matrix's parameter, m x n BF16
+                          row-major (16-byte aligned), which receives Root's update in the same
+                          call (Section 3.4: the orthogonalised matrix is applied to the
+                          projection; Section 3.3: BF16 weights, no FP32 master copy):
+                            W <- BF16( fl(W * fl(1 - fl(lr * weight_decay)))
+                                       - fl(fl(lr * update_scale) * X_steps) ),  nearest even,
+                          fused into the epilogue of the last product (into the final transpose for
+                          a tall matrix), so X_steps is not read back from memory.             */
+  float lr;            /* with weights: learning rate                                        */
+  float weight_decay;  /* with weights: decoupled decay                                      */
+  float update_scale;  /* with weights: the shape factor Root-style optimisers put on the
+                          orthogonalised step (e.g. sqrt(max(1, m/n))); the caller's choice     */
 } fp4_ns_params;
 
 const char* fp4_status_string(fp4_status s);

@@ -19,6 +19,7 @@ FP4_FLAG_KEEP_OPERANDS = 1
 FP4_FLAG_RHT = 2
 FP4_FLAG_FOUR_SIX = 4
 FP4_FLAG_STORE_BF16 = 8
+FP4_FLAG_NO_OUT = 16
 FP4_MOM_FLAG_SR = 1
 STATUS_NAMES = {0: "FP4_OK", 1: "FP4_ERR_INVALID_ARG", 2: "FP4_ERR_SHAPE", 3: "FP4_ERR_ALIGNMENT",
                 4: "FP4_ERR_WORKSPACE", 5: "FP4_ERR_ARCH", 6: "FP4_ERR_CUDA", 7: "FP4_ERR_DEVICE_TIMEOUT",
@@ -43,10 +44,12 @@ class NsParams(C.Structure):
     """fp4_ns_params"""
     _fields_ = [("a", C.c_float), ("b", C.c_float), ("c", C.c_float), ("clip_quantile", C.c_float),
                 ("eps", C.c_float), ("flags", C.c_uint32), ("max_group", C.c_uint32), ("seed", C.c_uint64),
-                ("top_hist", C.POINTER(C.c_void_p))]
+                ("top_hist", C.POINTER(C.c_void_p)), ("weights", C.POINTER(C.c_void_p)),
+                ("lr", C.c_float), ("weight_decay", C.c_float), ("update_scale", C.c_float)]
 
     @classmethod
-    def make(cls, abc=None, clip_quantile=0.99, eps=1e-7, flags=0, max_group=0, seed=0, top_hist=None):
+    def make(cls, abc=None, clip_quantile=0.99, eps=1e-7, flags=0, max_group=0, seed=0, top_hist=None,
+             weights=None, lr=0.0, weight_decay=0.0, update_scale=1.0):
         p = cls()
         if abc is None:
             p.a = p.b = p.c = float("nan")
@@ -60,6 +63,12 @@ class NsParams(C.Structure):
             arr = (C.c_void_p * len(top_hist))(*[h.data_ptr() if h is not None else None for h in top_hist])
             p._top_hist_keepalive = arr
             p.top_hist = C.cast(arr, C.POINTER(C.c_void_p))
+        if weights is not None:
+            # one entry per matrix of the call: a BF16 tensor of the matrix's shape, or None
+            arr = (C.c_void_p * len(weights))(*[w.data_ptr() if w is not None else None for w in weights])
+            p._weights_keepalive = arr
+            p.weights = C.cast(arr, C.POINTER(C.c_void_p))
+        p.lr, p.weight_decay, p.update_scale = float(lr), float(weight_decay), float(update_scale)
         return p
 
 

@@ -236,8 +236,21 @@ __device__ unsigned long long g_trace[160 * 18 * 8];
 // warp index, known to the compiler to be the same in all lanes
 __device__ __forceinline__ int uniform_warp_index() { return __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0); }
 
+// 32 bytes per lane, global memory
+__device__ __forceinline__ void ldg256(const void* p, uint32_t (&r)[8]) {
+  asm volatile("ld.global.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "l"(p));
+  asm volatile("ld.global.v4.b32 {%0, %1, %2, %3}, [%4+16];" : "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]) : "l"(p));
+}
+__device__ __forceinline__ void stg256(void* p, const uint32_t (&r)[8]) {
+  asm volatile("st.global.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]) : "memory");
+  asm volatile("st.global.v4.b32 [%0+16], {%1, %2, %3, %4};" ::"l"(p), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]) : "memory");
+}
+
 // BH: instantiation with BF16 storage of the FP32 tiles (args.aux_h / args.out_h may be set)
-template <int MODE, bool PF, bool BH>
+// UPD: the last G3 stage of a call that also applies Root's parameter update (args.update): every lane
+//   loads the 16 BF16 weights under its row of a chunk (one 32-byte sector, fetched a chunk ahead),
+//   forms W * decay - step * X+ from the values it holds and stores the sector back.
+template <int MODE, bool PF, bool BH, bool UPD = false>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
 k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ GemmLaunch args) {
   extern __shared__ uint8_t smem_raw[];
@@ -258,7 +271,7 @@ k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ Ge
   const int num_kb = args.K / BK;
   constexpr bool HAS_AUX = (MODE == kG2 || MODE == kG3);
   constexpr bool STORE_F32 = (MODE == kPlain || MODE == kG1 || MODE == kG3);
-  const bool do_q = (MODE != kPlain) && args.write_q;
+  const bool do_q = (MODE != kPlain) && !UPD && args.write_q;  // the update variant is launched without quantised outputs
   // Measurement of the tensor-pipe ceiling (plain product only): no operand is fetched, the MMAs run on
   // whatever the stages hold.
   const bool dry = (MODE == kPlain) && args.dry_operands != 0;
@@ -510,7 +523,9 @@ k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ Ge
       const int cg = x64 / (TEAM_CHUNKS * CHUNK) & 3;                   // 64-column group within the tile
       const int bj = tj * 2 + (cg >> 1);                                // 128-column block of this warp's columns
       const bool mirror = do_q && !below && (MODE == kG3 || (sym && bi != bj));
-      const bool stage = (STORE_F32 && !hout) || mirror;
+      // the FP32 (or BF16) result leaves by TMA - unless the caller wants the parameter update only
+      const bool store_out = STORE_F32 && !(UPD && args.no_out && pr->W != nullptr);
+      const bool stage = (store_out && !hout) || mirror;
       const bool rows_in = y32 < pr->out_rows;                          // else: zero padding of the work shape
       TR_COUNT(6)
       TR_BEGIN
@@ -561,6 +576,13 @@ k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ Ge
       const uint32_t tm_acc = tm_lane + par * ACC1_COL + cg * (TEAM_CHUNKS * CHUNK);
       uint32_t sfw = 0;
       uint32_t acc[16];
+      // parameter update: this lane's row of the weight under the tile, one 32-byte piece per chunk
+      uint16_t* wrow = nullptr;
+      uint32_t wnext[8];
+      if (UPD) {
+        if (pr->W && rows_in && y32 + lane < pr->out_rows) wrow = pr->W + ((int64_t)y32 + lane) * pr->W_ld + x64;
+        if (wrow && x64 + flip * CHUNK < pr->out_cols) ldg256(wrow + flip * CHUNK, wnext);
+      }
       tc_ld16_issue(tm_acc + flip * CHUNK, acc);
 #pragma unroll
       for (int i = 0; i < TEAM_CHUNKS; ++i) {
@@ -648,6 +670,23 @@ k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ Ge
           __syncwarp();
           if (lane == 0) mbar_arrive_cluster(acc_empty_leader);  // done with the buffer
         }
+        if (UPD) {
+          uint32_t wcur[8];
+#pragma unroll
+          for (int q = 0; q < 8; ++q) wcur[q] = wnext[q];
+          const bool upd_here = wrow && xcol < pr->out_cols;
+          if (i + 1 < TEAM_CHUNKS) {
+            const int e1 = (i + 1) ^ flip;
+            if (wrow && x64 + e1 * CHUNK < pr->out_cols) ldg256(wrow + e1 * CHUNK, wnext);
+          }
+          if (upd_here) {
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+              wcur[q] = cvt_bf16x2(param_update_value(bf16_lo(wcur[q]), v[2 * q], args.upd_decay, args.upd_step),
+                                   param_update_value(bf16_hi(wcur[q]), v[2 * q + 1], args.upd_decay, args.upd_step));
+            stg256(wrow + e * CHUNK, wcur);
+          }
+        }
         uint32_t hw_out[8];  // the row rounded to BF16 (before a quantiser option may transform v in place)
         if (BH && hout) {
 #pragma unroll
@@ -659,10 +698,10 @@ k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ Ge
 #pragma unroll
           for (int j = 0; j < 4; ++j)
             sts128((row_addr + boff) ^ (j << 4), v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-          if (STORE_F32 && !hout) fence_proxy_async_smem();
+          if (store_out && !hout) fence_proxy_async_smem();
         }
         __syncwarp();
-        if (STORE_F32 && !hout && send && lane == 0) {
+        if (store_out && !hout && send && lane == 0) {
           tma_store_2d_s(&pr->tmOut, xcol, y32, area + boff);
           bulk_commit();
         }
@@ -674,7 +713,7 @@ k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ Ge
 #pragma unroll
           for (int k = 0; k < 16; ++k) w[k] = lds32(col_addr[(k >> 1) & 3] + boff + k * 64);
         }
-        if (BH && hout) {
+        if (BH && hout && store_out) {
           // BF16 storage: the rounded rows take the place of the FP32 block once it has been read back,
           // 32 bytes per row at the start of the buffer
           __syncwarp();
@@ -768,14 +807,14 @@ k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ Ge
   if (threadIdx.x == 0 && bars->abort_flag) report_timeout(args.status);
 }
 
-template <int MODE, bool PF, bool BH>
+template <int MODE, bool PF, bool BH, bool UPD = false>
 cudaError_t launch_pair_mode(const ProblemPack& pack, const GemmLaunch& L, int sms, cudaStream_t st) {
   const int tpp = L.symmetric ? L.tiles_n * (L.tiles_n + 1) / 2 : L.tiles_m * L.tiles_n;
   const int num_tiles = tpp * L.num_problems;
   int pairs = sms / 2;
   if (pairs > num_tiles) pairs = num_tiles;
   count_launches(1);
-  k_gemm_pair<MODE, PF, BH><<<2 * pairs, NTHREADS, SMEM_BYTES, st>>>(pack, L);
+  k_gemm_pair<MODE, PF, BH, UPD><<<2 * pairs, NTHREADS, SMEM_BYTES, st>>>(pack, L);
   return cudaGetLastError();
 }
 
@@ -807,6 +846,8 @@ cudaError_t gemm_pair_set_attributes() {
   if ((e = cudaFuncSetAttribute(k_gemm_pair<kG3, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
   if ((e = cudaFuncSetAttribute(k_gemm_pair<kG3, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
   if ((e = cudaFuncSetAttribute(k_gemm_pair<kG3, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG3, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG3, false, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
   return cudaSuccess;
 }
 
@@ -825,6 +866,12 @@ cudaError_t launch_gemm_pair(GemmMode mode, const ProblemPack& pack, const GemmL
                   : launch_pair_mode<M, true, false>(pack, L, sms, st))                  \
             : (bh ? launch_pair_mode<M, false, true>(pack, L, sms, st)                   \
                   : launch_pair_mode<M, false, false>(pack, L, sms, st))
+  if (launch.update) {
+    // the last G3 stage with the parameter update: nothing is quantised there (write_q = 0)
+    if (mode != kG3 || launch.write_q) return cudaErrorInvalidValue;
+    return bh ? launch_pair_mode<kG3, false, true, true>(pack, L, sms, st)
+              : launch_pair_mode<kG3, false, false, true>(pack, L, sms, st);
+  }
   switch (mode) {
     case kPlain: return launch_pair_mode<kPlain, false, false>(pack, L, sms, st);
     case kG1: FP4_PAIR_CASE(kG1);

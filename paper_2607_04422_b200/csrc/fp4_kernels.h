@@ -83,6 +83,8 @@ struct alignas(64) GemmProblem {
   int out_rows, out_cols;    // extent of the matrix behind tmOut (chunks that start outside it are not stored)
   void* out_direct;          // out_h == 2: the FP32 tensor the epilogue warps store the rounded result to
   int64_t out_direct_ld;     //   (row-major, leading dimension in elements)
+  uint16_t* W;               // kG3 with launch.update: the BF16 parameter (same shape and orientation as the
+  int64_t W_ld;              //   result, row-major, leading dimension in elements) updated with the result; or null
 };
 
 // The problems of one launch travel as a kernel parameter (descriptors in parameter space need no
@@ -106,6 +108,10 @@ struct GemmLaunch {
   int aux_h;           // the combined tile is read from tmH (BF16)
   int out_h;           // 0: FP32 result by TMA store; 1: rounded to BF16, staged and stored through tmH (CTA-pair
                        // kernel); 2: rounded to BF16, stored as FP32 by the epilogue warps (single-CTA kernel)
+  int update;          // kG3, CTA-pair kernel, last iteration: Root's parameter update W <- BF16(W * upd_decay -
+  float upd_decay;     //   upd_step * X+) on every problem whose W is set, in the epilogue
+  float upd_step;
+  int no_out;          // with update: the FP32 result is not stored
   int dry_operands;    // kPlain, CTA-pair kernel: measurement of the tensor-pipe ceiling - no operand is fetched
   NsScalarIdx ix;
   uint32_t* status;
@@ -153,9 +159,22 @@ struct PrologueItem {
 // count matrices that share the shape (s, l) and the clip / eps parameters
 cudaError_t launch_prologue_group(const PrologueItem* items, int count, int write_q, const QuantOpts& q,
                                   cudaStream_t st);
-// out (l0 x s0, row-major) = the leading s0 x l0 part of X^T, X being s x l with row pitch l
+// Root's parameter update on BF16 weights: decay = fl(1 - fl(lr * wd)), step = fl(lr * scale),
+// w <- BF16(fl(fl(w * decay) - fl(step * o))).
+struct ParamUpdate {
+  uint16_t* W;     // null: no update
+  float decay, step;
+  int no_out;      // where the update is fused with the store of the FP32 result: skip that store
+};
+__device__ __forceinline__ float param_update_value(float w, float o, float decay, float step) {
+  return __fsub_rn(__fmul_rn(w, decay), __fmul_rn(step, o));
+}
+// out (l0 x s0, row-major) = the leading s0 x l0 part of X^T, X being s x l with row pitch l; with
+// upd.W set, W (l0 x s0 like out) takes the update from the same values
 cudaError_t launch_transpose_out(const float* X, int64_t s, int64_t l, float* out, int64_t s0, int64_t l0,
-                                 cudaStream_t st);
+                                 const ParamUpdate& upd, cudaStream_t st);
+// W (n elements) updated from the FP32 matrix O of the same layout
+cudaError_t launch_param_update(const float* O, int64_t n, const ParamUpdate& upd, int sms, cudaStream_t st);
 cudaError_t prologue_set_attributes();
 
 cudaError_t gemm_set_attributes();

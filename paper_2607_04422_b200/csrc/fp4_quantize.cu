@@ -101,7 +101,7 @@ __global__ void __launch_bounds__(256) k_quantize_rows_opts(const float* __restr
 // shared memory, 128-bit loads along the rows of X and 128-bit stores along the rows of out
 // (s0 and l0 are multiples of 16, so a 16-byte piece is all inside or all outside).
 __global__ void __launch_bounds__(256) k_transpose_out(const float* __restrict__ X, int64_t l, float* __restrict__ out,
-                                                       int64_t s0, int64_t l0) {
+                                                       int64_t s0, int64_t l0, const ParamUpdate upd) {
   __shared__ float t[64][65];
   const int64_t r0 = (int64_t)blockIdx.y * 64, c0 = (int64_t)blockIdx.x * 64;  // tile origin in X
   const int q = threadIdx.x & 15, row = threadIdx.x >> 4;                      // 16 pieces per row, 16 rows per sweep
@@ -115,9 +115,38 @@ __global__ void __launch_bounds__(256) k_transpose_out(const float* __restrict__
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
     const int c = row + 16 * j;  // column of X = row of out
-    if (c0 + c < l0 && r0 + 4 * q < s0)
-      *reinterpret_cast<float4*>(out + (c0 + c) * s0 + r0 + 4 * q) =
-          make_float4(t[4 * q][c], t[4 * q + 1][c], t[4 * q + 2][c], t[4 * q + 3][c]);
+    if (c0 + c < l0 && r0 + 4 * q < s0) {
+      const int64_t at = (c0 + c) * s0 + r0 + 4 * q;
+      const float4 o = make_float4(t[4 * q][c], t[4 * q + 1][c], t[4 * q + 2][c], t[4 * q + 3][c]);
+      if (!(upd.W && upd.no_out)) *reinterpret_cast<float4*>(out + at) = o;
+      if (upd.W) {
+        // Root's parameter update from the values on their way out (the parameter has the caller's
+        // orientation, like `out`)
+        uint2* wp = reinterpret_cast<uint2*>(upd.W + at);
+        const uint2 w = *wp;
+        *wp = make_uint2(cvt_bf16x2(param_update_value(bf16_lo(w.x), o.x, upd.decay, upd.step),
+                                    param_update_value(bf16_hi(w.x), o.y, upd.decay, upd.step)),
+                         cvt_bf16x2(param_update_value(bf16_lo(w.y), o.z, upd.decay, upd.step),
+                                    param_update_value(bf16_hi(w.y), o.w, upd.decay, upd.step)));
+      }
+    }
+  }
+}
+
+// W <- update(W, O) elementwise, 8 elements per thread
+__global__ void __launch_bounds__(256) k_param_update(const float* __restrict__ O, int64_t n8, const ParamUpdate upd) {
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n8; i += (int64_t)gridDim.x * blockDim.x) {
+    const float4 a = __ldg(reinterpret_cast<const float4*>(O) + 2 * i), b = __ldg(reinterpret_cast<const float4*>(O) + 2 * i + 1);
+    uint4* wp = reinterpret_cast<uint4*>(upd.W) + i;
+    const uint4 w = *wp;
+    *wp = make_uint4(cvt_bf16x2(param_update_value(bf16_lo(w.x), a.x, upd.decay, upd.step),
+                                param_update_value(bf16_hi(w.x), a.y, upd.decay, upd.step)),
+                     cvt_bf16x2(param_update_value(bf16_lo(w.y), a.z, upd.decay, upd.step),
+                                param_update_value(bf16_hi(w.y), a.w, upd.decay, upd.step)),
+                     cvt_bf16x2(param_update_value(bf16_lo(w.z), b.x, upd.decay, upd.step),
+                                param_update_value(bf16_hi(w.z), b.y, upd.decay, upd.step)),
+                     cvt_bf16x2(param_update_value(bf16_lo(w.w), b.z, upd.decay, upd.step),
+                                param_update_value(bf16_hi(w.w), b.w, upd.decay, upd.step)));
   }
 }
 
@@ -150,11 +179,19 @@ cudaError_t launch_quantize(const float* x, int64_t rows, int64_t cols, uint8_t*
 }
 
 cudaError_t launch_transpose_out(const float* X, int64_t s, int64_t l, float* out, int64_t s0, int64_t l0,
-                                 cudaStream_t st) {
+                                 const ParamUpdate& upd, cudaStream_t st) {
   dim3 grid((unsigned)((l0 + 63) / 64), (unsigned)((s0 + 63) / 64));
   (void)s;
   count_launches(1);
-  k_transpose_out<<<grid, 256, 0, st>>>(X, l, out, s0, l0);
+  k_transpose_out<<<grid, 256, 0, st>>>(X, l, out, s0, l0, upd);
+  return cudaGetLastError();
+}
+
+// n is a multiple of 256 (both dimensions are multiples of 16)
+cudaError_t launch_param_update(const float* O, int64_t n, const ParamUpdate& upd, int sms, cudaStream_t st) {
+  if (!upd.W) return cudaSuccess;
+  count_launches(1);
+  k_param_update<<<grid_for(n / 8, 256, sms), 256, 0, st>>>(O, n / 8, upd);
   return cudaGetLastError();
 }
 

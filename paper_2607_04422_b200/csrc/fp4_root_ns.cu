@@ -82,7 +82,8 @@ inline bool shape_ok(int64_t v) { return v >= 128 && v % 128 == 0 && v <= (1 << 
 inline bool ns_shape_ok(int64_t v) { return v >= 16 && v % 16 == 0 && v <= (1 << 20); }
 inline int64_t pad128(int64_t v) { return (v + 127) / 128 * 128; }
 // flag bits the Newton-Schulz entry points know
-constexpr uint32_t kNsFlags = FP4_FLAG_KEEP_OPERANDS | FP4_FLAG_RHT | FP4_FLAG_FOUR_SIX | FP4_FLAG_STORE_BF16;
+constexpr uint32_t kNsFlags =
+    FP4_FLAG_KEEP_OPERANDS | FP4_FLAG_RHT | FP4_FLAG_FOUR_SIX | FP4_FLAG_STORE_BF16 | FP4_FLAG_NO_OUT;
 
 // 2-D map over a row-major byte matrix (NVFP4 codes): box = one operand stage (64 or 128 bytes
 // x 128 rows), swizzled over the box width.
@@ -173,6 +174,9 @@ void default_params(fp4_ns_params* p) {
   p->max_group = 0;
   p->seed = 0;
   p->top_hist = nullptr;
+  p->weights = nullptr;
+  p->lr = p->weight_decay = 0.0f;
+  p->update_scale = 1.0f;
 }
 
 // The 16 signs of the j-th random Hadamard matrix of a call: splitmix64 on seed + j.
@@ -289,6 +293,7 @@ struct MatrixCtx {
   bool store_x0;              // the prologue writes X0 in FP32
   int64_t x_rows, x_cols;     // extent (and row pitch) of X
   uint32_t* hist_top;         // the caller's first-pass histogram of G, or null
+  uint16_t* W;                // the BF16 parameter that takes Root's update in this call, or null
 };
 
 fp4_status prepare_matrix(const DeviceInfo* d, const float* G, float* out, int64_t m, int64_t n, int steps,
@@ -299,6 +304,7 @@ fp4_status prepare_matrix(const DeviceInfo* d, const float* G, float* out, int64
   const int64_t s = c->pl.s, l = c->pl.l;
   c->G = G; c->out = out; c->ws = ws;
   c->hist_top = nullptr;
+  c->W = nullptr;
   c->X = c->pl.tall ? reinterpret_cast<float*>(ws + L.X) : out;
   // extent of X: the padded work shape in the workspace, the caller's shape in `out` (TMA fills what
   // lies outside with zeros on loads and drops it on stores)
@@ -393,6 +399,20 @@ fp4_status run_group(const DeviceInfo* d, MatrixCtx* mats, int count, int steps,
                      uint32_t* status, bool clear_first_status, cudaStream_t st) {
   if (count < 1 || count > kPackMax) return FP4_ERR_INVALID_ARG;
   const bool keep = (p->flags & FP4_FLAG_KEEP_OPERANDS) != 0;
+  ParamUpdate upd;
+  upd.W = nullptr;
+  {
+    // every operation rounded to FP32 on its own (volatile keeps the host compiler from fusing them)
+    volatile float t = p->lr * p->weight_decay;
+    volatile float dec = 1.0f - t;
+    volatile float stp = p->lr * p->update_scale;
+    upd.decay = dec;
+    upd.step = stp;
+  }
+  upd.no_out = (p->flags & FP4_FLAG_NO_OUT) ? 1 : 0;
+  bool any_update = false;
+  for (int i = 0; i < count; ++i) any_update = any_update || mats[i].W != nullptr;
+  std::vector<char> fused_update((size_t)count, 0);
   const NsPlan& pl0 = mats[0].pl;
   const int64_t s = pl0.s, l = pl0.l;
   {
@@ -413,6 +433,19 @@ fp4_status run_group(const DeviceInfo* d, MatrixCtx* mats, int count, int steps,
         const MatrixCtx& c = mats[j < count ? j : 0];
         packs[(size_t)kind].p[j] = kind == 0 ? c.g1 : kind == 1 ? c.g2 : kind == 4 ? c.g3_first : c.g3[kind - 2];
       }
+    }
+    // Root's parameter update: fused into the last G3 stage where the CTA-pair kernel runs it on a
+    // matrix in the caller's orientation and no operand copies are wanted from that stage; into the
+    // final transpose for a tall matrix; a separate elementwise pass otherwise (below).
+    const bool g3_pair = pair_kernel(s / 128, l / 128, s, d->sms, pl0.bf16_mode == 2);
+    if (g3_pair && !keep) {
+      for (int kind = 2; kind < 5; ++kind)
+        for (int j = 0; j < count; ++j)
+          if (mats[j].W && !mats[j].pl.tall) {
+            packs[(size_t)kind].p[j].W = mats[j].W;
+            packs[(size_t)kind].p[j].W_ld = mats[j].pl.n;
+            fused_update[(size_t)j] = 1;
+          }
     }
     GemmLaunch base;
     memset(&base, 0, sizeof(base));
@@ -452,6 +485,11 @@ fp4_status run_group(const DeviceInfo* d, MatrixCtx* mats, int count, int steps,
       L3.q = quant_opts(p, 2 * (uint64_t)k + 2);  // both copies of X_{k+1}
       L3.aux_h = (bmode == 1 && k > 0) ? 1 : 0;   // X_0 is FP32 (or the raw input)
       L3.out_h = last ? 0 : bmode;                 // the result itself is FP32
+      if (last && g3_pair && !keep && any_update) {
+        L3.update = 1;
+        L3.upd_decay = upd.decay; L3.upd_step = upd.step;
+        L3.no_out = upd.no_out;
+      }
       {
         ProfScope ps(FP4_PROF_G3, st);
         if (launch_gemm_auto(kG3, packs[k == 0 ? 4 : 2 + cur], L3, d->sms, st, fs) != cudaSuccess)
@@ -460,9 +498,14 @@ fp4_status run_group(const DeviceInfo* d, MatrixCtx* mats, int count, int steps,
     }
   }
   for (int i = 0; i < count; ++i) {
+    ParamUpdate u = upd;
+    u.W = mats[i].W;
     if (mats[i].pl.tall) {
       ProfScope ps(FP4_PROF_TRANSPOSE, st);
-      if (launch_transpose_out(mats[i].X, s, l, mats[i].out, pl0.s0, pl0.l0, st) != cudaSuccess) return FP4_ERR_CUDA;
+      if (launch_transpose_out(mats[i].X, s, l, mats[i].out, pl0.s0, pl0.l0, u, st) != cudaSuccess) return FP4_ERR_CUDA;
+    } else if (u.W && !fused_update[(size_t)i]) {
+      ProfScope ps(FP4_PROF_TRANSPOSE, st);
+      if (launch_param_update(mats[i].out, mats[i].pl.m * mats[i].pl.n, u, d->sms, st) != cudaSuccess) return FP4_ERR_CUDA;
     }
   }
   return FP4_OK;
@@ -475,6 +518,7 @@ fp4_status run_one(const DeviceInfo* d, const float* G, float* out, int64_t m, i
   fp4_status rc = prepare_matrix(d, G, out, m, n, steps, p, ws, &c);
   if (rc != FP4_OK) return rc;
   if (p->top_hist) c.hist_top = p->top_hist[0];
+  if (p->weights) c.W = p->weights[0];
   return run_group(d, &c, 1, steps, p, reinterpret_cast<uint32_t*>(ws + c.pl.lay.header), clear_status, st);
 }
 
@@ -666,6 +710,7 @@ fp4_status fp4_root_ns_batched(int count, const float* const* G, float* const* o
     rc = prepare_matrix(d, G[i], out[i], m[i], n[i], steps, p, base + off, &ctx[(size_t)i]);
     if (rc != FP4_OK) return rc;
     if (p->top_hist) ctx[(size_t)i].hist_top = p->top_hist[i];
+    if (p->weights) ctx[(size_t)i].W = p->weights[i];
     off += align_up(ctx[(size_t)i].pl.lay.total, 1024);
   }
   uint32_t* status = reinterpret_cast<uint32_t*>(base);  // header of the first matrix
