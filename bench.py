@@ -34,10 +34,10 @@ UNIT = "matrices/s"
 FP4_NOMINAL_TFLOPS = 9000.0  # dense NVFP4, nominal
 FP4_OVER_BF16 = 4.0          # nominal ratio of the dense FP4 and BF16 tensor peaks
 # DRAM bytes per element of X that one G3 launch moves (dram__bytes_read + dram__bytes_write of
-# k_gemm_pair<G3> on one 3072 x 8192 matrix with all quantised outputs written,
-# profiles/k_gemm_pair_3072x8192.md: 217.3 MB for 25.2 M elements); a grouped launch is scaled by
-# the elements it covers
-G3_DRAM_BYTES_PER_ELEMENT = 217.3e6 / (3072 * 8192)
+# k_gemm_pair<3, 0, 0> from an ncu capture of one 3072 x 8192 matrix with all quantised outputs
+# written: 217.0 MB for 25.2 M elements); a grouped launch is scaled by the elements it covers
+G3_DRAM_BYTES_PER_ELEMENT = 217.0e6 / (3072 * 8192)
+G3_KERNEL = "k_gemm_pair<3, 0, 0>"   # MODE = G3, base quantiser, FP32 storage
 
 
 def peaks():
@@ -178,6 +178,45 @@ def cpu_baseline_leg(mats_np, shapes):
             "gflops_algorithmic": alg_sample / dt / 1e9}
 
 
+def small_config_rows(full_cpu: bool):
+    """The single-matrix configurations measured in full on both sides: the oracle on the host cores
+    (whole step, 5 iterations) and fp4_root_ns on the GPU (median of 20 calls after 5 warm-ups).  The
+    256 x 512 and 2048 x 2048 cases take seconds; the 2048 x 8192 pair about a minute of host time
+    and is only run with --full-cpu."""
+    import torch
+    import oracle
+    import paper_2607_04422_b200 as fp4
+    from paper_2607_04422_b200 import workloads
+    cases = [("cfg1 256x512 Gaussian", workloads.config1()), ("cfg2 2048x2048 low-rank + outliers", workloads.config2())]
+    if full_cpu:
+        wide, tall = workloads.config3()
+        cases += [("cfg3 2048x8192 row-lognormal", wide), ("cfg3 8192x2048 row-lognormal", tall)]
+    rows = []
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for name, G_np in cases:
+        m, n = G_np.shape
+        t0 = time.perf_counter()
+        want = oracle.root_ns(G_np, steps=STEPS_NS)
+        cpu_s = time.perf_counter() - t0
+        G = torch.from_numpy(G_np).cuda()
+        out = torch.empty_like(G)
+        ws = torch.empty(fp4.fp4_root_ns_workspace_bytes(m, n, STEPS_NS), dtype=torch.uint8, device="cuda")
+        times = []
+        for it in range(25):
+            e0.record(); fp4.fp4_root_ns(G, out, STEPS_NS, None, ws); e1.record()
+            torch.cuda.synchronize()
+            if it >= 5:
+                times.append(e0.elapsed_time(e1))
+        got = out.cpu().numpy().astype(np.float64)
+        rel = float(np.linalg.norm(got - want) / np.linalg.norm(want))
+        alg, _ = batch_flops([(m, n)])
+        gpu_ms = float(np.median(times))
+        rows.append({"workload": name, "cpu_oracle_s": cpu_s, "cpu_matrices_per_s": 1.0 / cpu_s,
+                     "cpu_gflops_algorithmic": alg / cpu_s / 1e9, "gpu_ms": gpu_ms, "gpu_matrices_per_s": 1e3 / gpu_ms,
+                     "gpu_tflops_algorithmic": alg / gpu_ms / 1e9, "rel_frobenius_vs_oracle": rel})
+    return rows
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -223,8 +262,10 @@ def run_ours(args):
     sampler = ClockSampler(local) if rank == 0 else None
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
+    host_t0 = time.perf_counter()
     for _ in range(args.steps):
         step()
+    host_ms_per_call = (time.perf_counter() - host_t0) * 1e3 / args.steps   # the calls only enqueue work
     e1.record(stream)
     barrier()
     ms = e0.elapsed_time(e1)
@@ -262,6 +303,23 @@ def run_ours(args):
     if fp4.fp4_last_device_status(ws) != 0:
         raise SystemExit("device status after the paper-faithful pass")
 
+    # ---- the same step with BF16 storage of X_k / A_k between the stages (FP4_FLAG_STORE_BF16): a secondary row
+    bf_params = fp4.NsParams.make(flags=fp4.FP4_FLAG_STORE_BF16)
+    ws_bf = torch.empty(fp4.fp4_root_ns_batched_workspace_bytes(shapes, STEPS_NS, fp4.FP4_FLAG_STORE_BF16),
+                        dtype=torch.uint8, device="cuda")
+    for _ in range(2):
+        fp4.fp4_root_ns_batched(Gs, outs, STEPS_NS, bf_params, ws_bf, stream)
+    torch.cuda.synchronize()
+    e0.record(stream)
+    for _ in range(pf_steps):
+        fp4.fp4_root_ns_batched(Gs, outs, STEPS_NS, bf_params, ws_bf, stream)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    bf_ms = e0.elapsed_time(e1) / pf_steps
+    if fp4.fp4_last_device_status(ws_bf) != 0:
+        raise SystemExit("device status after the BF16-storage pass")
+    del ws_bf
+
     # ---- the optimiser step around it: momentum kept in the 5-bit NVFP4 state (stochastic
     # rounding), M_t = mu M_{t-1} + G_t written in FP32 together with the clip's first-pass
     # histogram, then the Root step on M_t with that histogram handed over: a secondary row
@@ -289,7 +347,38 @@ def run_ours(args):
     mr_ms = e0.elapsed_time(e1) / mr_steps
     if fp4.fp4_last_device_status(ws) != 0:
         raise SystemExit("device status after the momentum + Root pass")
-    del m_codes, m_scales, Ms
+    # ---- and with Root's parameter update on BF16 weights: fused into the step (last product's epilogue /
+    # final transpose, FP32 result not stored) against a separate update pass over the stored result
+    Wts = [(torch.randn(G.shape, device="cuda") * 0.05).to(torch.bfloat16) for G in Gs]
+    up_kw = dict(lr=0.02, weight_decay=0.1, update_scale=1.0)
+    fused_params = fp4.NsParams.make(flags=fp4.FP4_FLAG_NO_OUT, top_hist=[hists[i] for i in range(len(Gs))],
+                                     weights=Wts, **up_kw)
+
+    def momentum_root_update_step(t, fused):
+        for i, G in enumerate(Gs):
+            fp4.fp4_momentum_update(G, m_codes[i], m_scales[i], Ms[i], hists[i], 0.95, 1.0, fp4.FP4_MOM_FLAG_SR,
+                                    t, stream)
+        if fused:
+            fp4.fp4_root_ns_batched(Ms, outs, STEPS_NS, fused_params, ws, stream)
+        else:
+            fp4.fp4_root_ns_batched(Ms, outs, STEPS_NS, h_params, ws, stream)
+            for W, o in zip(Wts, outs):      # the separate pass: W <- W * (1 - lr wd) - lr X_k in BF16
+                W.mul_(1.0 - up_kw["lr"] * up_kw["weight_decay"]).add_(o, alpha=-up_kw["lr"])
+
+    mru = {}
+    for fused in (True, False):
+        for t in range(2):
+            momentum_root_update_step(10 + t, fused)
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for t in range(mr_steps):
+            momentum_root_update_step(20 + t, fused)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        mru[fused] = e0.elapsed_time(e1) / mr_steps
+    if fp4.fp4_last_device_status(ws) != 0:
+        raise SystemExit("device status after the momentum + Root + update pass")
+    del m_codes, m_scales, Ms, Wts
 
     # ---- the standalone quantiser on one 8192 x 8192 tensor (HBM-bound: 8.5625 B per element)
     qx = torch.randn((8192, 8192), device="cuda")
@@ -303,6 +392,26 @@ def run_ours(args):
         q_ms.append(e0.elapsed_time(e1))
     q_gbs = 8192 * 8192 * 8.5625 / (min(q_ms[1:]) / 1e3) / 1e9
     del qx, qc, qs
+
+    # ---- tensor-pipe ceiling of the GEMM kernel: the plain product on 8192^3 with the operands of each SM pair
+    # resident in shared memory (fetched once), i.e. MMAs, commits and the FP32 epilogue only; and the same
+    # product with its operand traffic
+    cq = torch.empty((8192, 4096), dtype=torch.uint8, device="cuda")
+    cs = torch.empty(fp4.fp4_scale_bytes(8192, 8192), dtype=torch.uint8, device="cuda")
+    ct = torch.empty(1, device="cuda")
+    fp4.fp4_quantize(torch.randn((8192, 8192), device="cuda"), cq, cs, ct, 0, stream)
+    torch.cuda.synchronize()
+    csg = float(ct.item())
+    cD = torch.empty((8192, 8192), device="cuda")
+    ceil = {}
+    for name, fn in (("resident", fp4.fp4_gemm_nt_resident), ("streamed", fp4.fp4_gemm_nt)):
+        t_ms = []
+        for _ in range(6):
+            e0.record(stream); fn(cq, cs, csg, cq, cs, csg, cD, None, stream); e1.record(stream)
+            torch.cuda.synchronize()
+            t_ms.append(e0.elapsed_time(e1))
+        ceil[name] = 2.0 * 8192 ** 3 / (min(t_ms[1:]) / 1e3) / 1e12
+    del cq, cs, cD
 
     # ---- the momentum step on one 8192 x 8192 matrix (HBM-bound: G in, M out, 5-bit state in
     # and out = 9.25 B per element), with the clip histogram and with stochastic rounding
@@ -461,7 +570,8 @@ def run_ours(args):
     per_launch_ms = dom_ms / max(prof[dom][1], 1)
     achieved = dom_flops / (dom_ms / 1e3) / 1e12
     fp4_peak = pk["bf16_tflops_sustained"] * FP4_OVER_BF16
-    roofline = {"kernel": f"k_gemm<{dom}>", "bound": "tensor", "achieved": achieved, "peak": fp4_peak,
+    kernel_names = {"G1": "k_gemm_pair<1, 0, 0>", "G2": "k_gemm_pair<2, 0, 0>", "G3": G3_KERNEL}
+    roofline = {"kernel": kernel_names[dom], "bound": "tensor", "achieved": achieved, "peak": fp4_peak,
                 "unit": "TFLOP/s", "frac": achieved / fp4_peak,
                 "traffic": (G3_DRAM_BYTES_PER_ELEMENT * sum(m * n for m, n in shapes) * STEPS_NS * prof_steps
                             / max(prof[dom][1], 1)) if dom == "G3" else None,
@@ -470,9 +580,14 @@ def run_ours(args):
                 "avg_launch_ms": per_launch_ms, "launches_profiled": prof[dom][1],
                 "flops_per_launch": dom_flops / max(prof[dom][1], 1),
                 "frac_of_nominal_9pf": achieved / FP4_NOMINAL_TFLOPS,
+                "mma_only_ceiling_tflops": ceil["resident"], "frac_of_mma_only_ceiling": achieved / ceil["resident"],
+                "ceiling_note": "fp4_gemm_nt on 8192^3 with each SM pair's operand stages resident in shared memory "
+                                "(no operand traffic): what the MMA issue, commit and FP32 epilogue of this kernel "
+                                f"reach under the power cap; the same product with operand traffic: {ceil['streamed']:.0f} TFLOP/s",
                 "time_share": shares}
 
     cpu = cpu_baseline_leg(mats_np, shapes)
+    cpu["configs_measured_in_full"] = small_config_rows(args.full_cpu)
     step_s = ms_per_step / 1e3
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
@@ -481,6 +596,11 @@ def run_ours(args):
                                    "(16x 3072x3072, 8x 3072x8192, 4x 8192x3072), 5 NVFP4 Newton-Schulz iterations, "
                                    "one fp4_root_ns_batched call per step",
                        "l2": f"inputs {in_bytes / 1e9:.2f} GB per step, larger than L2; no flush needed",
+                       "coefficients": "stand-in provider (the paper shows Root's values only in a figure): parity unpinned",
+                       "tensor_scales": "in-loop tensor scales are predicted from running maxima (a reading of the "
+                                        "paper's 'FP32 global scale'), shared by oracle and kernels",
+                       "storage": "X_k and A_k kept in FP32 between the stages (headline); BF16 storage is the "
+                                  "secondary row bf16_storage",
                        "parallelism": f"replicas x{world}, no collective"},
             "tflops_algorithmic": alg / step_s / 1e12, "tflops_dense_equivalent": dense / step_s / 1e12,
             "pct_of_nominal_fp4_peak": 100.0 * alg / step_s / 1e12 / FP4_NOMINAL_TFLOPS,
@@ -512,6 +632,15 @@ def run_ours(args):
                                        "(dense, no symmetry, same coefficients); clip and normalisation outside "
                                        "the timed region; compare with our stages G1+G2+G3",
                                "our_ns_loop_ms": ms_per_step * (shares["G1"] + shares["G2"] + shares["G3"])},
+            "host_ms_per_call": host_ms_per_call,
+            "bf16_storage": {"value": len(shapes) / (bf_ms / 1e3), "unit": UNIT, "ms_per_step": bf_ms,
+                             "what": "the same step with FP4_FLAG_STORE_BF16: X_k (k >= 1) and A_k stored in BF16 "
+                                     "between the stages, operand copies and maxima still from the FP32 values"},
+            "momentum_root_update": {"fused_ms_per_step": mru[True], "separate_ms_per_step": mru[False],
+                                     "what": "momentum update, Root step and the BF16 parameter update of all 28 "
+                                             "matrices: update fused into the step (last product's epilogue or the "
+                                             "final transpose, FP32 result not stored) against the step followed "
+                                             "by a separate torch pass W.mul_().add_() per matrix"},
             "rht_four_six": {"value": len(shapes) / (pf_ms / 1e3), "unit": UNIT, "ms_per_step": pf_ms,
                              "what": "the same step with FP4_FLAG_RHT | FP4_FLAG_FOUR_SIX (paper-faithful "
                                      "quantiser options); the headline value uses the base quantiser"},
@@ -528,6 +657,8 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--full-cpu", action="store_true",
+                    help="also time the oracle in full on the 2048 x 8192 pair (about a minute of host time)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -9,9 +9,10 @@
  * General rules
  *   - Every pointer named "device" is a CUDA device pointer on the current device;
  *     every other pointer is host memory that is read before the call returns.
- *   - The caller owns all buffers.  The library keeps no state between calls except
- *     the driver entry point it resolves on first use.  It allocates no device
- *     memory.
+ *   - The caller owns all buffers.  The library allocates no device memory.  Between calls it
+ *     keeps, on the host, the driver entry point it resolves on first use and a bounded cache of
+ *     the TMA descriptors and workspace plans of recent (buffers, shape, parameters)
+ *     combinations, so that a call with the same buffers as an earlier one skips their set-up.
  *   - All work is enqueued on `stream`; no call synchronises the host except
  *     fp4_last_device_status.
  *   - Shapes: for fp4_root_ns, fp4_root_ns_batched and fp4_root_ns_static every matrix
@@ -262,6 +263,16 @@ fp4_status fp4_gemm_nt(const uint8_t* a_codes, const uint8_t* a_scales, float a_
                        uint32_t* device_status /* device, may be NULL: receives
                        FP4_ERR_DEVICE_TIMEOUT if a bounded wait gives up */,
                        cudaStream_t stream);
+
+/* Measurement helper: the same launch as fp4_gemm_nt (same kernel, tiles, instruction stream and epilogue)
+ * in which every pair of SMs fetches only the first operand stages of its first tile and runs all
+ * later MMAs on those resident stages.  Times the tensor-core side of the product without any operand
+ * traffic: the ceiling the benchmark reports beside the nominal peak.  D receives meaningless values.
+ * M, N, K multiples of 256 (else FP4_ERR_SHAPE). */
+fp4_status fp4_gemm_nt_resident(const uint8_t* a_codes, const uint8_t* a_scales, float a_tensor_scale,
+                                const uint8_t* b_codes, const uint8_t* b_scales, float b_tensor_scale,
+                                int64_t M, int64_t N, int64_t K, float* D, uint32_t* device_status,
+                                cudaStream_t stream);
 
 /* ---- first-moment momentum in a 5-bit NVFP4 state ---------------------------------------------
  * Section 3.3 (first-moment recipe: Hadamard mixing, then stochastic rounding and adaptive 4/6

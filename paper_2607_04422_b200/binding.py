@@ -29,6 +29,7 @@ FP4_STATIC_SCRATCH_BYTES = 16 << 20
 EXPORTS = ("fp4_status_string", "fp4_scale_bytes", "fp4_quantize", "fp4_root_coeffs",
            "fp4_root_ns_workspace_bytes", "fp4_root_ns", "fp4_root_ns_batched_workspace_bytes",
            "fp4_root_ns_batched", "fp4_last_device_status", "fp4_root_ns_workspace_layout", "fp4_gemm_nt",
+           "fp4_gemm_nt_resident",
            "fp4_profile_enable", "fp4_profile_collect", "fp4_kernel_launches", "fp4_root_ns_static",
            "fp4_selftest_bounded_wait")
 PROF_CLASSES = ("clip", "stats", "prep", "G1", "G2", "G3", "transpose", "quantize", "momentum", "adamw")
@@ -130,6 +131,8 @@ def load_library():
     L.fp4_root_ns_workspace_layout.restype = C.c_int
     L.fp4_gemm_nt.argtypes = [vp, vp, C.c_float, vp, vp, C.c_float, i64, i64, i64, vp, vp, vp]
     L.fp4_gemm_nt.restype = C.c_int
+    L.fp4_gemm_nt_resident.argtypes = L.fp4_gemm_nt.argtypes
+    L.fp4_gemm_nt_resident.restype = C.c_int
     L.fp4_root_ns_static.argtypes = [vp, vp, i64, i64, C.c_int, C.POINTER(NsParams), vp, vp]
     L.fp4_root_ns_static.restype = C.c_int
     L.fp4_profile_enable.argtypes = [C.c_int]; L.fp4_profile_enable.restype = None
@@ -270,6 +273,18 @@ def fp4_gemm_nt(a_codes, a_scales, a_sg: float, b_codes, b_scales, b_sg: float, 
                                       b_scales.data_ptr(), float(b_sg), M, N, K, D.data_ptr(),
                                       status.data_ptr() if status is not None else None, _stream(stream)),
            "fp4_gemm_nt")
+
+
+def fp4_gemm_nt_resident(a_codes, a_scales, a_sg: float, b_codes, b_scales, b_sg: float, D: torch.Tensor,
+                         status: torch.Tensor | None = None, stream=None) -> None:
+    """The launch of fp4_gemm_nt with the operands fetched once per SM pair (tensor-pipe ceiling)."""
+    M, K = a_codes.shape[0], a_codes.shape[1] * 2
+    N = b_codes.shape[0]
+    _check(load_library().fp4_gemm_nt_resident(a_codes.data_ptr(), a_scales.data_ptr(), float(a_sg),
+                                               b_codes.data_ptr(), b_scales.data_ptr(), float(b_sg), M, N, K,
+                                               D.data_ptr(), status.data_ptr() if status is not None else None,
+                                               _stream(stream)),
+           "fp4_gemm_nt_resident")
 
 
 def fp4_profile_enable(on: bool) -> None:

@@ -272,8 +272,9 @@ k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ Ge
   constexpr bool HAS_AUX = (MODE == kG2 || MODE == kG3);
   constexpr bool STORE_F32 = (MODE == kPlain || MODE == kG1 || MODE == kG3);
   const bool do_q = (MODE != kPlain) && !UPD && args.write_q;  // the update variant is launched without quantised outputs
-  // Measurement of the tensor-pipe ceiling (plain product only): no operand is fetched, the MMAs run on
-  // whatever the stages hold.
+  // Measurement of the tensor-pipe ceiling (plain product only): each CTA pair fetches the first stages of
+  // its first tile once and every later MMA runs on those resident stages - no operand traffic, same
+  // instruction stream, same epilogue.
   const bool dry = (MODE == kPlain) && args.dry_operands != 0;
 
   if (threadIdx.x == 0) {
@@ -297,16 +298,16 @@ k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ Ge
 
   if (warp == 0) {
     // ------------------------------------------------------------ operand producer (both CTAs)
-    if (!dry && elect_one()) {
+    if (elect_one()) {
       int st = 0; uint32_t ph = 0;
       TR_DECL
-      for (int t = pair; t < num_tiles; t += num_pairs) {
+      for (int t = pair; t < (dry ? min(num_tiles, pair + 1) : num_tiles); t += num_pairs) {
         int p, ti, tj;
         decode_tile(t, args, tiles_per_problem, p, ti, tj, sym);
         const GemmProblem* pr = probs + p;
         const int arow = ti * PM + (int)rank * BM;   // this CTA's rows of the row operand
         const int brow = tj * PN + (int)rank * BM;   // this CTA's half of the column operand
-        for (int kb = 0; kb < num_kb; ++kb) {
+        for (int kb = 0; kb < (dry ? min(num_kb, STAGES) : num_kb); ++kb) {
           TR_BEGIN
           wait_or_abort(&bars->empty[st], ph ^ 1, abort_flag);
           TR_END(0)
@@ -344,7 +345,7 @@ k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ Ge
         const uint32_t d_tmem = tmem_base + par * ACC1_COL;
         for (int kb = 0; kb < num_kb; ++kb) {
           TR_BEGIN
-          if (!dry) wait_or_abort(&bars->full[st], ph, abort_flag);
+          if (!dry || (seq == 0 && kb < STAGES)) wait_or_abort(&bars->full[st], ph, abort_flag);
           TR_END(2)
           tc_fence_after();
           const uint32_t sf_t = tmem_base + TMEM_SF_COL;

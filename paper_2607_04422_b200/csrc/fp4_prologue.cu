@@ -15,8 +15,10 @@
 //           share an exponent, so their squares add as integers) and tau^2 for every clipped
 //           element, and derives nu, 1/(nu+eps), amax(X0) and the tensor scale of X0.
 // If the bin holds more candidates than the list can take (many equal values, e.g. a
-// constant matrix) a fallback continues the radix select with two more full passes and a
-// separate statistics pass; its kernels are always launched and return at once otherwise.
+// constant matrix) the finishing block itself continues the radix select with two more passes
+// over the matrix and a statistics pass (slow, rare, no extra launch).
+#include <stddef.h>
+
 #include "fp4_kernels.h"
 
 namespace fp4 {
@@ -67,12 +69,10 @@ __global__ void __launch_bounds__(256) kp_init(const __grid_constant__ PrepGroup
   const PrepMatrix& m = g.mat[blockIdx.y];
   uint32_t* w = reinterpret_cast<uint32_t*>(m.hdr);
   const int first = m.clear_status ? 0 : 4;
-  for (int i = first + blockIdx.x * blockDim.x + threadIdx.x; i < g.zero_words; i += gridDim.x * blockDim.x) w[i] = 0;
-}
-__global__ void kp_arm(const __grid_constant__ PrepGroup g) {
-  const PrepMatrix& m = g.mat[blockIdx.y];
-  m.hdr->sel_prefix = 0;
-  m.hdr->sel_rank = g.clip_rank;
+  // the select starts with an empty prefix and the wanted rank (written instead of the zero)
+  const int rank_word = (int)(offsetof(NsHeader, sel_rank) / 4);
+  for (int i = first + blockIdx.x * blockDim.x + threadIdx.x; i < g.zero_words; i += gridDim.x * blockDim.x)
+    w[i] = (i == rank_word) ? g.clip_rank : 0u;
 }
 
 constexpr int kTopBits = 13;                 // bits of the first radix pass
@@ -243,6 +243,63 @@ __device__ __forceinline__ void write_norm_scalars(float* scalars, const NsScala
   scalars[ix.sg_X0] = scale_exact(__fmul_rn(widen, amax0));
 }
 
+// ---- fallback when the candidate list overflowed (so many equal magnitudes that the picked bin holds more
+// than the list takes: constant matrices and the like).  One block finishes the job alone: two more
+// radix rounds over the whole matrix (bits 17..7, then 6..0) and the clamped sum of squares.  Slow
+// (three passes by 1024 threads) but rare, and it costs no launch when it is not needed.
+// hist: 2048 counters; shd: 1024 doubles.
+__device__ void fallback_select_and_stats(const PrepGroup& g, const PrepMatrix& m, uint32_t* hist, double* shd) {
+  __shared__ uint32_t s_fb_prefix, s_fb_rank;
+  NsHeader* hdr = m.hdr;
+  const float4* src = reinterpret_cast<const float4*>(m.G);
+  if (threadIdx.x == 0) { s_fb_prefix = hdr->sel_prefix; s_fb_rank = hdr->sel_rank; }
+  __syncthreads();
+  for (int round = 0; round < 2; ++round) {
+    const int shift = round == 0 ? 7 : 0, nbits = round == 0 ? 11 : 7;
+    const uint32_t nb = 1u << nbits;
+    const uint32_t high_mask = (0x7FFFFFFFu >> (shift + nbits)) << (shift + nbits);
+    for (uint32_t i = threadIdx.x; i < nb; i += blockDim.x) hist[i] = 0;
+    __syncthreads();
+    const uint32_t prefix = s_fb_prefix;
+    for (int64_t i = threadIdx.x; i < g.n4; i += blockDim.x) {
+      const float4 v = __ldg(src + i);
+      const uint32_t k[4] = {mag_bits(v.x), mag_bits(v.y), mag_bits(v.z), mag_bits(v.w)};
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        if ((k[j] & high_mask) == prefix) atomicAdd(&hist[(k[j] >> shift) & (nb - 1)], 1u);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      uint32_t run = 0;
+      const uint32_t rank = s_fb_rank;
+      for (uint32_t b = 0; b < nb; ++b) {
+        if (rank <= run + hist[b]) { s_fb_prefix = prefix | (b << shift); s_fb_rank = rank - run; break; }
+        run += hist[b];
+      }
+    }
+    __syncthreads();
+  }
+  const float tau = __uint_as_float(s_fb_prefix);
+  double acc = 0.0;
+  for (int64_t i = threadIdx.x; i < g.n4; i += blockDim.x) {
+    const float4 v = __ldg(src + i);
+    const float c[4] = {fminf(fabsf(v.x), tau), fminf(fabsf(v.y), tau), fminf(fabsf(v.z), tau), fminf(fabsf(v.w), tau)};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc += (double)c[j] * (double)c[j];
+  }
+  shd[threadIdx.x] = acc;
+  __syncthreads();
+  for (int o = blockDim.x / 2; o; o >>= 1) {
+    if ((int)threadIdx.x < o) shd[threadIdx.x] += shd[threadIdx.x + o];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    hdr->sel_prefix = s_fb_prefix;
+    m.scalars[g.ix.tau] = tau;
+    write_norm_scalars(m.scalars, g.ix, shd[0], tau, g.eps, g.q.widen);
+  }
+}
+
 // ---- finish: select tau among the candidates and derive the normalisation scalars
 __global__ void __launch_bounds__(1024) kp_finalize(const __grid_constant__ PrepGroup g) {
   const PrepMatrix& m = g.mat[blockIdx.y];
@@ -260,7 +317,9 @@ __global__ void __launch_bounds__(1024) kp_finalize(const __grid_constant__ Prep
   }
   const uint32_t count = hdr->cand_count;
   if (count > g.cand_cap) {
-    if (threadIdx.x == 0) hdr->overflow = 1;  // the fallback kernels take over
+    if (threadIdx.x == 0) hdr->overflow = 1;
+    __shared__ uint32_t fb_hist[2048];
+    fallback_select_and_stats(g, m, fb_hist, shd);
     return;
   }
   // two radix rounds over the low 18 bits of the candidates: 9 bits each.  The second round
@@ -378,73 +437,6 @@ __global__ void __launch_bounds__(1024) kp_finalize(const __grid_constant__ Prep
     m.scalars[g.ix.tau] = tau;
     write_norm_scalars(m.scalars, g.ix, total, tau, g.eps, g.q.widen);
     hdr->overflow = 0;
-  }
-}
-
-// ---- fallback when the candidate list overflowed: two more radix passes over the data
-// (bits 17..7, then 6..0), a clamp-statistics pass, and the scalars
-template <int SHIFT, int BITS>
-__global__ void __launch_bounds__(512) kp_fb_hist(const __grid_constant__ PrepGroup g) {
-  const PrepMatrix& m = g.mat[blockIdx.y];
-  if (!m.hdr->overflow) return;
-  constexpr int NB = 1 << BITS;
-  __shared__ uint32_t sh[NB];
-  for (int i = threadIdx.x; i < NB; i += blockDim.x) sh[i] = 0;
-  __syncthreads();
-  const uint32_t prefix = m.hdr->sel_prefix;
-  constexpr uint32_t HIGH_MASK = (0x7FFFFFFFu >> (SHIFT + BITS)) << (SHIFT + BITS);
-  const float4* src = reinterpret_cast<const float4*>(m.G);
-  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < g.n4; i += (int64_t)gridDim.x * blockDim.x) {
-    float4 v = __ldg(src + i);
-    const uint32_t k[4] = {mag_bits(v.x), mag_bits(v.y), mag_bits(v.z), mag_bits(v.w)};
-#pragma unroll
-    for (int j = 0; j < 4; ++j)
-      if ((k[j] & HIGH_MASK) == prefix) atomicAdd(&sh[(k[j] >> SHIFT) & (NB - 1)], 1u);
-  }
-  __syncthreads();
-  for (int i = threadIdx.x; i < NB; i += blockDim.x)
-    if (sh[i]) atomicAdd(&m.hist[i], sh[i]);
-}
-
-template <int SHIFT, int NB>
-__global__ void __launch_bounds__(256) kp_fb_pick(const __grid_constant__ PrepGroup g) {
-  const PrepMatrix& m = g.mat[blockIdx.y];
-  if (!m.hdr->overflow) return;
-  pick_bin<NB>(m.hdr, m.hist, SHIFT, nullptr, nullptr);
-}
-
-__global__ void __launch_bounds__(256) kp_fb_stats(const __grid_constant__ PrepGroup g) {
-  const PrepMatrix& m = g.mat[blockIdx.y];
-  if (!m.hdr->overflow) return;
-  const float tau = __uint_as_float(m.hdr->sel_prefix);
-  const float4* src = reinterpret_cast<const float4*>(m.G);
-  double acc = 0.0;
-  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < g.n4; i += (int64_t)gridDim.x * blockDim.x) {
-    float4 v = __ldg(src + i);
-    const float c[4] = {fminf(fabsf(v.x), tau), fminf(fabsf(v.y), tau), fminf(fabsf(v.z), tau), fminf(fabsf(v.w), tau)};
-#pragma unroll
-    for (int j = 0; j < 4; ++j) acc += (double)c[j] * (double)c[j];
-  }
-#pragma unroll
-  for (int o = 16; o; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-  __shared__ double wa[8];
-  if ((threadIdx.x & 31) == 0) wa[threadIdx.x >> 5] = acc;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    for (int w = 1; w < 8; ++w) acc += wa[w];
-    m.partial[blockIdx.x] = acc;
-  }
-}
-
-__global__ void __launch_bounds__(1024) kp_fb_finish(const __grid_constant__ PrepGroup g) {
-  const PrepMatrix& m = g.mat[blockIdx.y];
-  if (!m.hdr->overflow) return;
-  __shared__ double shd[1024];
-  const double total = sum_partials(m.partial, g.stat_blocks, shd);
-  if (threadIdx.x == 0) {
-    const float tau = __uint_as_float(m.hdr->sel_prefix);
-    m.scalars[g.ix.tau] = tau;
-    write_norm_scalars(m.scalars, g.ix, total, tau, g.eps, g.q.widen);
   }
 }
 
@@ -618,10 +610,9 @@ cudaError_t launch_prologue_group(const PrologueItem* items, int count, int writ
       kp_init<<<dim3(4, (unsigned)nn), 256, 0, st>>>(g);
       count_launches(1);
       if (g.clip) {
-        kp_arm<<<gy1, 1, 0, st>>>(g);
         if (!all_counted) kp_hist_top<<<gh, 512, 0, st>>>(g);
         kp_pick_top<<<gy1, 256, 0, st>>>(g);
-        count_launches(all_counted ? 2 : 3);
+        count_launches(all_counted ? 1 : 2);
       }
     }
     {
@@ -629,15 +620,6 @@ cudaError_t launch_prologue_group(const PrologueItem* items, int count, int writ
       kp_compact_stats<<<gs, 256, 0, st>>>(g);
       kp_finalize<<<gy1, 1024, 0, st>>>(g);
       count_launches(2);
-      if (g.clip) {
-        kp_fb_hist<7, 11><<<gh, 512, 0, st>>>(g);
-        kp_fb_pick<7, 2048><<<gy1, 256, 0, st>>>(g);
-        kp_fb_hist<0, 7><<<gh, 512, 0, st>>>(g);
-        kp_fb_pick<0, 256><<<gy1, 256, 0, st>>>(g);
-        kp_fb_stats<<<gs, 256, 0, st>>>(g);
-        kp_fb_finish<<<gy1, 1024, 0, st>>>(g);
-        count_launches(6);
-      }
     }
     {
       ProfScope ps(FP4_PROF_PREP, st);

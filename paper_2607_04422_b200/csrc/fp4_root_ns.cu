@@ -4,6 +4,7 @@
 #include <atomic>
 #include <cmath>
 #include <mutex>
+#include <unordered_map>
 #include <vector>
 
 #include "fp4_gemm_common.cuh"
@@ -296,8 +297,8 @@ struct MatrixCtx {
   uint16_t* W;                // the BF16 parameter that takes Root's update in this call, or null
 };
 
-fp4_status prepare_matrix(const DeviceInfo* d, const float* G, float* out, int64_t m, int64_t n, int steps,
-                          const fp4_ns_params* p, uint8_t* ws, MatrixCtx* c) {
+fp4_status build_matrix(const DeviceInfo* d, const float* G, float* out, int64_t m, int64_t n, int steps,
+                        const fp4_ns_params* p, uint8_t* ws, MatrixCtx* c) {
   fp4_status rc = make_plan(m, n, steps, p, d->sms, &c->pl);
   if (rc != FP4_OK) return rc;
   const fp4_ws_layout& L = c->pl.lay;
@@ -389,6 +390,56 @@ fp4_status prepare_matrix(const DeviceInfo* d, const float* G, float* out, int64
     c->g3_first.tmAux = tm_G;
     c->g3_first.aux_raw = 1;
   }
+  return FP4_OK;
+}
+
+// Everything build_matrix derives (workspace plan, a dozen and a half TMA descriptors, the problem
+// descriptions) depends only on the pointers, the shape and a few parameters: an optimiser calls with
+// the same buffers every step, so the results are kept, keyed by exactly those inputs.  The library
+// keeps no other state between calls; a hit costs one hash lookup instead of ~20 driver calls.
+struct CtxKey {
+  int dev; int steps; uint32_t flags;
+  const void* G; const void* out; const void* ws;
+  int64_t m, n;
+  uint32_t a, b, c, q, eps;   // bit patterns of the float parameters
+  bool operator==(const CtxKey& o) const {
+    return dev == o.dev && steps == o.steps && flags == o.flags && G == o.G && out == o.out && ws == o.ws && m == o.m &&
+           n == o.n && a == o.a && b == o.b && c == o.c && q == o.q && eps == o.eps;
+  }
+};
+struct CtxKeyHash {
+  size_t operator()(const CtxKey& k) const {
+    uint64_t h = 1469598103934665603ull;
+    auto mix = [&](uint64_t v) { h = (h ^ v) * 1099511628211ull; };
+    mix((uint64_t)k.dev); mix((uint64_t)k.steps); mix(k.flags);
+    mix((uint64_t)(uintptr_t)k.G); mix((uint64_t)(uintptr_t)k.out); mix((uint64_t)(uintptr_t)k.ws);
+    mix((uint64_t)k.m); mix((uint64_t)k.n); mix(k.a); mix(k.b); mix(k.c); mix(k.q); mix(k.eps);
+    return (size_t)h;
+  }
+};
+std::unordered_map<CtxKey, MatrixCtx, CtxKeyHash> g_ctx_cache;
+std::mutex g_ctx_mu;
+constexpr size_t kCtxCacheMax = 1024;   // entries (about 8 KB each); the cache is emptied when it is full
+
+inline uint32_t fbits(float v) { uint32_t u; memcpy(&u, &v, 4); return u; }
+
+fp4_status prepare_matrix(const DeviceInfo* d, const float* G, float* out, int64_t m, int64_t n, int steps,
+                          const fp4_ns_params* p, uint8_t* ws, MatrixCtx* c) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return FP4_ERR_CUDA;
+  // NO_OUT only matters to the launch sequence, not to what is prepared here
+  const CtxKey key{dev, steps, p->flags & ~FP4_FLAG_NO_OUT, G, out, ws, m, n,
+                   fbits(p->a), fbits(p->b), fbits(p->c), fbits(p->clip_quantile), fbits(p->eps)};
+  {
+    std::lock_guard<std::mutex> lock(g_ctx_mu);
+    auto it = g_ctx_cache.find(key);
+    if (it != g_ctx_cache.end()) { *c = it->second; return FP4_OK; }
+  }
+  fp4_status rc = build_matrix(d, G, out, m, n, steps, p, ws, c);
+  if (rc != FP4_OK) return rc;
+  std::lock_guard<std::mutex> lock(g_ctx_mu);
+  if (g_ctx_cache.size() >= kCtxCacheMax) g_ctx_cache.clear();
+  g_ctx_cache.emplace(key, *c);
   return FP4_OK;
 }
 
@@ -748,7 +799,7 @@ fp4_status fp4_last_device_status(const void* ws, cudaStream_t stream) {
   return word == 0 ? FP4_OK : (fp4_status)word;
 }
 
-fp4_status fp4_gemm_nt(const uint8_t* a_codes, const uint8_t* a_scales, float a_tensor_scale,
+static fp4_status gemm_nt_impl(int dry, const uint8_t* a_codes, const uint8_t* a_scales, float a_tensor_scale,
                        const uint8_t* b_codes, const uint8_t* b_scales, float b_tensor_scale, int64_t M, int64_t N,
                        int64_t K, float* D, uint32_t* device_status, cudaStream_t stream) {
   if (!a_codes || !a_scales || !b_codes || !b_scales || !D) return FP4_ERR_INVALID_ARG;
@@ -775,7 +826,23 @@ fp4_status fp4_gemm_nt(const uint8_t* a_codes, const uint8_t* a_scales, float a_
   L.num_problems = 1;
   L.K = (int)K; L.tiles_m = (int)(M / 128); L.tiles_n = (int)(N / 128);
   L.status = device_status;
+  L.dry_operands = dry;
+  if (dry && !pair_kernel(L.tiles_m, L.tiles_n, L.K, d->sms)) return FP4_ERR_SHAPE;
   return launch_gemm_auto(kPlain, pack, L, d->sms, stream) == cudaSuccess ? FP4_OK : FP4_ERR_CUDA;
+}
+
+fp4_status fp4_gemm_nt(const uint8_t* a_codes, const uint8_t* a_scales, float a_tensor_scale,
+                       const uint8_t* b_codes, const uint8_t* b_scales, float b_tensor_scale, int64_t M, int64_t N,
+                       int64_t K, float* D, uint32_t* device_status, cudaStream_t stream) {
+  return gemm_nt_impl(0, a_codes, a_scales, a_tensor_scale, b_codes, b_scales, b_tensor_scale, M, N, K, D, device_status,
+                      stream);
+}
+
+fp4_status fp4_gemm_nt_resident(const uint8_t* a_codes, const uint8_t* a_scales, float a_tensor_scale,
+                                const uint8_t* b_codes, const uint8_t* b_scales, float b_tensor_scale, int64_t M,
+                                int64_t N, int64_t K, float* D, uint32_t* device_status, cudaStream_t stream) {
+  return gemm_nt_impl(1, a_codes, a_scales, a_tensor_scale, b_codes, b_scales, b_tensor_scale, M, N, K, D, device_status,
+                      stream);
 }
 
 }  // extern "C"

@@ -395,7 +395,7 @@ def test_argument_errors():
     with pytest.raises(fp4.Fp4Error) as e:
         fp4.fp4_root_ns(G, G, 5, None, ws[1:])
     assert e.value.code == 3
-    for bad_flags in (16, FP4_FLAG_RHT | (0x1234 << 16)):      # unknown bits, fp4_quantize's sign bits
+    for bad_flags in (32, FP4_FLAG_RHT | (0x1234 << 16)):      # unknown bits, fp4_quantize's sign bits
         with pytest.raises(fp4.Fp4Error) as e:
             fp4.fp4_root_ns(G, G, 5, fp4.NsParams.make(flags=bad_flags), ws)
         assert e.value.code == 1
