@@ -130,6 +130,20 @@ __device__ __forceinline__ void tma_load_2d_pair(void* smem_dst, const void* tma
       "l"(tmap), "r"(x), "r"(y), "r"(bar_cluster)
       : "memory");
 }
+// The same load with an L2 eviction-priority hint (a policy made by createpolicy)
+__device__ __forceinline__ void tma_load_2d_pair_hint(void* smem_dst, const void* tmap, int x, int y, uint32_t bar_cluster,
+                                                      uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint "
+      "[%0], [%1, {%2, %3}], [%4], %5;" ::"r"(smem_u32(smem_dst)),
+      "l"(tmap), "r"(x), "r"(y), "r"(bar_cluster), "l"(policy)
+      : "memory");
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+  uint64_t p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
 __device__ __forceinline__ void tmem_alloc2(uint32_t* smem_dst, uint32_t ncols) {
   asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_dst)),
                "r"(ncols)
@@ -301,6 +315,17 @@ k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ Ge
     if (elect_one()) {
       int st = 0; uint32_t ph = 0;
       TR_DECL
+      // G3's operands (qB and the transposed copy of qX, some 20 MB per matrix) are re-read by every tile
+      // while 200 MB of FP32 X stream through the L2 beside them: a stage completes when its last byte
+      // has arrived, so even a small share of operand lines evicted to DRAM makes almost every stage wait
+      // for DRAM.  Loading them with evict-last priority took 6 % off G3; the same hint on the symmetric
+      // products' operands, and evict-first on the FP32 tiles, measured slower and are not used.
+      const uint64_t keep = l2_policy_evict_last();
+#define TMA_OPERAND(dst, map, x, y, bar)                                          \
+  do {                                                                            \
+    if (MODE == kG3) tma_load_2d_pair_hint(dst, map, x, y, bar, keep);            \
+    else tma_load_2d_pair(dst, map, x, y, bar);                                   \
+  } while (0)
       for (int t = pair; t < (dry ? min(num_tiles, pair + 1) : num_tiles); t += num_pairs) {
         int p, ti, tj;
         decode_tile(t, args, tiles_per_problem, p, ti, tj, sym);
@@ -313,13 +338,13 @@ k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ Ge
           TR_END(0)
           const uint32_t full_leader = map_to_cta(&bars->full[st], 0);
           if (leader) mbar_expect_tx(&bars->full[st], 2 * STAGE_BYTES_CTA);
-          tma_load_2d_pair(smem + OFF_A + st * OPER_BYTES, &pr->tmA, kb * (BK / 2), arow, full_leader);
-          tma_load_2d_pair(smem + OFF_B + st * OPER_BYTES, &pr->tmB, kb * (BK / 2), brow, full_leader);
+          TMA_OPERAND(smem + OFF_A + st * OPER_BYTES, &pr->tmA, kb * (BK / 2), arow, full_leader);
+          TMA_OPERAND(smem + OFF_B + st * OPER_BYTES, &pr->tmB, kb * (BK / 2), brow, full_leader);
           // scale atoms: 64-bit elements, one row of the map per 128-row block
           uint8_t* sf = smem + OFF_SF + st * SF_BYTES;
-          tma_load_2d_pair(sf, &pr->tmSfa, kb * (SF_ATOMS / 8), arow / 128, full_leader);
-          tma_load_2d_pair(sf + SF_ATOMS, &pr->tmSfb, kb * (SF_ATOMS / 8), tj * 2, full_leader);
-          tma_load_2d_pair(sf + 2 * SF_ATOMS, &pr->tmSfb, kb * (SF_ATOMS / 8), tj * 2 + 1, full_leader);
+          TMA_OPERAND(sf, &pr->tmSfa, kb * (SF_ATOMS / 8), arow / 128, full_leader);
+          TMA_OPERAND(sf + SF_ATOMS, &pr->tmSfb, kb * (SF_ATOMS / 8), tj * 2, full_leader);
+          TMA_OPERAND(sf + 2 * SF_ATOMS, &pr->tmSfb, kb * (SF_ATOMS / 8), tj * 2 + 1, full_leader);
           if (++st == STAGES) { st = 0; ph ^= 1; }
         }
       }
