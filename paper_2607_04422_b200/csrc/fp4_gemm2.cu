@@ -25,14 +25,17 @@ namespace fp4 {
 
 namespace {
 
-#ifndef FP4_STAGES2
-#define FP4_STAGES2 3
+#ifndef FP4_STAGES_AUX
+#define FP4_STAGES_AUX 3
+#endif
+#ifndef FP4_STAGES_NOAUX
+#define FP4_STAGES_NOAUX 4
 #endif
 constexpr int PM = 256, PN = 256;              // output tile of a CTA pair
 constexpr int BM = 128;                        // rows per CTA
 constexpr int BK = 256;                        // elements of K per stage: 128-byte operand rows
 constexpr int KSTEPS = BK / 64;
-constexpr int STAGES = FP4_STAGES2;
+constexpr int MAX_STAGES = 4;
 constexpr int OPER_BYTES = BM * BK / 2;        // 16 KB: 128 rows of one operand
 constexpr int SF_ATOMS = KSTEPS * 512;         // scale atoms of one 128-row block and stage
 constexpr int SF_BYTES = 3 * SF_ATOMS;         // row operand: own block; column operand: both blocks
@@ -42,10 +45,8 @@ constexpr int NCHUNK = PN / CHUNK;             // 16
 constexpr int TEAMS = 4;                       // column groups of a tile: 64 columns = one word of row scales
 constexpr int TEAM_CHUNKS = NCHUNK / TEAMS;    // 4
 constexpr int EPI_WARPS = 4 * TEAMS;           // one warp per (column group, lane quadrant)
-constexpr int XBUF = 2;                        // FP32 chunk buffers per warp
-constexpr int XBUF_BYTES = 32 * CHUNK * 4;     // 2 KB: 32 rows x 64 bytes (64-byte swizzle)
+constexpr int XBUF_BYTES = 32 * CHUNK * 4;     // a warp's FP32 chunk buffer, 2 KB: 32 rows x 64 bytes (64-byte swizzle)
 constexpr int RQ_BYTES = 32 * 32;              // row-quantised codes of 32 rows x 64 columns
-constexpr int WARP_AREA = XBUF * XBUF_BYTES + RQ_BYTES;
 // What a warp alone would write as partial 32-byte sectors is collected for one 128-column half of the
 // CTA's tile (two column groups = eight warps) and leaves as whole sectors: the column-quantised codes
 // [128 tile columns][64 bytes = the CTA's 128 rows], their scale bytes (two atoms) and the row scales
@@ -53,7 +54,7 @@ constexpr int WARP_AREA = XBUF * XBUF_BYTES + RQ_BYTES;
 constexpr int HALF_CQ_BYTES = 128 * 64;
 constexpr int HALF_SF_BYTES = 2 * 512;
 constexpr int HALF_AREA = HALF_CQ_BYTES + 2 * HALF_SF_BYTES;
-static_assert(TEAM_CHUNKS == 4 && XBUF == 2, "the chunk loop is written for four chunks on two buffers");
+static_assert(TEAM_CHUNKS == 4, "the chunk loop is written for four chunks");
 
 // Two consecutive tiles use two accumulator buffers that share one chunk of tensor memory
 // (512 columns cannot hold two 256-column accumulators plus the scale factors):
@@ -64,16 +65,29 @@ static_assert(TEAM_CHUNKS == 4 && XBUF == 2, "the chunk loop is written for four
 // may then start while the rest of the tile is still being drained.
 constexpr uint32_t ACC1_COL = PN - CHUNK;      // 240
 
-constexpr int OFF_A = 0;
-constexpr int OFF_B = OFF_A + STAGES * OPER_BYTES;
-constexpr int OFF_SF = OFF_B + STAGES * OPER_BYTES;
-constexpr int OFF_EPI = OFF_SF + STAGES * SF_BYTES;
-constexpr int OFF_HALF = OFF_EPI + EPI_WARPS * WARP_AREA;
-constexpr int OFF_BAR = OFF_HALF + 2 * HALF_AREA;
-constexpr int SMEM_BYTES = OFF_BAR + 512 + 1024;
-static_assert(OFF_EPI % 1024 == 0 && WARP_AREA % 1024 == 0, "chunk buffers keep the swizzle phase");
-static_assert(OFF_HALF % 1024 == 0 && HALF_AREA % 1024 == 0, "code staging keeps the swizzle phase");
-static_assert(SMEM_BYTES <= 232448, "at most 227 KB of dynamic shared memory");
+// Shared-memory layout, per epilogue mode.  The main loop is bound by how many operand bytes a pair of
+// SMs keeps in flight (the plain product runs at 2.9 / 3.9 / 4.7 PFLOP/s with 2 / 3 / 4 stages), so every
+// mode takes as many stages as its epilogue leaves room for: the modes that combine with an FP32 tile
+// (G2, G3) need two chunk buffers per warp - one in work, one being fetched - and fit three stages; the
+// others (G1, the plain product) stage their result in one buffer and fit four.
+template <int MODE>
+struct Lay {
+  static constexpr bool HAS_AUX = (MODE == kG2 || MODE == kG3);
+  static constexpr int STAGES = HAS_AUX ? FP4_STAGES_AUX : FP4_STAGES_NOAUX;
+  static constexpr int XBUF = HAS_AUX ? 2 : 1;                 // FP32 chunk buffers per warp
+  static constexpr int WARP_AREA = XBUF * XBUF_BYTES + RQ_BYTES;
+  static constexpr int OFF_A = 0;
+  static constexpr int OFF_B = OFF_A + STAGES * OPER_BYTES;
+  static constexpr int OFF_SF = OFF_B + STAGES * OPER_BYTES;
+  static constexpr int OFF_EPI = OFF_SF + STAGES * SF_BYTES;
+  static constexpr int OFF_HALF = OFF_EPI + EPI_WARPS * WARP_AREA;
+  static constexpr int OFF_BAR = OFF_HALF + 2 * HALF_AREA;
+  static constexpr int SMEM_BYTES = OFF_BAR + 512 + 1024;
+  static_assert(STAGES <= MAX_STAGES, "barrier arrays");
+  static_assert(OFF_EPI % 1024 == 0 && WARP_AREA % 1024 == 0, "chunk buffers keep the swizzle phase");
+  static_assert(OFF_HALF % 1024 == 0 && HALF_AREA % 1024 == 0, "code staging keeps the swizzle phase");
+  static_assert(SMEM_BYTES <= 232448, "at most 227 KB of dynamic shared memory");
+};
 
 constexpr int ROLE_WARPS = 3;                  // operand producer, MMA issuer, issuer of the half-tile stores
 constexpr int NTHREADS = (ROLE_WARPS + EPI_WARPS) * 32;
@@ -88,12 +102,12 @@ static_assert(TMEM_SF_COL + SF_COLS <= 512, "tensor memory columns");
 constexpr uint32_t IDESC = (1u << 7) | (1u << 10) | ((uint32_t)(PN >> 3) << 17) | ((uint32_t)(PM >> 4) << 24);
 
 struct Barriers {
-  uint64_t full[STAGES];     // even CTA: both CTAs' operand bytes of a stage have landed
-  uint64_t empty[STAGES];    // stage consumed (MMA commit, multicast to both CTAs)
+  uint64_t full[MAX_STAGES]; // even CTA: both CTAs' operand bytes of a stage have landed
+  uint64_t empty[MAX_STAGES];  // stage consumed (MMA commit, multicast to both CTAs)
   uint64_t acc_full[2];      // accumulator buffer complete (MMA commit, multicast)
   uint64_t acc_empty[2];     // even CTA: buffer drained by all epilogue warps of the pair
   uint64_t ov_free;          // even CTA: the columns shared with the other buffer are drained (8 warps)
-  uint64_t xfull[EPI_WARPS * XBUF];  // a warp's chunk buffer holds the FP32 block it asked for
+  uint64_t xfull[EPI_WARPS * 2];  // a warp's chunk buffer holds the FP32 block it asked for
   uint64_t half_done[2];     // the eight warps of a half have staged their quantised output of the tile
   uint64_t half_free[2];     // the stores of the half's staging area have read it
   uint32_t tmem_base;
@@ -267,6 +281,10 @@ __device__ __forceinline__ void stg256(void* p, const uint32_t (&r)[8]) {
 template <int MODE, bool PF, bool BH, bool UPD = false>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
 k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ GemmLaunch args) {
+  using L = Lay<MODE>;
+  constexpr int STAGES = L::STAGES, XBUF = L::XBUF, WARP_AREA = L::WARP_AREA;
+  constexpr int OFF_A = L::OFF_A, OFF_B = L::OFF_B, OFF_SF = L::OFF_SF, OFF_EPI = L::OFF_EPI, OFF_HALF = L::OFF_HALF,
+                OFF_BAR = L::OFF_BAR;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   Barriers* bars = reinterpret_cast<Barriers*>(smem + OFF_BAR);
@@ -295,7 +313,7 @@ k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ Ge
     for (int i = 0; i < STAGES; ++i) { mbar_init(&bars->full[i], 1); mbar_init(&bars->empty[i], 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&bars->acc_full[i], 1); mbar_init(&bars->acc_empty[i], 2 * EPI_WARPS); }
     mbar_init(&bars->ov_free, 8);
-    for (int i = 0; i < EPI_WARPS * XBUF; ++i) mbar_init(&bars->xfull[i], 1);
+    for (int i = 0; i < EPI_WARPS * 2; ++i) mbar_init(&bars->xfull[i], 1);
     for (int i = 0; i < 2; ++i) { mbar_init(&bars->half_done[i], EPI_WARPS / 2); mbar_init(&bars->half_free[i], 1); }
     bars->abort_flag = 0;
     mbar_fence_init();
@@ -438,7 +456,7 @@ k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ Ge
     const int half = team >> 1;                         // the staging area this warp shares with seven others
     const uint32_t half_st = smem_u32(smem + OFF_HALF + half * HALF_AREA);
     const uint32_t half_done = smem_u32(&bars->half_done[half]), half_free = smem_u32(&bars->half_free[half]);
-    const uint32_t xfull0 = smem_u32(&bars->xfull[ew * XBUF]);
+    const uint32_t xfull0 = smem_u32(&bars->xfull[ew * 2]);
     // row pass: this lane's row of a chunk buffer is 64 bytes whose 16-byte groups are XOR-swizzled with
     // bits 1-2 of the row; group j of the row sits at row_addr ^ (j << 4)
     const uint32_t row_addr = area + lane * 64 + (((lane >> 1) & 3) << 4);
@@ -614,7 +632,7 @@ k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ Ge
       for (int i = 0; i < TEAM_CHUNKS; ++i) {
         const int e = i ^ flip;                         // position of this chunk among the warp's 64 columns
         const int b = i & 1;
-        const uint32_t boff = b * XBUF_BYTES;
+        const uint32_t boff = (XBUF == 2 ? b : 0) * XBUF_BYTES;   // without a fetched tile: one staging buffer
         const int xcol = x64 + e * CHUNK;
         float v[16];
         if (HAS_AUX) {
@@ -773,6 +791,7 @@ k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ Ge
         TR_BEGIN
         if (lane == 0 && (STORE_F32 || i == 0)) bulk_wait_read<0>();
         TR_END(3)
+        if (XBUF == 1) __syncwarp();  // one buffer: the next chunk is staged over this one, after the store's read
         if (HAS_AUX) {
           if (i < 2) fetch(pr, x64, y32, (i + 2) ^ flip, false, b);
           else if (has_next) fetch(probs + nxt.p, nxt.x64, nxt.y32, (i - 2) ^ (flip ^ 3), nxt.below, b);
@@ -840,7 +859,7 @@ cudaError_t launch_pair_mode(const ProblemPack& pack, const GemmLaunch& L, int s
   int pairs = sms / 2;
   if (pairs > num_tiles) pairs = num_tiles;
   count_launches(1);
-  k_gemm_pair<MODE, PF, BH, UPD><<<2 * pairs, NTHREADS, SMEM_BYTES, st>>>(pack, L);
+  k_gemm_pair<MODE, PF, BH, UPD><<<2 * pairs, NTHREADS, Lay<MODE>::SMEM_BYTES, st>>>(pack, L);
   return cudaGetLastError();
 }
 
@@ -859,21 +878,21 @@ extern "C" int fp4_trace_read(unsigned long long* dst, int clear) {
 
 cudaError_t gemm_pair_set_attributes() {
   cudaError_t e;
-  if ((e = cudaFuncSetAttribute(k_gemm_pair<kPlain, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
-  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG1, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
-  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG1, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
-  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG1, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
-  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG1, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
-  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG2, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
-  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG2, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
-  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG2, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
-  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG2, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
-  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG3, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
-  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG3, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
-  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG3, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
-  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG3, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
-  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG3, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
-  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG3, false, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kPlain, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Lay<kPlain>::SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG1, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Lay<kG1>::SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG1, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Lay<kG1>::SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG1, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Lay<kG1>::SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG1, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Lay<kG1>::SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG2, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Lay<kG2>::SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG2, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Lay<kG2>::SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG2, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Lay<kG2>::SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG2, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Lay<kG2>::SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG3, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Lay<kG3>::SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG3, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Lay<kG3>::SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG3, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Lay<kG3>::SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG3, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Lay<kG3>::SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG3, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Lay<kG3>::SMEM_BYTES))) return e;
+  if ((e = cudaFuncSetAttribute(k_gemm_pair<kG3, false, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Lay<kG3>::SMEM_BYTES))) return e;
   return cudaSuccess;
 }
 
