@@ -34,10 +34,10 @@ UNIT = "matrices/s"
 FP4_NOMINAL_TFLOPS = 9000.0  # dense NVFP4, nominal
 FP4_OVER_BF16 = 4.0          # nominal ratio of the dense FP4 and BF16 tensor peaks
 # DRAM bytes per element of X that one G3 launch moves (dram__bytes_read + dram__bytes_write of
-# k_gemm_pair<3, 0, 0> from an ncu capture of one 3072 x 8192 matrix with all quantised outputs
+# k_gemm_pair<3, 0, 0, 0> from an ncu capture of one 3072 x 8192 matrix with all quantised outputs
 # written: 217.0 MB for 25.2 M elements); a grouped launch is scaled by the elements it covers
 G3_DRAM_BYTES_PER_ELEMENT = 217.0e6 / (3072 * 8192)
-G3_KERNEL = "k_gemm_pair<3, 0, 0>"   # MODE = G3, base quantiser, FP32 storage
+G3_KERNEL = "k_gemm_pair<3, 0, 0, 0>"   # MODE = G3, base quantiser, FP32 storage
 
 
 def peaks():
@@ -570,7 +570,7 @@ def run_ours(args):
     per_launch_ms = dom_ms / max(prof[dom][1], 1)
     achieved = dom_flops / (dom_ms / 1e3) / 1e12
     fp4_peak = pk["bf16_tflops_sustained"] * FP4_OVER_BF16
-    kernel_names = {"G1": "k_gemm_pair<1, 0, 0>", "G2": "k_gemm_pair<2, 0, 0>", "G3": G3_KERNEL}
+    kernel_names = {"G1": "k_gemm_pair<1, 0, 0, 0>", "G2": "k_gemm_pair<2, 0, 0, 0>", "G3": G3_KERNEL}
     roofline = {"kernel": kernel_names[dom], "bound": "tensor", "achieved": achieved, "peak": fp4_peak,
                 "unit": "TFLOP/s", "frac": achieved / fp4_peak,
                 "traffic": (G3_DRAM_BYTES_PER_ELEMENT * sum(m * n for m, n in shapes) * STEPS_NS * prof_steps
