@@ -25,6 +25,9 @@ namespace fp4 {
 
 namespace {
 
+#ifndef FP4_BK_AUX
+#define FP4_BK_AUX 256
+#endif
 #ifndef FP4_STAGES_AUX
 #define FP4_STAGES_AUX 3
 #endif
@@ -33,13 +36,7 @@ namespace {
 #endif
 constexpr int PM = 256, PN = 256;              // output tile of a CTA pair
 constexpr int BM = 128;                        // rows per CTA
-constexpr int BK = 256;                        // elements of K per stage: 128-byte operand rows
-constexpr int KSTEPS = BK / 64;
-constexpr int MAX_STAGES = 4;
-constexpr int OPER_BYTES = BM * BK / 2;        // 16 KB: 128 rows of one operand
-constexpr int SF_ATOMS = KSTEPS * 512;         // scale atoms of one 128-row block and stage
-constexpr int SF_BYTES = 3 * SF_ATOMS;         // row operand: own block; column operand: both blocks
-constexpr uint32_t STAGE_BYTES_CTA = 2 * OPER_BYTES + SF_BYTES;
+constexpr int MAX_STAGES = 8;
 constexpr int CHUNK = 16;                      // FP32 columns per epilogue step
 constexpr int NCHUNK = PN / CHUNK;             // 16
 constexpr int TEAMS = 4;                       // column groups of a tile: 64 columns = one word of row scales
@@ -73,6 +70,15 @@ constexpr uint32_t ACC1_COL = PN - CHUNK;      // 240
 template <int MODE>
 struct Lay {
   static constexpr bool HAS_AUX = (MODE == kG2 || MODE == kG3);
+  static constexpr int BK = HAS_AUX ? FP4_BK_AUX : 256;        // elements of K per stage: 64- or 128-byte operand rows
+  static_assert(BK == 128 || BK == 256, "operand rows of a stage are one TMA swizzle span");
+  static constexpr int KSTEPS = BK / 64;                       // MMAs (K = 64) per stage
+  static constexpr uint32_t OPER_SWIZZLE = (BK == 256) ? 2u : 4u;  // UMMA layout type: 128- or 64-byte swizzle
+  static constexpr uint32_t OPER_SBO = 8 * (BK / 2);           // bytes between 8-row groups of an operand tile
+  static constexpr int OPER_BYTES = BM * BK / 2;               // 128 rows of one operand
+  static constexpr int SF_ATOMS = KSTEPS * 512;                // scale atoms of one 128-row block and stage
+  static constexpr int SF_BYTES = 3 * SF_ATOMS;                // row operand: own block; column operand: both blocks
+  static constexpr uint32_t STAGE_BYTES_CTA = 2 * OPER_BYTES + SF_BYTES;
   static constexpr int STAGES = HAS_AUX ? FP4_STAGES_AUX : FP4_STAGES_NOAUX;
   static constexpr int XBUF = HAS_AUX ? 2 : 1;                 // FP32 chunk buffers per warp
   static constexpr int WARP_AREA = XBUF * XBUF_BYTES + RQ_BYTES;
@@ -283,6 +289,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NTHREADS, 1)
 k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ GemmLaunch args) {
   using L = Lay<MODE>;
   constexpr int STAGES = L::STAGES, XBUF = L::XBUF, WARP_AREA = L::WARP_AREA;
+  constexpr int BK = L::BK, KSTEPS = L::KSTEPS, OPER_BYTES = L::OPER_BYTES, SF_ATOMS = L::SF_ATOMS, SF_BYTES = L::SF_BYTES;
+  constexpr uint32_t STAGE_BYTES_CTA = L::STAGE_BYTES_CTA, OPER_SBO = L::OPER_SBO, OPER_SWIZZLE = L::OPER_SWIZZLE;
   constexpr int OFF_A = L::OFF_A, OFF_B = L::OFF_B, OFF_SF = L::OFF_SF, OFF_EPI = L::OFF_EPI, OFF_HALF = L::OFF_HALF,
                 OFF_BAR = L::OFF_BAR;
   extern __shared__ uint8_t smem_raw[];
@@ -393,8 +401,8 @@ k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ Ge
           tc_fence_after();
           const uint32_t sf_t = tmem_base + TMEM_SF_COL;
           const uint8_t* sf = smem + OFF_SF + st * SF_BYTES;
-          const uint64_t adesc = umma_desc(smem_u32(smem + OFF_A + st * OPER_BYTES), 1024, 2);
-          const uint64_t bdesc = umma_desc(smem_u32(smem + OFF_B + st * OPER_BYTES), 1024, 2);
+          const uint64_t adesc = umma_desc(smem_u32(smem + OFF_A + st * OPER_BYTES), OPER_SBO, OPER_SWIZZLE);
+          const uint64_t bdesc = umma_desc(smem_u32(smem + OFF_B + st * OPER_BYTES), OPER_SBO, OPER_SWIZZLE);
 #pragma unroll
           for (int k = 0; k < KSTEPS; ++k) {
             tc_cp_sf2(sf_t, umma_desc(smem_u32(sf + k * 512), 128, 0));
@@ -896,10 +904,21 @@ cudaError_t gemm_pair_set_attributes() {
   return cudaSuccess;
 }
 
+// Elements of K per operand stage of a mode: the operand and scale descriptors of a problem are built
+// with boxes of that depth.
+int gemm_pair_stage_k(GemmMode mode) {
+  switch (mode) {
+    case kG1: return Lay<kG1>::BK;
+    case kG2: return Lay<kG2>::BK;
+    case kG3: return Lay<kG3>::BK;
+    default: return Lay<kPlain>::BK;
+  }
+}
+
 // `launch` carries tile counts in 128-blocks; all of M, N, K must be multiples of 256.
 cudaError_t launch_gemm_pair(GemmMode mode, const ProblemPack& pack, const GemmLaunch& launch, int sms,
                              cudaStream_t st) {
-  if ((launch.tiles_m & 1) || (launch.tiles_n & 1) || (launch.K % BK)) return cudaErrorInvalidValue;
+  if ((launch.tiles_m & 1) || (launch.tiles_n & 1) || (launch.K % 256)) return cudaErrorInvalidValue;
   if (launch.num_problems < 1 || launch.num_problems > kPackMax) return cudaErrorInvalidValue;
   GemmLaunch L = launch;
   L.tiles_m = launch.tiles_m / 2;

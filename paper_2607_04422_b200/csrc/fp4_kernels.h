@@ -155,10 +155,11 @@ struct PrologueItem {
   bool store_x;   // write X0 in FP32 (not needed when the first G3 stage reads G itself)
   int64_t x_rows, x_cols;  // extent and row pitch of X: the work shape in the workspace, the caller's shape in `out`
   uint32_t* hist_top;      // the caller's histogram of the top 13 magnitude bits of G, or null
+  const CUtensorMap* tmG;  // G as an FP32 tensor: box = 32 columns x 128 rows, 128-byte swizzle
 };
 // count matrices that share the shape (s, l) and the clip / eps parameters
 cudaError_t launch_prologue_group(const PrologueItem* items, int count, int write_q, const QuantOpts& q,
-                                  cudaStream_t st);
+                                  uint32_t* status, cudaStream_t st);
 // Root's parameter update on BF16 weights: decay = fl(1 - fl(lr * wd)), step = fl(lr * scale),
 // w <- BF16(fl(fl(w * decay) - fl(step * o))).
 struct ParamUpdate {
@@ -183,6 +184,7 @@ cudaError_t gemm_pair_set_attributes();
 cudaError_t launch_gemm_pair(GemmMode mode, const ProblemPack& pack, const GemmLaunch& launch, int sms,
                              cudaStream_t st);
 int gemm_stage_k();  // elements of K per operand stage (the codes maps' box is this / 2 bytes wide)
+int gemm_pair_stage_k(GemmMode mode);  // the same for a mode of the CTA-pair kernel
 cudaError_t launch_gemm(GemmMode mode, const ProblemPack& pack, const GemmLaunch& launch, int sms, cudaStream_t st);
 
 }  // namespace fp4

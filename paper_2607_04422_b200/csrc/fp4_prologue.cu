@@ -19,6 +19,7 @@
 // over the matrix and a statistics pass (slow, rare, no extra launch).
 #include <stddef.h>
 
+#include "fp4_gemm_common.cuh"
 #include "fp4_kernels.h"
 
 namespace fp4 {
@@ -59,6 +60,8 @@ struct PrepGroup {
   int zero_words;      // 32-bit words of header + scalars + histogram to clear
   QuantOpts q;         // quantiser options of X0's operand copies
   NsScalarIdx ix;
+  uint32_t* status;    // the call's status word
+  CUtensorMap tmG[kMaxPack];  // the callers' matrices as FP32 tensors, box = 32 columns x 128 rows, 128-byte swizzle
 };
 
 __device__ __forceinline__ uint32_t mag_bits(float x) { return __float_as_uint(x) & 0x7FFFFFFFu; }
@@ -441,127 +444,424 @@ __global__ void __launch_bounds__(1024) kp_finalize(const __grid_constant__ Prep
 }
 
 // ---- X0 = clamp(G) * inv in the work orientation (s x l; transposed when G is tall), its FP32
-// copy (unless the first G3 stage will form X0 from G itself), and both NVFP4 operand copies.  One 128 x 128 tile of X per block, gridDim.z = matrix.
-// Row pitch of the shared tile in floats: 132 (16-byte aligned rows: 128-bit shared accesses
-// along a row, conflict-free per quarter-warp) when the tile is filled row by row; 129 (odd)
-// for a tall input, whose tile is filled transposed with 4-byte stores.
-constexpr int kPitchWide = 132, kPitchTall = 129;
+// copy (unless the first G3 stage will form X0 from G itself), and both NVFP4 operand copies.
+//
+// A persistent block per SM walks 128 x 128 tiles of G.  Three tiles are kept in flight with TMA
+// (64 KB each, four 32-column boxes with the 128-byte swizzle; what lies outside the caller's
+// matrix arrives as zeros, which is the padding of the work shape).  Thirty-two warps quantise the
+// tiles as they land: sixteen along the rows (a warp takes 8 rows, a thread one 32-column box of a
+// row), sixteen along the columns (a warp takes a band of 16 rows and 64 columns, a thread two
+// columns).  The tile is never transposed: for a tall G the two passes simply swap destinations
+// (blocks along the rows of G are blocks along the columns of X = G^T).  The row pass writes its
+// codes itself (the four lanes of a row fill 64 contiguous bytes); the column pass's codes (8 bytes
+// per column) and both kinds of scale bytes are staged in shared memory and leave as 64-byte rows
+// and whole 512-byte atoms.
+// One block-wide barrier per tile: after it the tile's buffer is refilled and the staged bytes go out.
+// Tile buffers and staging areas form rings of three.
+constexpr int kPrepBufs = 3;
+constexpr int kPrepTile = 128 * 128 * 4;       // bytes of a tile
+constexpr int kPrepBox = 32 * 128 * 4;         // bytes of one 32-column box
+constexpr int kQtSlot = 1024 + 16;             // staged column codes: [band][column][8 B], padded bands
+constexpr int kPrepStage = 8 * kQtSlot + 2 * 1024;  // + two scale atoms per pass
+constexpr int kPrepWarps = 32;
+constexpr int kPrepThreads = kPrepWarps * 32;
+
+struct PrepTileInfo { int mi, gr0, gc0, pad; };  // matrix, origin of the tile in G
+struct PrepShared {
+  uint64_t full[kPrepBufs];
+  uint32_t abort_flag;
+  PrepTileInfo info[4];           // tiles it .. it + 3 of this block (ring)
+  float rcp_tab[kMaxPack][8];     // per matrix: fl(1 / fl((8 + j) sg))
+};
+constexpr int kPrepSmem = kPrepBufs * (kPrepTile + kPrepStage) + (int)sizeof(PrepShared) + 1024;
+static_assert(kPrepSmem <= 232448, "at most 227 KB of dynamic shared memory");
+
+// address of the 16-byte piece c4 (0..31) of row r in a tile of four swizzled boxes
+__device__ __forceinline__ uint32_t prep_piece(uint32_t tile, int r, int c4) {
+  return tile + (uint32_t)((c4 >> 3) * kPrepBox + r * 128 + (((c4 & 7) ^ (r & 7)) << 4));
+}
+__device__ __forceinline__ float4 lds128f(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ float lds32f(uint32_t addr) {
+  float v;
+  asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
+  return v;
+}
+// Eight FP32 -> four bytes of E2M1 codes (v0 in bits 3:0 ... v7 in bits 31:28).
+__device__ __forceinline__ uint32_t cvt_e2m1x8(float v0, float v1, float v2, float v3, float v4, float v5, float v6,
+                                               float v7) {
+  uint32_t r;
+  asm("{\n\t.reg .b8 t0, t1, t2, t3;\n\t"
+      "cvt.rn.satfinite.e2m1x2.f32 t0, %2, %1;\n\t"
+      "cvt.rn.satfinite.e2m1x2.f32 t1, %4, %3;\n\t"
+      "cvt.rn.satfinite.e2m1x2.f32 t2, %6, %5;\n\t"
+      "cvt.rn.satfinite.e2m1x2.f32 t3, %8, %7;\n\t"
+      "mov.b32 %0, {t0, t1, t2, t3};\n\t}"
+      : "=r"(r)
+      : "f"(v0), "f"(v1), "f"(v2), "f"(v3), "f"(v4), "f"(v5), "f"(v6), "f"(v7));
+  return r;
+}
+
+// ---- block quantisers of the operand preparation.
+// They quantise x0 = clamp(g, +-tau) * inv (quantize_block16 applied to x0) with fewer instructions,
+// bit for bit the same result; whatever the short cuts do not cover goes to quantize_block16 itself.
+//  * No clamp per element.  With y = fl(g * inv) and tinv = fl(tau * inv), rounding is monotonic, so
+//    x0 = clamp(y, +-tinv) exactly and the block's amax is min(max |y|, tinv).  An element beyond the clip
+//    level would be quantised from fl(tinv * rcp), which lies near 6 (the block's scale maps its amax = tinv
+//    there); every larger product saturates to the same code 6.  Checked per matrix: fl(tinv * rcp) > 5
+//    for the scale byte of a block whose amax is tinv.
+//  * The scale byte is E4M3(fl(amax / 6sg)).  q = amax * fl(1 / 6sg) with one correction step
+//    (r = amax - q * 6sg exactly by FMA, q += r * fl(1 / 6sg)) is within one ulp of the correctly rounded
+//    quotient, so both convert to the same byte unless q lies within two ulps of a rounding boundary of
+//    E4M3 (mantissa bits 19..0 = 0x80000 in the normal range); those blocks, and scale bytes <= 8
+//    (subnormal E4M3, where the boundaries lie elsewhere), take the exact path.
+//  * The reciprocal of the decoded scale d = fl(s * sg), s = (8 + m) 2^(E - 10): for sg far from the ends
+//    of the exponent range d = fl((8 + m) sg) 2^(E - 10) exactly, so fl(1 / d) is one of eight values per
+//    matrix with the exponent shifted; the eight values fl(1 / fl((8 + j) sg)) lie in shared memory.
+struct PrepScalars {
+  float tau, inv, tinv, six_sg, rcp_six_sg, sg;
+  uint32_t rcp_tab;     // shared-memory address of the matrix's eight reciprocals
+  uint32_t near_limit;  // 4 when the short cuts hold for this matrix (sg in [2^-60, 2^60], and the clip level
+                        // itself is quantised to 6: fl(tinv * rcp) > 5 for the scale of a clipped block), else all ones
+};
+
+__device__ __noinline__ uint32_t prep_quant_exact(const float (&gv)[16], float tau, float inv, float six_sg, float sg,
+                                                  uint32_t& lo, uint32_t& hi) {
+  float v[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) v[i] = __fmul_rn(fminf(fmaxf(gv[i], -tau), tau), inv);
+  return quantize_block16(v, six_sg, sg, lo, hi);
+}
+
+// amax (of |y|, not yet limited to tinv) -> scale byte and fl(1 / d); `rare` is set when the block must take
+// the exact path.
+__device__ __forceinline__ uint32_t prep_scale(const PrepScalars& ps, float amax_y, float& rcp, bool& rare) {
+  const float amax = fminf(amax_y, ps.tinv);
+  float q = __fmul_rn(amax, ps.rcp_six_sg);
+  const float r = __fmaf_rn(-q, ps.six_sg, amax);
+  q = __fmaf_rn(r, ps.rcp_six_sg, q);
+  const uint32_t sb = cvt_ue4m3(q);
+  uint32_t tab;
+  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tab) : "r"(ps.rcp_tab + ((sb & 7u) << 2)));
+  rcp = __uint_as_float(tab - (((sb >> 3) - 10u) << 23));
+  const uint32_t near = (__float_as_uint(q) + 2u - 0x80000u) & 0xFFFFFu;
+  // q < 1.0625 * 2^-6: scale bytes <= 8 (and the boundary to 9)
+  rare = near <= ps.near_limit || q < 0.0166015625f;
+  return sb;
+}
+
+// One block of 16 consecutive elements, given as four 16-byte pieces of two packed pairs each.
+// `rare`: the caller must redo the block with prep_quant_exact.
+__device__ __forceinline__ uint32_t prep_quant_row(uint64_t (&y2)[8], const PrepScalars& ps, uint32_t& lo,
+                                                   uint32_t& hi, bool& rare) {
+  const uint64_t inv2 = pack2(ps.inv, ps.inv);
+  float m8[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    float a, b;
+    y2[i] = mul2(y2[i], inv2);
+    unpack2(y2[i], a, b);
+    m8[i] = fmaxf(fabsf(a), fabsf(b));
+  }
+  const float amax_y = fmaxf(fmaxf(fmaxf(m8[0], m8[1]), fmaxf(m8[2], m8[3])),
+                             fmaxf(fmaxf(m8[4], m8[5]), fmaxf(m8[6], m8[7])));
+  float rcp;
+  const uint32_t sb = prep_scale(ps, amax_y, rcp, rare);
+  const uint64_t rcp2 = pack2(rcp, rcp);
+  float z[16];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) unpack2(mul2(y2[i], rcp2), z[2 * i], z[2 * i + 1]);
+  lo = cvt_e2m1x8(z[0], z[1], z[2], z[3], z[4], z[5], z[6], z[7]);
+  hi = cvt_e2m1x8(z[8], z[9], z[10], z[11], z[12], z[13], z[14], z[15]);
+  return sb;
+}
+
+// Two blocks side by side: g2[i] = the elements of row i in two neighbouring columns; block j runs down
+// column j.  The pairs stay together through both multiplications.  Returns the two scale bytes.
+__device__ __forceinline__ void prep_quant_col2(uint64_t (&y2)[16], const PrepScalars& ps, uint32_t (&cw)[4],
+                                                uint32_t& sb0, uint32_t& sb1, bool& rare) {
+  const uint64_t inv2 = pack2(ps.inv, ps.inv);
+  float ax = 0.0f, ay = 0.0f;
+#pragma unroll
+  for (int i = 0; i < 16; i += 2) {
+    float a, b, c, d;
+    y2[i] = mul2(y2[i], inv2);
+    y2[i + 1] = mul2(y2[i + 1], inv2);
+    unpack2(y2[i], a, b);
+    unpack2(y2[i + 1], c, d);
+    ax = fmaxf(ax, fmaxf(fabsf(a), fabsf(c)));
+    ay = fmaxf(ay, fmaxf(fabsf(b), fabsf(d)));
+  }
+  float r0, r1;
+  bool rare0, rare1;
+  sb0 = prep_scale(ps, ax, r0, rare0);
+  sb1 = prep_scale(ps, ay, r1, rare1);
+  const uint64_t rcp2 = pack2(r0, r1);
+  float zx[16], zy[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) unpack2(mul2(y2[i], rcp2), zx[i], zy[i]);
+  cw[0] = cvt_e2m1x8(zx[0], zx[1], zx[2], zx[3], zx[4], zx[5], zx[6], zx[7]);
+  cw[1] = cvt_e2m1x8(zx[8], zx[9], zx[10], zx[11], zx[12], zx[13], zx[14], zx[15]);
+  cw[2] = cvt_e2m1x8(zy[0], zy[1], zy[2], zy[3], zy[4], zy[5], zy[6], zy[7]);
+  cw[3] = cvt_e2m1x8(zy[8], zy[9], zy[10], zy[11], zy[12], zy[13], zy[14], zy[15]);
+  rare = rare0 || rare1;
+}
 
 template <bool PF>
-__global__ void __launch_bounds__(512, 3) kp_prep_operands(const __grid_constant__ PrepGroup g) {
-  extern __shared__ float xs[];  // [128][pitch]
-  const PrepMatrix& m = g.mat[blockIdx.z];
-  const int64_t s = g.s, l = g.l;
-  const int tall = m.tall;
-  const int P = tall ? kPitchTall : kPitchWide;
-  const int64_t ldg = tall ? g.s0 : g.l0;  // row length of G: a tall G is l0 x s0
-  const float tau = g.clip ? m.scalars[g.ix.tau] : __int_as_float(0x7f800000);
-  const float inv = m.scalars[g.ix.inv];
-  const float sg = m.scalars[g.ix.sg_X0];
-  const float six_sg = __fmul_rn(6.0f, sg);
-  const int64_t r0 = (int64_t)blockIdx.y * 128, c0 = (int64_t)blockIdx.x * 128;  // tile origin in X
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+__global__ void __launch_bounds__(kPrepThreads, 1) kp_prep_operands(const __grid_constant__ PrepGroup g) {
+  extern __shared__ uint8_t prep_smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(prep_smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint8_t* stage_base = smem + kPrepBufs * kPrepTile;
+  PrepShared* sh = reinterpret_cast<PrepShared*>(stage_base + kPrepBufs * kPrepStage);
+  volatile uint32_t* abort_flag = &sh->abort_flag;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tiles_per_matrix = (int)((g.s >> 7) * (g.l >> 7));
+  const int total = tiles_per_matrix * g.count;
+  const int my_tiles = (total - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;  // tiles of this block
 
-  // The tile holds raw G values; clamp and scale are applied where a pass reads them.  A wide
-  // input's rows go straight to shared memory with asynchronous 16-byte copies (64 KB in flight
-  // per block without holding registers); a tall input's tile is filled transposed from registers.
-  auto x0 = [&](float gval) { return __fmul_rn(fminf(fmaxf(gval, -tau), tau), inv); };
-  // Rows and columns beyond the caller's matrix are zero padding (source size 0 of the copy
-  // fills with zeros); the dimensions are multiples of 16, so a 16-byte piece is all in or all out.
-  if (!tall) {
+  // Tile `it` of this block: work out where it lies, publish that in the ring and start its copy.  Called by
+  // one thread, a block-wide barrier before the tile's turn.
+  auto fetch = [&](int it_) {
+    if (it_ >= my_tiles) return;
+    const int t_ = (int)blockIdx.x + it_ * (int)gridDim.x;
+    const int b_ = it_ % kPrepBufs;
+    PrepTileInfo ti;
+    ti.pad = 0;
+    ti.mi = t_ / tiles_per_matrix;
+    const int r_ = t_ - ti.mi * tiles_per_matrix;
+    const int tiles_x = (int)((g.mat[ti.mi].tall ? g.s : g.l) >> 7);  // tiles along a row of G
+    const int ty = r_ / tiles_x;
+    ti.gr0 = ty * 128;
+    ti.gc0 = (r_ - ty * tiles_x) * 128;
+    sh->info[it_ & 3] = ti;
+    mbar_expect_tx(&sh->full[b_], kPrepTile);
 #pragma unroll
-    for (int rr = warp; rr < 128; rr += 16) {
-      const bool in = (r0 + rr) < g.s0 && (c0 + lane * 4) < g.l0;
-      const float* src = in ? m.G + (r0 + rr) * ldg + c0 + lane * 4 : m.G;
-      asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_u32(xs + rr * P + lane * 4)), "l"(src),
-                   "r"(in ? 16 : 0)
-                   : "memory");
-    }
-    asm volatile("cp.async.wait_all;" ::: "memory");
-  } else {
-#pragma unroll 4
-    for (int rr = warp; rr < 128; rr += 16) {
-      const bool in = (c0 + rr) < g.l0 && (r0 + lane * 4) < g.s0;
-      float4 v = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-      if (in) v = __ldg(reinterpret_cast<const float4*>(m.G + (c0 + rr) * ldg + r0) + lane);
-      xs[(lane * 4 + 0) * P + rr] = v.x; xs[(lane * 4 + 1) * P + rr] = v.y;
-      xs[(lane * 4 + 2) * P + rr] = v.z; xs[(lane * 4 + 3) * P + rr] = v.w;
-    }
+    for (int q = 0; q < 4; ++q)
+      tma_load_2d(smem + b_ * kPrepTile + q * kPrepBox, &g.tmG[ti.mi], ti.gc0 + 32 * q, ti.gr0, &sh->full[b_]);
+  };
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < kPrepBufs; ++i) mbar_init(&sh->full[i], 1);
+    sh->abort_flag = 0;
+    mbar_fence_init();
+    for (int i = 0; i < kPrepBufs; ++i) fetch(i);
+  }
+  if (threadIdx.x < g.count * 8) {
+    const float sg_ = g.mat[threadIdx.x >> 3].scalars[g.ix.sg_X0];
+    sh->rcp_tab[threadIdx.x >> 3][threadIdx.x & 7] = __frcp_rn(__fmul_rn((float)(8 + (threadIdx.x & 7)), sg_));
   }
   __syncthreads();
-  if (m.store_x) {
-#pragma unroll 4
-    for (int rr = warp; rr < 128; rr += 16) {
-      const float* row = xs + rr * P + lane * 4;
-      if ((r0 + rr) < m.x_rows && (c0 + lane * 4) < m.x_cols)
-        *reinterpret_cast<float4*>(m.X + (r0 + rr) * m.x_cols + c0 + lane * 4) =
-            make_float4(x0(row[0]), x0(row[1]), x0(row[2]), x0(row[3]));
+
+  // lane-dependent parts of the shared-memory addresses, fixed for the whole kernel
+  const bool row_warp = warp < kPrepWarps / 2;
+  //   row pass: a warp takes 8 rows, a thread one 32-column box of a row (two blocks)
+  const int rr = (warp & 15) * 8 + (lane & 7), box = lane >> 3;
+  //   column pass: a warp takes a band of 16 rows and 64 columns, a thread two columns
+  const int cwp = warp & 15, band = cwp >> 1, cp = (cwp & 1) * 32 + lane;  // cp: column pair 0..63
+  uint32_t base_off, sw;
+  if (row_warp) { base_off = (uint32_t)(box * kPrepBox + rr * 128); sw = (uint32_t)(rr & 7) << 4; }
+  else { base_off = (uint32_t)((cp >> 4) * kPrepBox + band * 16 * 128 + (cp & 1) * 8); sw = (uint32_t)((cp >> 1) & 7) << 4; }
+
+  int cur = -1;
+  PrepScalars ps;
+  ps.tau = ps.inv = ps.tinv = ps.six_sg = ps.rcp_six_sg = ps.sg = 0.0f; ps.rcp_tab = 0; ps.near_limit = 0;
+  for (int it = 0; it < my_tiles; ++it) {
+    const int b = it % kPrepBufs, use = it / kPrepBufs;
+    const PrepTileInfo ti = sh->info[it & 3];   // written before an earlier barrier
+    wait_or_abort(&sh->full[b], (uint32_t)use & 1u, abort_flag);
+    const int mi = ti.mi, gr0 = ti.gr0, gc0 = ti.gc0;
+    const PrepMatrix& m = g.mat[mi];
+    if (mi != cur) {
+      cur = mi;
+      ps.tau = g.clip ? m.scalars[g.ix.tau] : __int_as_float(0x7f800000);
+      ps.inv = m.scalars[g.ix.inv];
+      ps.tinv = __fmul_rn(ps.tau, ps.inv);
+      ps.sg = m.scalars[g.ix.sg_X0];
+      ps.six_sg = __fmul_rn(6.0f, ps.sg);
+      ps.rcp_six_sg = __frcp_rn(ps.six_sg);
+      ps.rcp_tab = smem_u32(&sh->rcp_tab[mi][0]);
+      const uint32_t esg = (__float_as_uint(ps.sg) >> 23) & 0xFFu;
+      bool ok = esg >= 67u && esg <= 187u;   // 2^-60 .. 2^60
+      if (ps.tinv < __int_as_float(0x7f800000)) {
+        // a block with clipped elements has amax = tinv: is the clip level quantised to 6 there?
+        const float dc = __fmul_rn(ue4m3_to_float(cvt_ue4m3(__fdiv_rn(ps.tinv, ps.six_sg))), ps.sg);
+        ok = ok && dc != 0.0f && __fmul_rn(ps.tinv, __frcp_rn(dc)) > 5.0f;
+      }
+      ps.near_limit = ok ? 4u : 0xFFFFFFFFu;
     }
-  }
-  if (!g.write_q) return;
-  const int part = (warp & 7) >> 2;  // which four of the eight 16-blocks this thread takes
-  uint32_t code[8];                  // the codes of those four blocks: 32 consecutive bytes of the operand row
-  uint32_t sfw = 0;
-  if (warp < 8) {
-    // blocks along the columns of X (contraction axis of G1): thread = row
-    const int rr = (warp & 3) * 32 + lane;
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const int kb = part * 4 + q;
-      float v[16];
-      if (tall) {
-#pragma unroll
-        for (int i = 0; i < 16; ++i) v[i] = x0(xs[rr * P + kb * 16 + i]);
+    auto x0 = [&](float gval) { return __fmul_rn(fminf(fmaxf(gval, -ps.tau), ps.tau), ps.inv); };
+    const uint32_t tile = smem_u32(smem + b * kPrepTile);
+    uint8_t* stage = stage_base + b * kPrepStage;
+    const int tall = m.tall;
+
+    if (m.store_x) {
+      if (!tall) {
+        // X = G: rows of the tile are rows of X
+#pragma unroll 4
+        for (int r = warp; r < 128; r += kPrepWarps) {
+          const float4 v = lds128f(prep_piece(tile, r, lane));
+          if ((gr0 + r) < m.x_rows && (gc0 + lane * 4) < m.x_cols)
+            *reinterpret_cast<float4*>(m.X + (int64_t)(gr0 + r) * m.x_cols + gc0 + lane * 4) =
+                make_float4(x0(v.x), x0(v.y), x0(v.z), x0(v.w));
+        }
       } else {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const float4 t = *reinterpret_cast<const float4*>(xs + rr * P + kb * 16 + i * 4);
-          v[4 * i] = x0(t.x); v[4 * i + 1] = x0(t.y); v[4 * i + 2] = x0(t.z); v[4 * i + 3] = x0(t.w);
+        // X = G^T: a lane group of 8 consecutive tile rows writes one 32-byte sector of a row of X;
+        // the 8 rows x 4 columns a warp reads at once lie in 32 different banks
+        const int r8 = lane & 7, cq = lane >> 3;
+#pragma unroll 4
+        for (int k = 0; k < 512 / kPrepWarps; ++k) {
+          const int p = warp * (512 / kPrepWarps) + k;
+          const int row = (p & 15) * 8 + r8, col = (p >> 4) * 4 + cq;
+          const float v = lds32f(prep_piece(tile, row, col >> 2) + (uint32_t)(col & 3) * 4u);
+          if ((gc0 + col) < m.x_rows && (gr0 + row) < m.x_cols) m.X[(int64_t)(gc0 + col) * m.x_cols + gr0 + row] = x0(v);
         }
       }
-      uint32_t sb;
-      float unused;
-      if (PF) sb = quantize_block16_opts(v, g.q, sg, code[2 * q], code[2 * q + 1], unused);
-      else sb = quantize_block16(v, six_sg, sg, code[2 * q], code[2 * q + 1]);
-      sfw |= sb << (8 * q);
     }
-    uint4* dst = reinterpret_cast<uint4*>(m.qx_codes + (r0 + rr) * (l / 2) + (c0 + part * 64) / 2);
-    dst[0] = make_uint4(code[0], code[1], code[2], code[3]);
-    dst[1] = make_uint4(code[4], code[5], code[6], code[7]);
-    *reinterpret_cast<uint32_t*>(m.qx_sf + sf_offset(r0 + rr, c0 / 16 + part * 4, l / 16)) = sfw;
-  } else {
-    // blocks along the rows of X (contraction axis of G3): thread = column of X = row of X^T
-    const int cc = (warp & 3) * 32 + lane;
+
+    // destinations of the two passes: blocks along the rows of G are qX for a wide G, qX^T for a tall one
+    const int64_t rp_k = tall ? g.s : g.l, cp_k = tall ? g.l : g.s;  // contraction length of each destination
+    if (g.write_q) {
+      uint8_t* sf_stage = stage + 8 * kQtSlot;
+      const uint32_t tb = tile + base_off;
+      if (row_warp) {
+        uint32_t code[4];
+        uint32_t sfw = 0;
+        bool redo = false;
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const int gq = part * 4 + q;
-      float v[16];
+        for (int q = 0; q < 2; ++q) {
+          uint64_t g2[8];
 #pragma unroll
-      for (int i = 0; i < 16; ++i) v[i] = x0(xs[(gq * 16 + i) * P + cc]);
-      uint32_t sb;
-      float unused;
-      if (PF) sb = quantize_block16_opts(v, g.q, sg, code[2 * q], code[2 * q + 1], unused);
-      else sb = quantize_block16(v, six_sg, sg, code[2 * q], code[2 * q + 1]);
-      sfw |= sb << (8 * q);
+          for (int i = 0; i < 4; ++i)
+            asm volatile("ld.shared.v2.b64 {%0, %1}, [%2];"
+                         : "=l"(g2[2 * i]), "=l"(g2[2 * i + 1])
+                         : "r"(tb + (((uint32_t)(q * 4 + i) << 4) ^ sw)));
+          uint32_t sb;
+          if (PF) {
+            float v[16], unused;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              float a, b2;
+              unpack2(g2[i], a, b2);
+              v[2 * i] = x0(a); v[2 * i + 1] = x0(b2);
+            }
+            sb = quantize_block16_opts(v, g.q, ps.sg, code[2 * q], code[2 * q + 1], unused);
+          } else {
+            bool rare;
+            sb = prep_quant_row(g2, ps, code[2 * q], code[2 * q + 1], rare);
+            redo = redo || rare;
+          }
+          sfw |= sb << (8 * q);
+        }
+        if (!PF && redo) {   // rare: both blocks again from the tile, with the plain quantiser
+          sfw = 0;
+#pragma unroll 1
+          for (int q = 0; q < 2; ++q) {
+            float gv[16];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const float4 f = lds128f(tb + (((uint32_t)(q * 4 + i) << 4) ^ sw));
+              gv[4 * i] = f.x; gv[4 * i + 1] = f.y; gv[4 * i + 2] = f.z; gv[4 * i + 3] = f.w;
+            }
+            sfw |= prep_quant_exact(gv, ps.tau, ps.inv, ps.six_sg, ps.sg, code[2 * q], code[2 * q + 1]) << (8 * q);
+          }
+        }
+        // the four lanes of a row write 64 contiguous bytes
+        uint8_t* rp_codes = tall ? m.qt_codes : m.qx_codes;
+        *reinterpret_cast<uint4*>(rp_codes + (int64_t)(gr0 + rr) * (rp_k / 2) + gc0 / 2 + box * 16) =
+            make_uint4(code[0], code[1], code[2], code[3]);
+        *reinterpret_cast<uint16_t*>(sf_stage + (box >> 1) * 512 + (rr & 31) * 16 + (rr >> 5) * 4 + (box & 1) * 2) =
+            (uint16_t)sfw;
+      } else {
+        uint64_t g2[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          // row band * 16 + i of the tile: its low three bits are those of i
+          const uint32_t a = tb + (uint32_t)(i * 128) + (sw ^ ((uint32_t)(i & 7) << 4));
+          asm volatile("ld.shared.b64 %0, [%1];" : "=l"(g2[i]) : "r"(a));
+        }
+        uint32_t cw[4], sb0 = 0, sb1 = 0;
+        if (PF) {
+          float unused;
+#pragma unroll
+          for (int j = 0; j < 2; ++j) {
+            float v[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              float a, b2;
+              unpack2(g2[i], a, b2);
+              v[i] = x0(j == 0 ? a : b2);
+            }
+            const uint32_t sb = quantize_block16_opts(v, g.q, ps.sg, cw[2 * j], cw[2 * j + 1], unused);
+            if (j == 0) sb0 = sb; else sb1 = sb;
+          }
+        } else {
+          bool rare;
+          prep_quant_col2(g2, ps, cw, sb0, sb1, rare);
+          if (rare) {   // redo both blocks from the tile with the plain quantiser
+#pragma unroll 1
+            for (int j = 0; j < 2; ++j) {
+              float gv[16];
+#pragma unroll
+              for (int i = 0; i < 16; ++i)
+                gv[i] = lds32f(tb + (uint32_t)(i * 128 + j * 4) + (sw ^ ((uint32_t)(i & 7) << 4)));
+              const uint32_t sb = prep_quant_exact(gv, ps.tau, ps.inv, ps.six_sg, ps.sg, cw[2 * j], cw[2 * j + 1]);
+              if (j == 0) sb0 = sb; else sb1 = sb;
+            }
+          }
+        }
+        uint8_t* sfc = sf_stage + 1024 + (band >> 2) * 512 + (band & 3);
+        const int c = cp * 2;
+        sfc[(c & 31) * 16 + (c >> 5) * 4] = (uint8_t)sb0;
+        sfc[((c + 1) & 31) * 16 + ((c + 1) >> 5) * 4] = (uint8_t)sb1;
+        *reinterpret_cast<uint4*>(stage + band * kQtSlot + cp * 16) = make_uint4(cw[0], cw[1], cw[2], cw[3]);
+      }
     }
-    uint4* dst = reinterpret_cast<uint4*>(m.qt_codes + (c0 + cc) * (s / 2) + (r0 + part * 64) / 2);
-    dst[0] = make_uint4(code[0], code[1], code[2], code[3]);
-    dst[1] = make_uint4(code[4], code[5], code[6], code[7]);
-    *reinterpret_cast<uint32_t*>(m.qt_sf + sf_offset(c0 + cc, r0 / 16 + part * 4, s / 16)) = sfw;
+
+    // Every warp has read the tile and staged its output: the buffer takes the tile three ahead, the
+    // staged bytes go out.
+    __syncthreads();
+    if (threadIdx.x == kPrepThreads - 32) {
+      fence_proxy_async_smem();
+      fetch(it + kPrepBufs);
+    }
+    if (g.write_q) {
+      const int tid = threadIdx.x;
+      if (tid < 512) {
+        // column-pass codes: row (gc0 + c) of the destination, 64 bytes from byte gr0 / 2; four lanes per row
+        uint8_t* cp_codes = tall ? m.qx_codes : m.qt_codes;
+        const int c = tid >> 2, h = tid & 3;
+        const uint8_t* src = stage + c * 8;
+        const uint2 a = *reinterpret_cast<const uint2*>(src + (2 * h) * kQtSlot);
+        const uint2 d = *reinterpret_cast<const uint2*>(src + (2 * h + 1) * kQtSlot);
+        *reinterpret_cast<uint4*>(cp_codes + (int64_t)(gc0 + c) * (cp_k / 2) + gr0 / 2 + h * 16) = make_uint4(a.x, a.y, d.x, d.y);
+      } else if (tid < 640) {
+        // scale atoms: two adjacent 512-byte atoms per pass
+        const bool rowpass = tid < 576;
+        uint8_t* sf_base = rowpass ? (tall ? m.qt_sf : m.qx_sf) : (tall ? m.qx_sf : m.qt_sf);
+        const int64_t row0 = rowpass ? gr0 : gc0, k0 = rowpass ? gc0 : gr0, kk = rowpass ? rp_k : cp_k;
+        const int j = tid & 63;
+        const uint4 w = *reinterpret_cast<const uint4*>(stage + 8 * kQtSlot + (rowpass ? 0 : 1024) + j * 16);
+        *reinterpret_cast<uint4*>(sf_base + sf_offset(row0, k0 / 16, kk / 16) + j * 16) = w;
+      }
+    }
   }
+  if (threadIdx.x == 0 && sh->abort_flag) report_timeout(g.status);
 }
 
 }  // namespace
 
 cudaError_t prologue_set_attributes() {
-  cudaError_t e = cudaFuncSetAttribute(kp_prep_operands<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * kPitchWide * 4);
+  cudaError_t e = cudaFuncSetAttribute(kp_prep_operands<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPrepSmem);
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(kp_prep_operands<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * kPitchWide * 4);
+  return cudaFuncSetAttribute(kp_prep_operands<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kPrepSmem);
 }
 
 // Enqueue the prologue for `count` matrices of one shape (s, l) and one parameter set.
 cudaError_t launch_prologue_group(const PrologueItem* items, int count, int write_q, const QuantOpts& q,
-                                  cudaStream_t st) {
+                                  uint32_t* status, cudaStream_t st) {
   for (int i0 = 0; i0 < count; i0 += kMaxPack) {
     const int nn = count - i0 < kMaxPack ? count - i0 : kMaxPack;
     const NsPlan& pl = *items[i0].pl;
@@ -581,6 +881,7 @@ cudaError_t launch_prologue_group(const PrologueItem* items, int count, int writ
     g.zero_words = (int)(pl.zero_bytes / 4);
     g.ix = pl.ix;
     g.q = q;
+    g.status = status;
     bool all_counted = true;
     for (int j = 0; j < nn; ++j) {
       const PrologueItem& it = items[i0 + j];
@@ -600,6 +901,7 @@ cudaError_t launch_prologue_group(const PrologueItem* items, int count, int writ
       m.x_rows = it.x_rows; m.x_cols = it.x_cols;
       m.hist_top = it.hist_top;
       if (!it.hist_top) all_counted = false;
+      g.tmG[j] = *it.tmG;
     }
     const int sms = pl.sms;
     int64_t hb = (g.n4 + 512 * 4 - 1) / (512 * 4);
@@ -623,9 +925,10 @@ cudaError_t launch_prologue_group(const PrologueItem* items, int count, int writ
     }
     {
       ProfScope ps(FP4_PROF_PREP, st);
-      const dim3 gp((unsigned)(pl.l / 128), (unsigned)(pl.s / 128), (unsigned)nn);
-      if (q.rht || q.four_six) kp_prep_operands<true><<<gp, 512, 128 * kPitchWide * 4, st>>>(g);
-      else kp_prep_operands<false><<<gp, 512, 128 * kPitchWide * 4, st>>>(g);
+      const int64_t tiles = (pl.l / 128) * (pl.s / 128) * nn;
+      const unsigned gp = (unsigned)(tiles < sms ? tiles : sms);
+      if (q.rht || q.four_six) kp_prep_operands<true><<<gp, kPrepThreads, kPrepSmem, st>>>(g);
+      else kp_prep_operands<false><<<gp, kPrepThreads, kPrepSmem, st>>>(g);
       count_launches(1);
     }
     cudaError_t e = cudaGetLastError();

@@ -86,10 +86,10 @@ inline int64_t pad128(int64_t v) { return (v + 127) / 128 * 128; }
 constexpr uint32_t kNsFlags =
     FP4_FLAG_KEEP_OPERANDS | FP4_FLAG_RHT | FP4_FLAG_FOUR_SIX | FP4_FLAG_STORE_BF16 | FP4_FLAG_NO_OUT;
 
-// 2-D map over a row-major byte matrix (NVFP4 codes): box = one operand stage (64 or 128 bytes
-// x 128 rows), swizzled over the box width.
-bool make_codes_map(const DeviceInfo* d, CUtensorMap* tm, const void* base, int64_t rows, int64_t row_bytes) {
-  const cuuint32_t bw = (cuuint32_t)(gemm_stage_k() / 2);
+// 2-D map over a row-major byte matrix (NVFP4 codes): box = one operand stage of `stage_k` elements of K
+// (64 or 128 bytes x 128 rows), swizzled over the box width.
+bool make_codes_map(const DeviceInfo* d, CUtensorMap* tm, const void* base, int64_t rows, int64_t row_bytes, int stage_k) {
+  const cuuint32_t bw = (cuuint32_t)(stage_k / 2);
   cuuint64_t dims[2] = {(cuuint64_t)row_bytes, (cuuint64_t)rows};
   cuuint64_t strides[1] = {(cuuint64_t)row_bytes};
   cuuint32_t box[2] = {bw, 128};
@@ -108,6 +108,18 @@ bool make_f32_map(const DeviceInfo* d, CUtensorMap* tm, const void* base, int64_
   cuuint32_t estr[2] = {1, 1};
   return d->encode(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box, estr,
                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// 2-D map over a row-major FP32 matrix for the operand preparation: box = 32 columns x 128 rows (a quarter
+// of a 128 x 128 tile), 128-byte swizzle.
+bool make_f32_tile_map(const DeviceInfo* d, CUtensorMap* tm, const void* base, int64_t rows, int64_t cols) {
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)cols * 4};
+  cuuint32_t box[2] = {32, 128};
+  cuuint32_t estr[2] = {1, 1};
+  return d->encode(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -139,12 +151,12 @@ bool make_code_store_map(const DeviceInfo* d, CUtensorMap* tm, const void* base,
 constexpr int kDefaultMaxGroup = kPackMax;
 
 // 2-D map over the scale atoms of a rows x K operand: one map row per 128-row block, 64-bit
-// elements, box = the atoms of one operand stage (256 elements = 2 KB), no swizzle.
-bool make_sf_map(const DeviceInfo* d, CUtensorMap* tm, const void* base, int64_t rows, int64_t K) {
+// elements, box = the atoms of one operand stage (`stage_k` elements of 8 bytes: 1 or 2 KB), no swizzle.
+bool make_sf_map(const DeviceInfo* d, CUtensorMap* tm, const void* base, int64_t rows, int64_t K, int stage_k) {
   if (K < 256) { memset(tm, 0, sizeof(*tm)); return true; }   // never used by the CTA-pair kernel
   cuuint64_t dims[2] = {(cuuint64_t)(K / 64) * 64, (cuuint64_t)(rows / 128)};
   cuuint64_t strides[1] = {(cuuint64_t)(K / 64) * 512};
-  cuuint32_t box[2] = {256, 1};
+  cuuint32_t box[2] = {(cuuint32_t)stage_k, 1};
   cuuint32_t estr[2] = {1, 1};
   return d->encode(tm, CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, const_cast<void*>(base), dims, strides, box, estr,
                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -295,6 +307,7 @@ struct MatrixCtx {
   int64_t x_rows, x_cols;     // extent (and row pitch) of X
   uint32_t* hist_top;         // the caller's first-pass histogram of G, or null
   uint16_t* W;                // the BF16 parameter that takes Root's update in this call, or null
+  CUtensorMap tm_G;           // the caller's matrix for the operand preparation (tiles of 128 x 128)
 };
 
 fp4_status build_matrix(const DeviceInfo* d, const float* G, float* out, int64_t m, int64_t n, int steps,
@@ -312,6 +325,7 @@ fp4_status build_matrix(const DeviceInfo* d, const float* G, float* out, int64_t
   const int64_t xr = c->pl.tall ? s : c->pl.s0, xc = c->pl.tall ? l : c->pl.l0;
   c->x_rows = xr; c->x_cols = xc;
   c->store_x0 = c->pl.tall || steps == 0;
+  if (!make_f32_tile_map(d, &c->tm_G, G, m, n)) return FP4_ERR_CUDA;
   if (steps == 0) return FP4_OK;
   float abc[3] = {p->a, p->b, p->c};
   if (std::isnan(p->a)) coeffs(m, n, abc);
@@ -321,14 +335,17 @@ fp4_status build_matrix(const DeviceInfo* d, const float* G, float* out, int64_t
              pair3 = pair_kernel(s / 128, l / 128, s, d->sms, fs);
   CUtensorMap tm_qX, tm_qXt[2], tm_qA, tm_qB, tm_A1, tm_A2, tm_X;
   CUtensorMap sf_qX, sf_qXt[2], sf_qA, sf_qB;
-  bool ok = make_sf_map(d, &sf_qX, ws + L.qX_scales, s, l) && make_sf_map(d, &sf_qXt[0], ws + L.qXt_scales[0], l, s) &&
-            make_sf_map(d, &sf_qXt[1], ws + L.qXt_scales[1], l, s) && make_sf_map(d, &sf_qA, ws + L.qA_scales, s, s) &&
-            make_sf_map(d, &sf_qB, ws + L.qB_scales, s, s) &&
-            make_codes_map(d, &tm_qX, ws + L.qX_codes, s, l / 2) &&
-            make_codes_map(d, &tm_qXt[0], ws + L.qXt_codes[0], l, s / 2) &&
-            make_codes_map(d, &tm_qXt[1], ws + L.qXt_codes[1], l, s / 2) &&
-            make_codes_map(d, &tm_qA, ws + L.qA_codes, s, s / 2) &&
-            make_codes_map(d, &tm_qB, ws + L.qB_codes, s, s / 2) &&
+  // every operand is read by exactly one stage: its descriptors take that stage's depth in K
+  const int k1 = pair1 ? gemm_pair_stage_k(kG1) : gemm_stage_k(), k2 = pair2 ? gemm_pair_stage_k(kG2) : gemm_stage_k(),
+            k3 = pair3 ? gemm_pair_stage_k(kG3) : gemm_stage_k();
+  bool ok = make_sf_map(d, &sf_qX, ws + L.qX_scales, s, l, k1) && make_sf_map(d, &sf_qXt[0], ws + L.qXt_scales[0], l, s, k3) &&
+            make_sf_map(d, &sf_qXt[1], ws + L.qXt_scales[1], l, s, k3) && make_sf_map(d, &sf_qA, ws + L.qA_scales, s, s, k2) &&
+            make_sf_map(d, &sf_qB, ws + L.qB_scales, s, s, k3) &&
+            make_codes_map(d, &tm_qX, ws + L.qX_codes, s, l / 2, k1) &&
+            make_codes_map(d, &tm_qXt[0], ws + L.qXt_codes[0], l, s / 2, k3) &&
+            make_codes_map(d, &tm_qXt[1], ws + L.qXt_codes[1], l, s / 2, k3) &&
+            make_codes_map(d, &tm_qA, ws + L.qA_codes, s, s / 2, k2) &&
+            make_codes_map(d, &tm_qB, ws + L.qB_codes, s, s / 2, k3) &&
             make_f32_map(d, &tm_A1, ws + L.A, s, s, pair1 ? 32 : 128) &&
             make_f32_map(d, &tm_A2, ws + L.A, s, s, pair2 ? 32 : 128) &&
             make_f32_map(d, &tm_X, c->X, xr, xc, pair3 ? 32 : 128);
@@ -471,9 +488,9 @@ fp4_status run_group(const DeviceInfo* d, MatrixCtx* mats, int count, int steps,
     for (int i = 0; i < count; ++i) {
       MatrixCtx& c = mats[i];
       items[(size_t)i] = PrologueItem{c.G, c.X, c.ws, &c.pl, clear_first_status && i == 0, c.store_x0, c.x_rows, c.x_cols,
-                                      c.hist_top};
+                                      c.hist_top, &c.tm_G};
     }
-    if (launch_prologue_group(items.data(), count, steps > 0 || keep, quant_opts(p, 0), st) != cudaSuccess)
+    if (launch_prologue_group(items.data(), count, steps > 0 || keep, quant_opts(p, 0), status, st) != cudaSuccess)
       return FP4_ERR_CUDA;
   }
   if (steps > 0) {
@@ -813,9 +830,11 @@ static fp4_status gemm_nt_impl(int dry, const uint8_t* a_codes, const uint8_t* a
   ProblemPack pack;
   memset(&pack, 0, sizeof(pack));
   GemmProblem& pr = pack.p[0];
-  if (!make_codes_map(d, &pr.tmA, a_codes, M, K / 2) || !make_codes_map(d, &pr.tmB, b_codes, N, K / 2) ||
-      !make_f32_map(d, &pr.tmOut, D, M, N, pair_kernel(M / 128, N / 128, K, d->sms) ? 32 : 128) || !make_sf_map(d, &pr.tmSfa, a_scales, M, K) ||
-      !make_sf_map(d, &pr.tmSfb, b_scales, N, K))
+  const bool pair = pair_kernel(M / 128, N / 128, K, d->sms);
+  const int sk = pair ? gemm_pair_stage_k(kPlain) : gemm_stage_k();
+  if (!make_codes_map(d, &pr.tmA, a_codes, M, K / 2, sk) || !make_codes_map(d, &pr.tmB, b_codes, N, K / 2, sk) ||
+      !make_f32_map(d, &pr.tmOut, D, M, N, pair ? 32 : 128) || !make_sf_map(d, &pr.tmSfa, a_scales, M, K, sk) ||
+      !make_sf_map(d, &pr.tmSfb, b_scales, N, K, sk))
     return FP4_ERR_CUDA;
   pr.tmAux = pr.tmOut;
   pr.sfa = a_scales; pr.sfb = b_scales;
