@@ -497,3 +497,65 @@ def test_clip_degenerate_inputs(kind):
     if kind != "zero":
         got2, _ = run_gpu(G, steps=2)
         assert rel(got2, oracle.root_ns(G, steps=2)) <= TOL_OUT
+
+
+def _first_copies_input(kind, m, n):
+    rng = np.random.default_rng(1234)
+    G = rng.standard_normal((m, n)).astype(np.float32)
+    if kind == "dynamic_range":
+        # blocks of 16 along the rows scaled by 2^-k, k up to 40: scale bytes down to the E4M3
+        # subnormals and to zero, next to ordinary blocks
+        k = rng.integers(0, 41, size=(m, n // 16))
+        G = (G * np.repeat(np.exp2(-k), 16, axis=1)).astype(np.float32)
+    elif kind == "column_dynamic_range":
+        k = rng.integers(0, 41, size=(m // 16, n))
+        G = (G * np.repeat(np.exp2(-k), 16, axis=0)).astype(np.float32)
+    elif kind == "tiny":
+        G = (G * np.float32(1e-30)).astype(np.float32)   # X0 = G / (nu + eps) stays tiny: tensor scale near 2^-90
+    elif kind == "heavy_tail":
+        G = (G * np.exp(2.0 * rng.standard_normal((m, n)))).astype(np.float32)
+    return G
+
+
+@pytest.mark.parametrize("kind", ["gaussian", "dynamic_range", "column_dynamic_range", "tiny", "heavy_tail"])
+@pytest.mark.parametrize("shape", [(256, 512), (512, 256), (144, 272), (272, 144), (1024, 2048)])
+def test_first_operand_copies_are_the_oracle_quantisation_of_x0(kind, shape):
+    """The prologue alone (no iteration): X0 and both NVFP4 copies of it.  The copies must be, bit for bit,
+    what the oracle's quantiser makes of the X0 the call returned - including blocks whose scale is an E4M3
+    subnormal or zero, blocks with clipped elements, and a tensor scale far from 1."""
+    m, n = shape
+    G = _first_copies_input(kind, m, n)
+    flags = FP4_FLAG_KEEP_OPERANDS
+    got, ws = run_gpu(G, steps=0, flags=flags)
+    lay, sc, f32, q, s, l = ws_view(ws, m, n, 0, flags)
+    s_pad, l_pad = -(-s // 128) * 128, -(-l // 128) * 128
+    X0 = np.zeros((s_pad, l_pad), dtype=np.float32)
+    X0[:s, :l] = got if m <= n else got.T
+    sg = float(sc[lay.idx_sg_X0])
+    assert sg == np.float32(np.abs(X0).max() / np.float32(2688.0)) or np.abs(X0).max() == 0
+    oc, os_, _ = oracle.quantize(X0, s_g=sg)
+    codes, sf = q(lay.qX_codes, lay.qX_scales, s_pad, l_pad)
+    assert np.array_equal(sf, os_), mismatch(sf, os_)
+    assert np.array_equal(codes, oc), mismatch(codes, oc)
+    row_scales = os_
+    oc, os_, _ = oracle.quantize(np.ascontiguousarray(X0.T), s_g=sg)
+    codes, sf = q(lay.qXt_codes[0], lay.qXt_scales[0], l_pad, s_pad)
+    assert np.array_equal(sf, os_), mismatch(sf, os_)
+    assert np.array_equal(codes, oc), mismatch(codes, oc)
+    if kind in ("dynamic_range", "column_dynamic_range"):
+        # the scaled blocks run along the rows of G: the copy that keeps them intact has the small scales
+        along_rows = (kind == "dynamic_range") == (m <= n)
+        small = row_scales if along_rows else os_
+        assert ((small > 0) & (small <= 8)).any() and (small == 0).any(), "the case is meant to reach small scale bytes"
+
+
+def mismatch(a, b):
+    bad = np.argwhere(a != b)
+    return "%d of %d differ, first at %s: %s vs %s" % (len(bad), a.size, bad[0], a[tuple(bad[0])], b[tuple(bad[0])])
+
+
+@pytest.mark.parametrize("kind", ["gaussian", "heavy_tail"])
+def test_first_operand_copies_two_million_blocks(kind):
+    """The same on 4096 x 4096: with 2 x 10^6 blocks some scale quotients fall within two ulps of an E4M3
+    rounding boundary, the case the preparation kernel hands to its exact path."""
+    test_first_operand_copies_are_the_oracle_quantisation_of_x0(kind, (4096, 4096))
