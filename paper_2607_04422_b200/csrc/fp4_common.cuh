@@ -287,6 +287,14 @@ __device__ __forceinline__ void report_timeout(uint32_t* status) {
 // ----------------------------------------------------------------------------------
 // PTX wrappers
 // ----------------------------------------------------------------------------------
+// Programmatic dependent launch.  Every kernel of a Newton-Schulz call lets the next launch of the stream
+// start early (its blocks become resident as soon as this grid's blocks have all started and resources are
+// free) and itself waits, after its set-up and before it touches global memory, until the launch before it
+// has completed and its writes are visible.  Every kernel waits unconditionally, so completion stays
+// transitive along the stream.  Both are no-ops for a kernel launched without the attribute.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return (uint32_t)__cvta_generic_to_shared(p);
 }

@@ -121,6 +121,7 @@ k_gemm(const __grid_constant__ ProblemPack pack, const __grid_constant__ GemmLau
   constexpr bool STORE_F32 = (MODE == kPlain || MODE == kG1 || MODE == kG3);
   const bool do_q = (MODE != kPlain) && args.write_q;
 
+  pdl_launch_dependents();
   if (threadIdx.x == 0) {
     for (int i = 0; i < STAGES; ++i) { mbar_init(&bars->full[i], 1); mbar_init(&bars->empty[i], 1); }
     for (int i = 0; i < NACC; ++i) { mbar_init(&bars->acc_full[i], 1); mbar_init(&bars->acc_empty[i], 8); }
@@ -140,6 +141,7 @@ k_gemm(const __grid_constant__ ProblemPack pack, const __grid_constant__ GemmLau
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = bars->tmem_base;
+  pdl_wait();   // set-up done; from here on the kernel reads what the launches before it wrote
 
   if (warp == 0) {
     // ------------------------------------------------------------ operand producer
@@ -486,7 +488,7 @@ cudaError_t launch_mode(const ProblemPack& pack, const GemmLaunch& L, int sms, c
   int grid = sms;
   if (grid > num_tiles) grid = num_tiles;
   count_launches(1);
-  k_gemm<MODE, PF><<<grid, NTHREADS, SMEM_BYTES, st>>>(pack, L);
+  launch_chained(k_gemm<MODE, PF>, dim3(grid), dim3(NTHREADS), SMEM_BYTES, st, pack, L);
   return cudaGetLastError();
 }
 

@@ -317,6 +317,7 @@ k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ Ge
   // instruction stream, same epilogue.
   const bool dry = (MODE == kPlain) && args.dry_operands != 0;
 
+  pdl_launch_dependents();
   if (threadIdx.x == 0) {
     for (int i = 0; i < STAGES; ++i) { mbar_init(&bars->full[i], 1); mbar_init(&bars->empty[i], 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(&bars->acc_full[i], 1); mbar_init(&bars->acc_empty[i], 2 * EPI_WARPS); }
@@ -335,6 +336,7 @@ k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ Ge
   cluster_sync_all();  // the peer's barriers are initialised before anything signals them
   tc_fence_after();
   const uint32_t tmem_base = bars->tmem_base;
+  pdl_wait();          // set-up done; from here on the kernel reads what the launches before it wrote
 
   if (warp == 0) {
     // ------------------------------------------------------------ operand producer (both CTAs)
@@ -867,7 +869,7 @@ cudaError_t launch_pair_mode(const ProblemPack& pack, const GemmLaunch& L, int s
   int pairs = sms / 2;
   if (pairs > num_tiles) pairs = num_tiles;
   count_launches(1);
-  k_gemm_pair<MODE, PF, BH, UPD><<<2 * pairs, NTHREADS, Lay<MODE>::SMEM_BYTES, st>>>(pack, L);
+  launch_chained(k_gemm_pair<MODE, PF, BH, UPD>, dim3(2 * pairs), dim3(NTHREADS), Lay<MODE>::SMEM_BYTES, st, pack, L);
   return cudaGetLastError();
 }
 

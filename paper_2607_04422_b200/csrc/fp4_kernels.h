@@ -1,6 +1,8 @@
 // Internal interfaces between the translation units of the library.
 #pragma once
 
+#include <utility>
+
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -120,6 +122,23 @@ struct GemmLaunch {
 // Measurement support: counts kernel launches and, when profiling is on, brackets a group of
 // launches with events.
 void count_launches(int n);
+
+// Launch of a kernel of the Newton-Schulz chain: with the programmatic-stream-serialisation attribute (the
+// kernel's blocks may become resident before the previous launch has completed; the kernel itself waits,
+// see pdl_wait) for the groups of a call that are bound by launch latency (pdl_select, called per group),
+// unless the environment variable FP4ROOT_NO_PDL is set.
+bool pdl_enabled();
+void pdl_select(int64_t group_elements);
+template <typename... KArgs, typename... Args>
+cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = pdl_enabled() ? 1 : 0;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
 
 // First-moment momentum state (fp4_momentum.cu): one step in place on codes/scales; M_out and
 // hist may be null.

@@ -69,6 +69,8 @@ __device__ __forceinline__ uint32_t mag_bits(float x) { return __float_as_uint(x
 // ---- init: clear header (keeping the status word of all but the first matrix of a call),
 // scalars and histogram; arm the select
 __global__ void __launch_bounds__(256) kp_init(const __grid_constant__ PrepGroup g) {
+  pdl_launch_dependents();
+  pdl_wait();
   const PrepMatrix& m = g.mat[blockIdx.y];
   uint32_t* w = reinterpret_cast<uint32_t*>(m.hdr);
   const int first = m.clear_status ? 0 : 4;
@@ -84,6 +86,8 @@ constexpr int kTopBins = 1 << kTopBits;      // 8192
 
 // ---- pass 1: histogram of the top 13 magnitude bits
 __global__ void __launch_bounds__(512) kp_hist_top(const __grid_constant__ PrepGroup g) {
+  pdl_launch_dependents();
+  pdl_wait();
   __shared__ uint32_t sh[kTopBins];
   const PrepMatrix& m = g.mat[blockIdx.y];
   if (m.hist_top) return;  // the caller counted this matrix already
@@ -153,6 +157,8 @@ __device__ __forceinline__ void pick_bin(NsHeader* hdr, uint32_t* hist, int shif
 }
 
 __global__ void __launch_bounds__(256) kp_pick_top(const __grid_constant__ PrepGroup g) {
+  pdl_launch_dependents();
+  pdl_wait();
   const PrepMatrix& m = g.mat[blockIdx.y];
   pick_bin<kTopBins>(m.hdr, m.hist_top ? m.hist_top : m.hist, kTopShift, &m.hdr->bin_count, &m.hdr->count_below);
 }
@@ -161,6 +167,8 @@ __global__ void __launch_bounds__(256) kp_pick_top(const __grid_constant__ PrepG
 // Candidates are rare: they are collected in a shared-memory buffer per block and copied to
 // the global list with one reservation per block (or directly when the buffer is full).
 __global__ void __launch_bounds__(256) kp_compact_stats(const __grid_constant__ PrepGroup g) {
+  pdl_launch_dependents();
+  pdl_wait();
   constexpr uint32_t kBuf = 2048;
   __shared__ uint32_t s_buf[kBuf];
   __shared__ uint32_t s_cnt, s_base;
@@ -305,6 +313,8 @@ __device__ void fallback_select_and_stats(const PrepGroup& g, const PrepMatrix& 
 
 // ---- finish: select tau among the candidates and derive the normalisation scalars
 __global__ void __launch_bounds__(1024) kp_finalize(const __grid_constant__ PrepGroup g) {
+  pdl_launch_dependents();
+  pdl_wait();
   const PrepMatrix& m = g.mat[blockIdx.y];
   __shared__ double shd[1024];
   __shared__ uint32_t hist[1024];
@@ -621,6 +631,7 @@ __global__ void __launch_bounds__(kPrepThreads, 1) kp_prep_operands(const __grid
   const int tiles_per_matrix = (int)((g.s >> 7) * (g.l >> 7));
   const int total = tiles_per_matrix * g.count;
   const int my_tiles = (total - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;  // tiles of this block
+  pdl_launch_dependents();
 
   // Tile `it` of this block: work out where it lies, publish that in the ring and start its copy.  Called by
   // one thread, a block-wide barrier before the tile's turn.
@@ -647,6 +658,9 @@ __global__ void __launch_bounds__(kPrepThreads, 1) kp_prep_operands(const __grid
     for (int i = 0; i < kPrepBufs; ++i) mbar_init(&sh->full[i], 1);
     sh->abort_flag = 0;
     mbar_fence_init();
+  }
+  pdl_wait();   // from here on the kernel reads what the launches before it wrote
+  if (threadIdx.x == 0) {
     for (int i = 0; i < kPrepBufs; ++i) fetch(i);
   }
   if (threadIdx.x < g.count * 8) {
@@ -909,26 +923,26 @@ cudaError_t launch_prologue_group(const PrologueItem* items, int count, int writ
     const dim3 gy1(1, (unsigned)nn), gh((unsigned)hist_blocks, (unsigned)nn), gs((unsigned)g.stat_blocks, (unsigned)nn);
     {
       ProfScope ps(FP4_PROF_CLIP, st);
-      kp_init<<<dim3(4, (unsigned)nn), 256, 0, st>>>(g);
+      launch_chained(kp_init, dim3(4, (unsigned)nn), dim3(256), 0, st, g);
       count_launches(1);
       if (g.clip) {
-        if (!all_counted) kp_hist_top<<<gh, 512, 0, st>>>(g);
-        kp_pick_top<<<gy1, 256, 0, st>>>(g);
+        if (!all_counted) launch_chained(kp_hist_top, gh, dim3(512), 0, st, g);
+        launch_chained(kp_pick_top, gy1, dim3(256), 0, st, g);
         count_launches(all_counted ? 1 : 2);
       }
     }
     {
       ProfScope ps(FP4_PROF_STATS, st);
-      kp_compact_stats<<<gs, 256, 0, st>>>(g);
-      kp_finalize<<<gy1, 1024, 0, st>>>(g);
+      launch_chained(kp_compact_stats, gs, dim3(256), 0, st, g);
+      launch_chained(kp_finalize, gy1, dim3(1024), 0, st, g);
       count_launches(2);
     }
     {
       ProfScope ps(FP4_PROF_PREP, st);
       const int64_t tiles = (pl.l / 128) * (pl.s / 128) * nn;
       const unsigned gp = (unsigned)(tiles < sms ? tiles : sms);
-      if (q.rht || q.four_six) kp_prep_operands<true><<<gp, kPrepThreads, kPrepSmem, st>>>(g);
-      else kp_prep_operands<false><<<gp, kPrepThreads, kPrepSmem, st>>>(g);
+      if (q.rht || q.four_six) launch_chained(kp_prep_operands<true>, dim3(gp), dim3(kPrepThreads), kPrepSmem, st, g);
+      else launch_chained(kp_prep_operands<false>, dim3(gp), dim3(kPrepThreads), kPrepSmem, st, g);
       count_launches(1);
     }
     cudaError_t e = cudaGetLastError();

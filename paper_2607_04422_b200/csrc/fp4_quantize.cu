@@ -103,6 +103,8 @@ __global__ void __launch_bounds__(256) k_quantize_rows_opts(const float* __restr
 __global__ void __launch_bounds__(256) k_transpose_out(const float* __restrict__ X, int64_t l, float* __restrict__ out,
                                                        int64_t s0, int64_t l0, const ParamUpdate upd) {
   __shared__ float t[64][65];
+  pdl_launch_dependents();
+  pdl_wait();
   const int64_t r0 = (int64_t)blockIdx.y * 64, c0 = (int64_t)blockIdx.x * 64;  // tile origin in X
   const int q = threadIdx.x & 15, row = threadIdx.x >> 4;                      // 16 pieces per row, 16 rows per sweep
 #pragma unroll
@@ -135,6 +137,8 @@ __global__ void __launch_bounds__(256) k_transpose_out(const float* __restrict__
 
 // W <- update(W, O) elementwise, 8 elements per thread
 __global__ void __launch_bounds__(256) k_param_update(const float* __restrict__ O, int64_t n8, const ParamUpdate upd) {
+  pdl_launch_dependents();
+  pdl_wait();
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n8; i += (int64_t)gridDim.x * blockDim.x) {
     const float4 a = __ldg(reinterpret_cast<const float4*>(O) + 2 * i), b = __ldg(reinterpret_cast<const float4*>(O) + 2 * i + 1);
     uint4* wp = reinterpret_cast<uint4*>(upd.W) + i;
@@ -183,7 +187,7 @@ cudaError_t launch_transpose_out(const float* X, int64_t s, int64_t l, float* ou
   dim3 grid((unsigned)((l0 + 63) / 64), (unsigned)((s0 + 63) / 64));
   (void)s;
   count_launches(1);
-  k_transpose_out<<<grid, 256, 0, st>>>(X, l, out, s0, l0, upd);
+  launch_chained(k_transpose_out, grid, dim3(256), 0, st, X, l, out, s0, l0, upd);
   return cudaGetLastError();
 }
 
@@ -191,7 +195,7 @@ cudaError_t launch_transpose_out(const float* X, int64_t s, int64_t l, float* ou
 cudaError_t launch_param_update(const float* O, int64_t n, const ParamUpdate& upd, int sms, cudaStream_t st) {
   if (!upd.W) return cudaSuccess;
   count_launches(1);
-  k_param_update<<<grid_for(n / 8, 256, sms), 256, 0, st>>>(O, n / 8, upd);
+  launch_chained(k_param_update, dim3(grid_for(n / 8, 256, sms)), dim3(256), 0, st, O, n / 8, upd);
   return cudaGetLastError();
 }
 
