@@ -478,6 +478,10 @@ k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ Ge
     const uint32_t acc_empty_leader0 = map_to_cta(&bars->acc_empty[0], 0);
     const uint32_t acc_empty_leader1 = map_to_cta(&bars->acc_empty[1], 0);
     const uint32_t ov_free_leader = map_to_cta(&bars->ov_free, 0);
+    // A tall input is worked on as its transpose.  With FP32 storage the first G3 stage reads the caller's
+    // matrix through a transposing box and the last one writes the caller's result the same way, so neither
+    // an FP32 copy of X0 nor a final transpose pass is needed (per-problem flags aux_tr / out_tr).
+    constexpr bool TR = (MODE == kG3) && !BH;
     const bool auxh = BH && HAS_AUX && args.aux_h != 0;                               // the combined tile is BF16
     const bool hout = BH && STORE_F32 && MODE != kPlain && args.out_h == 1;           // the result is stored as BF16
 
@@ -487,7 +491,7 @@ k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ Ge
     bool scale_pow2 = false;
     uint64_t scale2 = 0, ca2 = 0, cb2 = 0, ccs2 = 0;
     float tau = 0.0f, inv = 0.0f;  // first G3 stage on the raw input: X0 = clamp(G, tau) * inv
-    bool raw = false;
+    bool raw = false, aux_tr = false, out_tr = false;
     const GemmProblem* pr = nullptr;
     int cur_p = -1;
     float amax = 0.0f;
@@ -503,6 +507,11 @@ k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ Ge
         } else if (auxh) {
           mbar_expect_tx_s(bar, XBUF_BYTES / 2);
           tma_load_2d_s(area + b * XBUF_BYTES, &q->tmH, x64 + e * CHUNK, y32, bar);
+        } else if (TR && q->aux_tr) {
+          // the tile comes from a matrix stored the other way round (a tall input): the same 2 KB arrive as
+          // 16 rows (columns of the tile) of 32 elements (its rows)
+          mbar_expect_tx_s(bar, XBUF_BYTES);
+          tma_load_2d_s(area + b * XBUF_BYTES, &q->tmAux, y32, x64 + e * CHUNK, bar);
         } else {
           mbar_expect_tx_s(bar, XBUF_BYTES);
           tma_load_2d_s(area + b * XBUF_BYTES, &q->tmAux, x64 + e * CHUNK, y32, bar);
@@ -566,6 +575,8 @@ k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ Ge
         const float ccs = __fmul_rn(cc, scale);
         ccs2 = pack2(ccs, ccs);
         raw = (MODE == kG3) && pr->aux_raw != 0;
+        aux_tr = TR && pr->aux_tr != 0;
+        out_tr = TR && pr->out_tr != 0;
         if (raw) {
           tau = args.clip ? pr->scalars[args.ix.tau] : __int_as_float(0x7f800000);
           inv = pr->scalars[args.ix.inv];
@@ -667,9 +678,16 @@ k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ Ge
           __syncwarp();  // every lane has its row before FP32 rows are staged over them
         } else if (HAS_AUX) {
           float x[16];
+          if (TR && aux_tr) {
+            // the block lies transposed in the buffer: element (row = lane, column j) at j * 128 + lane * 4
 #pragma unroll
-          for (int j = 0; j < 4; ++j)
-            lds128((row_addr + boff) ^ (j << 4), x[4 * j], x[4 * j + 1], x[4 * j + 2], x[4 * j + 3]);
+            for (int j = 0; j < 16; ++j) x[j] = lds32(area + boff + j * 128 + lane * 4);
+            __syncwarp();  // every lane has its row before the result rows are staged over the block
+          } else {
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+              lds128((row_addr + boff) ^ (j << 4), x[4 * j], x[4 * j + 1], x[4 * j + 2], x[4 * j + 3]);
+          }
           TR_BEGIN
           tc_wait_ld16(acc);
           TR_END(2)
@@ -748,7 +766,12 @@ k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ Ge
         }
         // ---- stage the block (for the TMA store and / or the column pass) and send it off
         const bool send = rows_in && xcol < pr->out_cols;
-        if (stage) {
+        if (TR && out_tr) {
+          // the caller's matrix is the transpose: the block leaves as 16 rows of 32 elements
+#pragma unroll
+          for (int j = 0; j < 16; ++j) sts32(area + boff + j * 128 + lane * 4, __float_as_uint(v[j]));
+          fence_proxy_async_smem();
+        } else if (stage) {
 #pragma unroll
           for (int j = 0; j < 4; ++j)
             sts128((row_addr + boff) ^ (j << 4), v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
@@ -756,7 +779,8 @@ k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ Ge
         }
         __syncwarp();
         if (store_out && !hout && send && lane == 0) {
-          tma_store_2d_s(&pr->tmOut, xcol, y32, area + boff);
+          if (TR && out_tr) tma_store_2d_s(&pr->tmOut, y32, xcol, area + boff);
+          else tma_store_2d_s(&pr->tmOut, xcol, y32, area + boff);
           bulk_commit();
         }
         // ---- blocks of 16 down the rows of this warp's own 32 x 16 block (the transposed operand

@@ -82,6 +82,8 @@ struct alignas(64) GemmProblem {
   float ca, cb, cc;          // coefficients
   float sg_a, sg_b;          // kPlain: tensor scales from the host
   int aux_raw;               // kG3: tmAux maps the raw input G; X0 = clamp(G, tau) * inv is formed on the fly
+  int aux_tr;                // kG3, CTA-pair kernel: tmAux maps a matrix stored as the transpose of the tile grid (box = 32 x 16)
+  int out_tr;                // kG3, CTA-pair kernel: so does tmOut (the caller's result of a tall input)
   int out_rows, out_cols;    // extent of the matrix behind tmOut (chunks that start outside it are not stored)
   void* out_direct;          // out_h == 2: the FP32 tensor the epilogue warps store the rounded result to
   int64_t out_direct_ld;     //   (row-major, leading dimension in elements)

@@ -136,6 +136,18 @@ bool make_f32_tile_map(const DeviceInfo* d, CUtensorMap* tm, const void* base, i
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// 2-D map over a row-major FP32 matrix whose transpose the CTA-pair kernel works on: box = 32 columns x 16 rows
+// (one epilogue warp's 32 x 16 block, transposed), no swizzle.
+bool make_f32_tr_map(const DeviceInfo* d, CUtensorMap* tm, const void* base, int64_t rows, int64_t cols) {
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)cols * 4};
+  cuuint32_t box[2] = {32, 16};
+  cuuint32_t estr[2] = {1, 1};
+  return d->encode(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // 2-D map over a row-major BF16 matrix: box = 16 columns x 32 rows (32-byte rows), no swizzle: the block of
 // one epilogue warp of the CTA-pair kernel.
 bool make_bf16_map(const DeviceInfo* d, CUtensorMap* tm, const void* base, int64_t rows, int64_t cols) {
@@ -321,6 +333,10 @@ struct MatrixCtx {
   uint32_t* hist_top;         // the caller's first-pass histogram of G, or null
   uint16_t* W;                // the BF16 parameter that takes Root's update in this call, or null
   CUtensorMap tm_G;           // the caller's matrix for the operand preparation (tiles of 128 x 128)
+  // A tall input with FP32 storage in the CTA-pair kernel: the first G3 stage reads the caller's matrix and
+  // the last one writes the caller's result through transposing boxes.
+  bool native_tall;
+  CUtensorMap tm_outT;
 };
 
 fp4_status build_matrix(const DeviceInfo* d, const float* G, float* out, int64_t m, int64_t n, int steps,
@@ -338,6 +354,7 @@ fp4_status build_matrix(const DeviceInfo* d, const float* G, float* out, int64_t
   const int64_t xr = c->pl.tall ? s : c->pl.s0, xc = c->pl.tall ? l : c->pl.l0;
   c->x_rows = xr; c->x_cols = xc;
   c->store_x0 = c->pl.tall || steps == 0;
+  c->native_tall = false;
   if (!make_f32_tile_map(d, &c->tm_G, G, m, n)) return FP4_ERR_CUDA;
   if (steps == 0) return FP4_OK;
   float abc[3] = {p->a, p->b, p->c};
@@ -414,7 +431,17 @@ fp4_status build_matrix(const DeviceInfo* d, const float* G, float* out, int64_t
     g.tmRq = st_qX_r; g.tmCq = st_qXt_c[cur ^ 1];
   }
   c->g3_first = c->g3[0];
-  if (!c->store_x0) {
+  c->native_tall = c->pl.tall && pair3 && bmode == 0;
+  if (c->native_tall) {
+    // the caller's matrices are l0 x s0
+    CUtensorMap tm_Gt;
+    if (!make_f32_tr_map(d, &tm_Gt, G, c->pl.l0, c->pl.s0) || !make_f32_tr_map(d, &c->tm_outT, out, c->pl.l0, c->pl.s0))
+      return FP4_ERR_CUDA;
+    c->store_x0 = false;
+    c->g3_first.tmAux = tm_Gt;
+    c->g3_first.aux_raw = 1;
+    c->g3_first.aux_tr = 1;
+  } else if (!c->store_x0) {
     CUtensorMap tm_G;
     if (!make_f32_map(d, &tm_G, G, c->pl.s0, c->pl.l0, pair3 ? 32 : 128)) return FP4_ERR_CUDA;
     c->g3_first.tmAux = tm_G;
@@ -494,6 +521,12 @@ fp4_status run_group(const DeviceInfo* d, MatrixCtx* mats, int count, int steps,
   bool any_update = false;
   for (int i = 0; i < count; ++i) any_update = any_update || mats[i].W != nullptr;
   std::vector<char> fused_update((size_t)count, 0);
+  // a tall input's result leaves the last G3 stage transposed (no transpose pass) unless that stage also has to
+  // write operand copies, or the call updates parameters (the update of a tall matrix rides on the transpose)
+  std::vector<char> direct_out((size_t)count, 0);
+  bool any_direct = false;
+  for (int i = 0; i < count; ++i)
+    if (steps > 0 && mats[i].native_tall && !keep && !any_update) { direct_out[(size_t)i] = 1; any_direct = true; }
   const NsPlan& pl0 = mats[0].pl;
   const int64_t s = pl0.s, l = pl0.l;
   pdl_select(s * l * count);
@@ -572,9 +605,23 @@ fp4_status run_group(const DeviceInfo* d, MatrixCtx* mats, int count, int steps,
         L3.upd_decay = upd.decay; L3.upd_step = upd.step;
         L3.no_out = upd.no_out;
       }
+      const ProblemPack* pk = &packs[k == 0 ? 4 : 2 + cur];
+      ProblemPack last_pack;
+      if (last && any_direct) {
+        // tall inputs whose result goes straight to the caller's matrix, transposed on the way out
+        last_pack = *pk;
+        for (int j = 0; j < count; ++j)
+          if (direct_out[(size_t)j]) {
+            GemmProblem& g = last_pack.p[j];
+            g.tmOut = mats[j].tm_outT;
+            g.out_tr = 1;
+            g.out_rows = (int)pl0.s0; g.out_cols = (int)pl0.l0;
+          }
+        pk = &last_pack;
+      }
       {
         ProfScope ps(FP4_PROF_G3, st);
-        if (launch_gemm_auto(kG3, packs[k == 0 ? 4 : 2 + cur], L3, d->sms, st, fs) != cudaSuccess)
+        if (launch_gemm_auto(kG3, *pk, L3, d->sms, st, fs) != cudaSuccess)
           return FP4_ERR_CUDA;
       }
     }
@@ -582,6 +629,7 @@ fp4_status run_group(const DeviceInfo* d, MatrixCtx* mats, int count, int steps,
   for (int i = 0; i < count; ++i) {
     ParamUpdate u = upd;
     u.W = mats[i].W;
+    if (direct_out[(size_t)i]) continue;
     if (mats[i].pl.tall) {
       ProfScope ps(FP4_PROF_TRANSPOSE, st);
       if (launch_transpose_out(mats[i].X, s, l, mats[i].out, pl0.s0, pl0.l0, u, st) != cudaSuccess) return FP4_ERR_CUDA;

@@ -209,7 +209,8 @@ def test_batched_mixed_orientations_in_one_group_paper_options():
         assert rel(single, oracle.root_ns(g, steps=3, rht=True, four_six=True, seed=77)) <= TOL_OUT
 
 
-@pytest.mark.parametrize("shape", [(144, 272), (272, 144), (208, 208), (16, 64), (400, 1040), (1040, 400)])
+@pytest.mark.parametrize("shape", [(144, 272), (272, 144), (208, 208), (16, 64), (400, 1040), (1040, 400),
+                                   (496, 1008), (1008, 496)])   # the last two pad to 512 x 1024: CTA-pair kernel
 def test_shapes_that_are_not_multiples_of_128(shape):
     """Dimensions that are multiples of the block length 16 are zero-padded to the tile size
     inside the library; the oracle works on the matrix as it is.  Padding must be invisible:
