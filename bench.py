@@ -594,6 +594,19 @@ def run_ours(args):
                                 f"reach under the power cap; the same product with operand traffic: {ceil['streamed']:.0f} TFLOP/s",
                 "time_share": shares}
 
+    # the three passes of the prologue over the input (HBM-bound): bytes each moves per element of G
+    n_elem = float(sum(m * n for m, n in shapes))
+    pass_bytes = {"clip": 4.0, "stats": 4.0, "prep": 4.0 + 2 * 0.5625}
+    prologue = {"what": "clip: histogram of the top magnitude bits + bin pick; stats: candidates of the clip bin and "
+                        "sum of squares + select; prep: clamp, scale and both NVFP4 copies of X0 (no FP32 copy: "
+                        "the first G3 stage reads the input itself, transposed for tall matrices)",
+                "ms_per_step": sum(prof[k][0] for k in pass_bytes) / prof_steps, "passes": {}}
+    for k, bpe in pass_bytes.items():
+        ms_k = prof[k][0] / prof_steps
+        gbs_k = n_elem * bpe / (ms_k / 1e3) / 1e9 if ms_k > 0 else 0.0
+        prologue["passes"][k] = {"ms_per_step": ms_k, "bytes_per_element": bpe, "gbs": gbs_k,
+                                 "frac_of_measured_hbm": gbs_k / pk["hbm_gbs"]}
+
     cpu = cpu_baseline_leg(mats_np, shapes)
     cpu["configs_measured_in_full"] = small_config_rows(args.full_cpu)
     step_s = ms_per_step / 1e3
@@ -653,6 +666,7 @@ def run_ours(args):
                              "what": "the same step with FP4_FLAG_RHT | FP4_FLAG_FOUR_SIX (paper-faithful "
                                      "quantiser options); the headline value uses the base quantiser"},
             "paper_context": "paper: Root step 2.50x / 2.83x faster than optimised BF16 on one RTX 5090 (d=4096/6144)",
+            "prologue": prologue,
             "gpu_launches": int(launches), "clocks": clocks, "roofline": roofline, "cpu_baseline": cpu}
     print(json.dumps(line), flush=True)
     if world > 1:
