@@ -166,6 +166,12 @@ fp4_status fp4_root_coeffs(int64_t m, int64_t n, int steps, float abc[3]);
  *   an NVFP4 quantisation with 16-element blocks along the contraction axis; the
  *   result is X_steps (transposed back when m > n).
  * Two calls that share a workspace must not overlap in time.
+ * Launches: 6 kernels for clip, normalisation and the first quantisation plus 3 per iteration
+ *   (and a transpose pass for a tall matrix on the routes that cannot write the result
+ *   transposed from the last product).  Calls on small matrices (up to 8 M elements per group
+ *   of equal shapes) chain their kernels with programmatic dependent launch; the environment
+ *   variable FP4ROOT_NO_PDL (any value) switches that off.  Kernels launched before or after
+ *   the call on the same stream see ordinary stream order either way.
  */
 size_t fp4_root_ns_workspace_bytes(int64_t m, int64_t n, int steps, uint32_t flags);
 fp4_status fp4_root_ns(const float* G, float* out, int64_t m, int64_t n, int steps,
