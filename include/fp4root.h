@@ -185,6 +185,11 @@ fp4_status fp4_root_ns(const float* G, float* out, int64_t m, int64_t n, int ste
  * Matrices of equal shape (after orientation) are grouped: each Newton-Schulz stage of a
  * group is one launch whose tile list spans all its matrices.  Results are bit-identical to
  * calling fp4_root_ns on each matrix.
+ * Streams: with two or more groups the call also uses a second stream of its own (one per host
+ *   thread and device, created on first use), which waits for everything enqueued on `stream`
+ *   before the call and which `stream` waits for before the call returns, so callers see
+ *   ordinary stream order; the pattern can be captured in a CUDA graph.  The environment
+ *   variable FP4ROOT_NO_OVERLAP (any value) keeps all launches on `stream`.
  */
 size_t fp4_root_ns_batched_workspace_bytes(int count, const int64_t* m, const int64_t* n,
                                            int steps, uint32_t flags);

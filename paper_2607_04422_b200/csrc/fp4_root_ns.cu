@@ -799,6 +799,34 @@ fp4_status fp4_root_ns(const float* G, float* out, int64_t m, int64_t n, int ste
   return run_one(d, G, out, m, n, steps, p, static_cast<uint8_t*>(ws), true, stream);
 }
 
+// The second stream of a batched call, one per host thread and device, created on first use (never inside
+// fp4_root_ns or fp4_root_ns_static).  FP4ROOT_NO_OVERLAP in the environment keeps everything on the
+// caller's stream.
+struct SideStream {
+  int dev = -1;
+  cudaStream_t stream = nullptr;
+  cudaEvent_t fork = nullptr, join = nullptr;
+};
+SideStream* side_stream(int dev) {
+  static const bool allowed = getenv("FP4ROOT_NO_OVERLAP") == nullptr;
+  if (!allowed) return nullptr;
+  thread_local SideStream t;
+  if (t.stream && t.dev == dev) return &t;
+  if (t.stream) {   // the thread moved to another device
+    cudaEventDestroy(t.fork); cudaEventDestroy(t.join); cudaStreamDestroy(t.stream);
+    t = SideStream();
+  }
+  if (cudaStreamCreateWithFlags(&t.stream, cudaStreamNonBlocking) != cudaSuccess) { t = SideStream(); return nullptr; }
+  if (cudaEventCreateWithFlags(&t.fork, cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&t.join, cudaEventDisableTiming) != cudaSuccess) {
+    cudaStreamDestroy(t.stream);
+    t = SideStream();
+    return nullptr;
+  }
+  t.dev = dev;
+  return &t;
+}
+
 // Batched workspace: one workspace per matrix (the stages of equal-shape matrices run in
 // lockstep, so none can be shared).
 size_t fp4_root_ns_batched_workspace_bytes(int count, const int64_t* m, const int64_t* n, int steps,
@@ -851,11 +879,11 @@ fp4_status fp4_root_ns_batched(int count, const float* const* G, float* const* o
   // exceeds max_group matrices, which bounds the working set competing for L2.
   const int cap = p->max_group > 0 && (int)p->max_group < kPackMax ? (int)p->max_group : kDefaultMaxGroup;
   std::vector<char> done((size_t)count, 0);
-  std::vector<MatrixCtx> group;
-  bool first = true;
+  std::vector<std::vector<MatrixCtx>> groups;
   for (int i = 0; i < count; ++i) {
     if (done[(size_t)i]) continue;
-    group.clear();
+    groups.emplace_back();
+    std::vector<MatrixCtx>& group = groups.back();
     for (int j = i; j < count && (int)group.size() < cap; ++j) {
       if (done[(size_t)j]) continue;
       if (ctx[(size_t)j].pl.s0 == ctx[(size_t)i].pl.s0 && ctx[(size_t)j].pl.l0 == ctx[(size_t)i].pl.l0) {
@@ -863,11 +891,30 @@ fp4_status fp4_root_ns_batched(int count, const float* const* G, float* const* o
         done[(size_t)j] = 1;
       }
     }
-    rc = run_group(d, group.data(), (int)group.size(), steps, p, status, first, stream);
-    if (rc != FP4_OK) return rc;
-    first = false;
   }
-  return FP4_OK;
+  // Groups do not depend on one another.  With two or more, they alternate between the caller's stream
+  // and a second one that forks from it and joins it again before the call returns: every launch is a
+  // persistent grid that ends in a partial wave of tiles, and the next launch of the same group cannot
+  // start before it has drained - a launch of the other group can.
+  // (not while stage times are being collected: the event pairs of the two streams would overlap)
+  SideStream* side = groups.size() >= 2 && g_prof_on.load() == 0 ? side_stream((int)(d - g_dev)) : nullptr;
+  if (side) {
+    // the status word is cleared once, before the fork (a group's own clearing kernel could wipe what
+    // a kernel of the other group has just reported)
+    if (cudaMemsetAsync(status, 0, 4, stream) != cudaSuccess || cudaEventRecord(side->fork, stream) != cudaSuccess ||
+        cudaStreamWaitEvent(side->stream, side->fork, 0) != cudaSuccess)
+      return FP4_ERR_CUDA;
+  }
+  for (size_t gi = 0; gi < groups.size(); ++gi) {
+    cudaStream_t st = (side && (gi & 1)) ? side->stream : stream;
+    rc = run_group(d, groups[gi].data(), (int)groups[gi].size(), steps, p, status, !side && gi == 0, st);
+    if (rc != FP4_OK) break;
+  }
+  if (side) {
+    if (cudaEventRecord(side->join, side->stream) != cudaSuccess || cudaStreamWaitEvent(stream, side->join, 0) != cudaSuccess)
+      return FP4_ERR_CUDA;
+  }
+  return rc;
 }
 
 fp4_status fp4_last_device_status(const void* ws, cudaStream_t stream) {

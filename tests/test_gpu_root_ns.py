@@ -293,6 +293,38 @@ def test_cuda_graph_replay_matches_direct_call():
         assert torch.equal(out, direct)
 
 
+def test_cuda_graph_replay_of_a_batched_call_with_several_groups():
+    """A batched call with more than one group of shapes forks to a second stream and joins again:
+    captured as a whole, the replay gives the bytes of the direct call."""
+    shapes = [(256, 512), (512, 256), (512, 512), (256, 512), (768, 256), (512, 512)]
+    Gs = [torch.from_numpy(workloads.gradient_like(m, n, seed=60 + i)).cuda() for i, (m, n) in enumerate(shapes)]
+    direct = [torch.empty_like(x) for x in Gs]
+    ws = torch.empty(fp4.fp4_root_ns_batched_workspace_bytes(shapes, 3), dtype=torch.uint8, device="cuda")
+    fp4.fp4_root_ns_batched(Gs, direct, 3, None, ws)
+    torch.cuda.synchronize()
+    assert fp4.fp4_last_device_status(ws) == 0
+    singles = []
+    for x in Gs:
+        o = torch.empty_like(x)
+        w1 = torch.empty(fp4.fp4_root_ns_workspace_bytes(x.shape[0], x.shape[1], 3), dtype=torch.uint8, device="cuda")
+        fp4.fp4_root_ns(x, o, 3, None, w1)
+        singles.append(o)
+    for a, b in zip(direct, singles):
+        assert torch.equal(a, b)
+    outs = [torch.zeros_like(x) for x in Gs]
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        fp4.fp4_root_ns_batched(Gs, outs, 3, None, ws, torch.cuda.current_stream())
+    for _ in range(2):
+        for o in outs:
+            o.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert fp4.fp4_last_device_status(ws) == 0
+        for a, b in zip(outs, direct):
+            assert torch.equal(a, b)
+
+
 @pytest.mark.parametrize("shape", [(256, 512), (512, 256), (512, 512), (384, 384), (640, 384), (144, 272), (1024, 2048)])
 def test_bf16_storage_of_the_high_precision_copies(shape):
     """FP4_FLAG_STORE_BF16: A_k and X_k (k >= 1) are kept in BF16 between the stages; shapes whose
