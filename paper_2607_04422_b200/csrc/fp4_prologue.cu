@@ -36,7 +36,7 @@ struct PrepMatrix {
   uint32_t* hist;      // 8192 counters
   uint32_t* hist_top;  // the caller's counters of the first radix pass (then pass 1 is skipped), or null
   double* partial;     // one FP64 partial per statistics block
-  uint32_t* cand;      // candidate list (the A buffer of the workspace, unused until G1)
+  uint32_t* cand;      // candidate list (workspace that is unused until the first product)
   uint8_t* qx_codes; uint8_t* qx_sf;
   uint8_t* qt_codes; uint8_t* qt_sf;
   int tall;
@@ -887,7 +887,12 @@ cudaError_t launch_prologue_group(const PrologueItem* items, int count, int writ
     g.s0 = pl.s0; g.l0 = pl.l0;
     g.clip = pl.clip;
     g.clip_rank = (uint32_t)pl.clip_rank;
-    const int64_t cap = pl.s0 * pl.l0 / 8 < pl.s * pl.s ? pl.s0 * pl.l0 / 8 : pl.s * pl.s;
+    // The candidate list lives in workspace that nothing else uses before the first product: the A buffer
+    // (s x s words) or, for a matrix much longer than high, the second set of transposed operand codes
+    // (s x l / 8 words).  An eighth of the elements is more than any bin of a spread-out distribution holds.
+    const bool cand_in_qxt = pl.s * pl.l / 8 > pl.s * pl.s;
+    const int64_t region = cand_in_qxt ? pl.s * pl.l / 8 : pl.s * pl.s;
+    const int64_t cap = pl.s0 * pl.l0 / 8 < region ? pl.s0 * pl.l0 / 8 : region;
     g.cand_cap = (uint32_t)cap;
     g.eps = pl.eps;
     g.stat_blocks = pl.stat_blocks;
@@ -906,7 +911,7 @@ cudaError_t launch_prologue_group(const PrologueItem* items, int count, int writ
       m.scalars = reinterpret_cast<float*>(it.ws + L.scalars);
       m.hist = reinterpret_cast<uint32_t*>(it.ws + it.pl->off_hist);
       m.partial = reinterpret_cast<double*>(it.ws + it.pl->off_partial);
-      m.cand = reinterpret_cast<uint32_t*>(it.ws + L.A);
+      m.cand = reinterpret_cast<uint32_t*>(it.ws + (cand_in_qxt ? L.qXt_codes[1] : L.A));
       m.qx_codes = it.ws + L.qX_codes; m.qx_sf = it.ws + L.qX_scales;
       m.qt_codes = it.ws + L.qXt_codes[0]; m.qt_sf = it.ws + L.qXt_scales[0];
       m.tall = it.pl->tall;
