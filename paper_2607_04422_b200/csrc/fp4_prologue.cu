@@ -125,20 +125,34 @@ template <int NB>
 __device__ __forceinline__ void pick_bin(NsHeader* hdr, uint32_t* hist, int shift, uint32_t* bin_count_out,
                                          uint32_t* below_out) {
   constexpr int PER = NB / 256;
-  __shared__ uint32_t part[256];
+  static_assert(PER % 4 == 0, "a thread reads its counters as 16-byte pieces");
+  __shared__ uint32_t wtot[8];
   uint32_t local[PER];
   uint32_t sum = 0;
+  if ((reinterpret_cast<uintptr_t>(hist) & 15) == 0) {
 #pragma unroll
-  for (int j = 0; j < PER; ++j) { local[j] = hist[threadIdx.x * PER + j]; sum += local[j]; }
-  part[threadIdx.x] = sum;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    uint32_t run = 0;
-    for (int i = 0; i < 256; ++i) { uint32_t t = part[i]; part[i] = run; run += t; }
+    for (int j = 0; j < PER; j += 4) {
+      const uint4 v = *reinterpret_cast<const uint4*>(hist + threadIdx.x * PER + j);
+      local[j] = v.x; local[j + 1] = v.y; local[j + 2] = v.z; local[j + 3] = v.w;
+    }
+  } else {   // a caller's histogram need only be 4-byte aligned
+#pragma unroll
+    for (int j = 0; j < PER; ++j) local[j] = hist[threadIdx.x * PER + j];
   }
+#pragma unroll
+  for (int j = 0; j < PER; ++j) sum += local[j];
+  // exclusive prefix of the 256 chunk sums: scan inside each warp, then add the totals of the warps before
+  uint32_t incl = sum;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t t = __shfl_up_sync(0xffffffffu, incl, o);
+    if ((int)(threadIdx.x & 31) >= o) incl += t;
+  }
+  if ((threadIdx.x & 31) == 31) wtot[threadIdx.x >> 5] = incl;
   __syncthreads();
+  uint32_t before = incl - sum;
+  for (int w = 0; w < (int)(threadIdx.x >> 5); ++w) before += wtot[w];
   const uint32_t rank = hdr->sel_rank;
-  uint32_t before = part[threadIdx.x];
   __syncthreads();
   if (rank > before && rank <= before + sum) {
 #pragma unroll
