@@ -1,7 +1,7 @@
 // Prologue of the Root step for a group of equal-size matrices (Section 3.4: "p99 outlier
 // clipping"; normalisation; the first operand copies qX = Q_1x16(X), qX^{16x1} = Q_16x1(X)).
-// Every kernel covers the whole group (gridDim.y or .z = matrix), so a batch needs a dozen
-// launches instead of a dozen per matrix.
+// Every kernel covers the whole group (gridDim.y = matrix, or a tile list over all matrices), so a
+// group needs six launches instead of six per matrix.
 //
 // Clip threshold tau = nearest-rank quantile of |g|, found exactly with two passes over
 // the data where three were needed before:
