@@ -592,3 +592,30 @@ def test_first_operand_copies_two_million_blocks(kind):
     """The same on 4096 x 4096: with 2 x 10^6 blocks some scale quotients fall within two ulps of an E4M3
     rounding boundary, the case the preparation kernel hands to its exact path."""
     test_first_operand_copies_are_the_oracle_quantisation_of_x0(kind, (4096, 4096))
+
+
+@pytest.mark.parametrize("qmode", ["rht", "four_six", "paper"])
+@pytest.mark.parametrize("shape", [(256, 512), (512, 256), (144, 272)])
+def test_first_operand_copies_with_the_paper_quantiser_options(shape, qmode):
+    """The same check for the random Hadamard transform and adaptive 4/6 scaling of X0's copies (the
+    transform of the first copies uses the mask of index 0; the tensor scale then covers 4 amax)."""
+    m, n = shape
+    rht, fs = QMODES[qmode]
+    seed = 1234
+    G = _first_copies_input("heavy_tail", m, n)
+    flags = FP4_FLAG_KEEP_OPERANDS | qflags(qmode)
+    got, ws = run_gpu(G, steps=0, flags=flags, seed=seed)
+    lay, sc, f32, q, s, l = ws_view(ws, m, n, 0, flags)
+    s_pad, l_pad = -(-s // 128) * 128, -(-l // 128) * 128
+    X0 = np.zeros((s_pad, l_pad), dtype=np.float32)
+    X0[:s, :l] = got if m <= n else got.T
+    sg = float(sc[lay.idx_sg_X0])
+    qopt = dict(rht=rht, mask=oracle.rht_mask(seed, 0) if rht else 0, four_six=fs)
+    oc, os_, _ = oracle.quantize(X0, s_g=sg, **qopt)
+    codes, sf = q(lay.qX_codes, lay.qX_scales, s_pad, l_pad)
+    assert np.array_equal(sf, os_), mismatch(sf, os_)
+    assert np.array_equal(codes, oc), mismatch(codes, oc)
+    oc, os_, _ = oracle.quantize(np.ascontiguousarray(X0.T), s_g=sg, **qopt)
+    codes, sf = q(lay.qXt_codes[0], lay.qXt_scales[0], l_pad, s_pad)
+    assert np.array_equal(sf, os_), mismatch(sf, os_)
+    assert np.array_equal(codes, oc), mismatch(codes, oc)
