@@ -98,6 +98,16 @@ __device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
   asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
   return d;
 }
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
 // d = a * b + c per lane, one rounding (what the scalar fused multiply-add gives)
 __device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
   uint64_t d;
@@ -193,8 +203,71 @@ __device__ __forceinline__ float2 e2m1x2_to_float2(uint32_t byte) {
 }
 
 // v <- v diag(signs) H_16 / 4 in FP32: signs, the natural-order butterfly (strides 1, 2, 4, 8;
-// sum to the lower index, difference to the upper), then the factor 1/4.
+// sum to the lower index, difference to the upper), then the factor 1/4.  The stride-1 stage runs on
+// scalars, the strides 2, 4, 8 and the factor on packed pairs (v[2k], v[2k+1]): every lane is the same
+// single rounded operation as in a scalar butterfly, and no product meets a sum that could absorb it.
 __device__ __forceinline__ void hadamard16(float (&v)[16], uint32_t mask) {
+  uint64_t p[8];
+#pragma unroll
+  for (int k = 0; k < 8; ++k) {
+    const float a = __uint_as_float(__float_as_uint(v[2 * k]) ^ (((mask >> (2 * k)) & 1u) << 31));
+    const float b = __uint_as_float(__float_as_uint(v[2 * k + 1]) ^ (((mask >> (2 * k + 1)) & 1u) << 31));
+    p[k] = pack2(__fadd_rn(a, b), __fsub_rn(a, b));
+  }
+#pragma unroll
+  for (int h = 1; h < 8; h *= 2) {
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      if ((k & h) == 0) {
+        const uint64_t a = p[k], b = p[k + h];
+        p[k] = add2(a, b);
+        p[k + h] = sub2(a, b);
+      }
+    }
+  }
+  const uint64_t q = pack2(0.25f, 0.25f);
+#pragma unroll
+  for (int k = 0; k < 8; ++k) unpack2(mul2(p[k], q), v[2 * k], v[2 * k + 1]);
+}
+
+// Codes of one block for the scale byte sb; returns the sum of the squared FP32 errors,
+// accumulated in element order (the 4/6 choice compares two such sums, so the order of the
+// roundings is part of the definition).  Products are taken two at a time; every subtraction and
+// every addition of the error sum stays a scalar operation, so none can fuse with a product.
+__device__ __forceinline__ float encode_block16(const float (&v)[16], uint32_t sb, float sg, uint32_t& lo,
+                                                uint32_t& hi) {
+  const float d = __fmul_rn(ue4m3_to_float(sb), sg);
+  lo = 0; hi = 0;
+  float err = 0.0f;
+  if (d == 0.0f) {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) err = __fadd_rn(err, __fmul_rn(v[i], v[i]));
+    return err;
+  }
+  const float rcp = __frcp_rn(d);
+  const uint64_t rcp2 = pack2(rcp, rcp), d2 = pack2(d, d);
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    float y0, y1, p0, p1, s0, s1;
+    unpack2(mul2(pack2(v[2 * i], v[2 * i + 1]), rcp2), y0, y1);
+    const uint32_t byte = cvt_e2m1x2(y0, y1);
+    const float2 q = e2m1x2_to_float2(byte);
+    unpack2(mul2(pack2(q.x, q.y), d2), p0, p1);
+    const float d0 = __fsub_rn(v[2 * i], p0), d1 = __fsub_rn(v[2 * i + 1], p1);
+    const uint64_t dd = pack2(d0, d1);
+    unpack2(mul2(dd, dd), s0, s1);
+    err = __fadd_rn(err, s0);
+    err = __fadd_rn(err, s1);
+    if (i < 4) lo |= byte << (8 * i); else hi |= byte << (8 * (i - 4));
+  }
+  return err;
+}
+
+// The same two functions with scalar operations only (fewer live registers: G3's epilogue, which
+// quantises every block twice, is faster with these; the results are the same bit for bit).
+// v <- v diag(signs) H_16 / 4 in FP32: signs, the natural-order butterfly (strides 1, 2, 4, 8;
+// sum to the lower index, difference to the upper), then the factor 1/4.
+__device__ __forceinline__ void hadamard16_scalar(float (&v)[16], uint32_t mask) {
 #pragma unroll
   for (int i = 0; i < 16; ++i) v[i] = (mask >> i) & 1 ? -v[i] : v[i];
 #pragma unroll
@@ -215,7 +288,7 @@ __device__ __forceinline__ void hadamard16(float (&v)[16], uint32_t mask) {
 // Codes of one block for the scale byte sb; returns the sum of the squared FP32 errors,
 // accumulated in element order (the 4/6 choice compares two such sums, so the order of the
 // roundings is part of the definition).
-__device__ __forceinline__ float encode_block16(const float (&v)[16], uint32_t sb, float sg, uint32_t& lo,
+__device__ __forceinline__ float encode_block16_scalar(const float (&v)[16], uint32_t sb, float sg, uint32_t& lo,
                                                 uint32_t& hi) {
   const float d = __fmul_rn(ue4m3_to_float(sb), sg);
   lo = 0; hi = 0;
@@ -241,7 +314,9 @@ __device__ __forceinline__ float encode_block16(const float (&v)[16], uint32_t s
 
 // Quantise one block with the options above; any tensor scale.  v is transformed in place.
 // Returns the scale byte; amax_in is the block's amax before the transform (what the
-// predicted tensor scales of the next stage are derived from).
+// predicted tensor scales of the next stage are derived from).  PACKED selects the form of the
+// transform and of the error sums (same results).
+template <bool PACKED = true>
 __device__ __forceinline__ uint32_t quantize_block16_opts(float (&v)[16], const QuantOpts& q, float sg, uint32_t& lo,
                                                           uint32_t& hi, float& amax_in) {
   float a = 0.0f;
@@ -249,17 +324,17 @@ __device__ __forceinline__ uint32_t quantize_block16_opts(float (&v)[16], const 
   for (int i = 0; i < 16; ++i) a = fmaxf(a, fabsf(v[i]));
   amax_in = a;
   if (q.rht) {
-    hadamard16(v, q.mask);
+    if (PACKED) hadamard16(v, q.mask); else hadamard16_scalar(v, q.mask);
     a = 0.0f;
 #pragma unroll
     for (int i = 0; i < 16; ++i) a = fmaxf(a, fabsf(v[i]));
   }
   uint32_t sb = cvt_ue4m3(__fdiv_rn(a, __fmul_rn(6.0f, sg)));
-  const float err6 = encode_block16(v, sb, sg, lo, hi);
+  const float err6 = PACKED ? encode_block16(v, sb, sg, lo, hi) : encode_block16_scalar(v, sb, sg, lo, hi);
   if (q.four_six) {
     const uint32_t sb4 = cvt_ue4m3(__fdiv_rn(a, __fmul_rn(4.0f, sg)));
     uint32_t lo4, hi4;
-    const float err4 = encode_block16(v, sb4, sg, lo4, hi4);
+    const float err4 = PACKED ? encode_block16(v, sb4, sg, lo4, hi4) : encode_block16_scalar(v, sb4, sg, lo4, hi4);
     if (err4 < err6) { sb = sb4; lo = lo4; hi = hi4; }
   }
   return sb;

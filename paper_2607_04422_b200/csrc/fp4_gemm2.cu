@@ -809,7 +809,7 @@ k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ Ge
         if (do_q) {
           float bmax;
           uint32_t sb;
-          if (PF) sb = quantize_block16_opts(v, args.q, sg_out, rlo, rhi, bmax);
+          if (PF) sb = quantize_block16_opts<MODE != kG3>(v, args.q, sg_out, rlo, rhi, bmax);
           else sb = quantize_block16_pow2(v, sg_out, inv_sg, rcp_base, rlo, rhi, bmax);
           if (MODE == kG1 || MODE == kG3) amax = fmaxf(amax, bmax);
           sfw |= sb << (8 * e);
@@ -843,7 +843,7 @@ k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ Ge
           uint32_t lo, hi;
           float bmax;
           uint32_t sb;
-          if (PF) sb = quantize_block16_opts(w, args.q, sg_out, lo, hi, bmax);
+          if (PF) sb = quantize_block16_opts<MODE != kG3>(w, args.q, sg_out, lo, hi, bmax);
           else sb = quantize_block16_pow2(w, sg_out, inv_sg, rcp_base, lo, hi, bmax);
           sts64u(cq_st + e * (CHUNK * 64), lo, hi);
           // tensor row = x64 + e * 16 + cq: e % 2 selects the upper 16 of 32 rows of its scale atom,

@@ -14,17 +14,6 @@ __device__ __forceinline__ uint64_t splitmix64_at(uint64_t seed, uint64_t idx) {
   return z ^ (z >> 31);
 }
 
-__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
-  uint64_t d;
-  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-  return d;
-}
-__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
-  uint64_t d;
-  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-  return d;
-}
-
 // v <- v H_16 / 4, the natural-order butterfly of hadamard16 with no signs: the stride-1 stage on
 // scalars, the strides 2, 4, 8 and the factor 1/4 on packed pairs (v[2k], v[2k+1]); every lane
 // is the same single rounded operation as in the scalar form.
