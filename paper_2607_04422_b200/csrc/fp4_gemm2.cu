@@ -478,10 +478,10 @@ k_gemm_pair(const __grid_constant__ ProblemPack pack, const __grid_constant__ Ge
     const uint32_t acc_empty_leader0 = map_to_cta(&bars->acc_empty[0], 0);
     const uint32_t acc_empty_leader1 = map_to_cta(&bars->acc_empty[1], 0);
     const uint32_t ov_free_leader = map_to_cta(&bars->ov_free, 0);
-    // A tall input is worked on as its transpose.  With FP32 storage the first G3 stage reads the caller's
-    // matrix through a transposing box and the last one writes the caller's result the same way, so neither
+    // A tall input is worked on as its transpose.  The first G3 stage reads the caller's matrix through a
+    // transposing box and the last one writes the caller's result the same way, so neither
     // an FP32 copy of X0 nor a final transpose pass is needed (per-problem flags aux_tr / out_tr).
-    constexpr bool TR = (MODE == kG3) && !BH;
+    constexpr bool TR = (MODE == kG3);
     const bool auxh = BH && HAS_AUX && args.aux_h != 0;                               // the combined tile is BF16
     const bool hout = BH && STORE_F32 && MODE != kPlain && args.out_h == 1;           // the result is stored as BF16
 

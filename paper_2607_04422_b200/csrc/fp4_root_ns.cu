@@ -333,8 +333,8 @@ struct MatrixCtx {
   uint32_t* hist_top;         // the caller's first-pass histogram of G, or null
   uint16_t* W;                // the BF16 parameter that takes Root's update in this call, or null
   CUtensorMap tm_G;           // the caller's matrix for the operand preparation (tiles of 128 x 128)
-  // A tall input with FP32 storage in the CTA-pair kernel: the first G3 stage reads the caller's matrix and
-  // the last one writes the caller's result through transposing boxes.
+  // A tall input in the CTA-pair kernel: the first G3 stage reads the caller's matrix and the last one
+  // writes the caller's result through transposing boxes.
   bool native_tall;
   CUtensorMap tm_outT;
 };
@@ -431,7 +431,7 @@ fp4_status build_matrix(const DeviceInfo* d, const float* G, float* out, int64_t
     g.tmRq = st_qX_r; g.tmCq = st_qXt_c[cur ^ 1];
   }
   c->g3_first = c->g3[0];
-  c->native_tall = c->pl.tall && pair3 && bmode == 0;
+  c->native_tall = c->pl.tall && pair3;   // (rounded-FP32 storage, bmode 2, never runs in the CTA-pair kernel)
   if (c->native_tall) {
     // the caller's matrices are l0 x s0
     CUtensorMap tm_Gt;
