@@ -619,3 +619,39 @@ def test_first_operand_copies_with_the_paper_quantiser_options(shape, qmode):
     codes, sf = q(lay.qXt_codes[0], lay.qXt_scales[0], l_pad, s_pad)
     assert np.array_equal(sf, os_), mismatch(sf, os_)
     assert np.array_equal(codes, oc), mismatch(codes, oc)
+
+
+def test_two_host_threads_call_concurrently():
+    """The library keeps per-thread launch state (second stream of a batched call, launch mode) and a
+    locked descriptor cache: two host threads with their own streams and workspaces get the results of
+    single calls."""
+    import threading
+    shapes = [(256, 512), (512, 256), (512, 512), (768, 256)]
+    results = {}
+
+    def worker(tid):
+        torch.cuda.set_device(0)
+        st = torch.cuda.Stream()
+        Gs = [torch.from_numpy(workloads.gradient_like(m, n, seed=80 + 10 * tid + i)).cuda() for i, (m, n) in enumerate(shapes)]
+        outs = [torch.empty_like(x) for x in Gs]
+        ws = torch.empty(fp4.fp4_root_ns_batched_workspace_bytes(shapes, 3), dtype=torch.uint8, device="cuda")
+        with torch.cuda.stream(st):
+            for _ in range(20):
+                fp4.fp4_root_ns_batched(Gs, outs, 3, None, ws, st)
+        st.synchronize()
+        results[tid] = (Gs, outs, fp4.fp4_last_device_status(ws))
+
+    threads = [threading.Thread(target=worker, args=(t,)) for t in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    for tid in range(2):
+        Gs, outs, status = results[tid]
+        assert status == 0
+        for x, o in zip(Gs, outs):
+            single = torch.empty_like(x)
+            w1 = torch.empty(fp4.fp4_root_ns_workspace_bytes(x.shape[0], x.shape[1], 3), dtype=torch.uint8, device="cuda")
+            fp4.fp4_root_ns(x, single, 3, None, w1)
+            torch.cuda.synchronize()
+            assert torch.equal(o, single)
