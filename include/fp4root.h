@@ -84,6 +84,14 @@ typedef enum {
  * wants).  `out` is still required - it is the working copy of X during the iterations of a wide matrix -
  * and its contents are unspecified afterwards. */
 #define FP4_FLAG_NO_OUT 16u
+/* fp4_root_ns_batched only: groups of equal shapes, which do not depend on one another, alternate between
+ * the caller's stream and a second stream of the library's own (one per host thread and device, created on
+ * first use).  The second stream waits for everything enqueued on the caller's stream before the call, and
+ * the caller's stream waits for it before the call returns, so callers see ordinary stream order and the
+ * call can still be captured in a CUDA graph.  Off by default: with two large groups (the decoder-stack
+ * benchmark) the gain or loss of about 1.5 % depends on the order in which the two groups' launches meet
+ * on the device; the option is for batches of many small groups. */
+#define FP4_FLAG_OVERLAP_GROUPS 32u
 #define FP4_QUANT_SIGNS(mask) ((uint32_t)(mask) << 16)
 
 /* Parameters of the step.  Pass NULL for the defaults noted on each field. */
@@ -185,11 +193,7 @@ fp4_status fp4_root_ns(const float* G, float* out, int64_t m, int64_t n, int ste
  * Matrices of equal shape (after orientation) are grouped: each Newton-Schulz stage of a
  * group is one launch whose tile list spans all its matrices.  Results are bit-identical to
  * calling fp4_root_ns on each matrix.
- * Streams: with two or more groups the call also uses a second stream of its own (one per host
- *   thread and device, created on first use), which waits for everything enqueued on `stream`
- *   before the call and which `stream` waits for before the call returns, so callers see
- *   ordinary stream order; the pattern can be captured in a CUDA graph.  The environment
- *   variable FP4ROOT_NO_OVERLAP (any value) keeps all launches on `stream`.
+ * All launches go to `stream` unless FP4_FLAG_OVERLAP_GROUPS is set (see there).
  */
 size_t fp4_root_ns_batched_workspace_bytes(int count, const int64_t* m, const int64_t* n,
                                            int steps, uint32_t flags);

@@ -20,6 +20,7 @@ FP4_FLAG_RHT = 2
 FP4_FLAG_FOUR_SIX = 4
 FP4_FLAG_STORE_BF16 = 8
 FP4_FLAG_NO_OUT = 16
+FP4_FLAG_OVERLAP_GROUPS = 32
 FP4_MOM_FLAG_SR = 1
 STATUS_NAMES = {0: "FP4_OK", 1: "FP4_ERR_INVALID_ARG", 2: "FP4_ERR_SHAPE", 3: "FP4_ERR_ALIGNMENT",
                 4: "FP4_ERR_WORKSPACE", 5: "FP4_ERR_ARCH", 6: "FP4_ERR_CUDA", 7: "FP4_ERR_DEVICE_TIMEOUT",

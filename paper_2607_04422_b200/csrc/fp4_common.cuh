@@ -127,6 +127,21 @@ __device__ __forceinline__ uint32_t cvt_e2m1x4(float a, float b, float c, float 
   return r;
 }
 
+// Eight FP32 -> four bytes of E2M1 codes (v0 in bits 3:0 ... v7 in bits 31:28).
+__device__ __forceinline__ uint32_t cvt_e2m1x8(float v0, float v1, float v2, float v3, float v4, float v5, float v6,
+                                               float v7) {
+  uint32_t r;
+  asm("{\n\t.reg .b8 t0, t1, t2, t3;\n\t"
+      "cvt.rn.satfinite.e2m1x2.f32 t0, %2, %1;\n\t"
+      "cvt.rn.satfinite.e2m1x2.f32 t1, %4, %3;\n\t"
+      "cvt.rn.satfinite.e2m1x2.f32 t2, %6, %5;\n\t"
+      "cvt.rn.satfinite.e2m1x2.f32 t3, %8, %7;\n\t"
+      "mov.b32 %0, {t0, t1, t2, t3};\n\t}"
+      : "=r"(r)
+      : "f"(v0), "f"(v1), "f"(v2), "f"(v3), "f"(v4), "f"(v5), "f"(v6), "f"(v7));
+  return r;
+}
+
 // The same quantisation when the tensor scale is a power of two (every tensor produced
 // inside the Newton-Schulz loop), with the two IEEE divisions replaced by exact equivalents:
 //   amax / (6 sg)  = RN(amax / 6) * (1/sg): the division by the constant 6 is one multiply
@@ -161,16 +176,11 @@ __device__ __forceinline__ uint32_t quantize_block16_pow2(const float (&v)[16], 
   // y = v * rcp, two lanes per instruction; an all-zero block (rcp = 0) gets codes 0 with the
   // sign bits of its elements cleared below
   const uint64_t rcp2 = pack2(rcp, rcp);
-  uint32_t w[4];
+  float z[16];
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    float a, b, c, d;
-    unpack2(mul2(pack2(v[4 * i], v[4 * i + 1]), rcp2), a, b);
-    unpack2(mul2(pack2(v[4 * i + 2], v[4 * i + 3]), rcp2), c, d);
-    w[i] = cvt_e2m1x4(a, b, c, d);
-  }
-  lo = w[0] | (w[1] << 16);
-  hi = w[2] | (w[3] << 16);
+  for (int i = 0; i < 8; ++i) unpack2(mul2(pack2(v[2 * i], v[2 * i + 1]), rcp2), z[2 * i], z[2 * i + 1]);
+  lo = cvt_e2m1x8(z[0], z[1], z[2], z[3], z[4], z[5], z[6], z[7]);
+  hi = cvt_e2m1x8(z[8], z[9], z[10], z[11], z[12], z[13], z[14], z[15]);
   if (sb == 0) { lo = 0; hi = 0; }
   return sb;
 }

@@ -514,21 +514,6 @@ __device__ __forceinline__ float lds32f(uint32_t addr) {
   asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
   return v;
 }
-// Eight FP32 -> four bytes of E2M1 codes (v0 in bits 3:0 ... v7 in bits 31:28).
-__device__ __forceinline__ uint32_t cvt_e2m1x8(float v0, float v1, float v2, float v3, float v4, float v5, float v6,
-                                               float v7) {
-  uint32_t r;
-  asm("{\n\t.reg .b8 t0, t1, t2, t3;\n\t"
-      "cvt.rn.satfinite.e2m1x2.f32 t0, %2, %1;\n\t"
-      "cvt.rn.satfinite.e2m1x2.f32 t1, %4, %3;\n\t"
-      "cvt.rn.satfinite.e2m1x2.f32 t2, %6, %5;\n\t"
-      "cvt.rn.satfinite.e2m1x2.f32 t3, %8, %7;\n\t"
-      "mov.b32 %0, {t0, t1, t2, t3};\n\t}"
-      : "=r"(r)
-      : "f"(v0), "f"(v1), "f"(v2), "f"(v3), "f"(v4), "f"(v5), "f"(v6), "f"(v7));
-  return r;
-}
-
 // ---- block quantisers of the operand preparation.
 // They quantise x0 = clamp(g, +-tau) * inv (quantize_block16 applied to x0) with fewer instructions,
 // bit for bit the same result; whatever the short cuts do not cover goes to quantize_block16 itself.

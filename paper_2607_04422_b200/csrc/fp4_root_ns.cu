@@ -97,7 +97,8 @@ inline bool ns_shape_ok(int64_t v) { return v >= 16 && v % 16 == 0 && v <= (1 <<
 inline int64_t pad128(int64_t v) { return (v + 127) / 128 * 128; }
 // flag bits the Newton-Schulz entry points know
 constexpr uint32_t kNsFlags =
-    FP4_FLAG_KEEP_OPERANDS | FP4_FLAG_RHT | FP4_FLAG_FOUR_SIX | FP4_FLAG_STORE_BF16 | FP4_FLAG_NO_OUT;
+    FP4_FLAG_KEEP_OPERANDS | FP4_FLAG_RHT | FP4_FLAG_FOUR_SIX | FP4_FLAG_STORE_BF16 | FP4_FLAG_NO_OUT |
+    FP4_FLAG_OVERLAP_GROUPS;
 
 // 2-D map over a row-major byte matrix (NVFP4 codes): box = one operand stage of `stage_k` elements of K
 // (64 or 128 bytes x 128 rows), swizzled over the box width.
@@ -799,17 +800,14 @@ fp4_status fp4_root_ns(const float* G, float* out, int64_t m, int64_t n, int ste
   return run_one(d, G, out, m, n, steps, p, static_cast<uint8_t*>(ws), true, stream);
 }
 
-// The second stream of a batched call, one per host thread and device, created on first use (never inside
-// fp4_root_ns or fp4_root_ns_static).  FP4ROOT_NO_OVERLAP in the environment keeps everything on the
-// caller's stream.
+// The second stream of a batched call with FP4_FLAG_OVERLAP_GROUPS, one per host thread and device,
+// created on first use.
 struct SideStream {
   int dev = -1;
   cudaStream_t stream = nullptr;
   cudaEvent_t fork = nullptr, join = nullptr;
 };
 SideStream* side_stream(int dev) {
-  static const bool allowed = getenv("FP4ROOT_NO_OVERLAP") == nullptr;
-  if (!allowed) return nullptr;
   thread_local SideStream t;
   if (t.stream && t.dev == dev) return &t;
   if (t.stream) {   // the thread moved to another device
@@ -892,12 +890,13 @@ fp4_status fp4_root_ns_batched(int count, const float* const* G, float* const* o
       }
     }
   }
-  // Groups do not depend on one another.  With two or more, they alternate between the caller's stream
-  // and a second one that forks from it and joins it again before the call returns: every launch is a
-  // persistent grid that ends in a partial wave of tiles, and the next launch of the same group cannot
-  // start before it has drained - a launch of the other group can.
-  // (not while stage times are being collected: the event pairs of the two streams would overlap)
-  SideStream* side = groups.size() >= 2 && g_prof_on.load() == 0 ? side_stream((int)(d - g_dev)) : nullptr;
+  // Groups do not depend on one another.  On request (FP4_FLAG_OVERLAP_GROUPS) they alternate between the
+  // caller's stream and a second one that forks from it and joins it again before the call returns: every
+  // launch is a persistent grid that ends in a partial wave of tiles, and the next launch of the same
+  // group cannot start before it has drained - a launch of another group can.  (Not while stage times
+  // are being collected: the event pairs of the two streams would overlap.)
+  SideStream* side = (p->flags & FP4_FLAG_OVERLAP_GROUPS) && groups.size() >= 2 && g_prof_on.load() == 0
+                         ? side_stream((int)(d - g_dev)) : nullptr;
   if (side) {
     // the status word is cleared once, before the fork (a group's own clearing kernel could wipe what
     // a kernel of the other group has just reported)

@@ -6,7 +6,8 @@ import torch
 import oracle
 import paper_2607_04422_b200 as fp4
 from paper_2607_04422_b200 import workloads
-from paper_2607_04422_b200.binding import (FP4_FLAG_FOUR_SIX, FP4_FLAG_KEEP_OPERANDS, FP4_FLAG_RHT, FP4_FLAG_STORE_BF16,
+from paper_2607_04422_b200.binding import (FP4_FLAG_FOUR_SIX, FP4_FLAG_KEEP_OPERANDS, FP4_FLAG_OVERLAP_GROUPS, FP4_FLAG_RHT,
+                                           FP4_FLAG_STORE_BF16,
                                            fp4_root_ns_workspace_layout)
 from helpers import nibbles, sf_from_atoms
 
@@ -294,13 +295,14 @@ def test_cuda_graph_replay_matches_direct_call():
 
 
 def test_cuda_graph_replay_of_a_batched_call_with_several_groups():
-    """A batched call with more than one group of shapes forks to a second stream and joins again:
-    captured as a whole, the replay gives the bytes of the direct call."""
+    """With FP4_FLAG_OVERLAP_GROUPS a batched call with more than one group of shapes forks to a second
+    stream and joins again: captured as a whole, the replay gives the bytes of the direct call."""
     shapes = [(256, 512), (512, 256), (512, 512), (256, 512), (768, 256), (512, 512)]
     Gs = [torch.from_numpy(workloads.gradient_like(m, n, seed=60 + i)).cuda() for i, (m, n) in enumerate(shapes)]
     direct = [torch.empty_like(x) for x in Gs]
     ws = torch.empty(fp4.fp4_root_ns_batched_workspace_bytes(shapes, 3), dtype=torch.uint8, device="cuda")
-    fp4.fp4_root_ns_batched(Gs, direct, 3, None, ws)
+    p = fp4.NsParams.make(flags=FP4_FLAG_OVERLAP_GROUPS)
+    fp4.fp4_root_ns_batched(Gs, direct, 3, p, ws)
     torch.cuda.synchronize()
     assert fp4.fp4_last_device_status(ws) == 0
     singles = []
@@ -314,7 +316,7 @@ def test_cuda_graph_replay_of_a_batched_call_with_several_groups():
     outs = [torch.zeros_like(x) for x in Gs]
     graph = torch.cuda.CUDAGraph()
     with torch.cuda.graph(graph):
-        fp4.fp4_root_ns_batched(Gs, outs, 3, None, ws, torch.cuda.current_stream())
+        fp4.fp4_root_ns_batched(Gs, outs, 3, p, ws, torch.cuda.current_stream())
     for _ in range(2):
         for o in outs:
             o.zero_()
@@ -428,7 +430,7 @@ def test_argument_errors():
     with pytest.raises(fp4.Fp4Error) as e:
         fp4.fp4_root_ns(G, G, 5, None, ws[1:])
     assert e.value.code == 3
-    for bad_flags in (32, FP4_FLAG_RHT | (0x1234 << 16)):      # unknown bits, fp4_quantize's sign bits
+    for bad_flags in (64, FP4_FLAG_RHT | (0x1234 << 16)):      # unknown bits, fp4_quantize's sign bits
         with pytest.raises(fp4.Fp4Error) as e:
             fp4.fp4_root_ns(G, G, 5, fp4.NsParams.make(flags=bad_flags), ws)
         assert e.value.code == 1
@@ -637,7 +639,7 @@ def test_two_host_threads_call_concurrently():
         ws = torch.empty(fp4.fp4_root_ns_batched_workspace_bytes(shapes, 3), dtype=torch.uint8, device="cuda")
         with torch.cuda.stream(st):
             for _ in range(20):
-                fp4.fp4_root_ns_batched(Gs, outs, 3, None, ws, st)
+                fp4.fp4_root_ns_batched(Gs, outs, 3, fp4.NsParams.make(flags=FP4_FLAG_OVERLAP_GROUPS), ws, st)
         st.synchronize()
         results[tid] = (Gs, outs, fp4.fp4_last_device_status(ws))
 
