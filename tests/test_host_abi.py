@@ -58,6 +58,7 @@ def test_scale_bytes_and_workspace_sizes():
     assert both >= small + big and both < small + big + (1 << 16)  # one workspace per matrix
     # flag bits the library does not know are an error, not ignored: the size query answers 0
     assert fp4.fp4_root_ns_workspace_bytes(128, 256, 5, 64) == 0
+    assert fp4.fp4_root_ns_workspace_bytes(128, 256, 5, fp4.FP4_FLAG_OVERLAP_GROUPS) == small  # the newest known bit
     assert fp4.fp4_root_ns_workspace_bytes(128, 256, 5, 0xABCD0000) == 0
     assert fp4.fp4_root_ns_batched_workspace_bytes([(128, 256)], 5, 1 << 20) == 0
     lay = fp4.fp4_root_ns_workspace_layout(512, 256, 5)
