@@ -657,3 +657,15 @@ def test_two_host_threads_call_concurrently():
             fp4.fp4_root_ns(x, single, 3, None, w1)
             torch.cuda.synchronize()
             assert torch.equal(o, single)
+
+
+@pytest.mark.parametrize("shape", [(1024, 512), (512, 1024), (1008, 496)])
+def test_in_place_single_iteration(shape):
+    """One iteration in place: the only G3 launch reads the caller's matrix (through a transposing box when
+    it is tall) and writes the result over it."""
+    m, n = shape
+    G = workloads.gradient_like(m, n, seed=33)
+    apart, _ = run_gpu(G, steps=1)
+    inplace, _ = run_gpu(G, steps=1, in_place=True)
+    assert np.array_equal(inplace, apart)
+    assert rel(apart, oracle.root_ns(G, steps=1)) <= TOL_OUT
